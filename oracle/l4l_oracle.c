@@ -1,0 +1,241 @@
+/*
+ * CPU oracle for causal attention (prefill, decode) and the KV-cache copy.
+ *
+ * THIS IS TEST INFRASTRUCTURE, NOT THE PRODUCT. It is a slow, plain restatement of
+ * the definition of scaled-dot-product softmax attention in fp64, read from the same
+ * bf16 inputs the GPU path gets. It shares no code with the CUDA kernels and must be
+ * used only by the tests, the smoke check and the benchmark's CPU-baseline leg.
+ *
+ * What it follows. The paper (appendix, "Transformer attention") names the two
+ * phase-specialised kernels but prints no formula: a prefill kernel for q_len > 1
+ * that derives the KV head from the grouped-query structure and applies the causal
+ * mask in the score update, and a decode kernel for q_len = 1 that serves one KV
+ * head's whole query-head group from a populated cache. Both are exact
+ * reformulations (online softmax, tiling) of ordinary softmax attention, so the
+ * oracle is that definition written out:
+ *
+ *   s_j   = scale * sum_d q[d] * k_j[d]            (keys j = 0 .. n-1)
+ *   p_j   = exp(s_j - max_j s_j)
+ *   o[d]  = sum_j p_j * v_j[d] / sum_j p_j
+ *   lse   = max_j s_j + log(sum_j p_j)
+ *
+ * Readings where the paper is silent (declared choices):
+ *   - query head h uses KV head h / (Hq / Hkv) (consecutive query heads share a KV head);
+ *   - prefill is causal with square alignment: query i sees keys 0..i of its sequence;
+ *   - decode has no mask: the current token is already in the cache, the query sees
+ *     all kv_len tokens;
+ *   - n = 0 keys gives o = 0 and lse = -inf;
+ *   - q, k, v are [B, S, H, D] token-major, the cache is [B, Hkv, Lmax, D]; all dense.
+ *
+ * No tiling, no online softmax, no reordering: one function, attend_row(), is the
+ * definition; everything else is loops that call it or copy 16-bit words.
+ * Parallelism is OpenMP over independent output rows only.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* bf16 is the upper half of an IEEE binary32; widening is exact. */
+static double bf16_to_f64(uint16_t h)
+{
+    uint32_t u = (uint32_t)h << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+int l4l_oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/*
+ * Softmax attention of ONE query row over n keys (the definition above).
+ *   q        : D bf16 values
+ *   k, v     : row j at k + j*k_stride, v + j*v_stride (strides in elements), D values each
+ *   p        : scratch of n doubles
+ *   out      : D doubles;  lse : 1 double (may be NULL)
+ */
+static void attend_row(const uint16_t *q, const uint16_t *k, int64_t k_stride,
+                       const uint16_t *v, int64_t v_stride, int n, int D,
+                       double scale, double *p, double *out, double *lse)
+{
+    if (n <= 0) {
+        for (int d = 0; d < D; ++d) out[d] = 0.0;
+        if (lse) *lse = -INFINITY;
+        return;
+    }
+    double m = -INFINITY;
+    for (int j = 0; j < n; ++j) {
+        double dot = 0.0;
+        for (int d = 0; d < D; ++d)
+            dot += bf16_to_f64(q[d]) * bf16_to_f64(k[(int64_t)j * k_stride + d]);
+        p[j] = scale * dot;
+        if (p[j] > m) m = p[j];
+    }
+    double l = 0.0;
+    for (int j = 0; j < n; ++j) {
+        p[j] = exp(p[j] - m);
+        l += p[j];
+    }
+    for (int d = 0; d < D; ++d) {
+        double acc = 0.0;
+        for (int j = 0; j < n; ++j)
+            acc += p[j] * bf16_to_f64(v[(int64_t)j * v_stride + d]);
+        out[d] = acc / l;
+    }
+    if (lse) *lse = m + log(l);
+}
+
+/*
+ * Causal prefill, every valid row.
+ *   q        [B, S, Hq, D]  bf16 bits      k, v  [B, S, Hkv, D] bf16 bits
+ *   seq_len  [B]            tokens per sequence (<= S)
+ *   out      [B, S, Hq, D]  fp64; rows i >= seq_len[b] are left untouched
+ *   lse      [B, Hq, S]     fp64 or NULL; same rule
+ * Returns 0, or -1 on bad arguments / allocation failure.
+ */
+int l4l_oracle_prefill(const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                       const int32_t *seq_len, int B, int S, int Hq, int Hkv, int D,
+                       double scale, double *out, double *lse)
+{
+    if (Hkv <= 0 || Hq % Hkv != 0) return -1;
+    const int G = Hq / Hkv;
+    int fail = 0;
+#pragma omp parallel
+    {
+        double *p = (double *)malloc(sizeof(double) * (size_t)(S > 0 ? S : 1));
+        if (!p) {
+#pragma omp atomic write
+            fail = 1;
+        }
+#pragma omp for collapse(2) schedule(dynamic, 8)
+        for (int b = 0; b < B; ++b) {
+            for (int i = 0; i < S; ++i) {
+                if (!p || i >= seq_len[b]) continue;
+                for (int h = 0; h < Hq; ++h) {
+                    const int g = h / G;
+                    const uint16_t *qrow = q + (((int64_t)b * S + i) * Hq + h) * D;
+                    const uint16_t *kb = k + (((int64_t)b * S) * Hkv + g) * D;
+                    const uint16_t *vb = v + (((int64_t)b * S) * Hkv + g) * D;
+                    attend_row(qrow, kb, (int64_t)Hkv * D, vb, (int64_t)Hkv * D,
+                               i + 1, D, scale, p,
+                               out + (((int64_t)b * S + i) * Hq + h) * D,
+                               lse ? lse + ((int64_t)b * Hq + h) * S + i : NULL);
+                }
+            }
+        }
+        free(p);
+    }
+    return fail ? -1 : 0;
+}
+
+/*
+ * Causal prefill of a LIST of rows (for sizes where every row would take too long).
+ *   rows     [n_rows, 3]    (b, i, h) triples, each with i < seq_len[b]
+ *   out      [n_rows, D]    lse [n_rows] or NULL
+ */
+int l4l_oracle_prefill_rows(const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                            const int32_t *seq_len, int B, int S, int Hq, int Hkv, int D,
+                            double scale, const int32_t *rows, int n_rows,
+                            double *out, double *lse)
+{
+    if (Hkv <= 0 || Hq % Hkv != 0) return -1;
+    const int G = Hq / Hkv;
+    int fail = 0;
+    for (int r = 0; r < n_rows; ++r) {
+        int b = rows[3 * r], i = rows[3 * r + 1], h = rows[3 * r + 2];
+        if (b < 0 || b >= B || h < 0 || h >= Hq || i < 0 || i >= seq_len[b]) return -1;
+    }
+#pragma omp parallel
+    {
+        double *p = (double *)malloc(sizeof(double) * (size_t)(S > 0 ? S : 1));
+        if (!p) {
+#pragma omp atomic write
+            fail = 1;
+        }
+#pragma omp for schedule(dynamic, 1)
+        for (int r = 0; r < n_rows; ++r) {
+            if (!p) continue;
+            const int b = rows[3 * r], i = rows[3 * r + 1], h = rows[3 * r + 2];
+            const int g = h / G;
+            attend_row(q + (((int64_t)b * S + i) * Hq + h) * D,
+                       k + (((int64_t)b * S) * Hkv + g) * D, (int64_t)Hkv * D,
+                       v + (((int64_t)b * S) * Hkv + g) * D, (int64_t)Hkv * D,
+                       i + 1, D, scale, p, out + (int64_t)r * D, lse ? lse + r : NULL);
+        }
+        free(p);
+    }
+    return fail ? -1 : 0;
+}
+
+/*
+ * Decode: one query token per sequence over the populated cache (no mask).
+ *   q        [B, Hq, D]           cache_k, cache_v  [B, Hkv, Lmax, D]
+ *   kv_len   [B]   valid tokens, the current one included (<= Lmax)
+ *   out      [B, Hq, D] fp64      lse [B, Hq] fp64 or NULL
+ */
+int l4l_oracle_decode(const uint16_t *q, const uint16_t *cache_k, const uint16_t *cache_v,
+                      const int32_t *kv_len, int B, int Hq, int Hkv, int D, int Lmax,
+                      double scale, double *out, double *lse)
+{
+    if (Hkv <= 0 || Hq % Hkv != 0) return -1;
+    const int G = Hq / Hkv;
+    int fail = 0;
+#pragma omp parallel
+    {
+        double *p = (double *)malloc(sizeof(double) * (size_t)(Lmax > 0 ? Lmax : 1));
+        if (!p) {
+#pragma omp atomic write
+            fail = 1;
+        }
+#pragma omp for collapse(2) schedule(dynamic, 1)
+        for (int b = 0; b < B; ++b) {
+            for (int h = 0; h < Hq; ++h) {
+                if (!p) continue;
+                const int g = h / G;
+                const int64_t base = ((int64_t)b * Hkv + g) * Lmax * D;
+                attend_row(q + ((int64_t)b * Hq + h) * D, cache_k + base, D,
+                           cache_v + base, D, kv_len[b], D, scale, p,
+                           out + ((int64_t)b * Hq + h) * D,
+                           lse ? lse + (int64_t)b * Hq + h : NULL);
+            }
+        }
+        free(p);
+    }
+    return fail ? -1 : 0;
+}
+
+/*
+ * Cache copy. Writes n_new[b] tokens of k_new / v_new ([B, T, Hkv, D]) into the cache
+ * ([B, Hkv, Lmax, D]) at slots pos[b] .. pos[b]+n_new[b]-1, as raw 16-bit words.
+ * Everything else in the cache is left as it was. The prefill cache write is the case
+ * pos = 0, n_new = seq_len; the decode-step append is the case T = 1, n_new = 1.
+ * Returns -1 if a write would fall outside [0, Lmax).
+ */
+int l4l_oracle_kv_append(uint16_t *cache_k, uint16_t *cache_v, const uint16_t *k_new,
+                         const uint16_t *v_new, const int32_t *pos, const int32_t *n_new,
+                         int B, int T, int Hkv, int D, int Lmax)
+{
+    for (int b = 0; b < B; ++b)
+        if (n_new[b] < 0 || n_new[b] > T || pos[b] < 0 || pos[b] + n_new[b] > Lmax) return -1;
+    for (int b = 0; b < B; ++b)
+        for (int r = 0; r < n_new[b]; ++r)
+            for (int g = 0; g < Hkv; ++g)
+                for (int d = 0; d < D; ++d) {
+                    const int64_t src = (((int64_t)b * T + r) * Hkv + g) * D + d;
+                    const int64_t dst = (((int64_t)b * Hkv + g) * Lmax + pos[b] + r) * D + d;
+                    cache_k[dst] = k_new[src];
+                    cache_v[dst] = v_new[src];
+                }
+    return 0;
+}

@@ -1,0 +1,153 @@
+"""ctypes front end of the CPU oracle (``l4l_oracle.c``).
+
+TEST INFRASTRUCTURE, NOT THE PRODUCT: only the tests, the smoke check and the
+benchmark's CPU-baseline leg may import this module. It shares no code with the CUDA
+path. All arithmetic lives in the C file; this file only builds it with gcc, turns
+arrays into pointers and allocates the fp64 outputs.
+
+Inputs are bf16 given either as ``torch.bfloat16`` CPU tensors or as numpy ``uint16``
+arrays of the raw bits; outputs are numpy ``float64`` (caches: ``uint16`` bits).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "l4l_oracle.c")
+_LIB = os.path.join(_HERE, "libl4l_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (-O2, OpenMP); returns the path of the library."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(
+            ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", tmp, _SRC, "-lm"]
+        )
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        u16p = ctypes.POINTER(ctypes.c_uint16)
+        i32p = ctypes.POINTER(ctypes.c_int32)
+        f64p = ctypes.POINTER(ctypes.c_double)
+        i, d = ctypes.c_int, ctypes.c_double
+        lib.l4l_oracle_num_threads.restype = i
+        lib.l4l_oracle_prefill.argtypes = [u16p, u16p, u16p, i32p, i, i, i, i, i, d, f64p, f64p]
+        lib.l4l_oracle_prefill_rows.argtypes = [u16p, u16p, u16p, i32p, i, i, i, i, i, d,
+                                                i32p, i, f64p, f64p]
+        lib.l4l_oracle_decode.argtypes = [u16p, u16p, u16p, i32p, i, i, i, i, i, d, f64p, f64p]
+        lib.l4l_oracle_kv_append.argtypes = [u16p, u16p, u16p, u16p, i32p, i32p, i, i, i, i, i]
+        _lib = lib
+    return _lib
+
+
+def num_threads() -> int:
+    return int(_load().l4l_oracle_num_threads())
+
+
+def bits(x) -> np.ndarray:
+    """Raw bf16 bits as a C-contiguous uint16 array (accepts torch.bfloat16 or uint16)."""
+    if isinstance(x, np.ndarray):
+        if x.dtype != np.uint16:
+            raise TypeError("numpy input must be uint16 bf16 bits")
+        return np.ascontiguousarray(x)
+    import torch  # device memory / tensor container only
+
+    if x.dtype != torch.bfloat16:
+        raise TypeError("tensor input must be bfloat16")
+    return np.ascontiguousarray(x.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16))
+
+
+def _p(a, ty):
+    return a.ctypes.data_as(ctypes.POINTER(ty))
+
+
+def _i32(x) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(x, dtype=np.int32))
+
+
+def prefill(q, k, v, seq_len, scale: float):
+    """Causal prefill. q [B,S,Hq,D], k/v [B,S,Hkv,D]; returns (out [B,S,Hq,D], lse [B,Hq,S]).
+
+    Rows i >= seq_len[b] are NaN in both outputs (they are not defined)."""
+    q, k, v = bits(q), bits(k), bits(v)
+    B, S, Hq, D = q.shape
+    Hkv = k.shape[2]
+    assert k.shape == (B, S, Hkv, D) and v.shape == k.shape
+    sl = _i32(seq_len)
+    assert sl.shape == (B,) and (sl >= 0).all() and (sl <= S).all()
+    out = np.full((B, S, Hq, D), np.nan, dtype=np.float64)
+    lse = np.full((B, Hq, S), np.nan, dtype=np.float64)
+    rc = _load().l4l_oracle_prefill(_p(q, ctypes.c_uint16), _p(k, ctypes.c_uint16),
+                                    _p(v, ctypes.c_uint16), _p(sl, ctypes.c_int32),
+                                    B, S, Hq, Hkv, D, float(scale),
+                                    _p(out, ctypes.c_double), _p(lse, ctypes.c_double))
+    if rc != 0:
+        raise ValueError("l4l_oracle_prefill rejected its arguments")
+    return out, lse
+
+
+def prefill_rows(q, k, v, seq_len, scale: float, rows):
+    """Causal prefill of the listed (b, i, h) rows only; returns (out [n,D], lse [n])."""
+    q, k, v = bits(q), bits(k), bits(v)
+    B, S, Hq, D = q.shape
+    Hkv = k.shape[2]
+    sl = _i32(seq_len)
+    rows = _i32(rows).reshape(-1, 3)
+    n = rows.shape[0]
+    out = np.empty((n, D), dtype=np.float64)
+    lse = np.empty((n,), dtype=np.float64)
+    rc = _load().l4l_oracle_prefill_rows(_p(q, ctypes.c_uint16), _p(k, ctypes.c_uint16),
+                                         _p(v, ctypes.c_uint16), _p(sl, ctypes.c_int32),
+                                         B, S, Hq, Hkv, D, float(scale),
+                                         _p(rows, ctypes.c_int32), n,
+                                         _p(out, ctypes.c_double), _p(lse, ctypes.c_double))
+    if rc != 0:
+        raise ValueError("l4l_oracle_prefill_rows rejected its arguments")
+    return out, lse
+
+
+def decode(q, cache_k, cache_v, kv_len, scale: float):
+    """Decode. q [B,Hq,D], caches [B,Hkv,Lmax,D]; returns (out [B,Hq,D], lse [B,Hq])."""
+    q, ck, cv = bits(q), bits(cache_k), bits(cache_v)
+    B, Hq, D = q.shape
+    _, Hkv, Lmax, _ = ck.shape
+    assert ck.shape == (B, Hkv, Lmax, D) and cv.shape == ck.shape
+    kl = _i32(kv_len)
+    assert kl.shape == (B,) and (kl >= 0).all() and (kl <= Lmax).all()
+    out = np.empty((B, Hq, D), dtype=np.float64)
+    lse = np.empty((B, Hq), dtype=np.float64)
+    rc = _load().l4l_oracle_decode(_p(q, ctypes.c_uint16), _p(ck, ctypes.c_uint16),
+                                   _p(cv, ctypes.c_uint16), _p(kl, ctypes.c_int32),
+                                   B, Hq, Hkv, D, Lmax, float(scale),
+                                   _p(out, ctypes.c_double), _p(lse, ctypes.c_double))
+    if rc != 0:
+        raise ValueError("l4l_oracle_decode rejected its arguments")
+    return out, lse
+
+
+def kv_append(cache_k, cache_v, k_new, v_new, pos, n_new):
+    """Returns copies of the caches (uint16 bits) with the new tokens written in."""
+    ck, cv = bits(cache_k).copy(), bits(cache_v).copy()
+    kn, vn = bits(k_new), bits(v_new)
+    B, Hkv, Lmax, D = ck.shape
+    T = kn.shape[1]
+    assert kn.shape == (B, T, Hkv, D) and vn.shape == kn.shape
+    pos, n_new = _i32(pos), _i32(n_new)
+    rc = _load().l4l_oracle_kv_append(_p(ck, ctypes.c_uint16), _p(cv, ctypes.c_uint16),
+                                      _p(kn, ctypes.c_uint16), _p(vn, ctypes.c_uint16),
+                                      _p(pos, ctypes.c_int32), _p(n_new, ctypes.c_int32),
+                                      B, T, Hkv, D, Lmax)
+    if rc != 0:
+        raise ValueError("l4l_oracle_kv_append: write outside the cache")
+    return ck, cv

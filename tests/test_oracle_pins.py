@@ -1,0 +1,336 @@
+"""Pins of the CPU oracle against what softmax attention fixes by definition.
+
+The paper prints no formula and no worked numeric example for attention, so nothing
+here comes from a printed value; every pin is a closed form, an invariant, a special
+case that reduces to a textbook/library routine, or brute force on tiny inputs. Each is
+chosen so that a plausible slip in the oracle (dropped scale, wrong head mapping,
+off-by-one causal bound, transposed operand, missing normalisation) fails at least one.
+"""
+import math
+import struct
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import l4l_oracle as orc
+
+
+def bf16(x: torch.Tensor) -> torch.Tensor:
+    return x.to(torch.bfloat16)
+
+
+def randn(shape, seed, scale=1.0):
+    g = torch.Generator().manual_seed(seed)
+    return bf16(torch.randn(shape, generator=g) * scale)
+
+
+def f64(x: torch.Tensor) -> np.ndarray:
+    return x.to(torch.float64).numpy()
+
+
+def full_lens(B, S):
+    return np.full((B,), S, dtype=np.int32)
+
+
+def cache_from(k: torch.Tensor) -> torch.Tensor:
+    """[B, L, Hkv, D] token-major -> cache layout [B, Hkv, L, D]."""
+    return k.permute(0, 2, 1, 3).contiguous()
+
+
+# --------------------------------------------------------------------------- I5 brute force
+def _bf16_bits_to_float(bits: int) -> float:
+    return struct.unpack("<f", struct.pack("<I", (bits & 0xFFFF) << 16))[0]
+
+
+def brute_force_row(qrow, keys, vals, scale):
+    """Independent evaluation in pure Python: no max subtraction, d-outer loop order,
+    exact-sum accumulation with math.fsum."""
+    n, D = len(keys), len(qrow)
+    s = [0.0] * n
+    for d in range(D):
+        for j in range(n):
+            s[j] += qrow[d] * keys[j][d]
+    w = [math.exp(scale * sj) for sj in s]
+    z = math.fsum(w)
+    out = [math.fsum(w[j] * vals[j][d] for j in range(n)) / z for d in range(D)]
+    return out, math.log(z)
+
+
+@pytest.mark.parametrize("B,S,Hq,Hkv,D", [(2, 8, 4, 2, 8), (1, 5, 3, 1, 4), (2, 7, 2, 2, 6)])
+def test_I5_bruteforce_prefill_and_decode(B, S, Hq, Hkv, D):
+    q, k, v = randn((B, S, Hq, D), 1), randn((B, S, Hkv, D), 2), randn((B, S, Hkv, D), 3)
+    scale = 0.37
+    out, lse = orc.prefill(q, k, v, full_lens(B, S), scale)
+    qb, kb, vb = orc.bits(q), orc.bits(k), orc.bits(v)
+    G = Hq // Hkv
+    for b in range(B):
+        for i in range(S):
+            for h in range(Hq):
+                g = h // G
+                qrow = [_bf16_bits_to_float(int(x)) for x in qb[b, i, h]]
+                keys = [[_bf16_bits_to_float(int(x)) for x in kb[b, j, g]] for j in range(i + 1)]
+                vals = [[_bf16_bits_to_float(int(x)) for x in vb[b, j, g]] for j in range(i + 1)]
+                ref, ref_lse = brute_force_row(qrow, keys, vals, scale)
+                np.testing.assert_allclose(out[b, i, h], ref, rtol=0, atol=1e-12)
+                assert abs(lse[b, h, i] - ref_lse) < 1e-12
+    # decode over the same data, all tokens visible
+    dq = q[:, -1].contiguous()
+    dout, dlse = orc.decode(dq, cache_from(k), cache_from(v), full_lens(B, S), scale)
+    np.testing.assert_allclose(dout, out[:, -1], rtol=0, atol=1e-13)
+    np.testing.assert_allclose(dlse, lse[:, :, -1], rtol=0, atol=1e-13)
+
+
+# --------------------------------------------------------------------------- I1 identical keys
+def test_I1_identical_keys_give_prefix_mean_of_v():
+    B, S, Hq, Hkv, D = 2, 33, 4, 2, 16
+    q = randn((B, S, Hq, D), 4)
+    k = randn((B, 1, Hkv, D), 5).expand(B, S, Hkv, D).contiguous()
+    v = randn((B, S, Hkv, D), 6)
+    out, lse = orc.prefill(q, k, v, full_lens(B, S), 0.25)
+    vv = f64(v)
+    counts = np.arange(1, S + 1, dtype=np.float64)[None, :, None, None]
+    pm = np.cumsum(vv, axis=1) / counts                 # prefix mean  [B,S,Hkv,D]
+    np.testing.assert_allclose(out, np.repeat(pm, Hq // Hkv, axis=2), rtol=0, atol=1e-13)
+    # lse = common score + log(number of keys)
+    s = 0.25 * np.einsum("bihd,bhd->bih", f64(q), np.repeat(f64(k)[:, 0], Hq // Hkv, axis=1))
+    np.testing.assert_allclose(lse, (s + np.log(counts[..., 0])).transpose(0, 2, 1), rtol=0, atol=1e-12)
+    dout, _ = orc.decode(q[:, -1].contiguous(), cache_from(k), cache_from(v), full_lens(B, S), 0.25)
+    np.testing.assert_allclose(dout, np.repeat(vv.mean(axis=1), Hq // Hkv, axis=1), rtol=0, atol=1e-13)
+
+
+# --------------------------------------------------------------------------- I2 dominant key
+def test_I2_single_dominant_score_returns_its_v_row():
+    B, S, H, D = 1, 24, 2, 8
+    q = bf16(torch.ones(B, S, H, D))
+    k = bf16(torch.zeros(B, S, H, D))
+    jstar = 5
+    k[:, jstar] = 16.0                                   # score 16*8 = 128 above the rest
+    v = randn((B, S, H, D), 7)
+    out, _ = orc.prefill(q, k, v, full_lens(B, S), 1.0)
+    vv = f64(v)
+    for i in range(jstar, S):
+        np.testing.assert_allclose(out[0, i], vv[0, jstar], rtol=0, atol=1e-30 + i * math.exp(-128) * 10)
+    # before the dominant key is visible all scores tie: prefix mean
+    np.testing.assert_allclose(out[0, jstar - 1], vv[0, :jstar].mean(axis=0), rtol=0, atol=1e-13)
+    dout, _ = orc.decode(q[:, -1].contiguous(), cache_from(k), cache_from(v), full_lens(B, S), 1.0)
+    np.testing.assert_allclose(dout[0], vv[0, jstar], rtol=0, atol=1e-30)
+
+
+# --------------------------------------------------------------------------- I3 causality
+def test_I3_future_tokens_do_not_change_earlier_rows():
+    B, S, Hq, Hkv, D = 1, 20, 4, 2, 8
+    q, k, v = randn((B, S, Hq, D), 8), randn((B, S, Hkv, D), 9), randn((B, S, Hkv, D), 10)
+    out0, lse0 = orc.prefill(q, k, v, full_lens(B, S), 0.3)
+    cut = 11
+    q2, k2, v2 = q.clone(), k.clone(), v.clone()
+    q2[:, cut:], k2[:, cut:], v2[:, cut:] = randn((B, S - cut, Hq, D), 11), 7.0, -3.0
+    out1, lse1 = orc.prefill(q2, k2, v2, full_lens(B, S), 0.3)
+    assert np.array_equal(out0[:, :cut], out1[:, :cut])
+    assert np.array_equal(lse0[:, :, :cut], lse1[:, :, :cut])
+    assert not np.array_equal(out0[:, cut:], out1[:, cut:])
+    # the diagonal IS visible: changing token i's own k/v changes row i
+    k3 = k.clone()
+    k3[:, cut - 1] = 2.0
+    out2, _ = orc.prefill(q, k3, v, full_lens(B, S), 0.3)
+    assert np.array_equal(out0[:, : cut - 1], out2[:, : cut - 1])
+    assert not np.array_equal(out0[:, cut - 1], out2[:, cut - 1])
+
+
+def test_ragged_seq_len_ignores_padding_and_leaves_rows_undefined():
+    B, S, Hq, Hkv, D = 2, 12, 2, 1, 8
+    q, k, v = randn((B, S, Hq, D), 12), randn((B, S, Hkv, D), 13), randn((B, S, Hkv, D), 14)
+    lens = np.array([7, 12], dtype=np.int32)
+    out, lse = orc.prefill(q, k, v, lens, 0.5)
+    full, _ = orc.prefill(q, k, v, full_lens(B, S), 0.5)
+    assert np.array_equal(out[0, :7], full[0, :7]) and np.array_equal(out[1], full[1])
+    assert np.isnan(out[0, 7:]).all() and np.isnan(lse[0, :, 7:]).all()
+
+
+# --------------------------------------------------------------------------- I4 phase equivalence
+def test_I4_decode_step_equals_prefill_row():
+    B, L, Hq, Hkv, D = 2, 19, 4, 2, 8
+    q, k, v = randn((B, L, Hq, D), 15), randn((B, L, Hkv, D), 16), randn((B, L, Hkv, D), 17)
+    out, lse = orc.prefill(q, k, v, full_lens(B, L), 0.41)
+    Lmax = 32
+    ck = torch.zeros(B, Hkv, Lmax, D, dtype=torch.bfloat16)
+    cv = torch.zeros_like(ck)
+    ck[:, :, :L], cv[:, :, :L] = cache_from(k), cache_from(v)
+    ck[:, :, L:], cv[:, :, L:] = float("nan"), float("nan")      # must never be read
+    for t in (0, 1, 7, L - 1):
+        dout, dlse = orc.decode(q[:, t].contiguous(), ck, cv, full_lens(B, t + 1), 0.41)
+        np.testing.assert_allclose(dout, out[:, t], rtol=0, atol=1e-14)
+        np.testing.assert_allclose(dlse, lse[:, :, t], rtol=0, atol=1e-14)
+
+
+# --------------------------------------------------------------------------- I6, I7
+def test_I6_first_row_is_v0_exactly_and_empty_is_zero():
+    B, S, Hq, Hkv, D = 2, 4, 4, 2, 8
+    q, k, v = randn((B, S, Hq, D), 18), randn((B, S, Hkv, D), 19), randn((B, S, Hkv, D), 20)
+    out, lse = orc.prefill(q, k, v, full_lens(B, S), 0.7)
+    assert np.array_equal(out[:, 0], np.repeat(f64(v)[:, 0], Hq // Hkv, axis=1))
+    s00 = 0.7 * np.einsum("bhd,bhd->bh", f64(q)[:, 0], np.repeat(f64(k)[:, 0], Hq // Hkv, axis=1))
+    np.testing.assert_allclose(lse[:, :, 0], s00, rtol=0, atol=1e-14)
+    dout, _ = orc.decode(q[:, 0].contiguous(), cache_from(k), cache_from(v), full_lens(B, 1), 0.7)
+    assert np.array_equal(dout, out[:, 0])
+    dout0, dlse0 = orc.decode(q[:, 0].contiguous(), cache_from(k), cache_from(v), np.zeros(B, np.int32), 0.7)
+    assert (dout0 == 0).all() and np.isneginf(dlse0).all()
+
+
+def test_I7_zero_scale_gives_running_mean():
+    B, S, Hq, Hkv, D = 1, 40, 2, 2, 4
+    q, k, v = randn((B, S, Hq, D), 21), randn((B, S, Hkv, D), 22), randn((B, S, Hkv, D), 23)
+    out, lse = orc.prefill(q, k, v, full_lens(B, S), 0.0)
+    counts = np.arange(1, S + 1, dtype=np.float64)[None, :, None, None]
+    np.testing.assert_allclose(out, np.cumsum(f64(v), axis=1) / counts, rtol=0, atol=1e-13)
+    np.testing.assert_allclose(lse[0, 0], np.log(counts[0, :, 0, 0]), rtol=0, atol=1e-13)
+
+
+# --------------------------------------------------------------------------- I8 head mapping
+def test_I8_gqa_equals_mha_with_consecutively_repeated_kv_heads():
+    B, S, Hq, Hkv, D = 1, 16, 8, 2, 8
+    G = Hq // Hkv
+    q, k, v = randn((B, S, Hq, D), 24), randn((B, S, Hkv, D), 25), randn((B, S, Hkv, D), 26)
+    out, lse = orc.prefill(q, k, v, full_lens(B, S), 0.35)
+    kr, vr = k.repeat_interleave(G, dim=2), v.repeat_interleave(G, dim=2)
+    out_mha, lse_mha = orc.prefill(q, kr, vr, full_lens(B, S), 0.35)
+    assert np.array_equal(out, out_mha) and np.array_equal(lse, lse_mha)
+    # the rejected convention (h % Hkv) would tile, not interleave: it must differ
+    out_tiled, _ = orc.prefill(q, k.repeat(1, 1, G, 1), v.repeat(1, 1, G, 1), full_lens(B, S), 0.35)
+    assert not np.array_equal(out, out_tiled)
+    # decode uses the same mapping
+    dout, _ = orc.decode(q[:, -1].contiguous(), cache_from(k), cache_from(v), full_lens(B, S), 0.35)
+    dmha, _ = orc.decode(q[:, -1].contiguous(), cache_from(kr), cache_from(vr), full_lens(B, S), 0.35)
+    assert np.array_equal(dout, dmha)
+
+
+def test_kv_head_only_feeds_its_own_query_group():
+    B, S, Hq, Hkv, D = 1, 9, 6, 3, 4
+    G = Hq // Hkv
+    q, k, v = randn((B, S, Hq, D), 27), randn((B, S, Hkv, D), 28), randn((B, S, Hkv, D), 29)
+    out0, _ = orc.prefill(q, k, v, full_lens(B, S), 0.5)
+    v2 = v.clone()
+    v2[:, :, 1] += 1.0
+    out1, _ = orc.prefill(q, k, v2, full_lens(B, S), 0.5)
+    changed = [h for h in range(Hq) if not np.array_equal(out0[:, :, h], out1[:, :, h])]
+    assert changed == list(range(G, 2 * G))
+
+
+# --------------------------------------------------------------------------- I9, I10, I11
+def test_I9_adding_a_constant_vector_to_every_key_changes_nothing():
+    B, S, H, D = 1, 12, 2, 8
+    # dyadic values so that k + c is exact in bf16
+    g = torch.Generator().manual_seed(30)
+    q = bf16(torch.randint(-8, 9, (B, S, H, D), generator=g) / 8.0)
+    k = bf16(torch.randint(-8, 9, (B, S, H, D), generator=g) / 8.0)
+    v = randn((B, S, H, D), 31)
+    c = bf16(torch.randint(-8, 9, (1, 1, H, D), generator=g) / 4.0)
+    out0, lse0 = orc.prefill(q, k, v, full_lens(B, S), 0.125)
+    out1, lse1 = orc.prefill(q, bf16(k.float() + c.float()), v, full_lens(B, S), 0.125)
+    np.testing.assert_allclose(out0, out1, rtol=0, atol=1e-13)
+    shift = 0.125 * np.einsum("bihd,hd->bhi", f64(q), f64(c)[0, 0])
+    np.testing.assert_allclose(lse1 - lse0, shift, rtol=0, atol=1e-12)
+
+
+def test_I10_decode_is_invariant_to_a_joint_permutation_of_cache_tokens():
+    B, L, Hq, Hkv, D = 2, 23, 4, 2, 8
+    q = randn((B, Hq, D), 32)
+    ck, cv = randn((B, Hkv, L, D), 33), randn((B, Hkv, L, D), 34)
+    perm = torch.randperm(L, generator=torch.Generator().manual_seed(35))
+    out0, lse0 = orc.decode(q, ck, cv, full_lens(B, L), 0.3)
+    out1, lse1 = orc.decode(q, ck[:, :, perm].contiguous(), cv[:, :, perm].contiguous(), full_lens(B, L), 0.3)
+    np.testing.assert_allclose(out0, out1, rtol=0, atol=1e-13)
+    np.testing.assert_allclose(lse0, lse1, rtol=0, atol=1e-13)
+    # permuting K alone is a different problem
+    out2, _ = orc.decode(q, ck[:, :, perm].contiguous(), cv, full_lens(B, L), 0.3)
+    assert np.abs(out2 - out0).max() > 1e-3
+
+
+def test_I11_linear_in_v_and_constant_v_gives_constant():
+    B, S, H, D = 1, 14, 2, 8
+    q, k = randn((B, S, H, D), 36), randn((B, S, H, D), 37)
+    g = torch.Generator().manual_seed(38)
+    v1 = bf16(torch.randint(-16, 17, (B, S, H, D), generator=g) / 8.0)
+    v2 = bf16(torch.randint(-16, 17, (B, S, H, D), generator=g) / 8.0)
+    o1, _ = orc.prefill(q, k, v1, full_lens(B, S), 0.3)
+    o2, _ = orc.prefill(q, k, v2, full_lens(B, S), 0.3)
+    o12, _ = orc.prefill(q, k, bf16(2.0 * v1.float() - 0.5 * v2.float()), full_lens(B, S), 0.3)
+    np.testing.assert_allclose(o12, 2.0 * o1 - 0.5 * o2, rtol=0, atol=1e-13)
+    oc, _ = orc.prefill(q, k, bf16(torch.full((B, S, H, D), 1.75)), full_lens(B, S), 0.3)
+    np.testing.assert_allclose(oc, 1.75, rtol=0, atol=1e-14)
+
+
+# --------------------------------------------------------------------------- I12 split/merge
+def test_I12_lse_merge_of_any_partition_equals_the_whole():
+    B, L, Hq, Hkv, D = 1, 50, 4, 2, 8
+    q = randn((B, Hq, D), 39)
+    ck, cv = randn((B, Hkv, L, D), 40, 2.0), randn((B, Hkv, L, D), 41)
+    whole, whole_lse = orc.decode(q, ck, cv, full_lens(B, L), 0.4)
+    cuts = [0, 3, 4, 21, 50]
+    parts = []
+    for a, b in zip(cuts[:-1], cuts[1:]):
+        o, l = orc.decode(q, ck[:, :, a:b].contiguous(), cv[:, :, a:b].contiguous(), full_lens(B, b - a), 0.4)
+        parts.append((o, l))
+    lses = np.stack([l for _, l in parts])                # [C,B,Hq]
+    m = lses.max(axis=0)
+    w = np.exp(lses - m)
+    merged = sum(w[c][..., None] * parts[c][0] for c in range(len(parts))) / w.sum(axis=0)[..., None]
+    np.testing.assert_allclose(merged, whole, rtol=0, atol=1e-13)
+    np.testing.assert_allclose(m + np.log(w.sum(axis=0)), whole_lse, rtol=0, atol=1e-13)
+
+
+# --------------------------------------------------------------------------- I13 library routine
+@pytest.mark.parametrize("B,S,Hq,Hkv,D", [(2, 37, 4, 2, 16), (1, 64, 6, 6, 8)])
+def test_I13_matches_torch_sdpa_float64(B, S, Hq, Hkv, D):
+    q, k, v = randn((B, S, Hq, D), 42), randn((B, S, Hkv, D), 43), randn((B, S, Hkv, D), 44)
+    scale = 1.0 / math.sqrt(D)
+    out, _ = orc.prefill(q, k, v, full_lens(B, S), scale)
+    G = Hq // Hkv
+    qq = q.double().permute(0, 2, 1, 3)
+    kk = k.double().repeat_interleave(G, dim=2).permute(0, 2, 1, 3)
+    vv = v.double().repeat_interleave(G, dim=2).permute(0, 2, 1, 3)
+    ref = torch.nn.functional.scaled_dot_product_attention(qq, kk, vv, is_causal=True, scale=scale)
+    np.testing.assert_allclose(out, ref.permute(0, 2, 1, 3).numpy(), rtol=0, atol=1e-12)
+    dref = torch.nn.functional.scaled_dot_product_attention(qq[:, :, -1:], kk, vv, is_causal=False, scale=scale)
+    dout, _ = orc.decode(q[:, -1].contiguous(), cache_from(k), cache_from(v), full_lens(B, S), scale)
+    np.testing.assert_allclose(dout, dref[:, :, 0].numpy(), rtol=0, atol=1e-12)
+
+
+def test_prefill_rows_is_the_same_function_as_prefill():
+    B, S, Hq, Hkv, D = 2, 21, 4, 2, 8
+    q, k, v = randn((B, S, Hq, D), 45), randn((B, S, Hkv, D), 46), randn((B, S, Hkv, D), 47)
+    lens = np.array([21, 13], dtype=np.int32)
+    out, lse = orc.prefill(q, k, v, lens, 0.2)
+    rows = [(0, 0, 0), (0, 20, 3), (1, 12, 1), (1, 5, 2)]
+    o, l = orc.prefill_rows(q, k, v, lens, 0.2, rows)
+    for r, (b, i, h) in enumerate(rows):
+        assert np.array_equal(o[r], out[b, i, h]) and l[r] == lse[b, h, i]
+    with pytest.raises(ValueError):
+        orc.prefill_rows(q, k, v, lens, 0.2, [(1, 13, 0)])
+
+
+# --------------------------------------------------------------------------- cache copy
+def test_kv_append_is_a_bit_exact_copy_and_touches_nothing_else():
+    B, T, Hkv, D, Lmax = 3, 4, 2, 8, 16
+    g = torch.Generator().manual_seed(48)
+    # all 16-bit patterns are legal payload (NaNs, -0, denormals): use raw random bits
+    def rawbits(shape):
+        return torch.randint(0, 65536, shape, generator=g, dtype=torch.int32).to(torch.int16).view(torch.bfloat16)
+    ck, cv = rawbits((B, Hkv, Lmax, D)), rawbits((B, Hkv, Lmax, D))
+    kn, vn = rawbits((B, T, Hkv, D)), rawbits((B, T, Hkv, D))
+    pos = np.array([0, 5, 12], dtype=np.int32)
+    n_new = np.array([4, 0, 3], dtype=np.int32)
+    ok, ov = orc.kv_append(ck, cv, kn, vn, pos, n_new)
+    ek, ev = orc.bits(ck).copy(), orc.bits(cv).copy()
+    knb, vnb = orc.bits(kn), orc.bits(vn)
+    for b in range(B):
+        n = int(n_new[b])
+        ek[b, :, pos[b]:pos[b] + n] = knb[b, :n].transpose(1, 0, 2)
+        ev[b, :, pos[b]:pos[b] + n] = vnb[b, :n].transpose(1, 0, 2)
+    assert np.array_equal(ok, ek) and np.array_equal(ov, ev)
+    with pytest.raises(ValueError):
+        orc.kv_append(ck, cv, kn, vn, np.array([0, 5, 14], np.int32), n_new)
+
+
+def test_oracle_reports_thread_count():
+    assert orc.num_threads() >= 1
