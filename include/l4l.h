@@ -1,0 +1,155 @@
+/*
+ * l4l.h — C ABI of the B200 (sm_100a) causal-attention hot path.
+ *
+ * The operations are the ones the paper's appendix on accepted kernels ("Transformer
+ * attention", Table A.4) names as the attention module's two phases plus the cache
+ * update that surrounds them:
+ *
+ *   l4l_attn_prefill   q_len > 1 : causal grouped-query attention over the prompt; the KV
+ *                                  head of a query head follows from the grouped-query
+ *                                  structure, the causal mask is part of the score update,
+ *                                  softmax statistics are kept in fp32; the prompt's K and V
+ *                                  are written to the cache in the same pass.
+ *   l4l_attn_decode    q_len = 1 : one query token per sequence over a populated, ragged KV
+ *                                  cache; all query heads of a KV group are served by one
+ *                                  pass over that group's cache.
+ *   l4l_kv_append                : the cache update (an exact copy).
+ *
+ * Conventions shared by every call
+ *   - All tensors are bf16 (16-bit words) in DEVICE memory unless a parameter says "host".
+ *     head_dim (D) is the contiguous innermost dimension; the other strides are passed in
+ *     ELEMENTS. Every base pointer must be 16-byte aligned and every stride a multiple of 8
+ *     elements (16 bytes), because tiles move with TMA.
+ *   - Query head h reads KV head h / (Hq / Hkv): consecutive query heads share a KV head.
+ *   - The caller owns every buffer. The library allocates no device memory, enqueues its
+ *     kernels on the caller's stream and never synchronises (l4l_last_device_error excepted).
+ *     Sequence lengths live in device memory; only upper bounds come from the host.
+ *   - Errors: arguments are validated on the host BEFORE anything is launched; a non-zero
+ *     status means no kernel of that call ran. Nothing throws, nothing traps on the device.
+ *     Unsupported shapes return L4L_ERR_UNSUPPORTED; there is no fallback path.
+ *       supported: head_dim in {64, 128}; Hq % Hkv == 0; Hq / Hkv <= 16.
+ *   - Device-side waits (TMA / tensor-core pipeline barriers) are bounded. If one ever runs
+ *     out, the kernel records a code in the workspace's status block and returns; the host
+ *     sees it through l4l_last_device_error().
+ */
+#ifndef L4L_H
+#define L4L_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    L4L_OK = 0,
+    L4L_ERR_INVALID_ARG = 1, /* null pointer, negative size, misaligned pointer or stride      */
+    L4L_ERR_UNSUPPORTED = 2, /* head_dim / head grouping outside the supported set             */
+    L4L_ERR_WORKSPACE = 3,   /* workspace missing or too small                                  */
+    L4L_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed (launch, tensor-map encode) */
+    L4L_ERR_TIMEOUT = 5      /* a bounded device-side wait ran out (see l4l_last_device_error)  */
+} l4l_status;
+
+/* A cudaStream_t, passed as an opaque pointer (NULL = the legacy default stream). */
+typedef void *l4l_stream;
+
+/* bf16 [B, T, H, D] view: element (b, t, h, d) is at ptr + b*stride_b + t*stride_t + h*stride_h + d. */
+typedef struct {
+    void *ptr;
+    int64_t stride_b, stride_t, stride_h;
+} l4l_tensor4;
+
+/* bf16 KV cache: element (b, kv_head, slot, d) of K is at k + b*stride_b + kv_head*stride_h +
+ * slot*stride_t + d (V likewise). The default dense layout is [B, Hkv, max_len, D]; any
+ * layout expressible by these strides (e.g. [B, max_len, Hkv, D]) is accepted. Not paged.
+ * max_len = number of token slots per sequence. */
+typedef struct {
+    void *k;
+    void *v;
+    int64_t stride_b, stride_h, stride_t;
+    int32_t max_len;
+} l4l_kv_cache;
+
+enum { L4L_OP_PREFILL = 0, L4L_OP_DECODE = 1 };
+
+/*
+ * Bytes of device workspace the given operation needs for these sizes (max_len = the largest
+ * S_max / max_kv_len it will be called with). Always >= 256: the first 256 bytes are the
+ * status block. Returns 0 for unsupported arguments.
+ */
+size_t l4l_workspace_bytes(int op, int B, int Hq, int Hkv, int head_dim, int max_len);
+
+/*
+ * Zero the workspace's status block (enqueued on `stream`). Call once after allocating a
+ * workspace and again after a reported device error. The rest of the workspace needs no
+ * initialisation.
+ */
+l4l_status l4l_workspace_init(void *workspace, size_t ws_bytes, l4l_stream stream);
+
+/*
+ * Cache update: for every sequence b, copy n_new[b] tokens of k_new / v_new ([B, T, Hkv, D],
+ * T = n_new_max) into cache slots write_pos[b] .. write_pos[b] + n_new[b] - 1, bit for bit.
+ * (In the paper the cache update is the module code around the two kernels; it must happen
+ * exactly once per token.) Every other cache slot is left untouched. Writes that would fall
+ * outside [0, max_len) are dropped on the device, never performed.
+ *   d_write_pos  device int32 [B]
+ *   d_n_new      device int32 [B], or NULL meaning n_new[b] = n_new_max for all b
+ */
+l4l_status l4l_kv_append(l4l_kv_cache cache, l4l_tensor4 k_new, l4l_tensor4 v_new,
+                         const int32_t *d_write_pos, const int32_t *d_n_new, int n_new_max,
+                         int B, int Hkv, int head_dim, l4l_stream stream);
+
+/*
+ * Causal prefill. For every sequence b with L = seq_lens[b] tokens, query head h, row i < L:
+ *     o[b, i, h, :] = softmax_j( scale * q[b, i, h, :] . k[b, j, h/G, :],  j = 0..i ) @ v[b, 0..i, h/G, :]
+ * and, when cache.k != NULL, cache slots 0..L-1 of sequence b receive k and v bit for bit
+ * (the prompt starts an empty cache; prefill over an already populated cache is not
+ * supported). Rows i >= L of o / lse and cache slots >= L are left untouched; q/k/v rows
+ * >= L may hold anything.
+ *   q, o         [B, S_max, Hq, D] views       k, v   [B, S_max, Hkv, D] views
+ *   d_seq_lens   device int32 [B], each 0 <= L <= S_max (and <= cache.max_len when caching)
+ *   S_max        host upper bound of the lengths = extent of the token dimension
+ *   d_lse        device float [B, Hq, S_max] receiving max + ln(sum) of the scaled scores, or NULL
+ *   workspace    >= l4l_workspace_bytes(L4L_OP_PREFILL, ...) bytes, initialised once
+ */
+l4l_status l4l_attn_prefill(l4l_tensor4 q, l4l_tensor4 k, l4l_tensor4 v, l4l_tensor4 o,
+                            l4l_kv_cache cache, const int32_t *d_seq_lens, int S_max,
+                            int B, int Hq, int Hkv, int head_dim, float scale,
+                            float *d_lse, void *workspace, size_t ws_bytes, l4l_stream stream);
+
+/*
+ * Decode. For every sequence b with n = kv_lens[b] cached tokens (the current token has
+ * already been appended and is included), query head h:
+ *     o[b, h, :] = softmax_j( scale * q[b, h, :] . K[b, h/G, j, :],  j = 0..n-1 ) @ V[b, h/G, 0..n-1, :]
+ * with no mask. n = 0 gives o = 0 and lse = -inf. Cache slots >= n are never allowed to
+ * influence the result, whatever bits they hold.
+ *   q, o         dense [B, Hq, D]
+ *   d_kv_lens    device int32 [B], each 0 <= n <= max_kv_len
+ *   max_kv_len   host upper bound of kv_lens (<= cache.max_len); used to size the split
+ *   d_lse        device float [B, Hq] or NULL
+ *   workspace    >= l4l_workspace_bytes(L4L_OP_DECODE, ...) bytes; holds the fp32 partial
+ *                results of the KV splits between the two passes
+ */
+l4l_status l4l_attn_decode(const void *q, void *o, l4l_kv_cache cache,
+                           const int32_t *d_kv_lens, int max_kv_len,
+                           int B, int Hq, int Hkv, int head_dim, float scale,
+                           float *d_lse, void *workspace, size_t ws_bytes, l4l_stream stream);
+
+/* Static, human-readable name of a status code. */
+const char *l4l_status_string(l4l_status status);
+
+/*
+ * Synchronises `stream`, reads the workspace's status block and returns 0 if no bounded wait
+ * has run out since the last l4l_workspace_init(), else a non-zero code identifying the wait
+ * (bit 0: decode pipeline, bit 1: prefill pipeline). Returns -1 if the read itself fails.
+ */
+int l4l_last_device_error(void *workspace, l4l_stream stream);
+
+/* Library version, "major.minor". */
+const char *l4l_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* L4L_H */

@@ -1,0 +1,187 @@
+"""Thin ctypes binding of the C-ABI library ``libl4l.so`` (same names as ``include/l4l.h``).
+
+Argument marshalling only: tensors become pointers + strides, the current CUDA stream
+becomes a ``void*``. Every step of the attention path runs inside the library's kernels;
+PyTorch is used for device memory and streams. There is no fallback: if the library is
+missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libl4l.so")
+
+L4L_OK, L4L_ERR_INVALID_ARG, L4L_ERR_UNSUPPORTED, L4L_ERR_WORKSPACE, L4L_ERR_CUDA, L4L_ERR_TIMEOUT = range(6)
+L4L_OP_PREFILL, L4L_OP_DECODE = 0, 1
+
+EXPORTS = (
+    "l4l_version", "l4l_status_string", "l4l_workspace_bytes", "l4l_workspace_init",
+    "l4l_last_device_error", "l4l_kv_append", "l4l_attn_prefill", "l4l_attn_decode",
+)
+
+
+class Tensor4(ctypes.Structure):
+    _fields_ = [("ptr", ctypes.c_void_p), ("stride_b", ctypes.c_int64), ("stride_t", ctypes.c_int64),
+                ("stride_h", ctypes.c_int64)]
+
+
+class KVCache(ctypes.Structure):
+    _fields_ = [("k", ctypes.c_void_p), ("v", ctypes.c_void_p), ("stride_b", ctypes.c_int64),
+                ("stride_h", ctypes.c_int64), ("stride_t", ctypes.c_int64), ("max_len", ctypes.c_int32)]
+
+
+class L4LError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Opens libl4l.so; raises if it has not been built (``python -m paper_2608_21836_b200.build``)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise FileNotFoundError(
+            f"{LIB_PATH} not found: build it with `python -m paper_2608_21836_b200.build`; there is no fallback path")
+    lib = ctypes.CDLL(LIB_PATH)
+    c_int, c_size, vp, i32p = ctypes.c_int, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_void_p
+    lib.l4l_version.restype = ctypes.c_char_p
+    lib.l4l_status_string.restype = ctypes.c_char_p
+    lib.l4l_status_string.argtypes = [c_int]
+    lib.l4l_workspace_bytes.restype = c_size
+    lib.l4l_workspace_bytes.argtypes = [c_int] * 6
+    lib.l4l_workspace_init.restype = c_int
+    lib.l4l_workspace_init.argtypes = [vp, c_size, vp]
+    lib.l4l_last_device_error.restype = c_int
+    lib.l4l_last_device_error.argtypes = [vp, vp]
+    lib.l4l_kv_append.restype = c_int
+    lib.l4l_kv_append.argtypes = [KVCache, Tensor4, Tensor4, i32p, i32p, c_int, c_int, c_int, c_int, vp]
+    lib.l4l_attn_prefill.restype = c_int
+    lib.l4l_attn_prefill.argtypes = [Tensor4, Tensor4, Tensor4, Tensor4, KVCache, i32p, c_int, c_int, c_int, c_int,
+                                     c_int, ctypes.c_float, vp, vp, c_size, vp]
+    lib.l4l_attn_decode.restype = c_int
+    lib.l4l_attn_decode.argtypes = [vp, vp, KVCache, i32p, c_int, c_int, c_int, c_int, c_int, ctypes.c_float, vp,
+                                    vp, c_size, vp]
+    _lib = lib
+    return lib
+
+
+def version() -> str:
+    return load().l4l_version().decode()
+
+
+def status_string(status: int) -> str:
+    return load().l4l_status_string(int(status)).decode()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _check_bf16_cuda(t: torch.Tensor, name: str) -> None:
+    if not (t.is_cuda and t.dtype == torch.bfloat16 and t.stride(-1) == 1):
+        raise TypeError(f"{name} must be a CUDA bfloat16 tensor with a contiguous last dimension")
+
+
+def tensor4(t: torch.Tensor, name: str = "tensor") -> Tensor4:
+    """[B, T, H, D] view -> l4l_tensor4."""
+    _check_bf16_cuda(t, name)
+    if t.dim() != 4:
+        raise ValueError(f"{name} must have 4 dimensions [B, T, H, D]")
+    return Tensor4(t.data_ptr(), t.stride(0), t.stride(1), t.stride(2))
+
+
+def kv_cache(cache_k: Optional[torch.Tensor], cache_v: Optional[torch.Tensor]) -> KVCache:
+    """Caches indexed [B, Hkv, slot, D] (any strides with D contiguous) -> l4l_kv_cache; (None, None) -> no cache."""
+    if cache_k is None and cache_v is None:
+        return KVCache(None, None, 0, 0, 0, 0)
+    _check_bf16_cuda(cache_k, "cache_k")
+    _check_bf16_cuda(cache_v, "cache_v")
+    if cache_k.dim() != 4 or cache_k.shape != cache_v.shape or cache_k.stride() != cache_v.stride():
+        raise ValueError("cache_k and cache_v must be [B, Hkv, max_len, D] views with equal shapes and strides")
+    return KVCache(cache_k.data_ptr(), cache_v.data_ptr(), cache_k.stride(0), cache_k.stride(1), cache_k.stride(2),
+                   cache_k.shape[2])
+
+
+def _i32_dev(t: Optional[torch.Tensor], name: str) -> Optional[int]:
+    if t is None:
+        return None
+    if not (t.is_cuda and t.dtype == torch.int32 and t.is_contiguous()):
+        raise TypeError(f"{name} must be a contiguous CUDA int32 tensor")
+    return t.data_ptr()
+
+
+def l4l_workspace_bytes(op: int, B: int, Hq: int, Hkv: int, head_dim: int, max_len: int) -> int:
+    return int(load().l4l_workspace_bytes(op, B, Hq, Hkv, head_dim, max_len))
+
+
+def l4l_workspace_init(workspace: torch.Tensor) -> None:
+    st = load().l4l_workspace_init(workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream())
+    if st != L4L_OK:
+        raise L4LError(st, "l4l_workspace_init")
+
+
+def new_workspace(op: int, B: int, Hq: int, Hkv: int, head_dim: int, max_len: int, device="cuda") -> torch.Tensor:
+    """Allocates (with torch) and initialises a workspace of the size the library asks for."""
+    n = l4l_workspace_bytes(op, B, Hq, Hkv, head_dim, max_len)
+    if n == 0:
+        raise L4LError(L4L_ERR_UNSUPPORTED, "l4l_workspace_bytes")
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    l4l_workspace_init(ws)
+    return ws
+
+
+def l4l_last_device_error(workspace: torch.Tensor) -> int:
+    return int(load().l4l_last_device_error(workspace.data_ptr(), _stream()))
+
+
+def l4l_kv_append(cache_k, cache_v, k_new, v_new, write_pos, n_new=None) -> None:
+    """cache [B,Hkv,max_len,D]; k_new/v_new [B,T,Hkv,D]; write_pos, n_new: CUDA int32 [B]."""
+    B, T, Hkv, D = k_new.shape
+    st = load().l4l_kv_append(kv_cache(cache_k, cache_v), tensor4(k_new, "k_new"), tensor4(v_new, "v_new"),
+                              _i32_dev(write_pos, "write_pos"), _i32_dev(n_new, "n_new"), T, B, Hkv, D, _stream())
+    if st != L4L_OK:
+        raise L4LError(st, "l4l_kv_append")
+
+
+def l4l_attn_prefill(q, k, v, o, seq_lens, scale: float, workspace, cache_k=None, cache_v=None, lse=None) -> None:
+    """q,o [B,S,Hq,D]; k,v [B,S,Hkv,D]; seq_lens CUDA int32 [B]; lse optional CUDA float32 [B,Hq,S]."""
+    B, S, Hq, D = q.shape
+    Hkv = k.shape[2]
+    if lse is not None and not (lse.is_cuda and lse.dtype == torch.float32 and lse.is_contiguous()
+                                and tuple(lse.shape) == (B, Hq, S)):
+        raise TypeError("lse must be a contiguous CUDA float32 tensor [B, Hq, S]")
+    st = load().l4l_attn_prefill(tensor4(q, "q"), tensor4(k, "k"), tensor4(v, "v"), tensor4(o, "o"),
+                                 kv_cache(cache_k, cache_v), _i32_dev(seq_lens, "seq_lens"), S, B, Hq, Hkv, D,
+                                 float(scale), None if lse is None else lse.data_ptr(), workspace.data_ptr(),
+                                 workspace.numel() * workspace.element_size(), _stream())
+    if st != L4L_OK:
+        raise L4LError(st, "l4l_attn_prefill")
+
+
+def l4l_attn_decode(q, o, cache_k, cache_v, kv_lens, max_kv_len: int, scale: float, workspace, lse=None) -> None:
+    """q,o dense [B,Hq,D]; cache [B,Hkv,max_len,D]; kv_lens CUDA int32 [B] (current token included)."""
+    _check_bf16_cuda(q, "q")
+    _check_bf16_cuda(o, "o")
+    if not (q.is_contiguous() and o.is_contiguous() and q.dim() == 3 and q.shape == o.shape):
+        raise ValueError("q and o must be dense [B, Hq, D]")
+    B, Hq, D = q.shape
+    Hkv = cache_k.shape[1]
+    if lse is not None and not (lse.is_cuda and lse.dtype == torch.float32 and lse.is_contiguous()
+                                and tuple(lse.shape) == (B, Hq)):
+        raise TypeError("lse must be a contiguous CUDA float32 tensor [B, Hq]")
+    st = load().l4l_attn_decode(q.data_ptr(), o.data_ptr(), kv_cache(cache_k, cache_v),
+                                _i32_dev(kv_lens, "kv_lens"), int(max_kv_len), B, Hq, Hkv, D, float(scale),
+                                None if lse is None else lse.data_ptr(), workspace.data_ptr(),
+                                workspace.numel() * workspace.element_size(), _stream())
+    if st != L4L_OK:
+        raise L4LError(st, "l4l_attn_decode")

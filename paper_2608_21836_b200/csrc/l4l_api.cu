@@ -1,0 +1,192 @@
+// C-ABI entry points: host-side validation, workspace sizing, tensor-map construction.
+// Nothing here touches the data path; every operation runs in the kernels of the other
+// translation units.
+#include <mutex>
+
+#include "l4l_internal.h"
+#include "l4l_ptx.cuh"
+
+namespace l4l {
+
+namespace {
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    });
+    return fn;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool stride_ok(int64_t s) { return s >= 0 && (s % 8) == 0; }
+
+bool tensor4_ok(const l4l_tensor4 &t)
+{
+    return t.ptr && aligned16(t.ptr) && stride_ok(t.stride_b) && stride_ok(t.stride_t) && stride_ok(t.stride_h);
+}
+
+bool cache_ok(const l4l_kv_cache &c)
+{
+    return c.k && c.v && aligned16(c.k) && aligned16(c.v) && stride_ok(c.stride_b) && stride_ok(c.stride_h) &&
+           stride_ok(c.stride_t) && c.max_len > 0;
+}
+
+l4l_status shape_status(int B, int Hq, int Hkv, int D)
+{
+    if (B < 0 || Hq <= 0 || Hkv <= 0) return L4L_ERR_INVALID_ARG;
+    if (D != 64 && D != 128) return L4L_ERR_UNSUPPORTED;
+    if (Hq % Hkv != 0 || Hq / Hkv > 16) return L4L_ERR_UNSUPPORTED;
+    return L4L_OK;
+}
+
+}  // namespace
+
+int sm_count()
+{
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+            n = 148;
+    }
+    return n;
+}
+
+bool make_tmap_bf16(CUtensorMap *out, TmapCoord *coord, const void *base, int D, int64_t n_t, int64_t n_h,
+                    int64_t n_b, int64_t stride_t, int64_t stride_h, int64_t stride_b, int box_d, int box_t)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    // order the three outer dimensions by ascending stride (extent-1 dimensions last)
+    struct Dim { int64_t n, stride; int which; int box; };
+    Dim dims[3] = {{n_t, stride_t, 0, box_t}, {n_h, stride_h, 1, 1}, {n_b, stride_b, 2, 1}};
+    auto key = [](const Dim &d) { return d.n <= 1 ? INT64_MAX : d.stride; };
+    for (int i = 0; i < 3; ++i)
+        for (int j = i + 1; j < 3; ++j)
+            if (key(dims[j]) < key(dims[i])) { Dim t = dims[i]; dims[i] = dims[j]; dims[j] = t; }
+    cuuint64_t gdim[4] = {(cuuint64_t)D, 0, 0, 0};
+    cuuint64_t gstride[3];
+    cuuint32_t box[4] = {(cuuint32_t)box_d, 1, 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    int64_t prev_extent_bytes = (int64_t)D * 2;
+    for (int i = 0; i < 3; ++i) {
+        gdim[i + 1] = (cuuint64_t)(dims[i].n < 1 ? 1 : dims[i].n);
+        int64_t sb = dims[i].stride * 2;
+        if (dims[i].n <= 1 && sb < prev_extent_bytes) sb = prev_extent_bytes;   // never used for addressing
+        gstride[i] = (cuuint64_t)sb;
+        prev_extent_bytes = sb * (int64_t)gdim[i + 1];
+        box[i + 1] = (cuuint32_t)dims[i].box;
+        if (dims[i].which == 0) coord->pos_t = i + 1;
+        if (dims[i].which == 1) coord->pos_h = i + 1;
+        if (dims[i].which == 2) coord->pos_b = i + 1;
+    }
+    CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), gdim, gstride, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+}  // namespace l4l
+
+using namespace l4l;
+
+extern "C" {
+
+const char *l4l_version(void) { return "0.1"; }
+
+const char *l4l_status_string(l4l_status s)
+{
+    switch (s) {
+        case L4L_OK: return "ok";
+        case L4L_ERR_INVALID_ARG: return "invalid argument";
+        case L4L_ERR_UNSUPPORTED: return "unsupported shape";
+        case L4L_ERR_WORKSPACE: return "workspace missing or too small";
+        case L4L_ERR_CUDA: return "CUDA call failed";
+        case L4L_ERR_TIMEOUT: return "bounded device-side wait ran out";
+    }
+    return "unknown status";
+}
+
+size_t l4l_workspace_bytes(int op, int B, int Hq, int Hkv, int head_dim, int max_len)
+{
+    if (shape_status(B, Hq, Hkv, head_dim) != L4L_OK || max_len < 0) return 0;
+    if (op == L4L_OP_PREFILL) return kStatusBytes;
+    if (op == L4L_OP_DECODE) return plan_decode(B, Hq, Hkv, head_dim, max_len, (size_t)-1).ws_bytes;
+    return 0;
+}
+
+l4l_status l4l_workspace_init(void *workspace, size_t ws_bytes, l4l_stream stream)
+{
+    if (!workspace || ws_bytes < kStatusBytes) return L4L_ERR_WORKSPACE;
+    return cudaMemsetAsync(workspace, 0, kStatusBytes, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? L4L_OK
+               : L4L_ERR_CUDA;
+}
+
+int l4l_last_device_error(void *workspace, l4l_stream stream)
+{
+    if (!workspace) return -1;
+    unsigned words[2] = {0, 0};
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(words, workspace, sizeof(words), cudaMemcpyDeviceToHost, s) != cudaSuccess) return -1;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return -1;
+    return (int)words[kStatusErrWord];
+}
+
+l4l_status l4l_kv_append(l4l_kv_cache cache, l4l_tensor4 k_new, l4l_tensor4 v_new, const int32_t *d_write_pos,
+                         const int32_t *d_n_new, int n_new_max, int B, int Hkv, int head_dim, l4l_stream stream)
+{
+    if (B < 0 || Hkv <= 0 || n_new_max < 0) return L4L_ERR_INVALID_ARG;
+    if (head_dim != 64 && head_dim != 128) return L4L_ERR_UNSUPPORTED;
+    if (!cache_ok(cache) || !tensor4_ok(k_new) || !tensor4_ok(v_new) || !d_write_pos) return L4L_ERR_INVALID_ARG;
+    if (B == 0 || n_new_max == 0) return L4L_OK;
+    return launch_kv_append(cache, k_new, v_new, d_write_pos, d_n_new, n_new_max, B, Hkv, head_dim,
+                            static_cast<cudaStream_t>(stream));
+}
+
+l4l_status l4l_attn_prefill(l4l_tensor4 q, l4l_tensor4 k, l4l_tensor4 v, l4l_tensor4 o, l4l_kv_cache cache,
+                            const int32_t *d_seq_lens, int S_max, int B, int Hq, int Hkv, int head_dim, float scale,
+                            float *d_lse, void *workspace, size_t ws_bytes, l4l_stream stream)
+{
+    l4l_status st = shape_status(B, Hq, Hkv, head_dim);
+    if (st != L4L_OK) return st;
+    if (S_max < 0 || !d_seq_lens) return L4L_ERR_INVALID_ARG;
+    if (!tensor4_ok(q) || !tensor4_ok(k) || !tensor4_ok(v) || !tensor4_ok(o)) return L4L_ERR_INVALID_ARG;
+    if (cache.k || cache.v) {
+        if (!cache_ok(cache)) return L4L_ERR_INVALID_ARG;
+    }
+    if (!workspace || ws_bytes < kStatusBytes) return L4L_ERR_WORKSPACE;
+    if (B == 0 || S_max == 0) return L4L_OK;
+    return launch_prefill(q, k, v, o, cache, d_seq_lens, S_max, B, Hq, Hkv, head_dim, scale, d_lse, workspace,
+                          static_cast<cudaStream_t>(stream));
+}
+
+l4l_status l4l_attn_decode(const void *q, void *o, l4l_kv_cache cache, const int32_t *d_kv_lens, int max_kv_len,
+                           int B, int Hq, int Hkv, int head_dim, float scale, float *d_lse, void *workspace,
+                           size_t ws_bytes, l4l_stream stream)
+{
+    l4l_status st = shape_status(B, Hq, Hkv, head_dim);
+    if (st != L4L_OK) return st;
+    if (!q || !o || !d_kv_lens || !aligned16(q) || !aligned16(o)) return L4L_ERR_INVALID_ARG;
+    if (!cache_ok(cache) || max_kv_len < 0 || max_kv_len > cache.max_len) return L4L_ERR_INVALID_ARG;
+    if (!workspace || ws_bytes < kStatusBytes) return L4L_ERR_WORKSPACE;
+    if (B == 0) return L4L_OK;
+    const DecodePlan plan = plan_decode(B, Hq, Hkv, head_dim, max_kv_len, ws_bytes);
+    if (plan.ws_bytes > ws_bytes) return L4L_ERR_WORKSPACE;
+    return launch_decode(q, o, cache, d_kv_lens, max_kv_len, B, Hq, Hkv, head_dim, scale, d_lse, workspace, plan,
+                         static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

@@ -1,0 +1,47 @@
+// Host-side declarations shared by the translation units of libl4l (not part of the ABI).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/l4l.h"
+
+namespace l4l {
+
+// Where each logical coordinate (token, head, batch) sits among coordinates 1..3 of a 4-D
+// tensor map whose coordinate 0 is head_dim. Dimensions are ordered by ascending stride.
+struct TmapCoord {
+    int pos_t, pos_h, pos_b;
+};
+
+// Builds a tiled bf16 tensor map over a [batch, head, token, D]-indexable buffer with the
+// given element strides; the box is box_d x box_t (x1x1) with the 128-byte swizzle
+// (box_d must be 64). Returns false (and leaves *out undefined) if the driver refuses.
+bool make_tmap_bf16(CUtensorMap *out, TmapCoord *coord, const void *base, int D, int64_t n_t, int64_t n_h,
+                    int64_t n_b, int64_t stride_t, int64_t stride_h, int64_t stride_b, int box_d, int box_t);
+
+int sm_count();
+
+struct DecodePlan {
+    int chunk;       // tokens per KV split (multiple of 64)
+    int nsplit;      // max splits per sequence = ceil(max_kv_len / chunk)
+    size_t ws_bytes; // status block + partials
+};
+DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_limit);
+
+l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, const int32_t *d_kv_lens,
+                         int max_kv_len, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
+                         void *workspace, const DecodePlan &plan, cudaStream_t stream);
+
+l4l_status launch_kv_append(const l4l_kv_cache &cache, const l4l_tensor4 &k_new, const l4l_tensor4 &v_new,
+                            const int32_t *d_write_pos, const int32_t *d_n_new, int n_new_max, int B, int Hkv,
+                            int D, cudaStream_t stream);
+
+l4l_status launch_prefill(const l4l_tensor4 &q, const l4l_tensor4 &k, const l4l_tensor4 &v,
+                          const l4l_tensor4 &o, const l4l_kv_cache &cache, const int32_t *d_seq_lens,
+                          int S_max, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
+                          void *workspace, cudaStream_t stream);
+
+}  // namespace l4l

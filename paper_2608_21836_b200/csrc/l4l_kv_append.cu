@@ -1,0 +1,67 @@
+// KV-cache append: an exact copy of the new tokens' K and V rows into their cache slots.
+// One thread moves one 16-byte piece of a K row and the matching piece of the V row, so a
+// warp reads and writes whole contiguous rows (coalesced both ways).
+#include "l4l_internal.h"
+#include "l4l_ptx.cuh"
+
+namespace l4l {
+
+namespace {
+
+struct AppendParams {
+    const uint4 *k_new, *v_new;     // strides below are in 16-byte units
+    uint4 *cache_k, *cache_v;
+    int64_t new_sb, new_st, new_sh, vnew_sb, vnew_st, vnew_sh;
+    int64_t c_sb, c_sh, c_st;
+    const int32_t *write_pos, *n_new;
+    int B, T, Hkv, pieces, max_len;
+};
+
+__global__ void __launch_bounds__(256) kv_append_kernel(const AppendParams p)
+{
+    const long long total = (long long)p.B * p.T * p.Hkv * p.pieces;
+    for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const int piece = (int)(idx % p.pieces);
+        long long rest = idx / p.pieces;
+        const int g = (int)(rest % p.Hkv);
+        rest /= p.Hkv;
+        const int r = (int)(rest % p.T);
+        const int b = (int)(rest / p.T);
+        const int n = p.n_new ? p.n_new[b] : p.T;
+        if (r >= n) continue;
+        const long long slot = (long long)p.write_pos[b] + r;
+        if (slot < 0 || slot >= p.max_len) continue;          // dropped, never written out of range
+        const uint4 kk = p.k_new[b * p.new_sb + r * p.new_st + g * p.new_sh + piece];
+        const uint4 vv = p.v_new[b * p.vnew_sb + r * p.vnew_st + g * p.vnew_sh + piece];
+        const int64_t dst = b * p.c_sb + g * p.c_sh + slot * p.c_st + piece;
+        p.cache_k[dst] = kk;
+        p.cache_v[dst] = vv;
+    }
+}
+
+}  // namespace
+
+l4l_status launch_kv_append(const l4l_kv_cache &cache, const l4l_tensor4 &k_new, const l4l_tensor4 &v_new,
+                            const int32_t *d_write_pos, const int32_t *d_n_new, int n_new_max, int B, int Hkv,
+                            int D, cudaStream_t stream)
+{
+    AppendParams p;
+    p.k_new = static_cast<const uint4 *>(k_new.ptr);
+    p.v_new = static_cast<const uint4 *>(v_new.ptr);
+    p.cache_k = static_cast<uint4 *>(cache.k);
+    p.cache_v = static_cast<uint4 *>(cache.v);
+    p.new_sb = k_new.stride_b / 8; p.new_st = k_new.stride_t / 8; p.new_sh = k_new.stride_h / 8;
+    p.vnew_sb = v_new.stride_b / 8; p.vnew_st = v_new.stride_t / 8; p.vnew_sh = v_new.stride_h / 8;
+    p.c_sb = cache.stride_b / 8; p.c_sh = cache.stride_h / 8; p.c_st = cache.stride_t / 8;
+    p.write_pos = d_write_pos; p.n_new = d_n_new;
+    p.B = B; p.T = n_new_max; p.Hkv = Hkv; p.pieces = D / 8; p.max_len = cache.max_len;
+    const long long total = (long long)B * n_new_max * Hkv * p.pieces;
+    long long blocks = (total + 255) / 256;
+    const long long cap = 8ll * sm_count();
+    if (blocks > cap) blocks = cap;
+    kv_append_kernel<<<(int)blocks, 256, 0, stream>>>(p);
+    return cudaGetLastError() == cudaSuccess ? L4L_OK : L4L_ERR_CUDA;
+}
+
+}  // namespace l4l
