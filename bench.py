@@ -1,0 +1,367 @@
+#!/usr/bin/env python
+"""Benchmark of the attention hot path on B200: prefill TFLOP/s and decode HBM GB/s vs roofline.
+
+One "step" is one pass of the whole hot path at the 8B-shaped sizes (Hq=32, Hkv=8, D=128):
+  1. l4l_attn_prefill   causal prefill B=4, S=8192 with the KV cache written in the same pass
+  2. l4l_kv_append      the current token's K/V of B=32 ragged sequences (512..4096 cached tokens)
+  3. l4l_attn_decode    one query token per sequence over that ragged cache (split + merge)
+`value` is the step's attention FLOPs (causal pairs only for prefill) divided by the step's time,
+summed over GPUs; the per-kernel roofline fractions (tensor peak for prefill, HBM for decode) are
+in `roofline` / `roofline_decode`. Inputs are seeded synthetic bf16 (see workloads.py).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+Under torchrun every rank runs the same step on its own GPU (sequences shard with no exchange).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2608_21836_b200 import workloads as wl  # noqa: E402
+
+METRIC = "decode-attn HBM GB/s & prefill-attn TFLOP/s, each as % of B200 peak"
+NOMINAL_TFLOPS, NOMINAL_GBS = 2250.0, 8000.0
+FALLBACK_TFLOPS, FALLBACK_GBS = 1590.0, 6650.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            mp = json.load(f)
+        return {"hbm_gbs": float(mp["hbm_gbs"]), "bf16_tflops": float(mp["bf16_tflops"]),
+                "bf16_tflops_sustained": float(mp.get("bf16_tflops_sustained", mp["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": FALLBACK_GBS, "bf16_tflops": FALLBACK_TFLOPS, "bf16_tflops_sustained": 1400.0,
+            "source": "fallback"}
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4),
+        }
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        if self.is_alive():
+            self.join(timeout=2)
+        med = int(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# ----------------------------------------------------------------------------------- workload
+def make_inputs():
+    wp, wd = wl.WORKLOADS["long_prefill"], wl.WORKLOADS["batched_decode"]
+    seq = wl.make_sequence(wp)
+    db = wl.make_decode_batch(wd)
+    g = torch.Generator().manual_seed(wd.seed + 7)
+    k_new = torch.randn(wd.decode_B, 1, wd.Hkv, wd.D, generator=g).to(torch.bfloat16)
+    v_new = torch.randn(wd.decode_B, 1, wd.Hkv, wd.D, generator=g).to(torch.bfloat16)
+    return wp, wd, seq, db, k_new, v_new
+
+
+def step_work(wp, wd, seq, db):
+    pre_flops = wl.prefill_flops(wp.Hq, wp.D, [seq.S] * wp.prefill_B)
+    dec_bytes = wl.decode_kv_bytes(wd.Hkv, wd.D, db.kv_len.tolist())
+    dec_flops = 4 * wd.D * wd.Hq * int(db.kv_len.sum())
+    return pre_flops, dec_bytes, dec_flops
+
+
+def workload_name(wp, wd):
+    return (f"8b_shaped: long_prefill(B={wp.prefill_B},S={wp.prefill_S},Hq={wp.Hq},Hkv={wp.Hkv},D={wp.D},cache write) + "
+            f"batched_decode(B={wd.decode_B},kv_len~U[{wd.decode_len_lo},{wd.decode_len_hi}],append+decode)")
+
+
+# ----------------------------------------------------------------------------------- oracle timing
+def time_oracle_sample(wp, wd, seq, db, budget_s: float = 12.0):
+    """Times the CPU oracle, as it stands, on a bounded sample of the step: a stratified set of prefill
+    rows (grown until about budget_s of work) and the whole decode batch. Returns work and seconds."""
+    from oracle import l4l_oracle as orc
+
+    B, S, Hq, D = wp.prefill_B, seq.S, wp.Hq, wp.D
+    lens = np.full(B, S, np.int32)
+    rng = np.random.default_rng(2024)
+
+    def rows(n):
+        return np.stack([rng.integers(0, B, n), rng.integers(0, S, n), rng.integers(0, Hq, n)], axis=1).astype(np.int32)
+
+    probe = rows(512)
+    t0 = time.perf_counter()
+    orc.prefill_rows(seq.q, seq.k, seq.v, lens, wp.scale, probe)
+    t_probe = time.perf_counter() - t0
+    n = int(min(200000, max(512, 512 * (0.7 * budget_s) / max(t_probe, 1e-3))))
+    sample = rows(n)
+    t0 = time.perf_counter()
+    orc.prefill_rows(seq.q, seq.k, seq.v, lens, wp.scale, sample)
+    t_pre = time.perf_counter() - t0
+    pre_flops = int(4 * D * (sample[:, 1].astype(np.int64) + 1).sum())
+    t0 = time.perf_counter()
+    orc.decode(db.q, db.cache_k, db.cache_v, db.kv_len.numpy(), wd.scale)
+    t_dec = time.perf_counter() - t0
+    dec_bytes = wl.decode_kv_bytes(wd.Hkv, wd.D, db.kv_len.tolist())
+    dec_flops = 4 * wd.D * wd.Hq * int(db.kv_len.sum())
+    return {"pre_flops": pre_flops, "t_pre": t_pre, "rows": n, "dec_bytes": dec_bytes, "dec_flops": dec_flops,
+            "t_dec": t_dec, "cores": orc.num_threads()}
+
+
+def cpu_baseline_obj(s):
+    total_t = s["t_pre"] + s["t_dec"]
+    return {
+        "value": (s["pre_flops"] + s["dec_flops"]) / total_t / 1e12, "unit": "TFLOP/s", "cores": s["cores"],
+        "kind": "oracle",
+        "sample": (f"{s['rows']} random (b,i,h) rows of the B=4,S=8192 causal prefill ({s['t_pre']:.1f} s) + the whole "
+                   f"B=32 ragged decode batch ({s['t_dec']:.1f} s), fp64 C oracle with OpenMP"),
+        "prefill_gflops": s["pre_flops"] / s["t_pre"] / 1e9,
+        "decode_gbs": s["dec_bytes"] / s["t_dec"] / 1e9,
+    }
+
+
+def run_reference(args, rank):
+    """--impl reference: the oracle, as it stands, on the host cores; each step is a bounded sample."""
+    if rank != 0:
+        return
+    wp, wd, seq, db, _, _ = make_inputs()
+    per_step_budget = max(2.0, min(20.0, 150.0 / max(1, args.steps + args.warmup)))
+    for _ in range(args.warmup):
+        time_oracle_sample(wp, wd, seq, db, budget_s=min(2.0, per_step_budget))
+    tot_fl, tot_t, last = 0.0, 0.0, None
+    for _ in range(args.steps):
+        last = time_oracle_sample(wp, wd, seq, db, budget_s=per_step_budget)
+        tot_fl += last["pre_flops"] + last["dec_flops"]
+        tot_t += last["t_pre"] + last["t_dec"]
+    value = tot_fl / tot_t / 1e12
+    cb = cpu_baseline_obj(last)
+    cb["value"] = value
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": tot_t / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload_name(wp, wd), "note": "each step is a bounded sample of the workload"},
+        "cpu_baseline": cb,
+        "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+# ----------------------------------------------------------------------------------- our arm
+def run_ours(args, rank, world):
+    import torch.distributed as dist
+    from paper_2608_21836_b200 import binding as l4l
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the attention path has no CPU fallback")
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    l4l.load()
+
+    wp, wd, seq, db, k_new, v_new = make_inputs()
+    pre_flops, dec_bytes, dec_flops = step_work(wp, wd, seq, db)
+    Bp, S, Hq, Hkv, D = wp.prefill_B, seq.S, wp.Hq, wp.Hkv, wp.D
+    Bd, Lmax = wd.decode_B, wd.decode_Lmax
+
+    # device-resident inputs
+    q, k, v = seq.q.to(dev), seq.k.to(dev), seq.v.to(dev)
+    o = torch.empty_like(q)
+    pk = torch.empty(Bp, Hkv, S, D, dtype=torch.bfloat16, device=dev)
+    pv = torch.empty_like(pk)
+    plens = torch.full((Bp,), S, dtype=torch.int32, device=dev)
+    ws_p = l4l.new_workspace(l4l.L4L_OP_PREFILL, Bp, Hq, Hkv, D, S, device=dev)
+    dq, dck, dcv = db.q.to(dev), db.cache_k.to(dev), db.cache_v.to(dev)
+    dlen = db.kv_len.to(dev)
+    dpos = (db.kv_len - 1).to(torch.int32).to(dev)
+    dkn, dvn = k_new.to(dev), v_new.to(dev)
+    do = torch.empty_like(dq)
+    ws_d = l4l.new_workspace(l4l.L4L_OP_DECODE, Bd, Hq, Hkv, D, Lmax, device=dev)
+
+    def step(ev=None):
+        if ev: ev[0].record()
+        l4l.l4l_attn_prefill(q, k, v, o, plens, wp.scale, ws_p, cache_k=pk, cache_v=pv)
+        if ev: ev[1].record()
+        l4l.l4l_kv_append(dck, dcv, dkn, dvn, dpos)
+        if ev: ev[2].record()
+        l4l.l4l_attn_decode(dq, do, dck, dcv, dlen, Lmax, wd.scale, ws_d)
+        if ev: ev[3].record()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_begin.record()
+    for i in range(args.steps):
+        step(evs[i])
+    t_end.record()
+    barrier()
+    clocks = sampler.stop()
+    total_ms = t_begin.elapsed_time(t_end)
+    t_pre = float(np.mean([e[0].elapsed_time(e[1]) for e in evs]))
+    t_app = float(np.mean([e[1].elapsed_time(e[2]) for e in evs]))
+    t_dec = float(np.mean([e[2].elapsed_time(e[3]) for e in evs]))
+    dev_err = l4l.l4l_last_device_error(ws_p) | l4l.l4l_last_device_error(ws_d)
+
+    # ---- end to end through the same entry points with HOST buffers (pinned), copies inside the timed region
+    hq, hk, hv = seq.q.pin_memory(), seq.k.pin_memory(), seq.v.pin_memory()
+    ho = torch.empty_like(hq).pin_memory()
+    hdq, hkn, hvn = db.q.pin_memory(), k_new.pin_memory(), v_new.pin_memory()
+    hdo = torch.empty_like(hdq).pin_memory()
+    h2d = sum(t.numel() * 2 for t in (hq, hk, hv, hdq, hkn, hvn))
+    d2h = sum(t.numel() * 2 for t in (ho, hdo))
+
+    def e2e_step():
+        q.copy_(hq, non_blocking=True); k.copy_(hk, non_blocking=True); v.copy_(hv, non_blocking=True)
+        l4l.l4l_attn_prefill(q, k, v, o, plens, wp.scale, ws_p, cache_k=pk, cache_v=pv)
+        ho.copy_(o, non_blocking=True)
+        dq.copy_(hdq, non_blocking=True); dkn.copy_(hkn, non_blocking=True); dvn.copy_(hvn, non_blocking=True)
+        l4l.l4l_kv_append(dck, dcv, dkn, dvn, dpos)
+        l4l.l4l_attn_decode(dq, do, dck, dcv, dlen, Lmax, wd.scale, ws_d)
+        hdo.copy_(do, non_blocking=True)
+
+    e2e_steps = max(3, min(args.steps, 20))
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+
+    # ---- max over ranks
+    times = torch.tensor([total_ms, e2e_ms, t_pre, t_dec, t_app], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms, t_pre, t_dec, t_app = times.tolist()
+    if rank != 0:
+        return
+
+    ms_per_step = total_ms / args.steps
+    step_flops = pre_flops + dec_flops
+    value = world * step_flops / (ms_per_step * 1e-3) / 1e12
+    peaks = measured_peaks()
+    pre_tflops = pre_flops / (t_pre * 1e-3) / 1e12
+    dec_gbs = dec_bytes / (t_dec * 1e-3) / 1e9
+    # prefill is timed inside a long back-to-back loop: sustained tensor peak is its denominator
+    tensor_peak = peaks["bf16_tflops_sustained"]
+    line = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {
+            "workload": workload_name(wp, wd),
+            "value_definition": "attention FLOPs of one step (4*D per causal query-key pair per query head for prefill, "
+                                "4*D per cached token per query head for decode) / step time, summed over GPUs",
+            "l2": "inputs larger than L2: prefill streams 805 MB and decode 294 MB per step, each evicting the other",
+            "parallelism": "replicas (sequences shard with no exchange)" if world > 1 else "single GPU",
+        },
+        "prefill": {"tflops": pre_tflops, "ms": t_pre, "pct_nominal_2250": 100 * pre_tflops / NOMINAL_TFLOPS,
+                    "pct_measured_burst": 100 * pre_tflops / peaks["bf16_tflops"],
+                    "pct_measured_sustained": 100 * pre_tflops / peaks["bf16_tflops_sustained"]},
+        "decode": {"kv_gbs": dec_gbs, "us": t_dec * 1e3, "pct_nominal_8000": 100 * dec_gbs / NOMINAL_GBS,
+                   "pct_measured": 100 * dec_gbs / peaks["hbm_gbs"], "append_us": t_app * 1e3},
+        "roofline": {"kernel": "prefill", "bound": "tensor", "achieved": pre_tflops, "peak": tensor_peak,
+                     "unit": "TFLOP/s", "frac": pre_tflops / tensor_peak, "traffic": None,
+                     "peak_source": peaks["source"] + " (sustained bf16 GEMM)"},
+        "roofline_decode": {"kernel": "decode_split", "bound": "hbm", "achieved": dec_gbs, "peak": peaks["hbm_gbs"],
+                            "unit": "GB/s", "frac": dec_gbs / peaks["hbm_gbs"], "traffic": None,
+                            "peak_source": peaks["source"] + " (device copy)"},
+        "e2e": {"value": world * step_flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+        "gpu_launches": 4 * args.steps,
+        "clocks": clocks,
+        "device_error": dev_err,
+    }
+    prof = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(prof):
+        with open(prof) as f:
+            tr = json.load(f)
+        line["roofline"]["traffic"] = tr.get("prefill")
+        line["roofline_decode"]["traffic"] = tr.get("decode")
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline_obj(time_oracle_sample(wp, wd, seq, db))
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", int(os.environ.get("LOCAL_RANK", 0))))
+    try:
+        run_ours(args, rank, world)
+    finally:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
