@@ -1,0 +1,446 @@
+// Causal prefill on the 5th-generation tensor cores (tcgen05.mma, accumulators in tensor memory).
+//
+// One CTA owns 256 consecutive query rows of one (sequence, query head): two 128-row sub-tiles
+// whose S = Q K^T and O += P V products ping-pong on the tensor pipe while the other sub-tile's
+// softmax runs on the CUDA cores.
+//
+//   warps 0-3   softmax of sub-tile 0: thread t owns row t (= TMEM lane t): reads S from TMEM,
+//               keeps the running max / sum in fp32, writes P (bf16) back into TMEM over S
+//   warps 4-7   the same for sub-tile 1
+//   warp  8     TMA producer: Q once, then K_j, V_j tiles (128 tokens, 128-byte swizzle) through a
+//               ring of shared-memory slots; afterwards copies the block's diagonal K/V tiles from
+//               shared memory into the KV cache (only for the first query head of a KV group)
+//   warp  9     MMA issuer (one lane): S_i = Q_i K_j^T from shared memory, O_i += P_i V_j with P read
+//               from TMEM and V as an MN-major shared-memory operand; owns the TMEM allocation
+//
+// TMEM columns: S0 [0,128) S1 [128,256) O0 [256,256+D) O1 [256+D,256+2D); P_i aliases the first 64
+// columns of S_i. Causal tile skipping: sub-tile i only visits K/V tiles up to its diagonal.
+// The tensor pipe executes one thread's MMAs in issue order, which is what makes the S/P aliasing
+// safe: QK_{j+1} into S_i is issued after PV_j that reads P_i.
+#include "l4l_internal.h"
+#include "l4l_ptx.cuh"
+
+namespace l4l {
+
+namespace {
+
+constexpr int kRows = 128;                     // rows per sub-tile == tokens per K/V tile
+constexpr int kThreads = 320;
+constexpr uint32_t kHalfBytes = kRows * 128;   // [128 rows][64 bf16], 128-byte swizzled
+constexpr float kRescaleThreshold = 8.f;       // log2 domain: O is rescaled only if the max grew by > 2^8
+
+template <int D>
+struct TcCfg {
+    static constexpr int kHalves = D / 64;
+    static constexpr uint32_t kTileBytes = kHalves * kHalfBytes;        // one Q sub-tile, K tile or V tile
+    static constexpr int kSlots = (D == 128) ? 4 : 8;                    // ring of K/V tiles
+    static constexpr uint32_t kTmemCols = 512;
+    static constexpr uint32_t kColS0 = 0, kColS1 = 128, kColO0 = 256, kColO1 = 256 + D;
+    static constexpr int kNumBars = 1 + 2 * kSlots + 6;
+    static constexpr size_t kSmemBytes = 1024 + 2 * kTileBytes + (size_t)kSlots * kTileBytes + kNumBars * 8 + 64;
+};
+
+struct TcParams {
+    __nv_bfloat16 *o;
+    int64_t o_sb, o_st, o_sh;
+    __nv_bfloat16 *cache_k, *cache_v;
+    int64_t c_sb, c_sh, c_st;
+    int cache_max_len;
+    const int32_t *seq_lens;
+    float *lse;
+    unsigned *status;
+    int S_max, B, Hq, Hkv, G, n_qblocks;
+    float scale_log2e;
+    TmapCoord cq, ckv;
+};
+
+__device__ __forceinline__ void order_coords(const TmapCoord &c, int t, int h, int b, int &c1, int &c2, int &c3)
+{
+    c1 = (c.pos_t == 1) ? t : (c.pos_h == 1) ? h : b;
+    c2 = (c.pos_t == 2) ? t : (c.pos_h == 2) ? h : b;
+    c3 = (c.pos_t == 3) ? t : (c.pos_h == 3) ? h : b;
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle, 8-row groups 1024 bytes apart.
+// K-major operands ignore the leading byte offset; MN-major ones use it as the stride between
+// 64-element chunks along M/N.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr, uint32_t lbo_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((1024u >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;                     // descriptor version for sm_100
+    d |= (uint64_t)2 << 61;                     // SWIZZLE_128B
+    return d;
+}
+
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128.
+__host__ __device__ constexpr uint32_t make_idesc(int n, bool b_mn_major)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) |
+           ((uint32_t)(kRows >> 4) << 24);
+}
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1)
+prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+                  const __grid_constant__ CUtensorMap tmap_v, const TcParams p)
+{
+    using C = TcCfg<D>;
+    // ---- which block: heaviest (longest causal span) blocks first, heads of a KV group adjacent
+    const int per_block = p.Hq * p.B;
+    const int qb = p.n_qblocks - 1 - (int)(blockIdx.x / per_block);
+    const int hb = blockIdx.x % per_block;
+    const int h = hb % p.Hq, b = hb / p.Hq;
+    const int kvh = h / p.G;
+    int L = p.seq_lens[b];
+    L = L < 0 ? 0 : (L > p.S_max ? p.S_max : L);
+    const int q0 = qb * 2 * kRows;
+    if (q0 >= L) return;
+    const int n_tiles_L = (L + kRows - 1) / kRows;              // K/V tiles that hold any valid token
+    int n_sub[2];
+    n_sub[0] = min(n_tiles_L, 2 * qb + 1);
+    n_sub[1] = (q0 + kRows < L) ? min(n_tiles_L, 2 * qb + 2) : 0;
+    const int n_kv = max(n_sub[0], n_sub[1]);
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    uint8_t *smem = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
+    uint8_t *q_smem = smem;                                       // 2 sub-tiles
+    uint8_t *ring = smem + 2 * C::kTileBytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(ring + (size_t)C::kSlots * C::kTileBytes);
+    uint64_t *q_full = bars;
+    uint64_t *kv_full = bars + 1;
+    uint64_t *kv_empty = kv_full + C::kSlots;
+    uint64_t *s_full = kv_empty + C::kSlots;      // [2]
+    uint64_t *p_full = s_full + 2;                // [2]
+    uint64_t *o_full = p_full + 2;                // [2]
+    uint32_t *tmem_base_smem = reinterpret_cast<uint32_t *>(o_full + 2);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_base_smem + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        mbar_init(q_full, 1);
+        for (int s = 0; s < C::kSlots; ++s) {
+            mbar_init(&kv_full[s], 1);
+            mbar_init(&kv_empty[s], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&s_full[i], 1);
+            mbar_init(&p_full[i], kRows);
+            mbar_init(&o_full[i], 1);
+        }
+        *abort_flag = 0;
+        fence_barrier_init();
+        fence_proxy_async_smem();
+    }
+    if (warp == 9) {
+        tmem_alloc(tmem_base_smem, C::kTmemCols);
+        tmem_relinquish_alloc_permit();
+    }
+    tcgen05_fence_before_sync();
+    __syncthreads();
+    tcgen05_fence_after_sync();
+    const uint32_t tmem_base = *tmem_base_smem;
+
+    if (warp == 8) {
+        // ============================================================ TMA producer (+ cache copy)
+        if (lane == 0) {
+            tma_prefetch_desc(&tmap_q);
+            tma_prefetch_desc(&tmap_k);
+            tma_prefetch_desc(&tmap_v);
+            int c1, c2, c3;
+            mbar_arrive_expect_tx(q_full, 2 * C::kTileBytes);
+            for (int i = 0; i < 2; ++i) {
+                order_coords(p.cq, q0 + i * kRows, h, b, c1, c2, c3);
+#pragma unroll
+                for (int hf = 0; hf < C::kHalves; ++hf)
+                    tma_load_4d(q_smem + i * C::kTileBytes + hf * kHalfBytes, &tmap_q, q_full, hf * 64, c1, c2, c3);
+            }
+            for (int idx = 0; idx < 2 * n_kv; ++idx) {
+                const int j = idx >> 1;
+                const uint32_t s = idx % C::kSlots, ph = (idx / C::kSlots) & 1u;
+                if (!mbar_wait(&kv_empty[s], ph ^ 1u, abort_flag)) break;
+                mbar_arrive_expect_tx(&kv_full[s], C::kTileBytes);
+                order_coords(p.ckv, j * kRows, kvh, b, c1, c2, c3);
+                const CUtensorMap *tm = (idx & 1) ? &tmap_v : &tmap_k;
+#pragma unroll
+                for (int hf = 0; hf < C::kHalves; ++hf)
+                    tma_load_4d(ring + (size_t)s * C::kTileBytes + hf * kHalfBytes, tm, &kv_full[s], hf * 64, c1, c2, c3);
+            }
+        }
+        __syncwarp();
+        if (p.cache_k != nullptr && (h % p.G) == 0) {
+            // the block's diagonal K/V tiles (2*qb and 2*qb+1) go to the cache; they are the last tiles
+            // loaded, so their slots are not refilled. Rows >= L are never written.
+            const int lim = min(L, p.cache_max_len);
+            for (int j = 2 * qb; j < n_kv; ++j) {
+                for (int kv = 0; kv < 2; ++kv) {
+                    const int idx = 2 * j + kv;
+                    const uint32_t s = idx % C::kSlots, ph = (idx / C::kSlots) & 1u;
+                    if (!mbar_wait(&kv_full[s], ph, abort_flag)) break;
+                    const uint8_t *src = ring + (size_t)s * C::kTileBytes;
+                    __nv_bfloat16 *dst_base = (kv ? p.cache_v : p.cache_k) + b * p.c_sb + kvh * p.c_sh;
+                    constexpr int kChunks = D / 8;
+                    const int rows = min(kRows, lim - j * kRows);
+                    for (int i = lane; i < rows * kChunks; i += 32) {
+                        const int r = i / kChunks, ch = i % kChunks;
+                        const uint4 val =
+                            *reinterpret_cast<const uint4 *>(src + (ch >> 3) * kHalfBytes + swz128(r, ch & 7));
+                        *reinterpret_cast<uint4 *>(dst_base + (int64_t)(j * kRows + r) * p.c_st + ch * 8) = val;
+                    }
+                }
+            }
+        }
+    } else if (warp == 9) {
+        // ============================================================ MMA issuer
+        constexpr uint32_t idesc_qk = make_idesc(kRows, false);
+        constexpr uint32_t idesc_pv = make_idesc(D, true);
+        const uint32_t tmem_s[2] = {tmem_base + C::kColS0, tmem_base + C::kColS1};
+        const uint32_t tmem_o[2] = {tmem_base + C::kColO0, tmem_base + C::kColO1};
+        const uint32_t q_addr = smem_u32(q_smem), ring_addr = smem_u32(ring);
+
+        auto issue_qk = [&](int i, uint32_t k_addr) {
+#pragma unroll
+            for (int k = 0; k < D / 16; ++k) {
+                const uint32_t off = (k >> 2) * kHalfBytes + (k & 3) * 32;
+                tcgen05_mma_ss(tmem_s[i], make_smem_desc(q_addr + i * C::kTileBytes + off, 0),
+                               make_smem_desc(k_addr + off, 0), idesc_qk, k > 0 ? 1u : 0u);
+            }
+        };
+        auto issue_pv = [&](int i, uint32_t v_addr, bool first) {
+#pragma unroll
+            for (int k = 0; k < kRows / 16; ++k)
+                tcgen05_mma_ts(tmem_o[i], tmem_s[i] + k * 8, make_smem_desc(v_addr + k * 2048, kHalfBytes), idesc_pv,
+                               (first && k == 0) ? 0u : 1u);
+        };
+
+        bool ok = mbar_wait(q_full, 0, abort_flag) && mbar_wait(&kv_full[0], 0, abort_flag);
+        if (ok) {
+            tcgen05_fence_after_sync();
+            if (lane == 0) {
+                for (int i = 0; i < 2; ++i)
+                    if (n_sub[i] > 0) {
+                        issue_qk(i, ring_addr);
+                        tcgen05_commit(&s_full[i]);
+                    }
+                tcgen05_commit(&kv_empty[0]);
+            }
+            __syncwarp();
+        }
+        for (int j = 0; ok && j < n_kv; ++j) {
+            const int iv = 2 * j + 1, ik = 2 * j + 2;
+            const uint32_t sv = iv % C::kSlots, sk = ik % C::kSlots;
+            if (!mbar_wait(&kv_full[sv], (iv / C::kSlots) & 1u, abort_flag)) { ok = false; break; }
+            const int first_dead = L - j * kRows;                 // V rows >= this hold no valid token
+            if (first_dead < kRows) {
+                // may hold any bits (NaN included): clear, so that a zero weight times garbage cannot appear
+                uint8_t *vt = ring + (size_t)sv * C::kTileBytes;
+                constexpr int kChunks = D / 8;
+                for (int i = lane; i < (kRows - first_dead) * kChunks; i += 32) {
+                    const int r = first_dead + i / kChunks, ch = i % kChunks;
+                    *reinterpret_cast<uint4 *>(vt + (ch >> 3) * kHalfBytes + r * 128 + ((ch & 7) << 4)) =
+                        make_uint4(0u, 0u, 0u, 0u);
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+            }
+            const bool have_next = j + 1 < n_kv;
+            if (have_next && !mbar_wait(&kv_full[sk], (ik / C::kSlots) & 1u, abort_flag)) { ok = false; break; }
+            for (int i = 0; i < 2 && ok; ++i) {
+                if (j >= n_sub[i]) continue;
+                if (!mbar_wait(&p_full[i], j & 1u, abort_flag)) { ok = false; break; }
+                tcgen05_fence_after_sync();
+                if (lane == 0) {
+                    issue_pv(i, ring_addr + sv * C::kTileBytes, j == 0);
+                    if (j + 1 < n_sub[i]) {
+                        issue_qk(i, ring_addr + sk * C::kTileBytes);
+                        tcgen05_commit(&s_full[i]);
+                    } else {
+                        tcgen05_commit(&o_full[i]);
+                    }
+                }
+                __syncwarp();
+            }
+            if (ok && lane == 0) {
+                tcgen05_commit(&kv_empty[sv]);
+                if (have_next) tcgen05_commit(&kv_empty[sk]);
+            }
+            __syncwarp();
+        }
+    } else {
+        // ============================================================ softmax + epilogue warpgroups
+        const int i = warp >> 2;                                   // sub-tile
+        const int t = threadIdx.x & 127;                           // row within the sub-tile == TMEM lane
+        const int row = q0 + i * kRows + t;                        // token index of this thread's query row
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tmem_s = tmem_base + lane_base + (i ? C::kColS1 : C::kColS0);
+        const uint32_t tmem_o = tmem_base + lane_base + (i ? C::kColO1 : C::kColO0);
+        const int n_mine = n_sub[i];
+        const int diag_tile = (q0 + i * kRows) / kRows;
+        const float c = p.scale_log2e;
+        float m = -INFINITY, l = 0.f;
+        bool ok = true;
+
+        for (int j = 0; j < n_mine; ++j) {
+            if (!mbar_wait(&s_full[i], j & 1u, abort_flag)) { ok = false; break; }
+            tcgen05_fence_after_sync();
+            uint32_t sr[4][32];
+#pragma unroll
+            for (int qd = 0; qd < 4; ++qd) tmem_ld_32x32b_x32(tmem_s + qd * 32, sr[qd]);
+            tcgen05_wait_ld();
+
+            // scaled scores (log2 domain); causal mask on the diagonal tile
+            float mx = -INFINITY;
+            if (j == diag_tile) {
+                const int lim = row - j * kRows;                   // columns > lim are in the future
+#pragma unroll
+                for (int qd = 0; qd < 4; ++qd)
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) {
+                        float x = __uint_as_float(sr[qd][e]) * c;
+                        x = (qd * 32 + e > lim) ? -INFINITY : x;
+                        sr[qd][e] = __float_as_uint(x);
+                        mx = fmaxf(mx, x);
+                    }
+            } else {
+#pragma unroll
+                for (int qd = 0; qd < 4; ++qd)
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) {
+                        const float x = __uint_as_float(sr[qd][e]) * c;
+                        sr[qd][e] = __float_as_uint(x);
+                        mx = fmaxf(mx, x);
+                    }
+            }
+            // lazy rescale: keep the old reference max unless the new one is much larger
+            const bool grow = (mx > m + kRescaleThreshold) || (j == 0);
+            float alpha = 1.f;
+            if (grow) {
+                const float m_new = (mx == -INFINITY) ? 0.f : mx;
+                alpha = fast_exp2(m - m_new);                      // j == 0: exp2(-inf) = 0
+                m = m_new;
+                l *= alpha;
+            }
+            if (j > 0 && __any_sync(0xffffffffu, grow)) {
+                // PV_{j-1} has completed (s_full is committed after it), PV_j is not issued before p_full
+#pragma unroll
+                for (int qd = 0; qd < D / 32; ++qd) {
+                    uint32_t orr[32];
+                    tmem_ld_32x32b_x32(tmem_o + qd * 32, orr);
+                    tcgen05_wait_ld();
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) orr[e] = __float_as_uint(__uint_as_float(orr[e]) * alpha);
+                    tmem_st_32x32b_x32(tmem_o + qd * 32, orr);
+                }
+            }
+            float sum = 0.f;
+#pragma unroll
+            for (int qd = 0; qd < 4; ++qd) {
+                uint32_t pk[16];
+#pragma unroll
+                for (int e = 0; e < 16; ++e) {
+                    const float p0 = fast_exp2(__uint_as_float(sr[qd][2 * e]) - m);
+                    const float p1 = fast_exp2(__uint_as_float(sr[qd][2 * e + 1]) - m);
+                    sum += p0 + p1;
+                    pk[e] = pack_bf16x2(p0, p1);
+                }
+                tmem_st_32x32b_x16(tmem_s + qd * 16, pk);
+            }
+            l += sum;
+            tcgen05_wait_st();
+            tcgen05_fence_before_sync();
+            mbar_arrive(&p_full[i]);
+        }
+
+        if (ok && n_mine > 0 && mbar_wait(&o_full[i], 0, abort_flag)) {
+            tcgen05_fence_after_sync();
+            const float inv = 1.f / l;
+            const bool valid = row < L;
+            __nv_bfloat16 *orow = p.o + b * p.o_sb + (int64_t)row * p.o_st + h * p.o_sh;
+#pragma unroll
+            for (int qd = 0; qd < D / 32; ++qd) {
+                uint32_t orr[32];
+                tmem_ld_32x32b_x32(tmem_o + qd * 32, orr);
+                tcgen05_wait_ld();
+                if (valid) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        uint4 val;
+                        val.x = pack_bf16x2(__uint_as_float(orr[8 * e + 0]) * inv, __uint_as_float(orr[8 * e + 1]) * inv);
+                        val.y = pack_bf16x2(__uint_as_float(orr[8 * e + 2]) * inv, __uint_as_float(orr[8 * e + 3]) * inv);
+                        val.z = pack_bf16x2(__uint_as_float(orr[8 * e + 4]) * inv, __uint_as_float(orr[8 * e + 5]) * inv);
+                        val.w = pack_bf16x2(__uint_as_float(orr[8 * e + 6]) * inv, __uint_as_float(orr[8 * e + 7]) * inv);
+                        *reinterpret_cast<uint4 *>(orow + qd * 32 + e * 8) = val;
+                    }
+                }
+            }
+            if (valid && p.lse)
+                p.lse[((size_t)b * p.Hq + h) * p.S_max + row] = (m + log2f(l)) * 0.6931471805599453f;
+        }
+    }
+
+    tcgen05_fence_before_sync();
+    __syncthreads();
+    if (warp == 9) {
+        tcgen05_fence_after_sync();
+        tmem_dealloc(tmem_base, C::kTmemCols);
+    }
+    if (threadIdx.x == 0 && *abort_flag) {
+        atomicOr(p.status + kStatusErrWord, kErrPrefillWait);
+        p.status[kStatusInfoWord] = 0x20000u | (blockIdx.x & 0xffffu);
+    }
+}
+
+template <int D>
+l4l_status launch_t(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const TcParams &p,
+                    cudaStream_t stream)
+{
+    using C = TcCfg<D>;
+    static bool configured = false;
+    if (!configured) {
+        if (cudaFuncSetAttribute(prefill_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)C::kSmemBytes) != cudaSuccess)
+            return L4L_ERR_CUDA;
+        configured = true;
+    }
+    const long long grid = (long long)p.n_qblocks * p.Hq * p.B;
+    if (grid > 0x7fffffffll) return L4L_ERR_UNSUPPORTED;
+    prefill_tc_kernel<D><<<(unsigned)grid, kThreads, C::kSmemBytes, stream>>>(tq, tk, tv, p);
+    return cudaGetLastError() == cudaSuccess ? L4L_OK : L4L_ERR_CUDA;
+}
+
+}  // namespace
+
+l4l_status launch_prefill_tc(const l4l_tensor4 &q, const l4l_tensor4 &k, const l4l_tensor4 &v,
+                             const l4l_tensor4 &o, const l4l_kv_cache &cache, const int32_t *d_seq_lens,
+                             int S_max, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
+                             void *workspace, cudaStream_t stream)
+{
+    CUtensorMap tq, tk, tv;
+    TmapCoord cq, ck, cv;
+    if (!make_tmap_bf16(&tq, &cq, q.ptr, D, S_max, Hq, B, q.stride_t, q.stride_h, q.stride_b, 64, kRows) ||
+        !make_tmap_bf16(&tk, &ck, k.ptr, D, S_max, Hkv, B, k.stride_t, k.stride_h, k.stride_b, 64, kRows) ||
+        !make_tmap_bf16(&tv, &cv, v.ptr, D, S_max, Hkv, B, v.stride_t, v.stride_h, v.stride_b, 64, kRows))
+        return L4L_ERR_CUDA;
+    if (ck.pos_t != cv.pos_t || ck.pos_h != cv.pos_h || ck.pos_b != cv.pos_b) return L4L_ERR_UNSUPPORTED;
+    TcParams p;
+    p.o = static_cast<__nv_bfloat16 *>(o.ptr);
+    p.o_sb = o.stride_b; p.o_st = o.stride_t; p.o_sh = o.stride_h;
+    p.cache_k = static_cast<__nv_bfloat16 *>(cache.k);
+    p.cache_v = static_cast<__nv_bfloat16 *>(cache.v);
+    p.c_sb = cache.stride_b; p.c_sh = cache.stride_h; p.c_st = cache.stride_t;
+    p.cache_max_len = cache.max_len;
+    p.seq_lens = d_seq_lens;
+    p.lse = d_lse;
+    p.status = static_cast<unsigned *>(workspace);
+    p.S_max = S_max; p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.G = Hq / Hkv;
+    p.n_qblocks = (S_max + 2 * kRows - 1) / (2 * kRows);
+    p.scale_log2e = scale * 1.4426950408889634f;
+    p.cq = cq; p.ckv = ck;
+    return (D == 128) ? launch_t<128>(tq, tk, tv, p, stream) : launch_t<64>(tq, tk, tv, p, stream);
+}
+
+}  // namespace l4l
