@@ -49,7 +49,7 @@ def measured_peaks():
 class ClockSampler(threading.Thread):
     """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
 
-    def __init__(self, index: int, period_s: float = 0.02):
+    def __init__(self, index: int, period_s: float = 0.005):
         super().__init__(daemon=True)
         self.index, self.period = index, period_s
         self.samples, self.reasons, self.max_mhz = [], set(), None
@@ -338,6 +338,35 @@ def run_ours(args, rank, world):
     print(json.dumps(line))
 
 
+def run_profile_case(case: str):
+    """A few launches of ONE kernel on a small case, for `ncu` captures (not a benchmark):
+    prefill = B=1, S=8192 of the long_prefill workload (inputs 168 MB > L2); decode = the batched_decode batch."""
+    from paper_2608_21836_b200 import binding as l4l
+
+    torch.cuda.set_device(0)
+    if case == "prefill":
+        w = wl.WORKLOADS["long_prefill"]
+        seq = wl.make_sequence(w, B=1)
+        q, k, v = seq.q.cuda(), seq.k.cuda(), seq.v.cuda()
+        o = torch.empty_like(q)
+        ck = torch.empty(1, w.Hkv, seq.S, w.D, dtype=torch.bfloat16, device="cuda")
+        cv = torch.empty_like(ck)
+        lens = torch.full((1,), seq.S, dtype=torch.int32, device="cuda")
+        ws = l4l.new_workspace(l4l.L4L_OP_PREFILL, 1, w.Hq, w.Hkv, w.D, seq.S)
+        for _ in range(3):
+            l4l.l4l_attn_prefill(q, k, v, o, lens, w.scale, ws, cache_k=ck, cache_v=cv)
+    else:
+        w = wl.WORKLOADS["batched_decode"]
+        db = wl.make_decode_batch(w)
+        q, ck, cv, lens = db.q.cuda(), db.cache_k.cuda(), db.cache_v.cuda(), db.kv_len.cuda()
+        o = torch.empty_like(q)
+        ws = l4l.new_workspace(l4l.L4L_OP_DECODE, w.decode_B, w.Hq, w.Hkv, w.D, w.decode_Lmax)
+        for _ in range(3):
+            l4l.l4l_attn_decode(q, o, ck, cv, lens, w.decode_Lmax, w.scale, ws)
+    torch.cuda.synchronize()
+    print(json.dumps({"profile_case": case, "device_error": l4l.l4l_last_device_error(ws)}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -345,7 +374,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--profile-case", choices=["prefill", "decode"], default=None,
+                    help="run three launches of one kernel on a small case and exit (for ncu)")
     args = ap.parse_args()
+    if args.profile_case:
+        run_profile_case(args.profile_case)
+        return
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
     if args.impl == "reference":
