@@ -25,7 +25,7 @@ namespace l4l {
 namespace {
 
 constexpr int kRows = 128;                     // rows per sub-tile == tokens per K/V tile
-constexpr int kThreads = 320;
+constexpr int kThreads = 384;                  // 3 warpgroups: softmax 0, softmax 1, {producer, MMA, 2 idle}
 constexpr uint32_t kHalfBytes = kRows * 128;   // [128 rows][64 bf16], 128-byte swizzled
 constexpr float kRescaleThreshold = 8.f;       // log2 domain: O is rescaled only if the max grew by > 2^8
 
@@ -145,6 +145,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     tcgen05_fence_after_sync();
     const uint32_t tmem_base = *tmem_base_smem;
 
+    // Register reallocation: the data-movement warpgroup gives registers to the softmax warpgroups,
+    // whose threads hold a whole 128-column score row.
+    if (warp >= 8) {
+    setmaxnreg_dec<56>();
     if (warp == 8) {
         // ============================================================ TMA producer (+ cache copy)
         if (lane == 0) {
@@ -270,7 +274,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
             }
             __syncwarp();
         }
+    }
     } else {
+        setmaxnreg_inc<224>();
         // ============================================================ softmax + epilogue warpgroups
         const int i = warp >> 2;                                   // sub-tile
         const int t = threadIdx.x & 127;                           // row within the sub-tile == TMEM lane
@@ -292,28 +298,52 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
             for (int qd = 0; qd < 4; ++qd) tmem_ld_32x32b_x32(tmem_s + qd * 32, sr[qd]);
             tcgen05_wait_ld();
 
-            // scaled scores (log2 domain); causal mask on the diagonal tile
-            float mx = -INFINITY;
-            if (j == diag_tile) {
+            // Row maximum of the scaled scores (log2 domain). Off the diagonal the maximum is taken over the
+            // raw scores with independent 3-input max chains and scaled once (min for a negative scale);
+            // on the diagonal tile the causal mask is applied to the scaled scores first.
+            const bool diag = (j == diag_tile);
+            float mx;
+            if (diag) {
                 const int lim = row - j * kRows;                   // columns > lim are in the future
+                float a0 = -INFINITY, a1 = -INFINITY, a2 = -INFINITY, a3 = -INFINITY;
 #pragma unroll
                 for (int qd = 0; qd < 4; ++qd)
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) {
-                        float x = __uint_as_float(sr[qd][e]) * c;
-                        x = (qd * 32 + e > lim) ? -INFINITY : x;
-                        sr[qd][e] = __float_as_uint(x);
-                        mx = fmaxf(mx, x);
+                    for (int e = 0; e < 32; e += 4) {
+                        float x[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            x[u] = __uint_as_float(sr[qd][e + u]) * c;
+                            x[u] = (qd * 32 + e + u > lim) ? -INFINITY : x[u];
+                            sr[qd][e + u] = __float_as_uint(x[u]);
+                        }
+                        a0 = fmaxf(a0, x[0]); a1 = fmaxf(a1, x[1]); a2 = fmaxf(a2, x[2]); a3 = fmaxf(a3, x[3]);
                     }
+                mx = fmaxf(fmaxf(a0, a1), fmaxf(a2, a3));
+            } else if (c >= 0.f) {
+                float a0 = -INFINITY, a1 = -INFINITY, a2 = -INFINITY, a3 = -INFINITY;
+#pragma unroll
+                for (int qd = 0; qd < 4; ++qd)
+#pragma unroll
+                    for (int e = 0; e < 32; e += 8) {
+                        a0 = max3(a0, __uint_as_float(sr[qd][e + 0]), __uint_as_float(sr[qd][e + 1]));
+                        a1 = max3(a1, __uint_as_float(sr[qd][e + 2]), __uint_as_float(sr[qd][e + 3]));
+                        a2 = max3(a2, __uint_as_float(sr[qd][e + 4]), __uint_as_float(sr[qd][e + 5]));
+                        a3 = max3(a3, __uint_as_float(sr[qd][e + 6]), __uint_as_float(sr[qd][e + 7]));
+                    }
+                mx = fmaxf(fmaxf(a0, a1), fmaxf(a2, a3)) * c;
             } else {
+                float a0 = INFINITY, a1 = INFINITY, a2 = INFINITY, a3 = INFINITY;
 #pragma unroll
                 for (int qd = 0; qd < 4; ++qd)
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) {
-                        const float x = __uint_as_float(sr[qd][e]) * c;
-                        sr[qd][e] = __float_as_uint(x);
-                        mx = fmaxf(mx, x);
+                    for (int e = 0; e < 32; e += 4) {
+                        a0 = fminf(a0, __uint_as_float(sr[qd][e + 0]));
+                        a1 = fminf(a1, __uint_as_float(sr[qd][e + 1]));
+                        a2 = fminf(a2, __uint_as_float(sr[qd][e + 2]));
+                        a3 = fminf(a3, __uint_as_float(sr[qd][e + 3]));
                     }
+                mx = fminf(fminf(a0, a1), fminf(a2, a3)) * c;
             }
             // lazy rescale: keep the old reference max unless the new one is much larger
             const bool grow = (mx > m + kRescaleThreshold) || (j == 0);
@@ -336,19 +366,33 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
                     tmem_st_32x32b_x32(tmem_o + qd * 32, orr);
                 }
             }
-            float sum = 0.f;
+            // p = 2^(x - m): packed fp32x2 FMA feeds the exp2 unit; sums in two independent packed chains
+            const float fc = diag ? 1.f : c;                       // diagonal scores are already scaled
+            const uint64_t c2 = pack_f32x2(fc, fc), nm2 = pack_f32x2(-m, -m);
+            uint64_t sum_a = pack_f32x2(0.f, 0.f), sum_b = sum_a;
 #pragma unroll
             for (int qd = 0; qd < 4; ++qd) {
                 uint32_t pk[16];
 #pragma unroll
-                for (int e = 0; e < 16; ++e) {
-                    const float p0 = fast_exp2(__uint_as_float(sr[qd][2 * e]) - m);
-                    const float p1 = fast_exp2(__uint_as_float(sr[qd][2 * e + 1]) - m);
-                    sum += p0 + p1;
-                    pk[e] = pack_bf16x2(p0, p1);
+                for (int e = 0; e < 16; e += 2) {
+                    const uint64_t xa = fma_f32x2(pack_u32x2(sr[qd][2 * e], sr[qd][2 * e + 1]), c2, nm2);
+                    const uint64_t xb = fma_f32x2(pack_u32x2(sr[qd][2 * e + 2], sr[qd][2 * e + 3]), c2, nm2);
+                    float xa0, xa1, xb0, xb1;
+                    unpack_f32x2(xa, xa0, xa1);
+                    unpack_f32x2(xb, xb0, xb1);
+                    const float pa0 = fast_exp2(xa0), pa1 = fast_exp2(xa1);
+                    const float pb0 = fast_exp2(xb0), pb1 = fast_exp2(xb1);
+                    sum_a = add_f32x2(sum_a, pack_f32x2(pa0, pa1));
+                    sum_b = add_f32x2(sum_b, pack_f32x2(pb0, pb1));
+                    pk[e] = pack_bf16x2(pa0, pa1);
+                    pk[e + 1] = pack_bf16x2(pb0, pb1);
                 }
                 tmem_st_32x32b_x16(tmem_s + qd * 16, pk);
             }
+            float sa0, sa1, sb0, sb1;
+            unpack_f32x2(sum_a, sa0, sa1);
+            unpack_f32x2(sum_b, sb0, sb1);
+            const float sum = (sa0 + sa1) + (sb0 + sb1);
             l += sum;
             tcgen05_wait_st();
             tcgen05_fence_before_sync();
