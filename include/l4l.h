@@ -81,9 +81,10 @@ enum { L4L_OP_PREFILL = 0, L4L_OP_DECODE = 1 };
 size_t l4l_workspace_bytes(int op, int B, int Hq, int Hkv, int head_dim, int max_len);
 
 /*
- * Zero the workspace's status block (enqueued on `stream`). Call once after allocating a
- * workspace and again after a reported device error. The rest of the workspace needs no
- * initialisation.
+ * Zero the workspace (status block and the decode ticket counters; enqueued on `stream`).
+ * Call once after allocating a workspace and again after a reported device error. The
+ * kernels leave the counters at zero, so no re-initialisation is needed between calls. A
+ * workspace serves one call at a time: calls that may overlap on the device need their own.
  */
 l4l_status l4l_workspace_init(void *workspace, size_t ws_bytes, l4l_stream stream);
 

@@ -130,7 +130,7 @@ size_t l4l_workspace_bytes(int op, int B, int Hq, int Hkv, int head_dim, int max
 l4l_status l4l_workspace_init(void *workspace, size_t ws_bytes, l4l_stream stream)
 {
     if (!workspace || ws_bytes < kStatusBytes) return L4L_ERR_WORKSPACE;
-    return cudaMemsetAsync(workspace, 0, kStatusBytes, static_cast<cudaStream_t>(stream)) == cudaSuccess
+    return cudaMemsetAsync(workspace, 0, ws_bytes, static_cast<cudaStream_t>(stream)) == cudaSuccess
                ? L4L_OK
                : L4L_ERR_CUDA;
 }

@@ -1,16 +1,23 @@
 // Decode attention: one query token per sequence over a ragged bf16 KV cache.
 //
-// Pass 1 (decode_split_kernel): persistent CTAs stream the cache exactly once. A work item is
-// (sequence, KV head, chunk of `chunk` tokens); items are enumerated from the device-side
-// lengths (prefix sum over sequences) and dealt round-robin to the CTAs. One producer warp
-// keeps a ring of TMA tiles (64 tokens of K and V, 128-byte swizzle) full across item
-// boundaries; four consumer warps each take 16 tokens of every tile and serve ALL query heads
-// of the KV group from it: the group is the M dimension (zero padded to 16) of warp-level
-// bf16 MMAs, so the cache bytes are read once per group. Softmax statistics are fp32, row
-// maxima are reduced with warp shuffles, and the four warps' partial results are merged
-// through shared memory at the end of an item.
-// Pass 2 (decode_merge_kernel): log-sum-exp merge of the chunk partials of each
-// (sequence, query head); sequences that fit one chunk were already finished by pass 1.
+// One launch. The cache of every (sequence, KV head) is cut into 64-token tiles; the flattened
+// tile stream (sequence-major, then KV head, then position) is divided EVENLY among persistent
+// CTAs, so every CTA streams the same number of bytes whatever the length mix. A CTA's range may
+// start or end inside a sequence: each (sequence, KV head) is thus covered by one or more
+// "pieces", one per CTA that touches it.
+//
+//   producer warp    walks the CTA's tile range and keeps a ring of TMA tiles (K and V, 128-byte
+//                    swizzle) full, across piece boundaries
+//   4 consumer warps each take 16 tokens of every tile and serve ALL query heads of the KV group
+//                    from it: the group is the M dimension (zero-padded to 16) of warp-level bf16
+//                    MMAs, so cache bytes are read once per group. Softmax statistics are fp32;
+//                    row maxima are reduced with warp shuffles. At the end of a piece they drop
+//                    their (max, sum, O) into shared memory and go straight on to the next tile.
+//   finisher warp    merges the four warps' results of a piece off the critical path. A sequence
+//                    covered by a single piece is written out directly; otherwise the piece's
+//                    normalised fp32 partial and its log-sum-exp go to the workspace, and the LAST
+//                    piece to arrive (a self-resetting ticket counter per (sequence, KV head)) runs
+//                    the second pass: the log-sum-exp merge of all pieces.
 #include "l4l_internal.h"
 #include "l4l_warp_attn.cuh"
 
@@ -20,7 +27,9 @@ namespace {
 
 constexpr int kTileT = 64;                 // tokens per TMA tile
 constexpr int kConsumerWarps = 4;
-constexpr int kThreads = (kConsumerWarps + 1) * 32;
+constexpr int kProducerWarp = kConsumerWarps;
+constexpr int kFinisherWarp = kConsumerWarps + 1;
+constexpr int kThreads = (kConsumerWarps + 2) * 32;
 constexpr int kMaxB = 1024;                // sequences per launch (prefix sums live in shared memory)
 
 template <int D>
@@ -33,9 +42,13 @@ struct DecodeCfg {
 };
 
 struct TileMeta {
-    int b, kvh, t0, chunk_idx, kv_len, nchunks, flags, pad;
+    int b, kvh, t0, piece, kv_len, npieces, flags, pad;
 };
 constexpr int kFlagFirst = 1, kFlagLast = 2, kFlagStop = 4;
+
+struct PieceMeta {
+    int b, kvh, piece, npieces, stop, pad0, pad1, pad2;
+};
 
 struct DecodeParams {
     const __nv_bfloat16 *q;   // [B, Hq, D]
@@ -43,20 +56,21 @@ struct DecodeParams {
     float *lse;               // [B, Hq] or null
     const int32_t *kv_lens;   // [B]
     float *part_o;            // [B, Hq, nsplit, D]  normalised partial outputs
-    float *part_lse;          // [B, Hq, nsplit]     log2-domain log-sum-exp of the chunk
+    float *part_lse;          // [B, Hq, nsplit]     log2-domain log-sum-exp of the piece
+    int *tickets;             // [B, Hkv]            pieces arrived; zero between calls
     unsigned *status;
-    int B, Hq, Hkv, G, chunk, nsplit;
+    int B, Hq, Hkv, G, min_tiles, nsplit, max_kv_len;
     float scale_log2e;
     TmapCoord coord;
 };
 
 template <int D>
-size_t decode_smem_bytes(int G)
+size_t decode_smem_bytes(int G, int nsplit)
 {
     using C = DecodeCfg<D>;
-    size_t comb = (size_t)kConsumerWarps * G * (D + 2) * sizeof(float);
-    return 1024 /*alignment slack*/ + (size_t)C::kStages * C::kStageBytes + comb +
-           C::kStages * sizeof(TileMeta) + (2 * C::kStages + 2) * sizeof(uint64_t) + (kMaxB + 1) * sizeof(int) + 64;
+    size_t comb = (size_t)kConsumerWarps * G * (D + 4) * sizeof(float) + (size_t)((G * nsplit + 3) & ~3) * sizeof(float);
+    return 1024 /*alignment slack*/ + (size_t)C::kStages * C::kStageBytes + comb + C::kStages * sizeof(TileMeta) +
+           sizeof(PieceMeta) + (2 * C::kStages + 2) * sizeof(uint64_t) + (kMaxB + 1) * sizeof(int) + 64;
 }
 
 __device__ __forceinline__ void order_coords(const TmapCoord &c, int t, int h, int b, int &c1, int &c2, int &c3)
@@ -78,12 +92,17 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
 
     uint8_t *stages = smem;
     float *comb = reinterpret_cast<float *>(stages + (size_t)C::kStages * C::kStageBytes);
-    const int comb_floats = kConsumerWarps * p.G * (D + 2);
-    TileMeta *meta = reinterpret_cast<TileMeta *>(comb + comb_floats);
-    uint64_t *full = reinterpret_cast<uint64_t *>(meta + C::kStages);
+    constexpr int kPitch = D + 4;            // floats per row of `comb`: O[D], max, sum, pad (16-byte rows)
+    constexpr int kVec = D / 4;
+    const int comb_floats = kConsumerWarps * p.G * kPitch;
+    float *merge_lse = comb + comb_floats;   // [G][nsplit] scratch of the finisher's second pass
+    TileMeta *meta = reinterpret_cast<TileMeta *>(merge_lse + ((p.G * p.nsplit + 3) & ~3));   // keeps 16-byte alignment
+    PieceMeta *piece_meta = reinterpret_cast<PieceMeta *>(meta + C::kStages);
+    uint64_t *full = reinterpret_cast<uint64_t *>(piece_meta + 1);
     uint64_t *empty = full + C::kStages;
-    uint64_t *comb_bar = empty + C::kStages;   // [0]: partials written, [1]: partials consumed
-    int *cum = reinterpret_cast<int *>(comb_bar + 2);
+    uint64_t *comb_full = empty + C::kStages;   // consumers -> finisher: a piece's results are in `comb`
+    uint64_t *comb_empty = comb_full + 1;       // finisher -> consumers: `comb` may be overwritten
+    int *cum = reinterpret_cast<int *>(comb_empty + 1);   // cum[b] = tiles of sequences < b (times Hkv)
     volatile int *abort_flag = cum + (kMaxB + 1);
 
     const int warp = threadIdx.x >> 5;
@@ -94,26 +113,29 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             mbar_init(&full[s], 1);
             mbar_init(&empty[s], kConsumerWarps);
         }
-        mbar_init(&comb_bar[0], kConsumerWarps);
-        mbar_init(&comb_bar[1], kConsumerWarps);
+        mbar_init(comb_full, kConsumerWarps);
+        mbar_init(comb_empty, 1);
         *abort_flag = 0;
         fence_barrier_init();
         fence_proxy_async_smem();
     }
     __syncthreads();
 
-    if (warp == kConsumerWarps) {
+    if (warp == kProducerWarp) {
         // ------------------------------------------------------------------ producer warp
-        // exclusive prefix sum of chunks per sequence
+        if (lane == 0) {
+            tma_prefetch_desc(&tmap_k);
+            tma_prefetch_desc(&tmap_v);
+        }
+        // exclusive prefix sum over sequences of (tiles * Hkv)
         int running = 0;
         for (int b0 = 0; b0 < p.B; b0 += 32) {
             const int b = b0 + lane;
             int n = 0;
             if (b < p.B) {
                 int len = p.kv_lens[b];
-                len = len < 0 ? 0 : len;
-                n = (len + p.chunk - 1) / p.chunk;
-                n = n > p.nsplit ? p.nsplit : n;   // lengths beyond the host bound are clipped
+                len = len < 0 ? 0 : (len > p.max_kv_len ? p.max_kv_len : len);
+                n = ((len + kTileT - 1) / kTileT) * p.Hkv;
             }
             int incl = n;
 #pragma unroll
@@ -128,44 +150,51 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
         __syncwarp();
 
         if (lane == 0) {
-            tma_prefetch_desc(&tmap_k);
-            tma_prefetch_desc(&tmap_v);
-            const long long total_items = (long long)running * p.Hkv;
+            const int total = running;
+            int per_cta = (total + (int)gridDim.x - 1) / (int)gridDim.x;
+            per_cta = per_cta < p.min_tiles ? p.min_tiles : per_cta;
+            const int my_begin = min(total, (int)blockIdx.x * per_cta);
+            const int my_end = min(total, my_begin + per_cta);
             uint32_t it = 0;
             bool ok = true;
-            for (long long item = blockIdx.x; ok && item < total_items; item += gridDim.x) {
-                const int pair = (int)(item / p.Hkv);
-                const int kvh = (int)(item % p.Hkv);
-                int lo = 0, hi = p.B;          // largest b with cum[b] <= pair
+            int g = my_begin;
+            while (ok && g < my_end) {
+                int lo = 0, hi = p.B;          // largest b with cum[b] <= g
                 while (hi - lo > 1) {
                     const int mid = (lo + hi) >> 1;
-                    if (cum[mid] <= pair) lo = mid; else hi = mid;
+                    if (cum[mid] <= g) lo = mid; else hi = mid;
                 }
                 const int b = lo;
-                const int c = pair - cum[b];
                 int len = p.kv_lens[b];
-                const int cap = p.nsplit * p.chunk;
-                len = len > cap ? cap : len;
-                const int nchunks = cum[b + 1] - cum[b];
-                const int t_begin = c * p.chunk;
-                const int t_end = min(len, t_begin + p.chunk);
+                len = len > p.max_kv_len ? p.max_kv_len : len;
+                const int tiles_b = (len + kTileT - 1) / kTileT;
+                const int r = g - cum[b];
+                const int kvh = r / tiles_b;
+                const int seq_first = cum[b] + kvh * tiles_b;          // flattened index of this sequence's tile 0
+                const int tile_begin = g - seq_first;
+                const int tile_end = min(tiles_b, my_end - seq_first);
+                const int first_cta = seq_first / per_cta;
+                const int npieces = (seq_first + tiles_b - 1) / per_cta - first_cta + 1;
+                const int piece = (int)blockIdx.x - first_cta;
                 int c1, c2, c3;
-                for (int t0 = t_begin; t0 < t_end; t0 += kTileT, ++it) {
+                for (int tile = tile_begin; tile < tile_end; ++tile, ++it) {
                     const uint32_t s = it % C::kStages;
                     const uint32_t ph = (it / C::kStages) & 1u;
                     if (!mbar_wait(&empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
                     TileMeta &mt = meta[s];
-                    mt.b = b; mt.kvh = kvh; mt.t0 = t0; mt.chunk_idx = c; mt.kv_len = len; mt.nchunks = nchunks;
-                    mt.flags = (t0 == t_begin ? kFlagFirst : 0) | (t0 + kTileT >= t_end ? kFlagLast : 0);
+                    mt.b = b; mt.kvh = kvh; mt.t0 = tile * kTileT; mt.piece = piece; mt.kv_len = len;
+                    mt.npieces = npieces;
+                    mt.flags = (tile == tile_begin ? kFlagFirst : 0) | (tile + 1 == tile_end ? kFlagLast : 0);
                     mbar_arrive_expect_tx(&full[s], C::kStageBytes);
                     uint8_t *dst = stages + (size_t)s * C::kStageBytes;
-                    order_coords(p.coord, t0, kvh, b, c1, c2, c3);
+                    order_coords(p.coord, tile * kTileT, kvh, b, c1, c2, c3);
 #pragma unroll
                     for (int hf = 0; hf < C::kHalves; ++hf) {
                         tma_load_4d(dst + hf * C::kHalfBytes, &tmap_k, &full[s], hf * 64, c1, c2, c3);
                         tma_load_4d(dst + C::kTileBytes + hf * C::kHalfBytes, &tmap_v, &full[s], hf * 64, c1, c2, c3);
                     }
                 }
+                g = seq_first + tile_end;
             }
             if (ok) {
                 const uint32_t s = it % C::kStages;
@@ -176,6 +205,124 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 }
             }
         }
+    } else if (warp == kFinisherWarp) {
+        // ------------------------------------------------------------------ finisher warp
+        // sequences with no cached token get o = 0, lse = -inf (no tile ever refers to them)
+        for (int b = blockIdx.x; b < p.B; b += gridDim.x) {
+            if (p.kv_lens[b] <= 0) {
+                for (int i = lane; i < p.Hq * D; i += 32) p.o[(size_t)b * p.Hq * D + i] = __float2bfloat16_rn(0.f);
+                if (p.lse)
+                    for (int i = lane; i < p.Hq; i += 32) p.lse[(size_t)b * p.Hq + i] = -INFINITY;
+            }
+        }
+        for (uint32_t n = 0;; ++n) {
+            if (!mbar_wait(comb_full, n & 1u, abort_flag)) break;
+            const PieceMeta pm = *piece_meta;
+            if (pm.stop) break;
+            const bool single = (pm.npieces == 1);
+            // merge the four consumer warps' (max, sum, O); each lane owns float4 pieces of the G x D outputs
+            for (int item = lane; item < p.G * kVec; item += 32) {
+                const int r = item / kVec, d4 = item % kVec;
+                float mw[kConsumerWarps];
+                float mstar = -INFINITY;
+#pragma unroll
+                for (int w = 0; w < kConsumerWarps; ++w) {
+                    mw[w] = comb[((size_t)w * p.G + r) * kPitch + D];
+                    mstar = fmaxf(mstar, mw[w]);
+                }
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                float lsum = 0.f;
+#pragma unroll
+                for (int w = 0; w < kConsumerWarps; ++w) {
+                    const float *row = comb + ((size_t)w * p.G + r) * kPitch;
+                    const float wgt = fast_exp2(mw[w] - mstar);    // warp that saw no token: max = -inf -> 0
+                    const float4 v = *reinterpret_cast<const float4 *>(row + d4 * 4);
+                    acc.x += wgt * v.x; acc.y += wgt * v.y; acc.z += wgt * v.z; acc.w += wgt * v.w;
+                    lsum += wgt * row[D + 1];
+                }
+                const float inv = 1.f / lsum;
+                acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+                const size_t bh = (size_t)pm.b * p.Hq + pm.kvh * p.G + r;
+                const float lse2 = mstar + log2f(lsum);
+                if (single) {
+                    uint2 packed;
+                    packed.x = pack_bf16x2(acc.x, acc.y);
+                    packed.y = pack_bf16x2(acc.z, acc.w);
+                    *reinterpret_cast<uint2 *>(p.o + bh * D + d4 * 4) = packed;
+                    if (d4 == 0 && p.lse) p.lse[bh] = lse2 * 0.6931471805599453f;
+                } else {
+                    const size_t slot = bh * p.nsplit + pm.piece;
+                    *reinterpret_cast<float4 *>(p.part_o + slot * D + d4 * 4) = acc;
+                    if (d4 == 0) p.part_lse[slot] = lse2;
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(comb_empty);        // `comb` has been consumed
+            if (single) continue;
+
+            // ---- ticket: the last piece of this (sequence, KV head) to arrive merges all of them
+            __threadfence();                               // this warp's partials visible device-wide
+            __syncwarp();
+            int ticket = 0;
+            if (lane == 0) {
+                int *tk = p.tickets + (size_t)pm.b * p.Hkv + pm.kvh;
+                ticket = atomicAdd(tk, 1);
+                if (ticket == pm.npieces - 1) atomicExch(tk, 0);       // ready for the next call
+            }
+            ticket = __shfl_sync(0xffffffffu, ticket, 0);
+            if (ticket != pm.npieces - 1) continue;
+            __threadfence();
+            // second pass: out = sum_c w_c o_c / sum_c w_c with w_c = 2^(lse_c - max_c lse_c)
+            const int np = pm.npieces;
+            const size_t bh0 = (size_t)pm.b * p.Hq + pm.kvh * p.G;
+            for (int idx = lane; idx < p.G * np; idx += 32) {
+                const int r = idx / np, c = idx % np;
+                merge_lse[r * p.nsplit + c] = __ldcg(p.part_lse + (bh0 + r) * p.nsplit + c);
+            }
+            __syncwarp();
+            for (int base = 0; base < p.G * kVec; base += 4 * 32) {
+                float4 res[4];
+                float lse_out[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int item = base + u * 32 + lane;
+                    res[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    lse_out[u] = 0.f;
+                    if (item < p.G * kVec) {
+                        const int r = item / kVec, d4 = item % kVec;
+                        const float *wl = merge_lse + r * p.nsplit;
+                        float mstar = -INFINITY;
+                        for (int c = 0; c < np; ++c) mstar = fmaxf(mstar, wl[c]);
+                        const float4 *po = reinterpret_cast<const float4 *>(p.part_o + (bh0 + r) * p.nsplit * D) + d4;
+                        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                        float wsum = 0.f;
+#pragma unroll 4
+                        for (int c = 0; c < np; ++c) {
+                            const float w = fast_exp2(wl[c] - mstar);
+                            const float4 v = __ldcg(po + (size_t)c * kVec);
+                            acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+                            wsum += w;
+                        }
+                        const float inv = 1.f / wsum;
+                        res[u] = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+                        lse_out[u] = (mstar + log2f(wsum)) * 0.6931471805599453f;
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int item = base + u * 32 + lane;
+                    if (item < p.G * kVec) {
+                        const int r = item / kVec, d4 = item % kVec;
+                        uint2 packed;
+                        packed.x = pack_bf16x2(res[u].x, res[u].y);
+                        packed.y = pack_bf16x2(res[u].z, res[u].w);
+                        *reinterpret_cast<uint2 *>(p.o + (bh0 + r) * D + d4 * 4) = packed;
+                        if (d4 == 0 && p.lse) p.lse[bh0 + r] = lse_out[u];
+                    }
+                }
+            }
+            __syncwarp();
+        }
     } else {
         // ------------------------------------------------------------------ consumer warps
         WarpAttnState<D> st;
@@ -183,15 +330,22 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
         uint32_t qf[D / 16][4];
         const int r_lo = lane >> 2;          // query head within the group held in rows lane/4, lane/4+8
         const int r_hi = r_lo + 8;
-        const int ctid = threadIdx.x;        // 0..127
-        uint32_t item_par = 0;               // parity of the per-item merge barriers
+        uint32_t n_dumps = 0;                // pieces handed to the finisher so far
 
         for (uint32_t it = 0;; ++it) {
             const uint32_t s = it % C::kStages;
             const uint32_t ph = (it / C::kStages) & 1u;
             if (!mbar_wait(&full[s], ph, abort_flag)) break;
             const TileMeta mt = meta[s];
-            if (mt.flags & kFlagStop) break;
+            if (mt.flags & kFlagStop) {
+                // tell the finisher to stop (after it has drained the previous piece)
+                if (mbar_wait(comb_empty, (n_dumps & 1u) ^ 1u, abort_flag)) {
+                    if (warp == 0 && lane == 0) piece_meta->stop = 1;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(comb_full);
+                }
+                break;
+            }
 
             if (mt.flags & kFlagFirst) {
                 st.reset();
@@ -247,71 +401,40 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 warp_pv_16x16<D>(st, pa, v_tile, C::kHalfBytes, row0);
             }
 
-            const bool last = (mt.flags & kFlagLast) != 0;
             if (wrote_smem) fence_proxy_async_smem();   // generic writes before the next TMA fill
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty[s]);
 
-            if (last) {
-                // ---- merge the four warps' (m, l, O) and emit the item's result
+            if (mt.flags & kFlagLast) {
+                // ---- hand this piece's (max, sum, O) to the finisher warp and carry on
+                if (!mbar_wait(comb_empty, (n_dumps & 1u) ^ 1u, abort_flag)) break;
                 float l0 = st.l[0], l1 = st.l[1];
                 l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
                 l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
                 l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
                 l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
-                float *cw = comb + (size_t)warp * p.G * (D + 2);
+                float *cw = comb + (size_t)warp * p.G * kPitch;
                 if (r_lo < p.G) {
-                    float *row = cw + (size_t)r_lo * (D + 2);
+                    float *row = cw + (size_t)r_lo * kPitch;
                     if ((lane & 3) == 0) { row[D] = st.m[0]; row[D + 1] = l0; }
 #pragma unroll
-                    for (int nt = 0; nt < D / 8; ++nt) {
-                        row[nt * 8 + 2 * (lane & 3)] = st.o[nt][0];
-                        row[nt * 8 + 2 * (lane & 3) + 1] = st.o[nt][1];
-                    }
+                    for (int nt = 0; nt < D / 8; ++nt)
+                        *reinterpret_cast<float2 *>(row + nt * 8 + 2 * (lane & 3)) = make_float2(st.o[nt][0], st.o[nt][1]);
                 }
                 if (r_hi < p.G) {
-                    float *row = cw + (size_t)r_hi * (D + 2);
+                    float *row = cw + (size_t)r_hi * kPitch;
                     if ((lane & 3) == 0) { row[D] = st.m[1]; row[D + 1] = l1; }
 #pragma unroll
-                    for (int nt = 0; nt < D / 8; ++nt) {
-                        row[nt * 8 + 2 * (lane & 3)] = st.o[nt][2];
-                        row[nt * 8 + 2 * (lane & 3) + 1] = st.o[nt][3];
-                    }
+                    for (int nt = 0; nt < D / 8; ++nt)
+                        *reinterpret_cast<float2 *>(row + nt * 8 + 2 * (lane & 3)) = make_float2(st.o[nt][2], st.o[nt][3]);
+                }
+                if (warp == 0 && lane == 0) {
+                    piece_meta->b = mt.b; piece_meta->kvh = mt.kvh; piece_meta->piece = mt.piece;
+                    piece_meta->npieces = mt.npieces; piece_meta->stop = 0;
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&comb_bar[0]);
-                if (!mbar_wait(&comb_bar[0], item_par, abort_flag)) break;
-                for (int idx = ctid; idx < p.G * D; idx += kConsumerWarps * 32) {
-                    const int r = idx / D, d = idx % D;
-                    float mstar = -INFINITY;
-#pragma unroll
-                    for (int w = 0; w < kConsumerWarps; ++w)
-                        mstar = fmaxf(mstar, comb[((size_t)w * p.G + r) * (D + 2) + D]);
-                    float acc = 0.f, lsum = 0.f;
-#pragma unroll
-                    for (int w = 0; w < kConsumerWarps; ++w) {
-                        const float *row = comb + ((size_t)w * p.G + r) * (D + 2);
-                        const float wgt = fast_exp2(row[D] - mstar);   // idle warp: m = -inf -> 0
-                        acc += wgt * row[d];
-                        lsum += wgt * row[D + 1];
-                    }
-                    const float val = acc / lsum;
-                    const int head = mt.kvh * p.G + r;
-                    const size_t bh = (size_t)mt.b * p.Hq + head;
-                    const float lse2 = mstar + log2f(lsum);
-                    if (mt.nchunks == 1) {
-                        p.o[bh * D + d] = __float2bfloat16_rn(val);
-                        if (d == 0 && p.lse) p.lse[bh] = lse2 * 0.6931471805599453f;
-                    } else {
-                        const size_t slot = bh * p.nsplit + mt.chunk_idx;
-                        p.part_o[slot * D + d] = val;
-                        if (d == 0) p.part_lse[slot] = lse2;
-                    }
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&comb_bar[1]);
-                if (!mbar_wait(&comb_bar[1], item_par, abort_flag)) break;
-                item_par ^= 1u;
+                if (lane == 0) mbar_arrive(comb_full);
+                ++n_dumps;
             }
         }
     }
@@ -323,81 +446,62 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     }
 }
 
-// Pass 2: out[b,h,:] = sum_c w_c o_c / sum_c w_c with w_c = 2^(lse_c - max lse).
+// Resident CTAs per SM for a given dynamic shared-memory size (0 on failure).
 template <int D>
-__global__ void __launch_bounds__(D) decode_merge_kernel(const DecodeParams p)
+int decode_blocks_per_sm(size_t smem)
 {
-    const int h = blockIdx.x, b = blockIdx.y, d = threadIdx.x;
-    int len = p.kv_lens[b];
-    len = len < 0 ? 0 : len;
-    int n = (len + p.chunk - 1) / p.chunk;
-    n = n > p.nsplit ? p.nsplit : n;
-    if (n == 1) return;                       // finished by pass 1
-    const size_t bh = (size_t)b * p.Hq + h;
-    if (n == 0) {
-        p.o[bh * D + d] = __float2bfloat16_rn(0.f);
-        if (d == 0 && p.lse) p.lse[bh] = -INFINITY;
-        return;
+    static bool attr_set = false;
+    if (!attr_set) {
+        // the opt-in limit is per kernel: allow everything the SM has
+        if (cudaFuncSetAttribute(decode_split_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+            cudaSuccess)
+            return 0;
+        attr_set = true;
     }
-    const float *pl = p.part_lse + bh * p.nsplit;
-    const float *po = p.part_o + bh * p.nsplit * D;
-    float mstar = -INFINITY;
-    for (int c = 0; c < n; ++c) mstar = fmaxf(mstar, pl[c]);
-    float acc = 0.f, wsum = 0.f;
-    for (int c = 0; c < n; ++c) {
-        const float w = fast_exp2(pl[c] - mstar);
-        acc += w * po[(size_t)c * D + d];
-        wsum += w;
-    }
-    p.o[bh * D + d] = __float2bfloat16_rn(acc / wsum);
-    if (d == 0 && p.lse) p.lse[bh] = (mstar + log2f(wsum)) * 0.6931471805599453f;
-}
-
-template <int D>
-l4l_status launch_decode_t(const CUtensorMap &tk, const CUtensorMap &tv, const DecodeParams &p, int n_items_max,
-                           cudaStream_t stream)
-{
-    static int blocks_per_sm[17] = {0};
-    const size_t smem = decode_smem_bytes<D>(p.G);
-    if (blocks_per_sm[p.G] == 0) {
-        // the opt-in limit is per kernel: set it once to the largest group's need
-        if (cudaFuncSetAttribute(decode_split_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)decode_smem_bytes<D>(16)) != cudaSuccess)
-            return L4L_ERR_CUDA;
-        int n = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_split_kernel<D>, kThreads, smem) != cudaSuccess ||
-            n < 1)
-            return L4L_ERR_CUDA;
-        blocks_per_sm[p.G] = n;
-    }
-    int grid = sm_count() * blocks_per_sm[p.G];
-    if (grid > n_items_max) grid = n_items_max;
-    if (grid < 1) grid = 1;
-    decode_split_kernel<D><<<grid, kThreads, smem, stream>>>(tk, tv, p);
-    // always launched: it also covers kv_len == 0 (writes zeros); single-chunk sequences return at once
-    decode_merge_kernel<D><<<dim3(p.Hq, p.B), D, 0, stream>>>(p);
-    return cudaGetLastError() == cudaSuccess ? L4L_OK : L4L_ERR_CUDA;
+    if (smem > 227 * 1024) return 0;
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_split_kernel<D>, kThreads, smem) != cudaSuccess)
+        return 0;
+    return n;
 }
 
 }  // namespace
 
 DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_limit)
 {
-    // Largest chunk that still gives every CTA slot several items; then grown (fewer, larger
-    // partials) until the partials fit the workspace the caller provided.
-    const long long slots = 2ll * sm_count();
-    int chunk = 1024;
-    while (chunk > kTileT) {
-        const long long items = (long long)B * Hkv * ((max_kv_len + chunk - 1) / chunk);
-        if (items >= 8 * slots) break;
-        chunk >>= 1;
-    }
+    // Grid: every resident CTA slot of the device. A floor on the tiles per CTA bounds the number of
+    // pieces a sequence can be cut into (and with it the partials in the workspace and the finisher's
+    // scratch) when the real lengths are far below max_kv_len; it is raised until the partials fit the
+    // caller's workspace and the shared memory fits the SM.
     DecodePlan pl;
-    for (;; chunk <<= 1) {
-        pl.chunk = chunk;
-        pl.nsplit = max_kv_len > 0 ? (max_kv_len + chunk - 1) / chunk : 1;
-        pl.ws_bytes = kStatusBytes + (size_t)B * Hq * pl.nsplit * (D + 1) * sizeof(float);
-        if (pl.ws_bytes <= ws_limit || pl.nsplit == 1) break;
+    const int G = Hq / Hkv;
+    int n_dev = 0;
+    const bool have_dev = cudaGetDeviceCount(&n_dev) == cudaSuccess && n_dev > 0;
+    if (!have_dev) (void)cudaGetLastError();
+    auto blocks = [&](int nsplit) {
+        if (!have_dev) return 2;   // sizing without a device: assume the usual two CTAs per SM
+        return (D == 128) ? decode_blocks_per_sm<128>(decode_smem_bytes<128>(G, nsplit))
+                          : decode_blocks_per_sm<64>(decode_smem_bytes<64>(G, nsplit));
+    };
+    int per_sm = blocks(2);
+    if (per_sm < 1) per_sm = 1;
+    const long long slots = (long long)sm_count() * per_sm;
+    const long long tiles_max = max_kv_len > 0 ? (max_kv_len + kTileT - 1) / kTileT : 1;
+    const long long total_max = (long long)B * Hkv * tiles_max;
+    long long min_tiles = (total_max + 8 * slots - 1) / (8 * slots);
+    if (min_tiles < 1) min_tiles = 1;
+    for (;; min_tiles *= 2) {
+        // a sequence of n tiles meets at most ceil(n / tiles per CTA) + 1 CTAs, never more than it has tiles
+        long long nsplit = (tiles_max + min_tiles - 1) / min_tiles + 1;
+        if (nsplit > tiles_max) nsplit = tiles_max;
+        if (nsplit < 1) nsplit = 1;
+        pl.min_tiles = (int)min_tiles;
+        pl.nsplit = (int)nsplit;
+        pl.ws_bytes = kStatusBytes + (((size_t)B * Hkv * sizeof(int) + 255) / 256) * 256 +
+                      (size_t)B * Hq * pl.nsplit * (D + 1) * sizeof(float);
+        const int n = blocks(pl.nsplit);
+        pl.grid = sm_count() * (n > 0 ? n : 1);
+        if ((pl.ws_bytes <= ws_limit && n > 0) || min_tiles >= tiles_max) break;
     }
     return pl;
 }
@@ -406,47 +510,44 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
                          int max_kv_len, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
                          void *workspace, const DecodePlan &plan, cudaStream_t stream)
 {
-    CUtensorMap tk, tv;
-    TmapCoord coord, coord_v;
-    if (!make_tmap_bf16(&tk, &coord, cache.k, D, cache.max_len, Hkv, B, cache.stride_t, cache.stride_h,
-                        cache.stride_b, 64, kTileT) ||
-        !make_tmap_bf16(&tv, &coord_v, cache.v, D, cache.max_len, Hkv, B, cache.stride_t, cache.stride_h,
-                        cache.stride_b, 64, kTileT))
-        return L4L_ERR_CUDA;
-
+    const int G = Hq / Hkv;
+    const size_t smem = (D == 128) ? decode_smem_bytes<128>(G, plan.nsplit) : decode_smem_bytes<64>(G, plan.nsplit);
+    if (((D == 128) ? decode_blocks_per_sm<128>(smem) : decode_blocks_per_sm<64>(smem)) == 0) return L4L_ERR_CUDA;
     uint8_t *ws = static_cast<uint8_t *>(workspace);
+    int *tickets = reinterpret_cast<int *>(ws + kStatusBytes);
+    // partial outputs first: their float4 accesses need 16-byte alignment
+    float *part_o = reinterpret_cast<float *>(ws + kStatusBytes + (((size_t)B * Hkv * sizeof(int) + 255) / 256) * 256);
+    float *part_lse = part_o + (size_t)B * Hq * plan.nsplit * D;
+
     for (int b0 = 0; b0 < B; b0 += kMaxB) {
         const int nb = (B - b0 < kMaxB) ? (B - b0) : kMaxB;
+        CUtensorMap tk, tv;
+        TmapCoord coord, coord_v;
+        const __nv_bfloat16 *kb = static_cast<const __nv_bfloat16 *>(cache.k) + (size_t)b0 * cache.stride_b;
+        const __nv_bfloat16 *vb = static_cast<const __nv_bfloat16 *>(cache.v) + (size_t)b0 * cache.stride_b;
+        if (!make_tmap_bf16(&tk, &coord, kb, D, cache.max_len, Hkv, nb, cache.stride_t, cache.stride_h,
+                            cache.stride_b, 64, kTileT) ||
+            !make_tmap_bf16(&tv, &coord_v, vb, D, cache.max_len, Hkv, nb, cache.stride_t, cache.stride_h,
+                            cache.stride_b, 64, kTileT))
+            return L4L_ERR_CUDA;
         DecodeParams p;
         p.q = static_cast<const __nv_bfloat16 *>(q) + (size_t)b0 * Hq * D;
         p.o = static_cast<__nv_bfloat16 *>(o) + (size_t)b0 * Hq * D;
         p.lse = d_lse ? d_lse + (size_t)b0 * Hq : nullptr;
         p.kv_lens = d_kv_lens + b0;
-        p.part_o = reinterpret_cast<float *>(ws + kStatusBytes) + (size_t)b0 * Hq * plan.nsplit * D;
-        p.part_lse = reinterpret_cast<float *>(ws + kStatusBytes) + (size_t)B * Hq * plan.nsplit * D +
-                     (size_t)b0 * Hq * plan.nsplit;
+        p.part_o = part_o + (size_t)b0 * Hq * plan.nsplit * D;
+        p.part_lse = part_lse + (size_t)b0 * Hq * plan.nsplit;
+        p.tickets = tickets + (size_t)b0 * Hkv;
         p.status = reinterpret_cast<unsigned *>(ws);
-        p.B = nb; p.Hq = Hq; p.Hkv = Hkv; p.G = Hq / Hkv; p.chunk = plan.chunk; p.nsplit = plan.nsplit;
+        p.B = nb; p.Hq = Hq; p.Hkv = Hkv; p.G = G; p.min_tiles = plan.min_tiles; p.nsplit = plan.nsplit;
+        p.max_kv_len = max_kv_len;
         p.scale_log2e = scale * 1.4426950408889634f;
         p.coord = coord;
-        // batch slices address the cache through the tensor map: shift the batch coordinate
-        // by rebuilding the maps on the slice's base pointer
-        CUtensorMap tks = tk, tvs = tv;
-        if (b0 > 0) {
-            const __nv_bfloat16 *kb = static_cast<const __nv_bfloat16 *>(cache.k) + (size_t)b0 * cache.stride_b;
-            const __nv_bfloat16 *vb = static_cast<const __nv_bfloat16 *>(cache.v) + (size_t)b0 * cache.stride_b;
-            if (!make_tmap_bf16(&tks, &coord, kb, D, cache.max_len, Hkv, nb, cache.stride_t, cache.stride_h,
-                                cache.stride_b, 64, kTileT) ||
-                !make_tmap_bf16(&tvs, &coord_v, vb, D, cache.max_len, Hkv, nb, cache.stride_t, cache.stride_h,
-                                cache.stride_b, 64, kTileT))
-                return L4L_ERR_CUDA;
-            p.coord = coord;
-        }
-        const long long items = (long long)nb * Hkv * plan.nsplit;
-        const int n_items_max = items > (1ll << 30) ? (1 << 30) : (int)items;
-        l4l_status st = (D == 128) ? launch_decode_t<128>(tks, tvs, p, n_items_max, stream)
-                                   : launch_decode_t<64>(tks, tvs, p, n_items_max, stream);
-        if (st != L4L_OK) return st;
+        if (D == 128)
+            decode_split_kernel<128><<<plan.grid, kThreads, smem, stream>>>(tk, tv, p);
+        else
+            decode_split_kernel<64><<<plan.grid, kThreads, smem, stream>>>(tk, tv, p);
+        if (cudaGetLastError() != cudaSuccess) return L4L_ERR_CUDA;
     }
     return L4L_OK;
 }

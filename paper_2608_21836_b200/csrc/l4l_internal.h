@@ -25,9 +25,10 @@ bool make_tmap_bf16(CUtensorMap *out, TmapCoord *coord, const void *base, int D,
 int sm_count();
 
 struct DecodePlan {
-    int chunk;       // tokens per KV split (multiple of 64)
-    int nsplit;      // max splits per sequence = ceil(max_kv_len / chunk)
-    size_t ws_bytes; // status block + partials
+    int grid;        // persistent CTAs
+    int min_tiles;   // floor on the 64-token tiles per CTA (bounds the pieces per sequence)
+    int nsplit;      // max pieces a (sequence, KV head) can be cut into
+    size_t ws_bytes; // status block + ticket counters + partials
 };
 DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_limit);
 

@@ -78,7 +78,7 @@ def test_decode_many_splits_and_forced_large_chunks(D):
     q, ck, cv, kv_len = random_batch(2, 4, 1, D, 3072, lens, seed=7)
     o1, _ = check_decode(q, ck, cv, kv_len, 1.0 / math.sqrt(D))
     # a workspace too small for the preferred split: the library must grow the chunks, not fail
-    small = 256 + 2 * 4 * 3 * (D + 1) * 4
+    small = 256 + 256 + 2 * 4 * 3 * (D + 1) * 4
     o2, _ = check_decode(q, ck, cv, kv_len, 1.0 / math.sqrt(D), ws_bytes=small)
     # and an upper bound far above the real lengths is only a hint
     o3, _ = check_decode(q, ck, cv, torch.tensor([100, 77], dtype=torch.int32), 1.0 / math.sqrt(D))
