@@ -30,7 +30,7 @@ constexpr int kConsumerWarps = 4;
 constexpr int kProducerWarp = kConsumerWarps;
 constexpr int kFinisherWarp = kConsumerWarps + 1;
 constexpr int kThreads = (kConsumerWarps + 2) * 32;
-constexpr int kMaxB = 1024;                // sequences per launch (prefix sums live in shared memory)
+constexpr int kMaxB = 512;                 // sequences per launch (prefix sums live in shared memory)
 
 template <int D>
 struct DecodeCfg {
@@ -69,7 +69,8 @@ size_t decode_smem_bytes(int G, int nsplit)
 {
     using C = DecodeCfg<D>;
     size_t comb = (size_t)kConsumerWarps * G * (D + 4) * sizeof(float) + (size_t)((G * nsplit + 3) & ~3) * sizeof(float);
-    return 1024 /*alignment slack*/ + (size_t)C::kStages * C::kStageBytes + comb + C::kStages * sizeof(TileMeta) +
+    return 1024 /*alignment slack*/ + (size_t)C::kStages * (C::kStageBytes + (size_t)G * D * 2) + comb +
+           C::kStages * sizeof(TileMeta) +
            sizeof(PieceMeta) + (2 * C::kStages + 2) * sizeof(uint64_t) + (kMaxB + 1) * sizeof(int) + 64;
 }
 
@@ -91,7 +92,9 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     uint8_t *smem = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
 
     uint8_t *stages = smem;
-    float *comb = reinterpret_cast<float *>(stages + (size_t)C::kStages * C::kStageBytes);
+    uint8_t *q_slots = stages + (size_t)C::kStages * C::kStageBytes;     // per stage: the piece's G query rows
+    const uint32_t q_bytes = (uint32_t)p.G * D * 2;
+    float *comb = reinterpret_cast<float *>(q_slots + (size_t)C::kStages * q_bytes);
     constexpr int kPitch = D + 4;            // floats per row of `comb`: O[D], max, sum, pad (16-byte rows)
     constexpr int kVec = D / 4;
     const int comb_floats = kConsumerWarps * p.G * kPitch;
@@ -185,7 +188,12 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     mt.b = b; mt.kvh = kvh; mt.t0 = tile * kTileT; mt.piece = piece; mt.kv_len = len;
                     mt.npieces = npieces;
                     mt.flags = (tile == tile_begin ? kFlagFirst : 0) | (tile + 1 == tile_end ? kFlagLast : 0);
-                    mbar_arrive_expect_tx(&full[s], C::kStageBytes);
+                    // the first tile of a piece also brings the group's query rows (contiguous in q)
+                    const bool first = (tile == tile_begin);
+                    mbar_arrive_expect_tx(&full[s], C::kStageBytes + (first ? q_bytes : 0u));
+                    if (first)
+                        bulk_load_1d(q_slots + (size_t)s * q_bytes, p.q + ((size_t)b * p.Hq + (size_t)kvh * p.G) * D,
+                                     q_bytes, &full[s]);
                     uint8_t *dst = stages + (size_t)s * C::kStageBytes;
                     order_coords(p.coord, tile * kTileT, kvh, b, c1, c2, c3);
 #pragma unroll
@@ -275,6 +283,52 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             // second pass: out = sum_c w_c o_c / sum_c w_c with w_c = 2^(lse_c - max_c lse_c)
             const int np = pm.npieces;
             const size_t bh0 = (size_t)pm.b * p.Hq + pm.kvh * p.G;
+            if (np <= 4) {
+                // common case: all loads of a batch of outputs are issued before any is used (one round trip)
+                for (int base = 0; base < p.G * kVec; base += 2 * 32) {
+                    float4 v[2][4];
+                    float ls[2][4];
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        const int item = base + u * 32 + lane;
+                        const bool on = item < p.G * kVec;
+                        const int r = on ? item / kVec : 0, d4 = on ? item % kVec : 0;
+                        const float *pl = p.part_lse + (bh0 + r) * p.nsplit;
+                        const float4 *po = reinterpret_cast<const float4 *>(p.part_o + (bh0 + r) * p.nsplit * D) + d4;
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            const bool ld = on && c < np;
+                            ls[u][c] = ld ? __ldcg(pl + c) : -INFINITY;
+                            v[u][c] = ld ? __ldcg(po + (size_t)c * kVec) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        const int item = base + u * 32 + lane;
+                        if (item < p.G * kVec) {
+                            const int r = item / kVec, d4 = item % kVec;
+                            const float mstar = fmaxf(fmaxf(ls[u][0], ls[u][1]), fmaxf(ls[u][2], ls[u][3]));
+                            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                            float wsum = 0.f;
+#pragma unroll
+                            for (int c = 0; c < 4; ++c) {
+                                const float w = fast_exp2(ls[u][c] - mstar);       // absent piece: 2^-inf = 0
+                                acc.x += w * v[u][c].x; acc.y += w * v[u][c].y;
+                                acc.z += w * v[u][c].z; acc.w += w * v[u][c].w;
+                                wsum += w;
+                            }
+                            const float inv = 1.f / wsum;
+                            uint2 packed;
+                            packed.x = pack_bf16x2(acc.x * inv, acc.y * inv);
+                            packed.y = pack_bf16x2(acc.z * inv, acc.w * inv);
+                            *reinterpret_cast<uint2 *>(p.o + (bh0 + r) * D + d4 * 4) = packed;
+                            if (d4 == 0 && p.lse) p.lse[bh0 + r] = (mstar + log2f(wsum)) * 0.6931471805599453f;
+                        }
+                    }
+                }
+                __syncwarp();
+                continue;
+            }
             for (int idx = lane; idx < p.G * np; idx += 32) {
                 const int r = idx / np, c = idx % np;
                 merge_lse[r * p.nsplit + c] = __ldcg(p.part_lse + (bh0 + r) * p.nsplit + c);
@@ -349,17 +403,17 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
 
             if (mt.flags & kFlagFirst) {
                 st.reset();
-                const uint32_t *qrow_lo = reinterpret_cast<const uint32_t *>(
-                    p.q + ((size_t)mt.b * p.Hq + (size_t)mt.kvh * p.G + r_lo) * D);
-                const uint32_t *qrow_hi = qrow_lo + (size_t)8 * D / 2;
+                const uint32_t *qs = reinterpret_cast<const uint32_t *>(q_slots + (size_t)s * q_bytes);
+                const uint32_t *qrow_lo = qs + (size_t)r_lo * D / 2;
+                const uint32_t *qrow_hi = qs + (size_t)r_hi * D / 2;
                 const bool v_lo = r_lo < p.G, v_hi = r_hi < p.G;
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     const int w = ks * 8 + (lane & 3);               // 32-bit word index in the row
-                    qf[ks][0] = v_lo ? __ldg(qrow_lo + w) : 0u;
-                    qf[ks][1] = v_hi ? __ldg(qrow_hi + w) : 0u;
-                    qf[ks][2] = v_lo ? __ldg(qrow_lo + w + 4) : 0u;
-                    qf[ks][3] = v_hi ? __ldg(qrow_hi + w + 4) : 0u;
+                    qf[ks][0] = v_lo ? qrow_lo[w] : 0u;
+                    qf[ks][1] = v_hi ? qrow_hi[w] : 0u;
+                    qf[ks][2] = v_lo ? qrow_lo[w + 4] : 0u;
+                    qf[ks][3] = v_hi ? qrow_hi[w + 4] : 0u;
                 }
             }
 
