@@ -137,6 +137,43 @@ l4l_status l4l_attn_decode(const void *q, void *o, l4l_kv_cache cache,
                            int B, int Hq, int Hkv, int head_dim, float scale,
                            float *d_lse, void *workspace, size_t ws_bytes, l4l_stream stream);
 
+/*
+ * Decode for callers that cannot allocate device memory (no counterpart in the paper: it is the
+ * same operation as l4l_attn_decode, with the scratch moved inside the library).
+ *
+ * Who needs it: code that runs where cudaMalloc / cudaFree (or a framework allocator that may fall
+ * back to them) is off limits at the moment decode is needed. Typical cases are a serving loop whose
+ * memory plan is frozen after start-up because every spare byte of HBM already belongs to the KV
+ * pool, and a plug-in inside someone else's runtime, where an allocation would synchronise the
+ * device, stall the other streams and break the host's latency guarantees. Such callers have no
+ * workspace to hand over and no safe way to make one.
+ *
+ * What it does instead: the status block, the ticket counters and the fp32 partials live in a fixed
+ * array of L4L_STATIC_SCRATCH_BYTES inside the library's device image. Every GPU that loads the
+ * library carries that array until the process exits, whether or not this entry point is used. The
+ * call itself allocates nothing and frees nothing, through CUDA or any other library.
+ *
+ * Arguments, layouts, results and host-side validation are exactly those of l4l_attn_decode (inputs
+ * and outputs are still the caller's buffers); there is no workspace argument. Differences:
+ *   - Limit: the split of the KV axis is chosen so that its partials fit the fixed array. If even the
+ *     coarsest split needs more than L4L_STATIC_SCRATCH_BYTES (roughly B * Hq * (head_dim + 1) * 8
+ *     bytes plus 512), the call returns L4L_ERR_WORKSPACE and launches nothing; use l4l_attn_decode
+ *     with a workspace of your own for such sizes.
+ *   - First call on each device: the device address of the array is looked up (with that device
+ *     current) and remembered. Make this first call during start-up, before any stream capture.
+ *   - Shared state: all calls on a device use the same array, which keeps what the previous call left
+ *     in it; each call therefore clears the status block and the ticket counters on `stream` before its
+ *     kernel. Two calls that can overlap on the GPU (different streams, no ordering between them) race
+ *     on the array and give wrong results: order them, or give one of them a workspace.
+ *   - A bounded device-side wait that runs out is recorded in the array's status block, which this
+ *     entry point does not expose; callers that must observe it use l4l_attn_decode.
+ */
+#define L4L_STATIC_SCRATCH_BYTES (8u << 20)
+l4l_status l4l_attn_decode_static(const void *q, void *o, l4l_kv_cache cache,
+                                  const int32_t *d_kv_lens, int max_kv_len,
+                                  int B, int Hq, int Hkv, int head_dim, float scale,
+                                  float *d_lse, l4l_stream stream);
+
 /* Static, human-readable name of a status code. */
 const char *l4l_status_string(l4l_status status);
 

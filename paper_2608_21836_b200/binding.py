@@ -22,7 +22,9 @@ L4L_OP_PREFILL, L4L_OP_DECODE = 0, 1
 EXPORTS = (
     "l4l_version", "l4l_status_string", "l4l_workspace_bytes", "l4l_workspace_init",
     "l4l_last_device_error", "l4l_kv_append", "l4l_attn_prefill", "l4l_attn_decode",
+    "l4l_attn_decode_static",
 )
+STATIC_SCRATCH_BYTES = 8 << 20
 
 
 class Tensor4(ctypes.Structure):
@@ -71,6 +73,9 @@ def load() -> ctypes.CDLL:
     lib.l4l_attn_decode.restype = c_int
     lib.l4l_attn_decode.argtypes = [vp, vp, KVCache, i32p, c_int, c_int, c_int, c_int, c_int, ctypes.c_float, vp,
                                     vp, c_size, vp]
+    lib.l4l_attn_decode_static.restype = c_int
+    lib.l4l_attn_decode_static.argtypes = [vp, vp, KVCache, i32p, c_int, c_int, c_int, c_int, c_int, ctypes.c_float, vp,
+                                           vp]
     _lib = lib
     return lib
 
@@ -185,3 +190,25 @@ def l4l_attn_decode(q, o, cache_k, cache_v, kv_lens, max_kv_len: int, scale: flo
                                 workspace.numel() * workspace.element_size(), _stream())
     if st != L4L_OK:
         raise L4LError(st, "l4l_attn_decode")
+
+
+def l4l_attn_decode_static(q, o, cache_k, cache_v, kv_lens, max_kv_len: int, scale: float, lse=None) -> None:
+    """Decode for callers that may not allocate: same arguments as l4l_attn_decode but no workspace.
+
+    The scratch is a fixed array of STATIC_SCRATCH_BYTES inside the library, shared by every call on the
+    device, so calls that could overlap on the GPU must be ordered by the caller. Problems whose partials
+    do not fit raise L4LError(L4L_ERR_WORKSPACE). Make the first call on a device during start-up."""
+    _check_bf16_cuda(q, "q")
+    _check_bf16_cuda(o, "o")
+    if not (q.is_contiguous() and o.is_contiguous() and q.dim() == 3 and q.shape == o.shape):
+        raise ValueError("q and o must be dense [B, Hq, D]")
+    B, Hq, D = q.shape
+    Hkv = cache_k.shape[1]
+    if lse is not None and not (lse.is_cuda and lse.dtype == torch.float32 and lse.is_contiguous()
+                                and tuple(lse.shape) == (B, Hq)):
+        raise TypeError("lse must be a contiguous CUDA float32 tensor [B, Hq]")
+    st = load().l4l_attn_decode_static(q.data_ptr(), o.data_ptr(), kv_cache(cache_k, cache_v),
+                                       _i32_dev(kv_lens, "kv_lens"), int(max_kv_len), B, Hq, Hkv, D, float(scale),
+                                       None if lse is None else lse.data_ptr(), _stream())
+    if st != L4L_OK:
+        raise L4LError(st, "l4l_attn_decode_static")

@@ -18,6 +18,8 @@
 //                    normalised fp32 partial and its log-sum-exp go to the workspace, and the LAST
 //                    piece to arrive (a self-resetting ticket counter per (sequence, KV head)) runs
 //                    the second pass: the log-sum-exp merge of all pieces.
+#include <mutex>
+
 #include "l4l_internal.h"
 #include "l4l_warp_attn.cuh"
 
@@ -607,3 +609,75 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
 }
 
 }  // namespace l4l
+
+// =================================================================================================
+// Decode without a caller-provided workspace (and without any allocation).
+//
+// The scratch that l4l_attn_decode keeps in the caller's workspace (status block, ticket counters,
+// fp32 partials) lives here in a fixed array inside the library's device image. Host code cannot use
+// the array's name as a pointer: the name is only a handle on the host side, and a kernel handed it
+// would fault or scribble over unrelated memory. The device address is looked up once per device with
+// cudaGetSymbolAddress (that device being current) and passed to the very same launch path as the
+// workspace variant.
+namespace l4l {
+
+namespace {
+
+static __device__ __align__(256) unsigned char g_decode_static_scratch[L4L_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+void *g_static_scratch_addr[kMaxDevices] = {nullptr};
+std::mutex g_static_scratch_mutex;
+
+// Device address of the scratch array on the current device, or nullptr if the look-up fails.
+void *static_scratch_on_current_device()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+    if (g_static_scratch_addr[dev] == nullptr) {
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_decode_static_scratch) != cudaSuccess || ptr == nullptr) {
+            (void)cudaGetLastError();
+            return nullptr;
+        }
+        g_static_scratch_addr[dev] = ptr;
+    }
+    return g_static_scratch_addr[dev];
+}
+
+}  // namespace
+
+}  // namespace l4l
+
+extern "C" l4l_status l4l_attn_decode_static(const void *q, void *o, l4l_kv_cache cache, const int32_t *d_kv_lens,
+                                             int max_kv_len, int B, int Hq, int Hkv, int head_dim, float scale,
+                                             float *d_lse, l4l_stream stream)
+{
+    using namespace l4l;
+    if (B < 0 || Hq <= 0 || Hkv <= 0) return L4L_ERR_INVALID_ARG;
+    if (head_dim != 64 && head_dim != 128) return L4L_ERR_UNSUPPORTED;
+    if (Hq % Hkv != 0 || Hq / Hkv > 16) return L4L_ERR_UNSUPPORTED;
+    auto aligned16 = [](const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; };
+    auto stride_ok = [](int64_t s) { return s >= 0 && (s % 8) == 0; };
+    if (!q || !o || !d_kv_lens || !aligned16(q) || !aligned16(o)) return L4L_ERR_INVALID_ARG;
+    if (!cache.k || !cache.v || !aligned16(cache.k) || !aligned16(cache.v) || !stride_ok(cache.stride_b) ||
+        !stride_ok(cache.stride_h) || !stride_ok(cache.stride_t) || cache.max_len <= 0)
+        return L4L_ERR_INVALID_ARG;
+    if (max_kv_len < 0 || max_kv_len > cache.max_len) return L4L_ERR_INVALID_ARG;
+    if (B == 0) return L4L_OK;
+
+    // the split is chosen so that its partials fit the fixed array; if even the coarsest split does
+    // not fit, the problem is beyond this entry point
+    const DecodePlan plan = plan_decode(B, Hq, Hkv, head_dim, max_kv_len, (size_t)L4L_STATIC_SCRATCH_BYTES);
+    if (plan.ws_bytes > (size_t)L4L_STATIC_SCRATCH_BYTES) return L4L_ERR_WORKSPACE;
+
+    void *scratch = static_scratch_on_current_device();
+    if (!scratch) return L4L_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // the array keeps whatever the previous call left: the status block and the ticket counters must
+    // start at zero (the partials need no clearing, every slot is written before it is read)
+    const size_t zero_bytes = kStatusBytes + (((size_t)B * Hkv * sizeof(int) + 255) / 256) * 256;
+    if (cudaMemsetAsync(scratch, 0, zero_bytes, s) != cudaSuccess) return L4L_ERR_CUDA;
+    return launch_decode(q, o, cache, d_kv_lens, max_kv_len, B, Hq, Hkv, head_dim, scale, d_lse, scratch, plan, s);
+}
