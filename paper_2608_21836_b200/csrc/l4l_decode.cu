@@ -545,6 +545,11 @@ DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_
     const long long tiles_max = max_kv_len > 0 ? (max_kv_len + kTileT - 1) / kTileT : 1;
     const long long total_max = (long long)B * Hkv * tiles_max;
     long long min_tiles = (total_max + 8 * slots - 1) / (8 * slots);
+    // small problems are latency-bound: a CTA that streams only a tile or two spends longer in the
+    // merge of the many pieces than in the stream, so give every CTA at least 16 tiles (or a quarter
+    // of the longest sequence, if that is less)
+    const long long floor_tiles = (tiles_max + 3) / 4 < 16 ? (tiles_max + 3) / 4 : 16;
+    if (min_tiles < floor_tiles) min_tiles = floor_tiles;
     if (min_tiles < 1) min_tiles = 1;
     for (;; min_tiles *= 2) {
         // a sequence of n tiles meets at most ceil(n / tiles per CTA) + 1 CTAs, never more than it has tiles
