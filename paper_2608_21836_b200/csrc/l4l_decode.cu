@@ -124,14 +124,19 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
         fence_barrier_init();
         fence_proxy_async_smem();
     }
+    if (warp == kProducerWarp && lane == 0) {
+        tma_prefetch_desc(&tmap_k);
+        tma_prefetch_desc(&tmap_v);
+    }
+    // Programmatic dependent launch: everything above overlaps the tail of the previous kernel in the
+    // stream; nothing below (no global read or write) starts before that kernel has completed. The
+    // next kernel in the stream may begin its own prologue as soon as this grid's CTAs retire.
+    grid_dependency_wait();
+    grid_launch_dependents();
     __syncthreads();
 
     if (warp == kProducerWarp) {
         // ------------------------------------------------------------------ producer warp
-        if (lane == 0) {
-            tma_prefetch_desc(&tmap_k);
-            tma_prefetch_desc(&tmap_v);
-        }
         // exclusive prefix sum over sequences of (tiles * Hkv)
         int running = 0;
         for (int b0 = 0; b0 < p.B; b0 += 32) {
@@ -604,11 +609,19 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         p.max_kv_len = max_kv_len;
         p.scale_log2e = scale * 1.4426950408889634f;
         p.coord = coord;
-        if (D == 128)
-            decode_split_kernel<128><<<plan.grid, kThreads, smem, stream>>>(tk, tv, p);
-        else
-            decode_split_kernel<64><<<plan.grid, kThreads, smem, stream>>>(tk, tv, p);
-        if (cudaGetLastError() != cudaSuccess) return L4L_ERR_CUDA;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(plan.grid);
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        const cudaError_t err = (D == 128) ? cudaLaunchKernelEx(&cfg, decode_split_kernel<128>, tk, tv, p)
+                                           : cudaLaunchKernelEx(&cfg, decode_split_kernel<64>, tk, tv, p);
+        if (err != cudaSuccess) return L4L_ERR_CUDA;
     }
     return L4L_OK;
 }
