@@ -275,21 +275,75 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             if (lane == 0) mbar_arrive(comb_empty);        // `comb` has been consumed
             if (single) continue;
 
-            // ---- ticket: the last piece of this (sequence, KV head) to arrive merges all of them
-            __threadfence();                               // this warp's partials visible device-wide
-            __syncwarp();
-            int ticket = 0;
-            if (lane == 0) {
-                int *tk = p.tickets + (size_t)pm.b * p.Hkv + pm.kvh;
-                ticket = atomicAdd(tk, 1);
-                if (ticket == pm.npieces - 1) atomicExch(tk, 0);       // ready for the next call
-            }
-            ticket = __shfl_sync(0xffffffffu, ticket, 0);
-            if (ticket != pm.npieces - 1) continue;
-            __threadfence();
-            // second pass: out = sum_c w_c o_c / sum_c w_c with w_c = 2^(lse_c - max_c lse_c)
+            // ---- ticket: the last piece of this (sequence, KV head) to arrive merges all of them.
+            // The usual case at the end of a CTA's range is that every other piece arrived long ago. The
+            // counter is therefore read (acquire) before the fence; if it already shows all other pieces,
+            // their partials are loaded while this piece's own ticket is in flight, which takes one memory
+            // round trip off the tail (fence, then ticket and loads together, instead of three in a row).
             const int np = pm.npieces;
             const size_t bh0 = (size_t)pm.b * p.Hq + pm.kvh * p.G;
+            int *tk = p.tickets + (size_t)pm.b * p.Hkv + pm.kvh;
+            const bool small = (np <= 4) && (p.G * kVec <= 4 * 32);
+            int seen = 0;
+            if (small && lane == 0) seen = ld_acquire_gpu(tk);
+            __threadfence();                               // this warp's partials visible device-wide
+            seen = __shfl_sync(0xffffffffu, seen, 0);
+            const bool spec = small && (seen == np - 1);
+            float4 sv[4][4];
+            float sl[4][4];
+            auto load_pieces = [&]() {
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int item = u * 32 + lane;
+                    const bool on = item < p.G * kVec;
+                    const int r = on ? item / kVec : 0, d4 = on ? item % kVec : 0;
+                    const float *pl = p.part_lse + (bh0 + r) * p.nsplit;
+                    const float4 *po = reinterpret_cast<const float4 *>(p.part_o + (bh0 + r) * p.nsplit * D) + d4;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const bool ld = on && c < np;
+                        sl[u][c] = ld ? __ldcg(pl + c) : -INFINITY;
+                        sv[u][c] = ld ? __ldcg(po + (size_t)c * kVec) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                }
+            };
+            if (spec) load_pieces();
+            int ticket = 0;
+            if (lane == 0) {
+                ticket = atomicAdd(tk, 1);
+                if (ticket == np - 1) atomicExch(tk, 0);               // ready for the next call
+            }
+            ticket = __shfl_sync(0xffffffffu, ticket, 0);
+            if (ticket != np - 1) continue;
+            if (!spec) __threadfence();
+            if (small) {
+                if (!spec) load_pieces();
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int item = u * 32 + lane;
+                    if (item < p.G * kVec) {
+                        const int r = item / kVec, d4 = item % kVec;
+                        const float mstar = fmaxf(fmaxf(sl[u][0], sl[u][1]), fmaxf(sl[u][2], sl[u][3]));
+                        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                        float wsum = 0.f;
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            const float w = fast_exp2(sl[u][c] - mstar);           // absent piece: 2^-inf = 0
+                            acc.x += w * sv[u][c].x; acc.y += w * sv[u][c].y;
+                            acc.z += w * sv[u][c].z; acc.w += w * sv[u][c].w;
+                            wsum += w;
+                        }
+                        const float inv = 1.f / wsum;
+                        uint2 packed;
+                        packed.x = pack_bf16x2(acc.x * inv, acc.y * inv);
+                        packed.y = pack_bf16x2(acc.z * inv, acc.w * inv);
+                        *reinterpret_cast<uint2 *>(p.o + (bh0 + r) * D + d4 * 4) = packed;
+                        if (d4 == 0 && p.lse) p.lse[bh0 + r] = (mstar + log2f(wsum)) * 0.6931471805599453f;
+                    }
+                }
+                __syncwarp();
+                continue;
+            }
             if (np <= 4) {
                 // common case: all loads of a batch of outputs are issued before any is used (one round trip)
                 for (int base = 0; base < p.G * kVec; base += 2 * 32) {
