@@ -100,6 +100,22 @@ class ClockSampler(threading.Thread):
                 "samples": len(self.samples)}
 
 
+# ----------------------------------------------------------------------------------- multi-rank bookkeeping
+def max_over_ranks(values, world: int, device="cpu"):
+    """Every timing is the MAX over ranks (the job is as slow as its slowest replica). Works on any backend:
+    NCCL with CUDA tensors in the benchmark, gloo with CPU tensors in the tests."""
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def whole_job_value(world: int, step_flops: float, ms_per_step: float) -> float:
+    """Aggregate throughput of `world` replicas, each doing `step_flops` per step (weak scaling), in TFLOP/s."""
+    return world * step_flops / (ms_per_step * 1e-3) / 1e12
+
+
 # ----------------------------------------------------------------------------------- workload
 def make_inputs():
     wp, wd = wl.WORKLOADS["long_prefill"], wl.WORKLOADS["batched_decode"]
@@ -306,16 +322,14 @@ def run_ours(args, rank, world):
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
 
     # ---- max over ranks
-    times = torch.tensor([total_ms, e2e_ms, t_pre, t_dec, t_app, t_dec_b2b], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    total_ms, e2e_ms, t_pre, t_dec, t_app, t_dec_b2b = times.tolist()
+    total_ms, e2e_ms, t_pre, t_dec, t_app, t_dec_b2b = max_over_ranks(
+        [total_ms, e2e_ms, t_pre, t_dec, t_app, t_dec_b2b], world, dev)
     if rank != 0:
         return
 
     ms_per_step = total_ms / args.steps
     step_flops = pre_flops + dec_flops
-    value = world * step_flops / (ms_per_step * 1e-3) / 1e12
+    value = whole_job_value(world, step_flops, ms_per_step)
     peaks = measured_peaks()
     pre_tflops = pre_flops / (t_pre * 1e-3) / 1e12
     dec_gbs = dec_bytes / (t_dec_b2b * 1e-3) / 1e9          # average launch duration, back-to-back launches
@@ -345,7 +359,7 @@ def run_ours(args, rank, world):
         "roofline_decode": {"kernel": "decode_split", "bound": "hbm", "achieved": dec_gbs, "peak": peaks["hbm_gbs"],
                             "unit": "GB/s", "frac": dec_gbs / peaks["hbm_gbs"], "traffic": None,
                             "peak_source": peaks["source"] + " (device copy)"},
-        "e2e": {"value": world * step_flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+        "e2e": {"value": whole_job_value(world, step_flops, e2e_ms), "unit": "TFLOP/s", "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "gpu_launches": 3 * args.steps,
         "clocks": clocks,
