@@ -89,6 +89,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
 {
     using C = TcCfg<D>;
     // ---- which block: heaviest (longest causal span) blocks first, heads of a KV group adjacent
+    grid_dependency_wait();                       // seq_lens may have been written by the previous kernel
     const int per_block = p.Hq * p.B;
     const int qb = p.n_qblocks - 1 - (int)(blockIdx.x / per_block);
     const int hb = blockIdx.x % per_block;
@@ -118,6 +119,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     uint64_t *o_full = p_full + 2;                // [2]
     uint32_t *tmem_base_smem = reinterpret_cast<uint32_t *>(o_full + 2);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_base_smem + 1);
+    volatile int *copy_go = abort_flag + 1;       // producer -> helper warps: all loads issued
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -133,6 +135,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
             mbar_init(&o_full[i], 1);
         }
         *abort_flag = 0;
+        *copy_go = 0;
         fence_barrier_init();
         fence_proxy_async_smem();
     }
@@ -140,15 +143,43 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
         tmem_alloc(tmem_base_smem, C::kTmemCols);
         tmem_relinquish_alloc_permit();
     }
+    // Programmatic dependent launch: the set-up above may overlap the tail of the previous kernel of the
+    // stream; no global memory other than the kernel parameters is touched before it has completed.
+    grid_launch_dependents();
     tcgen05_fence_before_sync();
     __syncthreads();
     tcgen05_fence_after_sync();
     const uint32_t tmem_base = *tmem_base_smem;
 
+    // The block's diagonal K/V tiles (2*qb and 2*qb+1) go to the cache (first query head of a KV group
+    // only, so each row is written once). They are the last tiles loaded, so their ring slots are never
+    // refilled; the copy runs beside the last iterations, shared by three warps. Rows >= L are not written.
+    const bool writes_cache = p.cache_k != nullptr && (h % p.G) == 0;
+    auto copy_diagonal_tiles = [&](int part) {
+        if (!writes_cache) return;
+        const int lim = min(L, p.cache_max_len);
+        for (int j = 2 * qb; j < n_kv; ++j) {
+            for (int kv = 0; kv < 2; ++kv) {
+                const int idx = 2 * j + kv;
+                const uint32_t s = idx % C::kSlots, ph = (idx / C::kSlots) & 1u;
+                if (!mbar_wait(&kv_full[s], ph, abort_flag)) return;
+                const uint8_t *src = ring + (size_t)s * C::kTileBytes;
+                __nv_bfloat16 *dst_base = (kv ? p.cache_v : p.cache_k) + b * p.c_sb + kvh * p.c_sh;
+                constexpr int kChunks = D / 8;
+                const int rows = min(kRows, lim - j * kRows);
+                for (int i = part * 32 + lane; i < rows * kChunks; i += 96) {
+                    const int r = i / kChunks, ch = i % kChunks;
+                    const uint4 val = *reinterpret_cast<const uint4 *>(src + (ch >> 3) * kHalfBytes + swz128(r, ch & 7));
+                    *reinterpret_cast<uint4 *>(dst_base + (int64_t)(j * kRows + r) * p.c_st + ch * 8) = val;
+                }
+            }
+        }
+    };
+
     // Register reallocation: the data-movement warpgroup gives registers to the softmax warpgroups,
     // whose threads hold a whole 128-column score row.
     if (warp >= 8) {
-    setmaxnreg_dec<56>();
+    setmaxnreg_dec<64>();
     if (warp == 8) {
         // ============================================================ TMA producer (+ cache copy)
         if (lane == 0) {
@@ -175,28 +206,28 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
                     tma_load_4d(ring + (size_t)s * C::kTileBytes + hf * kHalfBytes, tm, &kv_full[s], hf * 64, c1, c2, c3);
             }
         }
+        // all loads are issued: the diagonal tiles' slots are in their last phase, the copy may start
+        if (lane == 0) {
+            __threadfence_block();
+            *copy_go = 1;
+        }
         __syncwarp();
-        if (p.cache_k != nullptr && (h % p.G) == 0) {
-            // the block's diagonal K/V tiles (2*qb and 2*qb+1) go to the cache; they are the last tiles
-            // loaded, so their slots are not refilled. Rows >= L are never written.
-            const int lim = min(L, p.cache_max_len);
-            for (int j = 2 * qb; j < n_kv; ++j) {
-                for (int kv = 0; kv < 2; ++kv) {
-                    const int idx = 2 * j + kv;
-                    const uint32_t s = idx % C::kSlots, ph = (idx / C::kSlots) & 1u;
-                    if (!mbar_wait(&kv_full[s], ph, abort_flag)) break;
-                    const uint8_t *src = ring + (size_t)s * C::kTileBytes;
-                    __nv_bfloat16 *dst_base = (kv ? p.cache_v : p.cache_k) + b * p.c_sb + kvh * p.c_sh;
-                    constexpr int kChunks = D / 8;
-                    const int rows = min(kRows, lim - j * kRows);
-                    for (int i = lane; i < rows * kChunks; i += 32) {
-                        const int r = i / kChunks, ch = i % kChunks;
-                        const uint4 val =
-                            *reinterpret_cast<const uint4 *>(src + (ch >> 3) * kHalfBytes + swz128(r, ch & 7));
-                        *reinterpret_cast<uint4 *>(dst_base + (int64_t)(j * kRows + r) * p.c_st + ch * 8) = val;
-                    }
-                }
+        copy_diagonal_tiles(0);
+    } else if (warp == 10 || warp == 11) {
+        // otherwise idle warps. First: if an earlier CTA of this launch already reported a dead wait, do
+        // not repeat its time-out in every remaining CTA. Then: help the producer warp copy the diagonal
+        // tiles to the cache.
+        if (warp == 10 && lane == 0 && *reinterpret_cast<volatile unsigned *>(p.status + kStatusErrWord) != 0u)
+            *abort_flag = 1;
+        if (writes_cache) {
+            const long long t0 = clock64();
+            bool go = true;
+            while (*copy_go == 0) {
+                if (*abort_flag || clock64() - t0 > kWaitCycleBudget) { go = false; break; }
+                __nanosleep(128);
             }
+            __threadfence_block();
+            if (go) copy_diagonal_tiles(warp - 9);
         }
     } else if (warp == 9) {
         // ============================================================ MMA issuer
@@ -276,7 +307,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
         }
     }
     } else {
-        setmaxnreg_inc<224>();
+        setmaxnreg_inc<216>();
         // ============================================================ softmax + epilogue warpgroups
         const int i = warp >> 2;                                   // sub-tile
         const int t = threadIdx.x & 127;                           // row within the sub-tile == TMEM lane
@@ -433,8 +464,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
         tmem_dealloc(tmem_base, C::kTmemCols);
     }
     if (threadIdx.x == 0 && *abort_flag) {
-        atomicOr(p.status + kStatusErrWord, kErrPrefillWait);
-        p.status[kStatusInfoWord] = 0x20000u | (blockIdx.x & 0xffffu);
+        if (atomicOr(p.status + kStatusErrWord, kErrPrefillWait) == 0u)
+            p.status[kStatusInfoWord] = 0x20000u | (blockIdx.x & 0xffffu);
     }
 }
 
@@ -452,8 +483,17 @@ l4l_status launch_t(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensor
     }
     const long long grid = (long long)p.n_qblocks * p.Hq * p.B;
     if (grid > 0x7fffffffll) return L4L_ERR_UNSUPPORTED;
-    prefill_tc_kernel<D><<<(unsigned)grid, kThreads, C::kSmemBytes, stream>>>(tq, tk, tv, p);
-    return cudaGetLastError() == cudaSuccess ? L4L_OK : L4L_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = C::kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, prefill_tc_kernel<D>, tq, tk, tv, p) == cudaSuccess ? L4L_OK : L4L_ERR_CUDA;
 }
 
 }  // namespace
