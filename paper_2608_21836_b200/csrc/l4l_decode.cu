@@ -32,6 +32,7 @@ constexpr int kConsumerWarps = 4;
 constexpr int kProducerWarp = kConsumerWarps;
 constexpr int kFinisherWarp = kConsumerWarps + 1;
 constexpr int kThreads = (kConsumerWarps + 2) * 32;
+constexpr int kPostRing = 16;               // pieces a producer can be ahead of its finisher (ring size)
 constexpr int kMaxB = 512;                 // sequences per launch (prefix sums live in shared memory)
 
 template <int D>
@@ -73,7 +74,8 @@ size_t decode_smem_bytes(int G, int nsplit)
     size_t comb = (size_t)kConsumerWarps * G * (D + 4) * sizeof(float) + (size_t)((G * nsplit + 3) & ~3) * sizeof(float);
     return 1024 /*alignment slack*/ + (size_t)C::kStages * (C::kStageBytes + (size_t)G * D * 2) + comb +
            C::kStages * sizeof(TileMeta) +
-           sizeof(PieceMeta) + (2 * C::kStages + 2) * sizeof(uint64_t) + (kMaxB + 1) * sizeof(int) + 64;
+           sizeof(PieceMeta) + (2 * C::kStages + 2) * sizeof(uint64_t) + (kMaxB + 1) * sizeof(int) + 64 +
+           kPostRing * sizeof(PieceMeta);
 }
 
 __device__ __forceinline__ void order_coords(const TmapCoord &c, int t, int h, int b, int &c1, int &c2, int &c3)
@@ -109,6 +111,10 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     uint64_t *comb_empty = comb_full + 1;       // finisher -> consumers: `comb` may be overwritten
     int *cum = reinterpret_cast<int *>(comb_empty + 1);   // cum[b] = tiles of sequences < b (times Hkv)
     volatile int *abort_flag = cum + (kMaxB + 1);
+    // producer -> finisher: the pieces this CTA has started, in order (so that the finisher can look at a
+    // piece's ticket while the piece is still being streamed)
+    volatile uint32_t *posted_count = reinterpret_cast<volatile uint32_t *>(abort_flag + 1);
+    PieceMeta *post_ring = reinterpret_cast<PieceMeta *>(cum + (kMaxB + 1) + 4);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -121,6 +127,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
         mbar_init(comb_full, kConsumerWarps);
         mbar_init(comb_empty, 1);
         *abort_flag = 0;
+        *posted_count = 0u;
         fence_barrier_init();
         fence_proxy_async_smem();
     }
@@ -165,7 +172,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             per_cta = per_cta < p.min_tiles ? p.min_tiles : per_cta;
             const int my_begin = min(total, (int)blockIdx.x * per_cta);
             const int my_end = min(total, my_begin + per_cta);
-            uint32_t it = 0;
+            uint32_t it = 0, n_posted = 0;
             bool ok = true;
             int g = my_begin;
             while (ok && g < my_end) {
@@ -186,6 +193,12 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 const int first_cta = seq_first / per_cta;
                 const int npieces = (seq_first + tiles_b - 1) / per_cta - first_cta + 1;
                 const int piece = (int)blockIdx.x - first_cta;
+                {
+                    PieceMeta &pp = post_ring[n_posted % kPostRing];
+                    pp.b = b; pp.kvh = kvh; pp.piece = piece; pp.npieces = npieces; pp.stop = 0;
+                    __threadfence_block();
+                    *posted_count = ++n_posted;
+                }
                 int c1, c2, c3;
                 for (int tile = tile_begin; tile < tile_end; ++tile, ++it) {
                     const uint32_t s = it % C::kStages;
@@ -230,11 +243,128 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     for (int i = lane; i < p.Hq; i += 32) p.lse[(size_t)b * p.Hq + i] = -INFINITY;
             }
         }
+        const bool few_items = (p.G * kVec <= 4 * 32);     // each lane owns at most four float4 outputs of a piece
         for (uint32_t n = 0;; ++n) {
-            if (!mbar_wait(comb_full, n & 1u, abort_flag)) break;
+            // ---- While the consumers are still streaming piece n: if every other piece of its sequence has
+            // already arrived (the usual case for the piece a CTA ends with), fetch their partials now, so
+            // that nothing but the local merge is left when the piece completes.
+            float4 sv[4][4];
+            float sl[4][4];
+            bool prefetched = false;
+            {
+                // every decision in this loop is taken by lane 0 and broadcast, so that the warp stays converged
+                const long long t0 = clock64();
+                bool have_post = false, dead = false;
+                while (true) {
+                    int st = 0;                                       // 0: keep polling
+                    if (lane == 0) {
+                        if (mbar_try_wait(comb_full, n & 1u)) st = 1;                                  // piece complete
+                        else if (*abort_flag || clock64() - t0 > kWaitCycleBudget) st = 3;             // give up
+                        else if (!have_post && (int32_t)(*posted_count - (n + 1u)) >= 0) st = 2;       // piece started
+                    }
+                    st = __shfl_sync(0xffffffffu, st, 0);
+                    if (st == 1) break;
+                    if (st == 3) { dead = true; break; }
+                    if (st == 2) {
+                        have_post = true;
+                        __threadfence_block();
+                        const PieceMeta pp = post_ring[n % kPostRing];
+                        if (few_items && pp.npieces > 1 && pp.npieces <= 4) {
+                            int *tk = p.tickets + (size_t)pp.b * p.Hkv + pp.kvh;
+                            int seen = (lane == 0) ? ld_acquire_gpu(tk) : 0;
+                            seen = __shfl_sync(0xffffffffu, seen, 0);
+                            if (seen == pp.npieces - 1) {
+                                const size_t bh0 = (size_t)pp.b * p.Hq + pp.kvh * p.G;
+#pragma unroll
+                                for (int u = 0; u < 4; ++u) {
+                                    const int item = u * 32 + lane;
+                                    const bool on = item < p.G * kVec;
+                                    const int r = on ? item / kVec : 0, d4 = on ? item % kVec : 0;
+                                    const float *pl = p.part_lse + (bh0 + r) * p.nsplit;
+                                    const float4 *po =
+                                        reinterpret_cast<const float4 *>(p.part_o + (bh0 + r) * p.nsplit * D) + d4;
+#pragma unroll
+                                    for (int c = 0; c < 4; ++c) {
+                                        const bool ld = on && c < pp.npieces && c != pp.piece;
+                                        sl[u][c] = ld ? __ldcg(pl + c) : -INFINITY;
+                                        sv[u][c] = ld ? __ldcg(po + (size_t)c * kVec) : make_float4(0.f, 0.f, 0.f, 0.f);
+                                    }
+                                }
+                                prefetched = true;
+                            }
+                        }
+                    } else {
+                        __nanosleep(64);
+                    }
+                }
+                if (dead) {
+                    *abort_flag = 1;
+                    break;
+                }
+                __syncwarp();                                         // lane 0's acquire covers the warp
+            }
             const PieceMeta pm = *piece_meta;
             if (pm.stop) break;
             const bool single = (pm.npieces == 1);
+            const size_t bh0 = (size_t)pm.b * p.Hq + pm.kvh * p.G;
+            int *tk = p.tickets + (size_t)pm.b * p.Hkv + pm.kvh;
+            const int np = pm.npieces;
+
+            if (prefetched) {
+                // ---- this piece completes its sequence: merge the four warps' results, fold in the other
+                // pieces' partials fetched above, write the final output; nothing goes through the workspace
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int item = u * 32 + lane;
+                    if (item < p.G * kVec) {
+                        const int r = item / kVec, d4 = item % kVec;
+                        float mw[kConsumerWarps];
+                        float mloc = -INFINITY;
+#pragma unroll
+                        for (int w = 0; w < kConsumerWarps; ++w) {
+                            mw[w] = comb[((size_t)w * p.G + r) * kPitch + D];
+                            mloc = fmaxf(mloc, mw[w]);
+                        }
+                        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                        float lsum = 0.f;
+#pragma unroll
+                        for (int w = 0; w < kConsumerWarps; ++w) {
+                            const float *row = comb + ((size_t)w * p.G + r) * kPitch;
+                            const float wgt = fast_exp2(mw[w] - mloc);
+                            const float4 v = *reinterpret_cast<const float4 *>(row + d4 * 4);
+                            acc.x += wgt * v.x; acc.y += wgt * v.y; acc.z += wgt * v.z; acc.w += wgt * v.w;
+                            lsum += wgt * row[D + 1];
+                        }
+                        // own piece in the same form as the stored partials: normalised output + log2-sum-exp
+                        const float inv_own = 1.f / lsum;
+                        const float lse_own = mloc + log2f(lsum);
+                        float mstar = fmaxf(lse_own, fmaxf(fmaxf(sl[u][0], sl[u][1]), fmaxf(sl[u][2], sl[u][3])));
+                        const float w_own = fast_exp2(lse_own - mstar) * inv_own;
+                        float4 out = make_float4(acc.x * w_own, acc.y * w_own, acc.z * w_own, acc.w * w_own);
+                        float wsum = fast_exp2(lse_own - mstar);
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            const float wc = fast_exp2(sl[u][c] - mstar);          // absent piece: 2^-inf = 0
+                            out.x += wc * sv[u][c].x; out.y += wc * sv[u][c].y;
+                            out.z += wc * sv[u][c].z; out.w += wc * sv[u][c].w;
+                            wsum += wc;
+                        }
+                        const float inv = 1.f / wsum;
+                        uint2 packed;
+                        packed.x = pack_bf16x2(out.x * inv, out.y * inv);
+                        packed.y = pack_bf16x2(out.z * inv, out.w * inv);
+                        *reinterpret_cast<uint2 *>(p.o + (bh0 + r) * D + d4 * 4) = packed;
+                        if (d4 == 0 && p.lse) p.lse[bh0 + r] = (mstar + log2f(wsum)) * 0.6931471805599453f;
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(comb_empty);                // `comb` has been consumed
+                    atomicExch(tk, 0);                      // every piece is accounted for: ready for the next call
+                }
+                continue;
+            }
+
             // merge the four consumer warps' (max, sum, O); each lane owns float4 pieces of the G x D outputs
             for (int item = lane; item < p.G * kVec; item += 32) {
                 const int r = item / kVec, d4 = item % kVec;
@@ -257,7 +387,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 }
                 const float inv = 1.f / lsum;
                 acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
-                const size_t bh = (size_t)pm.b * p.Hq + pm.kvh * p.G + r;
+                const size_t bh = bh0 + r;
                 const float lse2 = mstar + log2f(lsum);
                 if (single) {
                     uint2 packed;
@@ -276,21 +406,15 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             if (single) continue;
 
             // ---- ticket: the last piece of this (sequence, KV head) to arrive merges all of them.
-            // The usual case at the end of a CTA's range is that every other piece arrived long ago. The
-            // counter is therefore read (acquire) before the fence; if it already shows all other pieces,
-            // their partials are loaded while this piece's own ticket is in flight, which takes one memory
-            // round trip off the tail (fence, then ticket and loads together, instead of three in a row).
-            const int np = pm.npieces;
-            const size_t bh0 = (size_t)pm.b * p.Hq + pm.kvh * p.G;
-            int *tk = p.tickets + (size_t)pm.b * p.Hkv + pm.kvh;
-            const bool small = (np <= 4) && (p.G * kVec <= 4 * 32);
+            // The counter is read (acquire) before the fence; if it already shows every other piece, their
+            // partials are loaded while this piece's own ticket is in flight (fence, then ticket and loads
+            // together: two memory round trips instead of three).
+            const bool small = few_items && np <= 4;
             int seen = 0;
             if (small && lane == 0) seen = ld_acquire_gpu(tk);
             __threadfence();                               // this warp's partials visible device-wide
             seen = __shfl_sync(0xffffffffu, seen, 0);
             const bool spec = small && (seen == np - 1);
-            float4 sv[4][4];
-            float sl[4][4];
             auto load_pieces = [&]() {
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
@@ -344,52 +468,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 __syncwarp();
                 continue;
             }
-            if (np <= 4) {
-                // common case: all loads of a batch of outputs are issued before any is used (one round trip)
-                for (int base = 0; base < p.G * kVec; base += 2 * 32) {
-                    float4 v[2][4];
-                    float ls[2][4];
-#pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        const int item = base + u * 32 + lane;
-                        const bool on = item < p.G * kVec;
-                        const int r = on ? item / kVec : 0, d4 = on ? item % kVec : 0;
-                        const float *pl = p.part_lse + (bh0 + r) * p.nsplit;
-                        const float4 *po = reinterpret_cast<const float4 *>(p.part_o + (bh0 + r) * p.nsplit * D) + d4;
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            const bool ld = on && c < np;
-                            ls[u][c] = ld ? __ldcg(pl + c) : -INFINITY;
-                            v[u][c] = ld ? __ldcg(po + (size_t)c * kVec) : make_float4(0.f, 0.f, 0.f, 0.f);
-                        }
-                    }
-#pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        const int item = base + u * 32 + lane;
-                        if (item < p.G * kVec) {
-                            const int r = item / kVec, d4 = item % kVec;
-                            const float mstar = fmaxf(fmaxf(ls[u][0], ls[u][1]), fmaxf(ls[u][2], ls[u][3]));
-                            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                            float wsum = 0.f;
-#pragma unroll
-                            for (int c = 0; c < 4; ++c) {
-                                const float w = fast_exp2(ls[u][c] - mstar);       // absent piece: 2^-inf = 0
-                                acc.x += w * v[u][c].x; acc.y += w * v[u][c].y;
-                                acc.z += w * v[u][c].z; acc.w += w * v[u][c].w;
-                                wsum += w;
-                            }
-                            const float inv = 1.f / wsum;
-                            uint2 packed;
-                            packed.x = pack_bf16x2(acc.x * inv, acc.y * inv);
-                            packed.y = pack_bf16x2(acc.z * inv, acc.w * inv);
-                            *reinterpret_cast<uint2 *>(p.o + (bh0 + r) * D + d4 * 4) = packed;
-                            if (d4 == 0 && p.lse) p.lse[bh0 + r] = (mstar + log2f(wsum)) * 0.6931471805599453f;
-                        }
-                    }
-                }
-                __syncwarp();
-                continue;
-            }
+            // second pass: out = sum_c w_c o_c / sum_c w_c with w_c = 2^(lse_c - max_c lse_c)
             for (int idx = lane; idx < p.G * np; idx += 32) {
                 const int r = idx / np, c = idx % np;
                 merge_lse[r * p.nsplit + c] = __ldcg(p.part_lse + (bh0 + r) * p.nsplit + c);
