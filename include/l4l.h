@@ -157,7 +157,7 @@ l4l_status l4l_attn_decode(const void *q, void *o, l4l_kv_cache cache,
  * and outputs are still the caller's buffers); there is no workspace argument. Differences:
  *   - Limit: the split of the KV axis is chosen so that its partials fit the fixed array. If even the
  *     coarsest split needs more than L4L_STATIC_SCRATCH_BYTES (roughly B * Hq * (head_dim + 1) * 8
- *     bytes plus 512), the call returns L4L_ERR_WORKSPACE and launches nothing; use l4l_attn_decode
+ *     bytes plus 128 KiB of counters), the call returns L4L_ERR_WORKSPACE and launches nothing; use l4l_attn_decode
  *     with a workspace of your own for such sizes.
  *   - First call on each device: the device address of the array is looked up (with that device
  *     current) and remembered. Make this first call during start-up, before any stream capture.

@@ -33,6 +33,10 @@ constexpr int kProducerWarp = kConsumerWarps;
 constexpr int kFinisherWarp = kConsumerWarps + 1;
 constexpr int kThreads = (kConsumerWarps + 2) * 32;
 constexpr int kPostRing = 16;               // pieces a producer can be ahead of its finisher (ring size)
+// The ticket counters sit at a FIXED place and size in the workspace (right after the status block), so
+// that calls of different shapes on one workspace can never write partials over counters another call
+// relies on being zero.
+constexpr size_t kTicketBytes = 128 * 1024;  // 32768 (sequence, KV head) pairs per launch
 constexpr int kMaxB = 512;                 // sequences per launch (prefix sums live in shared memory)
 
 template <int D>
@@ -88,6 +92,7 @@ __device__ __forceinline__ void order_coords(const TmapCoord &c, int t, int h, i
 template <int D>
 __global__ void __launch_bounds__(kThreads)
 decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
+                    const __grid_constant__ CUtensorMap tmap_k16, const __grid_constant__ CUtensorMap tmap_v16,
                     const DecodeParams p)
 {
     using C = DecodeCfg<D>;
@@ -134,6 +139,8 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     if (warp == kProducerWarp && lane == 0) {
         tma_prefetch_desc(&tmap_k);
         tma_prefetch_desc(&tmap_v);
+        tma_prefetch_desc(&tmap_k16);
+        tma_prefetch_desc(&tmap_v16);
     }
     // Programmatic dependent launch: everything above overlaps the tail of the previous kernel in the
     // stream; nothing below (no global read or write) starts before that kernel has completed. The
@@ -210,16 +217,33 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     mt.flags = (tile == tile_begin ? kFlagFirst : 0) | (tile + 1 == tile_end ? kFlagLast : 0);
                     // the first tile of a piece also brings the group's query rows (contiguous in q)
                     const bool first = (tile == tile_begin);
-                    mbar_arrive_expect_tx(&full[s], C::kStageBytes + (first ? q_bytes : 0u));
+                    // the last tile of a sequence is fetched in 16-token groups, so that (almost) nothing past
+                    // the end of the sequence is read; rows not fetched are never looked at by the consumers
+                    const int rem = len - tile * kTileT;
+                    const int groups = rem >= kTileT ? kTileT / 16 : (rem + 15) / 16;
+                    const uint32_t kv_bytes = rem >= kTileT ? C::kStageBytes : (uint32_t)groups * 16u * 128u * C::kHalves * 2u;
+                    mbar_arrive_expect_tx(&full[s], kv_bytes + (first ? q_bytes : 0u));
                     if (first)
                         bulk_load_1d(q_slots + (size_t)s * q_bytes, p.q + ((size_t)b * p.Hq + (size_t)kvh * p.G) * D,
                                      q_bytes, &full[s]);
                     uint8_t *dst = stages + (size_t)s * C::kStageBytes;
-                    order_coords(p.coord, tile * kTileT, kvh, b, c1, c2, c3);
+                    if (rem >= kTileT) {
+                        order_coords(p.coord, tile * kTileT, kvh, b, c1, c2, c3);
 #pragma unroll
-                    for (int hf = 0; hf < C::kHalves; ++hf) {
-                        tma_load_4d(dst + hf * C::kHalfBytes, &tmap_k, &full[s], hf * 64, c1, c2, c3);
-                        tma_load_4d(dst + C::kTileBytes + hf * C::kHalfBytes, &tmap_v, &full[s], hf * 64, c1, c2, c3);
+                        for (int hf = 0; hf < C::kHalves; ++hf) {
+                            tma_load_4d(dst + hf * C::kHalfBytes, &tmap_k, &full[s], hf * 64, c1, c2, c3);
+                            tma_load_4d(dst + C::kTileBytes + hf * C::kHalfBytes, &tmap_v, &full[s], hf * 64, c1, c2, c3);
+                        }
+                    } else {
+                        for (int gq = 0; gq < groups; ++gq) {
+                            order_coords(p.coord, tile * kTileT + gq * 16, kvh, b, c1, c2, c3);
+                            uint8_t *dg = dst + gq * 16 * 128;        // 2 KB per group: the swizzle phase is kept
+#pragma unroll
+                            for (int hf = 0; hf < C::kHalves; ++hf) {
+                                tma_load_4d(dg + hf * C::kHalfBytes, &tmap_k16, &full[s], hf * 64, c1, c2, c3);
+                                tma_load_4d(dg + C::kTileBytes + hf * C::kHalfBytes, &tmap_v16, &full[s], hf * 64, c1, c2, c3);
+                            }
+                        }
                     }
                 }
                 g = seq_first + tile_end;
@@ -696,7 +720,7 @@ DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_
         if (nsplit < 1) nsplit = 1;
         pl.min_tiles = (int)min_tiles;
         pl.nsplit = (int)nsplit;
-        pl.ws_bytes = kStatusBytes + (((size_t)B * Hkv * sizeof(int) + 255) / 256) * 256 +
+        pl.ws_bytes = kStatusBytes + kTicketBytes +
                       (size_t)B * Hq * pl.nsplit * (D + 1) * sizeof(float);
         const int n = blocks(pl.nsplit);
         pl.grid = sm_count() * (n > 0 ? n : 1);
@@ -715,19 +739,27 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
     uint8_t *ws = static_cast<uint8_t *>(workspace);
     int *tickets = reinterpret_cast<int *>(ws + kStatusBytes);
     // partial outputs first: their float4 accesses need 16-byte alignment
-    float *part_o = reinterpret_cast<float *>(ws + kStatusBytes + (((size_t)B * Hkv * sizeof(int) + 255) / 256) * 256);
+    float *part_o = reinterpret_cast<float *>(ws + kStatusBytes + kTicketBytes);
     float *part_lse = part_o + (size_t)B * Hq * plan.nsplit * D;
 
-    for (int b0 = 0; b0 < B; b0 += kMaxB) {
-        const int nb = (B - b0 < kMaxB) ? (B - b0) : kMaxB;
-        CUtensorMap tk, tv;
+    // sequences per launch: bounded by the prefix-sum array in shared memory and by the ticket region
+    int slice = (int)(kTicketBytes / sizeof(int)) / Hkv;
+    if (slice > kMaxB) slice = kMaxB;
+    if (slice < 1) return L4L_ERR_UNSUPPORTED;
+    for (int b0 = 0; b0 < B; b0 += slice) {
+        const int nb = (B - b0 < slice) ? (B - b0) : slice;
+        CUtensorMap tk, tv, tk16, tv16;   // 64-token boxes, and 16-token boxes for the last tile of a sequence
         TmapCoord coord, coord_v;
         const __nv_bfloat16 *kb = static_cast<const __nv_bfloat16 *>(cache.k) + (size_t)b0 * cache.stride_b;
         const __nv_bfloat16 *vb = static_cast<const __nv_bfloat16 *>(cache.v) + (size_t)b0 * cache.stride_b;
         if (!make_tmap_bf16(&tk, &coord, kb, D, cache.max_len, Hkv, nb, cache.stride_t, cache.stride_h,
                             cache.stride_b, 64, kTileT) ||
             !make_tmap_bf16(&tv, &coord_v, vb, D, cache.max_len, Hkv, nb, cache.stride_t, cache.stride_h,
-                            cache.stride_b, 64, kTileT))
+                            cache.stride_b, 64, kTileT) ||
+            !make_tmap_bf16(&tk16, &coord_v, kb, D, cache.max_len, Hkv, nb, cache.stride_t, cache.stride_h,
+                            cache.stride_b, 64, 16) ||
+            !make_tmap_bf16(&tv16, &coord_v, vb, D, cache.max_len, Hkv, nb, cache.stride_t, cache.stride_h,
+                            cache.stride_b, 64, 16))
             return L4L_ERR_CUDA;
         DecodeParams p;
         p.q = static_cast<const __nv_bfloat16 *>(q) + (size_t)b0 * Hq * D;
@@ -736,7 +768,7 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         p.kv_lens = d_kv_lens + b0;
         p.part_o = part_o + (size_t)b0 * Hq * plan.nsplit * D;
         p.part_lse = part_lse + (size_t)b0 * Hq * plan.nsplit;
-        p.tickets = tickets + (size_t)b0 * Hkv;
+        p.tickets = tickets;                       // every launch leaves them at zero for the next
         p.status = reinterpret_cast<unsigned *>(ws);
         p.B = nb; p.Hq = Hq; p.Hkv = Hkv; p.G = G; p.min_tiles = plan.min_tiles; p.nsplit = plan.nsplit;
         p.max_kv_len = max_kv_len;
@@ -752,8 +784,8 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        const cudaError_t err = (D == 128) ? cudaLaunchKernelEx(&cfg, decode_split_kernel<128>, tk, tv, p)
-                                           : cudaLaunchKernelEx(&cfg, decode_split_kernel<64>, tk, tv, p);
+        const cudaError_t err = (D == 128) ? cudaLaunchKernelEx(&cfg, decode_split_kernel<128>, tk, tv, tk16, tv16, p)
+                                           : cudaLaunchKernelEx(&cfg, decode_split_kernel<64>, tk, tv, tk16, tv16, p);
         if (err != cudaSuccess) return L4L_ERR_CUDA;
     }
     return L4L_OK;
@@ -828,7 +860,7 @@ extern "C" l4l_status l4l_attn_decode_static(const void *q, void *o, l4l_kv_cach
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // the array keeps whatever the previous call left: the status block and the ticket counters must
     // start at zero (the partials need no clearing, every slot is written before it is read)
-    const size_t zero_bytes = kStatusBytes + (((size_t)B * Hkv * sizeof(int) + 255) / 256) * 256;
+    const size_t zero_bytes = kStatusBytes + kTicketBytes;
     if (cudaMemsetAsync(scratch, 0, zero_bytes, s) != cudaSuccess) return L4L_ERR_CUDA;
     return launch_decode(q, o, cache, d_kv_lens, max_kv_len, B, Hq, Hkv, head_dim, scale, d_lse, scratch, plan, s);
 }

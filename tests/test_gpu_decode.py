@@ -78,7 +78,7 @@ def test_decode_many_splits_and_forced_large_chunks(D):
     q, ck, cv, kv_len = random_batch(2, 4, 1, D, 3072, lens, seed=7)
     o1, _ = check_decode(q, ck, cv, kv_len, 1.0 / math.sqrt(D))
     # a workspace too small for the preferred split: the library must grow the chunks, not fail
-    small = 256 + 256 + 2 * 4 * 3 * (D + 1) * 4
+    small = 256 + 128 * 1024 + 2 * 4 * 3 * (D + 1) * 4
     o2, _ = check_decode(q, ck, cv, kv_len, 1.0 / math.sqrt(D), ws_bytes=small)
     # and an upper bound far above the real lengths is only a hint
     o3, _ = check_decode(q, ck, cv, torch.tensor([100, 77], dtype=torch.int32), 1.0 / math.sqrt(D))
@@ -159,3 +159,28 @@ def test_config_append_then_decode_steps_equal_prefill_rows(name):
     ref, _ = orc.prefill_rows(seq.q, seq.k, seq.v, np.full(B, S + T, np.int32), w.scale, rows)
     got = torch.stack([outs[b, t, h] for b in range(B) for t in steps for h in range(Hq)])
     assert_close_to_oracle(got, ref, f"{name} decode steps")
+
+
+def test_decode_repeated_calls_on_one_workspace_stay_correct():
+    """The ticket counters and partials live in the workspace across calls: alternate two different
+    batches many times on ONE workspace (every merge path: sequences cut in 2, 3 and more pieces) and
+    check each result against the oracle's."""
+    D, Hq, Hkv, Lmax = 128, 32, 8, 4096
+    rng = np.random.default_rng(77)
+    batches = []
+    for seed, B in ((1, 32), (2, 24)):
+        lens = rng.integers(512, 4097, B).tolist()
+        lens[0], lens[1] = 4096, 1                      # the longest possible and a trivial one
+        q, ck, cv, kv_len = random_batch(B, Hq, Hkv, D, Lmax, lens, seed=900 + seed)
+        ref, _ = orc.decode(q, ck, cv, kv_len.numpy(), 0.09)
+        batches.append((q.cuda(), ck.cuda(), cv.cuda(), kv_len.cuda(), ref))
+    ws = l4l.new_workspace(l4l.L4L_OP_DECODE, 32, Hq, Hkv, D, Lmax)
+    for it in range(12):
+        q, ck, cv, kv_len, ref = batches[it % 2]
+        o = torch.zeros_like(q)
+        l4l.l4l_attn_decode(q, o, ck, cv, kv_len, Lmax, 0.09, ws)
+        if it in (0, 1, 6, 11):
+            torch.cuda.synchronize()
+            assert_close_to_oracle(o, ref, f"repeated decode, call {it}")
+    torch.cuda.synchronize()
+    assert l4l.l4l_last_device_error(ws) == 0
