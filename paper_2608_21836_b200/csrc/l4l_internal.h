@@ -45,12 +45,6 @@ l4l_status launch_prefill(const l4l_tensor4 &q, const l4l_tensor4 &k, const l4l_
                           int S_max, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
                           void *workspace, cudaStream_t stream);
 
-// Warp-MMA (mma.sync) prefill kernel.
-l4l_status launch_prefill_mma(const l4l_tensor4 &q, const l4l_tensor4 &k, const l4l_tensor4 &v,
-                              const l4l_tensor4 &o, const l4l_kv_cache &cache, const int32_t *d_seq_lens,
-                              int S_max, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
-                              void *workspace, cudaStream_t stream);
-
 // tcgen05 / tensor-memory prefill kernel.
 l4l_status launch_prefill_tc(const l4l_tensor4 &q, const l4l_tensor4 &k, const l4l_tensor4 &v,
                              const l4l_tensor4 &o, const l4l_kv_cache &cache, const int32_t *d_seq_lens,

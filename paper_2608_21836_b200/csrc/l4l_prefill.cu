@@ -1,6 +1,4 @@
-// Prefill dispatch: picks the kernel for the shape. (Host code only.)
-#include <cstdlib>
-
+// Prefill entry on the host side: one kernel serves every supported shape.
 #include "l4l_internal.h"
 
 namespace l4l {
@@ -10,14 +8,7 @@ l4l_status launch_prefill(const l4l_tensor4 &q, const l4l_tensor4 &k, const l4l_
                           int S_max, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
                           void *workspace, cudaStream_t stream)
 {
-    // L4L_PREFILL_KERNEL=mma selects the warp-MMA kernel (debugging aid); the default is tcgen05
-    static const bool use_mma = [] {
-        const char *e = getenv("L4L_PREFILL_KERNEL");
-        return e && e[0] == 'm';
-    }();
-    if (!use_mma)
-        return launch_prefill_tc(q, k, v, o, cache, d_seq_lens, S_max, B, Hq, Hkv, D, scale, d_lse, workspace, stream);
-    return launch_prefill_mma(q, k, v, o, cache, d_seq_lens, S_max, B, Hq, Hkv, D, scale, d_lse, workspace, stream);
+    return launch_prefill_tc(q, k, v, o, cache, d_seq_lens, S_max, B, Hq, Hkv, D, scale, d_lse, workspace, stream);
 }
 
 }  // namespace l4l

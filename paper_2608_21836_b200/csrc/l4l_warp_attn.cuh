@@ -1,7 +1,8 @@
 // Warp-level building blocks on the legacy tensor path (mma.sync m16n8k16, bf16 -> fp32):
 // one warp holds 16 query rows and consumes 16 tokens of K and V at a time from a shared-
 // memory tile written by TMA with the 128-byte swizzle. Used by the decode kernel, where
-// the 16 rows are the (zero-padded) query-head group of one KV head.
+// the 16 rows are the (zero-padded) query-head group of one KV head. (Prefill runs on
+// tcgen05 instead: see l4l_prefill_tc.cu.)
 //
 // Tile layout in shared memory: D/64 "halves", each [tile_tokens][64] bf16 (128-byte rows,
 // swizzled), half h covering head_dim [64h, 64h+64).
