@@ -33,10 +33,10 @@ METRIC = "decode-attn HBM GB/s & prefill-attn TFLOP/s, each as % of B200 peak"
 NOMINAL_TFLOPS, NOMINAL_GBS = 2250.0, 8000.0
 FALLBACK_TFLOPS, FALLBACK_GBS = 1590.0, 6650.0
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
-# profiles/: prefill captured at B=1,S=8192 (166.98 MB) and scaled x4 to the bench's B=4 (traffic is proportional
+# profiles/: prefill captured at B=1,S=8192 (155.8 MB) and scaled x4 to the bench's B=4 (traffic is proportional
 # to B); decode captured on the bench's own batch.
-NCU_TRAFFIC_PREFILL = 667.9e6
-NCU_TRAFFIC_DECODE = 306.0e6
+NCU_TRAFFIC_PREFILL = 623.1e6   # 4 x (101.0 MB read + 54.8 MB written)
+NCU_TRAFFIC_DECODE = 299.9e6    # 296.0 MB read + 3.9 MB written
 
 
 def measured_peaks():
