@@ -12,6 +12,7 @@
 //               shared memory into the KV cache (only for the first query head of a KV group)
 //   warp  9     MMA issuer (one lane): S_i = Q_i K_j^T from shared memory, O_i += P_i V_j with P read
 //               from TMEM and V as an MN-major shared-memory operand; owns the TMEM allocation
+//   warps 10-11 help with the cache copy, which runs beside the last iterations
 //
 // TMEM columns: S0 [0,128) S1 [128,256) O0 [256,256+D) O1 [256+D,256+2D); P_i aliases the first 64
 // columns of S_i. Causal tile skipping: sub-tile i only visits K/V tiles up to its diagonal.
