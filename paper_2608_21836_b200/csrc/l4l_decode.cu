@@ -18,6 +18,7 @@
 //                    normalised fp32 partial and its log-sum-exp go to the workspace, and the LAST
 //                    piece to arrive (a self-resetting ticket counter per (sequence, KV head)) runs
 //                    the second pass: the log-sum-exp merge of all pieces.
+#include <cstdlib>
 #include <mutex>
 
 #include "l4l_internal.h"
@@ -27,11 +28,9 @@ namespace l4l {
 
 namespace {
 
-constexpr int kTileT = 64;                 // tokens per TMA tile
-constexpr int kConsumerWarps = 4;
-constexpr int kProducerWarp = kConsumerWarps;
-constexpr int kFinisherWarp = kConsumerWarps + 1;
-constexpr int kThreads = (kConsumerWarps + 2) * 32;
+// The kernel comes in two shapes, W = 4 or 8 consumer warps. A tile is 16*W tokens (each consumer warp takes
+// 16 of them); with W = 4 two CTAs share an SM, with W = 8 one CTA owns it and streams ranges twice as long,
+// so that fewer sequences are cut between CTAs. W + 2 warps in all: consumers, producer, finisher.
 constexpr int kPostRing = 16;               // pieces a producer can be ahead of its finisher (ring size)
 // The ticket counters sit at a FIXED place and size in the workspace (right after the status block), so
 // that calls of different shapes on one workspace can never write partials over counters another call
@@ -39,10 +38,11 @@ constexpr int kPostRing = 16;               // pieces a producer can be ahead of
 constexpr size_t kTicketBytes = 128 * 1024;  // 32768 (sequence, KV head) pairs per launch
 constexpr int kMaxB = 512;                 // sequences per launch (prefix sums live in shared memory)
 
-template <int D>
+template <int D, int W>
 struct DecodeCfg {
+    static constexpr int kTileT = 16 * W;                         // tokens per TMA tile
     static constexpr int kHalves = D / 64;
-    static constexpr uint32_t kHalfBytes = kTileT * 128;          // [64 tokens][64 dims] bf16
+    static constexpr uint32_t kHalfBytes = kTileT * 128;          // [tile tokens][64 dims] bf16
     static constexpr uint32_t kTileBytes = kHalves * kHalfBytes;  // one of K or V
     static constexpr uint32_t kStageBytes = 2 * kTileBytes;
     static constexpr int kStages = (D == 128) ? 3 : 6;
@@ -71,11 +71,11 @@ struct DecodeParams {
     TmapCoord coord;
 };
 
-template <int D>
+template <int D, int W>
 size_t decode_smem_bytes(int G, int nsplit)
 {
-    using C = DecodeCfg<D>;
-    size_t comb = (size_t)kConsumerWarps * G * (D + 4) * sizeof(float) + (size_t)((G * nsplit + 3) & ~3) * sizeof(float);
+    using C = DecodeCfg<D, W>;
+    size_t comb = (size_t)W * G * (D + 4) * sizeof(float) + (size_t)((G * nsplit + 3) & ~3) * sizeof(float);
     return 1024 /*alignment slack*/ + (size_t)C::kStages * (C::kStageBytes + (size_t)G * D * 2) + comb +
            C::kStages * sizeof(TileMeta) +
            sizeof(PieceMeta) + (2 * C::kStages + 2) * sizeof(uint64_t) + (kMaxB + 1) * sizeof(int) + 64 +
@@ -89,13 +89,15 @@ __device__ __forceinline__ void order_coords(const TmapCoord &c, int t, int h, i
     c3 = (c.pos_t == 3) ? t : (c.pos_h == 3) ? h : b;
 }
 
-template <int D>
-__global__ void __launch_bounds__(kThreads)
+template <int D, int W>
+__global__ void __launch_bounds__((W + 2) * 32)
 decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
                     const __grid_constant__ CUtensorMap tmap_k16, const __grid_constant__ CUtensorMap tmap_v16,
                     const DecodeParams p)
 {
-    using C = DecodeCfg<D>;
+    using C = DecodeCfg<D, W>;
+    constexpr int kTileT = C::kTileT;
+    constexpr int kConsumerWarps = W, kProducerWarp = W, kFinisherWarp = W + 1;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     uint8_t *smem = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
@@ -175,10 +177,16 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
 
         if (lane == 0) {
             const int total = running;
-            int per_cta = (total + (int)gridDim.x - 1) / (int)gridDim.x;
-            per_cta = per_cta < p.min_tiles ? p.min_tiles : per_cta;
-            const int my_begin = min(total, (int)blockIdx.x * per_cta);
-            const int my_end = min(total, my_begin + per_cta);
+            // Even split of the tile stream: the first `rem` CTAs take q+1 tiles, the others q, so that
+            // no CTA idles; if that would be fewer than the floor, every CTA takes the floor instead (and
+            // the last CTAs get nothing).
+            int q = total / (int)gridDim.x, rem = total % (int)gridDim.x;
+            if (q < p.min_tiles) { q = p.min_tiles; rem = 0; }
+            const int big = rem * (q + 1);                 // tiles covered by the CTAs that take q+1
+            auto range_begin = [&](int c) { return min(total, c * q + min(c, rem)); };
+            auto cta_of = [&](int t) { return t < big ? t / (q + 1) : rem + (t - big) / q; };
+            const int my_begin = range_begin((int)blockIdx.x);
+            const int my_end = range_begin((int)blockIdx.x + 1);
             uint32_t it = 0, n_posted = 0;
             bool ok = true;
             int g = my_begin;
@@ -197,8 +205,8 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 const int seq_first = cum[b] + kvh * tiles_b;          // flattened index of this sequence's tile 0
                 const int tile_begin = g - seq_first;
                 const int tile_end = min(tiles_b, my_end - seq_first);
-                const int first_cta = seq_first / per_cta;
-                const int npieces = (seq_first + tiles_b - 1) / per_cta - first_cta + 1;
+                const int first_cta = cta_of(seq_first);
+                const int npieces = cta_of(seq_first + tiles_b - 1) - first_cta + 1;
                 const int piece = (int)blockIdx.x - first_cta;
                 {
                     PieceMeta &pp = post_ring[n_posted % kPostRing];
@@ -665,52 +673,74 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
 }
 
 // Resident CTAs per SM for a given dynamic shared-memory size (0 on failure).
-template <int D>
+template <int D, int W>
 int decode_blocks_per_sm(size_t smem)
 {
     static bool attr_set = false;
     if (!attr_set) {
         // the opt-in limit is per kernel: allow everything the SM has
-        if (cudaFuncSetAttribute(decode_split_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+        if (cudaFuncSetAttribute(decode_split_kernel<D, W>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
             cudaSuccess)
             return 0;
         attr_set = true;
     }
     if (smem > 227 * 1024) return 0;
     int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_split_kernel<D>, kThreads, smem) != cudaSuccess)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_split_kernel<D, W>, (W + 2) * 32, smem) != cudaSuccess)
         return 0;
     return n;
 }
 
 }  // namespace
 
-DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_limit)
+namespace {
+
+// Host-side view of one kernel shape.
+struct ShapeOps {
+    int warps, tile_t;
+    size_t (*smem_bytes)(int G, int nsplit);
+    int (*blocks_per_sm)(size_t smem);
+};
+
+template <int D, int W>
+ShapeOps shape_ops()
+{
+    return ShapeOps{W, 16 * W, &decode_smem_bytes<D, W>, &decode_blocks_per_sm<D, W>};
+}
+
+ShapeOps pick_shape(int D, int warps)
+{
+    if (D == 128) return warps == 8 ? shape_ops<128, 8>() : shape_ops<128, 4>();
+    return warps == 8 ? shape_ops<64, 8>() : shape_ops<64, 4>();
+}
+
+// Plan for one kernel shape (warps = 4 or 8).
+DecodePlan plan_for_shape(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_limit, int warps, bool have_dev)
 {
     // Grid: every resident CTA slot of the device. A floor on the tiles per CTA bounds the number of
     // pieces a sequence can be cut into (and with it the partials in the workspace and the finisher's
     // scratch) when the real lengths are far below max_kv_len; it is raised until the partials fit the
     // caller's workspace and the shared memory fits the SM.
     DecodePlan pl;
+    const ShapeOps ops = pick_shape(D, warps);
+    pl.warps = warps;
     const int G = Hq / Hkv;
-    int n_dev = 0;
-    const bool have_dev = cudaGetDeviceCount(&n_dev) == cudaSuccess && n_dev > 0;
-    if (!have_dev) (void)cudaGetLastError();
     auto blocks = [&](int nsplit) {
-        if (!have_dev) return 2;   // sizing without a device: assume the usual two CTAs per SM
-        return (D == 128) ? decode_blocks_per_sm<128>(decode_smem_bytes<128>(G, nsplit))
-                          : decode_blocks_per_sm<64>(decode_smem_bytes<64>(G, nsplit));
+        const size_t smem = ops.smem_bytes(G, nsplit);
+        if (!have_dev) return smem <= 227 * 1024 ? (warps == 8 ? 1 : 2) : 0;   // sizing without a device
+        return ops.blocks_per_sm(smem);
     };
     int per_sm = blocks(2);
     if (per_sm < 1) per_sm = 1;
     const long long slots = (long long)sm_count() * per_sm;
-    const long long tiles_max = max_kv_len > 0 ? (max_kv_len + kTileT - 1) / kTileT : 1;
+    const long long tiles_max = max_kv_len > 0 ? (max_kv_len + ops.tile_t - 1) / ops.tile_t : 1;
     const long long total_max = (long long)B * Hkv * tiles_max;
     long long min_tiles = (total_max + 8 * slots - 1) / (8 * slots);
     // small problems are latency-bound: a CTA that streams only a tile or two spends longer in the
-    // merge of the many pieces than in the stream, so give every CTA at least 16 tiles (or a quarter
+    // merge of the many pieces than in the stream, so give every CTA at least 1024 tokens (or a quarter
     // of the longest sequence, if that is less)
-    const long long floor_tiles = (tiles_max + 3) / 4 < 16 ? (tiles_max + 3) / 4 : 16;
+    const long long floor_cap = 1024 / ops.tile_t;
+    const long long floor_tiles = (tiles_max + 3) / 4 < floor_cap ? (tiles_max + 3) / 4 : floor_cap;
     if (min_tiles < floor_tiles) min_tiles = floor_tiles;
     if (min_tiles < 1) min_tiles = 1;
     for (;; min_tiles *= 2) {
@@ -724,9 +754,31 @@ DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_
                       (size_t)B * Hq * pl.nsplit * (D + 1) * sizeof(float);
         const int n = blocks(pl.nsplit);
         pl.grid = sm_count() * (n > 0 ? n : 1);
+        pl.fits = n > 0;
         if ((pl.ws_bytes <= ws_limit && n > 0) || min_tiles >= tiles_max) break;
     }
     return pl;
+}
+
+}  // namespace
+
+DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_limit)
+{
+    int n_dev = 0;
+    const bool have_dev = cudaGetDeviceCount(&n_dev) == cudaSuccess && n_dev > 0;
+    if (!have_dev) (void)cudaGetLastError();
+    // Prefer the 8-warp shape (one CTA per SM, ranges twice as long, so fewer sequences are cut between
+    // CTAs) whenever its shared memory fits, which it does for query-head groups of up to 4; else 4 warps.
+    static const int forced = [] {
+        const char *e = getenv("L4L_DECODE_WARPS");      // debugging aid: force a shape
+        return e ? atoi(e) : 0;
+    }();
+    if (forced != 4) {
+        const DecodePlan p8 = plan_for_shape(B, Hq, Hkv, D, max_kv_len, ws_limit, 8, have_dev);
+        if (p8.fits && p8.ws_bytes <= ws_limit) return p8;
+        if (forced == 8) return p8;
+    }
+    return plan_for_shape(B, Hq, Hkv, D, max_kv_len, ws_limit, 4, have_dev);
 }
 
 l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, const int32_t *d_kv_lens,
@@ -734,8 +786,10 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
                          void *workspace, const DecodePlan &plan, cudaStream_t stream)
 {
     const int G = Hq / Hkv;
-    const size_t smem = (D == 128) ? decode_smem_bytes<128>(G, plan.nsplit) : decode_smem_bytes<64>(G, plan.nsplit);
-    if (((D == 128) ? decode_blocks_per_sm<128>(smem) : decode_blocks_per_sm<64>(smem)) == 0) return L4L_ERR_CUDA;
+    const ShapeOps ops = pick_shape(D, plan.warps);
+    const int kTileT = ops.tile_t;
+    const size_t smem = ops.smem_bytes(G, plan.nsplit);
+    if (ops.blocks_per_sm(smem) == 0) return L4L_ERR_CUDA;
     uint8_t *ws = static_cast<uint8_t *>(workspace);
     int *tickets = reinterpret_cast<int *>(ws + kStatusBytes);
     // partial outputs first: their float4 accesses need 16-byte alignment
@@ -776,7 +830,7 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         p.coord = coord;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(plan.grid);
-        cfg.blockDim = dim3(kThreads);
+        cfg.blockDim = dim3((plan.warps + 2) * 32);
         cfg.dynamicSmemBytes = smem;
         cfg.stream = stream;
         cudaLaunchAttribute attr[1];
@@ -784,8 +838,13 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        const cudaError_t err = (D == 128) ? cudaLaunchKernelEx(&cfg, decode_split_kernel<128>, tk, tv, tk16, tv16, p)
-                                           : cudaLaunchKernelEx(&cfg, decode_split_kernel<64>, tk, tv, tk16, tv16, p);
+        cudaError_t err;
+        if (D == 128)
+            err = plan.warps == 8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 8>, tk, tv, tk16, tv16, p)
+                                  : cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 4>, tk, tv, tk16, tv16, p);
+        else
+            err = plan.warps == 8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<64, 8>, tk, tv, tk16, tv16, p)
+                                  : cudaLaunchKernelEx(&cfg, decode_split_kernel<64, 4>, tk, tv, tk16, tv16, p);
         if (err != cudaSuccess) return L4L_ERR_CUDA;
     }
     return L4L_OK;

@@ -25,6 +25,8 @@ bool make_tmap_bf16(CUtensorMap *out, TmapCoord *coord, const void *base, int D,
 int sm_count();
 
 struct DecodePlan {
+    int warps;       // kernel shape: 4 or 8 consumer warps (tile = 16 tokens per warp)
+    bool fits;       // the shape's shared memory fits an SM
     int grid;        // persistent CTAs
     int min_tiles;   // floor on the 64-token tiles per CTA (bounds the pieces per sequence)
     int nsplit;      // max pieces a (sequence, KV head) can be cut into
