@@ -282,6 +282,11 @@ def run_ours(args, rank, world):
         l4l.l4l_attn_decode(dq, do, caches[i][0], caches[i][1], dlen, Lmax, wd.scale, ws_d)
     barrier()
     d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # a few milliseconds of unrelated GPU work queued first, so that the host has every launch of the timed
+    # run enqueued before the GPU reaches it: the figure is device time, not Python call overhead
+    filler = torch.empty(1 << 28, dtype=torch.float32, device=dev)
+    for _ in range(6):
+        filler.zero_()
     d0.record()
     for i in range(n_dec):
         ck_i, cv_i = caches[i % 3]
@@ -289,7 +294,7 @@ def run_ours(args, rank, world):
     d1.record()
     barrier()
     t_dec_b2b = d0.elapsed_time(d1) / n_dec
-    del caches
+    del caches, filler
     dev_err = l4l.l4l_last_device_error(ws_p) | l4l.l4l_last_device_error(ws_d)
 
     # ---- end to end through the same entry points with HOST buffers (pinned), copies inside the timed region

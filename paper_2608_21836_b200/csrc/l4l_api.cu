@@ -64,8 +64,61 @@ int sm_count()
     return n;
 }
 
+namespace {
+
+// A serving loop calls with the same buffers step after step: remember the last few encoded maps
+// (a tensor map is a pure function of these arguments).
+struct TmapKey {
+    const void *base;
+    int D, box_d, box_t;
+    int64_t n_t, n_h, n_b, stride_t, stride_h, stride_b;
+    bool operator==(const TmapKey &o) const
+    {
+        return base == o.base && D == o.D && box_d == o.box_d && box_t == o.box_t && n_t == o.n_t && n_h == o.n_h &&
+               n_b == o.n_b && stride_t == o.stride_t && stride_h == o.stride_h && stride_b == o.stride_b;
+    }
+};
+struct TmapEntry {
+    TmapKey key;
+    CUtensorMap map;
+    TmapCoord coord;
+    bool valid = false;
+};
+constexpr int kTmapCache = 32;
+TmapEntry g_tmap_cache[kTmapCache];
+int g_tmap_next = 0;
+std::mutex g_tmap_mutex;
+
+bool encode_tmap_bf16(CUtensorMap *out, TmapCoord *coord, const void *base, int D, int64_t n_t, int64_t n_h,
+                      int64_t n_b, int64_t stride_t, int64_t stride_h, int64_t stride_b, int box_d, int box_t);
+
+}  // namespace
+
 bool make_tmap_bf16(CUtensorMap *out, TmapCoord *coord, const void *base, int D, int64_t n_t, int64_t n_h,
                     int64_t n_b, int64_t stride_t, int64_t stride_h, int64_t stride_b, int box_d, int box_t)
+{
+    const TmapKey key{base, D, box_d, box_t, n_t, n_h, n_b, stride_t, stride_h, stride_b};
+    {
+        std::lock_guard<std::mutex> lock(g_tmap_mutex);
+        for (int i = 0; i < kTmapCache; ++i)
+            if (g_tmap_cache[i].valid && g_tmap_cache[i].key == key) {
+                *out = g_tmap_cache[i].map;
+                *coord = g_tmap_cache[i].coord;
+                return true;
+            }
+    }
+    if (!encode_tmap_bf16(out, coord, base, D, n_t, n_h, n_b, stride_t, stride_h, stride_b, box_d, box_t)) return false;
+    std::lock_guard<std::mutex> lock(g_tmap_mutex);
+    TmapEntry &e = g_tmap_cache[g_tmap_next];
+    g_tmap_next = (g_tmap_next + 1) % kTmapCache;
+    e.key = key; e.map = *out; e.coord = *coord; e.valid = true;
+    return true;
+}
+
+namespace {
+
+bool encode_tmap_bf16(CUtensorMap *out, TmapCoord *coord, const void *base, int D, int64_t n_t, int64_t n_h,
+                      int64_t n_b, int64_t stride_t, int64_t stride_h, int64_t stride_b, int box_d, int box_t)
 {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
@@ -97,6 +150,8 @@ bool make_tmap_bf16(CUtensorMap *out, TmapCoord *coord, const void *base, int D,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
+
+}  // namespace
 
 }  // namespace l4l
 
