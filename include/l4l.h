@@ -138,6 +138,22 @@ l4l_status l4l_attn_decode(const void *q, void *o, l4l_kv_cache cache,
                            float *d_lse, void *workspace, size_t ws_bytes, l4l_stream stream);
 
 /*
+ * Decode with the cache update fused in (one launch per decode step instead of two; the paper leaves
+ * the cache update to the module code around its decode kernel, and notes that the state must be
+ * updated exactly once). For every sequence b with n = kv_lens[b] >= 1: cache slot n-1 receives
+ * k_new[b, 0, :, :] and v_new[b, 0, :, :] bit for bit, and o[b] is the attention of q[b] over slots
+ * 0..n-1 with that newest token taken from k_new / v_new. Equivalent to l4l_kv_append at slot n-1
+ * followed by l4l_attn_decode; sequences with n = 0 append nothing and give o = 0.
+ *   k_new, v_new  [B, 1, Hkv, D] views (stride_t unused); both with the same strides
+ * Everything else as in l4l_attn_decode.
+ */
+l4l_status l4l_attn_decode_append(const void *q, void *o, l4l_kv_cache cache,
+                                  l4l_tensor4 k_new, l4l_tensor4 v_new,
+                                  const int32_t *d_kv_lens, int max_kv_len,
+                                  int B, int Hq, int Hkv, int head_dim, float scale,
+                                  float *d_lse, void *workspace, size_t ws_bytes, l4l_stream stream);
+
+/*
  * Decode for callers that cannot allocate device memory (no counterpart in the paper: it is the
  * same operation as l4l_attn_decode, with the scratch moved inside the library).
  *

@@ -22,7 +22,7 @@ L4L_OP_PREFILL, L4L_OP_DECODE = 0, 1
 EXPORTS = (
     "l4l_version", "l4l_status_string", "l4l_workspace_bytes", "l4l_workspace_init",
     "l4l_last_device_error", "l4l_kv_append", "l4l_attn_prefill", "l4l_attn_decode",
-    "l4l_attn_decode_static",
+    "l4l_attn_decode_static", "l4l_attn_decode_append",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -76,6 +76,9 @@ def load() -> ctypes.CDLL:
     lib.l4l_attn_decode_static.restype = c_int
     lib.l4l_attn_decode_static.argtypes = [vp, vp, KVCache, i32p, c_int, c_int, c_int, c_int, c_int, ctypes.c_float, vp,
                                            vp]
+    lib.l4l_attn_decode_append.restype = c_int
+    lib.l4l_attn_decode_append.argtypes = [vp, vp, KVCache, Tensor4, Tensor4, i32p, c_int, c_int, c_int, c_int, c_int,
+                                           ctypes.c_float, vp, vp, c_size, vp]
     _lib = lib
     return lib
 
@@ -212,3 +215,27 @@ def l4l_attn_decode_static(q, o, cache_k, cache_v, kv_lens, max_kv_len: int, sca
                                        None if lse is None else lse.data_ptr(), _stream())
     if st != L4L_OK:
         raise L4LError(st, "l4l_attn_decode_static")
+
+
+def l4l_attn_decode_append(q, o, cache_k, cache_v, k_new, v_new, kv_lens, max_kv_len: int, scale: float, workspace,
+                           lse=None) -> None:
+    """One launch per decode step: writes k_new / v_new ([B,1,Hkv,D]) into cache slot kv_lens[b]-1 and attends
+    over slots 0..kv_lens[b]-1. Same result as l4l_kv_append followed by l4l_attn_decode."""
+    _check_bf16_cuda(q, "q")
+    _check_bf16_cuda(o, "o")
+    if not (q.is_contiguous() and o.is_contiguous() and q.dim() == 3 and q.shape == o.shape):
+        raise ValueError("q and o must be dense [B, Hq, D]")
+    B, Hq, D = q.shape
+    Hkv = cache_k.shape[1]
+    if tuple(k_new.shape) != (B, 1, Hkv, D) or tuple(v_new.shape) != (B, 1, Hkv, D):
+        raise ValueError("k_new and v_new must be [B, 1, Hkv, D]")
+    if lse is not None and not (lse.is_cuda and lse.dtype == torch.float32 and lse.is_contiguous()
+                                and tuple(lse.shape) == (B, Hq)):
+        raise TypeError("lse must be a contiguous CUDA float32 tensor [B, Hq]")
+    st = load().l4l_attn_decode_append(q.data_ptr(), o.data_ptr(), kv_cache(cache_k, cache_v),
+                                       tensor4(k_new, "k_new"), tensor4(v_new, "v_new"),
+                                       _i32_dev(kv_lens, "kv_lens"), int(max_kv_len), B, Hq, Hkv, D, float(scale),
+                                       None if lse is None else lse.data_ptr(), workspace.data_ptr(),
+                                       workspace.numel() * workspace.element_size(), _stream())
+    if st != L4L_OK:
+        raise L4LError(st, "l4l_attn_decode_append")

@@ -65,6 +65,12 @@ struct DecodeParams {
     float *part_o;            // [B, Hq, nsplit, D]  normalised partial outputs
     float *part_lse;          // [B, Hq, nsplit]     log2-domain log-sum-exp of the piece
     int *tickets;             // [B, Hkv]            pieces arrived; zero between calls
+    // fused append (null: none): the newest token of every sequence (slot kv_len-1) comes from here and
+    // is written to the cache by the CTA that streams its tile
+    const __nv_bfloat16 *k_new, *v_new;       // element (b, kv head, d) at b*new_sb + kvh*new_sh + d
+    int64_t new_sb, new_sh;
+    __nv_bfloat16 *cache_k, *cache_v;
+    int64_t c_sb, c_sh, c_st;
     unsigned *status;
     int B, Hq, Hkv, G, min_tiles, nsplit, max_kv_len;
     float scale_log2e;
@@ -594,6 +600,28 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             const int row0 = warp * 16;
             const int nvalid = mt.kv_len - (mt.t0 + row0);       // valid tokens in this warp's slice
             bool wrote_smem = false;
+            if (p.k_new != nullptr && nvalid > 0 && nvalid <= 16) {
+                // fused append: this slice holds the sequence's newest token (row `last` of the tile). Its K/V
+                // arrive from the caller, not from the cache: patch the tile in shared memory and write the
+                // cache slot (each slot belongs to exactly one CTA's range and one warp's slice).
+                const int last = row0 + nvalid - 1;
+                constexpr int kChunks = D / 8;
+                if (lane < kChunks) {
+                    const size_t src = (size_t)mt.b * p.new_sb + (size_t)mt.kvh * p.new_sh + lane * 8;
+                    const uint4 kk = __ldg(reinterpret_cast<const uint4 *>(p.k_new + src));
+                    const uint4 vv = __ldg(reinterpret_cast<const uint4 *>(p.v_new + src));
+                    uint8_t *kt = stages + (size_t)s * C::kStageBytes;
+                    const uint32_t off = (lane >> 3) * C::kHalfBytes + swz128(last, lane & 7);
+                    *reinterpret_cast<uint4 *>(kt + off) = kk;
+                    *reinterpret_cast<uint4 *>(kt + C::kTileBytes + off) = vv;
+                    const size_t dst = (size_t)mt.b * p.c_sb + (size_t)mt.kvh * p.c_sh +
+                                       (size_t)(mt.kv_len - 1) * p.c_st + lane * 8;
+                    *reinterpret_cast<uint4 *>(p.cache_k + dst) = kk;
+                    *reinterpret_cast<uint4 *>(p.cache_v + dst) = vv;
+                }
+                wrote_smem = true;
+                __syncwarp();
+            }
             if (nvalid > 0) {
                 float s_lo[4], s_hi[4];
                 warp_qk_16x16<D>(qf, k_tile, C::kHalfBytes, row0, s_lo, s_hi);
@@ -783,7 +811,8 @@ DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_
 
 l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, const int32_t *d_kv_lens,
                          int max_kv_len, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
-                         void *workspace, const DecodePlan &plan, cudaStream_t stream)
+                         void *workspace, const DecodePlan &plan, cudaStream_t stream, const l4l_tensor4 *k_new,
+                         const l4l_tensor4 *v_new)
 {
     const int G = Hq / Hkv;
     const ShapeOps ops = pick_shape(D, plan.warps);
@@ -826,6 +855,17 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         p.status = reinterpret_cast<unsigned *>(ws);
         p.B = nb; p.Hq = Hq; p.Hkv = Hkv; p.G = G; p.min_tiles = plan.min_tiles; p.nsplit = plan.nsplit;
         p.max_kv_len = max_kv_len;
+        p.k_new = p.v_new = nullptr;
+        p.new_sb = p.new_sh = 0;
+        p.cache_k = static_cast<__nv_bfloat16 *>(cache.k) + (size_t)b0 * cache.stride_b;
+        p.cache_v = static_cast<__nv_bfloat16 *>(cache.v) + (size_t)b0 * cache.stride_b;
+        p.c_sb = cache.stride_b; p.c_sh = cache.stride_h; p.c_st = cache.stride_t;
+        if (k_new && v_new) {
+            if (k_new->stride_b != v_new->stride_b || k_new->stride_h != v_new->stride_h) return L4L_ERR_UNSUPPORTED;
+            p.k_new = static_cast<const __nv_bfloat16 *>(k_new->ptr) + (size_t)b0 * k_new->stride_b;
+            p.v_new = static_cast<const __nv_bfloat16 *>(v_new->ptr) + (size_t)b0 * v_new->stride_b;
+            p.new_sb = k_new->stride_b; p.new_sh = k_new->stride_h;
+        }
         p.scale_log2e = scale * 1.4426950408889634f;
         p.coord = coord;
         cudaLaunchConfig_t cfg = {};
@@ -921,5 +961,6 @@ extern "C" l4l_status l4l_attn_decode_static(const void *q, void *o, l4l_kv_cach
     // start at zero (the partials need no clearing, every slot is written before it is read)
     const size_t zero_bytes = kStatusBytes + kTicketBytes;
     if (cudaMemsetAsync(scratch, 0, zero_bytes, s) != cudaSuccess) return L4L_ERR_CUDA;
-    return launch_decode(q, o, cache, d_kv_lens, max_kv_len, B, Hq, Hkv, head_dim, scale, d_lse, scratch, plan, s);
+    return launch_decode(q, o, cache, d_kv_lens, max_kv_len, B, Hq, Hkv, head_dim, scale, d_lse, scratch, plan, s,
+                         nullptr, nullptr);
 }

@@ -36,7 +36,8 @@ DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_
 
 l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, const int32_t *d_kv_lens,
                          int max_kv_len, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
-                         void *workspace, const DecodePlan &plan, cudaStream_t stream);
+                         void *workspace, const DecodePlan &plan, cudaStream_t stream,
+                         const l4l_tensor4 *k_new = nullptr, const l4l_tensor4 *v_new = nullptr);
 
 l4l_status launch_kv_append(const l4l_kv_cache &cache, const l4l_tensor4 &k_new, const l4l_tensor4 &v_new,
                             const int32_t *d_write_pos, const int32_t *d_n_new, int n_new_max, int B, int Hkv,
