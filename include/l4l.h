@@ -120,6 +120,24 @@ l4l_status l4l_attn_prefill(l4l_tensor4 q, l4l_tensor4 k, l4l_tensor4 v, l4l_ten
                             float *d_lse, void *workspace, size_t ws_bytes, l4l_stream stream);
 
 /*
+ * Prefill of a chunk of new tokens over an already populated cache (the regime between the paper's
+ * two phases: q_len > 1 AND a populated cache; bottom-right causal alignment). For sequence b with
+ * P = past_lens[b] tokens already cached and L = q_lens[b] new tokens, whose K and V the caller has
+ * ALREADY written to cache slots P .. P+L-1 (l4l_kv_append), query row i < L and query head h:
+ *     o[b, i, h, :] = softmax_j( scale * q[b, i, h, :] . K[b, h/G, j, :],  j = 0 .. P+i ) @ V[b, h/G, 0..P+i, :]
+ * Keys and values are read from the cache; nothing is written to it. P = 0 is an ordinary prefill
+ * whose keys happen to live in the cache. Rows i >= L of o / lse are left untouched; cache slots
+ * >= P+L may hold anything.
+ *   q, o          [B, S_max, Hq, D] views (the chunk's tokens)
+ *   d_past_lens   device int32 [B], P >= 0;   d_q_lens  device int32 [B], 0 <= L <= S_max; P + L <= cache.max_len
+ *   d_lse         device float [B, Hq, S_max] or NULL;   workspace as for l4l_attn_prefill
+ */
+l4l_status l4l_attn_prefill_chunk(l4l_tensor4 q, l4l_tensor4 o, l4l_kv_cache cache,
+                                  const int32_t *d_past_lens, const int32_t *d_q_lens, int S_max,
+                                  int B, int Hq, int Hkv, int head_dim, float scale,
+                                  float *d_lse, void *workspace, size_t ws_bytes, l4l_stream stream);
+
+/*
  * Decode. For every sequence b with n = kv_lens[b] cached tokens (the current token has
  * already been appended and is included), query head h:
  *     o[b, h, :] = softmax_j( scale * q[b, h, :] . K[b, h/G, j, :],  j = 0..n-1 ) @ V[b, h/G, 0..n-1, :]

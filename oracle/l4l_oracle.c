@@ -179,6 +179,48 @@ int l4l_oracle_prefill_rows(const uint16_t *q, const uint16_t *k, const uint16_t
 }
 
 /*
+ * Prefill of a chunk of new tokens over a populated cache (q_len > 1 AND a populated cache, the regime
+ * between the paper's two phases), bottom-right causal alignment: row i of the chunk is the token at
+ * absolute position past[b] + i and sees cache slots 0 .. past[b] + i. The chunk's own K/V are expected in
+ * the cache already (slots past[b] .. past[b] + q_len[b] - 1).
+ *   q        [B, S, Hq, D]        cache_k, cache_v  [B, Hkv, Lmax, D]
+ *   out      [B, S, Hq, D] fp64; rows i >= q_len[b] are left untouched     lse [B, Hq, S] or NULL
+ */
+int l4l_oracle_prefill_chunk(const uint16_t *q, const uint16_t *cache_k, const uint16_t *cache_v,
+                             const int32_t *past, const int32_t *q_len, int B, int S, int Hq, int Hkv, int D,
+                             int Lmax, double scale, double *out, double *lse)
+{
+    if (Hkv <= 0 || Hq % Hkv != 0) return -1;
+    for (int b = 0; b < B; ++b)
+        if (past[b] < 0 || q_len[b] < 0 || q_len[b] > S || past[b] + q_len[b] > Lmax) return -1;
+    const int G = Hq / Hkv;
+    int fail = 0;
+#pragma omp parallel
+    {
+        double *p = (double *)malloc(sizeof(double) * (size_t)(Lmax > 0 ? Lmax : 1));
+        if (!p) {
+#pragma omp atomic write
+            fail = 1;
+        }
+#pragma omp for collapse(2) schedule(dynamic, 8)
+        for (int b = 0; b < B; ++b) {
+            for (int i = 0; i < S; ++i) {
+                if (!p || i >= q_len[b]) continue;
+                for (int h = 0; h < Hq; ++h) {
+                    const int g = h / G;
+                    const int64_t base = ((int64_t)b * Hkv + g) * Lmax * D;
+                    attend_row(q + (((int64_t)b * S + i) * Hq + h) * D, cache_k + base, D, cache_v + base, D,
+                               past[b] + i + 1, D, scale, p, out + (((int64_t)b * S + i) * Hq + h) * D,
+                               lse ? lse + ((int64_t)b * Hq + h) * S + i : NULL);
+                }
+            }
+        }
+        free(p);
+    }
+    return fail ? -1 : 0;
+}
+
+/*
  * Decode: one query token per sequence over the populated cache (no mask).
  *   q        [B, Hq, D]           cache_k, cache_v  [B, Hkv, Lmax, D]
  *   kv_len   [B]   valid tokens, the current one included (<= Lmax)

@@ -46,6 +46,7 @@ def _load():
         lib.l4l_oracle_prefill_rows.argtypes = [u16p, u16p, u16p, i32p, i, i, i, i, i, d,
                                                 i32p, i, f64p, f64p]
         lib.l4l_oracle_decode.argtypes = [u16p, u16p, u16p, i32p, i, i, i, i, i, d, f64p, f64p]
+        lib.l4l_oracle_prefill_chunk.argtypes = [u16p, u16p, u16p, i32p, i32p, i, i, i, i, i, i, d, f64p, f64p]
         lib.l4l_oracle_kv_append.argtypes = [u16p, u16p, u16p, u16p, i32p, i32p, i, i, i, i, i]
         _lib = lib
     return _lib
@@ -114,6 +115,24 @@ def prefill_rows(q, k, v, seq_len, scale: float, rows):
                                          _p(out, ctypes.c_double), _p(lse, ctypes.c_double))
     if rc != 0:
         raise ValueError("l4l_oracle_prefill_rows rejected its arguments")
+    return out, lse
+
+
+def prefill_chunk(q, cache_k, cache_v, past, q_len, scale: float):
+    """Chunk of new tokens over a populated cache. q [B,S,Hq,D], caches [B,Hkv,Lmax,D] already holding the
+    chunk's K/V at slots past..past+q_len-1; returns (out [B,S,Hq,D], lse [B,Hq,S]), NaN in undefined rows."""
+    q, ck, cv = bits(q), bits(cache_k), bits(cache_v)
+    B, S, Hq, D = q.shape
+    _, Hkv, Lmax, _ = ck.shape
+    assert ck.shape == (B, Hkv, Lmax, D) and cv.shape == ck.shape
+    past, q_len = _i32(past), _i32(q_len)
+    out = np.full((B, S, Hq, D), np.nan, dtype=np.float64)
+    lse = np.full((B, Hq, S), np.nan, dtype=np.float64)
+    rc = _load().l4l_oracle_prefill_chunk(_p(q, ctypes.c_uint16), _p(ck, ctypes.c_uint16), _p(cv, ctypes.c_uint16),
+                                          _p(past, ctypes.c_int32), _p(q_len, ctypes.c_int32), B, S, Hq, Hkv, D,
+                                          Lmax, float(scale), _p(out, ctypes.c_double), _p(lse, ctypes.c_double))
+    if rc != 0:
+        raise ValueError("l4l_oracle_prefill_chunk rejected its arguments")
     return out, lse
 
 

@@ -22,7 +22,7 @@ L4L_OP_PREFILL, L4L_OP_DECODE = 0, 1
 EXPORTS = (
     "l4l_version", "l4l_status_string", "l4l_workspace_bytes", "l4l_workspace_init",
     "l4l_last_device_error", "l4l_kv_append", "l4l_attn_prefill", "l4l_attn_decode",
-    "l4l_attn_decode_static", "l4l_attn_decode_append",
+    "l4l_attn_decode_static", "l4l_attn_decode_append", "l4l_attn_prefill_chunk",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -76,6 +76,9 @@ def load() -> ctypes.CDLL:
     lib.l4l_attn_decode_static.restype = c_int
     lib.l4l_attn_decode_static.argtypes = [vp, vp, KVCache, i32p, c_int, c_int, c_int, c_int, c_int, ctypes.c_float, vp,
                                            vp]
+    lib.l4l_attn_prefill_chunk.restype = c_int
+    lib.l4l_attn_prefill_chunk.argtypes = [Tensor4, Tensor4, KVCache, i32p, i32p, c_int, c_int, c_int, c_int, c_int,
+                                           ctypes.c_float, vp, vp, c_size, vp]
     lib.l4l_attn_decode_append.restype = c_int
     lib.l4l_attn_decode_append.argtypes = [vp, vp, KVCache, Tensor4, Tensor4, i32p, c_int, c_int, c_int, c_int, c_int,
                                            ctypes.c_float, vp, vp, c_size, vp]
@@ -239,3 +242,19 @@ def l4l_attn_decode_append(q, o, cache_k, cache_v, k_new, v_new, kv_lens, max_kv
                                        workspace.numel() * workspace.element_size(), _stream())
     if st != L4L_OK:
         raise L4LError(st, "l4l_attn_decode_append")
+
+
+def l4l_attn_prefill_chunk(q, o, cache_k, cache_v, past_lens, q_lens, scale: float, workspace, lse=None) -> None:
+    """Chunk of new tokens over a populated cache. q,o [B,S,Hq,D]; the chunk's K/V are already in the cache at
+    slots past..past+q_len-1; past_lens, q_lens CUDA int32 [B]; lse optional CUDA float32 [B,Hq,S]."""
+    B, S, Hq, D = q.shape
+    Hkv = cache_k.shape[1]
+    if lse is not None and not (lse.is_cuda and lse.dtype == torch.float32 and lse.is_contiguous()
+                                and tuple(lse.shape) == (B, Hq, S)):
+        raise TypeError("lse must be a contiguous CUDA float32 tensor [B, Hq, S]")
+    st = load().l4l_attn_prefill_chunk(tensor4(q, "q"), tensor4(o, "o"), kv_cache(cache_k, cache_v),
+                                       _i32_dev(past_lens, "past_lens"), _i32_dev(q_lens, "q_lens"), S, B, Hq, Hkv, D,
+                                       float(scale), None if lse is None else lse.data_ptr(), workspace.data_ptr(),
+                                       workspace.numel() * workspace.element_size(), _stream())
+    if st != L4L_OK:
+        raise L4LError(st, "l4l_attn_prefill_chunk")

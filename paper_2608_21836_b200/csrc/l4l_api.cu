@@ -228,6 +228,20 @@ l4l_status l4l_attn_prefill(l4l_tensor4 q, l4l_tensor4 k, l4l_tensor4 v, l4l_ten
                           static_cast<cudaStream_t>(stream));
 }
 
+l4l_status l4l_attn_prefill_chunk(l4l_tensor4 q, l4l_tensor4 o, l4l_kv_cache cache, const int32_t *d_past_lens,
+                                  const int32_t *d_q_lens, int S_max, int B, int Hq, int Hkv, int head_dim,
+                                  float scale, float *d_lse, void *workspace, size_t ws_bytes, l4l_stream stream)
+{
+    l4l_status st = shape_status(B, Hq, Hkv, head_dim);
+    if (st != L4L_OK) return st;
+    if (S_max < 0 || !d_past_lens || !d_q_lens) return L4L_ERR_INVALID_ARG;
+    if (!tensor4_ok(q) || !tensor4_ok(o) || !cache_ok(cache)) return L4L_ERR_INVALID_ARG;
+    if (!workspace || ws_bytes < kStatusBytes) return L4L_ERR_WORKSPACE;
+    if (B == 0 || S_max == 0) return L4L_OK;
+    return launch_prefill_chunk(q, o, cache, d_past_lens, d_q_lens, S_max, B, Hq, Hkv, head_dim, scale, d_lse,
+                                workspace, static_cast<cudaStream_t>(stream));
+}
+
 l4l_status l4l_attn_decode(const void *q, void *o, l4l_kv_cache cache, const int32_t *d_kv_lens, int max_kv_len,
                            int B, int Hq, int Hkv, int head_dim, float scale, float *d_lse, void *workspace,
                            size_t ws_bytes, l4l_stream stream)

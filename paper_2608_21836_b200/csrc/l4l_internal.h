@@ -48,10 +48,15 @@ l4l_status launch_prefill(const l4l_tensor4 &q, const l4l_tensor4 &k, const l4l_
                           int S_max, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
                           void *workspace, cudaStream_t stream);
 
-// tcgen05 / tensor-memory prefill kernel.
+// tcgen05 / tensor-memory prefill kernel. k, v: where the keys and values are read from, as [B, T, Hkv, D]
+// views with kv_extent token slots. d_past_lens (may be null): tokens ahead of the chunk, per sequence.
 l4l_status launch_prefill_tc(const l4l_tensor4 &q, const l4l_tensor4 &k, const l4l_tensor4 &v,
                              const l4l_tensor4 &o, const l4l_kv_cache &cache, const int32_t *d_seq_lens,
                              int S_max, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
-                             void *workspace, cudaStream_t stream);
+                             void *workspace, cudaStream_t stream, const int32_t *d_past_lens, int kv_extent);
+
+l4l_status launch_prefill_chunk(const l4l_tensor4 &q, const l4l_tensor4 &o, const l4l_kv_cache &cache,
+                                const int32_t *d_past_lens, const int32_t *d_q_lens, int S_max, int B, int Hq,
+                                int Hkv, int D, float scale, float *d_lse, void *workspace, cudaStream_t stream);
 
 }  // namespace l4l

@@ -48,6 +48,7 @@ struct TcParams {
     int64_t c_sb, c_sh, c_st;
     int cache_max_len;
     const int32_t *seq_lens;
+    const int32_t *past_lens;   // null: fresh prompt (keys come from k/v); else keys come from the cache views
     float *lse;
     unsigned *status;
     int S_max, B, Hq, Hkv, G, n_qblocks;
@@ -100,10 +101,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     L = L < 0 ? 0 : (L > p.S_max ? p.S_max : L);
     const int q0 = qb * 2 * kRows;
     if (q0 >= L) return;
-    const int n_tiles_L = (L + kRows - 1) / kRows;              // K/V tiles that hold any valid token
+    // Tokens already in the cache ahead of this chunk (0 for a fresh prompt): query row i sees keys
+    // 0 .. past + i. kv_total keys exist in all.
+    int past = p.past_lens ? p.past_lens[b] : 0;
+    past = past < 0 ? 0 : past;
+    const int kv_total = past + L;
+    // sub-tile i (rows q0 + 128 i ..) visits K/V tiles 0 .. tile of its last valid row's last key
     int n_sub[2];
-    n_sub[0] = min(n_tiles_L, 2 * qb + 1);
-    n_sub[1] = (q0 + kRows < L) ? min(n_tiles_L, 2 * qb + 2) : 0;
+    n_sub[0] = (past + min(q0 + kRows - 1, L - 1)) / kRows + 1;
+    n_sub[1] = (q0 + kRows < L) ? (past + min(q0 + 2 * kRows - 1, L - 1)) / kRows + 1 : 0;
     const int n_kv = max(n_sub[0], n_sub[1]);
 
     extern __shared__ uint8_t smem_raw[];
@@ -270,7 +276,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
             const int iv = 2 * j + 1, ik = 2 * j + 2;
             const uint32_t sv = iv % C::kSlots, sk = ik % C::kSlots;
             if (!mbar_wait(&kv_full[sv], (iv / C::kSlots) & 1u, abort_flag)) { ok = false; break; }
-            const int first_dead = L - j * kRows;                 // V rows >= this hold no valid token
+            const int first_dead = kv_total - j * kRows;          // V rows >= this hold no valid token
             if (first_dead < kRows) {
                 // may hold any bits (NaN included): clear, so that a zero weight times garbage cannot appear
                 uint8_t *vt = ring + (size_t)sv * C::kTileBytes;
@@ -317,7 +323,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
         const uint32_t tmem_s = tmem_base + lane_base + (i ? C::kColS1 : C::kColS0);
         const uint32_t tmem_o = tmem_base + lane_base + (i ? C::kColO1 : C::kColO0);
         const int n_mine = n_sub[i];
-        const int diag_tile = (q0 + i * kRows) / kRows;
+        const int mask_from = (past + q0 + i * kRows) / kRows;   // first K/V tile that holds a key some row must not see
         const float c = p.scale_log2e;
         float m = -INFINITY, l = 0.f;
         bool ok = true;
@@ -333,10 +339,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
             // Row maximum of the scaled scores (log2 domain). Off the diagonal the maximum is taken over the
             // raw scores with independent 3-input max chains and scaled once (min for a negative scale);
             // on the diagonal tile the causal mask is applied to the scaled scores first.
-            const bool diag = (j == diag_tile);
+            const bool diag = (j >= mask_from);
             float mx;
             if (diag) {
-                const int lim = row - j * kRows;                   // columns > lim are in the future
+                const int lim = past + row - j * kRows;            // columns > lim are in the future
                 float a0 = -INFINITY, a1 = -INFINITY, a2 = -INFINITY, a3 = -INFINITY;
 #pragma unroll
                 for (int qd = 0; qd < 4; ++qd)
@@ -502,13 +508,13 @@ l4l_status launch_t(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensor
 l4l_status launch_prefill_tc(const l4l_tensor4 &q, const l4l_tensor4 &k, const l4l_tensor4 &v,
                              const l4l_tensor4 &o, const l4l_kv_cache &cache, const int32_t *d_seq_lens,
                              int S_max, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
-                             void *workspace, cudaStream_t stream)
+                             void *workspace, cudaStream_t stream, const int32_t *d_past_lens, int kv_extent)
 {
     CUtensorMap tq, tk, tv;
     TmapCoord cq, ck, cv;
     if (!make_tmap_bf16(&tq, &cq, q.ptr, D, S_max, Hq, B, q.stride_t, q.stride_h, q.stride_b, 64, kRows) ||
-        !make_tmap_bf16(&tk, &ck, k.ptr, D, S_max, Hkv, B, k.stride_t, k.stride_h, k.stride_b, 64, kRows) ||
-        !make_tmap_bf16(&tv, &cv, v.ptr, D, S_max, Hkv, B, v.stride_t, v.stride_h, v.stride_b, 64, kRows))
+        !make_tmap_bf16(&tk, &ck, k.ptr, D, kv_extent, Hkv, B, k.stride_t, k.stride_h, k.stride_b, 64, kRows) ||
+        !make_tmap_bf16(&tv, &cv, v.ptr, D, kv_extent, Hkv, B, v.stride_t, v.stride_h, v.stride_b, 64, kRows))
         return L4L_ERR_CUDA;
     if (ck.pos_t != cv.pos_t || ck.pos_h != cv.pos_h || ck.pos_b != cv.pos_b) return L4L_ERR_UNSUPPORTED;
     TcParams p;
@@ -519,6 +525,7 @@ l4l_status launch_prefill_tc(const l4l_tensor4 &q, const l4l_tensor4 &k, const l
     p.c_sb = cache.stride_b; p.c_sh = cache.stride_h; p.c_st = cache.stride_t;
     p.cache_max_len = cache.max_len;
     p.seq_lens = d_seq_lens;
+    p.past_lens = d_past_lens;
     p.lse = d_lse;
     p.status = static_cast<unsigned *>(workspace);
     p.S_max = S_max; p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.G = Hq / Hkv;

@@ -296,6 +296,39 @@ def test_I13_matches_torch_sdpa_float64(B, S, Hq, Hkv, D):
     np.testing.assert_allclose(dout, dref[:, :, 0].numpy(), rtol=0, atol=1e-12)
 
 
+def test_chunk_over_populated_cache_equals_rows_of_the_full_prefill():
+    """Prefill of tokens [P, P+L) over a cache that holds tokens [0, P+L) must give rows P..P+L-1 of the causal
+    prefill of the whole sequence, and with L = 1 it is decode; padding slots must not matter."""
+    B, T, Hq, Hkv, D = 2, 29, 4, 2, 8
+    q, k, v = randn((B, T, Hq, D), 50), randn((B, T, Hkv, D), 51), randn((B, T, Hkv, D), 52)
+    full, full_lse = orc.prefill(q, k, v, full_lens(B, T), 0.33)
+    Lmax = 40
+    ck = torch.full((B, Hkv, Lmax, D), float("nan")).to(torch.bfloat16)
+    cv = ck.clone()
+    ck[:, :, :T], cv[:, :, :T] = cache_from(k), cache_from(v)
+    past = np.array([11, 0], np.int32)
+    qlen = np.array([T - 11, 17], np.int32)
+    S = int(qlen.max())
+    qc = torch.zeros(B, S, Hq, D, dtype=torch.bfloat16)
+    for b in range(B):
+        qc[b, :qlen[b]] = q[b, past[b]:past[b] + qlen[b]]
+    # the second sequence's cache is cut at past+qlen: later slots are poison
+    ck[1, :, 17:], cv[1, :, 17:] = float("nan"), float("nan")
+    out, lse = orc.prefill_chunk(qc, ck, cv, past, qlen, 0.33)
+    for b in range(B):
+        sl = slice(past[b], past[b] + qlen[b])
+        np.testing.assert_allclose(out[b, :qlen[b]], full[b, sl], rtol=0, atol=1e-14)
+        np.testing.assert_allclose(lse[b, :, :qlen[b]], full_lse[b, :, sl], rtol=0, atol=1e-14)
+        assert np.isnan(out[b, qlen[b]:]).all()
+    # one new token over P cached ones is decode with kv_len = P + 1
+    d_out, d_lse = orc.decode(q[:, 20].contiguous(), ck, cv, np.array([21, 17], np.int32), 0.33)
+    c_out, c_lse = orc.prefill_chunk(q[:, 20:21].contiguous(), ck, cv, np.array([20, 16], np.int32),
+                                     np.array([1, 1], np.int32), 0.33)
+    np.testing.assert_allclose(c_out[:, 0], d_out, rtol=0, atol=1e-14)
+    with pytest.raises(ValueError):
+        orc.prefill_chunk(qc, ck, cv, np.array([30, 0], np.int32), qlen, 0.33)       # past + q_len > Lmax
+
+
 def test_prefill_rows_is_the_same_function_as_prefill():
     B, S, Hq, Hkv, D = 2, 21, 4, 2, 8
     q, k, v = randn((B, S, Hq, D), 45), randn((B, S, Hkv, D), 46), randn((B, S, Hkv, D), 47)
