@@ -1,19 +1,20 @@
 // Decode attention: one query token per sequence over a ragged bf16 KV cache.
 //
-// One launch. The cache of every (sequence, KV head) is cut into 64-token tiles; the flattened
-// tile stream (sequence-major, then KV head, then position) is divided EVENLY among persistent
-// CTAs, so every CTA streams the same number of bytes whatever the length mix. A CTA's range may
+// One launch. The cache of every (sequence, KV head) is cut into tiles of 16*W tokens (W = 4 or 8
+// consumer warps); the flattened tile stream (sequence-major, then KV head, then position) is divided
+// among persistent CTAs as evenly as whole tiles allow, so every CTA streams the same number of bytes
+// (to within one tile) whatever the length mix. A CTA's range may
 // start or end inside a sequence: each (sequence, KV head) is thus covered by one or more
 // "pieces", one per CTA that touches it.
 //
 //   producer warp    walks the CTA's tile range and keeps a ring of TMA tiles (K and V, 128-byte
 //                    swizzle) full, across piece boundaries
-//   4 consumer warps each take 16 tokens of every tile and serve ALL query heads of the KV group
+//   W consumer warps each take 16 tokens of every tile and serve ALL query heads of the KV group
 //                    from it: the group is the M dimension (zero-padded to 16) of warp-level bf16
 //                    MMAs, so cache bytes are read once per group. Softmax statistics are fp32;
 //                    row maxima are reduced with warp shuffles. At the end of a piece they drop
 //                    their (max, sum, O) into shared memory and go straight on to the next tile.
-//   finisher warp    merges the four warps' results of a piece off the critical path. A sequence
+//   finisher warp    merges the consumer warps' results of a piece off the critical path. A sequence
 //                    covered by a single piece is written out directly; otherwise the piece's
 //                    normalised fp32 partial and its log-sum-exp go to the workspace, and the LAST
 //                    piece to arrive (a self-resetting ticket counter per (sequence, KV head)) runs
