@@ -102,6 +102,34 @@ l4l_status l4l_kv_append(l4l_kv_cache cache, l4l_tensor4 k_new, l4l_tensor4 v_ne
                          int B, int Hkv, int head_dim, l4l_stream stream);
 
 /*
+ * Rotary position embedding (and optional per-head RMS normalisation of q and k) fused with the
+ * cache update: the projection outputs of the new tokens go through ONE streaming pass that
+ * leaves q ready for the attention calls and K, V in the cache. (The paper's prefill kernel is
+ * described as causal attention "with fused QKV wiring" and its decode path as keeping the cache
+ * update's tensor contract; the paper prints no formula for the rotation, so the reading is the
+ * half-split convention of the Llama / Qwen3 modules it names.) For sequence b, new token
+ * t < n_new[b] at position P = pos[b] + t, every head row x of q and k_new (D values):
+ *     if a norm weight w is given:   x[d] <- x[d] / sqrt(mean_d(x[d]^2) + eps) * w[d]
+ *     for i < D/2:   y[i]       = x[i] * cos[P, i] - x[i + D/2] * sin[P, i]
+ *                    y[i + D/2] = x[i + D/2] * cos[P, i] + x[i] * sin[P, i]
+ * computed in fp32 and rounded once to bf16 (round to nearest even). q is overwritten with its y;
+ * cache_k slot P of (b, kv head) receives k_new's y; cache_v slot P receives v_new bit for bit.
+ * Tokens whose position falls outside [0, min(cache.max_len, n_pos)) are skipped entirely (q row
+ * left as it was, nothing written). Afterwards: l4l_attn_prefill_chunk(q, ..., past = pos,
+ * q_lens = n_new) for a prompt or a chunk, l4l_attn_decode for single tokens.
+ *   q            [B, T, Hq, D] view, read and written     k_new, v_new  [B, T, Hkv, D] views, read
+ *   d_pos        device int32 [B]      d_n_new  device int32 [B] or NULL (= T for all)
+ *   d_cos, d_sin device float [n_pos, D/2], row P holding cos / sin of P * theta_i
+ *   d_q_weight, d_k_weight   device float [D] or NULL (no normalisation of that tensor)
+ */
+l4l_status l4l_rope_kv_append(l4l_tensor4 q, l4l_tensor4 k_new, l4l_tensor4 v_new, l4l_kv_cache cache,
+                              const int32_t *d_pos, const int32_t *d_n_new, int T,
+                              int B, int Hq, int Hkv, int head_dim,
+                              const float *d_cos, const float *d_sin, int n_pos,
+                              const float *d_q_weight, const float *d_k_weight, float norm_eps,
+                              l4l_stream stream);
+
+/*
  * Causal prefill. For every sequence b with L = seq_lens[b] tokens, query head h, row i < L:
  *     o[b, i, h, :] = softmax_j( scale * q[b, i, h, :] . k[b, j, h/G, :],  j = 0..i ) @ v[b, 0..i, h/G, :]
  * and, when cache.k != NULL, cache slots 0..L-1 of sequence b receive k and v bit for bit

@@ -220,6 +220,105 @@ int l4l_oracle_prefill_chunk(const uint16_t *q, const uint16_t *cache_k, const u
     return fail ? -1 : 0;
 }
 
+/* Round an fp64 value to bf16: to nearest, ties to even; overflow goes to infinity, NaN stays NaN. */
+static uint16_t f64_to_bf16(double x)
+{
+    float f;
+    uint32_t u;
+    if (x != x) return 0x7FC0;
+    if (x != 0.0 && !isinf(x)) {
+        int e;
+        (void)frexp(fabs(x), &e);                                 /* |x| = m 2^e with 0.5 <= m < 1 */
+        /* spacing of the bf16 values around |x|: 8 significant bits, subnormals below 2^-126 */
+        const double quantum = ldexp(1.0, (e - 8 < -133) ? -133 : e - 8);
+        const double r = nearbyint(fabs(x) / quantum) * quantum; /* ties to even (default rounding mode) */
+        x = x < 0 ? -r : r;                                       /* now exactly a bf16 value, or 2^128 */
+    }
+    f = (float)x;
+    memcpy(&u, &f, sizeof u);
+    return (uint16_t)(u >> 16);
+}
+
+/* Exposed for the tests that pin the rounding against a library conversion. */
+void l4l_oracle_round_bf16(const double *x, uint16_t *out, int64_t n)
+{
+    for (int64_t i = 0; i < n; ++i) out[i] = f64_to_bf16(x[i]);
+}
+
+/*
+ * Rotary position embedding with optional per-head RMS normalisation, for ONE head row.
+ * Half-split convention: element i < D/2 is paired with element i + D/2;
+ *     y[i]       = x[i] cos_i - x[i + D/2] sin_i,     y[i + D/2] = x[i + D/2] cos_i + x[i] sin_i
+ * and, before that, when w != NULL:  x[d] <- x[d] / sqrt(mean_d x[d]^2 + eps) * w[d].
+ * Everything in fp64; `y` receives the unrounded result.
+ */
+static void rope_row(const uint16_t *x, int D, const float *cosr, const float *sinr, const float *w, double eps,
+                     double *y)
+{
+    double xs[256];
+    double ss = 0.0;
+    for (int d = 0; d < D; ++d) {
+        xs[d] = bf16_to_f64(x[d]);
+        ss += xs[d] * xs[d];
+    }
+    if (w) {
+        const double r = 1.0 / sqrt(ss / D + eps);
+        for (int d = 0; d < D; ++d) xs[d] = xs[d] * r * (double)w[d];
+    }
+    const int H = D / 2;
+    for (int i = 0; i < H; ++i) {
+        const double c = (double)cosr[i], sn = (double)sinr[i];
+        y[i] = xs[i] * c - xs[i + H] * sn;
+        y[i + H] = xs[i + H] * c + xs[i] * sn;
+    }
+}
+
+/*
+ * Rotary embedding (+ optional RMS normalisation) of the new tokens' q and k, fused with the cache
+ * update: token t < n_new[b] of sequence b sits at position P = pos[b] + t; its q rows are replaced
+ * by their rotated values, its rotated k rows and its v rows (bit for bit) go to cache slot P.
+ * Tokens with P outside [0, min(Lmax, n_pos)) are skipped.
+ *   q [B,T,Hq,D] in/out (bf16 bits)   k_new, v_new [B,T,Hkv,D]   caches [B,Hkv,Lmax,D] in/out
+ *   cos, sin [n_pos, D/2] fp32        q_w, k_w [D] fp32 or NULL
+ *   q_exact [B,T,Hq,D], k_exact [B,T,Hkv,D]: the unrounded fp64 results (or NULL); skipped rows untouched
+ */
+int l4l_oracle_rope_kv_append(uint16_t *q, const uint16_t *k_new, const uint16_t *v_new, uint16_t *cache_k,
+                              uint16_t *cache_v, const int32_t *pos, const int32_t *n_new, int B, int T, int Hq,
+                              int Hkv, int D, int Lmax, const float *cosv, const float *sinv, int n_pos,
+                              const float *q_w, const float *k_w, double eps, double *q_exact, double *k_exact)
+{
+    if (D <= 0 || D > 256 || (D & 1)) return -1;
+    const int lim = Lmax < n_pos ? Lmax : n_pos;
+    double y[256];
+    for (int b = 0; b < B; ++b) {
+        const int n = n_new ? n_new[b] : T;
+        for (int t = 0; t < T && t < n; ++t) {
+            const int64_t P = (int64_t)pos[b] + t;
+            if (P < 0 || P >= lim) continue;
+            const float *cr = cosv + P * (D / 2), *sr = sinv + P * (D / 2);
+            for (int h = 0; h < Hq; ++h) {
+                uint16_t *row = q + (((int64_t)b * T + t) * Hq + h) * D;
+                rope_row(row, D, cr, sr, q_w, eps, y);
+                for (int d = 0; d < D; ++d) {
+                    row[d] = f64_to_bf16(y[d]);
+                    if (q_exact) q_exact[(((int64_t)b * T + t) * Hq + h) * D + d] = y[d];
+                }
+            }
+            for (int g = 0; g < Hkv; ++g) {
+                const int64_t src = (((int64_t)b * T + t) * Hkv + g) * D;
+                const int64_t dst = (((int64_t)b * Hkv + g) * Lmax + P) * D;
+                rope_row(k_new + src, D, cr, sr, k_w, eps, y);
+                for (int d = 0; d < D; ++d) {
+                    cache_k[dst + d] = f64_to_bf16(y[d]);
+                    if (k_exact) k_exact[src + d] = y[d];
+                }
+                memcpy(cache_v + dst, v_new + src, sizeof(uint16_t) * (size_t)D);
+            }
+        }
+    }
+    return 0;
+}
+
 /*
  * Decode: one query token per sequence over the populated cache (no mask).
  *   q        [B, Hq, D]           cache_k, cache_v  [B, Hkv, Lmax, D]

@@ -47,6 +47,11 @@ def _load():
                                                 i32p, i, f64p, f64p]
         lib.l4l_oracle_decode.argtypes = [u16p, u16p, u16p, i32p, i, i, i, i, i, d, f64p, f64p]
         lib.l4l_oracle_prefill_chunk.argtypes = [u16p, u16p, u16p, i32p, i32p, i, i, i, i, i, i, d, f64p, f64p]
+        f32p = ctypes.POINTER(ctypes.c_float)
+        lib.l4l_oracle_round_bf16.argtypes = [f64p, u16p, ctypes.c_int64]
+        lib.l4l_oracle_round_bf16.restype = None
+        lib.l4l_oracle_rope_kv_append.argtypes = [u16p, u16p, u16p, u16p, u16p, i32p, i32p, i, i, i, i, i, i,
+                                                  f32p, f32p, i, f32p, f32p, d, f64p, f64p]
         lib.l4l_oracle_kv_append.argtypes = [u16p, u16p, u16p, u16p, i32p, i32p, i, i, i, i, i]
         _lib = lib
     return _lib
@@ -170,3 +175,43 @@ def kv_append(cache_k, cache_v, k_new, v_new, pos, n_new):
     if rc != 0:
         raise ValueError("l4l_oracle_kv_append: write outside the cache")
     return ck, cv
+
+
+def round_bf16(x) -> np.ndarray:
+    """fp64 array -> bf16 bits (uint16), round to nearest even."""
+    x = np.ascontiguousarray(np.asarray(x, dtype=np.float64))
+    out = np.empty(x.shape, dtype=np.uint16)
+    _load().l4l_oracle_round_bf16(_p(x, ctypes.c_double), _p(out, ctypes.c_uint16), x.size)
+    return out
+
+
+def rope_kv_append(q, k_new, v_new, cache_k, cache_v, pos, n_new, cos, sin, q_weight=None, k_weight=None,
+                   eps: float = 0.0):
+    """Rotary embedding (+ optional RMS norm) of q and k fused with the cache update.
+
+    q [B,T,Hq,D], k_new/v_new [B,T,Hkv,D], caches [B,Hkv,Lmax,D], cos/sin float32 [n_pos, D/2].
+    Returns (q_bits, cache_k_bits, cache_v_bits, q_exact, k_exact): the first three as uint16 bf16 bits after
+    the update, the last two the unrounded fp64 rotations (NaN in skipped rows)."""
+    qb, kn, vn = bits(q).copy(), bits(k_new), bits(v_new)
+    ck, cv = bits(cache_k).copy(), bits(cache_v).copy()
+    B, T, Hq, D = qb.shape
+    Hkv, Lmax = ck.shape[1], ck.shape[2]
+    assert kn.shape == (B, T, Hkv, D) and vn.shape == kn.shape and ck.shape == (B, Hkv, Lmax, D)
+    cos = np.ascontiguousarray(np.asarray(cos, dtype=np.float32))
+    sin = np.ascontiguousarray(np.asarray(sin, dtype=np.float32))
+    assert cos.shape == sin.shape and cos.shape[1] == D // 2
+    pos = _i32(pos)
+    n_new = _i32(n_new) if n_new is not None else np.full((B,), T, np.int32)
+    f32 = ctypes.c_float
+    qw = None if q_weight is None else np.ascontiguousarray(np.asarray(q_weight, dtype=np.float32))
+    kw = None if k_weight is None else np.ascontiguousarray(np.asarray(k_weight, dtype=np.float32))
+    q_exact = np.full(qb.shape, np.nan)
+    k_exact = np.full(kn.shape, np.nan)
+    rc = _load().l4l_oracle_rope_kv_append(
+        _p(qb, ctypes.c_uint16), _p(kn, ctypes.c_uint16), _p(vn, ctypes.c_uint16), _p(ck, ctypes.c_uint16),
+        _p(cv, ctypes.c_uint16), _p(pos, ctypes.c_int32), _p(n_new, ctypes.c_int32), B, T, Hq, Hkv, D, Lmax,
+        _p(cos, f32), _p(sin, f32), cos.shape[0], None if qw is None else _p(qw, f32),
+        None if kw is None else _p(kw, f32), float(eps), _p(q_exact, ctypes.c_double), _p(k_exact, ctypes.c_double))
+    if rc != 0:
+        raise ValueError("l4l_oracle_rope_kv_append rejected its arguments")
+    return qb, ck, cv, q_exact, k_exact

@@ -22,7 +22,7 @@ L4L_OP_PREFILL, L4L_OP_DECODE = 0, 1
 EXPORTS = (
     "l4l_version", "l4l_status_string", "l4l_workspace_bytes", "l4l_workspace_init",
     "l4l_last_device_error", "l4l_kv_append", "l4l_attn_prefill", "l4l_attn_decode",
-    "l4l_attn_decode_static", "l4l_attn_decode_append", "l4l_attn_prefill_chunk",
+    "l4l_attn_decode_static", "l4l_attn_decode_append", "l4l_attn_prefill_chunk", "l4l_rope_kv_append",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -76,6 +76,9 @@ def load() -> ctypes.CDLL:
     lib.l4l_attn_decode_static.restype = c_int
     lib.l4l_attn_decode_static.argtypes = [vp, vp, KVCache, i32p, c_int, c_int, c_int, c_int, c_int, ctypes.c_float, vp,
                                            vp]
+    lib.l4l_rope_kv_append.restype = c_int
+    lib.l4l_rope_kv_append.argtypes = [Tensor4, Tensor4, Tensor4, KVCache, i32p, i32p, c_int, c_int, c_int, c_int, c_int,
+                                       vp, vp, c_int, vp, vp, ctypes.c_float, vp]
     lib.l4l_attn_prefill_chunk.restype = c_int
     lib.l4l_attn_prefill_chunk.argtypes = [Tensor4, Tensor4, KVCache, i32p, i32p, c_int, c_int, c_int, c_int, c_int,
                                            ctypes.c_float, vp, vp, c_size, vp]
@@ -258,3 +261,31 @@ def l4l_attn_prefill_chunk(q, o, cache_k, cache_v, past_lens, q_lens, scale: flo
                                        workspace.numel() * workspace.element_size(), _stream())
     if st != L4L_OK:
         raise L4LError(st, "l4l_attn_prefill_chunk")
+
+
+def _f32_dev(t, name: str, shape=None):
+    if t is None:
+        return None
+    if not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()):
+        raise TypeError(f"{name} must be a contiguous CUDA float32 tensor")
+    if shape is not None and tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name} must have shape {tuple(shape)}")
+    return t.data_ptr()
+
+
+def l4l_rope_kv_append(q, k_new, v_new, cache_k, cache_v, pos, n_new, cos, sin, q_weight=None, k_weight=None,
+                       eps: float = 0.0) -> None:
+    """Rotary embedding (+ optional per-head RMS norm) of q (in place) and k, with K and V written to the cache.
+    q [B,T,Hq,D]; k_new, v_new [B,T,Hkv,D]; pos CUDA int32 [B]; n_new CUDA int32 [B] or None;
+    cos, sin CUDA float32 [n_pos, D/2]; q_weight, k_weight CUDA float32 [D] or None."""
+    B, T, Hq, D = q.shape
+    Hkv = k_new.shape[2]
+    n_pos = cos.shape[0]
+    st = load().l4l_rope_kv_append(tensor4(q, "q"), tensor4(k_new, "k_new"), tensor4(v_new, "v_new"),
+                                   kv_cache(cache_k, cache_v), _i32_dev(pos, "pos"),
+                                   None if n_new is None else _i32_dev(n_new, "n_new"), T, B, Hq, Hkv, D,
+                                   _f32_dev(cos, "cos", (n_pos, D // 2)), _f32_dev(sin, "sin", (n_pos, D // 2)), n_pos,
+                                   _f32_dev(q_weight, "q_weight", (D,)), _f32_dev(k_weight, "k_weight", (D,)),
+                                   float(eps), _stream())
+    if st != L4L_OK:
+        raise L4LError(st, "l4l_rope_kv_append")

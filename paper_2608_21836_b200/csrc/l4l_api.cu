@@ -211,6 +211,22 @@ l4l_status l4l_kv_append(l4l_kv_cache cache, l4l_tensor4 k_new, l4l_tensor4 v_ne
                             static_cast<cudaStream_t>(stream));
 }
 
+l4l_status l4l_rope_kv_append(l4l_tensor4 q, l4l_tensor4 k_new, l4l_tensor4 v_new, l4l_kv_cache cache,
+                              const int32_t *d_pos, const int32_t *d_n_new, int T, int B, int Hq, int Hkv, int head_dim,
+                              const float *d_cos, const float *d_sin, int n_pos, const float *d_q_weight,
+                              const float *d_k_weight, float norm_eps, l4l_stream stream)
+{
+    l4l_status st = shape_status(B, Hq, Hkv, head_dim);
+    if (st != L4L_OK) return st;
+    if (T < 0 || n_pos < 0 || !d_pos || !d_cos || !d_sin || !(norm_eps >= 0.f)) return L4L_ERR_INVALID_ARG;
+    if (!tensor4_ok(q) || !tensor4_ok(k_new) || !tensor4_ok(v_new) || !cache_ok(cache)) return L4L_ERR_INVALID_ARG;
+    if (!aligned16(d_cos) || !aligned16(d_sin) || !aligned16(d_q_weight) || !aligned16(d_k_weight))
+        return L4L_ERR_INVALID_ARG;
+    if (B == 0 || T == 0) return L4L_OK;
+    return launch_rope_kv_append(q, k_new, v_new, cache, d_pos, d_n_new, T, B, Hq, Hkv, head_dim, d_cos, d_sin, n_pos,
+                                 d_q_weight, d_k_weight, norm_eps, static_cast<cudaStream_t>(stream));
+}
+
 l4l_status l4l_attn_prefill(l4l_tensor4 q, l4l_tensor4 k, l4l_tensor4 v, l4l_tensor4 o, l4l_kv_cache cache,
                             const int32_t *d_seq_lens, int S_max, int B, int Hq, int Hkv, int head_dim, float scale,
                             float *d_lse, void *workspace, size_t ws_bytes, l4l_stream stream)

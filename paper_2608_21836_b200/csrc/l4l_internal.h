@@ -39,6 +39,10 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
                          void *workspace, const DecodePlan &plan, cudaStream_t stream,
                          const l4l_tensor4 *k_new = nullptr, const l4l_tensor4 *v_new = nullptr);
 
+l4l_status launch_rope_kv_append(const l4l_tensor4 &q, const l4l_tensor4 &k_new, const l4l_tensor4 &v_new,
+                                 const l4l_kv_cache &cache, const int32_t *d_pos, const int32_t *d_n_new, int T, int B,
+                                 int Hq, int Hkv, int D, const float *d_cos, const float *d_sin, int n_pos,
+                                 const float *d_q_weight, const float *d_k_weight, float norm_eps, cudaStream_t stream);
 l4l_status launch_kv_append(const l4l_kv_cache &cache, const l4l_tensor4 &k_new, const l4l_tensor4 &v_new,
                             const int32_t *d_write_pos, const int32_t *d_n_new, int n_new_max, int B, int Hkv,
                             int D, cudaStream_t stream);

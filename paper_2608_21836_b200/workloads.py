@@ -148,3 +148,13 @@ def prefill_flops(Hq: int, D: int, seq_lens) -> int:
 def decode_kv_bytes(Hkv: int, D: int, kv_lens) -> int:
     """Algorithmic traffic of decode: K and V of every cached token read once (bf16)."""
     return sum(int(L) * 2 * Hkv * D * 2 for L in kv_lens)
+
+
+def make_rope_tables(n_pos: int, D: int, base: float = 10000.0):
+    """cos / sin tables [n_pos, D/2] (float32) of angle P * base^(-2i/D): inputs of the rotary step, computed
+    in float64 and rounded once, as the models' rotary-embedding module hands them to the attention module."""
+    import numpy as np
+
+    inv_freq = base ** (-np.arange(0, D, 2, dtype=np.float64) / D)
+    ang = np.arange(n_pos, dtype=np.float64)[:, None] * inv_freq[None, :]
+    return torch.from_numpy(np.cos(ang).astype(np.float32)), torch.from_numpy(np.sin(ang).astype(np.float32))

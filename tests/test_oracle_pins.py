@@ -367,3 +367,108 @@ def test_kv_append_is_a_bit_exact_copy_and_touches_nothing_else():
 
 def test_oracle_reports_thread_count():
     assert orc.num_threads() >= 1
+
+
+# --------------------------------------------------------------------------- rotary embedding + RMS norm + cache update
+def _rope_inputs(B=2, T=7, Hq=4, Hkv=2, D=16, Lmax=24, n_pos=32, seed=90):
+    from paper_2608_21836_b200.workloads import make_rope_tables
+
+    q, k, v = randn((B, T, Hq, D), seed), randn((B, T, Hkv, D), seed + 1), randn((B, T, Hkv, D), seed + 2)
+    ck = torch.full((B, Hkv, Lmax, D), 3.0).to(torch.bfloat16)
+    cv = torch.full((B, Hkv, Lmax, D), 5.0).to(torch.bfloat16)
+    cos, sin = make_rope_tables(n_pos, D)
+    return q, k, v, ck, cv, cos.numpy(), sin.numpy()
+
+
+def test_bf16_rounding_matches_the_library_conversion():
+    """The oracle's fp64 -> bf16 rounding against torch's float32 -> bfloat16 (RNE), ties and extremes included."""
+    g = torch.Generator().manual_seed(5)
+    x = torch.randn(20000, generator=g) * torch.exp(torch.randn(20000, generator=g) * 8)
+    ties = torch.tensor([1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, -(2.0 + 2.0 ** -7), 1.0 + 2.0 ** -8 + 2.0 ** -20,
+                         0.0, -0.0, 3.3895313892515355e38, float("inf"), 2.0 ** -130, 1e-40])
+    x = torch.cat([x, ties])
+    want = x.to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    got = orc.round_bf16(x.double().numpy())
+    assert np.array_equal(got, want)
+    # a value just above a tie in fp64 that fp32 cannot distinguish from the tie must round up
+    assert orc.round_bf16(np.array([1.0 + 2.0 ** -8 + 2.0 ** -40]))[0] == 0x3F81
+
+
+def test_rope_is_a_complex_rotation_and_keeps_relative_position():
+    q, k, v, ck, cv, cos, sin = _rope_inputs()
+    B, T, Hq, D = q.shape
+    pos = np.array([3, 0], np.int32)
+    qb, ckb, cvb, q_ex, k_ex = orc.rope_kv_append(q, k, v, ck, cv, pos, None, cos, sin)
+    H = D // 2
+    # (x_i, x_{i+D/2}) as a complex number times e^{i P theta_i}, with numpy's complex product
+    for b in range(B):
+        for t in range(T):
+            P = pos[b] + t
+            z = f64(q)[b, t, :, :H] + 1j * f64(q)[b, t, :, H:]
+            w = z * (cos[P].astype(np.float64) + 1j * sin[P].astype(np.float64))[None, :]
+            np.testing.assert_allclose(q_ex[b, t, :, :H], w.real, rtol=0, atol=1e-14)
+            np.testing.assert_allclose(q_ex[b, t, :, H:], w.imag, rtol=0, atol=1e-14)
+    # a rotation keeps the length of every pair
+    np.testing.assert_allclose(k_ex[..., :H] ** 2 + k_ex[..., H:] ** 2, f64(k)[..., :H] ** 2 + f64(k)[..., H:] ** 2,
+                               rtol=1e-6, atol=0)        # tables are float32: cos^2 + sin^2 = 1 to ~1e-7
+    # position 0 is the identity, bit for bit after rounding
+    assert np.array_equal(qb[1, 0], orc.bits(q)[1, 0])
+    # relative position: <rope(q, m), rope(k, n)> depends on m - n only (same vectors placed 5 positions later)
+    q1, k1 = q[:1, :1].contiguous(), k[:1, :1].contiguous()
+    dots = []
+    for shift in (0, 5, 11):
+        _, _, _, qe, _ = orc.rope_kv_append(q1, k1, v[:1, :1].contiguous(), ck[:1], cv[:1], [7 + shift], None, cos, sin)
+        _, _, _, _, ke = orc.rope_kv_append(q1, k1, v[:1, :1].contiguous(), ck[:1], cv[:1], [2 + shift], None, cos, sin)
+        dots.append(np.einsum("d,d->", qe[0, 0, 0], ke[0, 0, 0]))
+    np.testing.assert_allclose(dots[1:], dots[0], rtol=0, atol=2e-5)
+
+
+def test_rope_append_writes_the_right_slots_and_nothing_else():
+    q, k, v, ck, cv, cos, sin = _rope_inputs()
+    B, T, Hq, D = q.shape
+    Lmax = ck.shape[2]
+    pos = np.array([20, 1], np.int32)                    # sequence 0 runs off the cache after 4 tokens
+    n_new = np.array([7, 3], np.int32)
+    qb, ckb, cvb, q_ex, k_ex = orc.rope_kv_append(q, k, v, ck, cv, pos, n_new, cos, sin)
+    vb, ck0, cv0 = orc.bits(v), orc.bits(ck), orc.bits(cv)
+    for b in range(B):
+        written = [pos[b] + t for t in range(n_new[b]) if pos[b] + t < Lmax]
+        for slot in range(Lmax):
+            if slot in written:
+                t = slot - pos[b]
+                assert np.array_equal(cvb[b, :, slot], vb[b, t])                 # v: exact copy
+                assert np.array_equal(ckb[b, :, slot], orc.round_bf16(k_ex[b, t]))
+            else:
+                assert np.array_equal(ckb[b, :, slot], ck0[b, :, slot]) and np.array_equal(cvb[b, :, slot], cv0[b, :, slot])
+        for t in range(T):
+            if t < n_new[b] and pos[b] + t < Lmax:
+                assert np.array_equal(qb[b, t], orc.round_bf16(q_ex[b, t]))
+            else:
+                assert np.array_equal(qb[b, t], orc.bits(q)[b, t]) and np.isnan(q_ex[b, t]).all()
+
+
+def test_rms_norm_part_of_rope_has_unit_rms_scale_invariance_and_weight_linearity():
+    q, k, v, ck, cv, cos, sin = _rope_inputs(D=32)
+    D = q.shape[-1]
+    ones = np.ones(D, np.float32)
+    pos = np.array([0, 0], np.int32)
+    # at position 0 the rotation is the identity, so the exact output is the normalised row
+    _, _, _, qn, kn = orc.rope_kv_append(q[:, :1].contiguous(), k[:, :1].contiguous(), v[:, :1].contiguous(), ck, cv,
+                                         pos, None, cos, sin, q_weight=ones, k_weight=ones, eps=0.0)
+    np.testing.assert_allclose(np.sqrt((qn ** 2).mean(-1)), 1.0, rtol=1e-13)
+    np.testing.assert_allclose(np.sqrt((kn ** 2).mean(-1)), 1.0, rtol=1e-13)
+    # scaling the input by a power of two (exact in bf16) changes nothing when eps = 0
+    _, _, _, qn4, _ = orc.rope_kv_append((q[:, :1] * 4).contiguous(), k[:, :1].contiguous(), v[:, :1].contiguous(), ck,
+                                         cv, pos, None, cos, sin, q_weight=ones, k_weight=ones, eps=0.0)
+    np.testing.assert_allclose(qn4, qn, rtol=1e-14)
+    # the weight multiplies element-wise; k without a weight is left un-normalised
+    w = np.linspace(0.5, 2.0, D).astype(np.float32)
+    _, _, _, qw, kraw = orc.rope_kv_append(q[:, :1].contiguous(), k[:, :1].contiguous(), v[:, :1].contiguous(), ck, cv,
+                                           pos, None, cos, sin, q_weight=w, k_weight=None, eps=0.0)
+    np.testing.assert_allclose(qw, qn * w.astype(np.float64), rtol=1e-14)
+    np.testing.assert_allclose(kraw, f64(k[:, :1]), rtol=0, atol=0)
+    # eps enters under the root: a row of constant c gives c / sqrt(c^2 + eps)
+    const = torch.full((1, 1, 1, D), 0.5).to(torch.bfloat16)
+    _, _, _, qc, _ = orc.rope_kv_append(const, const, const, ck[:1, :1], cv[:1, :1], [0], None, cos, sin,
+                                        q_weight=ones, eps=0.75)
+    np.testing.assert_allclose(qc, 0.5 / math.sqrt(0.25 + 0.75), rtol=1e-14)
