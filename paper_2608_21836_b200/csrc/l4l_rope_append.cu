@@ -48,16 +48,16 @@ __global__ void __launch_bounds__(256) rope_kv_append_kernel(const RopeParams p)
     constexpr int kLanes = D / 16;                  // lanes per head row
     constexpr int kHalfPieces = D / 16;             // 16-byte pieces per half row
     const int heads = p.Hq + 2 * p.Hkv;             // q heads, then k heads, then v heads
-    const long long rows = (long long)p.B * p.T * heads;
+    const unsigned rows = (unsigned)p.B * p.T * heads;        // < 2^31, checked by the launcher
     const int u = threadIdx.x % kLanes;
     const uint32_t group_mask = ((1u << kLanes) - 1u) << ((threadIdx.x & 31) & ~(kLanes - 1));
-    const long long first = (blockIdx.x * (long long)blockDim.x + threadIdx.x) / kLanes;
-    const long long step = (long long)gridDim.x * blockDim.x / kLanes;
+    const unsigned first = (blockIdx.x * blockDim.x + threadIdx.x) / kLanes;
+    const unsigned step = gridDim.x * blockDim.x / kLanes;
     // all lanes of a row group take the same trips through the loop (rows is tested per group)
-    for (long long r = first; r < rows; r += step) {
-        const int hh = (int)(r % heads);
-        const long long bt = r / heads;
-        const int t = (int)(bt % p.T), b = (int)(bt / p.T);
+    for (unsigned r = first; r < rows; r += step) {
+        const int hh = (int)(r % (unsigned)heads);
+        const unsigned bt = r / (unsigned)heads;
+        const int t = (int)(bt % (unsigned)p.T), b = (int)(bt / (unsigned)p.T);
         const int n = p.n_new ? p.n_new[b] : p.T;
         const long long P = (long long)p.pos[b] + t;
         // the lanes of a row group skip together, so the group-masked shuffles below see the full group
@@ -141,7 +141,9 @@ l4l_status launch_rope_kv_append(const l4l_tensor4 &q, const l4l_tensor4 &k_new,
     p.eps = norm_eps;
     p.B = B; p.T = T; p.Hq = Hq; p.Hkv = Hkv;
     p.max_pos = cache.max_len < n_pos ? cache.max_len : n_pos;
-    const long long threads = (long long)B * T * (Hq + 2 * Hkv) * (D / 16);
+    const long long rows = (long long)B * T * (Hq + 2 * Hkv);
+    if (rows >= (1ll << 31) - (1ll << 24)) return L4L_ERR_UNSUPPORTED;   // the kernel indexes rows in 32 bits
+    const long long threads = rows * (D / 16);
     long long blocks = (threads + 255) / 256;
     const long long cap = 16ll * sm_count();      // grid-stride beyond that: 8 resident blocks per SM, two waves
     if (blocks > cap) blocks = cap;
