@@ -71,6 +71,21 @@ typedef struct {
     int32_t max_len;
 } l4l_kv_cache;
 
+/*
+ * A paged KV cache: a pool of fixed-size pages, element (page, kv head g, slot t, d) at
+ * k + page*stride_page + g*stride_h + t*stride_t + d. A per-sequence block table (device int32,
+ * [B, table_stride]) names the page that holds tokens [i*page_size, (i+1)*page_size) of a
+ * sequence in entry i. page_size must be a power of two >= 16. The dense layout is
+ * [num_pages, Hkv, page_size, D].
+ */
+typedef struct {
+    void *k;
+    void *v;
+    int64_t stride_page, stride_h, stride_t;
+    int32_t page_size;
+    int32_t num_pages;
+} l4l_paged_kv;
+
 enum { L4L_OP_PREFILL = 0, L4L_OP_DECODE = 1 };
 
 /*
@@ -100,6 +115,28 @@ l4l_status l4l_workspace_init(void *workspace, size_t ws_bytes, l4l_stream strea
 l4l_status l4l_kv_append(l4l_kv_cache cache, l4l_tensor4 k_new, l4l_tensor4 v_new,
                          const int32_t *d_write_pos, const int32_t *d_n_new, int n_new_max,
                          int B, int Hkv, int head_dim, l4l_stream stream);
+
+/*
+ * The same two operations over a paged cache (what serving runtimes hold: the paper's related-work
+ * discussion of KV-cache management; the paper's own kernels read a contiguous cache, so this
+ * layout has no counterpart there). Results are those of l4l_kv_append / l4l_attn_decode on the
+ * contiguous cache one gets by laying every sequence's pages end to end.
+ *   l4l_kv_append_paged : token slot s of sequence b goes to page block_table[b][s / page_size],
+ *                         offset s % page_size; slots beyond table_stride * page_size and slots
+ *                         whose table entry is outside [0, num_pages) are dropped.
+ *   l4l_attn_decode_paged : kv_lens[b] <= table_stride * page_size; a table entry outside
+ *                         [0, num_pages) reads as zeros (never as memory); entries past the last
+ *                         token of a sequence are not looked at. Workspace as for l4l_attn_decode
+ *                         with max_len = max_kv_len.
+ */
+l4l_status l4l_kv_append_paged(l4l_paged_kv pool, const int32_t *d_block_table, int table_stride,
+                               l4l_tensor4 k_new, l4l_tensor4 v_new, const int32_t *d_write_pos,
+                               const int32_t *d_n_new, int n_new_max, int B, int Hkv, int head_dim,
+                               l4l_stream stream);
+l4l_status l4l_attn_decode_paged(const void *q, void *o, l4l_paged_kv pool, const int32_t *d_block_table,
+                                 int table_stride, const int32_t *d_kv_lens, int max_kv_len,
+                                 int B, int Hq, int Hkv, int head_dim, float scale, float *d_lse,
+                                 void *workspace, size_t ws_bytes, l4l_stream stream);
 
 /*
  * Rotary position embedding (and optional per-head RMS normalisation of q and k) fused with the

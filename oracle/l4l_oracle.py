@@ -215,3 +215,49 @@ def rope_kv_append(q, k_new, v_new, cache_k, cache_v, pos, n_new, cos, sin, q_we
     if rc != 0:
         raise ValueError("l4l_oracle_rope_kv_append rejected its arguments")
     return qb, ck, cv, q_exact, k_exact
+
+
+def gather_pages(pool, block_table, n_slots: int) -> np.ndarray:
+    """Paged cache -> the contiguous cache it stands for. pool [pages, Hkv, page_size, D] (bf16 bits or tensor),
+    block_table [B, n] ints; returns uint16 [B, Hkv, n_slots, D]: slot s of sequence b is row s % page_size of page
+    block_table[b, s // page_size]. Entries outside the pool read as zeros (as the GPU path defines)."""
+    pb = bits(pool)
+    n_pages, Hkv, page, D = pb.shape
+    bt = np.asarray(block_table, dtype=np.int64)
+    B = bt.shape[0]
+    out = np.zeros((B, Hkv, n_slots, D), dtype=np.uint16)
+    for b in range(B):
+        for s0 in range(0, n_slots, page):
+            pg = bt[b, s0 // page] if s0 // page < bt.shape[1] else -1
+            if 0 <= pg < n_pages:
+                n = min(page, n_slots - s0)
+                out[b, :, s0:s0 + n] = pb[pg, :, :n]
+    return out
+
+
+def decode_paged(q, pool_k, pool_v, block_table, kv_len, scale: float):
+    """Decode over a paged cache = decode over the gathered contiguous cache."""
+    kl = _i32(kv_len)
+    n_slots = max(int(kl.max()) if kl.size else 0, 1)
+    return decode(q, gather_pages(pool_k, block_table, n_slots), gather_pages(pool_v, block_table, n_slots), kl, scale)
+
+
+def kv_append_paged(pool_k, pool_v, block_table, k_new, v_new, pos, n_new):
+    """Returns copies of the pools (uint16 bits) with the new tokens written to their pages."""
+    pk, pv = bits(pool_k).copy(), bits(pool_v).copy()
+    kn, vn = bits(k_new), bits(v_new)
+    n_pages, Hkv, page, D = pk.shape
+    bt = np.asarray(block_table, dtype=np.int64)
+    B, T = kn.shape[0], kn.shape[1]
+    pos = _i32(pos)
+    n_new = _i32(n_new) if n_new is not None else np.full((B,), T, np.int32)
+    for b in range(B):
+        for t in range(min(T, int(n_new[b]))):
+            s = int(pos[b]) + t
+            if s < 0 or s // page >= bt.shape[1]:
+                continue
+            pg = bt[b, s // page]
+            if 0 <= pg < n_pages:
+                pk[pg, :, s % page] = kn[b, t]
+                pv[pg, :, s % page] = vn[b, t]
+    return pk, pv

@@ -23,6 +23,7 @@ EXPORTS = (
     "l4l_version", "l4l_status_string", "l4l_workspace_bytes", "l4l_workspace_init",
     "l4l_last_device_error", "l4l_kv_append", "l4l_attn_prefill", "l4l_attn_decode",
     "l4l_attn_decode_static", "l4l_attn_decode_append", "l4l_attn_prefill_chunk", "l4l_rope_kv_append",
+    "l4l_kv_append_paged", "l4l_attn_decode_paged",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -30,6 +31,12 @@ STATIC_SCRATCH_BYTES = 8 << 20
 class Tensor4(ctypes.Structure):
     _fields_ = [("ptr", ctypes.c_void_p), ("stride_b", ctypes.c_int64), ("stride_t", ctypes.c_int64),
                 ("stride_h", ctypes.c_int64)]
+
+
+class PagedKV(ctypes.Structure):
+    _fields_ = [("k", ctypes.c_void_p), ("v", ctypes.c_void_p), ("stride_page", ctypes.c_int64),
+                ("stride_h", ctypes.c_int64), ("stride_t", ctypes.c_int64), ("page_size", ctypes.c_int32),
+                ("num_pages", ctypes.c_int32)]
 
 
 class KVCache(ctypes.Structure):
@@ -76,6 +83,11 @@ def load() -> ctypes.CDLL:
     lib.l4l_attn_decode_static.restype = c_int
     lib.l4l_attn_decode_static.argtypes = [vp, vp, KVCache, i32p, c_int, c_int, c_int, c_int, c_int, ctypes.c_float, vp,
                                            vp]
+    lib.l4l_kv_append_paged.restype = c_int
+    lib.l4l_kv_append_paged.argtypes = [PagedKV, i32p, c_int, Tensor4, Tensor4, i32p, i32p, c_int, c_int, c_int, c_int, vp]
+    lib.l4l_attn_decode_paged.restype = c_int
+    lib.l4l_attn_decode_paged.argtypes = [vp, vp, PagedKV, i32p, c_int, i32p, c_int, c_int, c_int, c_int, c_int,
+                                          ctypes.c_float, vp, vp, c_size, vp]
     lib.l4l_rope_kv_append.restype = c_int
     lib.l4l_rope_kv_append.argtypes = [Tensor4, Tensor4, Tensor4, KVCache, i32p, i32p, c_int, c_int, c_int, c_int, c_int,
                                        vp, vp, c_int, vp, vp, ctypes.c_float, vp]
@@ -289,3 +301,51 @@ def l4l_rope_kv_append(q, k_new, v_new, cache_k, cache_v, pos, n_new, cos, sin, 
                                    float(eps), _stream())
     if st != L4L_OK:
         raise L4LError(st, "l4l_rope_kv_append")
+
+
+def paged_kv(pool_k, pool_v) -> PagedKV:
+    """Page pools indexed [page, Hkv, slot, D] (any strides with D contiguous) -> l4l_paged_kv."""
+    _check_bf16_cuda(pool_k, "pool_k")
+    _check_bf16_cuda(pool_v, "pool_v")
+    if pool_k.dim() != 4 or pool_k.shape != pool_v.shape or pool_k.stride() != pool_v.stride():
+        raise ValueError("pool_k and pool_v must be [pages, Hkv, page_size, D] views with equal shapes and strides")
+    return PagedKV(pool_k.data_ptr(), pool_v.data_ptr(), pool_k.stride(0), pool_k.stride(1), pool_k.stride(2),
+                   pool_k.shape[2], pool_k.shape[0])
+
+
+def _block_table(t, B: int):
+    if not (t.is_cuda and t.dtype == torch.int32 and t.dim() == 2 and t.shape[0] == B and t.is_contiguous()):
+        raise TypeError("block_table must be a contiguous CUDA int32 tensor [B, pages per sequence]")
+    return t.data_ptr(), t.shape[1]
+
+
+def l4l_kv_append_paged(pool_k, pool_v, block_table, k_new, v_new, write_pos, n_new=None) -> None:
+    """k_new, v_new [B,T,Hkv,D] into the pages of a paged cache; write_pos CUDA int32 [B]."""
+    B, T, Hkv, D = k_new.shape
+    tbl, stride = _block_table(block_table, B)
+    st = load().l4l_kv_append_paged(paged_kv(pool_k, pool_v), tbl, stride, tensor4(k_new, "k_new"),
+                                    tensor4(v_new, "v_new"), _i32_dev(write_pos, "write_pos"),
+                                    None if n_new is None else _i32_dev(n_new, "n_new"), T, B, Hkv, D, _stream())
+    if st != L4L_OK:
+        raise L4LError(st, "l4l_kv_append_paged")
+
+
+def l4l_attn_decode_paged(q, o, pool_k, pool_v, block_table, kv_lens, max_kv_len: int, scale: float, workspace,
+                          lse=None) -> None:
+    """Decode over a paged cache. q,o dense [B,Hq,D]; pools [pages,Hkv,page_size,D]; block_table CUDA int32 [B, n]."""
+    _check_bf16_cuda(q, "q")
+    _check_bf16_cuda(o, "o")
+    if not (q.is_contiguous() and o.is_contiguous() and q.dim() == 3 and q.shape == o.shape):
+        raise ValueError("q and o must be dense [B, Hq, D]")
+    B, Hq, D = q.shape
+    Hkv = pool_k.shape[1]
+    if lse is not None and not (lse.is_cuda and lse.dtype == torch.float32 and lse.is_contiguous()
+                                and tuple(lse.shape) == (B, Hq)):
+        raise TypeError("lse must be a contiguous CUDA float32 tensor [B, Hq]")
+    tbl, stride = _block_table(block_table, B)
+    st = load().l4l_attn_decode_paged(q.data_ptr(), o.data_ptr(), paged_kv(pool_k, pool_v), tbl, stride,
+                                      _i32_dev(kv_lens, "kv_lens"), int(max_kv_len), B, Hq, Hkv, D, float(scale),
+                                      None if lse is None else lse.data_ptr(), workspace.data_ptr(),
+                                      workspace.numel() * workspace.element_size(), _stream())
+    if st != L4L_OK:
+        raise L4LError(st, "l4l_attn_decode_paged")

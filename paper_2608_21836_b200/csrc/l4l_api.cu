@@ -211,6 +211,60 @@ l4l_status l4l_kv_append(l4l_kv_cache cache, l4l_tensor4 k_new, l4l_tensor4 v_ne
                             static_cast<cudaStream_t>(stream));
 }
 
+namespace {
+
+// A page pool is valid if a page size is a power of two >= 16 (tiles are fetched in 16-token groups).
+bool pool_ok(const l4l_paged_kv &pool)
+{
+    return pool.k && pool.v && aligned16(pool.k) && aligned16(pool.v) && stride_ok(pool.stride_page) &&
+           stride_ok(pool.stride_h) && stride_ok(pool.stride_t) && pool.num_pages > 0 && pool.page_size >= 16 &&
+           pool.page_size <= (1 << 20) && (pool.page_size & (pool.page_size - 1)) == 0;
+}
+
+l4l_kv_cache pool_as_cache(const l4l_paged_kv &pool)
+{
+    l4l_kv_cache c;
+    c.k = pool.k; c.v = pool.v;
+    c.stride_b = pool.stride_page; c.stride_h = pool.stride_h; c.stride_t = pool.stride_t;
+    c.max_len = pool.page_size;
+    return c;
+}
+
+}  // namespace
+
+l4l_status l4l_kv_append_paged(l4l_paged_kv pool, const int32_t *d_block_table, int table_stride, l4l_tensor4 k_new,
+                               l4l_tensor4 v_new, const int32_t *d_write_pos, const int32_t *d_n_new, int n_new_max,
+                               int B, int Hkv, int head_dim, l4l_stream stream)
+{
+    if (B < 0 || Hkv <= 0 || n_new_max < 0 || table_stride <= 0) return L4L_ERR_INVALID_ARG;
+    if (head_dim != 64 && head_dim != 128) return L4L_ERR_UNSUPPORTED;
+    if (!pool_ok(pool) || !tensor4_ok(k_new) || !tensor4_ok(v_new) || !d_write_pos || !d_block_table)
+        return L4L_ERR_INVALID_ARG;
+    if (B == 0 || n_new_max == 0) return L4L_OK;
+    const PagedTable pt{d_block_table, table_stride, pool.num_pages};
+    return launch_kv_append(pool_as_cache(pool), k_new, v_new, d_write_pos, d_n_new, n_new_max, B, Hkv, head_dim,
+                            static_cast<cudaStream_t>(stream), &pt);
+}
+
+l4l_status l4l_attn_decode_paged(const void *q, void *o, l4l_paged_kv pool, const int32_t *d_block_table,
+                                 int table_stride, const int32_t *d_kv_lens, int max_kv_len, int B, int Hq, int Hkv,
+                                 int head_dim, float scale, float *d_lse, void *workspace, size_t ws_bytes,
+                                 l4l_stream stream)
+{
+    l4l_status st = shape_status(B, Hq, Hkv, head_dim);
+    if (st != L4L_OK) return st;
+    if (!q || !o || !d_kv_lens || !d_block_table || !aligned16(q) || !aligned16(o)) return L4L_ERR_INVALID_ARG;
+    if (!pool_ok(pool) || table_stride <= 0) return L4L_ERR_INVALID_ARG;
+    if (max_kv_len < 0 || (long long)max_kv_len > (long long)table_stride * pool.page_size) return L4L_ERR_INVALID_ARG;
+    if (!workspace || ws_bytes < kStatusBytes) return L4L_ERR_WORKSPACE;
+    if (B == 0) return L4L_OK;
+    const DecodePlan plan = plan_decode(B, Hq, Hkv, head_dim, max_kv_len, ws_bytes);
+    if (plan.ws_bytes > ws_bytes) return L4L_ERR_WORKSPACE;
+    const PagedTable pt{d_block_table, table_stride, pool.num_pages};
+    return launch_decode(q, o, pool_as_cache(pool), d_kv_lens, max_kv_len, B, Hq, Hkv, head_dim, scale, d_lse, workspace,
+                         plan, static_cast<cudaStream_t>(stream), nullptr, nullptr, &pt);
+}
+
 l4l_status l4l_rope_kv_append(l4l_tensor4 q, l4l_tensor4 k_new, l4l_tensor4 v_new, l4l_kv_cache cache,
                               const int32_t *d_pos, const int32_t *d_n_new, int T, int B, int Hq, int Hkv, int head_dim,
                               const float *d_cos, const float *d_sin, int n_pos, const float *d_q_weight,

@@ -73,6 +73,10 @@ struct DecodeParams {
     __nv_bfloat16 *cache_k, *cache_v;
     int64_t c_sb, c_sh, c_st;
     unsigned *status;
+    // paged cache (null: contiguous): token t of sequence b lives in page block_table[b * table_stride + t / page_size]
+    // at offset t % page_size; the tensor maps then describe the page pool [pages, Hkv, page_size, D]
+    const int32_t *block_table;
+    int table_stride, page_size, page_shift;
     int B, Hq, Hkv, G, min_tiles, nsplit, max_kv_len;
     float scale_log2e;
     TmapCoord coord;
@@ -242,16 +246,34 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                         bulk_load_1d(q_slots + (size_t)s * q_bytes, p.q + ((size_t)b * p.Hq + (size_t)kvh * p.G) * D,
                                      q_bytes, &full[s]);
                     uint8_t *dst = stages + (size_t)s * C::kStageBytes;
-                    if (rem >= kTileT) {
-                        order_coords(p.coord, tile * kTileT, kvh, b, c1, c2, c3);
+                    // With a paged cache a tile is one box only if a page holds whole tiles; smaller pages
+                    // are fetched in 16-token groups (a group never straddles pages: page sizes are multiples
+                    // of 16). A page id outside the pool makes the box read zeros, never memory.
+                    const bool paged = p.block_table != nullptr;
+                    const int32_t *pages = paged ? p.block_table + (size_t)b * p.table_stride : nullptr;
+                    if (rem >= kTileT && (!paged || p.page_size >= kTileT)) {
+                        int tt = tile * kTileT, bb = b;
+                        if (paged) {
+                            bb = __ldg(pages + (tt >> p.page_shift));
+                            tt &= p.page_size - 1;
+                        }
+                        order_coords(p.coord, tt, kvh, bb, c1, c2, c3);
 #pragma unroll
                         for (int hf = 0; hf < C::kHalves; ++hf) {
                             tma_load_4d(dst + hf * C::kHalfBytes, &tmap_k, &full[s], hf * 64, c1, c2, c3);
                             tma_load_4d(dst + C::kTileBytes + hf * C::kHalfBytes, &tmap_v, &full[s], hf * 64, c1, c2, c3);
                         }
                     } else {
-                        for (int gq = 0; gq < groups; ++gq) {
-                            order_coords(p.coord, tile * kTileT + gq * 16, kvh, b, c1, c2, c3);
+                        int page_of[kTileT / 16];                    // looked up together: independent loads
+#pragma unroll
+                        for (int gq = 0; gq < kTileT / 16; ++gq)
+                            page_of[gq] = (paged && gq < groups) ? __ldg(pages + ((tile * kTileT + gq * 16) >> p.page_shift)) : b;
+#pragma unroll
+                        for (int gq = 0; gq < kTileT / 16; ++gq) {
+                            if (gq >= groups) break;
+                            int tt = tile * kTileT + gq * 16;
+                            if (paged) tt &= p.page_size - 1;
+                            order_coords(p.coord, tt, kvh, page_of[gq], c1, c2, c3);
                             uint8_t *dg = dst + gq * 16 * 128;        // 2 KB per group: the swizzle phase is kept
 #pragma unroll
                             for (int hf = 0; hf < C::kHalves; ++hf) {
@@ -813,8 +835,10 @@ DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_
 l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, const int32_t *d_kv_lens,
                          int max_kv_len, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
                          void *workspace, const DecodePlan &plan, cudaStream_t stream, const l4l_tensor4 *k_new,
-                         const l4l_tensor4 *v_new)
+                         const l4l_tensor4 *v_new, const PagedTable *paged)
 {
+    // paged: `cache` describes the page pool (stride_b = stride between pages, max_len = page size)
+    if (paged && (k_new || v_new)) return L4L_ERR_UNSUPPORTED;
     const int G = Hq / Hkv;
     const ShapeOps ops = pick_shape(D, plan.warps);
     const int kTileT = ops.tile_t;
@@ -834,15 +858,20 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         const int nb = (B - b0 < slice) ? (B - b0) : slice;
         CUtensorMap tk, tv, tk16, tv16;   // 64-token boxes, and 16-token boxes for the last tile of a sequence
         TmapCoord coord, coord_v;
-        const __nv_bfloat16 *kb = static_cast<const __nv_bfloat16 *>(cache.k) + (size_t)b0 * cache.stride_b;
-        const __nv_bfloat16 *vb = static_cast<const __nv_bfloat16 *>(cache.v) + (size_t)b0 * cache.stride_b;
-        if (!make_tmap_bf16(&tk, &coord, kb, D, cache.max_len, Hkv, nb, cache.stride_t, cache.stride_h,
-                            cache.stride_b, 64, kTileT) ||
-            !make_tmap_bf16(&tv, &coord_v, vb, D, cache.max_len, Hkv, nb, cache.stride_t, cache.stride_h,
-                            cache.stride_b, 64, kTileT) ||
-            !make_tmap_bf16(&tk16, &coord_v, kb, D, cache.max_len, Hkv, nb, cache.stride_t, cache.stride_h,
+        // contiguous: the maps cover this slice's sequences; paged: the whole pool, whatever the slice
+        const size_t first = paged ? 0 : (size_t)b0 * cache.stride_b;
+        const int outer = paged ? paged->num_pages : nb;
+        const __nv_bfloat16 *kb = static_cast<const __nv_bfloat16 *>(cache.k) + first;
+        const __nv_bfloat16 *vb = static_cast<const __nv_bfloat16 *>(cache.v) + first;
+        // pages smaller than a tile are only ever fetched in 16-token groups: no box may exceed the page
+        const int box_t = (paged && cache.max_len < kTileT) ? 16 : kTileT;
+        if (!make_tmap_bf16(&tk, &coord, kb, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
+                            cache.stride_b, 64, box_t) ||
+            !make_tmap_bf16(&tv, &coord_v, vb, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
+                            cache.stride_b, 64, box_t) ||
+            !make_tmap_bf16(&tk16, &coord_v, kb, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
                             cache.stride_b, 64, 16) ||
-            !make_tmap_bf16(&tv16, &coord_v, vb, D, cache.max_len, Hkv, nb, cache.stride_t, cache.stride_h,
+            !make_tmap_bf16(&tv16, &coord_v, vb, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
                             cache.stride_b, 64, 16))
             return L4L_ERR_CUDA;
         DecodeParams p;
@@ -858,6 +887,11 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         p.max_kv_len = max_kv_len;
         p.k_new = p.v_new = nullptr;
         p.new_sb = p.new_sh = 0;
+        p.block_table = paged ? paged->block_table + (size_t)b0 * paged->table_stride : nullptr;
+        p.table_stride = paged ? paged->table_stride : 0;
+        p.page_size = paged ? cache.max_len : 0;
+        p.page_shift = 0;
+        while (paged && (1 << p.page_shift) < cache.max_len) ++p.page_shift;
         p.cache_k = static_cast<__nv_bfloat16 *>(cache.k) + (size_t)b0 * cache.stride_b;
         p.cache_v = static_cast<__nv_bfloat16 *>(cache.v) + (size_t)b0 * cache.stride_b;
         p.c_sb = cache.stride_b; p.c_sh = cache.stride_h; p.c_st = cache.stride_t;
@@ -963,5 +997,5 @@ extern "C" l4l_status l4l_attn_decode_static(const void *q, void *o, l4l_kv_cach
     const size_t zero_bytes = kStatusBytes + kTicketBytes;
     if (cudaMemsetAsync(scratch, 0, zero_bytes, s) != cudaSuccess) return L4L_ERR_CUDA;
     return launch_decode(q, o, cache, d_kv_lens, max_kv_len, B, Hq, Hkv, head_dim, scale, d_lse, scratch, plan, s,
-                         nullptr, nullptr);
+                         nullptr, nullptr, nullptr);
 }

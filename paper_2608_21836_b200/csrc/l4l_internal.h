@@ -34,10 +34,19 @@ struct DecodePlan {
 };
 DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_limit);
 
+// Block table of a paged cache: token t of sequence b is in page block_table[b * table_stride + t / page_size].
+struct PagedTable {
+    const int32_t *block_table;   // device
+    int table_stride;             // entries per sequence
+    int num_pages;                // pages in the pool
+};
+
+// With `paged`, `cache` describes the page pool: stride_b = stride between pages, max_len = page size.
 l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, const int32_t *d_kv_lens,
                          int max_kv_len, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
                          void *workspace, const DecodePlan &plan, cudaStream_t stream,
-                         const l4l_tensor4 *k_new = nullptr, const l4l_tensor4 *v_new = nullptr);
+                         const l4l_tensor4 *k_new = nullptr, const l4l_tensor4 *v_new = nullptr,
+                         const PagedTable *paged = nullptr);
 
 l4l_status launch_rope_kv_append(const l4l_tensor4 &q, const l4l_tensor4 &k_new, const l4l_tensor4 &v_new,
                                  const l4l_kv_cache &cache, const int32_t *d_pos, const int32_t *d_n_new, int T, int B,
@@ -45,7 +54,7 @@ l4l_status launch_rope_kv_append(const l4l_tensor4 &q, const l4l_tensor4 &k_new,
                                  const float *d_q_weight, const float *d_k_weight, float norm_eps, cudaStream_t stream);
 l4l_status launch_kv_append(const l4l_kv_cache &cache, const l4l_tensor4 &k_new, const l4l_tensor4 &v_new,
                             const int32_t *d_write_pos, const int32_t *d_n_new, int n_new_max, int B, int Hkv,
-                            int D, cudaStream_t stream);
+                            int D, cudaStream_t stream, const PagedTable *paged = nullptr);
 
 l4l_status launch_prefill(const l4l_tensor4 &q, const l4l_tensor4 &k, const l4l_tensor4 &v,
                           const l4l_tensor4 &o, const l4l_kv_cache &cache, const int32_t *d_seq_lens,

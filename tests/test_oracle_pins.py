@@ -472,3 +472,39 @@ def test_rms_norm_part_of_rope_has_unit_rms_scale_invariance_and_weight_linearit
     _, _, _, qc, _ = orc.rope_kv_append(const, const, const, ck[:1, :1], cv[:1, :1], [0], None, cos, sin,
                                         q_weight=ones, eps=0.75)
     np.testing.assert_allclose(qc, 0.5 / math.sqrt(0.25 + 0.75), rtol=1e-14)
+
+
+# --------------------------------------------------------------------------- paged cache = the cache its pages spell out
+def test_paged_decode_is_decode_over_the_pages_laid_end_to_end():
+    B, Hq, Hkv, D, page, n_per = 3, 4, 2, 8, 4, 5
+    Lmax = page * n_per
+    q = randn((B, Hq, D), 60)
+    ck, cv = randn((B, Hkv, Lmax, D), 61), randn((B, Hkv, Lmax, D), 62)
+    lens = np.array([Lmax, 7, 1], np.int32)
+    want, want_lse = orc.decode(q, ck, cv, lens, 0.4)
+    # scatter the contiguous caches into a shuffled pool with spare, poisoned pages
+    rng = np.random.default_rng(3)
+    n_pages = B * n_per + 4
+    perm = rng.permutation(n_pages)[: B * n_per].reshape(B, n_per)
+    pool_k = torch.full((n_pages, Hkv, page, D), float("nan")).to(torch.bfloat16)
+    pool_v = pool_k.clone()
+    for b in range(B):
+        for i in range(n_per):
+            pool_k[perm[b, i]] = ck[b, :, i * page:(i + 1) * page]
+            pool_v[perm[b, i]] = cv[b, :, i * page:(i + 1) * page]
+    got, got_lse = orc.decode_paged(q, pool_k, pool_v, perm, lens, 0.4)
+    assert np.array_equal(got, want) and np.array_equal(got_lse, want_lse)
+    assert np.array_equal(orc.gather_pages(pool_k, perm, Lmax), orc.bits(ck))
+    # entries past a sequence's last token are never looked at
+    perm2 = perm.copy()
+    perm2[1, 2:] = -1
+    perm2[2, 1:] = 10 ** 6
+    got2, _ = orc.decode_paged(q, pool_k, pool_v, perm2, lens, 0.4)
+    assert np.array_equal(got2, want)
+    # appending through the table lands where the gather finds it
+    k_new, v_new = randn((B, 3, Hkv, D), 63), randn((B, 3, Hkv, D), 64)
+    pos = np.array([Lmax - 2, 7, 1], np.int32)                     # sequence 0: third token falls off its table
+    pk2, pv2 = orc.kv_append_paged(pool_k, pool_v, perm, k_new, v_new, pos, None)
+    ck2, cv2 = orc.kv_append(ck, cv, k_new, v_new, pos, np.array([2, 3, 3], np.int32))
+    assert np.array_equal(orc.gather_pages(pk2, perm, Lmax), ck2)
+    assert np.array_equal(orc.gather_pages(pv2, perm, Lmax), cv2)
