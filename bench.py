@@ -323,7 +323,26 @@ def run_ours(args, rank, world):
     rope_bytes = 2 * q.numel() * 2 + 2 * (k.numel() + v.numel()) * 2       # q read + written, k/v read, cache written
     t_chunk = timed(lambda: l4l.l4l_attn_prefill_chunk(q, o, pk, pv, zeros_b, plens, wp.scale, ws_p), 5)
     t_fused = timed(lambda: l4l.l4l_attn_decode_append(dq, do, dck, dcv, dkn, dvn, dlen, Lmax, wd.scale, ws_d), 20)
-    del filler
+    # decode over a paged cache: the same batch cut into 64-token pages scattered over a pool, three pools in rotation
+    page = 64
+    n_per = Lmax // page
+    pools = []
+    for i in range(3):
+        perm = torch.randperm(Bd * n_per, generator=torch.Generator().manual_seed(7 + i)).to(dev)
+        pool_k = torch.empty(Bd * n_per, Hkv, page, D, dtype=torch.bfloat16, device=dev)
+        pool_v = torch.empty_like(pool_k)
+        pool_k[perm] = dck.view(Bd, Hkv, n_per, page, D).permute(0, 2, 1, 3, 4).reshape(Bd * n_per, Hkv, page, D)
+        pool_v[perm] = dcv.view(Bd, Hkv, n_per, page, D).permute(0, 2, 1, 3, 4).reshape(Bd * n_per, Hkv, page, D)
+        pools.append((pool_k, pool_v, perm.view(Bd, n_per).to(torch.int32).contiguous()))
+    rot = [0]
+
+    def paged_step():
+        pk_i, pv_i, tbl_i = pools[rot[0] % 3]
+        rot[0] += 1
+        l4l.l4l_attn_decode_paged(dq, do, pk_i, pv_i, tbl_i, dlen, Lmax, wd.scale, ws_d)
+
+    t_paged = timed(paged_step, 21)
+    del pools, filler
     dev_err = l4l.l4l_last_device_error(ws_p) | l4l.l4l_last_device_error(ws_d)
 
     # ---- end to end through the same entry points with HOST buffers (pinned), copies inside the timed region
@@ -356,8 +375,8 @@ def run_ours(args, rank, world):
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
 
     # ---- max over ranks
-    total_ms, e2e_ms, t_pre, t_dec, t_app, t_dec_b2b, t_rope, t_chunk, t_fused = max_over_ranks(
-        [total_ms, e2e_ms, t_pre, t_dec, t_app, t_dec_b2b, t_rope, t_chunk, t_fused], world, dev)
+    total_ms, e2e_ms, t_pre, t_dec, t_app, t_dec_b2b, t_rope, t_chunk, t_fused, t_paged = max_over_ranks(
+        [total_ms, e2e_ms, t_pre, t_dec, t_app, t_dec_b2b, t_rope, t_chunk, t_fused, t_paged], world, dev)
     if rank != 0:
         return
 
@@ -401,6 +420,7 @@ def run_ours(args, rank, world):
                                     "bytes": rope_bytes},
             "prefill_from_cache": {"ms": t_chunk, "tflops": pre_flops / (t_chunk * 1e-3) / 1e12},
             "decode_with_fused_append": {"us": t_fused * 1e3, "kv_gbs": dec_bytes / (t_fused * 1e-3) / 1e9},
+            "decode_paged_64": {"us": t_paged * 1e3, "kv_gbs": dec_bytes / (t_paged * 1e-3) / 1e9},
         },
         "gpu_launches": 3 * args.steps,
         "clocks": clocks,

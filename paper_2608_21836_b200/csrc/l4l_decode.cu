@@ -246,22 +246,31 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                         bulk_load_1d(q_slots + (size_t)s * q_bytes, p.q + ((size_t)b * p.Hq + (size_t)kvh * p.G) * D,
                                      q_bytes, &full[s]);
                     uint8_t *dst = stages + (size_t)s * C::kStageBytes;
-                    // With a paged cache a tile is one box only if a page holds whole tiles; smaller pages
-                    // are fetched in 16-token groups (a group never straddles pages: page sizes are multiples
-                    // of 16). A page id outside the pool makes the box read zeros, never memory.
+                    // With a paged cache a full tile is one box if a page holds whole tiles, else one box per
+                    // page (tmap_k / tmap_v then have page-sized boxes); the last tile of a sequence comes in
+                    // 16-token groups either way. Neither a box nor a group straddles pages: page sizes are
+                    // powers of two >= 16. A page id outside the pool makes the box read zeros, never memory.
                     const bool paged = p.block_table != nullptr;
                     const int32_t *pages = paged ? p.block_table + (size_t)b * p.table_stride : nullptr;
-                    if (rem >= kTileT && (!paged || p.page_size >= kTileT)) {
-                        int tt = tile * kTileT, bb = b;
-                        if (paged) {
-                            bb = __ldg(pages + (tt >> p.page_shift));
-                            tt &= p.page_size - 1;
-                        }
-                        order_coords(p.coord, tt, kvh, bb, c1, c2, c3);
+                    if (rem >= kTileT) {
+                        const int box_rows = (paged && p.page_size < kTileT) ? p.page_size : kTileT;
+                        const int n_box = kTileT / box_rows;
+                        int page_of[kTileT / 16];                    // looked up together: independent loads
 #pragma unroll
-                        for (int hf = 0; hf < C::kHalves; ++hf) {
-                            tma_load_4d(dst + hf * C::kHalfBytes, &tmap_k, &full[s], hf * 64, c1, c2, c3);
-                            tma_load_4d(dst + C::kTileBytes + hf * C::kHalfBytes, &tmap_v, &full[s], hf * 64, c1, c2, c3);
+                        for (int bx = 0; bx < kTileT / 16; ++bx)
+                            page_of[bx] = (paged && bx < n_box) ? __ldg(pages + ((tile * kTileT + bx * box_rows) >> p.page_shift)) : b;
+#pragma unroll
+                        for (int bx = 0; bx < kTileT / 16; ++bx) {
+                            if (bx >= n_box) break;
+                            int tt = tile * kTileT + bx * box_rows;
+                            if (paged) tt &= p.page_size - 1;
+                            order_coords(p.coord, tt, kvh, page_of[bx], c1, c2, c3);
+                            uint8_t *db = dst + bx * box_rows * 128;  // whole 8-row groups: the swizzle phase is kept
+#pragma unroll
+                            for (int hf = 0; hf < C::kHalves; ++hf) {
+                                tma_load_4d(db + hf * C::kHalfBytes, &tmap_k, &full[s], hf * 64, c1, c2, c3);
+                                tma_load_4d(db + C::kTileBytes + hf * C::kHalfBytes, &tmap_v, &full[s], hf * 64, c1, c2, c3);
+                            }
                         }
                     } else {
                         int page_of[kTileT / 16];                    // looked up together: independent loads
@@ -863,8 +872,8 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         const int outer = paged ? paged->num_pages : nb;
         const __nv_bfloat16 *kb = static_cast<const __nv_bfloat16 *>(cache.k) + first;
         const __nv_bfloat16 *vb = static_cast<const __nv_bfloat16 *>(cache.v) + first;
-        // pages smaller than a tile are only ever fetched in 16-token groups: no box may exceed the page
-        const int box_t = (paged && cache.max_len < kTileT) ? 16 : kTileT;
+        // pages smaller than a tile are fetched page by page: no box may exceed the page
+        const int box_t = (paged && cache.max_len < kTileT) ? cache.max_len : kTileT;
         if (!make_tmap_bf16(&tk, &coord, kb, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
                             cache.stride_b, 64, box_t) ||
             !make_tmap_bf16(&tv, &coord_v, vb, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
