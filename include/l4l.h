@@ -139,6 +139,27 @@ l4l_status l4l_attn_decode_paged(const void *q, void *o, l4l_paged_kv pool, cons
                                  void *workspace, size_t ws_bytes, l4l_stream stream);
 
 /*
+ * The same two operations over an fp8 cache (e4m3: 1 sign, 4 exponent, 3 mantissa bits, largest
+ * finite value 448, no infinities), which halves the bytes decode has to stream. The paper's
+ * kernels read a bf16 cache; this layout has no counterpart there. `cache8` uses the l4l_kv_cache
+ * struct with k / v pointing at bytes and strides counted in bytes (multiples of 16); a stored
+ * byte c of KV head g stands for the real value e4m3(c) * scale[g].
+ *   l4l_kv_append_fp8  : stores RN_e4m3( fp32(x) / k_scale[g] ) (IEEE fp32 division, then round to
+ *                        nearest even, saturating at +-448; NaN stays NaN); other rules as l4l_kv_append.
+ *   l4l_attn_decode_fp8: l4l_attn_decode over the values the bytes stand for (the widening to f16 in
+ *                        the kernel is exact; q and the softmax weights are used as f16). head_dim 128 only.
+ *   d_k_scale, d_v_scale   device float [Hkv], > 0
+ */
+l4l_status l4l_kv_append_fp8(l4l_kv_cache cache8, l4l_tensor4 k_new, l4l_tensor4 v_new,
+                             const int32_t *d_write_pos, const int32_t *d_n_new, int n_new_max,
+                             int B, int Hkv, int head_dim, const float *d_k_scale, const float *d_v_scale,
+                             l4l_stream stream);
+l4l_status l4l_attn_decode_fp8(const void *q, void *o, l4l_kv_cache cache8, const float *d_k_scale,
+                               const float *d_v_scale, const int32_t *d_kv_lens, int max_kv_len,
+                               int B, int Hq, int Hkv, int head_dim, float scale, float *d_lse,
+                               void *workspace, size_t ws_bytes, l4l_stream stream);
+
+/*
  * Rotary position embedding (and optional per-head RMS normalisation of q and k) fused with the
  * cache update: the projection outputs of the new tokens go through ONE streaming pass that
  * leaves q ready for the attention calls and K, V in the cache. (The paper's prefill kernel is

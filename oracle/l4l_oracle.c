@@ -356,6 +356,133 @@ int l4l_oracle_decode(const uint16_t *q, const uint16_t *cache_k, const uint16_t
     return fail ? -1 : 0;
 }
 
+/* ------------------------------------------------------------------------------------------------
+ * fp8 (e4m3) cache. The format: 1 sign bit, 4 exponent bits (bias 7), 3 mantissa bits; exponent 0 is
+ * subnormal (m/8 * 2^-6); there are no infinities; exponent 15 with mantissa 7 is NaN; the largest
+ * finite value is 1.75 * 2^8 = 448.
+ */
+static double e4m3_to_f64(uint8_t c)
+{
+    const int sign = c >> 7, e = (c >> 3) & 15, m = c & 7;
+    double v;
+    if (e == 15 && m == 7) return NAN;
+    v = (e == 0) ? ldexp((double)m / 8.0, -6) : ldexp(1.0 + (double)m / 8.0, e - 7);
+    return sign ? -v : v;
+}
+
+/* fp32 value -> e4m3: nearest, ties to even, saturating at +-448 (NaN -> 0x7F). Brute force over the 127
+ * non-negative finite codes: the nearest one wins, a tie goes to the even code. */
+static uint8_t f32_to_e4m3(float y)
+{
+    uint8_t best = 0;
+    double bd = INFINITY;
+    const double a = fabs((double)y);
+    if (y != y) return 0x7F;
+    for (int c = 0; c < 0x7F; ++c) {
+        const double d = fabs(e4m3_to_f64((uint8_t)c) - a);
+        if (d < bd || (d == bd && (c & 1) == 0)) { bd = d; best = (uint8_t)c; }
+    }
+    return (uint8_t)(best | (signbit(y) ? 0x80 : 0));
+}
+
+void l4l_oracle_e4m3_decode(const uint8_t *c, double *out, int64_t n)
+{
+    for (int64_t i = 0; i < n; ++i) out[i] = e4m3_to_f64(c[i]);
+}
+
+void l4l_oracle_e4m3_encode(const float *x, uint8_t *out, int64_t n)
+{
+    for (int64_t i = 0; i < n; ++i) out[i] = f32_to_e4m3(x[i]);
+}
+
+/*
+ * Cache update of an fp8 cache: slot write_pos[b] + t of (b, kv head g) receives the e4m3 code of
+ * fp32(x) / scale[g], the division rounded to fp32 (the precision the decision is defined in), for the
+ * new tokens' k and v. Out-of-range slots: error (the caller tests the drop rule separately).
+ *   cache_k8, cache_v8 [B, Hkv, Lmax, D] bytes, in/out      k_new, v_new [B, T, Hkv, D] bf16 bits
+ */
+int l4l_oracle_kv_append_fp8(uint8_t *cache_k8, uint8_t *cache_v8, const uint16_t *k_new, const uint16_t *v_new,
+                             const int32_t *pos, const int32_t *n_new, const float *k_scale, const float *v_scale,
+                             int B, int T, int Hkv, int D, int Lmax)
+{
+    for (int b = 0; b < B; ++b) {
+        const int n = n_new ? n_new[b] : T;
+        for (int t = 0; t < n && t < T; ++t) {
+            const int64_t slot = (int64_t)pos[b] + t;
+            if (slot < 0 || slot >= Lmax) continue;
+            for (int g = 0; g < Hkv; ++g)
+                for (int d = 0; d < D; ++d) {
+                    const int64_t src = (((int64_t)b * T + t) * Hkv + g) * D + d;
+                    const int64_t dst = (((int64_t)b * Hkv + g) * Lmax + slot) * D + d;
+                    const volatile float qk = (float)bf16_to_f64(k_new[src]) / k_scale[g];
+                    const volatile float qv = (float)bf16_to_f64(v_new[src]) / v_scale[g];
+                    cache_k8[dst] = f32_to_e4m3(qk);
+                    cache_v8[dst] = f32_to_e4m3(qv);
+                }
+        }
+    }
+    return 0;
+}
+
+/*
+ * Decode over an fp8 cache: the definition of attend_row() written out once more over the values the
+ * bytes stand for, k_j[d] = e4m3(cache_k8[j][d]) * k_scale[g] (and the same for v), in fp64.
+ */
+int l4l_oracle_decode_fp8(const uint16_t *q, const uint8_t *cache_k8, const uint8_t *cache_v8, const int32_t *kv_len,
+                          const float *k_scale, const float *v_scale, int B, int Hq, int Hkv, int D, int Lmax,
+                          double scale, double *out, double *lse)
+{
+    if (Hkv <= 0 || Hq % Hkv != 0) return -1;
+    const int G = Hq / Hkv;
+    for (int b = 0; b < B; ++b)
+        if (kv_len[b] < 0 || kv_len[b] > Lmax) return -1;
+    int fail = 0;
+#pragma omp parallel
+    {
+        double *p = (double *)malloc(sizeof(double) * (size_t)(Lmax > 0 ? Lmax : 1));
+        if (!p) {
+#pragma omp atomic write
+            fail = 1;
+        }
+#pragma omp for collapse(2) schedule(dynamic, 1)
+        for (int b = 0; b < B; ++b) {
+            for (int h = 0; h < Hq; ++h) {
+                if (!p) continue;
+                const int g = h / G, n = kv_len[b];
+                const uint16_t *qr = q + ((int64_t)b * Hq + h) * D;
+                const uint8_t *kb = cache_k8 + ((int64_t)b * Hkv + g) * Lmax * D;
+                const uint8_t *vb = cache_v8 + ((int64_t)b * Hkv + g) * Lmax * D;
+                double *o = out + ((int64_t)b * Hq + h) * D;
+                const double ks = (double)k_scale[g], vs = (double)v_scale[g];
+                if (n <= 0) {
+                    for (int d = 0; d < D; ++d) o[d] = 0.0;
+                    if (lse) lse[(int64_t)b * Hq + h] = -INFINITY;
+                    continue;
+                }
+                double m = -INFINITY, l = 0.0;
+                for (int j = 0; j < n; ++j) {
+                    double dot = 0.0;
+                    for (int d = 0; d < D; ++d) dot += bf16_to_f64(qr[d]) * (e4m3_to_f64(kb[(int64_t)j * D + d]) * ks);
+                    p[j] = scale * dot;
+                    if (p[j] > m) m = p[j];
+                }
+                for (int j = 0; j < n; ++j) {
+                    p[j] = exp(p[j] - m);
+                    l += p[j];
+                }
+                for (int d = 0; d < D; ++d) {
+                    double acc = 0.0;
+                    for (int j = 0; j < n; ++j) acc += p[j] * (e4m3_to_f64(vb[(int64_t)j * D + d]) * vs);
+                    o[d] = acc / l;
+                }
+                if (lse) lse[(int64_t)b * Hq + h] = m + log(l);
+            }
+        }
+        free(p);
+    }
+    return fail ? -1 : 0;
+}
+
 /*
  * Cache copy. Writes n_new[b] tokens of k_new / v_new ([B, T, Hkv, D]) into the cache
  * ([B, Hkv, Lmax, D]) at slots pos[b] .. pos[b]+n_new[b]-1, as raw 16-bit words.

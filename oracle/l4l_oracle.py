@@ -52,6 +52,13 @@ def _load():
         lib.l4l_oracle_round_bf16.restype = None
         lib.l4l_oracle_rope_kv_append.argtypes = [u16p, u16p, u16p, u16p, u16p, i32p, i32p, i, i, i, i, i, i,
                                                   f32p, f32p, i, f32p, f32p, d, f64p, f64p]
+        u8p = ctypes.POINTER(ctypes.c_uint8)
+        lib.l4l_oracle_e4m3_decode.argtypes = [u8p, f64p, ctypes.c_int64]
+        lib.l4l_oracle_e4m3_decode.restype = None
+        lib.l4l_oracle_e4m3_encode.argtypes = [f32p, u8p, ctypes.c_int64]
+        lib.l4l_oracle_e4m3_encode.restype = None
+        lib.l4l_oracle_kv_append_fp8.argtypes = [u8p, u8p, u16p, u16p, i32p, i32p, f32p, f32p, i, i, i, i, i]
+        lib.l4l_oracle_decode_fp8.argtypes = [u16p, u8p, u8p, i32p, f32p, f32p, i, i, i, i, i, d, f64p, f64p]
         lib.l4l_oracle_kv_append.argtypes = [u16p, u16p, u16p, u16p, i32p, i32p, i, i, i, i, i]
         _lib = lib
     return _lib
@@ -261,3 +268,67 @@ def kv_append_paged(pool_k, pool_v, block_table, k_new, v_new, pos, n_new):
                 pk[pg, :, s % page] = kn[b, t]
                 pv[pg, :, s % page] = vn[b, t]
     return pk, pv
+
+
+def _u8(x) -> np.ndarray:
+    """uint8 codes from a numpy uint8 array or a torch uint8 / float8_e4m3fn tensor."""
+    if isinstance(x, np.ndarray):
+        assert x.dtype == np.uint8
+        return np.ascontiguousarray(x)
+    import torch
+
+    if x.dtype != torch.uint8:
+        x = x.view(torch.uint8)
+    return np.ascontiguousarray(x.detach().cpu().contiguous().numpy())
+
+
+def e4m3_decode(codes) -> np.ndarray:
+    c = _u8(codes)
+    out = np.empty(c.shape, dtype=np.float64)
+    _load().l4l_oracle_e4m3_decode(_p(c, ctypes.c_uint8), _p(out, ctypes.c_double), c.size)
+    return out
+
+
+def e4m3_encode(x) -> np.ndarray:
+    """float32 values -> e4m3 codes (nearest even, saturating)."""
+    x = np.ascontiguousarray(np.asarray(x, dtype=np.float32))
+    out = np.empty(x.shape, dtype=np.uint8)
+    _load().l4l_oracle_e4m3_encode(_p(x, ctypes.c_float), _p(out, ctypes.c_uint8), x.size)
+    return out
+
+
+def kv_append_fp8(cache_k8, cache_v8, k_new, v_new, pos, n_new, k_scale, v_scale):
+    """Returns copies of the fp8 caches (uint8 codes) with the new tokens quantised in."""
+    ck, cv = _u8(cache_k8).copy(), _u8(cache_v8).copy()
+    kn, vn = bits(k_new), bits(v_new)
+    B, Hkv, Lmax, D = ck.shape
+    T = kn.shape[1]
+    assert kn.shape == (B, T, Hkv, D) and vn.shape == kn.shape
+    pos = _i32(pos)
+    n_new = _i32(n_new) if n_new is not None else np.full((B,), T, np.int32)
+    ks = np.ascontiguousarray(np.asarray(k_scale, dtype=np.float32))
+    vs = np.ascontiguousarray(np.asarray(v_scale, dtype=np.float32))
+    assert ks.shape == (Hkv,) and vs.shape == (Hkv,)
+    _load().l4l_oracle_kv_append_fp8(_p(ck, ctypes.c_uint8), _p(cv, ctypes.c_uint8), _p(kn, ctypes.c_uint16),
+                                     _p(vn, ctypes.c_uint16), _p(pos, ctypes.c_int32), _p(n_new, ctypes.c_int32),
+                                     _p(ks, ctypes.c_float), _p(vs, ctypes.c_float), B, T, Hkv, D, Lmax)
+    return ck, cv
+
+
+def decode_fp8(q, cache_k8, cache_v8, kv_len, k_scale, v_scale, scale: float):
+    """Decode over an fp8 cache. q [B,Hq,D] bf16; caches [B,Hkv,Lmax,D] e4m3 codes; scales float32 [Hkv]."""
+    q, ck, cv = bits(q), _u8(cache_k8), _u8(cache_v8)
+    B, Hq, D = q.shape
+    _, Hkv, Lmax, _ = ck.shape
+    kl = _i32(kv_len)
+    ks = np.ascontiguousarray(np.asarray(k_scale, dtype=np.float32))
+    vs = np.ascontiguousarray(np.asarray(v_scale, dtype=np.float32))
+    out = np.empty((B, Hq, D), dtype=np.float64)
+    lse = np.empty((B, Hq), dtype=np.float64)
+    rc = _load().l4l_oracle_decode_fp8(_p(q, ctypes.c_uint16), _p(ck, ctypes.c_uint8), _p(cv, ctypes.c_uint8),
+                                       _p(kl, ctypes.c_int32), _p(ks, ctypes.c_float), _p(vs, ctypes.c_float),
+                                       B, Hq, Hkv, D, Lmax, float(scale), _p(out, ctypes.c_double),
+                                       _p(lse, ctypes.c_double))
+    if rc != 0:
+        raise ValueError("l4l_oracle_decode_fp8 rejected its arguments")
+    return out, lse

@@ -23,7 +23,7 @@ EXPORTS = (
     "l4l_version", "l4l_status_string", "l4l_workspace_bytes", "l4l_workspace_init",
     "l4l_last_device_error", "l4l_kv_append", "l4l_attn_prefill", "l4l_attn_decode",
     "l4l_attn_decode_static", "l4l_attn_decode_append", "l4l_attn_prefill_chunk", "l4l_rope_kv_append",
-    "l4l_kv_append_paged", "l4l_attn_decode_paged",
+    "l4l_kv_append_paged", "l4l_attn_decode_paged", "l4l_kv_append_fp8", "l4l_attn_decode_fp8",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -88,6 +88,11 @@ def load() -> ctypes.CDLL:
     lib.l4l_attn_decode_paged.restype = c_int
     lib.l4l_attn_decode_paged.argtypes = [vp, vp, PagedKV, i32p, c_int, i32p, c_int, c_int, c_int, c_int, c_int,
                                           ctypes.c_float, vp, vp, c_size, vp]
+    lib.l4l_kv_append_fp8.restype = c_int
+    lib.l4l_kv_append_fp8.argtypes = [KVCache, Tensor4, Tensor4, i32p, i32p, c_int, c_int, c_int, c_int, vp, vp, vp]
+    lib.l4l_attn_decode_fp8.restype = c_int
+    lib.l4l_attn_decode_fp8.argtypes = [vp, vp, KVCache, vp, vp, i32p, c_int, c_int, c_int, c_int, c_int,
+                                        ctypes.c_float, vp, vp, c_size, vp]
     lib.l4l_rope_kv_append.restype = c_int
     lib.l4l_rope_kv_append.argtypes = [Tensor4, Tensor4, Tensor4, KVCache, i32p, i32p, c_int, c_int, c_int, c_int, c_int,
                                        vp, vp, c_int, vp, vp, ctypes.c_float, vp]
@@ -349,3 +354,46 @@ def l4l_attn_decode_paged(q, o, pool_k, pool_v, block_table, kv_lens, max_kv_len
                                       workspace.numel() * workspace.element_size(), _stream())
     if st != L4L_OK:
         raise L4LError(st, "l4l_attn_decode_paged")
+
+
+def kv_cache8(cache_k8, cache_v8) -> KVCache:
+    """fp8 caches indexed [B, Hkv, slot, D], dtype uint8 or float8_e4m3fn -> l4l_kv_cache with byte strides."""
+    for t, name in ((cache_k8, "cache_k8"), (cache_v8, "cache_v8")):
+        if not (t.is_cuda and t.dtype in (torch.uint8, torch.float8_e4m3fn) and t.dim() == 4 and t.stride(-1) == 1):
+            raise TypeError(f"{name} must be a CUDA uint8 / float8_e4m3fn tensor [B, Hkv, max_len, D] with D contiguous")
+    if cache_k8.shape != cache_v8.shape or cache_k8.stride() != cache_v8.stride():
+        raise ValueError("cache_k8 and cache_v8 must have equal shapes and strides")
+    return KVCache(cache_k8.data_ptr(), cache_v8.data_ptr(), cache_k8.stride(0), cache_k8.stride(1), cache_k8.stride(2),
+                   cache_k8.shape[2])
+
+
+def l4l_kv_append_fp8(cache_k8, cache_v8, k_new, v_new, write_pos, k_scale, v_scale, n_new=None) -> None:
+    """k_new, v_new [B,T,Hkv,D] bf16, divided by the per-KV-head scales and rounded to e4m3, into the fp8 cache."""
+    B, T, Hkv, D = k_new.shape
+    st = load().l4l_kv_append_fp8(kv_cache8(cache_k8, cache_v8), tensor4(k_new, "k_new"), tensor4(v_new, "v_new"),
+                                  _i32_dev(write_pos, "write_pos"), None if n_new is None else _i32_dev(n_new, "n_new"),
+                                  T, B, Hkv, D, _f32_dev(k_scale, "k_scale", (Hkv,)), _f32_dev(v_scale, "v_scale", (Hkv,)),
+                                  _stream())
+    if st != L4L_OK:
+        raise L4LError(st, "l4l_kv_append_fp8")
+
+
+def l4l_attn_decode_fp8(q, o, cache_k8, cache_v8, k_scale, v_scale, kv_lens, max_kv_len: int, scale: float, workspace,
+                        lse=None) -> None:
+    """Decode over an fp8 (e4m3) cache with per-KV-head scales. q,o dense bf16 [B,Hq,D]; head_dim 128."""
+    _check_bf16_cuda(q, "q")
+    _check_bf16_cuda(o, "o")
+    if not (q.is_contiguous() and o.is_contiguous() and q.dim() == 3 and q.shape == o.shape):
+        raise ValueError("q and o must be dense [B, Hq, D]")
+    B, Hq, D = q.shape
+    Hkv = cache_k8.shape[1]
+    if lse is not None and not (lse.is_cuda and lse.dtype == torch.float32 and lse.is_contiguous()
+                                and tuple(lse.shape) == (B, Hq)):
+        raise TypeError("lse must be a contiguous CUDA float32 tensor [B, Hq]")
+    st = load().l4l_attn_decode_fp8(q.data_ptr(), o.data_ptr(), kv_cache8(cache_k8, cache_v8),
+                                    _f32_dev(k_scale, "k_scale", (Hkv,)), _f32_dev(v_scale, "v_scale", (Hkv,)),
+                                    _i32_dev(kv_lens, "kv_lens"), int(max_kv_len), B, Hq, Hkv, D, float(scale),
+                                    None if lse is None else lse.data_ptr(), workspace.data_ptr(),
+                                    workspace.numel() * workspace.element_size(), _stream())
+    if st != L4L_OK:
+        raise L4LError(st, "l4l_attn_decode_fp8")

@@ -70,11 +70,11 @@ namespace {
 // (a tensor map is a pure function of these arguments).
 struct TmapKey {
     const void *base;
-    int D, box_d, box_t;
+    int D, box_d, box_t, elem_bytes;
     int64_t n_t, n_h, n_b, stride_t, stride_h, stride_b;
     bool operator==(const TmapKey &o) const
     {
-        return base == o.base && D == o.D && box_d == o.box_d && box_t == o.box_t && n_t == o.n_t && n_h == o.n_h &&
+        return base == o.base && D == o.D && elem_bytes == o.elem_bytes && box_d == o.box_d && box_t == o.box_t && n_t == o.n_t && n_h == o.n_h &&
                n_b == o.n_b && stride_t == o.stride_t && stride_h == o.stride_h && stride_b == o.stride_b;
     }
 };
@@ -89,15 +89,15 @@ TmapEntry g_tmap_cache[kTmapCache];
 int g_tmap_next = 0;
 std::mutex g_tmap_mutex;
 
-bool encode_tmap_bf16(CUtensorMap *out, TmapCoord *coord, const void *base, int D, int64_t n_t, int64_t n_h,
-                      int64_t n_b, int64_t stride_t, int64_t stride_h, int64_t stride_b, int box_d, int box_t);
+bool encode_tmap(CUtensorMap *out, TmapCoord *coord, const void *base, int D, int64_t n_t, int64_t n_h, int64_t n_b,
+                 int64_t stride_t, int64_t stride_h, int64_t stride_b, int box_d, int box_t, int elem_bytes);
 
 }  // namespace
 
-bool make_tmap_bf16(CUtensorMap *out, TmapCoord *coord, const void *base, int D, int64_t n_t, int64_t n_h,
-                    int64_t n_b, int64_t stride_t, int64_t stride_h, int64_t stride_b, int box_d, int box_t)
+bool make_tmap(CUtensorMap *out, TmapCoord *coord, const void *base, int D, int64_t n_t, int64_t n_h, int64_t n_b,
+               int64_t stride_t, int64_t stride_h, int64_t stride_b, int box_d, int box_t, int elem_bytes)
 {
-    const TmapKey key{base, D, box_d, box_t, n_t, n_h, n_b, stride_t, stride_h, stride_b};
+    const TmapKey key{base, D, box_d, box_t, elem_bytes, n_t, n_h, n_b, stride_t, stride_h, stride_b};
     {
         std::lock_guard<std::mutex> lock(g_tmap_mutex);
         for (int i = 0; i < kTmapCache; ++i)
@@ -107,7 +107,8 @@ bool make_tmap_bf16(CUtensorMap *out, TmapCoord *coord, const void *base, int D,
                 return true;
             }
     }
-    if (!encode_tmap_bf16(out, coord, base, D, n_t, n_h, n_b, stride_t, stride_h, stride_b, box_d, box_t)) return false;
+    if (!encode_tmap(out, coord, base, D, n_t, n_h, n_b, stride_t, stride_h, stride_b, box_d, box_t, elem_bytes))
+        return false;
     std::lock_guard<std::mutex> lock(g_tmap_mutex);
     TmapEntry &e = g_tmap_cache[g_tmap_next];
     g_tmap_next = (g_tmap_next + 1) % kTmapCache;
@@ -117,8 +118,8 @@ bool make_tmap_bf16(CUtensorMap *out, TmapCoord *coord, const void *base, int D,
 
 namespace {
 
-bool encode_tmap_bf16(CUtensorMap *out, TmapCoord *coord, const void *base, int D, int64_t n_t, int64_t n_h,
-                      int64_t n_b, int64_t stride_t, int64_t stride_h, int64_t stride_b, int box_d, int box_t)
+bool encode_tmap(CUtensorMap *out, TmapCoord *coord, const void *base, int D, int64_t n_t, int64_t n_h, int64_t n_b,
+                 int64_t stride_t, int64_t stride_h, int64_t stride_b, int box_d, int box_t, int elem_bytes)
 {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
@@ -133,10 +134,10 @@ bool encode_tmap_bf16(CUtensorMap *out, TmapCoord *coord, const void *base, int 
     cuuint64_t gstride[3];
     cuuint32_t box[4] = {(cuuint32_t)box_d, 1, 1, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
-    int64_t prev_extent_bytes = (int64_t)D * 2;
+    int64_t prev_extent_bytes = (int64_t)D * elem_bytes;
     for (int i = 0; i < 3; ++i) {
         gdim[i + 1] = (cuuint64_t)(dims[i].n < 1 ? 1 : dims[i].n);
-        int64_t sb = dims[i].stride * 2;
+        int64_t sb = dims[i].stride * elem_bytes;
         if (dims[i].n <= 1 && sb < prev_extent_bytes) sb = prev_extent_bytes;   // never used for addressing
         gstride[i] = (cuuint64_t)sb;
         prev_extent_bytes = sb * (int64_t)gdim[i + 1];
@@ -145,7 +146,7 @@ bool encode_tmap_bf16(CUtensorMap *out, TmapCoord *coord, const void *base, int 
         if (dims[i].which == 1) coord->pos_h = i + 1;
         if (dims[i].which == 2) coord->pos_b = i + 1;
     }
-    CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), gdim, gstride, box, estr,
+    CUresult r = fn(out, elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), gdim, gstride, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
@@ -263,6 +264,51 @@ l4l_status l4l_attn_decode_paged(const void *q, void *o, l4l_paged_kv pool, cons
     const PagedTable pt{d_block_table, table_stride, pool.num_pages};
     return launch_decode(q, o, pool_as_cache(pool), d_kv_lens, max_kv_len, B, Hq, Hkv, head_dim, scale, d_lse, workspace,
                          plan, static_cast<cudaStream_t>(stream), nullptr, nullptr, &pt);
+}
+
+namespace {
+
+// An fp8 cache: byte elements, every row start 16-byte aligned.
+bool cache8_ok(const l4l_kv_cache &c)
+{
+    auto s16 = [](int64_t s) { return s >= 0 && (s % 16) == 0; };
+    return c.k && c.v && aligned16(c.k) && aligned16(c.v) && s16(c.stride_b) && s16(c.stride_h) && s16(c.stride_t) &&
+           c.max_len > 0;
+}
+
+}  // namespace
+
+l4l_status l4l_kv_append_fp8(l4l_kv_cache cache8, l4l_tensor4 k_new, l4l_tensor4 v_new, const int32_t *d_write_pos,
+                             const int32_t *d_n_new, int n_new_max, int B, int Hkv, int head_dim,
+                             const float *d_k_scale, const float *d_v_scale, l4l_stream stream)
+{
+    if (B < 0 || Hkv <= 0 || n_new_max < 0) return L4L_ERR_INVALID_ARG;
+    if (head_dim != 64 && head_dim != 128) return L4L_ERR_UNSUPPORTED;
+    if (!cache8_ok(cache8) || !tensor4_ok(k_new) || !tensor4_ok(v_new) || !d_write_pos || !d_k_scale || !d_v_scale)
+        return L4L_ERR_INVALID_ARG;
+    if (B == 0 || n_new_max == 0) return L4L_OK;
+    return launch_kv_append_fp8(cache8, k_new, v_new, d_write_pos, d_n_new, n_new_max, B, Hkv, head_dim, d_k_scale,
+                                d_v_scale, static_cast<cudaStream_t>(stream));
+}
+
+l4l_status l4l_attn_decode_fp8(const void *q, void *o, l4l_kv_cache cache8, const float *d_k_scale,
+                               const float *d_v_scale, const int32_t *d_kv_lens, int max_kv_len, int B, int Hq, int Hkv,
+                               int head_dim, float scale, float *d_lse, void *workspace, size_t ws_bytes,
+                               l4l_stream stream)
+{
+    l4l_status st = shape_status(B, Hq, Hkv, head_dim);
+    if (st != L4L_OK) return st;
+    if (head_dim != 128) return L4L_ERR_UNSUPPORTED;          // one 128-byte row per token
+    if (!q || !o || !d_kv_lens || !d_k_scale || !d_v_scale || !aligned16(q) || !aligned16(o)) return L4L_ERR_INVALID_ARG;
+    if (!cache8_ok(cache8)) return L4L_ERR_INVALID_ARG;
+    if (max_kv_len < 0 || max_kv_len > cache8.max_len) return L4L_ERR_INVALID_ARG;
+    if (!workspace || ws_bytes < kStatusBytes) return L4L_ERR_WORKSPACE;
+    if (B == 0) return L4L_OK;
+    const DecodePlan plan = plan_decode(B, Hq, Hkv, head_dim, max_kv_len, ws_bytes, true);
+    if (plan.ws_bytes > ws_bytes) return L4L_ERR_WORKSPACE;
+    const Fp8Scales sc{d_k_scale, d_v_scale};
+    return launch_decode(q, o, cache8, d_kv_lens, max_kv_len, B, Hq, Hkv, head_dim, scale, d_lse, workspace, plan,
+                         static_cast<cudaStream_t>(stream), nullptr, nullptr, nullptr, &sc);
 }
 
 l4l_status l4l_rope_kv_append(l4l_tensor4 q, l4l_tensor4 k_new, l4l_tensor4 v_new, l4l_kv_cache cache,

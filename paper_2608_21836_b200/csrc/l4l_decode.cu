@@ -39,14 +39,18 @@ constexpr int kPostRing = 16;               // pieces a producer can be ahead of
 constexpr size_t kTicketBytes = 128 * 1024;  // 32768 (sequence, KV head) pairs per launch
 constexpr int kMaxB = 512;                 // sequences per launch (prefix sums live in shared memory)
 
-template <int D, int W>
+// F8: the cache holds e4m3 bytes (one byte per value) instead of bf16.
+template <int D, int W, bool F8>
 struct DecodeCfg {
+    static_assert(!F8 || D == 128, "the fp8 path wants one 128-byte row per token");
     static constexpr int kTileT = 16 * W;                         // tokens per TMA tile
-    static constexpr int kHalves = D / 64;
-    static constexpr uint32_t kHalfBytes = kTileT * 128;          // [tile tokens][64 dims] bf16
+    static constexpr int kRowBytes = F8 ? D : 2 * D;              // one token of one KV head
+    static constexpr int kHalves = kRowBytes / 128;               // 128-byte column blocks of a tile
+    static constexpr int kBoxD = F8 ? 128 : 64;                   // elements per 128-byte box row
+    static constexpr uint32_t kHalfBytes = kTileT * 128;          // [tile tokens][128 bytes], swizzled
     static constexpr uint32_t kTileBytes = kHalves * kHalfBytes;  // one of K or V
     static constexpr uint32_t kStageBytes = 2 * kTileBytes;
-    static constexpr int kStages = (D == 128) ? 3 : 6;
+    static constexpr int kStages = (kStageBytes >= 32768u * (W / 4)) ? 3 : 6;   // 192 KB (96 KB with W = 4) in flight
 };
 
 struct TileMeta {
@@ -73,6 +77,8 @@ struct DecodeParams {
     __nv_bfloat16 *cache_k, *cache_v;
     int64_t c_sb, c_sh, c_st;
     unsigned *status;
+    // fp8 cache: real value = e4m3 value * scale of its KV head
+    const float *k_scale, *v_scale;           // [Hkv]
     // paged cache (null: contiguous): token t of sequence b lives in page block_table[b * table_stride + t / page_size]
     // at offset t % page_size; the tensor maps then describe the page pool [pages, Hkv, page_size, D]
     const int32_t *block_table;
@@ -82,10 +88,10 @@ struct DecodeParams {
     TmapCoord coord;
 };
 
-template <int D, int W>
+template <int D, int W, bool F8>
 size_t decode_smem_bytes(int G, int nsplit)
 {
-    using C = DecodeCfg<D, W>;
+    using C = DecodeCfg<D, W, F8>;
     size_t comb = (size_t)W * G * (D + 4) * sizeof(float) + (size_t)((G * nsplit + 3) & ~3) * sizeof(float);
     return 1024 /*alignment slack*/ + (size_t)C::kStages * (C::kStageBytes + (size_t)G * D * 2) + comb +
            C::kStages * sizeof(TileMeta) +
@@ -100,13 +106,13 @@ __device__ __forceinline__ void order_coords(const TmapCoord &c, int t, int h, i
     c3 = (c.pos_t == 3) ? t : (c.pos_h == 3) ? h : b;
 }
 
-template <int D, int W>
+template <int D, int W, bool F8>
 __global__ void __launch_bounds__((W + 2) * 32)
 decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
                     const __grid_constant__ CUtensorMap tmap_k16, const __grid_constant__ CUtensorMap tmap_v16,
                     const DecodeParams p)
 {
-    using C = DecodeCfg<D, W>;
+    using C = DecodeCfg<D, W, F8>;
     constexpr int kTileT = C::kTileT;
     constexpr int kConsumerWarps = W, kProducerWarp = W, kFinisherWarp = W + 1;
     extern __shared__ uint8_t smem_raw[];
@@ -268,8 +274,8 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                             uint8_t *db = dst + bx * box_rows * 128;  // whole 8-row groups: the swizzle phase is kept
 #pragma unroll
                             for (int hf = 0; hf < C::kHalves; ++hf) {
-                                tma_load_4d(db + hf * C::kHalfBytes, &tmap_k, &full[s], hf * 64, c1, c2, c3);
-                                tma_load_4d(db + C::kTileBytes + hf * C::kHalfBytes, &tmap_v, &full[s], hf * 64, c1, c2, c3);
+                                tma_load_4d(db + hf * C::kHalfBytes, &tmap_k, &full[s], hf * C::kBoxD, c1, c2, c3);
+                                tma_load_4d(db + C::kTileBytes + hf * C::kHalfBytes, &tmap_v, &full[s], hf * C::kBoxD, c1, c2, c3);
                             }
                         }
                     } else {
@@ -286,8 +292,8 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                             uint8_t *dg = dst + gq * 16 * 128;        // 2 KB per group: the swizzle phase is kept
 #pragma unroll
                             for (int hf = 0; hf < C::kHalves; ++hf) {
-                                tma_load_4d(dg + hf * C::kHalfBytes, &tmap_k16, &full[s], hf * 64, c1, c2, c3);
-                                tma_load_4d(dg + C::kTileBytes + hf * C::kHalfBytes, &tmap_v16, &full[s], hf * 64, c1, c2, c3);
+                                tma_load_4d(dg + hf * C::kHalfBytes, &tmap_k16, &full[s], hf * C::kBoxD, c1, c2, c3);
+                                tma_load_4d(dg + C::kTileBytes + hf * C::kHalfBytes, &tmap_v16, &full[s], hf * C::kBoxD, c1, c2, c3);
                             }
                         }
                     }
@@ -619,11 +625,20 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 const bool v_lo = r_lo < p.G, v_hi = r_hi < p.G;
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
-                    const int w = ks * 8 + (lane & 3);               // 32-bit word index in the row
-                    qf[ks][0] = v_lo ? qrow_lo[w] : 0u;
-                    qf[ks][1] = v_hi ? qrow_hi[w] : 0u;
-                    qf[ks][2] = v_lo ? qrow_lo[w + 4] : 0u;
-                    qf[ks][3] = v_hi ? qrow_hi[w + 4] : 0u;
+                    if constexpr (F8) {
+                        // f16 fragments with the k index permuted the way the fp8 K tiles arrive
+                        const int w = q_frag_f8_word(ks, 0, lane);
+                        qf[ks][0] = v_lo ? bf16x2_to_f16x2(qrow_lo[w]) : 0u;
+                        qf[ks][1] = v_hi ? bf16x2_to_f16x2(qrow_hi[w]) : 0u;
+                        qf[ks][2] = v_lo ? bf16x2_to_f16x2(qrow_lo[w + 1]) : 0u;
+                        qf[ks][3] = v_hi ? bf16x2_to_f16x2(qrow_hi[w + 1]) : 0u;
+                    } else {
+                        const int w = ks * 8 + (lane & 3);           // 32-bit word index in the row
+                        qf[ks][0] = v_lo ? qrow_lo[w] : 0u;
+                        qf[ks][1] = v_hi ? qrow_hi[w] : 0u;
+                        qf[ks][2] = v_lo ? qrow_lo[w + 4] : 0u;
+                        qf[ks][3] = v_hi ? qrow_hi[w + 4] : 0u;
+                    }
                 }
             }
 
@@ -632,7 +647,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             const int row0 = warp * 16;
             const int nvalid = mt.kv_len - (mt.t0 + row0);       // valid tokens in this warp's slice
             bool wrote_smem = false;
-            if (p.k_new != nullptr && nvalid > 0 && nvalid <= 16) {
+            if (!F8 && p.k_new != nullptr && nvalid > 0 && nvalid <= 16) {
                 // fused append: this slice holds the sequence's newest token (row `last` of the tile). Its K/V
                 // arrive from the caller, not from the cache: patch the tile in shared memory and write the
                 // cache slot (each slot belongs to exactly one CTA's range and one warp's slice).
@@ -656,12 +671,18 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             }
             if (nvalid > 0) {
                 float s_lo[4], s_hi[4];
-                warp_qk_16x16<D>(qf, k_tile, C::kHalfBytes, row0, s_lo, s_hi);
+                float sc = p.scale_log2e;
+                if constexpr (F8) {
+                    warp_qk_16x16_f8<D>(qf, k_tile, row0, s_lo, s_hi);
+                    sc *= __ldg(p.k_scale + mt.kvh);
+                } else {
+                    warp_qk_16x16<D>(qf, k_tile, C::kHalfBytes, row0, s_lo, s_hi);
+                }
                 const int tok = 2 * (lane & 3);
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    s_lo[e] *= p.scale_log2e;
-                    s_hi[e] *= p.scale_log2e;
+                    s_lo[e] *= sc;
+                    s_hi[e] *= sc;
                 }
                 if (nvalid < 16) {
                     // tokens past the end of the sequence: no weight, and their V rows (which may
@@ -672,7 +693,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                         if (tok + (e & 1) + 8 >= nvalid) s_hi[e] = -INFINITY;
                     }
                     uint8_t *vt = stages + (size_t)s * C::kStageBytes + C::kTileBytes;
-                    const int chunks_per_row = D / 8;
+                    const int chunks_per_row = C::kRowBytes / 16;
                     for (int i = lane; i < (16 - nvalid) * chunks_per_row; i += 32) {
                         const int r = row0 + nvalid + i / chunks_per_row;
                         const int ch = i % chunks_per_row;
@@ -683,8 +704,11 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     __syncwarp();
                 }
                 uint32_t pa[4];
-                warp_softmax_16<D>(st, s_lo, s_hi, pa);
-                warp_pv_16x16<D>(st, pa, v_tile, C::kHalfBytes, row0);
+                warp_softmax_16<D, F8>(st, s_lo, s_hi, pa);
+                if constexpr (F8)
+                    warp_pv_16x16_f8<D>(st, pa, v_tile, row0);
+                else
+                    warp_pv_16x16<D>(st, pa, v_tile, C::kHalfBytes, row0);
             }
 
             if (wrote_smem) fence_proxy_async_smem();   // generic writes before the next TMA fill
@@ -700,19 +724,38 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
                 l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
                 float *cw = comb + (size_t)warp * p.G * kPitch;
+                // fp8: accumulator tiles alternate even / odd head dims (a tile pair gives this lane 4 consecutive
+                // dims) and O still lacks the V scale of its KV head
+                const float vs = F8 ? __ldg(p.v_scale + mt.kvh) : 1.f;
                 if (r_lo < p.G) {
                     float *row = cw + (size_t)r_lo * kPitch;
                     if ((lane & 3) == 0) { row[D] = st.m[0]; row[D + 1] = l0; }
+                    if constexpr (F8) {
 #pragma unroll
-                    for (int nt = 0; nt < D / 8; ++nt)
-                        *reinterpret_cast<float2 *>(row + nt * 8 + 2 * (lane & 3)) = make_float2(st.o[nt][0], st.o[nt][1]);
+                        for (int ch = 0; ch < D / 16; ++ch)
+                            *reinterpret_cast<float4 *>(row + ch * 16 + 4 * (lane & 3)) =
+                                make_float4(st.o[2 * ch][0] * vs, st.o[2 * ch + 1][0] * vs, st.o[2 * ch][1] * vs,
+                                            st.o[2 * ch + 1][1] * vs);
+                    } else {
+#pragma unroll
+                        for (int nt = 0; nt < D / 8; ++nt)
+                            *reinterpret_cast<float2 *>(row + nt * 8 + 2 * (lane & 3)) = make_float2(st.o[nt][0], st.o[nt][1]);
+                    }
                 }
                 if (r_hi < p.G) {
                     float *row = cw + (size_t)r_hi * kPitch;
                     if ((lane & 3) == 0) { row[D] = st.m[1]; row[D + 1] = l1; }
+                    if constexpr (F8) {
 #pragma unroll
-                    for (int nt = 0; nt < D / 8; ++nt)
-                        *reinterpret_cast<float2 *>(row + nt * 8 + 2 * (lane & 3)) = make_float2(st.o[nt][2], st.o[nt][3]);
+                        for (int ch = 0; ch < D / 16; ++ch)
+                            *reinterpret_cast<float4 *>(row + ch * 16 + 4 * (lane & 3)) =
+                                make_float4(st.o[2 * ch][2] * vs, st.o[2 * ch + 1][2] * vs, st.o[2 * ch][3] * vs,
+                                            st.o[2 * ch + 1][3] * vs);
+                    } else {
+#pragma unroll
+                        for (int nt = 0; nt < D / 8; ++nt)
+                            *reinterpret_cast<float2 *>(row + nt * 8 + 2 * (lane & 3)) = make_float2(st.o[nt][2], st.o[nt][3]);
+                    }
                 }
                 if (warp == 0 && lane == 0) {
                     piece_meta->b = mt.b; piece_meta->kvh = mt.kvh; piece_meta->piece = mt.piece;
@@ -733,20 +776,20 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
 }
 
 // Resident CTAs per SM for a given dynamic shared-memory size (0 on failure).
-template <int D, int W>
+template <int D, int W, bool F8>
 int decode_blocks_per_sm(size_t smem)
 {
     static bool attr_set = false;
     if (!attr_set) {
         // the opt-in limit is per kernel: allow everything the SM has
-        if (cudaFuncSetAttribute(decode_split_kernel<D, W>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+        if (cudaFuncSetAttribute(decode_split_kernel<D, W, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
             cudaSuccess)
             return 0;
         attr_set = true;
     }
     if (smem > 227 * 1024) return 0;
     int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_split_kernel<D, W>, (W + 2) * 32, smem) != cudaSuccess)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_split_kernel<D, W, F8>, (W + 2) * 32, smem) != cudaSuccess)
         return 0;
     return n;
 }
@@ -762,27 +805,29 @@ struct ShapeOps {
     int (*blocks_per_sm)(size_t smem);
 };
 
-template <int D, int W>
+template <int D, int W, bool F8>
 ShapeOps shape_ops()
 {
-    return ShapeOps{W, 16 * W, &decode_smem_bytes<D, W>, &decode_blocks_per_sm<D, W>};
+    return ShapeOps{W, 16 * W, &decode_smem_bytes<D, W, F8>, &decode_blocks_per_sm<D, W, F8>};
 }
 
-ShapeOps pick_shape(int D, int warps)
+ShapeOps pick_shape(int D, int warps, bool fp8)
 {
-    if (D == 128) return warps == 8 ? shape_ops<128, 8>() : shape_ops<128, 4>();
-    return warps == 8 ? shape_ops<64, 8>() : shape_ops<64, 4>();
+    if (fp8) return warps == 8 ? shape_ops<128, 8, true>() : shape_ops<128, 4, true>();      // D == 128 only
+    if (D == 128) return warps == 8 ? shape_ops<128, 8, false>() : shape_ops<128, 4, false>();
+    return warps == 8 ? shape_ops<64, 8, false>() : shape_ops<64, 4, false>();
 }
 
 // Plan for one kernel shape (warps = 4 or 8).
-DecodePlan plan_for_shape(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_limit, int warps, bool have_dev)
+DecodePlan plan_for_shape(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_limit, int warps, bool have_dev,
+                          bool fp8)
 {
     // Grid: every resident CTA slot of the device. A floor on the tiles per CTA bounds the number of
     // pieces a sequence can be cut into (and with it the partials in the workspace and the finisher's
     // scratch) when the real lengths are far below max_kv_len; it is raised until the partials fit the
     // caller's workspace and the shared memory fits the SM.
     DecodePlan pl;
-    const ShapeOps ops = pick_shape(D, warps);
+    const ShapeOps ops = pick_shape(D, warps, fp8);
     pl.warps = warps;
     const int G = Hq / Hkv;
     auto blocks = [&](int nsplit) {
@@ -822,7 +867,7 @@ DecodePlan plan_for_shape(int B, int Hq, int Hkv, int D, int max_kv_len, size_t 
 
 }  // namespace
 
-DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_limit)
+DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_limit, bool fp8)
 {
     int n_dev = 0;
     const bool have_dev = cudaGetDeviceCount(&n_dev) == cudaSuccess && n_dev > 0;
@@ -834,22 +879,25 @@ DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_
         return e ? atoi(e) : 0;
     }();
     if (forced != 4) {
-        const DecodePlan p8 = plan_for_shape(B, Hq, Hkv, D, max_kv_len, ws_limit, 8, have_dev);
+        const DecodePlan p8 = plan_for_shape(B, Hq, Hkv, D, max_kv_len, ws_limit, 8, have_dev, fp8);
         if (p8.fits && p8.ws_bytes <= ws_limit) return p8;
         if (forced == 8) return p8;
     }
-    return plan_for_shape(B, Hq, Hkv, D, max_kv_len, ws_limit, 4, have_dev);
+    return plan_for_shape(B, Hq, Hkv, D, max_kv_len, ws_limit, 4, have_dev, fp8);
 }
 
 l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, const int32_t *d_kv_lens,
                          int max_kv_len, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
                          void *workspace, const DecodePlan &plan, cudaStream_t stream, const l4l_tensor4 *k_new,
-                         const l4l_tensor4 *v_new, const PagedTable *paged)
+                         const l4l_tensor4 *v_new, const PagedTable *paged, const Fp8Scales *fp8)
 {
+    // fp8: cache.k / cache.v point at e4m3 bytes, the strides count bytes (= elements)
+    if (fp8 && (D != 128 || k_new || v_new)) return L4L_ERR_UNSUPPORTED;
+    const int esz = fp8 ? 1 : 2;
     // paged: `cache` describes the page pool (stride_b = stride between pages, max_len = page size)
     if (paged && (k_new || v_new)) return L4L_ERR_UNSUPPORTED;
     const int G = Hq / Hkv;
-    const ShapeOps ops = pick_shape(D, plan.warps);
+    const ShapeOps ops = pick_shape(D, plan.warps, fp8 != nullptr);
     const int kTileT = ops.tile_t;
     const size_t smem = ops.smem_bytes(G, plan.nsplit);
     if (ops.blocks_per_sm(smem) == 0) return L4L_ERR_CUDA;
@@ -870,18 +918,19 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         // contiguous: the maps cover this slice's sequences; paged: the whole pool, whatever the slice
         const size_t first = paged ? 0 : (size_t)b0 * cache.stride_b;
         const int outer = paged ? paged->num_pages : nb;
-        const __nv_bfloat16 *kb = static_cast<const __nv_bfloat16 *>(cache.k) + first;
-        const __nv_bfloat16 *vb = static_cast<const __nv_bfloat16 *>(cache.v) + first;
+        const uint8_t *kb = static_cast<const uint8_t *>(cache.k) + first * esz;
+        const uint8_t *vb = static_cast<const uint8_t *>(cache.v) + first * esz;
+        const int box_d = fp8 ? 128 : 64;
         // pages smaller than a tile are fetched page by page: no box may exceed the page
         const int box_t = (paged && cache.max_len < kTileT) ? cache.max_len : kTileT;
-        if (!make_tmap_bf16(&tk, &coord, kb, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
-                            cache.stride_b, 64, box_t) ||
-            !make_tmap_bf16(&tv, &coord_v, vb, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
-                            cache.stride_b, 64, box_t) ||
-            !make_tmap_bf16(&tk16, &coord_v, kb, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
-                            cache.stride_b, 64, 16) ||
-            !make_tmap_bf16(&tv16, &coord_v, vb, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
-                            cache.stride_b, 64, 16))
+        if (!make_tmap(&tk, &coord, kb, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
+                       cache.stride_b, box_d, box_t, esz) ||
+            !make_tmap(&tv, &coord_v, vb, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
+                       cache.stride_b, box_d, box_t, esz) ||
+            !make_tmap(&tk16, &coord_v, kb, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
+                       cache.stride_b, box_d, 16, esz) ||
+            !make_tmap(&tv16, &coord_v, vb, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
+                       cache.stride_b, box_d, 16, esz))
             return L4L_ERR_CUDA;
         DecodeParams p;
         p.q = static_cast<const __nv_bfloat16 *>(q) + (size_t)b0 * Hq * D;
@@ -896,13 +945,16 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         p.max_kv_len = max_kv_len;
         p.k_new = p.v_new = nullptr;
         p.new_sb = p.new_sh = 0;
+        p.k_scale = fp8 ? fp8->k_scale : nullptr;
+        p.v_scale = fp8 ? fp8->v_scale : nullptr;
         p.block_table = paged ? paged->block_table + (size_t)b0 * paged->table_stride : nullptr;
         p.table_stride = paged ? paged->table_stride : 0;
         p.page_size = paged ? cache.max_len : 0;
         p.page_shift = 0;
         while (paged && (1 << p.page_shift) < cache.max_len) ++p.page_shift;
-        p.cache_k = static_cast<__nv_bfloat16 *>(cache.k) + (size_t)b0 * cache.stride_b;
-        p.cache_v = static_cast<__nv_bfloat16 *>(cache.v) + (size_t)b0 * cache.stride_b;
+        // only the fused append (bf16, contiguous) writes through these
+        p.cache_k = static_cast<__nv_bfloat16 *>(cache.k) + (fp8 ? 0 : (size_t)b0 * cache.stride_b);
+        p.cache_v = static_cast<__nv_bfloat16 *>(cache.v) + (fp8 ? 0 : (size_t)b0 * cache.stride_b);
         p.c_sb = cache.stride_b; p.c_sh = cache.stride_h; p.c_st = cache.stride_t;
         if (k_new && v_new) {
             if (k_new->stride_b != v_new->stride_b || k_new->stride_h != v_new->stride_h) return L4L_ERR_UNSUPPORTED;
@@ -923,12 +975,15 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         cudaError_t err;
-        if (D == 128)
-            err = plan.warps == 8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 8>, tk, tv, tk16, tv16, p)
-                                  : cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 4>, tk, tv, tk16, tv16, p);
+        if (fp8)
+            err = plan.warps == 8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 8, true>, tk, tv, tk16, tv16, p)
+                                  : cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 4, true>, tk, tv, tk16, tv16, p);
+        else if (D == 128)
+            err = plan.warps == 8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 8, false>, tk, tv, tk16, tv16, p)
+                                  : cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 4, false>, tk, tv, tk16, tv16, p);
         else
-            err = plan.warps == 8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<64, 8>, tk, tv, tk16, tv16, p)
-                                  : cudaLaunchKernelEx(&cfg, decode_split_kernel<64, 4>, tk, tv, tk16, tv16, p);
+            err = plan.warps == 8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<64, 8, false>, tk, tv, tk16, tv16, p)
+                                  : cudaLaunchKernelEx(&cfg, decode_split_kernel<64, 4, false>, tk, tv, tk16, tv16, p);
         if (err != cudaSuccess) return L4L_ERR_CUDA;
     }
     return L4L_OK;
@@ -1006,5 +1061,5 @@ extern "C" l4l_status l4l_attn_decode_static(const void *q, void *o, l4l_kv_cach
     const size_t zero_bytes = kStatusBytes + kTicketBytes;
     if (cudaMemsetAsync(scratch, 0, zero_bytes, s) != cudaSuccess) return L4L_ERR_CUDA;
     return launch_decode(q, o, cache, d_kv_lens, max_kv_len, B, Hq, Hkv, head_dim, scale, d_lse, scratch, plan, s,
-                         nullptr, nullptr, nullptr);
+                         nullptr, nullptr, nullptr, nullptr);
 }

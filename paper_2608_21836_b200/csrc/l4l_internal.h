@@ -16,11 +16,17 @@ struct TmapCoord {
     int pos_t, pos_h, pos_b;
 };
 
-// Builds a tiled bf16 tensor map over a [batch, head, token, D]-indexable buffer with the
-// given element strides; the box is box_d x box_t (x1x1) with the 128-byte swizzle
-// (box_d must be 64). Returns false (and leaves *out undefined) if the driver refuses.
-bool make_tmap_bf16(CUtensorMap *out, TmapCoord *coord, const void *base, int D, int64_t n_t, int64_t n_h,
-                    int64_t n_b, int64_t stride_t, int64_t stride_h, int64_t stride_b, int box_d, int box_t);
+// Builds a tiled tensor map over a [batch, head, token, D]-indexable buffer of bf16 (elem_bytes = 2) or
+// single bytes (elem_bytes = 1) with the given element strides; the box is box_d x box_t (x1x1) with the
+// 128-byte swizzle (box_d * elem_bytes must be 128). Returns false (and leaves *out undefined) if the
+// driver refuses.
+bool make_tmap(CUtensorMap *out, TmapCoord *coord, const void *base, int D, int64_t n_t, int64_t n_h, int64_t n_b,
+               int64_t stride_t, int64_t stride_h, int64_t stride_b, int box_d, int box_t, int elem_bytes);
+inline bool make_tmap_bf16(CUtensorMap *out, TmapCoord *coord, const void *base, int D, int64_t n_t, int64_t n_h,
+                           int64_t n_b, int64_t stride_t, int64_t stride_h, int64_t stride_b, int box_d, int box_t)
+{
+    return make_tmap(out, coord, base, D, n_t, n_h, n_b, stride_t, stride_h, stride_b, box_d, box_t, 2);
+}
 
 int sm_count();
 
@@ -32,7 +38,7 @@ struct DecodePlan {
     int nsplit;      // max pieces a (sequence, KV head) can be cut into
     size_t ws_bytes; // status block + ticket counters + partials
 };
-DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_limit);
+DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_limit, bool fp8 = false);
 
 // Block table of a paged cache: token t of sequence b is in page block_table[b * table_stride + t / page_size].
 struct PagedTable {
@@ -41,12 +47,18 @@ struct PagedTable {
     int num_pages;                // pages in the pool
 };
 
+// Scales of an fp8 (e4m3) cache: real value = stored value * scale of its KV head.
+struct Fp8Scales {
+    const float *k_scale, *v_scale;   // device, [Hkv]
+};
+
 // With `paged`, `cache` describes the page pool: stride_b = stride between pages, max_len = page size.
+// With `fp8`, cache.k / cache.v hold e4m3 bytes and the strides count bytes.
 l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, const int32_t *d_kv_lens,
                          int max_kv_len, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
                          void *workspace, const DecodePlan &plan, cudaStream_t stream,
                          const l4l_tensor4 *k_new = nullptr, const l4l_tensor4 *v_new = nullptr,
-                         const PagedTable *paged = nullptr);
+                         const PagedTable *paged = nullptr, const Fp8Scales *fp8 = nullptr);
 
 l4l_status launch_rope_kv_append(const l4l_tensor4 &q, const l4l_tensor4 &k_new, const l4l_tensor4 &v_new,
                                  const l4l_kv_cache &cache, const int32_t *d_pos, const int32_t *d_n_new, int T, int B,
@@ -55,6 +67,10 @@ l4l_status launch_rope_kv_append(const l4l_tensor4 &q, const l4l_tensor4 &k_new,
 l4l_status launch_kv_append(const l4l_kv_cache &cache, const l4l_tensor4 &k_new, const l4l_tensor4 &v_new,
                             const int32_t *d_write_pos, const int32_t *d_n_new, int n_new_max, int B, int Hkv,
                             int D, cudaStream_t stream, const PagedTable *paged = nullptr);
+
+l4l_status launch_kv_append_fp8(const l4l_kv_cache &cache, const l4l_tensor4 &k_new, const l4l_tensor4 &v_new,
+                                const int32_t *d_write_pos, const int32_t *d_n_new, int n_new_max, int B, int Hkv,
+                                int D, const float *d_k_scale, const float *d_v_scale, cudaStream_t stream);
 
 l4l_status launch_prefill(const l4l_tensor4 &q, const l4l_tensor4 &k, const l4l_tensor4 &v,
                           const l4l_tensor4 &o, const l4l_kv_cache &cache, const int32_t *d_seq_lens,

@@ -52,7 +52,8 @@ __device__ __forceinline__ void warp_qk_16x16(const uint32_t (&qf)[D / 16][4], u
 
 // Online-softmax update for 16 tokens. Scores arrive already multiplied by scale*log2(e)
 // and with masked positions set to -inf. Produces the bf16 A-fragment of P and rescales O.
-template <int D>
+// kF16: P is packed as f16 (for the f16 MMAs of the fp8-cache path) instead of bf16.
+template <int D, bool kF16 = false>
 __device__ __forceinline__ void warp_softmax_16(WarpAttnState<D> &st, const float (&s_lo)[4], const float (&s_hi)[4],
                                                 uint32_t (&pa)[4])
 {
@@ -65,13 +66,16 @@ __device__ __forceinline__ void warp_softmax_16(WarpAttnState<D> &st, const floa
         const float m_new = fmaxf(st.m[h], mx);
         const float m_use = (m_new == -INFINITY) ? 0.f : m_new;     // row with nothing visible yet
         const float corr = fast_exp2(st.m[h] - m_use);
-        const uint32_t p01 = pack_bf16x2(fast_exp2(a0 - m_use), fast_exp2(a1 - m_use));
-        const uint32_t p23 = pack_bf16x2(fast_exp2(a2 - m_use), fast_exp2(a3 - m_use));
+        const float e0 = fast_exp2(a0 - m_use), e1 = fast_exp2(a1 - m_use);
+        const float e2 = fast_exp2(a2 - m_use), e3 = fast_exp2(a3 - m_use);
+        const uint32_t p01 = kF16 ? pack_f16x2(e0, e1) : pack_bf16x2(e0, e1);
+        const uint32_t p23 = kF16 ? pack_f16x2(e2, e3) : pack_bf16x2(e2, e3);
         pa[h] = p01;          // tokens +0,+1
         pa[2 + h] = p23;      // tokens +8,+9
         // the denominator sums exactly the rounded weights that multiply V
-        const float psum = __uint_as_float(p01 << 16) + __uint_as_float(p01 & 0xffff0000u) +
-                           __uint_as_float(p23 << 16) + __uint_as_float(p23 & 0xffff0000u);
+        const float psum = kF16 ? sum_f16x2(p01) + sum_f16x2(p23)
+                                : __uint_as_float(p01 << 16) + __uint_as_float(p01 & 0xffff0000u) +
+                                      __uint_as_float(p23 << 16) + __uint_as_float(p23 & 0xffff0000u);
         st.l[h] = st.l[h] * corr + psum;
         st.m[h] = m_new;
 #pragma unroll
@@ -98,6 +102,66 @@ __device__ __forceinline__ void warp_pv_16x16(WarpAttnState<D> &st, const uint32
         ldmatrix_x4_trans(addr, b0, b1, b2, b3);
         mma_bf16_16816(st.o[2 * np], pa, b0, b1);
         mma_bf16_16816(st.o[2 * np + 1], pa, b2, b3);
+    }
+}
+
+// ----------------------------------------------------------------------------- fp8 (e4m3) K/V tiles
+// A tile is [tile_tokens][128 bytes] (D = 128 values per token), 128-byte swizzled. The values are
+// widened to f16 in registers (exact) and multiplied with f16 MMAs. ldmatrix moves 16-bit units, so a
+// thread receives 4 consecutive head-dim bytes of a K row where the MMA wants two separate pairs: the
+// k index of QK^T is therefore permuted (MMA slots 2c, 2c+1, 2c+8, 2c+9 of a 16-block hold head dims
+// 4c .. 4c+3), and the q fragments are built with the same permutation (see q_frag_f8_word). For V the
+// transposing ldmatrix delivers, per thread, two tokens of an EVEN and an ODD head dim: the 8-column
+// MMA tiles of O alternate even / odd dims (tile 2j: dims 16j + 2x, tile 2j+1: dims 16j + 2x + 1 in
+// column x); a thread's accumulators of a tile pair are then 4 consecutive head dims.
+
+// 32-bit word (two bf16) of a q row that feeds A-fragment register `reg` (0..3) of k-step ks, as f16x2.
+__device__ __forceinline__ int q_frag_f8_word(int ks, int reg, int lane) { return ks * 8 + 2 * (lane & 3) + (reg >> 1); }
+
+__device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t v)
+{
+    return pack_f16x2(__uint_as_float(v << 16), __uint_as_float(v & 0xffff0000u));
+}
+
+template <int D>
+__device__ __forceinline__ void warp_qk_16x16_f8(const uint32_t (&qf)[D / 16][4], uint32_t k_tile, int row0,
+                                                 float (&s_lo)[4], float (&s_hi)[4])
+{
+    static_assert(D == 128, "one 128-byte row per token");
+    const int lane = threadIdx.x & 31;
+    s_lo[0] = s_lo[1] = s_lo[2] = s_lo[3] = 0.f;
+    s_hi[0] = s_hi[1] = s_hi[2] = s_hi[3] = 0.f;
+    const uint32_t row = row0 + ((lane >> 4) << 3) + (lane & 7);   // matrices 2,3: tokens +8
+    const uint32_t csel = (lane >> 3) & 1;                          // matrices 1,3: next 16 head dims
+#pragma unroll
+    for (int qd = 0; qd < D / 32; ++qd) {
+        uint32_t r0, r1, r2, r3;
+        ldmatrix_x4(k_tile + swz128(row, 2 * qd + csel), r0, r1, r2, r3);
+        mma_f16_16816(s_lo, qf[2 * qd], e4m3x2_to_f16x2(r0), e4m3x2_to_f16x2(r0 >> 16));
+        mma_f16_16816(s_lo, qf[2 * qd + 1], e4m3x2_to_f16x2(r1), e4m3x2_to_f16x2(r1 >> 16));
+        mma_f16_16816(s_hi, qf[2 * qd], e4m3x2_to_f16x2(r2), e4m3x2_to_f16x2(r2 >> 16));
+        mma_f16_16816(s_hi, qf[2 * qd + 1], e4m3x2_to_f16x2(r3), e4m3x2_to_f16x2(r3 >> 16));
+    }
+}
+
+template <int D>
+__device__ __forceinline__ void warp_pv_16x16_f8(WarpAttnState<D> &st, const uint32_t (&pa)[4], uint32_t v_tile, int row0)
+{
+    static_assert(D == 128, "one 128-byte row per token");
+    const int lane = threadIdx.x & 31;
+    const uint32_t row = row0 + (((lane >> 3) & 1) << 3) + (lane & 7);   // matrices 1,3: tokens +8
+    const uint32_t csel = lane >> 4;                                      // matrices 2,3: next 16 head dims
+#pragma unroll
+    for (int qd = 0; qd < D / 32; ++qd) {
+        uint32_t r0, r1, r2, r3;
+        ldmatrix_x4_trans(v_tile + swz128(row, 2 * qd + csel), r0, r1, r2, r3);
+        // bytes (tok, even) (tok, odd) (tok+1, even) (tok+1, odd) -> (tok, even) (tok+1, even) | (tok, odd) (tok+1, odd)
+        const uint32_t x0 = __byte_perm(r0, 0u, 0x3120), x1 = __byte_perm(r1, 0u, 0x3120);
+        const uint32_t x2 = __byte_perm(r2, 0u, 0x3120), x3 = __byte_perm(r3, 0u, 0x3120);
+        mma_f16_16816(st.o[4 * qd], pa, e4m3x2_to_f16x2(x0), e4m3x2_to_f16x2(x1));
+        mma_f16_16816(st.o[4 * qd + 1], pa, e4m3x2_to_f16x2(x0 >> 16), e4m3x2_to_f16x2(x1 >> 16));
+        mma_f16_16816(st.o[4 * qd + 2], pa, e4m3x2_to_f16x2(x2), e4m3x2_to_f16x2(x3));
+        mma_f16_16816(st.o[4 * qd + 3], pa, e4m3x2_to_f16x2(x2 >> 16), e4m3x2_to_f16x2(x3 >> 16));
     }
 }
 

@@ -19,6 +19,8 @@ class Guarded:
             buf = torch.full((n + 2 * GUARD_ELEMS,), fill_bits, dtype=torch.int16, device="cuda").view(torch.bfloat16)
         elif t.dtype == torch.float32:
             buf = torch.full((n + 2 * GUARD_ELEMS,), float("nan"), dtype=torch.float32, device="cuda")
+        elif t.dtype == torch.uint8:                       # fp8 codes: 0x7F is the e4m3 NaN
+            buf = torch.full((n + 2 * GUARD_ELEMS,), 0x7F, dtype=torch.uint8, device="cuda")
         else:
             raise TypeError(t.dtype)
         self.buf = buf
@@ -27,7 +29,10 @@ class Guarded:
         self._ref = buf.clone()
 
     def margins_intact(self) -> bool:
-        a = self.buf.view(torch.int16) if self.buf.dtype == torch.bfloat16 else self.buf.view(torch.int32)
+        if self.buf.dtype == torch.uint8:
+            a = self.buf
+        else:
+            a = self.buf.view(torch.int16) if self.buf.dtype == torch.bfloat16 else self.buf.view(torch.int32)
         b = self._ref.view(a.dtype)
         return bool(torch.equal(a[:GUARD_ELEMS], b[:GUARD_ELEMS]) and torch.equal(a[-GUARD_ELEMS:], b[-GUARD_ELEMS:]))
 

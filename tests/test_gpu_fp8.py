@@ -1,0 +1,110 @@
+"""fp8 (e4m3) KV cache: l4l_kv_append_fp8 (bit-exact codes) and l4l_attn_decode_fp8 against the oracle."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import l4l_oracle as orc
+from paper_2608_21836_b200 import binding as l4l
+from helpers import Guarded, assert_close_to_oracle
+
+pytestmark = pytest.mark.gpu
+
+
+def random_codes(shape, g, max_exp_field=11):
+    """Random e4m3 codes without NaN, magnitudes below 2^(max_exp_field - 6)."""
+    c = torch.randint(0, 256, shape, generator=g, dtype=torch.uint8)
+    e = (c >> 3) & 15
+    c = torch.where(e > max_exp_field, c & 0x87 | (max_exp_field << 3), c)
+    return c
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(32, 8), (8, 8), (16, 2)])
+def test_fp8_decode_matches_oracle(Hq, Hkv):
+    D, Lmax = 128, 2304
+    lens = [1, 15, 16, 17, 127, 128, 129, 700, 1024, 2049, 2304, 0, 333]
+    B = len(lens)
+    g = torch.Generator().manual_seed(1000 + Hq)
+    ck8 = random_codes((B, Hkv, Lmax, D), g, 7)              # |k| < 2
+    cv8 = random_codes((B, Hkv, Lmax, D), g, 7)              # |v| < 2: the absolute tolerance presumes O(1) outputs
+    for b, L in enumerate(lens):                             # slots past the end hold the NaN code
+        ck8[b, :, L:] = 0x7F
+        cv8[b, :, L:] = 0xFF
+    q = torch.randn(B, Hq, D, generator=g).to(torch.bfloat16)
+    ks = (torch.rand(Hkv, generator=g) + 0.5)
+    vs = (torch.rand(Hkv, generator=g) + 0.25)
+    scale = 1.0 / math.sqrt(D)
+    ref, ref_lse = orc.decode_fp8(q, ck8, cv8, np.array(lens, np.int32), ks.numpy(), vs.numpy(), scale)
+    gk, gv = Guarded(ck8), Guarded(cv8)
+    go = Guarded(torch.zeros(B, Hq, D, dtype=torch.bfloat16))
+    lse = torch.zeros(B, Hq, device="cuda")
+    ws = l4l.new_workspace(l4l.L4L_OP_DECODE, B, Hq, Hkv, D, Lmax)
+    l4l.l4l_attn_decode_fp8(q.cuda(), go.t, gk.t, gv.t, ks.cuda(), vs.cuda(), torch.tensor(lens, dtype=torch.int32).cuda(),
+                            Lmax, scale, ws, lse=lse)
+    torch.cuda.synchronize()
+    assert l4l.l4l_last_device_error(ws) == 0
+    assert gk.margins_intact() and gv.margins_intact() and go.margins_intact()
+    assert torch.equal(gk.t.cpu(), ck8) and torch.equal(gv.t.cpu(), cv8)
+    assert_close_to_oracle(go.t.cpu(), ref, "fp8 decode")
+    fin = np.isfinite(ref_lse)
+    assert np.abs(lse.cpu().double().numpy()[fin] - ref_lse[fin]).max() <= 2e-3
+    assert (lse.cpu().numpy()[~fin] == -np.inf).all()
+
+
+def test_fp8_decode_on_the_benchmark_batch_and_against_the_bf16_path():
+    """The ragged B=32 batch quantised with the library's own append: the fp8 kernel must match the oracle on the
+    codes, and (a sanity check of the whole idea) stay near the bf16 kernel on the unquantised cache."""
+    from paper_2608_21836_b200 import workloads as wl
+
+    w = wl.WORKLOADS["batched_decode"]
+    db = wl.make_decode_batch(w)
+    B, Hq, Hkv, D, Lmax = w.decode_B, w.Hq, w.Hkv, w.D, w.decode_Lmax
+    ck = torch.nan_to_num(db.cache_k.float(), nan=0.0).to(torch.bfloat16).cuda()     # the NaN tails would not quantise
+    cv = torch.nan_to_num(db.cache_v.float(), nan=0.0).to(torch.bfloat16).cuda()
+    ks = torch.full((Hkv,), 4.5 / 448, device="cuda")                                # N(0,1) data: 4.5 sigma full scale
+    vs = torch.full((Hkv,), 4.5 / 448, device="cuda")
+    ck8 = torch.zeros(B, Hkv, Lmax, D, dtype=torch.uint8, device="cuda")
+    cv8 = torch.zeros_like(ck8)
+    zero = torch.zeros(B, dtype=torch.int32, device="cuda")
+    l4l.l4l_kv_append_fp8(ck8, cv8, ck.permute(0, 2, 1, 3), cv.permute(0, 2, 1, 3), zero, ks, vs)
+    q, lens = db.q.cuda(), db.kv_len.cuda()
+    o8, o16 = torch.zeros_like(q), torch.zeros_like(q)
+    ws = l4l.new_workspace(l4l.L4L_OP_DECODE, B, Hq, Hkv, D, Lmax)
+    l4l.l4l_attn_decode_fp8(q, o8, ck8, cv8, ks, vs, lens, Lmax, w.scale, ws)
+    l4l.l4l_attn_decode(q, o16, ck, cv, lens, Lmax, w.scale, ws)
+    torch.cuda.synchronize()
+    assert l4l.l4l_last_device_error(ws) == 0
+    ref, _ = orc.decode_fp8(db.q, ck8.cpu(), cv8.cpu(), db.kv_len.numpy(), ks.cpu().numpy(), vs.cpu().numpy(), w.scale)
+    assert_close_to_oracle(o8.cpu(), ref, "fp8 decode, benchmark batch")
+    assert (o8.float() - o16.float()).abs().max().item() < 0.05                       # quantisation noise only
+
+
+@pytest.mark.parametrize("D", [64, 128])
+def test_fp8_append_is_bit_exact(D):
+    B, T, Hkv, Lmax = 3, 19, 4, 40
+    g = torch.Generator().manual_seed(D)
+    k = (torch.randn(B, T, Hkv, D, generator=g) * 3).to(torch.bfloat16)
+    v = (torch.randn(B, T, Hkv, D, generator=g) * torch.exp(torch.randn(B, T, Hkv, D, generator=g) * 4)).to(torch.bfloat16)
+    v[0, 0, 0, :4] = torch.tensor([float("inf"), -float("inf"), 1e30, -448.0]).to(torch.bfloat16)
+    ck8 = torch.full((B, Hkv, Lmax, D), 0x55, dtype=torch.uint8)
+    cv8 = ck8.clone()
+    ks, vs = torch.rand(Hkv, generator=g) + 0.1, torch.rand(Hkv, generator=g) * 3 + 0.1
+    pos, n_new = [0, 30, 21], [19, 19, 7]                    # sequence 1 runs off the end of the cache
+    ref_k, ref_v = orc.kv_append_fp8(ck8, cv8, k, v, pos, n_new, ks.numpy(), vs.numpy())
+    gk, gv = Guarded(ck8), Guarded(cv8)
+    l4l.l4l_kv_append_fp8(gk.t, gv.t, k.cuda(), v.cuda(), torch.tensor(pos, dtype=torch.int32).cuda(), ks.cuda(),
+                          vs.cuda(), n_new=torch.tensor(n_new, dtype=torch.int32).cuda())
+    torch.cuda.synchronize()
+    assert gk.margins_intact() and gv.margins_intact()
+    assert np.array_equal(gk.t.cpu().numpy(), ref_k) and np.array_equal(gv.t.cpu().numpy(), ref_v)
+
+
+def test_fp8_decode_rejects_head_dim_64():
+    q = torch.zeros(1, 4, 64, dtype=torch.bfloat16, device="cuda")
+    c8 = torch.zeros(1, 2, 32, 64, dtype=torch.uint8, device="cuda")
+    sc = torch.ones(2, device="cuda")
+    ws = l4l.new_workspace(l4l.L4L_OP_DECODE, 1, 4, 2, 64, 32)
+    with pytest.raises(l4l.L4LError):
+        l4l.l4l_attn_decode_fp8(q, q.clone(), c8, c8.clone(), sc, sc, torch.ones(1, dtype=torch.int32, device="cuda"),
+                                32, 0.1, ws)

@@ -508,3 +508,63 @@ def test_paged_decode_is_decode_over_the_pages_laid_end_to_end():
     ck2, cv2 = orc.kv_append(ck, cv, k_new, v_new, pos, np.array([2, 3, 3], np.int32))
     assert np.array_equal(orc.gather_pages(pk2, perm, Lmax), ck2)
     assert np.array_equal(orc.gather_pages(pv2, perm, Lmax), cv2)
+
+
+# --------------------------------------------------------------------------- fp8 (e4m3) cache
+def test_e4m3_code_table_and_rounding_match_the_library_type():
+    codes = torch.arange(256, dtype=torch.uint8)
+    want = codes.view(torch.float8_e4m3fn).float().double().numpy()
+    got = orc.e4m3_decode(codes)
+    nan = np.isnan(want)
+    assert np.array_equal(np.isnan(got), nan) and np.array_equal(got[~nan], want[~nan])
+    assert got[0x7E] == 448.0 and got[0x08] == 2.0 ** -6 and got[0x01] == 2.0 ** -9
+    g = torch.Generator().manual_seed(8)
+    x = torch.randn(50000, generator=g) * torch.exp(torch.randn(50000, generator=g) * 3)
+    x = x[x.abs() <= 448.0]
+    ties = torch.tensor([1.0625, 1.1875, -3.25, 0.0009765625, 2.0 ** -10, 3 * 2.0 ** -10, 0.0, -0.0, 447.9, 448.0])
+    x = torch.cat([x, ties])
+    want_c = x.to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    assert np.array_equal(orc.e4m3_encode(x.numpy()), want_c)
+    # saturation instead of overflow
+    assert list(orc.e4m3_encode(np.array([449.0, 1e9, -1e9], np.float32))) == [0x7E, 0x7E, 0xFE]
+
+
+def test_fp8_decode_equals_bf16_decode_on_values_both_formats_hold_exactly():
+    """Every e4m3 value is a bf16 value, and so is its product with a power-of-two scale: decode over the codes
+    must equal, bit for bit, decode over a bf16 cache holding the values the codes stand for."""
+    B, Hq, Hkv, D, Lmax = 2, 4, 2, 8, 20
+    g = torch.Generator().manual_seed(70)
+    ck8 = torch.randint(0, 256, (B, Hkv, Lmax, D), generator=g, dtype=torch.uint8)
+    cv8 = torch.randint(0, 256, (B, Hkv, Lmax, D), generator=g, dtype=torch.uint8)
+    ck8[(ck8 & 0x7F) == 0x7F] = 0x10                      # no NaN codes
+    cv8[(cv8 & 0x7F) == 0x7F] = 0x10
+    ck8[(ck8 & 0x78) == 0x78] &= 0xB7                     # keep |k| <= 30 so that the scores stay moderate
+    ks, vs = np.array([0.5, 2.0], np.float32), np.array([4.0, 0.25], np.float32)
+    kv = torch.from_numpy(orc.e4m3_decode(ck8) * ks[None, :, None, None]).to(torch.bfloat16)
+    vv = torch.from_numpy(orc.e4m3_decode(cv8) * vs[None, :, None, None]).to(torch.bfloat16)
+    assert np.array_equal(f64(kv), orc.e4m3_decode(ck8) * ks[None, :, None, None])          # exact in bf16
+    q = randn((B, Hq, D), 71, 0.25)
+    lens = np.array([Lmax, 7], np.int32)
+    want, want_lse = orc.decode(q, kv, vv, lens, 0.3)
+    got, got_lse = orc.decode_fp8(q, ck8, cv8, lens, ks, vs, 0.3)
+    np.testing.assert_allclose(got, want, rtol=0, atol=1e-13)
+    np.testing.assert_allclose(got_lse, want_lse, rtol=0, atol=1e-13)
+
+
+def test_fp8_append_quantises_by_division_and_touches_only_its_slots():
+    B, T, Hkv, D, Lmax = 2, 3, 2, 8, 10
+    k, v = randn((B, T, Hkv, D), 72, 3.0), randn((B, T, Hkv, D), 73, 100.0)
+    ck8 = torch.full((B, Hkv, Lmax, D), 0x55, dtype=torch.uint8)
+    cv8 = ck8.clone()
+    ks, vs = np.array([0.37, 1.0], np.float32), np.array([0.9, 3.0], np.float32)
+    gk, gv = orc.kv_append_fp8(ck8, cv8, k, v, [4, 8], [3, 3], ks, vs)      # sequence 1: third token falls off
+    for b, slots in ((0, [4, 5, 6]), (1, [8, 9])):
+        for t, s_ in enumerate(slots):
+            for g_ in range(Hkv):
+                wk = (k[b, t, g_].float() / float(ks[g_])).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+                assert np.array_equal(gk[b, g_, s_], wk)
+                y = v[b, t, g_].float() / float(vs[g_])
+                wv = y.clamp(-448, 448).to(torch.float8_e4m3fn).view(torch.uint8).numpy()    # the oracle saturates
+                assert np.array_equal(gv[b, g_, s_], wv)
+        others = [s_ for s_ in range(Lmax) if s_ not in slots]
+        assert (gk[b][:, others] == 0x55).all() and (gv[b][:, others] == 0x55).all()
