@@ -342,7 +342,26 @@ def run_ours(args, rank, world):
         l4l.l4l_attn_decode_paged(dq, do, pk_i, pv_i, tbl_i, dlen, Lmax, wd.scale, ws_d)
 
     t_paged = timed(paged_step, 21)
-    del pools, filler
+    del pools
+    # decode over an fp8 (e4m3) cache: the same batch quantised by the library's own append (N(0,1) data, 4.5 sigma
+    # at full scale), three copies in rotation
+    k_sc = torch.full((Hkv,), 4.5 / 448, dtype=torch.float32, device=dev)
+    c8 = []
+    for i in range(3):
+        k8 = torch.zeros(Bd, Hkv, Lmax, D, dtype=torch.uint8, device=dev)
+        v8 = torch.zeros_like(k8)
+        l4l.l4l_kv_append_fp8(k8, v8, torch.nan_to_num(dck.float()).to(torch.bfloat16).permute(0, 2, 1, 3),
+                              torch.nan_to_num(dcv.float()).to(torch.bfloat16).permute(0, 2, 1, 3),
+                              torch.zeros(Bd, dtype=torch.int32, device=dev), k_sc, k_sc)
+        c8.append((k8, v8))
+
+    def fp8_step():
+        k8, v8 = c8[rot[0] % 3]
+        rot[0] += 1
+        l4l.l4l_attn_decode_fp8(dq, do, k8, v8, k_sc, k_sc, dlen, Lmax, wd.scale, ws_d)
+
+    t_fp8 = timed(fp8_step, 21)
+    del c8, filler
     dev_err = l4l.l4l_last_device_error(ws_p) | l4l.l4l_last_device_error(ws_d)
 
     # ---- end to end through the same entry points with HOST buffers (pinned), copies inside the timed region
@@ -375,8 +394,8 @@ def run_ours(args, rank, world):
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
 
     # ---- max over ranks
-    total_ms, e2e_ms, t_pre, t_dec, t_app, t_dec_b2b, t_rope, t_chunk, t_fused, t_paged = max_over_ranks(
-        [total_ms, e2e_ms, t_pre, t_dec, t_app, t_dec_b2b, t_rope, t_chunk, t_fused, t_paged], world, dev)
+    total_ms, e2e_ms, t_pre, t_dec, t_app, t_dec_b2b, t_rope, t_chunk, t_fused, t_paged, t_fp8 = max_over_ranks(
+        [total_ms, e2e_ms, t_pre, t_dec, t_app, t_dec_b2b, t_rope, t_chunk, t_fused, t_paged, t_fp8], world, dev)
     if rank != 0:
         return
 
@@ -421,6 +440,8 @@ def run_ours(args, rank, world):
             "prefill_from_cache": {"ms": t_chunk, "tflops": pre_flops / (t_chunk * 1e-3) / 1e12},
             "decode_with_fused_append": {"us": t_fused * 1e3, "kv_gbs": dec_bytes / (t_fused * 1e-3) / 1e9},
             "decode_paged_64": {"us": t_paged * 1e3, "kv_gbs": dec_bytes / (t_paged * 1e-3) / 1e9},
+            "decode_fp8_cache": {"us": t_fp8 * 1e3, "kv_gbs_fp8_bytes": dec_bytes / 2 / (t_fp8 * 1e-3) / 1e9,
+                                 "speedup_over_bf16_cache": t_dec_b2b / t_fp8},
         },
         "gpu_launches": 3 * args.steps,
         "clocks": clocks,

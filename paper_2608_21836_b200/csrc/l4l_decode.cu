@@ -43,7 +43,8 @@ constexpr int kMaxB = 512;                 // sequences per launch (prefix sums 
 template <int D, int W, bool F8>
 struct DecodeCfg {
     static_assert(!F8 || D == 128, "the fp8 path wants one 128-byte row per token");
-    static constexpr int kTileT = 16 * W;                         // tokens per TMA tile
+    static constexpr int kSub = F8 ? 2 : 1;                       // 16-token blocks a consumer warp takes per tile
+    static constexpr int kTileT = 16 * W * kSub;                  // tokens per TMA tile
     static constexpr int kRowBytes = F8 ? D : 2 * D;              // one token of one KV head
     static constexpr int kHalves = kRowBytes / 128;               // 128-byte column blocks of a tile
     static constexpr int kBoxD = F8 ? 128 : 64;                   // elements per 128-byte box row
@@ -644,7 +645,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
 
             const uint32_t k_tile = smem_u32(stages + (size_t)s * C::kStageBytes);
             const uint32_t v_tile = k_tile + C::kTileBytes;
-            const int row0 = warp * 16;
+            const int row0 = warp * 16 * C::kSub;
             const int nvalid = mt.kv_len - (mt.t0 + row0);       // valid tokens in this warp's slice
             bool wrote_smem = false;
             if (!F8 && p.k_new != nullptr && nvalid > 0 && nvalid <= 16) {
@@ -669,15 +670,53 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 wrote_smem = true;
                 __syncwarp();
             }
-            if (nvalid > 0) {
+            if constexpr (F8) {
+                if (nvalid > 0) {
+                    // 32 tokens per step: two 16-token blocks share one softmax update. A block with no valid
+                    // token is skipped (its rows may never have been fetched); in the last valid block the
+                    // tokens past the end get no weight and their V rows are cleared.
+                    constexpr int kSub = C::kSub;
+                    float sv[2 * kSub][4];
+                    const float sc = p.scale_log2e * __ldg(p.k_scale + mt.kvh);
+#pragma unroll
+                    for (int u = 0; u < kSub; ++u) {
+                        if (u == 0 || nvalid > 16 * u) {
+                            warp_qk_16x16_f8<D>(qf, k_tile, row0 + 16 * u, sv[2 * u], sv[2 * u + 1]);
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                sv[2 * u][e] *= sc;
+                                sv[2 * u + 1][e] *= sc;
+                            }
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) sv[2 * u][e] = sv[2 * u + 1][e] = -INFINITY;
+                        }
+                    }
+                    if (nvalid < 16 * kSub) {
+                        const int tok = 2 * (lane & 3);
+#pragma unroll
+                        for (int j = 0; j < 2 * kSub; ++j)
+#pragma unroll
+                            for (int e = 0; e < 4; ++e)
+                                if (8 * j + tok + (e & 1) >= nvalid) sv[j][e] = -INFINITY;
+                        uint8_t *vt = stages + (size_t)s * C::kStageBytes + C::kTileBytes;
+                        const int fetched_end = (nvalid + 15) & ~15;                 // end of the last valid block
+                        for (int i = lane; i < (fetched_end - nvalid) * 8; i += 32)
+                            *reinterpret_cast<uint4 *>(vt + (row0 + nvalid + i / 8) * 128 + ((i & 7) << 4)) =
+                                make_uint4(0u, 0u, 0u, 0u);
+                        wrote_smem = true;
+                        __syncwarp();
+                    }
+                    uint32_t pa[kSub][4];
+                    warp_softmax_tiles<D, true, 2 * kSub>(st, sv, pa);
+#pragma unroll
+                    for (int u = 0; u < kSub; ++u)
+                        if (u == 0 || nvalid > 16 * u) warp_pv_16x16_f8<D>(st, pa[u], v_tile, row0 + 16 * u);
+                }
+            } else if (nvalid > 0) {
                 float s_lo[4], s_hi[4];
                 float sc = p.scale_log2e;
-                if constexpr (F8) {
-                    warp_qk_16x16_f8<D>(qf, k_tile, row0, s_lo, s_hi);
-                    sc *= __ldg(p.k_scale + mt.kvh);
-                } else {
-                    warp_qk_16x16<D>(qf, k_tile, C::kHalfBytes, row0, s_lo, s_hi);
-                }
+                warp_qk_16x16<D>(qf, k_tile, C::kHalfBytes, row0, s_lo, s_hi);
                 const int tok = 2 * (lane & 3);
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
@@ -704,11 +743,8 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     __syncwarp();
                 }
                 uint32_t pa[4];
-                warp_softmax_16<D, F8>(st, s_lo, s_hi, pa);
-                if constexpr (F8)
-                    warp_pv_16x16_f8<D>(st, pa, v_tile, row0);
-                else
-                    warp_pv_16x16<D>(st, pa, v_tile, C::kHalfBytes, row0);
+                warp_softmax_16<D>(st, s_lo, s_hi, pa);
+                warp_pv_16x16<D>(st, pa, v_tile, C::kHalfBytes, row0);
             }
 
             if (wrote_smem) fence_proxy_async_smem();   // generic writes before the next TMA fill
@@ -808,7 +844,7 @@ struct ShapeOps {
 template <int D, int W, bool F8>
 ShapeOps shape_ops()
 {
-    return ShapeOps{W, 16 * W, &decode_smem_bytes<D, W, F8>, &decode_blocks_per_sm<D, W, F8>};
+    return ShapeOps{W, DecodeCfg<D, W, F8>::kTileT, &decode_smem_bytes<D, W, F8>, &decode_blocks_per_sm<D, W, F8>};
 }
 
 ShapeOps pick_shape(int D, int warps, bool fp8)

@@ -78,10 +78,14 @@ __device__ __forceinline__ void warp_softmax_16(WarpAttnState<D> &st, const floa
                                       __uint_as_float(p23 << 16) + __uint_as_float(p23 & 0xffff0000u);
         st.l[h] = st.l[h] * corr + psum;
         st.m[h] = m_new;
+        // O is rescaled only if some row of this half saw its maximum grow (after the first tiles of a long
+        // sequence that is rare): corr == 1 exactly otherwise
+        if (__any_sync(0xffffffffu, corr != 1.f)) {
 #pragma unroll
-        for (int nt = 0; nt < D / 8; ++nt) {
-            st.o[nt][2 * h] *= corr;
-            st.o[nt][2 * h + 1] *= corr;
+            for (int nt = 0; nt < D / 8; ++nt) {
+                st.o[nt][2 * h] *= corr;
+                st.o[nt][2 * h + 1] *= corr;
+            }
         }
     }
 }
@@ -102,6 +106,44 @@ __device__ __forceinline__ void warp_pv_16x16(WarpAttnState<D> &st, const uint32
         ldmatrix_x4_trans(addr, b0, b1, b2, b3);
         mma_bf16_16816(st.o[2 * np], pa, b0, b1);
         mma_bf16_16816(st.o[2 * np + 1], pa, b2, b3);
+    }
+}
+
+// Online-softmax update over NT 8-token score tiles at once (NT = 2 is warp_softmax_16; the fp8 path takes 32
+// tokens per step so that the shuffles and the bookkeeping are paid once per 32 tokens). s[j] holds tokens
+// 8j + 2*(lane%4) + {0,1} (elements 0,1: row lane/4; 2,3: row lane/4 + 8); pa[u] is the A fragment of P for
+// tokens 16u .. 16u+15.
+template <int D, bool kF16, int NT>
+__device__ __forceinline__ void warp_softmax_tiles(WarpAttnState<D> &st, const float (&s)[NT][4], uint32_t (&pa)[NT / 2][4])
+{
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        float mx = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < NT; ++j) mx = fmaxf(mx, fmaxf(s[j][2 * h], s[j][2 * h + 1]));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        const float m_new = fmaxf(st.m[h], mx);
+        const float m_use = (m_new == -INFINITY) ? 0.f : m_new;     // row with nothing visible yet
+        const float corr = fast_exp2(st.m[h] - m_use);
+        float psum = 0.f;
+#pragma unroll
+        for (int j = 0; j < NT; ++j) {
+            const float e0 = fast_exp2(s[j][2 * h] - m_use), e1 = fast_exp2(s[j][2 * h + 1] - m_use);
+            const uint32_t pk = kF16 ? pack_f16x2(e0, e1) : pack_bf16x2(e0, e1);
+            pa[j >> 1][(j & 1) * 2 + h] = pk;
+            // the denominator sums exactly the rounded weights that multiply V
+            psum += kF16 ? sum_f16x2(pk) : __uint_as_float(pk << 16) + __uint_as_float(pk & 0xffff0000u);
+        }
+        st.l[h] = st.l[h] * corr + psum;
+        st.m[h] = m_new;
+        if (__any_sync(0xffffffffu, corr != 1.f)) {
+#pragma unroll
+            for (int nt = 0; nt < D / 8; ++nt) {
+                st.o[nt][2 * h] *= corr;
+                st.o[nt][2 * h + 1] *= corr;
+            }
+        }
     }
 }
 
