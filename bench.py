@@ -35,8 +35,8 @@ FALLBACK_TFLOPS, FALLBACK_GBS = 1590.0, 6650.0
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
 # profiles/: prefill captured at B=1,S=8192 (155.8 MB) and scaled x4 to the bench's B=4 (traffic is proportional
 # to B); decode captured on the bench's own batch.
-NCU_TRAFFIC_PREFILL = 623.1e6   # 4 x (101.0 MB read + 54.8 MB written)
-NCU_TRAFFIC_DECODE = 299.9e6    # 296.0 MB read + 3.9 MB written
+NCU_TRAFFIC_PREFILL = 628.1e6   # 4 x (101.0 MB read + 56.1 MB written)
+NCU_TRAFFIC_DECODE = 300.1e6    # 295.9 MB read + 4.2 MB written
 
 
 def measured_peaks():
