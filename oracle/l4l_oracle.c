@@ -357,6 +357,51 @@ int l4l_oracle_decode(const uint16_t *q, const uint16_t *cache_k, const uint16_t
 }
 
 /* ------------------------------------------------------------------------------------------------
+ * Second workload: the gated linear recurrence of the RecurrentGemma block (RG-LRU), which the paper's
+ * appendix lists as an accepted kernel that fuses "sigmoid, softplus-derived recurrent gating, reset
+ * handling, normalization, and the recurrent scan" with the state carried through the sequence and
+ * the final state written once. The paper prints no formula; this is the published recurrence of that
+ * block, per sequence b, channel c, step t (all in fp64 here):
+ *     i_t = sigmoid(gate_x[b,t,c])                      input gate
+ *     r_t = sigmoid(gate_a[b,t,c])                      recurrence gate
+ *     log a_t = -8 * r_t * softplus(a_param[c])
+ *     a_t = exp(log a_t),   m_t = sqrt(1 - a_t^2)       (m_t keeps the state's variance bounded)
+ *     at a reset step (position[b,t] == 0):  a_t = 0, m_t = 1
+ *     h_t = a_t * h_{t-1} + m_t * i_t * x[b,t,c]
+ *     y[b,t,c] = h_t
+ * x, gate_x, gate_a: bf16 bits [B, T, W]; a_param: fp32 [W]; position: int32 [B, T] or NULL (no resets);
+ * state: fp64 [B, W] in/out (h before the first step / after step seq_len[b]-1); seq_len [B] or NULL (= T).
+ * y: fp64 [B, T, W]; rows t >= seq_len[b] untouched.
+ */
+int l4l_oracle_rglru(const uint16_t *x, const uint16_t *gate_x, const uint16_t *gate_a, const float *a_param,
+                     const int32_t *position, const int32_t *seq_len, double *state, double *y, int B, int T, int W)
+{
+    for (int b = 0; b < B; ++b) {
+        const int L = seq_len ? seq_len[b] : T;
+        if (L < 0 || L > T) return -1;
+        for (int c = 0; c < W; ++c) {
+            const double sp = log1p(exp((double)a_param[c]));        /* softplus */
+            double h = state[(int64_t)b * W + c];
+            for (int t = 0; t < L; ++t) {
+                const int64_t idx = ((int64_t)b * T + t) * W + c;
+                const double in_gate = 1.0 / (1.0 + exp(-bf16_to_f64(gate_x[idx])));
+                const double rec_gate = 1.0 / (1.0 + exp(-bf16_to_f64(gate_a[idx])));
+                double a = exp(-8.0 * rec_gate * sp);
+                double m = sqrt(1.0 - a * a);
+                if (position && position[(int64_t)b * T + t] == 0) {
+                    a = 0.0;
+                    m = 1.0;
+                }
+                h = a * h + m * in_gate * bf16_to_f64(x[idx]);
+                y[idx] = h;
+            }
+            state[(int64_t)b * W + c] = h;
+        }
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------------------------------------
  * fp8 (e4m3) cache. The format: 1 sign bit, 4 exponent bits (bias 7), 3 mantissa bits; exponent 0 is
  * subnormal (m/8 * 2^-6); there are no infinities; exponent 15 with mantissa 7 is NaN; the largest
  * finite value is 1.75 * 2^8 = 448.

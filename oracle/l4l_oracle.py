@@ -59,6 +59,7 @@ def _load():
         lib.l4l_oracle_e4m3_encode.restype = None
         lib.l4l_oracle_kv_append_fp8.argtypes = [u8p, u8p, u16p, u16p, i32p, i32p, f32p, f32p, i, i, i, i, i]
         lib.l4l_oracle_decode_fp8.argtypes = [u16p, u8p, u8p, i32p, f32p, f32p, i, i, i, i, i, d, f64p, f64p]
+        lib.l4l_oracle_rglru.argtypes = [u16p, u16p, u16p, f32p, i32p, i32p, f64p, f64p, i, i, i]
         lib.l4l_oracle_kv_append.argtypes = [u16p, u16p, u16p, u16p, i32p, i32p, i, i, i, i, i]
         _lib = lib
     return _lib
@@ -332,3 +333,25 @@ def decode_fp8(q, cache_k8, cache_v8, kv_len, k_scale, v_scale, scale: float):
     if rc != 0:
         raise ValueError("l4l_oracle_decode_fp8 rejected its arguments")
     return out, lse
+
+
+def rglru(x, gate_x, gate_a, a_param, state=None, position=None, seq_len=None):
+    """Gated linear recurrence (RG-LRU). x, gate_x, gate_a bf16 [B,T,W]; a_param float32 [W]; state fp64 [B,W] or
+    None (zeros); position int32 [B,T] or None; seq_len [B] or None. Returns (y fp64 [B,T,W] with NaN in rows past
+    seq_len, final state fp64 [B,W])."""
+    xb, gx, ga = bits(x), bits(gate_x), bits(gate_a)
+    B, T, W = xb.shape
+    assert gx.shape == xb.shape and ga.shape == xb.shape
+    ap = np.ascontiguousarray(np.asarray(a_param, dtype=np.float32))
+    assert ap.shape == (W,)
+    st = np.zeros((B, W)) if state is None else np.ascontiguousarray(np.asarray(state, dtype=np.float64)).copy()
+    pos = None if position is None else _i32(position)
+    sl = None if seq_len is None else _i32(seq_len)
+    y = np.full((B, T, W), np.nan)
+    rc = _load().l4l_oracle_rglru(_p(xb, ctypes.c_uint16), _p(gx, ctypes.c_uint16), _p(ga, ctypes.c_uint16),
+                                  _p(ap, ctypes.c_float), None if pos is None else _p(pos, ctypes.c_int32),
+                                  None if sl is None else _p(sl, ctypes.c_int32), _p(st, ctypes.c_double),
+                                  _p(y, ctypes.c_double), B, T, W)
+    if rc != 0:
+        raise ValueError("l4l_oracle_rglru rejected its arguments")
+    return y, st

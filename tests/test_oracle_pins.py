@@ -568,3 +568,88 @@ def test_fp8_append_quantises_by_division_and_touches_only_its_slots():
                 assert np.array_equal(gv[b, g_, s_], wv)
         others = [s_ for s_ in range(Lmax) if s_ not in slots]
         assert (gk[b][:, others] == 0x55).all() and (gv[b][:, others] == 0x55).all()
+
+
+# --------------------------------------------------------------------------- gated linear recurrence (RG-LRU)
+def _sig(z):
+    return 1.0 / (1.0 + np.exp(-z))
+
+
+def test_rglru_constant_gates_give_the_geometric_series():
+    """With constant gate inputs a and b are constant: h_t = b (1 - a^t) / (1 - a) + a^t h_0."""
+    B, T, W = 1, 50, 3
+    gx_v, ga_v, x_v = 0.5, -1.0, 0.75                     # all exact in bf16
+    ap = np.array([-2.0, 0.0, 1.5], np.float32)
+    ones = torch.ones(B, T, W)
+    y, st = orc.rglru(bf16(ones * x_v), bf16(ones * gx_v), bf16(ones * ga_v), ap, state=np.full((B, W), 0.3))
+    a = np.exp(-8.0 * _sig(ga_v) * np.log1p(np.exp(ap.astype(np.float64))))
+    b = np.sqrt(1 - a * a) * _sig(gx_v) * x_v
+    t = np.arange(1, T + 1)[:, None]
+    want = b * (1 - a ** t) / (1 - a) + a ** t * 0.3
+    np.testing.assert_allclose(y[0], want, rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose(st[0], want[-1], rtol=1e-12)
+
+
+def test_rglru_equals_the_unrolled_sum_and_brute_force():
+    """h_t = sum_s (prod_{u=s+1..t} a_u) b_s + (prod_{u<=t} a_u) h_0, evaluated with cumulative products (a different
+    route from the step-by-step recurrence), and a pure-Python loop on the first channel."""
+    B, T, W = 2, 24, 5
+    x, gx, ga = randn((B, T, W), 80), randn((B, T, W), 81), randn((B, T, W), 82)
+    ap = np.linspace(-3, -1, W).astype(np.float32)        # a stays well away from 0: the division below is safe
+    h0 = np.random.default_rng(0).normal(size=(B, W))
+    y, st = orc.rglru(x, gx, ga, ap, state=h0)
+    sp = np.log1p(np.exp(ap.astype(np.float64)))
+    a = np.exp(-8.0 * _sig(f64(ga)) * sp)
+    bterm = np.sqrt(1 - a * a) * _sig(f64(gx)) * f64(x)
+    P = np.cumprod(a, axis=1)
+    want = P * (h0[:, None, :] + np.cumsum(bterm / P, axis=1))
+    np.testing.assert_allclose(y, want, rtol=1e-9, atol=1e-12)
+    np.testing.assert_allclose(st, want[:, -1], rtol=1e-9, atol=1e-12)
+    h = h0[1, 0]
+    for t in range(T):
+        r = 1 / (1 + math.exp(-float(ga[1, t, 0])))
+        i = 1 / (1 + math.exp(-float(gx[1, t, 0])))
+        at = math.exp(-8 * r * math.log1p(math.exp(float(ap[0]))))
+        h = at * h + math.sqrt(1 - at * at) * i * float(x[1, t, 0])
+        assert abs(h - y[1, t, 0]) < 1e-13
+
+
+def test_rglru_reset_ragged_and_chunking():
+    B, T, W = 2, 30, 4
+    x, gx, ga = randn((B, T, W), 83), randn((B, T, W), 84), randn((B, T, W), 85)
+    ap = np.array([-1.0, 0.0, 0.5, 2.0], np.float32)
+    pos = np.tile(np.arange(T, dtype=np.int32), (B, 1))
+    pos[1, 12:] = np.arange(T - 12)                       # a second segment starts at t = 12 of sequence 1
+    h0 = np.ones((B, W))
+    y, st = orc.rglru(x, gx, ga, ap, state=h0, position=pos, seq_len=[T, 20])
+    # a reset step forgets everything before it and passes the gated input through un-normalised
+    np.testing.assert_allclose(y[:, 0], _sig(f64(gx))[:, 0] * f64(x)[:, 0], rtol=1e-14)
+    np.testing.assert_allclose(y[1, 12], _sig(f64(gx))[1, 12] * f64(x)[1, 12], rtol=1e-14)
+    y2, _ = orc.rglru(x[1:, 12:20].contiguous(), gx[1:, 12:20].contiguous(), ga[1:, 12:20].contiguous(), ap,
+                      state=np.full((1, W), 123.0), position=pos[1:, 12:20])
+    np.testing.assert_allclose(y[1, 12:20], y2[0], rtol=0, atol=0)
+    assert np.isnan(y[1, 20:]).all()
+    # the state after seq_len steps; processing in two chunks with the state carried over changes nothing
+    np.testing.assert_allclose(st[1], y[1, 19], rtol=0, atol=0)
+    ya, sa = orc.rglru(x[:, :11].contiguous(), gx[:, :11].contiguous(), ga[:, :11].contiguous(), ap, state=h0,
+                       position=pos[:, :11])
+    yb, sb = orc.rglru(x[:, 11:].contiguous(), gx[:, 11:].contiguous(), ga[:, 11:].contiguous(), ap, state=sa,
+                       position=pos[:, 11:], seq_len=[T - 11, 9])
+    np.testing.assert_allclose(np.concatenate([ya, yb], 1)[0], y[0], rtol=0, atol=0)
+    np.testing.assert_allclose(sb, st, rtol=0, atol=0)
+    # without positions there is no reset: step 0 uses the incoming state
+    y3, _ = orc.rglru(x, gx, ga, ap, state=h0)
+    assert not np.allclose(y3[:, 0], y[:, 0])
+
+
+def test_rglru_keeps_unit_variance_for_white_inputs():
+    """The sqrt(1 - a^2) factor is there so that white unit-variance inputs (gate fully open) give a state of unit
+    variance whatever a is: a statistical pin of that factor."""
+    B, T, W = 1, 20000, 3
+    g = torch.Generator().manual_seed(86)
+    x = torch.randn(B, T, W, generator=g).to(torch.bfloat16)
+    gx = torch.full((B, T, W), 30.0).to(torch.bfloat16)    # sigmoid = 1 to 1e-13
+    ga = torch.zeros(B, T, W).to(torch.bfloat16)           # r = 1/2
+    y, _ = orc.rglru(x, gx, ga, np.array([-3.0, -1.0, 0.5], np.float32))
+    var = (y[0, 2000:] ** 2).mean(axis=0)
+    np.testing.assert_allclose(var, 1.0, rtol=0.12)
