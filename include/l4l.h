@@ -160,6 +160,29 @@ l4l_status l4l_attn_decode_fp8(const void *q, void *o, l4l_kv_cache cache8, cons
                                void *workspace, size_t ws_bytes, l4l_stream stream);
 
 /*
+ * Second workload: the gated linear recurrence of the RecurrentGemma block (RG-LRU). The paper's
+ * appendix ("RecurrentGemma RGLRU", Table A.4) describes the accepted kernel as fusing sigmoid,
+ * softplus-derived recurrent gating, reset handling, normalisation and the recurrent scan, with the
+ * state carried through the sequence inside the kernel and the final state written once; it prints
+ * no formula, so the recurrence is the published one of that block. For sequence b, channel c,
+ * step t < seq_lens[b]:
+ *     i = sigmoid(gate_x[b,t,c]),  r = sigmoid(gate_a[b,t,c]),  a = exp(-8 r softplus(a_param[c])),
+ *     m = sqrt(1 - a^2);   if position[b,t] == 0:  a = 0, m = 1        (first token of a segment)
+ *     h <- a h + m i x[b,t,c];   y[b,t,c] = h
+ * with h starting from state[b,c] and state[b,c] receiving the last h (after seq_lens[b] steps).
+ * fp32 arithmetic, y rounded to bf16. Rows t >= seq_lens[b] of y are left untouched.
+ *   x, gate_x, gate_a, y   device bf16, dense [B, T, W] (W a multiple of 8; x / gate_x / gate_a 16-byte aligned)
+ *   d_a_param    device float [W]
+ *   d_position   device int32 [B, T], or NULL: no resets (a chunk that continues its sequence)
+ *   d_seq_lens   device int32 [B], or NULL meaning T for all
+ *   d_state      device float [B, W], read and written
+ *   workspace    >= 256 bytes, initialised once (status block only)
+ */
+l4l_status l4l_rglru_scan(const void *x, const void *gate_x, const void *gate_a, const float *d_a_param,
+                          const int32_t *d_position, const int32_t *d_seq_lens, float *d_state, void *y,
+                          int B, int T, int W, void *workspace, size_t ws_bytes, l4l_stream stream);
+
+/*
  * Rotary position embedding (and optional per-head RMS normalisation of q and k) fused with the
  * cache update: the projection outputs of the new tokens go through ONE streaming pass that
  * leaves q ready for the attention calls and K, V in the cache. (The paper's prefill kernel is

@@ -23,7 +23,7 @@ EXPORTS = (
     "l4l_version", "l4l_status_string", "l4l_workspace_bytes", "l4l_workspace_init",
     "l4l_last_device_error", "l4l_kv_append", "l4l_attn_prefill", "l4l_attn_decode",
     "l4l_attn_decode_static", "l4l_attn_decode_append", "l4l_attn_prefill_chunk", "l4l_rope_kv_append",
-    "l4l_kv_append_paged", "l4l_attn_decode_paged", "l4l_kv_append_fp8", "l4l_attn_decode_fp8",
+    "l4l_kv_append_paged", "l4l_attn_decode_paged", "l4l_kv_append_fp8", "l4l_attn_decode_fp8", "l4l_rglru_scan",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -93,6 +93,8 @@ def load() -> ctypes.CDLL:
     lib.l4l_attn_decode_fp8.restype = c_int
     lib.l4l_attn_decode_fp8.argtypes = [vp, vp, KVCache, vp, vp, i32p, c_int, c_int, c_int, c_int, c_int,
                                         ctypes.c_float, vp, vp, c_size, vp]
+    lib.l4l_rglru_scan.restype = c_int
+    lib.l4l_rglru_scan.argtypes = [vp, vp, vp, vp, i32p, i32p, vp, vp, c_int, c_int, c_int, vp, c_size, vp]
     lib.l4l_rope_kv_append.restype = c_int
     lib.l4l_rope_kv_append.argtypes = [Tensor4, Tensor4, Tensor4, KVCache, i32p, i32p, c_int, c_int, c_int, c_int, c_int,
                                        vp, vp, c_int, vp, vp, ctypes.c_float, vp]
@@ -397,3 +399,24 @@ def l4l_attn_decode_fp8(q, o, cache_k8, cache_v8, k_scale, v_scale, kv_lens, max
                                     workspace.numel() * workspace.element_size(), _stream())
     if st != L4L_OK:
         raise L4LError(st, "l4l_attn_decode_fp8")
+
+
+def l4l_rglru_scan(x, gate_x, gate_a, a_param, state, y, workspace, position=None, seq_lens=None) -> None:
+    """Gated linear recurrence (RG-LRU) over the sequence. x, gate_x, gate_a, y dense CUDA bf16 [B,T,W];
+    a_param CUDA float32 [W]; state CUDA float32 [B,W] (in/out); position CUDA int32 [B,T] or None;
+    seq_lens CUDA int32 [B] or None."""
+    for t, name in ((x, "x"), (gate_x, "gate_x"), (gate_a, "gate_a"), (y, "y")):
+        _check_bf16_cuda(t, name)
+        if not (t.dim() == 3 and t.is_contiguous() and t.shape == x.shape):
+            raise ValueError(f"{name} must be a dense [B, T, W] tensor of the same shape as x")
+    B, T, W = x.shape
+    if position is not None and not (position.is_cuda and position.dtype == torch.int32 and position.is_contiguous()
+                                     and tuple(position.shape) == (B, T)):
+        raise TypeError("position must be a contiguous CUDA int32 tensor [B, T]")
+    st = load().l4l_rglru_scan(x.data_ptr(), gate_x.data_ptr(), gate_a.data_ptr(), _f32_dev(a_param, "a_param", (W,)),
+                               None if position is None else position.data_ptr(),
+                               None if seq_lens is None else _i32_dev(seq_lens, "seq_lens"),
+                               _f32_dev(state, "state", (B, W)), y.data_ptr(), B, T, W, workspace.data_ptr(),
+                               workspace.numel() * workspace.element_size(), _stream())
+    if st != L4L_OK:
+        raise L4LError(st, "l4l_rglru_scan")

@@ -94,6 +94,21 @@ bool encode_tmap(CUtensorMap *out, TmapCoord *coord, const void *base, int D, in
 
 }  // namespace
 
+bool make_tmap_rows_bf16(CUtensorMap *out, const void *base, int64_t n_cols, int64_t n_rows, int64_t n_outer,
+                         int64_t stride_row, int64_t stride_outer, int box_cols, int box_rows)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t gdim[3] = {(cuuint64_t)n_cols, (cuuint64_t)(n_rows < 1 ? 1 : n_rows), (cuuint64_t)(n_outer < 1 ? 1 : n_outer)};
+    cuuint64_t gstride[2] = {(cuuint64_t)stride_row * 2, (cuuint64_t)stride_outer * 2};
+    if (gstride[1] < gstride[0] * gdim[1]) gstride[1] = gstride[0] * gdim[1];      // extent-1 outer dimension
+    cuuint32_t box[3] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), gdim, gstride, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool make_tmap(CUtensorMap *out, TmapCoord *coord, const void *base, int D, int64_t n_t, int64_t n_h, int64_t n_b,
                int64_t stride_t, int64_t stride_h, int64_t stride_b, int box_d, int box_t, int elem_bytes)
 {
@@ -309,6 +324,20 @@ l4l_status l4l_attn_decode_fp8(const void *q, void *o, l4l_kv_cache cache8, cons
     const Fp8Scales sc{d_k_scale, d_v_scale};
     return launch_decode(q, o, cache8, d_kv_lens, max_kv_len, B, Hq, Hkv, head_dim, scale, d_lse, workspace, plan,
                          static_cast<cudaStream_t>(stream), nullptr, nullptr, nullptr, &sc);
+}
+
+l4l_status l4l_rglru_scan(const void *x, const void *gate_x, const void *gate_a, const float *d_a_param,
+                          const int32_t *d_position, const int32_t *d_seq_lens, float *d_state, void *y, int B, int T,
+                          int W, void *workspace, size_t ws_bytes, l4l_stream stream)
+{
+    if (B < 0 || T < 0 || W <= 0) return L4L_ERR_INVALID_ARG;
+    if (W % 8 != 0 || B > 65535) return L4L_ERR_UNSUPPORTED;       // 16-byte rows for the tensor maps; grid.y
+    if (!x || !gate_x || !gate_a || !d_a_param || !d_state || !y) return L4L_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(gate_x) || !aligned16(gate_a)) return L4L_ERR_INVALID_ARG;
+    if (!workspace || ws_bytes < kStatusBytes) return L4L_ERR_WORKSPACE;
+    if (B == 0 || T == 0) return L4L_OK;
+    return launch_rglru_scan(x, gate_x, gate_a, d_a_param, d_position, d_seq_lens, d_state, y, B, T, W, workspace,
+                             static_cast<cudaStream_t>(stream));
 }
 
 l4l_status l4l_rope_kv_append(l4l_tensor4 q, l4l_tensor4 k_new, l4l_tensor4 v_new, l4l_kv_cache cache,

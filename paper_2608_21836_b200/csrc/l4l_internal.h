@@ -28,6 +28,11 @@ inline bool make_tmap_bf16(CUtensorMap *out, TmapCoord *coord, const void *base,
     return make_tmap(out, coord, base, D, n_t, n_h, n_b, stride_t, stride_h, stride_b, box_d, box_t, 2);
 }
 
+// Tiled bf16 tensor map without swizzle over a dense [outer, rows, cols] array (cols contiguous): box =
+// box_cols x box_rows x 1. Coordinates are (col, row, outer).
+bool make_tmap_rows_bf16(CUtensorMap *out, const void *base, int64_t n_cols, int64_t n_rows, int64_t n_outer,
+                         int64_t stride_row, int64_t stride_outer, int box_cols, int box_rows);
+
 int sm_count();
 
 struct DecodePlan {
@@ -71,6 +76,10 @@ l4l_status launch_kv_append(const l4l_kv_cache &cache, const l4l_tensor4 &k_new,
 l4l_status launch_kv_append_fp8(const l4l_kv_cache &cache, const l4l_tensor4 &k_new, const l4l_tensor4 &v_new,
                                 const int32_t *d_write_pos, const int32_t *d_n_new, int n_new_max, int B, int Hkv,
                                 int D, const float *d_k_scale, const float *d_v_scale, cudaStream_t stream);
+
+l4l_status launch_rglru_scan(const void *x, const void *gate_x, const void *gate_a, const float *d_a_param,
+                             const int32_t *d_position, const int32_t *d_seq_lens, float *d_state, void *y, int B, int T,
+                             int W, void *workspace, cudaStream_t stream);
 
 l4l_status launch_prefill(const l4l_tensor4 &q, const l4l_tensor4 &k, const l4l_tensor4 &v,
                           const l4l_tensor4 &o, const l4l_kv_cache &cache, const int32_t *d_seq_lens,

@@ -16,6 +16,7 @@ constexpr int kStatusErrWord = 0;       // bitmask of waits that ran out
 constexpr int kStatusInfoWord = 1;      // where it happened (role / barrier id), best effort
 constexpr unsigned kErrDecodeWait = 1u;
 constexpr unsigned kErrPrefillWait = 2u;
+constexpr unsigned kErrScanWait = 4u;
 constexpr size_t kStatusBytes = 256;
 
 // Cycle budget of one bounded wait (~0.25 s at 2 GHz): far above any legitimate latency.
@@ -148,6 +149,16 @@ __device__ __forceinline__ void tma_load_4d(void *smem_dst, const void *tmap, ui
         " [%0], [%1, {%3, %4, %5, %6}], [%2];"
         ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_u32(bar)), "r"(c0), "r"(c1),
         "r"(c2), "r"(c3)
+        : "memory");
+}
+
+// 3-D tiled load global -> shared (same rules as the 4-D form).
+__device__ __forceinline__ void tma_load_3d(void *smem_dst, const void *tmap, uint64_t *bar, int c0, int c1, int c2)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
 }
 
