@@ -23,7 +23,7 @@ EXPORTS = (
     "l4l_version", "l4l_status_string", "l4l_workspace_bytes", "l4l_workspace_init",
     "l4l_last_device_error", "l4l_kv_append", "l4l_attn_prefill", "l4l_attn_decode",
     "l4l_attn_decode_static", "l4l_attn_decode_append", "l4l_attn_prefill_chunk", "l4l_rope_kv_append",
-    "l4l_kv_append_paged", "l4l_attn_decode_paged", "l4l_kv_append_fp8", "l4l_attn_decode_fp8", "l4l_rglru_scan",
+    "l4l_kv_append_paged", "l4l_attn_decode_paged", "l4l_kv_append_fp8", "l4l_attn_decode_fp8", "l4l_rglru_scan", "l4l_rglru_workspace_bytes",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -93,6 +93,8 @@ def load() -> ctypes.CDLL:
     lib.l4l_attn_decode_fp8.restype = c_int
     lib.l4l_attn_decode_fp8.argtypes = [vp, vp, KVCache, vp, vp, i32p, c_int, c_int, c_int, c_int, c_int,
                                         ctypes.c_float, vp, vp, c_size, vp]
+    lib.l4l_rglru_workspace_bytes.restype = c_size
+    lib.l4l_rglru_workspace_bytes.argtypes = [c_int, c_int, c_int]
     lib.l4l_rglru_scan.restype = c_int
     lib.l4l_rglru_scan.argtypes = [vp, vp, vp, vp, i32p, i32p, vp, vp, c_int, c_int, c_int, vp, c_size, vp]
     lib.l4l_rope_kv_append.restype = c_int
@@ -420,3 +422,12 @@ def l4l_rglru_scan(x, gate_x, gate_a, a_param, state, y, workspace, position=Non
                                workspace.numel() * workspace.element_size(), _stream())
     if st != L4L_OK:
         raise L4LError(st, "l4l_rglru_scan")
+
+
+def new_rglru_workspace(B: int, T: int, W: int, device=None) -> torch.Tensor:
+    """Zeroed workspace for l4l_rglru_scan, large enough for the segment-parallel mode at these sizes."""
+    n = int(load().l4l_rglru_workspace_bytes(B, T, W))
+    if n == 0:
+        raise ValueError("unsupported sizes")
+    ws = torch.zeros((n + 7) // 8, dtype=torch.int64, device=device or "cuda")
+    return ws

@@ -337,7 +337,13 @@ l4l_status l4l_rglru_scan(const void *x, const void *gate_x, const void *gate_a,
     if (!workspace || ws_bytes < kStatusBytes) return L4L_ERR_WORKSPACE;
     if (B == 0 || T == 0) return L4L_OK;
     return launch_rglru_scan(x, gate_x, gate_a, d_a_param, d_position, d_seq_lens, d_state, y, B, T, W, workspace,
-                             static_cast<cudaStream_t>(stream));
+                             ws_bytes, static_cast<cudaStream_t>(stream));
+}
+
+size_t l4l_rglru_workspace_bytes(int B, int T, int W)
+{
+    if (B < 0 || T < 0 || W <= 0) return 0;
+    return rglru_workspace_bytes(B, T, W);
 }
 
 l4l_status l4l_rope_kv_append(l4l_tensor4 q, l4l_tensor4 k_new, l4l_tensor4 v_new, l4l_kv_cache cache,

@@ -79,7 +79,8 @@ l4l_status launch_kv_append_fp8(const l4l_kv_cache &cache, const l4l_tensor4 &k_
 
 l4l_status launch_rglru_scan(const void *x, const void *gate_x, const void *gate_a, const float *d_a_param,
                              const int32_t *d_position, const int32_t *d_seq_lens, float *d_state, void *y, int B, int T,
-                             int W, void *workspace, cudaStream_t stream);
+                             int W, void *workspace, size_t ws_bytes, cudaStream_t stream);
+size_t rglru_workspace_bytes(int B, int T, int W);
 
 l4l_status launch_prefill(const l4l_tensor4 &q, const l4l_tensor4 &k, const l4l_tensor4 &v,
                           const l4l_tensor4 &o, const l4l_kv_cache &cache, const int32_t *d_seq_lens,
