@@ -361,8 +361,22 @@ def run_ours(args, rank, world):
         l4l.l4l_attn_decode_fp8(dq, do, k8, v8, k_sc, k_sc, dlen, Lmax, wd.scale, ws_d)
 
     t_fp8 = timed(fp8_step, 21)
-    del c8, filler
-    dev_err = l4l.l4l_last_device_error(ws_p) | l4l.l4l_last_device_error(ws_d)
+    del c8
+    # second workload: the RG-LRU recurrence of a RecurrentGemma-2B-sized block (2560 channels) over a long prompt
+    rB, rT, rW = 4, 8192, 2560
+    gen = torch.Generator(device="cpu").manual_seed(1006)
+    rx = torch.randn(rB, rT, rW, generator=gen).to(torch.bfloat16).to(dev)
+    rgx = (torch.randn(rB, rT, rW, generator=gen) * 2).to(torch.bfloat16).to(dev)
+    rga = (torch.randn(rB, rT, rW, generator=gen) * 2).to(torch.bfloat16).to(dev)
+    r_ap = torch.log(torch.expm1(-torch.log(torch.rand(rW, generator=gen) * 0.099 + 0.9) / 8)).float().to(dev)
+    r_state = torch.zeros(rB, rW, dtype=torch.float32, device=dev)
+    ry = torch.empty_like(rx)
+    ws_r = l4l.new_rglru_workspace(rB, rT, rW, device=dev)
+    t_rglru = timed(lambda: l4l.l4l_rglru_scan(rx, rgx, rga, r_ap, r_state, ry, ws_r), 10)
+    rglru_bytes = rx.numel() * 8                          # 3 bf16 read + 1 written per (step, channel)
+    dev_err_r = l4l.l4l_last_device_error(ws_r)
+    del rx, rgx, rga, ry, filler
+    dev_err = l4l.l4l_last_device_error(ws_p) | l4l.l4l_last_device_error(ws_d) | dev_err_r
 
     # ---- end to end through the same entry points with HOST buffers (pinned), copies inside the timed region
     hq, hk, hv = seq.q.pin_memory(), seq.k.pin_memory(), seq.v.pin_memory()
@@ -394,8 +408,8 @@ def run_ours(args, rank, world):
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
 
     # ---- max over ranks
-    total_ms, e2e_ms, t_pre, t_dec, t_app, t_dec_b2b, t_rope, t_chunk, t_fused, t_paged, t_fp8 = max_over_ranks(
-        [total_ms, e2e_ms, t_pre, t_dec, t_app, t_dec_b2b, t_rope, t_chunk, t_fused, t_paged, t_fp8], world, dev)
+    total_ms, e2e_ms, t_pre, t_dec, t_app, t_dec_b2b, t_rope, t_chunk, t_fused, t_paged, t_fp8, t_rglru = max_over_ranks(
+        [total_ms, e2e_ms, t_pre, t_dec, t_app, t_dec_b2b, t_rope, t_chunk, t_fused, t_paged, t_fp8, t_rglru], world, dev)
     if rank != 0:
         return
 
@@ -440,6 +454,9 @@ def run_ours(args, rank, world):
             "prefill_from_cache": {"ms": t_chunk, "tflops": pre_flops / (t_chunk * 1e-3) / 1e12},
             "decode_with_fused_append": {"us": t_fused * 1e3, "kv_gbs": dec_bytes / (t_fused * 1e-3) / 1e9},
             "decode_paged_64": {"us": t_paged * 1e3, "kv_gbs": dec_bytes / (t_paged * 1e-3) / 1e9},
+            "rglru_scan_B4_T8192_W2560": {"us": t_rglru * 1e3, "gbs": rglru_bytes / (t_rglru * 1e-3) / 1e9,
+                                          "frac_of_measured_hbm": rglru_bytes / (t_rglru * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                          "bytes": rglru_bytes},
             "decode_fp8_cache": {"us": t_fp8 * 1e3, "kv_gbs_fp8_bytes": dec_bytes / 2 / (t_fp8 * 1e-3) / 1e9,
                                  "speedup_over_bf16_cache": t_dec_b2b / t_fp8},
         },
