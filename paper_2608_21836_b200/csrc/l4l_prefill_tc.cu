@@ -37,7 +37,7 @@ struct TcCfg {
     static constexpr int kSlots = (D == 128) ? 4 : 8;                    // ring of K/V tiles
     static constexpr uint32_t kTmemCols = 512;
     static constexpr uint32_t kColS0 = 0, kColS1 = 128, kColO0 = 256, kColO1 = 256 + D;
-    static constexpr int kNumBars = 1 + 2 * kSlots + 6;
+    static constexpr int kNumBars = 1 + 2 * kSlots + 8;
     static constexpr size_t kSmemBytes = 1024 + 2 * kTileBytes + (size_t)kSlots * kTileBytes + kNumBars * 8 + 64;
 };
 
@@ -53,7 +53,7 @@ struct TcParams {
     unsigned *status;
     int S_max, B, Hq, Hkv, G, n_qblocks;
     float scale_log2e;
-    TmapCoord cq, ckv;
+    TmapCoord cq, ckv, co;
 };
 
 __device__ __forceinline__ void order_coords(const TmapCoord &c, int t, int h, int b, int &c1, int &c2, int &c3)
@@ -87,7 +87,8 @@ __host__ __device__ constexpr uint32_t make_idesc(int n, bool b_mn_major)
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
-                  const __grid_constant__ CUtensorMap tmap_v, const TcParams p)
+                  const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_o,
+                  const TcParams p)
 {
     using C = TcCfg<D>;
     // ---- which block: heaviest (longest causal span) blocks first, heads of a KV group adjacent
@@ -97,20 +98,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     const int hb = blockIdx.x % per_block;
     const int h = hb % p.Hq, b = hb / p.Hq;
     const int kvh = h / p.G;
-    int L = p.seq_lens[b];
-    L = L < 0 ? 0 : (L > p.S_max ? p.S_max : L);
+    // The two lengths are requested now and first looked at after the barrier / TMEM set-up below, so that
+    // their latency is hidden behind it.
+    const int L_raw = __ldg(p.seq_lens + b);
+    const int past_raw = p.past_lens ? __ldg(p.past_lens + b) : 0;
     const int q0 = qb * 2 * kRows;
-    if (q0 >= L) return;
-    // Tokens already in the cache ahead of this chunk (0 for a fresh prompt): query row i sees keys
-    // 0 .. past + i. kv_total keys exist in all.
-    int past = p.past_lens ? p.past_lens[b] : 0;
-    past = past < 0 ? 0 : past;
-    const int kv_total = past + L;
-    // sub-tile i (rows q0 + 128 i ..) visits K/V tiles 0 .. tile of its last valid row's last key
-    int n_sub[2];
-    n_sub[0] = (past + min(q0 + kRows - 1, L - 1)) / kRows + 1;
-    n_sub[1] = (q0 + kRows < L) ? (past + min(q0 + 2 * kRows - 1, L - 1)) / kRows + 1 : 0;
-    const int n_kv = max(n_sub[0], n_sub[1]);
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -124,7 +116,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     uint64_t *s_full = kv_empty + C::kSlots;      // [2]
     uint64_t *p_full = s_full + 2;                // [2]
     uint64_t *o_full = p_full + 2;                // [2]
-    uint32_t *tmem_base_smem = reinterpret_cast<uint32_t *>(o_full + 2);
+    uint64_t *o_staged = o_full + 2;              // [2] a sub-tile's output rows are in shared memory
+    uint32_t *tmem_base_smem = reinterpret_cast<uint32_t *>(o_staged + 2);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_base_smem + 1);
     volatile int *copy_go = abort_flag + 1;       // producer -> helper warps: all loads issued
 
@@ -140,18 +133,31 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
             mbar_init(&s_full[i], 1);
             mbar_init(&p_full[i], kRows);
             mbar_init(&o_full[i], 1);
+            mbar_init(&o_staged[i], kRows);
         }
         *abort_flag = 0;
         *copy_go = 0;
         fence_barrier_init();
         fence_proxy_async_smem();
     }
+    // first use of the lengths. A block past the end of its sequence has nothing to do (decided before any
+    // TMEM is taken).
+    const int L = L_raw < 0 ? 0 : (L_raw > p.S_max ? p.S_max : L_raw);
+    if (q0 >= L) return;
+    // Tokens already in the cache ahead of this chunk (0 for a fresh prompt): query row i sees keys
+    // 0 .. past + i. kv_total keys exist in all.
+    const int past = past_raw < 0 ? 0 : past_raw;
+    const int kv_total = past + L;
+    // sub-tile i (rows q0 + 128 i ..) visits K/V tiles 0 .. tile of its last valid row's last key
+    int n_sub[2];
+    n_sub[0] = (past + min(q0 + kRows - 1, L - 1)) / kRows + 1;
+    n_sub[1] = (q0 + kRows < L) ? (past + min(q0 + 2 * kRows - 1, L - 1)) / kRows + 1 : 0;
+    const int n_kv = max(n_sub[0], n_sub[1]);
     if (warp == 9) {
         tmem_alloc(tmem_base_smem, C::kTmemCols);
         tmem_relinquish_alloc_permit();
     }
-    // Programmatic dependent launch: the set-up above may overlap the tail of the previous kernel of the
-    // stream; no global memory other than the kernel parameters is touched before it has completed.
+    // Programmatic dependent launch: the next kernel of the stream may start its own prologue now.
     grid_launch_dependents();
     tcgen05_fence_before_sync();
     __syncthreads();
@@ -442,12 +448,28 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
             const float inv = 1.f / l;
             const bool valid = row < L;
             __nv_bfloat16 *orow = p.o + b * p.o_sb + (int64_t)row * p.o_st + h * p.o_sh;
+            // A sub-tile whose 128 rows are all valid leaves through shared memory and one TMA store per 64
+            // columns (coalesced, asynchronous): the rows are staged where Q_i was, which no MMA reads any more
+            // (o_full follows the last of them). A ragged sub-tile writes its valid rows directly.
+            const bool whole = q0 + i * kRows + kRows <= L;
+            uint8_t *stage = q_smem + i * C::kTileBytes;
 #pragma unroll
             for (int qd = 0; qd < D / 32; ++qd) {
                 uint32_t orr[32];
                 tmem_ld_32x32b_x32(tmem_o + qd * 32, orr);
                 tcgen05_wait_ld();
-                if (valid) {
+                if (whole) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        uint4 val;
+                        val.x = pack_bf16x2(__uint_as_float(orr[8 * e + 0]) * inv, __uint_as_float(orr[8 * e + 1]) * inv);
+                        val.y = pack_bf16x2(__uint_as_float(orr[8 * e + 2]) * inv, __uint_as_float(orr[8 * e + 3]) * inv);
+                        val.z = pack_bf16x2(__uint_as_float(orr[8 * e + 4]) * inv, __uint_as_float(orr[8 * e + 5]) * inv);
+                        val.w = pack_bf16x2(__uint_as_float(orr[8 * e + 6]) * inv, __uint_as_float(orr[8 * e + 7]) * inv);
+                        const int ch = qd * 4 + e;                 // 16-byte chunk of the row
+                        *reinterpret_cast<uint4 *>(stage + (ch >> 3) * kHalfBytes + swz128(t, ch & 7)) = val;
+                    }
+                } else if (valid) {
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         uint4 val;
@@ -457,6 +479,18 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
                         val.w = pack_bf16x2(__uint_as_float(orr[8 * e + 6]) * inv, __uint_as_float(orr[8 * e + 7]) * inv);
                         *reinterpret_cast<uint4 *>(orow + qd * 32 + e * 8) = val;
                     }
+                }
+            }
+            if (whole) {
+                fence_proxy_async_smem();                          // this thread's rows, for the TMA store
+                mbar_arrive(&o_staged[i]);
+                if (t == 0 && mbar_wait(&o_staged[i], 0, abort_flag)) {
+                    int c1, c2, c3;
+                    order_coords(p.co, q0 + i * kRows, h, b, c1, c2, c3);
+#pragma unroll
+                    for (int hf = 0; hf < C::kHalves; ++hf) tma_store_4d(&tmap_o, stage + hf * kHalfBytes, hf * 64, c1, c2, c3);
+                    tma_store_commit();
+                    tma_store_wait_read_all();                     // shared memory must outlive the reads
                 }
             }
             if (valid && p.lse)
@@ -477,8 +511,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
 }
 
 template <int D>
-l4l_status launch_t(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const TcParams &p,
-                    cudaStream_t stream)
+l4l_status launch_t(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const CUtensorMap &to,
+                    const TcParams &p, cudaStream_t stream)
 {
     using C = TcCfg<D>;
     static bool configured = false;
@@ -500,7 +534,7 @@ l4l_status launch_t(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensor
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, prefill_tc_kernel<D>, tq, tk, tv, p) == cudaSuccess ? L4L_OK : L4L_ERR_CUDA;
+    return cudaLaunchKernelEx(&cfg, prefill_tc_kernel<D>, tq, tk, tv, to, p) == cudaSuccess ? L4L_OK : L4L_ERR_CUDA;
 }
 
 }  // namespace
@@ -510,9 +544,10 @@ l4l_status launch_prefill_tc(const l4l_tensor4 &q, const l4l_tensor4 &k, const l
                              int S_max, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
                              void *workspace, cudaStream_t stream, const int32_t *d_past_lens, int kv_extent)
 {
-    CUtensorMap tq, tk, tv;
-    TmapCoord cq, ck, cv;
+    CUtensorMap tq, tk, tv, to;
+    TmapCoord cq, ck, cv, co;
     if (!make_tmap_bf16(&tq, &cq, q.ptr, D, S_max, Hq, B, q.stride_t, q.stride_h, q.stride_b, 64, kRows) ||
+        !make_tmap_bf16(&to, &co, o.ptr, D, S_max, Hq, B, o.stride_t, o.stride_h, o.stride_b, 64, kRows) ||
         !make_tmap_bf16(&tk, &ck, k.ptr, D, kv_extent, Hkv, B, k.stride_t, k.stride_h, k.stride_b, 64, kRows) ||
         !make_tmap_bf16(&tv, &cv, v.ptr, D, kv_extent, Hkv, B, v.stride_t, v.stride_h, v.stride_b, 64, kRows))
         return L4L_ERR_CUDA;
@@ -531,8 +566,8 @@ l4l_status launch_prefill_tc(const l4l_tensor4 &q, const l4l_tensor4 &k, const l
     p.S_max = S_max; p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.G = Hq / Hkv;
     p.n_qblocks = (S_max + 2 * kRows - 1) / (2 * kRows);
     p.scale_log2e = scale * 1.4426950408889634f;
-    p.cq = cq; p.ckv = ck;
-    return (D == 128) ? launch_t<128>(tq, tk, tv, p, stream) : launch_t<64>(tq, tk, tv, p, stream);
+    p.cq = cq; p.ckv = ck; p.co = co;
+    return (D == 128) ? launch_t<128>(tq, tk, tv, to, p, stream) : launch_t<64>(tq, tk, tv, to, p, stream);
 }
 
 }  // namespace l4l
