@@ -176,9 +176,8 @@ l4l_status l4l_attn_decode_fp8(const void *q, void *o, l4l_kv_cache cache8, cons
  *   d_position   device int32 [B, T], or NULL: no resets (a chunk that continues its sequence)
  *   d_seq_lens   device int32 [B], or NULL meaning T for all
  *   d_state      device float [B, W], read and written
- *   workspace    >= 256 bytes, initialised once. With l4l_rglru_workspace_bytes(B, T, W) bytes the time axis
- *                of short batches is cut into segments that run in parallel (same results up to fp32
- *                rounding order); with less, one warp walks each 64-channel strip from start to end.
+ *   workspace    >= l4l_rglru_workspace_bytes(B, T, W) bytes, initialised once (at present the 256-byte
+ *                status block: the state is handed from tile to tile on chip)
  */
 size_t l4l_rglru_workspace_bytes(int B, int T, int W);
 l4l_status l4l_rglru_scan(const void *x, const void *gate_x, const void *gate_a, const float *d_a_param,

@@ -40,11 +40,11 @@ def check(y_gpu, st_gpu, y_ref, st_ref, valid):
     assert serr.max() <= 5e-3, f"state max-abs {serr.max():.3g}"
 
 
-@pytest.mark.parametrize("segmented", [False, True])
-@pytest.mark.parametrize("B,T,W", [(2, 300, 2560), (3, 65, 40), (1, 1, 64), (5, 1000, 96)])
-def test_rglru_matches_oracle(B, T, W, segmented):
-    """segmented: the workspace is large enough for the time axis to be cut into parallel segments (these batches
-    are small enough for that to happen whenever T >= 128); otherwise the status block alone forces one pass."""
+@pytest.mark.parametrize("B,T,W", [(2, 300, 2560), (3, 65, 40), (1, 1, 64), (5, 1000, 96), (1, 16, 64), (2, 17, 128)])
+def test_rglru_matches_oracle(B, T, W):
+    """Sequences of many tiles (eight warps hand the state on from tile to tile), of exactly one tile (the one-warp
+    variant) and just past it; a second segment inside a sequence, ragged lengths, a channel count that does not fill
+    the last 64-channel strip."""
     x, gx, ga, ap, h0 = make(B, T, W, 1100 + T)
     pos = torch.arange(T, dtype=torch.int32).repeat(B, 1)
     if T > 40:
@@ -53,7 +53,7 @@ def test_rglru_matches_oracle(B, T, W, segmented):
     y_ref, st_ref = orc.rglru(x, gx, ga, ap.numpy(), state=h0.double().numpy(), position=pos.numpy(), seq_len=lens)
     gy = Guarded(torch.full((B, T, W), SENTINEL, dtype=torch.int16).view(torch.bfloat16))
     gs = Guarded(h0)
-    ws = l4l.new_rglru_workspace(B, T, W) if segmented else l4l.new_workspace(l4l.L4L_OP_PREFILL, 1, 1, 1, 64, 1)
+    ws = l4l.new_rglru_workspace(B, T, W)
     l4l.l4l_rglru_scan(x.cuda(), gx.cuda(), ga.cuda(), ap.cuda(), gs.t, gy.t, ws, position=pos.cuda(),
                        seq_lens=torch.tensor(lens, dtype=torch.int32).cuda())
     torch.cuda.synchronize()
