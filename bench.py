@@ -473,7 +473,8 @@ def run_ours(args, rank, world):
 
 def run_profile_case(case: str):
     """A few launches of ONE kernel on a small case, for `ncu` captures (not a benchmark):
-    prefill = B=1, S=8192 of the long_prefill workload (inputs 168 MB > L2); decode = the batched_decode batch."""
+    prefill = B=1, S=8192 of the long_prefill workload (inputs 168 MB > L2); decode = the batched_decode batch;
+    rglru = the RG-LRU scan on B=16, T=2048, W=2560."""
     from paper_2608_21836_b200 import binding as l4l
 
     torch.cuda.set_device(0)
@@ -488,6 +489,18 @@ def run_profile_case(case: str):
         ws = l4l.new_workspace(l4l.L4L_OP_PREFILL, 1, w.Hq, w.Hkv, w.D, seq.S)
         for _ in range(3):
             l4l.l4l_attn_prefill(q, k, v, o, lens, w.scale, ws, cache_k=ck, cache_v=cv)
+    elif case == "rglru":
+        B, T, W = 16, 2048, 2560                          # 503 MB of inputs, 168 MB of output
+        gen = torch.Generator().manual_seed(1006)
+        x = torch.randn(B, T, W, generator=gen).to(torch.bfloat16).cuda()
+        gx = (torch.randn(B, T, W, generator=gen) * 2).to(torch.bfloat16).cuda()
+        ga = (torch.randn(B, T, W, generator=gen) * 2).to(torch.bfloat16).cuda()
+        ap = torch.log(torch.expm1(-torch.log(torch.rand(W, generator=gen) * 0.099 + 0.9) / 8)).float().cuda()
+        state = torch.zeros(B, W, device="cuda")
+        y = torch.empty_like(x)
+        ws = l4l.new_rglru_workspace(B, T, W)
+        for _ in range(3):
+            l4l.l4l_rglru_scan(x, gx, ga, ap, state, y, ws)
     else:
         w = wl.WORKLOADS["batched_decode"]
         db = wl.make_decode_batch(w)
@@ -507,7 +520,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--profile-case", choices=["prefill", "decode"], default=None,
+    ap.add_argument("--profile-case", choices=["prefill", "decode", "rglru"], default=None,
                     help="run three launches of one kernel on a small case and exit (for ncu)")
     args = ap.parse_args()
     if args.profile_case:
