@@ -332,6 +332,7 @@ l4l_status l4l_rglru_scan(const void *x, const void *gate_x, const void *gate_a,
 {
     if (B < 0 || T < 0 || W <= 0) return L4L_ERR_INVALID_ARG;
     if (W % 8 != 0 || B > 65535) return L4L_ERR_UNSUPPORTED;       // 16-byte rows for the tensor maps; grid.y
+    if (B == 0 || T == 0) return L4L_OK;                            // nothing to do (empty tensors have no address)
     if (!x || !gate_x || !gate_a || !d_a_param || !d_state || !y) return L4L_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(gate_x) || !aligned16(gate_a)) return L4L_ERR_INVALID_ARG;
     if (!workspace || ws_bytes < kStatusBytes) return L4L_ERR_WORKSPACE;

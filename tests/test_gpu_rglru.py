@@ -96,3 +96,17 @@ def test_rglru_rejects_bad_shapes():
     with pytest.raises(l4l.L4LError):
         l4l.l4l_rglru_scan(x, x.clone(), x.clone(), torch.zeros(12, device="cuda"), torch.zeros(1, 12, device="cuda"),
                            x.clone(), ws)
+
+
+def test_rglru_empty_inputs_are_a_no_op():
+    ws = l4l.new_workspace(l4l.L4L_OP_PREFILL, 1, 1, 1, 64, 1)
+    state = torch.full((2, 64), 7.0, device="cuda")
+    e = torch.zeros(2, 0, 64, dtype=torch.bfloat16, device="cuda")
+    l4l.l4l_rglru_scan(e, e.clone(), e.clone(), torch.zeros(64, device="cuda"), state, e.clone(), ws)
+    # all sequences of length 0: the state comes back unchanged
+    x = torch.randn(2, 8, 64, device="cuda").to(torch.bfloat16)
+    y = torch.full((2, 8, 64), 3.0, device="cuda").to(torch.bfloat16)
+    l4l.l4l_rglru_scan(x, x.clone(), x.clone(), torch.zeros(64, device="cuda"), state, y, ws,
+                       seq_lens=torch.zeros(2, dtype=torch.int32, device="cuda"))
+    torch.cuda.synchronize()
+    assert (state == 7.0).all() and (y == 3.0).all() and l4l.l4l_last_device_error(ws) == 0
