@@ -15,6 +15,13 @@
  *                                  pass over that group's cache.
  *   l4l_kv_append                : the cache update (an exact copy).
  *
+ * Further entry points widen that path, each documented at its declaration:
+ *   l4l_attn_prefill_chunk (new tokens over a populated cache), l4l_attn_decode_append (cache
+ *   update fused into the decode step), l4l_rope_kv_append (rotary embedding and QK-norm fused
+ *   with the cache update), l4l_attn_decode_paged / l4l_kv_append_paged (page pool + block
+ *   table), l4l_attn_decode_fp8 / l4l_kv_append_fp8 (e4m3 cache), l4l_attn_decode_static (no
+ *   caller workspace), and a second workload, l4l_rglru_scan (gated linear recurrence).
+ *
  * Conventions shared by every call
  *   - All tensors are bf16 (16-bit words) in DEVICE memory unless a parameter says "host".
  *     head_dim (D) is the contiguous innermost dimension; the other strides are passed in
