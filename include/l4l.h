@@ -165,6 +165,13 @@ l4l_status l4l_attn_decode_fp8(const void *q, void *o, l4l_kv_cache cache8, cons
                                const float *d_v_scale, const int32_t *d_kv_lens, int max_kv_len,
                                int B, int Hq, int Hkv, int head_dim, float scale, float *d_lse,
                                void *workspace, size_t ws_bytes, l4l_stream stream);
+/* Both at once: an fp8 page pool (l4l_paged_kv with k / v pointing at bytes, strides in bytes, multiples
+ * of 16) read through a block table. Rules of l4l_attn_decode_paged and l4l_attn_decode_fp8 combined. */
+l4l_status l4l_attn_decode_paged_fp8(const void *q, void *o, l4l_paged_kv pool8, const float *d_k_scale,
+                                     const float *d_v_scale, const int32_t *d_block_table, int table_stride,
+                                     const int32_t *d_kv_lens, int max_kv_len, int B, int Hq, int Hkv,
+                                     int head_dim, float scale, float *d_lse, void *workspace,
+                                     size_t ws_bytes, l4l_stream stream);
 
 /*
  * Second workload: the gated linear recurrence of the RecurrentGemma block (RG-LRU). The paper's

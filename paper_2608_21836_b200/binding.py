@@ -24,6 +24,7 @@ EXPORTS = (
     "l4l_last_device_error", "l4l_kv_append", "l4l_attn_prefill", "l4l_attn_decode",
     "l4l_attn_decode_static", "l4l_attn_decode_append", "l4l_attn_prefill_chunk", "l4l_rope_kv_append",
     "l4l_kv_append_paged", "l4l_attn_decode_paged", "l4l_kv_append_fp8", "l4l_attn_decode_fp8", "l4l_rglru_scan", "l4l_rglru_workspace_bytes",
+    "l4l_attn_decode_paged_fp8",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -93,6 +94,9 @@ def load() -> ctypes.CDLL:
     lib.l4l_attn_decode_fp8.restype = c_int
     lib.l4l_attn_decode_fp8.argtypes = [vp, vp, KVCache, vp, vp, i32p, c_int, c_int, c_int, c_int, c_int,
                                         ctypes.c_float, vp, vp, c_size, vp]
+    lib.l4l_attn_decode_paged_fp8.restype = c_int
+    lib.l4l_attn_decode_paged_fp8.argtypes = [vp, vp, PagedKV, vp, vp, i32p, c_int, i32p, c_int, c_int, c_int, c_int, c_int,
+                                              ctypes.c_float, vp, vp, c_size, vp]
     lib.l4l_rglru_workspace_bytes.restype = c_size
     lib.l4l_rglru_workspace_bytes.argtypes = [c_int, c_int, c_int]
     lib.l4l_rglru_scan.restype = c_int
@@ -431,3 +435,24 @@ def new_rglru_workspace(B: int, T: int, W: int, device=None) -> torch.Tensor:
         raise ValueError("unsupported sizes")
     ws = torch.zeros((n + 7) // 8, dtype=torch.int64, device=device or "cuda")
     return ws
+
+
+def l4l_attn_decode_paged_fp8(q, o, pool_k8, pool_v8, k_scale, v_scale, block_table, kv_lens, max_kv_len: int, scale: float,
+                              workspace, lse=None) -> None:
+    """Decode over an fp8 page pool [pages, Hkv, page_size, 128] (uint8 / float8_e4m3fn) read through a block table."""
+    _check_bf16_cuda(q, "q")
+    _check_bf16_cuda(o, "o")
+    if not (q.is_contiguous() and o.is_contiguous() and q.dim() == 3 and q.shape == o.shape):
+        raise ValueError("q and o must be dense [B, Hq, D]")
+    B, Hq, D = q.shape
+    c = kv_cache8(pool_k8, pool_v8)                     # same checks; fields reinterpreted as a page pool
+    pool = PagedKV(c.k, c.v, c.stride_b, c.stride_h, c.stride_t, pool_k8.shape[2], pool_k8.shape[0])
+    Hkv = pool_k8.shape[1]
+    tbl, stride = _block_table(block_table, B)
+    st = load().l4l_attn_decode_paged_fp8(q.data_ptr(), o.data_ptr(), pool, _f32_dev(k_scale, "k_scale", (Hkv,)),
+                                          _f32_dev(v_scale, "v_scale", (Hkv,)), tbl, stride, _i32_dev(kv_lens, "kv_lens"),
+                                          int(max_kv_len), B, Hq, Hkv, D, float(scale),
+                                          None if lse is None else lse.data_ptr(), workspace.data_ptr(),
+                                          workspace.numel() * workspace.element_size(), _stream())
+    if st != L4L_OK:
+        raise L4LError(st, "l4l_attn_decode_paged_fp8")

@@ -326,6 +326,32 @@ l4l_status l4l_attn_decode_fp8(const void *q, void *o, l4l_kv_cache cache8, cons
                          static_cast<cudaStream_t>(stream), nullptr, nullptr, nullptr, &sc);
 }
 
+l4l_status l4l_attn_decode_paged_fp8(const void *q, void *o, l4l_paged_kv pool8, const float *d_k_scale,
+                                     const float *d_v_scale, const int32_t *d_block_table, int table_stride,
+                                     const int32_t *d_kv_lens, int max_kv_len, int B, int Hq, int Hkv, int head_dim,
+                                     float scale, float *d_lse, void *workspace, size_t ws_bytes, l4l_stream stream)
+{
+    l4l_status st = shape_status(B, Hq, Hkv, head_dim);
+    if (st != L4L_OK) return st;
+    if (head_dim != 128) return L4L_ERR_UNSUPPORTED;
+    if (!q || !o || !d_kv_lens || !d_block_table || !d_k_scale || !d_v_scale || !aligned16(q) || !aligned16(o))
+        return L4L_ERR_INVALID_ARG;
+    auto s16 = [](int64_t s) { return s >= 0 && (s % 16) == 0; };
+    if (!pool8.k || !pool8.v || !aligned16(pool8.k) || !aligned16(pool8.v) || !s16(pool8.stride_page) ||
+        !s16(pool8.stride_h) || !s16(pool8.stride_t) || pool8.num_pages <= 0 || pool8.page_size < 16 ||
+        pool8.page_size > (1 << 20) || (pool8.page_size & (pool8.page_size - 1)) != 0 || table_stride <= 0)
+        return L4L_ERR_INVALID_ARG;
+    if (max_kv_len < 0 || (long long)max_kv_len > (long long)table_stride * pool8.page_size) return L4L_ERR_INVALID_ARG;
+    if (!workspace || ws_bytes < kStatusBytes) return L4L_ERR_WORKSPACE;
+    if (B == 0) return L4L_OK;
+    const DecodePlan plan = plan_decode(B, Hq, Hkv, head_dim, max_kv_len, ws_bytes, true);
+    if (plan.ws_bytes > ws_bytes) return L4L_ERR_WORKSPACE;
+    const PagedTable pt{d_block_table, table_stride, pool8.num_pages};
+    const Fp8Scales sc{d_k_scale, d_v_scale};
+    return launch_decode(q, o, pool_as_cache(pool8), d_kv_lens, max_kv_len, B, Hq, Hkv, head_dim, scale, d_lse, workspace,
+                         plan, static_cast<cudaStream_t>(stream), nullptr, nullptr, &pt, &sc);
+}
+
 l4l_status l4l_rglru_scan(const void *x, const void *gate_x, const void *gate_a, const float *d_a_param,
                           const int32_t *d_position, const int32_t *d_seq_lens, float *d_state, void *y, int B, int T,
                           int W, void *workspace, size_t ws_bytes, l4l_stream stream)

@@ -108,3 +108,47 @@ def test_fp8_decode_rejects_head_dim_64():
     with pytest.raises(l4l.L4LError):
         l4l.l4l_attn_decode_fp8(q, q.clone(), c8, c8.clone(), sc, sc, torch.ones(1, dtype=torch.int32, device="cuda"),
                                 32, 0.1, ws)
+
+
+@pytest.mark.parametrize("page", [16, 64, 256])
+def test_fp8_paged_decode_matches_oracle(page):
+    """An fp8 page pool behind a block table: the oracle gathers the pages (codes are bytes: the gather is the same
+    indexing as for bf16) and decodes over the codes."""
+    Hq, Hkv, D = 16, 4, 128
+    lens = [1, 17, 255, 256, 257, 1500, 0, 640]
+    B = len(lens)
+    g = torch.Generator().manual_seed(2000 + page)
+    need = [(L + page - 1) // page for L in lens]
+    n_pages = sum(need) + 4
+    table = np.full((B, max(need) + 1), -1, np.int32)
+    perm = iter(torch.randperm(n_pages, generator=g).tolist())
+    pool_k = torch.full((n_pages, Hkv, page, D), 0x7F, dtype=torch.uint8)
+    pool_v = torch.full((n_pages, Hkv, page, D), 0xFF, dtype=torch.uint8)
+    for b in range(B):
+        for i in range(need[b]):
+            pg = next(perm)
+            table[b, i] = pg
+            n = min(page, lens[b] - i * page)
+            pool_k[pg, :, :n] = random_codes((Hkv, n, D), g, 7)
+            pool_v[pg, :, :n] = random_codes((Hkv, n, D), g, 7)
+    q = torch.randn(B, Hq, D, generator=g).to(torch.bfloat16)
+    ks, vs = torch.rand(Hkv, generator=g) + 0.5, torch.rand(Hkv, generator=g) + 0.25
+    Lmax = max(lens)
+    # gather the code pages into contiguous code caches (reusing the bf16 gather on 16-bit views is not possible for
+    # bytes, so index directly: slot s of sequence b = row s % page of page table[b, s // page])
+    ck8 = torch.zeros(B, Hkv, Lmax, D, dtype=torch.uint8)
+    cv8 = torch.zeros(B, Hkv, Lmax, D, dtype=torch.uint8)
+    for b in range(B):
+        for s0 in range(0, lens[b], page):
+            n = min(page, lens[b] - s0)
+            ck8[b, :, s0:s0 + n] = pool_k[table[b, s0 // page], :, :n]
+            cv8[b, :, s0:s0 + n] = pool_v[table[b, s0 // page], :, :n]
+    ref, _ = orc.decode_fp8(q, ck8, cv8, np.array(lens, np.int32), ks.numpy(), vs.numpy(), 0.09)
+    o = torch.zeros(B, Hq, D, dtype=torch.bfloat16, device="cuda")
+    ws = l4l.new_workspace(l4l.L4L_OP_DECODE, B, Hq, Hkv, D, Lmax)
+    l4l.l4l_attn_decode_paged_fp8(q.cuda(), o, pool_k.cuda(), pool_v.cuda(), ks.cuda(), vs.cuda(),
+                                  torch.from_numpy(table).cuda(), torch.tensor(lens, dtype=torch.int32).cuda(), Lmax,
+                                  0.09, ws)
+    torch.cuda.synchronize()
+    assert l4l.l4l_last_device_error(ws) == 0
+    assert_close_to_oracle(o.cpu(), ref, f"fp8 paged decode, page {page}")
