@@ -1,0 +1,98 @@
+"""The entry points enqueue on the caller's stream and never synchronise, so a decode step (append + decode, or the
+fused form) and a prefill can be captured in a CUDA graph and replayed with new data in the same buffers."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import l4l_oracle as orc
+from paper_2608_21836_b200 import binding as l4l
+from helpers import assert_close_to_oracle
+
+pytestmark = pytest.mark.gpu
+
+
+def test_decode_step_in_a_cuda_graph_replays_with_new_inputs():
+    B, Hq, Hkv, D, Lmax = 4, 8, 2, 128, 512
+    g = torch.Generator().manual_seed(11)
+    ck = torch.randn(B, Hkv, Lmax, D, generator=g).to(torch.bfloat16)
+    cv = torch.randn(B, Hkv, Lmax, D, generator=g).to(torch.bfloat16)
+    lens0 = np.array([100, 257, 1, 400], np.int32)
+    dck, dcv = ck.cuda(), cv.cuda()
+    q = torch.zeros(B, Hq, D, dtype=torch.bfloat16, device="cuda")
+    kn = torch.zeros(B, 1, Hkv, D, dtype=torch.bfloat16, device="cuda")
+    vn = torch.zeros_like(kn)
+    pos = torch.zeros(B, dtype=torch.int32, device="cuda")
+    lens = torch.zeros(B, dtype=torch.int32, device="cuda")
+    o = torch.zeros_like(q)
+    ws = l4l.new_workspace(l4l.L4L_OP_DECODE, B, Hq, Hkv, D, Lmax)
+    scale = 1.0 / math.sqrt(D)
+
+    def step():
+        l4l.l4l_kv_append(dck, dcv, kn, vn, pos)
+        l4l.l4l_attn_decode(q, o, dck, dcv, lens, Lmax, scale, ws)
+
+    # warm up on a side stream (first calls set function attributes), then capture
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        pos.copy_(torch.from_numpy(lens0)); lens.copy_(torch.from_numpy(lens0 + 1))
+        step()
+    torch.cuda.current_stream().wait_stream(s)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    cur = lens0.copy()
+    ref_k, ref_v = orc.bits(ck).copy(), orc.bits(cv).copy()
+    # the warm-up step already appended zeros at lens0: mirror that
+    ref_k, ref_v = orc.kv_append(ref_k, ref_v, torch.zeros(B, 1, Hkv, D).to(torch.bfloat16),
+                                 torch.zeros(B, 1, Hkv, D).to(torch.bfloat16), cur, np.ones(B, np.int32))
+    for it in range(3):
+        qi = torch.randn(B, Hq, D, generator=g).to(torch.bfloat16)
+        ki = torch.randn(B, 1, Hkv, D, generator=g).to(torch.bfloat16)
+        vi = torch.randn(B, 1, Hkv, D, generator=g).to(torch.bfloat16)
+        q.copy_(qi); kn.copy_(ki); vn.copy_(vi)
+        pos.copy_(torch.from_numpy(cur)); lens.copy_(torch.from_numpy(cur + 1))
+        graph.replay()
+        torch.cuda.synchronize()
+        ref_k, ref_v = orc.kv_append(ref_k, ref_v, ki, vi, cur, np.ones(B, np.int32))
+        ref, _ = orc.decode(qi, ref_k, ref_v, cur + 1, scale)
+        assert l4l.l4l_last_device_error(ws) == 0
+        assert_close_to_oracle(o.cpu(), ref, f"graph replay {it}")
+        cur = cur + 1
+    assert np.array_equal(orc.bits(dck.cpu()), ref_k)
+
+
+def test_prefill_in_a_cuda_graph():
+    B, S, Hq, Hkv, D = 2, 300, 8, 2, 128
+    g = torch.Generator().manual_seed(12)
+    q = torch.zeros(B, S, Hq, D, dtype=torch.bfloat16, device="cuda")
+    k = torch.zeros(B, S, Hkv, D, dtype=torch.bfloat16, device="cuda")
+    v = torch.zeros_like(k)
+    o = torch.zeros_like(q)
+    ck = torch.zeros(B, Hkv, S, D, dtype=torch.bfloat16, device="cuda")
+    cv = torch.zeros_like(ck)
+    lens = torch.tensor([S, 77], dtype=torch.int32, device="cuda")
+    ws = l4l.new_workspace(l4l.L4L_OP_PREFILL, B, Hq, Hkv, D, S)
+    scale = 1.0 / math.sqrt(D)
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        l4l.l4l_attn_prefill(q, k, v, o, lens, scale, ws, cache_k=ck, cache_v=cv)
+    torch.cuda.current_stream().wait_stream(s)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        l4l.l4l_attn_prefill(q, k, v, o, lens, scale, ws, cache_k=ck, cache_v=cv)
+    qi = torch.randn(B, S, Hq, D, generator=g).to(torch.bfloat16)
+    ki = torch.randn(B, S, Hkv, D, generator=g).to(torch.bfloat16)
+    vi = torch.randn(B, S, Hkv, D, generator=g).to(torch.bfloat16)
+    q.copy_(qi); k.copy_(ki); v.copy_(vi)
+    graph.replay()
+    torch.cuda.synchronize()
+    ref, _ = orc.prefill(qi, ki, vi, np.array([S, 77], np.int32), scale)
+    assert l4l.l4l_last_device_error(ws) == 0
+    valid = torch.arange(S).view(1, S) < torch.tensor([S, 77]).view(B, 1)
+    assert_close_to_oracle(o.cpu()[valid], ref[valid.numpy()], "prefill in a graph")
