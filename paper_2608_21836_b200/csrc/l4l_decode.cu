@@ -602,6 +602,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
         const int r_lo = lane >> 2;          // query head within the group held in rows lane/4, lane/4+8
         const int r_hi = r_lo + 8;
         uint32_t n_dumps = 0;                // pieces handed to the finisher so far
+        float k_sc = 1.f, v_sc = 1.f;        // fp8 cache: scales of the piece's KV head (read once per piece)
 
         for (uint32_t it = 0;; ++it) {
             const uint32_t s = it % C::kStages;
@@ -620,6 +621,10 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
 
             if (mt.flags & kFlagFirst) {
                 st.reset();
+                if constexpr (F8) {
+                    k_sc = __ldg(p.k_scale + mt.kvh);
+                    v_sc = __ldg(p.v_scale + mt.kvh);
+                }
                 const uint32_t *qs = reinterpret_cast<const uint32_t *>(q_slots + (size_t)s * q_bytes);
                 const uint32_t *qrow_lo = qs + (size_t)r_lo * D / 2;
                 const uint32_t *qrow_hi = qs + (size_t)r_hi * D / 2;
@@ -677,7 +682,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     // tokens past the end get no weight and their V rows are cleared.
                     constexpr int kSub = C::kSub;
                     float sv[2 * kSub][4];
-                    const float sc = p.scale_log2e * __ldg(p.k_scale + mt.kvh);
+                    const float sc = p.scale_log2e * k_sc;
 #pragma unroll
                     for (int u = 0; u < kSub; ++u) {
                         if (u == 0 || nvalid > 16 * u) {
@@ -762,7 +767,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 float *cw = comb + (size_t)warp * p.G * kPitch;
                 // fp8: accumulator tiles alternate even / odd head dims (a tile pair gives this lane 4 consecutive
                 // dims) and O still lacks the V scale of its KV head
-                const float vs = F8 ? __ldg(p.v_scale + mt.kvh) : 1.f;
+                const float vs = F8 ? v_sc : 1.f;
                 if (r_lo < p.G) {
                     float *row = cw + (size_t)r_lo * kPitch;
                     if ((lane & 3) == 0) { row[D] = st.m[0]; row[D + 1] = l0; }
