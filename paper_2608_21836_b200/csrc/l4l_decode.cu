@@ -1,7 +1,9 @@
-// Decode attention: one query token per sequence over a ragged bf16 KV cache.
+// Decode attention: one query token per sequence over a ragged KV cache (bf16, or e4m3 bytes with a scale
+// per KV head; contiguous, or pages behind a block table: the template flag F8 and the optional page table
+// change the tile element type and the producer's coordinates, nothing else).
 //
 // One launch. The cache of every (sequence, KV head) is cut into tiles of 16*W tokens (W = 4 or 8
-// consumer warps); the flattened tile stream (sequence-major, then KV head, then position) is divided
+// consumer warps; twice that for fp8, where a warp takes 32 tokens per step); the flattened tile stream (sequence-major, then KV head, then position) is divided
 // among persistent CTAs as evenly as whole tiles allow, so every CTA streams the same number of bytes
 // (to within one tile) whatever the length mix. A CTA's range may
 // start or end inside a sequence: each (sequence, KV head) is thus covered by one or more

@@ -14,6 +14,10 @@
 //               from TMEM and V as an MN-major shared-memory operand; owns the TMEM allocation
 //   warps 10-11 help with the cache copy, which runs beside the last iterations
 //
+// The same kernel serves a chunk of new tokens over a populated cache (per-sequence offset `past`: row i is
+// position past + i, K/V come from the cache layout, the causal diagonal may then cross two tiles per sub-tile).
+// A whole sub-tile's output leaves through the shared memory that held its Q rows and TMA stores.
+//
 // TMEM columns: S0 [0,128) S1 [128,256) O0 [256,256+D) O1 [256+D,256+2D); P_i aliases the first 64
 // columns of S_i. Causal tile skipping: sub-tile i only visits K/V tiles up to its diagonal.
 // The tensor pipe executes one thread's MMAs in issue order, which is what makes the S/P aliasing
