@@ -174,6 +174,20 @@ l4l_status l4l_attn_decode_paged_fp8(const void *q, void *o, l4l_paged_kv pool8,
                                      size_t ws_bytes, l4l_stream stream);
 
 /*
+ * Merge of R partial decode results over DISJOINT parts of the same sequences' caches: the step that
+ * context-parallel decode adds (one sequence's cache sharded over R GPUs: every rank calls
+ * l4l_attn_decode over its shard with d_lse set, the R (o, lse) pairs are gathered, this call combines
+ * them). The paper runs on one GPU and has no counterpart; the formula is the one the split decode
+ * kernel uses between its pieces:
+ *     o = sum_r w_r o_r / sum_r w_r,   lse = m + ln sum_r w_r,   w_r = exp(lse_r - m),  m = max_r lse_r
+ * A shard without keys has lse_r = -inf and weight 0; if all are empty, o = 0 and lse = -inf.
+ *   o_parts      device bf16 [R, B, Hq, D] dense        d_lse_parts  device float [R, B, Hq]
+ *   o            device bf16 [B, Hq, D] dense           d_lse        device float [B, Hq] or NULL
+ */
+l4l_status l4l_attn_merge(const void *o_parts, const float *d_lse_parts, int R, void *o, float *d_lse,
+                          int B, int Hq, int head_dim, l4l_stream stream);
+
+/*
  * Second workload: the gated linear recurrence of the RecurrentGemma block (RG-LRU). The paper's
  * appendix ("RecurrentGemma RGLRU", Table A.4) describes the accepted kernel as fusing sigmoid,
  * softplus-derived recurrent gating, reset handling, normalisation and the recurrent scan, with the

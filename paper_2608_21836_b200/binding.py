@@ -24,7 +24,7 @@ EXPORTS = (
     "l4l_last_device_error", "l4l_kv_append", "l4l_attn_prefill", "l4l_attn_decode",
     "l4l_attn_decode_static", "l4l_attn_decode_append", "l4l_attn_prefill_chunk", "l4l_rope_kv_append",
     "l4l_kv_append_paged", "l4l_attn_decode_paged", "l4l_kv_append_fp8", "l4l_attn_decode_fp8", "l4l_rglru_scan", "l4l_rglru_workspace_bytes",
-    "l4l_attn_decode_paged_fp8",
+    "l4l_attn_decode_paged_fp8", "l4l_attn_merge",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -97,6 +97,8 @@ def load() -> ctypes.CDLL:
     lib.l4l_attn_decode_paged_fp8.restype = c_int
     lib.l4l_attn_decode_paged_fp8.argtypes = [vp, vp, PagedKV, vp, vp, i32p, c_int, i32p, c_int, c_int, c_int, c_int, c_int,
                                               ctypes.c_float, vp, vp, c_size, vp]
+    lib.l4l_attn_merge.restype = c_int
+    lib.l4l_attn_merge.argtypes = [vp, vp, c_int, vp, vp, c_int, c_int, c_int, vp]
     lib.l4l_rglru_workspace_bytes.restype = c_size
     lib.l4l_rglru_workspace_bytes.argtypes = [c_int, c_int, c_int]
     lib.l4l_rglru_scan.restype = c_int
@@ -456,3 +458,17 @@ def l4l_attn_decode_paged_fp8(q, o, pool_k8, pool_v8, k_scale, v_scale, block_ta
                                           workspace.numel() * workspace.element_size(), _stream())
     if st != L4L_OK:
         raise L4LError(st, "l4l_attn_decode_paged_fp8")
+
+
+def l4l_attn_merge(o_parts, lse_parts, o, lse=None) -> None:
+    """Combines R partial decode results over disjoint key ranges. o_parts CUDA bf16 [R,B,Hq,D]; lse_parts CUDA
+    float32 [R,B,Hq]; o CUDA bf16 [B,Hq,D]; lse optional CUDA float32 [B,Hq]."""
+    _check_bf16_cuda(o_parts, "o_parts")
+    _check_bf16_cuda(o, "o")
+    R, B, Hq, D = o_parts.shape
+    if not (o_parts.is_contiguous() and o.is_contiguous() and tuple(o.shape) == (B, Hq, D)):
+        raise ValueError("o_parts must be dense [R, B, Hq, D] and o dense [B, Hq, D]")
+    st = load().l4l_attn_merge(o_parts.data_ptr(), _f32_dev(lse_parts, "lse_parts", (R, B, Hq)), R, o.data_ptr(),
+                               None if lse is None else _f32_dev(lse, "lse", (B, Hq)), B, Hq, D, _stream())
+    if st != L4L_OK:
+        raise L4LError(st, "l4l_attn_merge")

@@ -352,6 +352,16 @@ l4l_status l4l_attn_decode_paged_fp8(const void *q, void *o, l4l_paged_kv pool8,
                          plan, static_cast<cudaStream_t>(stream), nullptr, nullptr, &pt, &sc);
 }
 
+l4l_status l4l_attn_merge(const void *o_parts, const float *d_lse_parts, int R, void *o, float *d_lse, int B, int Hq,
+                          int head_dim, l4l_stream stream)
+{
+    if (B < 0 || Hq <= 0 || R <= 0) return L4L_ERR_INVALID_ARG;
+    if (head_dim != 64 && head_dim != 128) return L4L_ERR_UNSUPPORTED;
+    if (B == 0) return L4L_OK;
+    if (!o_parts || !d_lse_parts || !o || !aligned16(o_parts) || !aligned16(o)) return L4L_ERR_INVALID_ARG;
+    return launch_attn_merge(o_parts, d_lse_parts, R, o, d_lse, B, Hq, head_dim, static_cast<cudaStream_t>(stream));
+}
+
 l4l_status l4l_rglru_scan(const void *x, const void *gate_x, const void *gate_a, const float *d_a_param,
                           const int32_t *d_position, const int32_t *d_seq_lens, float *d_state, void *y, int B, int T,
                           int W, void *workspace, size_t ws_bytes, l4l_stream stream)

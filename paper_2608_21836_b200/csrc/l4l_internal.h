@@ -77,6 +77,9 @@ l4l_status launch_kv_append_fp8(const l4l_kv_cache &cache, const l4l_tensor4 &k_
                                 const int32_t *d_write_pos, const int32_t *d_n_new, int n_new_max, int B, int Hkv,
                                 int D, const float *d_k_scale, const float *d_v_scale, cudaStream_t stream);
 
+l4l_status launch_attn_merge(const void *o_parts, const float *lse_parts, int R, void *o, float *d_lse, int B, int Hq,
+                             int D, cudaStream_t stream);
+
 l4l_status launch_rglru_scan(const void *x, const void *gate_x, const void *gate_a, const float *d_a_param,
                              const int32_t *d_position, const int32_t *d_seq_lens, float *d_state, void *y, int B, int T,
                              int W, void *workspace, size_t ws_bytes, cudaStream_t stream);
