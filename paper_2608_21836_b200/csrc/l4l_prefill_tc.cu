@@ -127,7 +127,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    if (threadIdx.x == 0) {
+    // The producer's lane sets the barriers up itself, so that it can start the first loads right away, while
+    // the other warps are still on their way to the block-wide barrier below (TMEM allocation included).
+    const bool producer_lane = threadIdx.x == 8 * 32;
+    if (producer_lane) {
         mbar_init(q_full, 1);
         for (int s = 0; s < C::kSlots; ++s) {
             mbar_init(&kv_full[s], 1);
@@ -157,6 +160,34 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     n_sub[0] = (past + min(q0 + kRows - 1, L - 1)) / kRows + 1;
     n_sub[1] = (q0 + kRows < L) ? (past + min(q0 + 2 * kRows - 1, L - 1)) / kRows + 1 : 0;
     const int n_kv = max(n_sub[0], n_sub[1]);
+    // Q and the first ring-ful of K/V tiles need no waiting: requested before the block-wide barrier
+    const int n_pre = min(2 * n_kv, C::kSlots);
+    auto request_tile = [&](int idx) {
+        const uint32_t s = idx % C::kSlots;
+        int c1, c2, c3;
+        mbar_arrive_expect_tx(&kv_full[s], C::kTileBytes);
+        order_coords(p.ckv, (idx >> 1) * kRows, kvh, b, c1, c2, c3);
+        const CUtensorMap *tm = (idx & 1) ? &tmap_v : &tmap_k;
+#pragma unroll
+        for (int hf = 0; hf < C::kHalves; ++hf)
+            tma_load_4d(ring + (size_t)s * C::kTileBytes + hf * kHalfBytes, tm, &kv_full[s], hf * 64, c1, c2, c3);
+    };
+    if (producer_lane) {
+        tma_prefetch_desc(&tmap_q);
+        tma_prefetch_desc(&tmap_k);
+        tma_prefetch_desc(&tmap_v);
+        int c1, c2, c3;
+        mbar_arrive_expect_tx(q_full, 2 * C::kTileBytes);
+        order_coords(p.cq, q0, h, b, c1, c2, c3);
+#pragma unroll
+        for (int hf = 0; hf < C::kHalves; ++hf) tma_load_4d(q_smem + hf * kHalfBytes, &tmap_q, q_full, hf * 64, c1, c2, c3);
+        request_tile(0);                                   // K_0 right behind Q_0: the first product needs both
+        order_coords(p.cq, q0 + kRows, h, b, c1, c2, c3);
+#pragma unroll
+        for (int hf = 0; hf < C::kHalves; ++hf)
+            tma_load_4d(q_smem + C::kTileBytes + hf * kHalfBytes, &tmap_q, q_full, hf * 64, c1, c2, c3);
+        for (int idx = 1; idx < n_pre; ++idx) request_tile(idx);
+    }
     if (warp == 9) {
         tmem_alloc(tmem_base_smem, C::kTmemCols);
         tmem_relinquish_alloc_permit();
@@ -200,27 +231,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     if (warp == 8) {
         // ============================================================ TMA producer (+ cache copy)
         if (lane == 0) {
-            tma_prefetch_desc(&tmap_q);
-            tma_prefetch_desc(&tmap_k);
-            tma_prefetch_desc(&tmap_v);
-            int c1, c2, c3;
-            mbar_arrive_expect_tx(q_full, 2 * C::kTileBytes);
-            for (int i = 0; i < 2; ++i) {
-                order_coords(p.cq, q0 + i * kRows, h, b, c1, c2, c3);
-#pragma unroll
-                for (int hf = 0; hf < C::kHalves; ++hf)
-                    tma_load_4d(q_smem + i * C::kTileBytes + hf * kHalfBytes, &tmap_q, q_full, hf * 64, c1, c2, c3);
-            }
-            for (int idx = 0; idx < 2 * n_kv; ++idx) {
-                const int j = idx >> 1;
+            for (int idx = n_pre; idx < 2 * n_kv; ++idx) {
                 const uint32_t s = idx % C::kSlots, ph = (idx / C::kSlots) & 1u;
                 if (!mbar_wait(&kv_empty[s], ph ^ 1u, abort_flag)) break;
-                mbar_arrive_expect_tx(&kv_full[s], C::kTileBytes);
-                order_coords(p.ckv, j * kRows, kvh, b, c1, c2, c3);
-                const CUtensorMap *tm = (idx & 1) ? &tmap_v : &tmap_k;
-#pragma unroll
-                for (int hf = 0; hf < C::kHalves; ++hf)
-                    tma_load_4d(ring + (size_t)s * C::kTileBytes + hf * kHalfBytes, tm, &kv_full[s], hf * 64, c1, c2, c3);
+                request_tile(idx);
             }
         }
         // all loads are issued: the diagonal tiles' slots are in their last phase, the copy may start
