@@ -24,7 +24,7 @@ EXPORTS = (
     "l4l_last_device_error", "l4l_kv_append", "l4l_attn_prefill", "l4l_attn_decode",
     "l4l_attn_decode_static", "l4l_attn_decode_append", "l4l_attn_prefill_chunk", "l4l_rope_kv_append",
     "l4l_kv_append_paged", "l4l_attn_decode_paged", "l4l_kv_append_fp8", "l4l_attn_decode_fp8", "l4l_rglru_scan", "l4l_rglru_workspace_bytes",
-    "l4l_attn_decode_paged_fp8", "l4l_attn_merge",
+    "l4l_attn_decode_paged_fp8", "l4l_attn_merge", "l4l_attn_decode_rope_append",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -97,6 +97,9 @@ def load() -> ctypes.CDLL:
     lib.l4l_attn_decode_paged_fp8.restype = c_int
     lib.l4l_attn_decode_paged_fp8.argtypes = [vp, vp, PagedKV, vp, vp, i32p, c_int, i32p, c_int, c_int, c_int, c_int, c_int,
                                               ctypes.c_float, vp, vp, c_size, vp]
+    lib.l4l_attn_decode_rope_append.restype = c_int
+    lib.l4l_attn_decode_rope_append.argtypes = [vp, vp, KVCache, Tensor4, Tensor4, i32p, c_int, c_int, c_int, c_int, c_int,
+                                                ctypes.c_float, vp, vp, c_int, vp, vp, ctypes.c_float, vp, vp, c_size, vp]
     lib.l4l_attn_merge.restype = c_int
     lib.l4l_attn_merge.argtypes = [vp, vp, c_int, vp, vp, c_int, c_int, c_int, vp]
     lib.l4l_rglru_workspace_bytes.restype = c_size
@@ -472,3 +475,25 @@ def l4l_attn_merge(o_parts, lse_parts, o, lse=None) -> None:
                                None if lse is None else _f32_dev(lse, "lse", (B, Hq)), B, Hq, D, _stream())
     if st != L4L_OK:
         raise L4LError(st, "l4l_attn_merge")
+
+
+def l4l_attn_decode_rope_append(q, o, cache_k, cache_v, k_new, v_new, kv_lens, max_kv_len: int, scale: float, cos, sin,
+                                workspace, q_weight=None, k_weight=None, eps: float = 0.0, lse=None) -> None:
+    """One launch per decode step: rotary embedding (+ optional RMS norm) of q and k_new at position kv_lens - 1, cache
+    update and attention. q,o dense [B,Hq,D] (q is not modified); k_new, v_new [B,1,Hkv,D]; cos, sin CUDA float32
+    [n_pos, D/2]."""
+    _check_bf16_cuda(q, "q")
+    _check_bf16_cuda(o, "o")
+    if not (q.is_contiguous() and o.is_contiguous() and q.dim() == 3 and q.shape == o.shape):
+        raise ValueError("q and o must be dense [B, Hq, D]")
+    B, Hq, D = q.shape
+    Hkv = cache_k.shape[1]
+    n_pos = cos.shape[0]
+    st = load().l4l_attn_decode_rope_append(
+        q.data_ptr(), o.data_ptr(), kv_cache(cache_k, cache_v), tensor4(k_new, "k_new"), tensor4(v_new, "v_new"),
+        _i32_dev(kv_lens, "kv_lens"), int(max_kv_len), B, Hq, Hkv, D, float(scale),
+        _f32_dev(cos, "cos", (n_pos, D // 2)), _f32_dev(sin, "sin", (n_pos, D // 2)), n_pos,
+        _f32_dev(q_weight, "q_weight", (D,)), _f32_dev(k_weight, "k_weight", (D,)), float(eps),
+        None if lse is None else lse.data_ptr(), workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream())
+    if st != L4L_OK:
+        raise L4LError(st, "l4l_attn_decode_rope_append")

@@ -82,6 +82,12 @@ struct DecodeParams {
     unsigned *status;
     // fp8 cache: real value = e4m3 value * scale of its KV head
     const float *k_scale, *v_scale;           // [Hkv]
+    // rotary embedding (+ optional RMS norm) of the step's q and k_new inside the kernel (null: inputs are final);
+    // only together with the fused append. The new token's position is kv_len - 1.
+    const float *rope_cos, *rope_sin;         // [rope_n_pos, D/2]
+    const float *q_weight, *k_weight;         // [D] or null
+    float norm_eps;
+    int rope_n_pos;
     // paged cache (null: contiguous): token t of sequence b lives in page block_table[b * table_stride + t / page_size]
     // at offset t % page_size; the tensor maps then describe the page pool [pages, Hkv, page_size, D]
     const int32_t *block_table;
@@ -107,6 +113,106 @@ __device__ __forceinline__ void order_coords(const TmapCoord &c, int t, int h, i
     c1 = (c.pos_t == 1) ? t : (c.pos_h == 1) ? h : b;
     c2 = (c.pos_t == 2) ? t : (c.pos_h == 2) ? h : b;
     c3 = (c.pos_t == 3) ? t : (c.pos_h == 3) ? h : b;
+}
+
+// ---- rotary embedding (+ optional RMS norm) of the step's own token, inside the decode kernel ----------
+// Same arithmetic as the streaming rope kernel: xn = (x * rinv) * w, y1 = fma(-x2, sin, x1 * cos),
+// y2 = fma(x1, sin, x2 * cos) in fp32, one rounding to bf16. A position outside the table leaves the row as it is.
+
+// The q rows live in the A fragments of the warp MMA: a thread holds, per 16-column k-step, columns 2c, 2c+1
+// (registers 0: row lane/4, 1: row lane/4 + 8) and 2c+8, 2c+9 (registers 2, 3), c = lane % 4. The partner of
+// column i is column i + D/2, i.e. the same register of the k-step D/32 further on: no data leaves the thread.
+template <int D>
+__device__ __forceinline__ void rope_q_fragments(uint32_t (&qf)[D / 16][4], const DecodeParams &p, int pos, int lane)
+{
+    if (pos < 0 || pos >= p.rope_n_pos) return;
+    constexpr int kSteps = D / 16, kHalf = kSteps / 2;
+    const int c = lane & 3;
+    const bool valid[2] = {(lane >> 2) < p.G, (lane >> 2) + 8 < p.G};
+    float rinv[2] = {1.f, 1.f};
+    if (p.q_weight != nullptr) {
+        float ss[2] = {0.f, 0.f};
+#pragma unroll
+        for (int ks = 0; ks < kSteps; ++ks)
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                const float a = __uint_as_float(qf[ks][r] << 16), b = __uint_as_float(qf[ks][r] & 0xffff0000u);
+                ss[r & 1] = fmaf(a, a, fmaf(b, b, ss[r & 1]));
+            }
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            ss[h] += __shfl_xor_sync(0xffffffffu, ss[h], 1);
+            ss[h] += __shfl_xor_sync(0xffffffffu, ss[h], 2);
+            rinv[h] = valid[h] ? rsqrtf(ss[h] * (1.f / D) + p.norm_eps) : 0.f;
+        }
+    }
+    const float *cr = p.rope_cos + (size_t)pos * (D / 2), *sr = p.rope_sin + (size_t)pos * (D / 2);
+#pragma unroll
+    for (int ks = 0; ks < kHalf; ++ks)
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const int col = 16 * ks + 2 * c + ((r >> 1) << 3);               // first-half column of element 0
+            float x1[2] = {__uint_as_float(qf[ks][r] << 16), __uint_as_float(qf[ks][r] & 0xffff0000u)};
+            float x2[2] = {__uint_as_float(qf[ks + kHalf][r] << 16), __uint_as_float(qf[ks + kHalf][r] & 0xffff0000u)};
+            float y1[2], y2[2];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                if (p.q_weight != nullptr) {
+                    x1[e] = x1[e] * rinv[r & 1] * __ldg(p.q_weight + col + e);
+                    x2[e] = x2[e] * rinv[r & 1] * __ldg(p.q_weight + col + e + D / 2);
+                }
+                const float cs = __ldg(cr + col + e), sn = __ldg(sr + col + e);
+                y1[e] = fmaf(-x2[e], sn, x1[e] * cs);
+                y2[e] = fmaf(x1[e], sn, x2[e] * cs);
+            }
+            if (valid[r & 1]) {
+                qf[ks][r] = pack_bf16x2(y1[0], y1[1]);
+                qf[ks + kHalf][r] = pack_bf16x2(y2[0], y2[1]);
+            }
+        }
+}
+
+// The new token's k row as the patching warp holds it: lane l < D/8 has elements [8l, 8l + 8). The partner chunk
+// is D/16 lanes away. Every lane of the warp must call this (shuffles); lanes >= D/8 pass zeros.
+template <int D>
+__device__ __forceinline__ uint4 rope_k_row(uint4 kk, const DecodeParams &p, int pos, int lane)
+{
+    constexpr int kChunks = D / 8, kHalfChunks = D / 16;
+    float x[8];
+    const uint32_t w[4] = {kk.x, kk.y, kk.z, kk.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        x[2 * i] = __uint_as_float(w[i] << 16);
+        x[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+    const bool in_table = pos >= 0 && pos < p.rope_n_pos;
+    if (p.k_weight != nullptr) {
+        float ss = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) ss = fmaf(x[i], x[i], ss);
+#pragma unroll
+        for (int off = 1; off < kChunks; off <<= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+        const float rinv = rsqrtf(ss * (1.f / D) + p.norm_eps);
+        if (lane < kChunks && in_table) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) x[i] = x[i] * rinv * __ldg(p.k_weight + 8 * lane + i);
+        }
+    }
+    float y[8];
+    const bool first = (lane & kHalfChunks) == 0;
+    const int col0 = 8 * (lane & (kHalfChunks - 1));
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float px = __shfl_xor_sync(0xffffffffu, x[i], kHalfChunks);
+        float cs = 1.f, sn = 0.f;
+        if (lane < kChunks && in_table) {
+            cs = __ldg(p.rope_cos + (size_t)pos * (D / 2) + col0 + i);
+            sn = __ldg(p.rope_sin + (size_t)pos * (D / 2) + col0 + i);
+        }
+        y[i] = first ? fmaf(-px, sn, x[i] * cs) : fmaf(px, sn, x[i] * cs);
+    }
+    if (!in_table) return kk;
+    return make_uint4(pack_bf16x2(y[0], y[1]), pack_bf16x2(y[2], y[3]), pack_bf16x2(y[4], y[5]), pack_bf16x2(y[6], y[7]));
 }
 
 template <int D, int W, bool F8>
@@ -648,6 +754,9 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                         qf[ks][3] = v_hi ? qrow_hi[w + 4] : 0u;
                     }
                 }
+                if constexpr (!F8) {
+                    if (p.rope_cos != nullptr) rope_q_fragments<D>(qf, p, mt.kv_len - 1, lane);
+                }
             }
 
             const uint32_t k_tile = smem_u32(stages + (size_t)s * C::kStageBytes);
@@ -661,10 +770,14 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 // cache slot (each slot belongs to exactly one CTA's range and one warp's slice).
                 const int last = row0 + nvalid - 1;
                 constexpr int kChunks = D / 8;
+                uint4 kk = make_uint4(0u, 0u, 0u, 0u), vv = kk;
                 if (lane < kChunks) {
                     const size_t src = (size_t)mt.b * p.new_sb + (size_t)mt.kvh * p.new_sh + lane * 8;
-                    const uint4 kk = __ldg(reinterpret_cast<const uint4 *>(p.k_new + src));
-                    const uint4 vv = __ldg(reinterpret_cast<const uint4 *>(p.v_new + src));
+                    kk = __ldg(reinterpret_cast<const uint4 *>(p.k_new + src));
+                    vv = __ldg(reinterpret_cast<const uint4 *>(p.v_new + src));
+                }
+                if (p.rope_cos != nullptr) kk = rope_k_row<D>(kk, p, mt.kv_len - 1, lane);   // all lanes: shuffles inside
+                if (lane < kChunks) {
                     uint8_t *kt = stages + (size_t)s * C::kStageBytes;
                     const uint32_t off = (lane >> 3) * C::kHalfBytes + swz128(last, lane & 7);
                     *reinterpret_cast<uint4 *>(kt + off) = kk;
@@ -932,8 +1045,9 @@ DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_
 l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, const int32_t *d_kv_lens,
                          int max_kv_len, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
                          void *workspace, const DecodePlan &plan, cudaStream_t stream, const l4l_tensor4 *k_new,
-                         const l4l_tensor4 *v_new, const PagedTable *paged, const Fp8Scales *fp8)
+                         const l4l_tensor4 *v_new, const PagedTable *paged, const Fp8Scales *fp8, const RopeArgs *rope)
 {
+    if (rope && (!k_new || !v_new || fp8 || paged)) return L4L_ERR_UNSUPPORTED;   // only with the plain fused append
     // fp8: cache.k / cache.v point at e4m3 bytes, the strides count bytes (= elements)
     if (fp8 && (D != 128 || k_new || v_new)) return L4L_ERR_UNSUPPORTED;
     const int esz = fp8 ? 1 : 2;
@@ -988,6 +1102,12 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         p.max_kv_len = max_kv_len;
         p.k_new = p.v_new = nullptr;
         p.new_sb = p.new_sh = 0;
+        p.rope_cos = rope ? rope->cos : nullptr;
+        p.rope_sin = rope ? rope->sin : nullptr;
+        p.q_weight = rope ? rope->q_weight : nullptr;
+        p.k_weight = rope ? rope->k_weight : nullptr;
+        p.norm_eps = rope ? rope->eps : 0.f;
+        p.rope_n_pos = rope ? rope->n_pos : 0;
         p.k_scale = fp8 ? fp8->k_scale : nullptr;
         p.v_scale = fp8 ? fp8->v_scale : nullptr;
         p.block_table = paged ? paged->block_table + (size_t)b0 * paged->table_stride : nullptr;
@@ -1104,5 +1224,5 @@ extern "C" l4l_status l4l_attn_decode_static(const void *q, void *o, l4l_kv_cach
     const size_t zero_bytes = kStatusBytes + kTicketBytes;
     if (cudaMemsetAsync(scratch, 0, zero_bytes, s) != cudaSuccess) return L4L_ERR_CUDA;
     return launch_decode(q, o, cache, d_kv_lens, max_kv_len, B, Hq, Hkv, head_dim, scale, d_lse, scratch, plan, s,
-                         nullptr, nullptr, nullptr, nullptr);
+                         nullptr, nullptr, nullptr, nullptr, nullptr);
 }

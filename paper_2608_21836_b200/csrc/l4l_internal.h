@@ -57,13 +57,22 @@ struct Fp8Scales {
     const float *k_scale, *v_scale;   // device, [Hkv]
 };
 
+// Rotary embedding (+ optional RMS norm) of the step's q and k_new inside the decode kernel.
+struct RopeArgs {
+    const float *cos, *sin;           // device, [n_pos, D/2]
+    const float *q_weight, *k_weight; // device [D] or null
+    float eps;
+    int n_pos;
+};
+
 // With `paged`, `cache` describes the page pool: stride_b = stride between pages, max_len = page size.
 // With `fp8`, cache.k / cache.v hold e4m3 bytes and the strides count bytes.
 l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, const int32_t *d_kv_lens,
                          int max_kv_len, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
                          void *workspace, const DecodePlan &plan, cudaStream_t stream,
                          const l4l_tensor4 *k_new = nullptr, const l4l_tensor4 *v_new = nullptr,
-                         const PagedTable *paged = nullptr, const Fp8Scales *fp8 = nullptr);
+                         const PagedTable *paged = nullptr, const Fp8Scales *fp8 = nullptr,
+                         const RopeArgs *rope = nullptr);
 
 l4l_status launch_rope_kv_append(const l4l_tensor4 &q, const l4l_tensor4 &k_new, const l4l_tensor4 &v_new,
                                  const l4l_kv_cache &cache, const int32_t *d_pos, const int32_t *d_n_new, int T, int B,

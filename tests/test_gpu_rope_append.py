@@ -145,3 +145,46 @@ def test_rope_append_rejects_bad_arguments():
         l4l.l4l_rope_kv_append(q, k, k.clone(), ck, ck.clone(), pos, None, cos, sin.cuda())     # host table
     with pytest.raises(l4l.L4LError):
         l4l.l4l_rope_kv_append(q, k, k.clone(), ck, ck.clone(), pos, None, cos.cuda(), sin.cuda(), eps=-1.0)
+
+
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("Hq,Hkv", [(8, 2), (4, 4), (16, 1)])
+@pytest.mark.parametrize("norm", [False, True])
+def test_decode_step_with_rope_and_append_in_one_launch(D, Hq, Hkv, norm):
+    """l4l_attn_decode_rope_append against the oracle chain rope -> append -> decode, over several steps, with lengths
+    that put the new token at the start, in the middle and at the end of tiles."""
+    B, Lmax, steps = 6, 700, 3
+    lens = np.array([1, 16, 17, 128, 129, 600], np.int32)        # kv_len INCLUDING the new token at the first step
+    g = torch.Generator().manual_seed(900 + D + Hq + norm)
+    ck = torch.randn(B, Hkv, Lmax, D, generator=g).to(torch.bfloat16)
+    cv = torch.randn(B, Hkv, Lmax, D, generator=g).to(torch.bfloat16)
+    cos, sin = make_rope_tables(Lmax, D)
+    qw = (torch.rand(D, generator=g) + 0.5) if norm else None
+    kw = (torch.rand(D, generator=g) + 0.5) if norm else None
+    eps = 1e-6 if norm else 0.0
+    scale = 1.0 / math.sqrt(D)
+    dck, dcv = ck.cuda(), cv.cuda()
+    ock, ocv = orc.bits(ck), orc.bits(cv)
+    ws = l4l.new_workspace(l4l.L4L_OP_DECODE, B, Hq, Hkv, D, Lmax)
+    dcos, dsin = cos.cuda(), sin.cuda()
+    for s in range(steps):
+        q = torch.randn(B, Hq, D, generator=g).to(torch.bfloat16)
+        kn = torch.randn(B, 1, Hkv, D, generator=g).to(torch.bfloat16)
+        vn = torch.randn(B, 1, Hkv, D, generator=g).to(torch.bfloat16)
+        cur = lens + s
+        oq, ock, ocv, _, _ = orc.rope_kv_append(q.view(B, 1, Hq, D), kn, vn, ock, ocv, cur - 1, None, cos.numpy(),
+                                                sin.numpy(), None if qw is None else qw.numpy(),
+                                                None if kw is None else kw.numpy(), eps)
+        ref, _ = orc.decode(oq[:, 0], ock, ocv, cur, scale)
+        dq = q.cuda()
+        q_before = dq.clone()
+        o = torch.zeros(B, Hq, D, dtype=torch.bfloat16, device="cuda")
+        l4l.l4l_attn_decode_rope_append(dq, o, dck, dcv, kn.cuda(), vn.cuda(), torch.from_numpy(cur).cuda(), Lmax, scale,
+                                        dcos, dsin, ws, q_weight=None if qw is None else qw.cuda(),
+                                        k_weight=None if kw is None else kw.cuda(), eps=eps)
+        torch.cuda.synchronize()
+        assert l4l.l4l_last_device_error(ws) == 0
+        assert bits_equal(dq, q_before)                                          # q is read only
+        assert_close_to_oracle(o.cpu(), ref, f"rope + append + decode, step {s}")
+    assert_bf16_close(dck, ock, "cache k after the fused steps")
+    assert np.array_equal(orc.bits(dcv.cpu()), ocv)
