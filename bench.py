@@ -323,6 +323,19 @@ def run_ours(args, rank, world):
     rope_bytes = 2 * q.numel() * 2 + 2 * (k.numel() + v.numel()) * 2       # q read + written, k/v read, cache written
     t_chunk = timed(lambda: l4l.l4l_attn_prefill_chunk(q, o, pk, pv, zeros_b, plens, wp.scale, ws_p), 5)
     t_fused = timed(lambda: l4l.l4l_attn_decode_append(dq, do, dck, dcv, dkn, dvn, dlen, Lmax, wd.scale, ws_d), 20)
+    # the whole decode step of a layer: rope + norm of the new token's q and k, append, attention: one launch, against
+    # the three launches rope_kv_append (T = 1) + decode
+    cos_d, sin_d = wl.make_rope_tables(Lmax, D)
+    cos_d, sin_d = cos_d.to(dev), sin_d.to(dev)
+    t_step1 = timed(lambda: l4l.l4l_attn_decode_rope_append(dq, do, dck, dcv, dkn, dvn, dlen, Lmax, wd.scale, cos_d, sin_d,
+                                                            ws_d, q_weight=gamma, k_weight=gamma, eps=1e-6), 20)
+    dq4 = dq.view(Bd, 1, Hq, D)
+
+    def three_launches():
+        l4l.l4l_rope_kv_append(dq4, dkn, dvn, dck, dcv, dpos, None, cos_d, sin_d, gamma, gamma, 1e-6)
+        l4l.l4l_attn_decode(dq, do, dck, dcv, dlen, Lmax, wd.scale, ws_d)
+
+    t_step3 = timed(three_launches, 20)
     # decode over a paged cache: the same batch cut into 64-token pages scattered over a pool, three pools in rotation
     page = 64
     n_per = Lmax // page
@@ -433,8 +446,9 @@ def run_ours(args, rank, world):
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
 
     # ---- max over ranks
-    total_ms, e2e_ms, t_pre, t_dec, t_app, t_dec_b2b, t_rope, t_chunk, t_fused, t_paged, t_fp8, t_rglru = max_over_ranks(
-        [total_ms, e2e_ms, t_pre, t_dec, t_app, t_dec_b2b, t_rope, t_chunk, t_fused, t_paged, t_fp8, t_rglru], world, dev)
+    total_ms, e2e_ms, t_pre, t_dec, t_app, t_dec_b2b, t_rope, t_chunk, t_fused, t_paged, t_fp8, t_rglru, t_step1, t_step3 = max_over_ranks(
+        [total_ms, e2e_ms, t_pre, t_dec, t_app, t_dec_b2b, t_rope, t_chunk, t_fused, t_paged, t_fp8, t_rglru, t_step1, t_step3], world,
+        dev)
     if rank != 0:
         return
 
@@ -478,6 +492,7 @@ def run_ours(args, rank, world):
                                     "bytes": rope_bytes},
             "prefill_from_cache": {"ms": t_chunk, "tflops": pre_flops / (t_chunk * 1e-3) / 1e12},
             "decode_with_fused_append": {"us": t_fused * 1e3, "kv_gbs": dec_bytes / (t_fused * 1e-3) / 1e9},
+            "decode_step_rope_norm_append_attention": {"one_launch_us": t_step1 * 1e3, "two_launches_us": t_step3 * 1e3},
             "decode_paged_64": {"us": t_paged * 1e3, "kv_gbs": dec_bytes / (t_paged * 1e-3) / 1e9},
             "rglru_scan_B4_T8192_W2560": {"us": t_rglru * 1e3, "gbs": rglru_bytes / (t_rglru * 1e-3) / 1e9,
                                           "frac_of_measured_hbm": rglru_bytes / (t_rglru * 1e-3) / 1e9 / peaks["hbm_gbs"],

@@ -475,6 +475,7 @@ l4l_status l4l_attn_decode_rope_append(const void *q, void *o, l4l_kv_cache cach
     if (!cache_ok(cache) || max_kv_len < 0 || max_kv_len > cache.max_len) return L4L_ERR_INVALID_ARG;
     if (!tensor4_ok(k_new) || !tensor4_ok(v_new)) return L4L_ERR_INVALID_ARG;
     if (!d_cos || !d_sin || n_pos < 0 || !(norm_eps >= 0.f)) return L4L_ERR_INVALID_ARG;
+    if (!aligned16(d_cos) || !aligned16(d_sin)) return L4L_ERR_INVALID_ARG;      // rows are fetched with bulk copies
     if (!workspace || ws_bytes < kStatusBytes) return L4L_ERR_WORKSPACE;
     if (B == 0) return L4L_OK;
     const DecodePlan plan = plan_decode(B, Hq, Hkv, head_dim, max_kv_len, ws_bytes);

@@ -102,7 +102,10 @@ size_t decode_smem_bytes(int G, int nsplit)
 {
     using C = DecodeCfg<D, W, F8>;
     size_t comb = (size_t)W * G * (D + 4) * sizeof(float) + (size_t)((G * nsplit + 3) & ~3) * sizeof(float);
-    return 1024 /*alignment slack*/ + (size_t)C::kStages * (C::kStageBytes + (size_t)G * D * 2) + comb +
+    // per stage: the K/V tiles, the piece's query rows and (rope fused into the step) the cos / sin rows of the
+    // new token's position; per consumer warp: its private copy of those rows for the piece it is working on
+    return 1024 /*alignment slack*/ + (size_t)C::kStages * (C::kStageBytes + (size_t)G * D * 2 + D * 4) + (size_t)W * D * 4 + 2 * D * 4 +
+           comb +
            C::kStages * sizeof(TileMeta) +
            sizeof(PieceMeta) + (2 * C::kStages + 2) * sizeof(uint64_t) + (kMaxB + 1) * sizeof(int) + 64 +
            kPostRing * sizeof(PieceMeta);
@@ -118,14 +121,15 @@ __device__ __forceinline__ void order_coords(const TmapCoord &c, int t, int h, i
 // ---- rotary embedding (+ optional RMS norm) of the step's own token, inside the decode kernel ----------
 // Same arithmetic as the streaming rope kernel: xn = (x * rinv) * w, y1 = fma(-x2, sin, x1 * cos),
 // y2 = fma(x1, sin, x2 * cos) in fp32, one rounding to bf16. A position outside the table leaves the row as it is.
+// The cos | sin rows of the position come from shared memory: the producer fetches them with the piece's first tile.
 
 // The q rows live in the A fragments of the warp MMA: a thread holds, per 16-column k-step, columns 2c, 2c+1
 // (registers 0: row lane/4, 1: row lane/4 + 8) and 2c+8, 2c+9 (registers 2, 3), c = lane % 4. The partner of
 // column i is column i + D/2, i.e. the same register of the k-step D/32 further on: no data leaves the thread.
 template <int D>
-__device__ __forceinline__ void rope_q_fragments(uint32_t (&qf)[D / 16][4], const DecodeParams &p, int pos, int lane)
+__device__ __forceinline__ void rope_q_fragments(uint32_t (&qf)[D / 16][4], const DecodeParams &p, const float *cos_sin,
+                                                 const float *weight, int lane)
 {
-    if (pos < 0 || pos >= p.rope_n_pos) return;
     constexpr int kSteps = D / 16, kHalf = kSteps / 2;
     const int c = lane & 3;
     const bool valid[2] = {(lane >> 2) < p.G, (lane >> 2) + 8 < p.G};
@@ -146,7 +150,7 @@ __device__ __forceinline__ void rope_q_fragments(uint32_t (&qf)[D / 16][4], cons
             rinv[h] = valid[h] ? rsqrtf(ss[h] * (1.f / D) + p.norm_eps) : 0.f;
         }
     }
-    const float *cr = p.rope_cos + (size_t)pos * (D / 2), *sr = p.rope_sin + (size_t)pos * (D / 2);
+    const float *cr = cos_sin, *sr = cos_sin + D / 2;              // shared memory: cos | sin of the position
 #pragma unroll
     for (int ks = 0; ks < kHalf; ++ks)
 #pragma unroll
@@ -158,10 +162,10 @@ __device__ __forceinline__ void rope_q_fragments(uint32_t (&qf)[D / 16][4], cons
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
                 if (p.q_weight != nullptr) {
-                    x1[e] = x1[e] * rinv[r & 1] * __ldg(p.q_weight + col + e);
-                    x2[e] = x2[e] * rinv[r & 1] * __ldg(p.q_weight + col + e + D / 2);
+                    x1[e] = x1[e] * rinv[r & 1] * weight[col + e];
+                    x2[e] = x2[e] * rinv[r & 1] * weight[col + e + D / 2];
                 }
-                const float cs = __ldg(cr + col + e), sn = __ldg(sr + col + e);
+                const float cs = cr[col + e], sn = sr[col + e];
                 y1[e] = fmaf(-x2[e], sn, x1[e] * cs);
                 y2[e] = fmaf(x1[e], sn, x2[e] * cs);
             }
@@ -175,7 +179,8 @@ __device__ __forceinline__ void rope_q_fragments(uint32_t (&qf)[D / 16][4], cons
 // The new token's k row as the patching warp holds it: lane l < D/8 has elements [8l, 8l + 8). The partner chunk
 // is D/16 lanes away. Every lane of the warp must call this (shuffles); lanes >= D/8 pass zeros.
 template <int D>
-__device__ __forceinline__ uint4 rope_k_row(uint4 kk, const DecodeParams &p, int pos, int lane)
+__device__ __forceinline__ uint4 rope_k_row(uint4 kk, const DecodeParams &p, const float *cos_sin, const float *weight,
+                                            bool in_table, int lane)
 {
     constexpr int kChunks = D / 8, kHalfChunks = D / 16;
     float x[8];
@@ -185,7 +190,6 @@ __device__ __forceinline__ uint4 rope_k_row(uint4 kk, const DecodeParams &p, int
         x[2 * i] = __uint_as_float(w[i] << 16);
         x[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
     }
-    const bool in_table = pos >= 0 && pos < p.rope_n_pos;
     if (p.k_weight != nullptr) {
         float ss = 0.f;
 #pragma unroll
@@ -195,7 +199,7 @@ __device__ __forceinline__ uint4 rope_k_row(uint4 kk, const DecodeParams &p, int
         const float rinv = rsqrtf(ss * (1.f / D) + p.norm_eps);
         if (lane < kChunks && in_table) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) x[i] = x[i] * rinv * __ldg(p.k_weight + 8 * lane + i);
+            for (int i = 0; i < 8; ++i) x[i] = x[i] * rinv * weight[8 * lane + i];
         }
     }
     float y[8];
@@ -206,8 +210,8 @@ __device__ __forceinline__ uint4 rope_k_row(uint4 kk, const DecodeParams &p, int
         const float px = __shfl_xor_sync(0xffffffffu, x[i], kHalfChunks);
         float cs = 1.f, sn = 0.f;
         if (lane < kChunks && in_table) {
-            cs = __ldg(p.rope_cos + (size_t)pos * (D / 2) + col0 + i);
-            sn = __ldg(p.rope_sin + (size_t)pos * (D / 2) + col0 + i);
+            cs = cos_sin[col0 + i];
+            sn = cos_sin[D / 2 + col0 + i];
         }
         y[i] = first ? fmaf(-px, sn, x[i] * cs) : fmaf(px, sn, x[i] * cs);
     }
@@ -229,9 +233,13 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     uint8_t *smem = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
 
     uint8_t *stages = smem;
-    uint8_t *q_slots = stages + (size_t)C::kStages * C::kStageBytes;     // per stage: the piece's G query rows
+    uint8_t *q_slots = stages + (size_t)C::kStages * C::kStageBytes;     // per stage: the piece's G query rows ...
     const uint32_t q_bytes = (uint32_t)p.G * D * 2;
-    float *comb = reinterpret_cast<float *>(q_slots + (size_t)C::kStages * q_bytes);
+    constexpr uint32_t kRopeBytes = D * 4;                               // ... and cos | sin of the new token's position
+    const uint32_t q_stride = q_bytes + kRopeBytes;
+    float *rope_priv = reinterpret_cast<float *>(q_slots + (size_t)C::kStages * q_stride);   // [W][D] per-warp copy
+    float *norm_w = rope_priv + (size_t)W * D;                           // q_weight | k_weight (when given)
+    float *comb = norm_w + 2 * D;
     constexpr int kPitch = D + 4;            // floats per row of `comb`: O[D], max, sum, pad (16-byte rows)
     constexpr int kVec = D / 4;
     const int comb_floats = kConsumerWarps * p.G * kPitch;
@@ -275,6 +283,12 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     // next kernel in the stream may begin its own prologue as soon as this grid's CTAs retire.
     grid_dependency_wait();
     grid_launch_dependents();
+    if (p.rope_cos != nullptr) {
+        for (int i = threadIdx.x; i < D; i += blockDim.x) {
+            norm_w[i] = p.q_weight ? __ldg(p.q_weight + i) : 1.f;
+            norm_w[D + i] = p.k_weight ? __ldg(p.k_weight + i) : 1.f;
+        }
+    }
     __syncthreads();
 
     if (warp == kProducerWarp) {
@@ -356,10 +370,18 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     const int rem = len - tile * kTileT;
                     const int groups = rem >= kTileT ? kTileT / 16 : (rem + 15) / 16;
                     const uint32_t kv_bytes = rem >= kTileT ? C::kStageBytes : (uint32_t)groups * 16u * 128u * C::kHalves * 2u;
-                    mbar_arrive_expect_tx(&full[s], kv_bytes + (first ? q_bytes : 0u));
+                    // with the rope fused into the step, the piece's first tile also brings the cos / sin rows of
+                    // the new token's position (kv_len - 1), if the table has it
+                    const bool with_rope = first && p.rope_cos != nullptr && len - 1 < p.rope_n_pos;
+                    mbar_arrive_expect_tx(&full[s], kv_bytes + (first ? q_bytes : 0u) + (with_rope ? kRopeBytes : 0u));
                     if (first)
-                        bulk_load_1d(q_slots + (size_t)s * q_bytes, p.q + ((size_t)b * p.Hq + (size_t)kvh * p.G) * D,
+                        bulk_load_1d(q_slots + (size_t)s * q_stride, p.q + ((size_t)b * p.Hq + (size_t)kvh * p.G) * D,
                                      q_bytes, &full[s]);
+                    if (with_rope) {
+                        uint8_t *rs = q_slots + (size_t)s * q_stride + q_bytes;
+                        bulk_load_1d(rs, p.rope_cos + (size_t)(len - 1) * (D / 2), kRopeBytes / 2, &full[s]);
+                        bulk_load_1d(rs + kRopeBytes / 2, p.rope_sin + (size_t)(len - 1) * (D / 2), kRopeBytes / 2, &full[s]);
+                    }
                     uint8_t *dst = stages + (size_t)s * C::kStageBytes;
                     // With a paged cache a full tile is one box if a page holds whole tiles, else one box per
                     // page (tmap_k / tmap_v then have page-sized boxes); the last tile of a sequence comes in
@@ -733,7 +755,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     k_sc = __ldg(p.k_scale + mt.kvh);
                     v_sc = __ldg(p.v_scale + mt.kvh);
                 }
-                const uint32_t *qs = reinterpret_cast<const uint32_t *>(q_slots + (size_t)s * q_bytes);
+                const uint32_t *qs = reinterpret_cast<const uint32_t *>(q_slots + (size_t)s * q_stride);
                 const uint32_t *qrow_lo = qs + (size_t)r_lo * D / 2;
                 const uint32_t *qrow_hi = qs + (size_t)r_hi * D / 2;
                 const bool v_lo = r_lo < p.G, v_hi = r_hi < p.G;
@@ -755,7 +777,15 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     }
                 }
                 if constexpr (!F8) {
-                    if (p.rope_cos != nullptr) rope_q_fragments<D>(qf, p, mt.kv_len - 1, lane);
+                    if (p.rope_cos != nullptr && mt.kv_len - 1 < p.rope_n_pos) {
+                        // keep this piece's cos | sin rows in the warp's own scratch (the stage is recycled long
+                        // before the tile with the new token arrives), then rotate the q fragments in registers
+                        float *mine = rope_priv + (size_t)warp * D;
+                        const float4 *src = reinterpret_cast<const float4 *>(q_slots + (size_t)s * q_stride + q_bytes);
+                        for (int i = lane; i < D / 4; i += 32) reinterpret_cast<float4 *>(mine)[i] = src[i];
+                        __syncwarp();
+                        rope_q_fragments<D>(qf, p, mine, norm_w, lane);
+                    }
                 }
             }
 
@@ -776,7 +806,8 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     kk = __ldg(reinterpret_cast<const uint4 *>(p.k_new + src));
                     vv = __ldg(reinterpret_cast<const uint4 *>(p.v_new + src));
                 }
-                if (p.rope_cos != nullptr) kk = rope_k_row<D>(kk, p, mt.kv_len - 1, lane);   // all lanes: shuffles inside
+                if (p.rope_cos != nullptr)                                      // all lanes: shuffles inside
+                    kk = rope_k_row<D>(kk, p, rope_priv + (size_t)warp * D, norm_w + D, mt.kv_len - 1 < p.rope_n_pos, lane);
                 if (lane < kChunks) {
                     uint8_t *kt = stages + (size_t)s * C::kStageBytes;
                     const uint32_t off = (lane >> 3) * C::kHalfBytes + swz128(last, lane & 7);
