@@ -1,0 +1,553 @@
+// Decode attention for small batches: one thread-block cluster per (sequence, KV head).
+//
+// When the whole problem is a handful of tiles per SM, a decode step is a chain of latencies, not a stream:
+// the split kernel's workspace round trips (partials -> fence -> ticket -> partial loads) then cost more than
+// the attention itself. Here the CTAs that share a (sequence, KV head) form a cluster of C = 1, 2, 4 or 8 CTAs: CTA
+// `rank` streams the rank-th share of the sequence's 128-token tiles, the eight consumer warps merge their
+// results in shared memory, and after ONE cluster barrier every CTA reads the C partials straight out of its
+// peers' shared memory (distributed shared memory) and writes its 1/C of the output rows. No workspace, no
+// atomics, no global-memory fence.
+//
+//   warp 8      TMA producer: the group's query rows with the first tile, then K/V tiles (128-byte swizzle)
+//               through a small ring; the last tile of a sequence in 16-token groups
+//   warps 0-7   16 tokens of every tile each, all query heads of the KV group as the M dimension of the warp
+//               MMAs (the same building blocks as the split kernel), fused append of the step's new token
+//
+// bf16 cache, contiguous or paged. The fp8 cache and the rope-fused step stay on the split kernel.
+#include <cstdlib>
+
+#include "l4l_internal.h"
+#include "l4l_warp_attn.cuh"
+
+namespace l4l {
+
+namespace {
+
+constexpr int kW = 8;                          // consumer warps
+constexpr int kTileT = 16 * kW;                // tokens per tile
+constexpr int kThreads = (kW + 1) * 32;
+constexpr int kMaxCluster = 8;             // the portable limit; wider clusters schedule in too few places to pay
+constexpr uint32_t kHalfBytes = kTileT * 128;  // [tile tokens][64 bf16], swizzled
+
+template <int D>
+struct ClusterCfg {
+    static constexpr int kHalves = D / 64;
+    static constexpr uint32_t kTileBytes = kHalves * kHalfBytes;     // one of K or V
+    static constexpr uint32_t kStageBytes = 2 * kTileBytes;
+    static constexpr int kPitch = D + 4;                             // floats per row: O[D], max, sum, pad
+    static constexpr int kMaxStages = (D == 128) ? 3 : 6;
+};
+
+struct ClusterParams {
+    const __nv_bfloat16 *q;   // [B, Hq, D]
+    __nv_bfloat16 *o;         // [B, Hq, D]
+    float *lse;               // [B, Hq] or null
+    const int32_t *kv_lens;   // [B]
+    const __nv_bfloat16 *k_new, *v_new;       // fused append (null: none): element (b, kv head, d) at b*new_sb + kvh*new_sh + d
+    int64_t new_sb, new_sh;
+    __nv_bfloat16 *cache_k, *cache_v;
+    int64_t c_sb, c_sh, c_st;
+    unsigned *status;
+    const int32_t *block_table;               // paged cache (null: contiguous)
+    int table_stride, page_size, page_shift;
+    int B, Hq, Hkv, G, C, max_kv_len, stages;
+    float scale_log2e;
+    TmapCoord coord;
+};
+
+template <int D>
+size_t cluster_smem_bytes(int G, int stages)
+{
+    using C = ClusterCfg<D>;
+    return 1024 /*alignment slack*/ + (size_t)stages * C::kStageBytes + (size_t)G * D * 2 +
+           (size_t)(kW + 1) * G * C::kPitch * sizeof(float) + 2 * C::kMaxStages * sizeof(uint64_t) + 64;
+}
+
+__device__ __forceinline__ void order_coords(const TmapCoord &c, int t, int h, int b, int &c1, int &c2, int &c3)
+{
+    c1 = (c.pos_t == 1) ? t : (c.pos_h == 1) ? h : b;
+    c2 = (c.pos_t == 2) ? t : (c.pos_h == 2) ? h : b;
+    c3 = (c.pos_t == 3) ? t : (c.pos_h == 3) ? h : b;
+}
+
+// Cluster-wide barrier in two halves, so that work that needs no peer can sit between them. Hardware
+// barrier (no spinning): every thread of every CTA of the cluster executes both halves exactly once per use.
+__device__ __forceinline__ void cluster_arrive()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait()
+{
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+// Address of the same shared-memory location in the CTA of the given rank of this cluster.
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t smem_addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t addr)
+{
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                 : "r"(addr)
+                 : "memory");
+    return v;
+}
+__device__ __forceinline__ float2 ld_cluster_f2(uint32_t addr)
+{
+    float2 v;
+    asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
+    return v;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1)
+decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
+                      const __grid_constant__ CUtensorMap tmap_k16, const __grid_constant__ CUtensorMap tmap_v16,
+                      const ClusterParams p)
+{
+    using C = ClusterCfg<D>;
+    constexpr int kPitch = C::kPitch, kVec = D / 4;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    // the same offset in every CTA of the cluster (the dynamic segment starts at the same shared address)
+    uint8_t *smem = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
+    uint8_t *stages = smem;
+    uint8_t *q_smem = stages + (size_t)p.stages * C::kStageBytes;
+    const uint32_t q_bytes = (uint32_t)p.G * D * 2;
+    float *comb = reinterpret_cast<float *>(q_smem + q_bytes);       // [kW][G][kPitch] per-warp results
+    float *part = comb + (size_t)kW * p.G * kPitch;                  // [G][kPitch] this CTA's merged partial
+    uint64_t *full = reinterpret_cast<uint64_t *>(part + (size_t)p.G * kPitch);
+    uint64_t *empty = full + C::kMaxStages;
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(empty + C::kMaxStages);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int rank = blockIdx.x;                 // cluster = the gridDim.x CTAs of one blockIdx.y
+    const int unit = blockIdx.y;
+    const int b = unit / p.Hkv, kvh = unit % p.Hkv;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], kW);
+        }
+        *abort_flag = 0;
+        fence_barrier_init();
+        fence_proxy_async_smem();
+    }
+    if (warp == kW && lane == 0) {
+        tma_prefetch_desc(&tmap_k);
+        tma_prefetch_desc(&tmap_v);
+        tma_prefetch_desc(&tmap_k16);
+        tma_prefetch_desc(&tmap_v16);
+    }
+    // Programmatic dependent launch: everything above overlaps the tail of the previous kernel of the stream
+    grid_dependency_wait();
+    grid_launch_dependents();
+    int len = __ldg(p.kv_lens + b);
+    len = len < 0 ? 0 : (len > p.max_kv_len ? p.max_kv_len : len);
+    __syncthreads();
+
+    // this CTA's share of the sequence's tiles: as even as whole tiles allow
+    const int tiles_b = (len + kTileT - 1) / kTileT;
+    const int t_begin = (int)(((long long)rank * tiles_b) / p.C);
+    const int t_end = (int)(((long long)(rank + 1) * tiles_b) / p.C);
+    const int n_mine = t_end - t_begin;
+
+    if (warp == kW) {
+        // ------------------------------------------------------------------ producer
+        if (lane == 0) {
+            const bool paged = p.block_table != nullptr;
+            const int32_t *pages = paged ? p.block_table + (size_t)b * p.table_stride : nullptr;
+            for (int it = 0; it < n_mine; ++it) {
+                const int tile = t_begin + it;
+                const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
+                if (!mbar_wait(&empty[s], ph ^ 1u, abort_flag)) break;
+                const int rem = len - tile * kTileT;
+                // the last tile of a sequence is fetched in 16-token groups: (almost) nothing past the end is read
+                const int groups = rem >= kTileT ? kTileT / 16 : (rem + 15) / 16;
+                const uint32_t kv_bytes = rem >= kTileT ? C::kStageBytes : (uint32_t)groups * 16u * 128u * C::kHalves * 2u;
+                mbar_arrive_expect_tx(&full[s], kv_bytes + (it == 0 ? q_bytes : 0u));
+                if (it == 0)
+                    bulk_load_1d(q_smem, p.q + ((size_t)b * p.Hq + (size_t)kvh * p.G) * D, q_bytes, &full[s]);
+                uint8_t *dst = stages + (size_t)s * C::kStageBytes;
+                int c1, c2, c3;
+                // a full tile is one box (or one box per page when pages are smaller than the tile); neither a
+                // box nor a 16-token group straddles pages: page sizes are powers of two >= 16
+                const int box_rows = rem >= kTileT ? ((paged && p.page_size < kTileT) ? p.page_size : kTileT) : 16;
+                const int n_box = rem >= kTileT ? kTileT / box_rows : groups;
+                const CUtensorMap *tk = rem >= kTileT ? &tmap_k : &tmap_k16;
+                const CUtensorMap *tv = rem >= kTileT ? &tmap_v : &tmap_v16;
+                int page_of[kTileT / 16];                            // looked up together: independent loads
+#pragma unroll
+                for (int bx = 0; bx < kTileT / 16; ++bx)
+                    page_of[bx] = (paged && bx < n_box) ? __ldg(pages + ((tile * kTileT + bx * box_rows) >> p.page_shift)) : b;
+#pragma unroll
+                for (int bx = 0; bx < kTileT / 16; ++bx) {
+                    if (bx >= n_box) break;
+                    int tt = tile * kTileT + bx * box_rows;
+                    if (paged) tt &= p.page_size - 1;
+                    order_coords(p.coord, tt, kvh, page_of[bx], c1, c2, c3);
+                    uint8_t *db = dst + bx * box_rows * 128;          // whole 8-row groups: the swizzle phase is kept
+#pragma unroll
+                    for (int hf = 0; hf < C::kHalves; ++hf) {
+                        tma_load_4d(db + hf * kHalfBytes, tk, &full[s], hf * 64, c1, c2, c3);
+                        tma_load_4d(db + C::kTileBytes + hf * kHalfBytes, tv, &full[s], hf * 64, c1, c2, c3);
+                    }
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ consumer warps
+        WarpAttnState<D> st;
+        st.reset();
+        uint32_t qf[D / 16][4];
+        const int r_lo = lane >> 2, r_hi = r_lo + 8;    // query heads of the group held in rows lane/4, lane/4 + 8
+        for (int it = 0; it < n_mine; ++it) {
+            const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
+            if (!mbar_wait(&full[s], ph, abort_flag)) break;
+            if (it == 0) {
+                const uint32_t *qs = reinterpret_cast<const uint32_t *>(q_smem);
+                const uint32_t *qrow_lo = qs + (size_t)r_lo * D / 2;
+                const uint32_t *qrow_hi = qs + (size_t)r_hi * D / 2;
+                const bool v_lo = r_lo < p.G, v_hi = r_hi < p.G;
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const int w = ks * 8 + (lane & 3);               // 32-bit word index in the row
+                    qf[ks][0] = v_lo ? qrow_lo[w] : 0u;
+                    qf[ks][1] = v_hi ? qrow_hi[w] : 0u;
+                    qf[ks][2] = v_lo ? qrow_lo[w + 4] : 0u;
+                    qf[ks][3] = v_hi ? qrow_hi[w + 4] : 0u;
+                }
+            }
+            const int t0 = (t_begin + it) * kTileT;
+            const uint32_t k_tile = smem_u32(stages + (size_t)s * C::kStageBytes);
+            const uint32_t v_tile = k_tile + C::kTileBytes;
+            const int row0 = warp * 16;
+            const int nvalid = len - (t0 + row0);                    // valid tokens in this warp's slice
+            bool wrote_smem = false;
+            if (p.k_new != nullptr && nvalid > 0 && nvalid <= 16) {
+                // fused append: this slice holds the sequence's newest token. Its K/V arrive from the caller, not
+                // from the cache: patch the tile in shared memory and write the cache slot (exactly one warp of
+                // one CTA owns it)
+                const int last = row0 + nvalid - 1;
+                constexpr int kChunks = D / 8;
+                if (lane < kChunks) {
+                    const size_t src = (size_t)b * p.new_sb + (size_t)kvh * p.new_sh + lane * 8;
+                    const uint4 kk = __ldg(reinterpret_cast<const uint4 *>(p.k_new + src));
+                    const uint4 vv = __ldg(reinterpret_cast<const uint4 *>(p.v_new + src));
+                    uint8_t *kt = stages + (size_t)s * C::kStageBytes;
+                    const uint32_t off = (lane >> 3) * kHalfBytes + swz128(last, lane & 7);
+                    *reinterpret_cast<uint4 *>(kt + off) = kk;
+                    *reinterpret_cast<uint4 *>(kt + C::kTileBytes + off) = vv;
+                    const size_t dst = (size_t)b * p.c_sb + (size_t)kvh * p.c_sh + (size_t)(len - 1) * p.c_st + lane * 8;
+                    *reinterpret_cast<uint4 *>(p.cache_k + dst) = kk;
+                    *reinterpret_cast<uint4 *>(p.cache_v + dst) = vv;
+                }
+                wrote_smem = true;
+                __syncwarp();
+            }
+            if (nvalid > 0) {
+                float s_lo[4], s_hi[4];
+                warp_qk_16x16<D>(qf, k_tile, kHalfBytes, row0, s_lo, s_hi);
+                const int tok = 2 * (lane & 3);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    s_lo[e] *= p.scale_log2e;
+                    s_hi[e] *= p.scale_log2e;
+                }
+                if (nvalid < 16) {
+                    // tokens past the end of the sequence: no weight, and their V rows (any bits, NaN included)
+                    // are cleared so that 0 * garbage cannot appear
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        if (tok + (e & 1) >= nvalid) s_lo[e] = -INFINITY;
+                        if (tok + (e & 1) + 8 >= nvalid) s_hi[e] = -INFINITY;
+                    }
+                    uint8_t *vt = stages + (size_t)s * C::kStageBytes + C::kTileBytes;
+                    constexpr int kChunksPerRow = D / 8;
+                    for (int i = lane; i < (16 - nvalid) * kChunksPerRow; i += 32) {
+                        const int r = row0 + nvalid + i / kChunksPerRow, ch = i % kChunksPerRow;
+                        *reinterpret_cast<uint4 *>(vt + (ch >> 3) * kHalfBytes + r * 128 + ((ch & 7) << 4)) =
+                            make_uint4(0u, 0u, 0u, 0u);
+                    }
+                    wrote_smem = true;
+                    __syncwarp();
+                }
+                uint32_t pa[4];
+                warp_softmax_16<D>(st, s_lo, s_hi, pa);
+                warp_pv_16x16<D>(st, pa, v_tile, kHalfBytes, row0);
+            }
+            if (wrote_smem) fence_proxy_async_smem();   // generic writes before the next TMA fill
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty[s]);
+        }
+        // ---- this warp's (max, sum, O) into shared memory
+        float l0 = st.l[0], l1 = st.l[1];
+        l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+        l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+        l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+        l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+        float *cw = comb + (size_t)warp * p.G * kPitch;
+        if (r_lo < p.G) {
+            float *row = cw + (size_t)r_lo * kPitch;
+            if ((lane & 3) == 0) { row[D] = st.m[0]; row[D + 1] = l0; }
+#pragma unroll
+            for (int nt = 0; nt < D / 8; ++nt)
+                *reinterpret_cast<float2 *>(row + nt * 8 + 2 * (lane & 3)) = make_float2(st.o[nt][0], st.o[nt][1]);
+        }
+        if (r_hi < p.G) {
+            float *row = cw + (size_t)r_hi * kPitch;
+            if ((lane & 3) == 0) { row[D] = st.m[1]; row[D + 1] = l1; }
+#pragma unroll
+            for (int nt = 0; nt < D / 8; ++nt)
+                *reinterpret_cast<float2 *>(row + nt * 8 + 2 * (lane & 3)) = make_float2(st.o[nt][2], st.o[nt][3]);
+        }
+    }
+    __syncthreads();
+
+    // ---- merge of the eight warps: every thread owns float4 pieces of the G x D partial (unnormalised, relative
+    // to the CTA's row maximum). A warp (or a CTA) that saw no token has max = -inf and weight 0.
+    const int items = p.G * kVec;
+    for (int item = threadIdx.x; item < items; item += kThreads) {
+        const int r = item / kVec, d4 = item % kVec;
+        float mw[kW];
+        float mstar = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < kW; ++w) {
+            mw[w] = comb[((size_t)w * p.G + r) * kPitch + D];
+            mstar = fmaxf(mstar, mw[w]);
+        }
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        float lsum = 0.f;
+#pragma unroll
+        for (int w = 0; w < kW; ++w) {
+            const float *row = comb + ((size_t)w * p.G + r) * kPitch;
+            const float wgt = (mw[w] == -INFINITY) ? 0.f : fast_exp2(mw[w] - mstar);
+            const float4 v = *reinterpret_cast<const float4 *>(row + d4 * 4);
+            acc.x += wgt * v.x; acc.y += wgt * v.y; acc.z += wgt * v.z; acc.w += wgt * v.w;
+            lsum += wgt * row[D + 1];
+        }
+        *reinterpret_cast<float4 *>(part + (size_t)r * kPitch + d4 * 4) = acc;
+        if (d4 == 0) *reinterpret_cast<float2 *>(part + (size_t)r * kPitch + D) = make_float2(mstar, lsum);
+    }
+    __syncwarp();
+    if (p.C > 1) {
+        cluster_arrive();
+        cluster_wait();
+    } else {
+        __syncthreads();
+    }
+
+    // ---- every CTA merges the C partials for its share of the output (peers' shared memory read directly)
+    const int per = (items + p.C - 1) / p.C;
+    for (int t = threadIdx.x; t < per; t += kThreads) {
+        const int item = rank * per + t;
+        if (item >= items) break;
+        const int r = item / kVec, d4 = item % kVec;
+        const uint32_t a_val = smem_u32(part + (size_t)r * kPitch + d4 * 4);
+        const uint32_t a_ml = smem_u32(part + (size_t)r * kPitch + D);
+        float2 ml[kMaxCluster];
+        float4 val[kMaxCluster];
+#pragma unroll
+        for (int c = 0; c < kMaxCluster; ++c) {
+            if (c < p.C) {
+                ml[c] = ld_cluster_f2(map_to_rank(a_ml, c));
+                val[c] = ld_cluster_f4(map_to_rank(a_val, c));
+            } else {
+                ml[c] = make_float2(-INFINITY, 0.f);
+                val[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
+        float mstar = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < kMaxCluster; ++c) mstar = fmaxf(mstar, ml[c].x);
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        float lsum = 0.f;
+#pragma unroll
+        for (int c = 0; c < kMaxCluster; ++c) {
+            const float wgt = (ml[c].x == -INFINITY) ? 0.f : fast_exp2(ml[c].x - mstar);
+            acc.x += wgt * val[c].x; acc.y += wgt * val[c].y; acc.z += wgt * val[c].z; acc.w += wgt * val[c].w;
+            lsum += wgt * ml[c].y;
+        }
+        // a sequence with no cached token gets o = 0, lse = -inf
+        const float inv = len > 0 ? 1.f / lsum : 0.f;
+        const size_t bh = (size_t)b * p.Hq + (size_t)kvh * p.G + r;
+        uint2 packed;
+        packed.x = pack_bf16x2(acc.x * inv, acc.y * inv);
+        packed.y = pack_bf16x2(acc.z * inv, acc.w * inv);
+        *reinterpret_cast<uint2 *>(p.o + bh * D + d4 * 4) = packed;
+        if (d4 == 0 && p.lse) p.lse[bh] = len > 0 ? (mstar + log2f(lsum)) * 0.6931471805599453f : -INFINITY;
+    }
+    __syncwarp();
+    // no CTA may leave while a peer can still read its shared memory
+    if (p.C > 1) {
+        cluster_arrive();
+        cluster_wait();
+    }
+    if (threadIdx.x == 0 && *abort_flag) {
+        atomicOr(p.status + kStatusErrWord, kErrDecodeWait);
+        p.status[kStatusInfoWord] = 0x30000u | (blockIdx.y & 0xffffu);
+    }
+}
+
+template <int D>
+bool configure_kernel()
+{
+    static bool done = false, ok = false;
+    if (!done) {
+        done = true;
+        ok = cudaFuncSetAttribute(decode_cluster_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) ==
+             cudaSuccess;
+        if (!ok) (void)cudaGetLastError();
+    }
+    return ok;
+}
+
+// Shared-memory stages that fit beside the merge scratch (0: none do).
+template <int D>
+int pick_stages(int G)
+{
+    for (int s = ClusterCfg<D>::kMaxStages; s >= 2; --s)
+        if (cluster_smem_bytes<D>(G, s) <= 227 * 1024) return s;
+    return 0;
+}
+
+// Clusters of C CTAs that the device can hold at once (0 if the shape cannot launch). Looked up once per shape.
+template <int D>
+int resident_clusters(int C, size_t smem)
+{
+    struct Entry { int C; size_t smem; int n; };
+    static Entry cache[16];
+    static int n_cached = 0;
+    for (int i = 0; i < n_cached; ++i)
+        if (cache[i].C == C && cache[i].smem == smem) return cache[i].n;
+    if (!configure_kernel<D>()) return 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(C, 1, 1);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = C; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, decode_cluster_kernel<D>, &cfg) != cudaSuccess) {
+        (void)cudaGetLastError();
+        n = 0;
+    }
+    if (n_cached < 16) cache[n_cached++] = Entry{C, smem, n};
+    return n;
+}
+
+}  // namespace
+
+int decode_cluster_width(int B, int Hq, int Hkv, int D, int max_kv_len)
+{
+    // debugging aid: L4L_DECODE_CLUSTER=0 keeps every call on the split kernel, =N forces clusters of N where they fit
+    int forced = -1;
+    if (const char *e = getenv("L4L_DECODE_CLUSTER")) forced = atoi(e);
+    if (forced == 0) return 0;
+    const int G = Hq / Hkv;
+    const long long units = (long long)B * Hkv;
+    const int sms = sm_count();
+    if (units <= 0 || units > 65535 || units > sms) return 0;
+    const int stages = (D == 128) ? pick_stages<128>(G) : pick_stages<64>(G);
+    if (stages == 0) return 0;
+    const size_t smem = (D == 128) ? cluster_smem_bytes<128>(G, stages) : cluster_smem_bytes<64>(G, stages);
+    const int tiles_max = max_kv_len > 0 ? (max_kv_len + kTileT - 1) / kTileT : 1;
+    // the widest power of two that keeps every cluster resident at once and gives every CTA at least one tile
+    int C = 1;
+    while (2 * C <= kMaxCluster && units * 2 * C <= sms && 2 * C <= tiles_max) C *= 2;
+    if (forced > 0) {
+        C = 1;
+        while (2 * C <= forced && 2 * C <= kMaxCluster) C *= 2;
+    }
+    for (; C >= 1; C /= 2) {
+        const int n = (D == 128) ? resident_clusters<128>(C, smem) : resident_clusters<64>(C, smem);
+        if (n >= units || (forced > 0 && n > 0)) break;
+    }
+    if (C < 1) return 0;
+    if (forced > 0) return C;
+    // Beyond these bounds the even split of the whole tile stream over all SMs (the split kernel) wins: a lone CTA
+    // per sequence streams at one SM's rate, and ragged lengths leave short sequences' CTAs idle.
+    const int per_cta = (tiles_max + C - 1) / C;
+    if (per_cta > 32) return 0;
+    return C;
+}
+
+l4l_status launch_decode_cluster(const void *q, void *o, const l4l_kv_cache &cache, const int32_t *d_kv_lens,
+                                 int max_kv_len, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
+                                 void *workspace, cudaStream_t stream, const l4l_tensor4 *k_new,
+                                 const l4l_tensor4 *v_new, const PagedTable *paged, int width)
+{
+    if (paged && (k_new || v_new)) return L4L_ERR_UNSUPPORTED;
+    const int G = Hq / Hkv;
+    const int stages = (D == 128) ? pick_stages<128>(G) : pick_stages<64>(G);
+    if (stages == 0 || width < 1 || width > kMaxCluster) return L4L_ERR_UNSUPPORTED;
+    const size_t smem = (D == 128) ? cluster_smem_bytes<128>(G, stages) : cluster_smem_bytes<64>(G, stages);
+    if (!((D == 128) ? configure_kernel<128>() : configure_kernel<64>())) return L4L_ERR_CUDA;
+
+    CUtensorMap tk, tv, tk16, tv16;   // tile-sized boxes, and 16-token boxes for the last tile of a sequence
+    TmapCoord coord, coord_v;
+    const int outer = paged ? paged->num_pages : B;
+    // pages smaller than a tile are fetched page by page: no box may exceed the page
+    const int box_t = (paged && cache.max_len < kTileT) ? cache.max_len : kTileT;
+    if (!make_tmap(&tk, &coord, cache.k, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h, cache.stride_b, 64,
+                   box_t, 2) ||
+        !make_tmap(&tv, &coord_v, cache.v, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h, cache.stride_b,
+                   64, box_t, 2) ||
+        !make_tmap(&tk16, &coord_v, cache.k, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
+                   cache.stride_b, 64, 16, 2) ||
+        !make_tmap(&tv16, &coord_v, cache.v, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
+                   cache.stride_b, 64, 16, 2))
+        return L4L_ERR_CUDA;
+    ClusterParams p;
+    p.q = static_cast<const __nv_bfloat16 *>(q);
+    p.o = static_cast<__nv_bfloat16 *>(o);
+    p.lse = d_lse;
+    p.kv_lens = d_kv_lens;
+    p.k_new = p.v_new = nullptr;
+    p.new_sb = p.new_sh = 0;
+    if (k_new && v_new) {
+        if (k_new->stride_b != v_new->stride_b || k_new->stride_h != v_new->stride_h) return L4L_ERR_UNSUPPORTED;
+        p.k_new = static_cast<const __nv_bfloat16 *>(k_new->ptr);
+        p.v_new = static_cast<const __nv_bfloat16 *>(v_new->ptr);
+        p.new_sb = k_new->stride_b; p.new_sh = k_new->stride_h;
+    }
+    p.cache_k = static_cast<__nv_bfloat16 *>(cache.k);
+    p.cache_v = static_cast<__nv_bfloat16 *>(cache.v);
+    p.c_sb = cache.stride_b; p.c_sh = cache.stride_h; p.c_st = cache.stride_t;
+    p.status = static_cast<unsigned *>(workspace);
+    p.block_table = paged ? paged->block_table : nullptr;
+    p.table_stride = paged ? paged->table_stride : 0;
+    p.page_size = paged ? cache.max_len : 0;
+    p.page_shift = 0;
+    while (paged && (1 << p.page_shift) < cache.max_len) ++p.page_shift;
+    p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.G = G; p.C = width; p.max_kv_len = max_kv_len; p.stages = stages;
+    p.scale_log2e = scale * 1.4426950408889634f;
+    p.coord = coord;
+
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(width, B * Hkv, 1);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = width; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    const cudaError_t err = (D == 128) ? cudaLaunchKernelEx(&cfg, decode_cluster_kernel<128>, tk, tv, tk16, tv16, p)
+                                       : cudaLaunchKernelEx(&cfg, decode_cluster_kernel<64>, tk, tv, tk16, tv16, p);
+    return err == cudaSuccess ? L4L_OK : L4L_ERR_CUDA;
+}
+
+}  // namespace l4l

@@ -74,6 +74,14 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
                          const PagedTable *paged = nullptr, const Fp8Scales *fp8 = nullptr,
                          const RopeArgs *rope = nullptr);
 
+// Small batches: one thread-block cluster per (sequence, KV head), partials merged through distributed shared
+// memory. decode_cluster_width returns the cluster size to use, or 0 if the split kernel should run.
+int decode_cluster_width(int B, int Hq, int Hkv, int D, int max_kv_len);
+l4l_status launch_decode_cluster(const void *q, void *o, const l4l_kv_cache &cache, const int32_t *d_kv_lens,
+                                 int max_kv_len, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
+                                 void *workspace, cudaStream_t stream, const l4l_tensor4 *k_new,
+                                 const l4l_tensor4 *v_new, const PagedTable *paged, int width);
+
 l4l_status launch_rope_kv_append(const l4l_tensor4 &q, const l4l_tensor4 &k_new, const l4l_tensor4 &v_new,
                                  const l4l_kv_cache &cache, const int32_t *d_pos, const int32_t *d_n_new, int T, int B,
                                  int Hq, int Hkv, int D, const float *d_cos, const float *d_sin, int n_pos,
