@@ -92,6 +92,7 @@ struct DecodeParams {
     // at offset t % page_size; the tensor maps then describe the page pool [pages, Hkv, page_size, D]
     const int32_t *block_table;
     int table_stride, page_size, page_shift;
+    int tail_rows;            // tokens per box of tmap_k_tail / tmap_v_tail (32, or the page size if that is smaller)
     int B, Hq, Hkv, G, min_tiles, nsplit, max_kv_len;
     float scale_log2e;
     TmapCoord coord;
@@ -107,7 +108,7 @@ size_t decode_smem_bytes(int G, int nsplit)
     return 1024 /*alignment slack*/ + (size_t)C::kStages * (C::kStageBytes + (size_t)G * D * 2 + D * 4) + (size_t)W * D * 4 + 2 * D * 4 +
            comb +
            C::kStages * sizeof(TileMeta) +
-           sizeof(PieceMeta) + (2 * C::kStages + 2) * sizeof(uint64_t) + (kMaxB + 1) * sizeof(int) + 64 +
+           sizeof(PieceMeta) + (2 * C::kStages + 2) * sizeof(uint64_t) + (2 * kMaxB + 1) * sizeof(int) + 64 +
            kPostRing * sizeof(PieceMeta);
 }
 
@@ -222,7 +223,7 @@ __device__ __forceinline__ uint4 rope_k_row(uint4 kk, const DecodeParams &p, con
 template <int D, int W, bool F8>
 __global__ void __launch_bounds__((W + 2) * 32)
 decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
-                    const __grid_constant__ CUtensorMap tmap_k16, const __grid_constant__ CUtensorMap tmap_v16,
+                    const __grid_constant__ CUtensorMap tmap_k_tail, const __grid_constant__ CUtensorMap tmap_v_tail,
                     const DecodeParams p)
 {
     using C = DecodeCfg<D, W, F8>;
@@ -251,11 +252,12 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     uint64_t *comb_full = empty + C::kStages;   // consumers -> finisher: a piece's results are in `comb`
     uint64_t *comb_empty = comb_full + 1;       // finisher -> consumers: `comb` may be overwritten
     int *cum = reinterpret_cast<int *>(comb_empty + 1);   // cum[b] = tiles of sequences < b (times Hkv)
-    volatile int *abort_flag = cum + (kMaxB + 1);
+    int *lens_s = cum + (kMaxB + 1);                      // clamped kv_lens
+    volatile int *abort_flag = lens_s + kMaxB;
     // producer -> finisher: the pieces this CTA has started, in order (so that the finisher can look at a
     // piece's ticket while the piece is still being streamed)
     volatile uint32_t *posted_count = reinterpret_cast<volatile uint32_t *>(abort_flag + 1);
-    PieceMeta *post_ring = reinterpret_cast<PieceMeta *>(cum + (kMaxB + 1) + 4);
+    PieceMeta *post_ring = reinterpret_cast<PieceMeta *>(lens_s + kMaxB + 4);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -275,8 +277,8 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     if (warp == kProducerWarp && lane == 0) {
         tma_prefetch_desc(&tmap_k);
         tma_prefetch_desc(&tmap_v);
-        tma_prefetch_desc(&tmap_k16);
-        tma_prefetch_desc(&tmap_v16);
+        tma_prefetch_desc(&tmap_k_tail);
+        tma_prefetch_desc(&tmap_v_tail);
     }
     // Programmatic dependent launch: everything above overlaps the tail of the previous kernel in the
     // stream; nothing below (no global read or write) starts before that kernel has completed. The
@@ -301,6 +303,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             if (b < p.B) {
                 int len = p.kv_lens[b];
                 len = len < 0 ? 0 : (len > p.max_kv_len ? p.max_kv_len : len);
+                lens_s[b] = len;
                 n = ((len + kTileT - 1) / kTileT) * p.Hkv;
             }
             int incl = n;
@@ -329,24 +332,41 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             const int my_end = range_begin((int)blockIdx.x + 1);
             uint32_t it = 0, n_posted = 0;
             bool ok = true;
+            // The walk over this CTA's pieces: the first one is located by a binary search over the prefix sums, every
+            // later one starts a sequence (the next KV head of the same sequence, or the next sequence with tokens),
+            // so its numbers follow from the previous piece without a search or a division.
             int g = my_begin;
+            int b = 0, kvh = 0, len = 0, tiles_b = 0, seq_first = 0;
+            bool located = false;
             while (ok && g < my_end) {
-                int lo = 0, hi = p.B;          // largest b with cum[b] <= g
-                while (hi - lo > 1) {
-                    const int mid = (lo + hi) >> 1;
-                    if (cum[mid] <= g) lo = mid; else hi = mid;
+                int first_cta;
+                if (!located) {
+                    int lo = 0, hi = p.B;          // largest b with cum[b] <= g
+                    while (hi - lo > 1) {
+                        const int mid = (lo + hi) >> 1;
+                        if (cum[mid] <= g) lo = mid; else hi = mid;
+                    }
+                    b = lo;
+                    len = lens_s[b];
+                    tiles_b = (len + kTileT - 1) / kTileT;
+                    kvh = (g - cum[b]) / tiles_b;
+                    seq_first = cum[b] + kvh * tiles_b;          // flattened index of this sequence's tile 0
+                    first_cta = cta_of(seq_first);
+                    located = true;
+                } else {
+                    seq_first += tiles_b;                         // == g: the previous piece ran to the end of its sequence
+                    if (++kvh == p.Hkv) {
+                        kvh = 0;
+                        do { ++b; } while (lens_s[b] == 0);       // g < total: a sequence with tokens follows
+                        len = lens_s[b];
+                        tiles_b = (len + kTileT - 1) / kTileT;
+                    }
+                    first_cta = (int)blockIdx.x;
                 }
-                const int b = lo;
-                int len = p.kv_lens[b];
-                len = len > p.max_kv_len ? p.max_kv_len : len;
-                const int tiles_b = (len + kTileT - 1) / kTileT;
-                const int r = g - cum[b];
-                const int kvh = r / tiles_b;
-                const int seq_first = cum[b] + kvh * tiles_b;          // flattened index of this sequence's tile 0
                 const int tile_begin = g - seq_first;
                 const int tile_end = min(tiles_b, my_end - seq_first);
-                const int first_cta = cta_of(seq_first);
-                const int npieces = cta_of(seq_first + tiles_b - 1) - first_cta + 1;
+                const int npieces = (seq_first + tiles_b <= my_end) ? (int)blockIdx.x - first_cta + 1
+                                                                    : cta_of(seq_first + tiles_b - 1) - first_cta + 1;
                 const int piece = (int)blockIdx.x - first_cta;
                 {
                     PieceMeta &pp = post_ring[n_posted % kPostRing];
@@ -365,11 +385,19 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     mt.flags = (tile == tile_begin ? kFlagFirst : 0) | (tile + 1 == tile_end ? kFlagLast : 0);
                     // the first tile of a piece also brings the group's query rows (contiguous in q)
                     const bool first = (tile == tile_begin);
-                    // the last tile of a sequence is fetched in 16-token groups, so that (almost) nothing past
-                    // the end of the sequence is read; rows not fetched are never looked at by the consumers
+                    // The last tile of a sequence: if at most half of it holds tokens it is fetched in groups of
+                    // p.tail_rows tokens (a few small boxes, nothing past the group that holds the last token); else as
+                    // a whole tile like the others (one box; rows past the end of the sequence are never looked at
+                    // by the consumers, rows past the end of the cache arrive as zeros). With pages smaller than a
+                    // tile only the pages that hold tokens are fetched.
+                    const bool paged = p.block_table != nullptr;
                     const int rem = len - tile * kTileT;
-                    const int groups = rem >= kTileT ? kTileT / 16 : (rem + 15) / 16;
-                    const uint32_t kv_bytes = rem >= kTileT ? C::kStageBytes : (uint32_t)groups * 16u * 128u * C::kHalves * 2u;
+                    const int groups = (rem + p.tail_rows - 1) / p.tail_rows;
+                    const bool by_groups = rem < kTileT && groups * p.tail_rows * 2 <= kTileT;
+                    const int box_rows = by_groups ? p.tail_rows : ((paged && p.page_size < kTileT) ? p.page_size : kTileT);
+                    const int n_box = by_groups ? groups : ((rem >= kTileT || box_rows == kTileT) ? kTileT / box_rows
+                                                                                                  : (rem + box_rows - 1) / box_rows);
+                    const uint32_t kv_bytes = (uint32_t)n_box * box_rows * 128u * C::kHalves * 2u;
                     // with the rope fused into the step, the piece's first tile also brings the cos / sin rows of
                     // the new token's position (kv_len - 1), if the table has it
                     const bool with_rope = first && p.rope_cos != nullptr && len - 1 < p.rope_n_pos;
@@ -383,49 +411,26 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                         bulk_load_1d(rs + kRopeBytes / 2, p.rope_sin + (size_t)(len - 1) * (D / 2), kRopeBytes / 2, &full[s]);
                     }
                     uint8_t *dst = stages + (size_t)s * C::kStageBytes;
-                    // With a paged cache a full tile is one box if a page holds whole tiles, else one box per
-                    // page (tmap_k / tmap_v then have page-sized boxes); the last tile of a sequence comes in
-                    // 16-token groups either way. Neither a box nor a group straddles pages: page sizes are
-                    // powers of two >= 16. A page id outside the pool makes the box read zeros, never memory.
-                    const bool paged = p.block_table != nullptr;
+                    // Neither a box nor a group straddles pages: page sizes are powers of two >= 16 and p.tail_rows is at
+                    // most the page size. A page id outside the pool makes the box read zeros, never memory.
                     const int32_t *pages = paged ? p.block_table + (size_t)b * p.table_stride : nullptr;
-                    if (rem >= kTileT) {
-                        const int box_rows = (paged && p.page_size < kTileT) ? p.page_size : kTileT;
-                        const int n_box = kTileT / box_rows;
-                        int page_of[kTileT / 16];                    // looked up together: independent loads
+                    const CUtensorMap *tk = by_groups ? &tmap_k_tail : &tmap_k;
+                    const CUtensorMap *tv = by_groups ? &tmap_v_tail : &tmap_v;
+                    int page_of[kTileT / 16];                    // looked up together: independent loads
 #pragma unroll
-                        for (int bx = 0; bx < kTileT / 16; ++bx)
-                            page_of[bx] = (paged && bx < n_box) ? __ldg(pages + ((tile * kTileT + bx * box_rows) >> p.page_shift)) : b;
+                    for (int bx = 0; bx < kTileT / 16; ++bx)
+                        page_of[bx] = (paged && bx < n_box) ? __ldg(pages + ((tile * kTileT + bx * box_rows) >> p.page_shift)) : b;
 #pragma unroll
-                        for (int bx = 0; bx < kTileT / 16; ++bx) {
-                            if (bx >= n_box) break;
-                            int tt = tile * kTileT + bx * box_rows;
-                            if (paged) tt &= p.page_size - 1;
-                            order_coords(p.coord, tt, kvh, page_of[bx], c1, c2, c3);
-                            uint8_t *db = dst + bx * box_rows * 128;  // whole 8-row groups: the swizzle phase is kept
+                    for (int bx = 0; bx < kTileT / 16; ++bx) {
+                        if (bx >= n_box) break;
+                        int tt = tile * kTileT + bx * box_rows;
+                        if (paged) tt &= p.page_size - 1;
+                        order_coords(p.coord, tt, kvh, page_of[bx], c1, c2, c3);
+                        uint8_t *db = dst + bx * box_rows * 128;  // whole 8-row groups: the swizzle phase is kept
 #pragma unroll
-                            for (int hf = 0; hf < C::kHalves; ++hf) {
-                                tma_load_4d(db + hf * C::kHalfBytes, &tmap_k, &full[s], hf * C::kBoxD, c1, c2, c3);
-                                tma_load_4d(db + C::kTileBytes + hf * C::kHalfBytes, &tmap_v, &full[s], hf * C::kBoxD, c1, c2, c3);
-                            }
-                        }
-                    } else {
-                        int page_of[kTileT / 16];                    // looked up together: independent loads
-#pragma unroll
-                        for (int gq = 0; gq < kTileT / 16; ++gq)
-                            page_of[gq] = (paged && gq < groups) ? __ldg(pages + ((tile * kTileT + gq * 16) >> p.page_shift)) : b;
-#pragma unroll
-                        for (int gq = 0; gq < kTileT / 16; ++gq) {
-                            if (gq >= groups) break;
-                            int tt = tile * kTileT + gq * 16;
-                            if (paged) tt &= p.page_size - 1;
-                            order_coords(p.coord, tt, kvh, page_of[gq], c1, c2, c3);
-                            uint8_t *dg = dst + gq * 16 * 128;        // 2 KB per group: the swizzle phase is kept
-#pragma unroll
-                            for (int hf = 0; hf < C::kHalves; ++hf) {
-                                tma_load_4d(dg + hf * C::kHalfBytes, &tmap_k16, &full[s], hf * C::kBoxD, c1, c2, c3);
-                                tma_load_4d(dg + C::kTileBytes + hf * C::kHalfBytes, &tmap_v16, &full[s], hf * C::kBoxD, c1, c2, c3);
-                            }
+                        for (int hf = 0; hf < C::kHalves; ++hf) {
+                            tma_load_4d(db + hf * C::kHalfBytes, tk, &full[s], hf * C::kBoxD, c1, c2, c3);
+                            tma_load_4d(db + C::kTileBytes + hf * C::kHalfBytes, tv, &full[s], hf * C::kBoxD, c1, c2, c3);
                         }
                     }
                 }
@@ -1108,7 +1113,7 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
     if (slice < 1) return L4L_ERR_UNSUPPORTED;
     for (int b0 = 0; b0 < B; b0 += slice) {
         const int nb = (B - b0 < slice) ? (B - b0) : slice;
-        CUtensorMap tk, tv, tk16, tv16;   // 64-token boxes, and 16-token boxes for the last tile of a sequence
+        CUtensorMap tk, tv, tk_tail, tv_tail;   // tile-sized boxes, and small boxes for a mostly empty last tile of a sequence
         TmapCoord coord, coord_v;
         // contiguous: the maps cover this slice's sequences; paged: the whole pool, whatever the slice
         const size_t first = paged ? 0 : (size_t)b0 * cache.stride_b;
@@ -1118,14 +1123,15 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         const int box_d = fp8 ? 128 : 64;
         // pages smaller than a tile are fetched page by page: no box may exceed the page
         const int box_t = (paged && cache.max_len < kTileT) ? cache.max_len : kTileT;
+        const int tail_rows = (paged && cache.max_len < 32) ? cache.max_len : 32;
         if (!make_tmap(&tk, &coord, kb, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
                        cache.stride_b, box_d, box_t, esz) ||
             !make_tmap(&tv, &coord_v, vb, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
                        cache.stride_b, box_d, box_t, esz) ||
-            !make_tmap(&tk16, &coord_v, kb, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
-                       cache.stride_b, box_d, 16, esz) ||
-            !make_tmap(&tv16, &coord_v, vb, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
-                       cache.stride_b, box_d, 16, esz))
+            !make_tmap(&tk_tail, &coord_v, kb, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
+                       cache.stride_b, box_d, tail_rows, esz) ||
+            !make_tmap(&tv_tail, &coord_v, vb, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
+                       cache.stride_b, box_d, tail_rows, esz))
             return L4L_ERR_CUDA;
         DecodeParams p;
         p.q = static_cast<const __nv_bfloat16 *>(q) + (size_t)b0 * Hq * D;
@@ -1151,6 +1157,7 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         p.block_table = paged ? paged->block_table + (size_t)b0 * paged->table_stride : nullptr;
         p.table_stride = paged ? paged->table_stride : 0;
         p.page_size = paged ? cache.max_len : 0;
+        p.tail_rows = tail_rows;
         p.page_shift = 0;
         while (paged && (1 << p.page_shift) < cache.max_len) ++p.page_shift;
         // only the fused append (bf16, contiguous) writes through these
@@ -1177,14 +1184,14 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         cfg.numAttrs = 1;
         cudaError_t err;
         if (fp8)
-            err = plan.warps == 8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 8, true>, tk, tv, tk16, tv16, p)
-                                  : cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 4, true>, tk, tv, tk16, tv16, p);
+            err = plan.warps == 8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 8, true>, tk, tv, tk_tail, tv_tail, p)
+                                  : cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 4, true>, tk, tv, tk_tail, tv_tail, p);
         else if (D == 128)
-            err = plan.warps == 8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 8, false>, tk, tv, tk16, tv16, p)
-                                  : cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 4, false>, tk, tv, tk16, tv16, p);
+            err = plan.warps == 8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 8, false>, tk, tv, tk_tail, tv_tail, p)
+                                  : cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 4, false>, tk, tv, tk_tail, tv_tail, p);
         else
-            err = plan.warps == 8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<64, 8, false>, tk, tv, tk16, tv16, p)
-                                  : cudaLaunchKernelEx(&cfg, decode_split_kernel<64, 4, false>, tk, tv, tk16, tv16, p);
+            err = plan.warps == 8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<64, 8, false>, tk, tv, tk_tail, tv_tail, p)
+                                  : cudaLaunchKernelEx(&cfg, decode_split_kernel<64, 4, false>, tk, tv, tk_tail, tv_tail, p);
         if (err != cudaSuccess) return L4L_ERR_CUDA;
     }
     return L4L_OK;
