@@ -251,7 +251,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     uint64_t *empty = full + C::kStages;
     uint64_t *comb_full = empty + C::kStages;   // consumers -> finisher: a piece's results are in `comb`
     uint64_t *comb_empty = comb_full + 1;       // finisher -> consumers: `comb` may be overwritten
-    int *cum = reinterpret_cast<int *>(comb_empty + 1);   // cum[b] = tiles of sequences < b (times Hkv)
+    int *cum = reinterpret_cast<int *>(comb_empty + 1);   // cum[b] = stream items (tiles + one marker per KV head) of sequences < b
     int *lens_s = cum + (kMaxB + 1);                      // clamped kv_lens
     volatile int *abort_flag = lens_s + kMaxB;
     // producer -> finisher: the pieces this CTA has started, in order (so that the finisher can look at a
@@ -295,7 +295,10 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
 
     if (warp == kProducerWarp) {
         // ------------------------------------------------------------------ producer warp
-        // exclusive prefix sum over sequences of (tiles * Hkv)
+        // Exclusive prefix sum over sequences of ((tiles + 1) * Hkv): the flattened stream that is divided among
+        // the CTAs holds, ahead of the tiles of every (sequence, KV head), one marker that stands for the fixed
+        // cost of starting a piece there (query rows, a mostly short last tile, the hand-over to the finisher:
+        // about one tile's time). A CTA whose range covers many short sequences thus gets fewer tiles.
         int running = 0;
         for (int b0 = 0; b0 < p.B; b0 += 32) {
             const int b = b0 + lane;
@@ -304,7 +307,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 int len = p.kv_lens[b];
                 len = len < 0 ? 0 : (len > p.max_kv_len ? p.max_kv_len : len);
                 lens_s[b] = len;
-                n = ((len + kTileT - 1) / kTileT) * p.Hkv;
+                n = len > 0 ? ((len + kTileT - 1) / kTileT + 1) * p.Hkv : 0;
             }
             int incl = n;
 #pragma unroll
@@ -349,12 +352,12 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     b = lo;
                     len = lens_s[b];
                     tiles_b = (len + kTileT - 1) / kTileT;
-                    kvh = (g - cum[b]) / tiles_b;
-                    seq_first = cum[b] + kvh * tiles_b;          // flattened index of this sequence's tile 0
-                    first_cta = cta_of(seq_first);
+                    kvh = (g - cum[b]) / (tiles_b + 1);
+                    seq_first = cum[b] + kvh * (tiles_b + 1);    // flattened index of this sequence's marker; tile t at +1+t
+                    first_cta = cta_of(seq_first + 1);
                     located = true;
                 } else {
-                    seq_first += tiles_b;                         // == g: the previous piece ran to the end of its sequence
+                    seq_first += tiles_b + 1;                     // == g: the previous piece ran to the end of its sequence
                     if (++kvh == p.Hkv) {
                         kvh = 0;
                         do { ++b; } while (lens_s[b] == 0);       // g < total: a sequence with tokens follows
@@ -363,10 +366,11 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     }
                     first_cta = (int)blockIdx.x;
                 }
-                const int tile_begin = g - seq_first;
-                const int tile_end = min(tiles_b, my_end - seq_first);
-                const int npieces = (seq_first + tiles_b <= my_end) ? (int)blockIdx.x - first_cta + 1
-                                                                    : cta_of(seq_first + tiles_b - 1) - first_cta + 1;
+                const int tile_begin = max(g - seq_first - 1, 0);
+                const int tile_end = min(tiles_b, my_end - seq_first - 1);
+                if (tile_end <= tile_begin) break;                // only the marker fell into this range (at its very end)
+                const int npieces = (seq_first + tiles_b + 1 <= my_end) ? (int)blockIdx.x - first_cta + 1
+                                                                        : cta_of(seq_first + tiles_b) - first_cta + 1;
                 const int piece = (int)blockIdx.x - first_cta;
                 {
                     PieceMeta &pp = post_ring[n_posted % kPostRing];
@@ -434,7 +438,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                         }
                     }
                 }
-                g = seq_first + tile_end;
+                g = seq_first + 1 + tile_end;
             }
             if (ok) {
                 const uint32_t s = it % C::kStages;
