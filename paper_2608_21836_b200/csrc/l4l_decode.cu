@@ -25,6 +25,7 @@
 #include <mutex>
 
 #include "l4l_internal.h"
+#include "l4l_rope_frag.cuh"
 #include "l4l_warp_attn.cuh"
 
 namespace l4l {
@@ -117,107 +118,6 @@ __device__ __forceinline__ void order_coords(const TmapCoord &c, int t, int h, i
     c1 = (c.pos_t == 1) ? t : (c.pos_h == 1) ? h : b;
     c2 = (c.pos_t == 2) ? t : (c.pos_h == 2) ? h : b;
     c3 = (c.pos_t == 3) ? t : (c.pos_h == 3) ? h : b;
-}
-
-// ---- rotary embedding (+ optional RMS norm) of the step's own token, inside the decode kernel ----------
-// Same arithmetic as the streaming rope kernel: xn = (x * rinv) * w, y1 = fma(-x2, sin, x1 * cos),
-// y2 = fma(x1, sin, x2 * cos) in fp32, one rounding to bf16. A position outside the table leaves the row as it is.
-// The cos | sin rows of the position come from shared memory: the producer fetches them with the piece's first tile.
-
-// The q rows live in the A fragments of the warp MMA: a thread holds, per 16-column k-step, columns 2c, 2c+1
-// (registers 0: row lane/4, 1: row lane/4 + 8) and 2c+8, 2c+9 (registers 2, 3), c = lane % 4. The partner of
-// column i is column i + D/2, i.e. the same register of the k-step D/32 further on: no data leaves the thread.
-template <int D>
-__device__ __forceinline__ void rope_q_fragments(uint32_t (&qf)[D / 16][4], const DecodeParams &p, const float *cos_sin,
-                                                 const float *weight, int lane)
-{
-    constexpr int kSteps = D / 16, kHalf = kSteps / 2;
-    const int c = lane & 3;
-    const bool valid[2] = {(lane >> 2) < p.G, (lane >> 2) + 8 < p.G};
-    float rinv[2] = {1.f, 1.f};
-    if (p.q_weight != nullptr) {
-        float ss[2] = {0.f, 0.f};
-#pragma unroll
-        for (int ks = 0; ks < kSteps; ++ks)
-#pragma unroll
-            for (int r = 0; r < 4; ++r) {
-                const float a = __uint_as_float(qf[ks][r] << 16), b = __uint_as_float(qf[ks][r] & 0xffff0000u);
-                ss[r & 1] = fmaf(a, a, fmaf(b, b, ss[r & 1]));
-            }
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            ss[h] += __shfl_xor_sync(0xffffffffu, ss[h], 1);
-            ss[h] += __shfl_xor_sync(0xffffffffu, ss[h], 2);
-            rinv[h] = valid[h] ? rsqrtf(ss[h] * (1.f / D) + p.norm_eps) : 0.f;
-        }
-    }
-    const float *cr = cos_sin, *sr = cos_sin + D / 2;              // shared memory: cos | sin of the position
-#pragma unroll
-    for (int ks = 0; ks < kHalf; ++ks)
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            const int col = 16 * ks + 2 * c + ((r >> 1) << 3);               // first-half column of element 0
-            float x1[2] = {__uint_as_float(qf[ks][r] << 16), __uint_as_float(qf[ks][r] & 0xffff0000u)};
-            float x2[2] = {__uint_as_float(qf[ks + kHalf][r] << 16), __uint_as_float(qf[ks + kHalf][r] & 0xffff0000u)};
-            float y1[2], y2[2];
-#pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                if (p.q_weight != nullptr) {
-                    x1[e] = x1[e] * rinv[r & 1] * weight[col + e];
-                    x2[e] = x2[e] * rinv[r & 1] * weight[col + e + D / 2];
-                }
-                const float cs = cr[col + e], sn = sr[col + e];
-                y1[e] = fmaf(-x2[e], sn, x1[e] * cs);
-                y2[e] = fmaf(x1[e], sn, x2[e] * cs);
-            }
-            if (valid[r & 1]) {
-                qf[ks][r] = pack_bf16x2(y1[0], y1[1]);
-                qf[ks + kHalf][r] = pack_bf16x2(y2[0], y2[1]);
-            }
-        }
-}
-
-// The new token's k row as the patching warp holds it: lane l < D/8 has elements [8l, 8l + 8). The partner chunk
-// is D/16 lanes away. Every lane of the warp must call this (shuffles); lanes >= D/8 pass zeros.
-template <int D>
-__device__ __forceinline__ uint4 rope_k_row(uint4 kk, const DecodeParams &p, const float *cos_sin, const float *weight,
-                                            bool in_table, int lane)
-{
-    constexpr int kChunks = D / 8, kHalfChunks = D / 16;
-    float x[8];
-    const uint32_t w[4] = {kk.x, kk.y, kk.z, kk.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        x[2 * i] = __uint_as_float(w[i] << 16);
-        x[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-    }
-    if (p.k_weight != nullptr) {
-        float ss = 0.f;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) ss = fmaf(x[i], x[i], ss);
-#pragma unroll
-        for (int off = 1; off < kChunks; off <<= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
-        const float rinv = rsqrtf(ss * (1.f / D) + p.norm_eps);
-        if (lane < kChunks && in_table) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) x[i] = x[i] * rinv * weight[8 * lane + i];
-        }
-    }
-    float y[8];
-    const bool first = (lane & kHalfChunks) == 0;
-    const int col0 = 8 * (lane & (kHalfChunks - 1));
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const float px = __shfl_xor_sync(0xffffffffu, x[i], kHalfChunks);
-        float cs = 1.f, sn = 0.f;
-        if (lane < kChunks && in_table) {
-            cs = cos_sin[col0 + i];
-            sn = cos_sin[D / 2 + col0 + i];
-        }
-        y[i] = first ? fmaf(-px, sn, x[i] * cs) : fmaf(px, sn, x[i] * cs);
-    }
-    if (!in_table) return kk;
-    return make_uint4(pack_bf16x2(y[0], y[1]), pack_bf16x2(y[2], y[3]), pack_bf16x2(y[4], y[5]), pack_bf16x2(y[6], y[7]));
 }
 
 template <int D, int W, bool F8>
@@ -793,7 +693,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                         const float4 *src = reinterpret_cast<const float4 *>(q_slots + (size_t)s * q_stride + q_bytes);
                         for (int i = lane; i < D / 4; i += 32) reinterpret_cast<float4 *>(mine)[i] = src[i];
                         __syncwarp();
-                        rope_q_fragments<D>(qf, p, mine, norm_w, lane);
+                        rope_q_fragments<D>(qf, p.G, p.q_weight != nullptr, p.norm_eps, mine, norm_w, lane);
                     }
                 }
             }
@@ -816,7 +716,8 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     vv = __ldg(reinterpret_cast<const uint4 *>(p.v_new + src));
                 }
                 if (p.rope_cos != nullptr)                                      // all lanes: shuffles inside
-                    kk = rope_k_row<D>(kk, p, rope_priv + (size_t)warp * D, norm_w + D, mt.kv_len - 1 < p.rope_n_pos, lane);
+                    kk = rope_k_row<D>(kk, p.k_weight != nullptr, p.norm_eps, rope_priv + (size_t)warp * D, norm_w + D,
+                                        mt.kv_len - 1 < p.rope_n_pos, lane);
                 if (lane < kChunks) {
                     uint8_t *kt = stages + (size_t)s * C::kStageBytes;
                     const uint32_t off = (lane >> 3) * C::kHalfBytes + swz128(last, lane & 7);
@@ -1093,12 +994,12 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
     const int esz = fp8 ? 1 : 2;
     // paged: `cache` describes the page pool (stride_b = stride between pages, max_len = page size)
     if (paged && (k_new || v_new)) return L4L_ERR_UNSUPPORTED;
-    if (!fp8 && !rope) {
+    if (!fp8) {
         // small batches are latency-bound: one cluster per (sequence, KV head), no workspace round trips
         const int width = decode_cluster_width(B, Hq, Hkv, D, max_kv_len);
         if (width > 0)
             return launch_decode_cluster(q, o, cache, d_kv_lens, max_kv_len, B, Hq, Hkv, D, scale, d_lse, workspace,
-                                         stream, k_new, v_new, paged, width);
+                                         stream, k_new, v_new, paged, rope, width);
     }
     const int G = Hq / Hkv;
     const ShapeOps ops = pick_shape(D, plan.warps, fp8 != nullptr);

@@ -13,10 +13,12 @@
 //   warps 0-7   16 tokens of every tile each, all query heads of the KV group as the M dimension of the warp
 //               MMAs (the same building blocks as the split kernel), fused append of the step's new token
 //
-// bf16 cache, contiguous or paged. The fp8 cache and the rope-fused step stay on the split kernel.
+// bf16 cache, contiguous or paged, with or without the rotary embedding (+ RMS norm) of the step's q and k fused
+// in. The fp8 cache stays on the split kernel.
 #include <cstdlib>
 
 #include "l4l_internal.h"
+#include "l4l_rope_frag.cuh"
 #include "l4l_warp_attn.cuh"
 
 namespace l4l {
@@ -50,6 +52,12 @@ struct ClusterParams {
     unsigned *status;
     const int32_t *block_table;               // paged cache (null: contiguous)
     int table_stride, page_size, page_shift;
+    // rotary embedding (+ optional RMS norm) of the step's q and k_new (null: inputs are final); only with the fused
+    // append. The new token's position is kv_len - 1.
+    const float *rope_cos, *rope_sin;         // [rope_n_pos, D/2]
+    const float *q_weight, *k_weight;         // [D] or null
+    float norm_eps;
+    int rope_n_pos;
     int B, Hq, Hkv, G, C, max_kv_len, stages;
     float scale_log2e;
     TmapCoord coord;
@@ -60,7 +68,8 @@ size_t cluster_smem_bytes(int G, int stages)
 {
     using C = ClusterCfg<D>;
     return 1024 /*alignment slack*/ + (size_t)stages * C::kStageBytes + (size_t)G * D * 2 +
-           (size_t)(kW + 1) * G * C::kPitch * sizeof(float) + 2 * C::kMaxStages * sizeof(uint64_t) + 64;
+           (size_t)(kW + 1) * G * C::kPitch * sizeof(float) + 3 * D * sizeof(float) +
+           2 * C::kMaxStages * sizeof(uint64_t) + 64;
 }
 
 __device__ __forceinline__ void order_coords(const TmapCoord &c, int t, int h, int b, int &c1, int &c2, int &c3)
@@ -121,7 +130,10 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
     const uint32_t q_bytes = (uint32_t)p.G * D * 2;
     float *comb = reinterpret_cast<float *>(q_smem + q_bytes);       // [kW][G][kPitch] per-warp results
     float *part = comb + (size_t)kW * p.G * kPitch;                  // [G][kPitch] this CTA's merged partial
-    uint64_t *full = reinterpret_cast<uint64_t *>(part + (size_t)p.G * kPitch);
+    float *rope_cs = part + (size_t)p.G * kPitch;                    // cos | sin of the new token's position
+    float *norm_w = rope_cs + D;                                     // q_weight | k_weight
+    constexpr uint32_t kRopeBytes = D * 4;
+    uint64_t *full = reinterpret_cast<uint64_t *>(norm_w + 2 * D);
     uint64_t *empty = full + C::kMaxStages;
     volatile int *abort_flag = reinterpret_cast<volatile int *>(empty + C::kMaxStages);
 
@@ -150,6 +162,13 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
     grid_launch_dependents();
     int len = __ldg(p.kv_lens + b);
     len = len < 0 ? 0 : (len > p.max_kv_len ? p.max_kv_len : len);
+    const bool with_rope = p.rope_cos != nullptr && len - 1 < p.rope_n_pos;   // a position outside the table: rows stay as they are
+    if (p.rope_cos != nullptr) {
+        for (int i = threadIdx.x; i < D; i += kThreads) {
+            norm_w[i] = p.q_weight ? __ldg(p.q_weight + i) : 1.f;
+            norm_w[D + i] = p.k_weight ? __ldg(p.k_weight + i) : 1.f;
+        }
+    }
     __syncthreads();
 
     // this CTA's share of the sequence's tiles: as even as whole tiles allow
@@ -171,9 +190,14 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                 // the last tile of a sequence is fetched in 16-token groups: (almost) nothing past the end is read
                 const int groups = rem >= kTileT ? kTileT / 16 : (rem + 15) / 16;
                 const uint32_t kv_bytes = rem >= kTileT ? C::kStageBytes : (uint32_t)groups * 16u * 128u * C::kHalves * 2u;
-                mbar_arrive_expect_tx(&full[s], kv_bytes + (it == 0 ? q_bytes : 0u));
-                if (it == 0)
+                mbar_arrive_expect_tx(&full[s], kv_bytes + (it == 0 ? q_bytes + (with_rope ? kRopeBytes : 0u) : 0u));
+                if (it == 0) {
                     bulk_load_1d(q_smem, p.q + ((size_t)b * p.Hq + (size_t)kvh * p.G) * D, q_bytes, &full[s]);
+                    if (with_rope) {
+                        bulk_load_1d(rope_cs, p.rope_cos + (size_t)(len - 1) * (D / 2), kRopeBytes / 2, &full[s]);
+                        bulk_load_1d(rope_cs + D / 2, p.rope_sin + (size_t)(len - 1) * (D / 2), kRopeBytes / 2, &full[s]);
+                    }
+                }
                 uint8_t *dst = stages + (size_t)s * C::kStageBytes;
                 int c1, c2, c3;
                 // a full tile is one box (or one box per page when pages are smaller than the tile); neither a
@@ -223,6 +247,7 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                     qf[ks][2] = v_lo ? qrow_lo[w + 4] : 0u;
                     qf[ks][3] = v_hi ? qrow_hi[w + 4] : 0u;
                 }
+                if (with_rope) rope_q_fragments<D>(qf, p.G, p.q_weight != nullptr, p.norm_eps, rope_cs, norm_w, lane);
             }
             const int t0 = (t_begin + it) * kTileT;
             const uint32_t k_tile = smem_u32(stages + (size_t)s * C::kStageBytes);
@@ -236,10 +261,15 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                 // one CTA owns it)
                 const int last = row0 + nvalid - 1;
                 constexpr int kChunks = D / 8;
+                uint4 kk = make_uint4(0u, 0u, 0u, 0u), vv = kk;
                 if (lane < kChunks) {
                     const size_t src = (size_t)b * p.new_sb + (size_t)kvh * p.new_sh + lane * 8;
-                    const uint4 kk = __ldg(reinterpret_cast<const uint4 *>(p.k_new + src));
-                    const uint4 vv = __ldg(reinterpret_cast<const uint4 *>(p.v_new + src));
+                    kk = __ldg(reinterpret_cast<const uint4 *>(p.k_new + src));
+                    vv = __ldg(reinterpret_cast<const uint4 *>(p.v_new + src));
+                }
+                if (p.rope_cos != nullptr)                                      // all lanes: shuffles inside
+                    kk = rope_k_row<D>(kk, p.k_weight != nullptr, p.norm_eps, rope_cs, norm_w + D, with_rope, lane);
+                if (lane < kChunks) {
                     uint8_t *kt = stages + (size_t)s * C::kStageBytes;
                     const uint32_t off = (lane >> 3) * kHalfBytes + swz128(last, lane & 7);
                     *reinterpret_cast<uint4 *>(kt + off) = kk;
@@ -484,9 +514,10 @@ int decode_cluster_width(int B, int Hq, int Hkv, int D, int max_kv_len)
 l4l_status launch_decode_cluster(const void *q, void *o, const l4l_kv_cache &cache, const int32_t *d_kv_lens,
                                  int max_kv_len, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
                                  void *workspace, cudaStream_t stream, const l4l_tensor4 *k_new,
-                                 const l4l_tensor4 *v_new, const PagedTable *paged, int width)
+                                 const l4l_tensor4 *v_new, const PagedTable *paged, const RopeArgs *rope, int width)
 {
     if (paged && (k_new || v_new)) return L4L_ERR_UNSUPPORTED;
+    if (rope && (!k_new || !v_new)) return L4L_ERR_UNSUPPORTED;      // only with the fused append
     const int G = Hq / Hkv;
     const int stages = (D == 128) ? pick_stages<128>(G) : pick_stages<64>(G);
     if (stages == 0 || width < 1 || width > kMaxCluster) return L4L_ERR_UNSUPPORTED;
@@ -529,6 +560,12 @@ l4l_status launch_decode_cluster(const void *q, void *o, const l4l_kv_cache &cac
     p.page_size = paged ? cache.max_len : 0;
     p.page_shift = 0;
     while (paged && (1 << p.page_shift) < cache.max_len) ++p.page_shift;
+    p.rope_cos = rope ? rope->cos : nullptr;
+    p.rope_sin = rope ? rope->sin : nullptr;
+    p.q_weight = rope ? rope->q_weight : nullptr;
+    p.k_weight = rope ? rope->k_weight : nullptr;
+    p.norm_eps = rope ? rope->eps : 0.f;
+    p.rope_n_pos = rope ? rope->n_pos : 0;
     p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.G = G; p.C = width; p.max_kv_len = max_kv_len; p.stages = stages;
     p.scale_log2e = scale * 1.4426950408889634f;
     p.coord = coord;

@@ -122,6 +122,14 @@ def test_cluster_decode_paged(cluster_width, page_size):
     assert_close_to_oracle(o, ref, "cluster paged decode")
 
 
+@pytest.mark.parametrize("cluster_width", WIDTHS, indirect=True)
+@pytest.mark.parametrize("D,Hq,Hkv,norm", [(128, 8, 2, True), (64, 4, 4, False), (128, 16, 1, True)])
+def test_cluster_decode_step_with_rope_and_append(cluster_width, D, Hq, Hkv, norm):
+    from test_gpu_rope_append import test_decode_step_with_rope_and_append_in_one_launch as rope_step_case
+
+    rope_step_case(D, Hq, Hkv, norm)
+
+
 def test_library_choice_matches_split_kernel_result():
     # the same call on both kernels: results agree to rounding of the merge order
     lens = [2304]
