@@ -375,6 +375,50 @@ def run_ours(args, rank, world):
 
     t_fp8 = timed(fp8_step, 21)
     del c8
+    # The decode phase of the 8B-shaped layer config (B = 1, 2048-token prompt, 256 steps): latency-bound, so the
+    # steps (cache update fused in) are replayed from a CUDA graph, as a serving loop would issue them; once on the
+    # kernel the library picks for this size (a thread-block cluster per KV head) and once held on the split kernel.
+    def small_batch_step_us(L, split_only, n=64):
+        w8 = wl.WORKLOADS["layer8b"]
+        sb = wl.make_decode_batch(w8, B=1, len_lo=L, len_hi=L, Lmax=L, poison_tail=False)
+        sq, sck, scv, slen = sb.q.to(dev), sb.cache_k.to(dev), sb.cache_v.to(dev), sb.kv_len.to(dev)
+        skn = torch.zeros(1, 1, w8.Hkv, w8.D, dtype=torch.bfloat16, device=dev)
+        so = torch.empty_like(sq)
+        sws = l4l.new_workspace(l4l.L4L_OP_DECODE, 1, w8.Hq, w8.Hkv, w8.D, L, device=dev)
+        old = os.environ.get("L4L_DECODE_CLUSTER")
+        if split_only:
+            os.environ["L4L_DECODE_CLUSTER"] = "0"
+        try:
+            fn = lambda: l4l.l4l_attn_decode_append(sq, so, sck, scv, skn, skn, slen, L, w8.scale, sws)
+            side = torch.cuda.Stream(dev)
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                fn()
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                for _ in range(n):
+                    fn()
+        finally:
+            if old is None:
+                os.environ.pop("L4L_DECODE_CLUSTER", None)
+            else:
+                os.environ["L4L_DECODE_CLUSTER"] = old
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record()
+        for _ in range(5):
+            graph.replay()
+        a1.record()
+        torch.cuda.synchronize()
+        err = l4l.l4l_last_device_error(sws)
+        return a0.elapsed_time(a1) / (5 * n) * 1e3, err
+
+    t_small, err_small = small_batch_step_us(2304, False)
+    t_small_split, err_small2 = small_batch_step_us(2304, True)
     # second workload: the RG-LRU recurrence of a RecurrentGemma-2B-sized block (2560 channels) over a long prompt
     rB, rT, rW = 4, 8192, 2560
     gen = torch.Generator(device="cpu").manual_seed(1006)
@@ -389,7 +433,7 @@ def run_ours(args, rank, world):
     rglru_bytes = rx.numel() * 8                          # 3 bf16 read + 1 written per (step, channel)
     dev_err_r = l4l.l4l_last_device_error(ws_r)
     del rx, rgx, rga, ry, filler
-    dev_err = l4l.l4l_last_device_error(ws_p) | l4l.l4l_last_device_error(ws_d) | dev_err_r
+    dev_err = l4l.l4l_last_device_error(ws_p) | l4l.l4l_last_device_error(ws_d) | dev_err_r | err_small | err_small2
 
     # ---- end to end through the same entry points with HOST buffers (pinned), copies inside the timed region
     hq, hk, hv = seq.q.pin_memory(), seq.k.pin_memory(), seq.v.pin_memory()
@@ -499,6 +543,7 @@ def run_ours(args, rank, world):
                                           "bytes": rglru_bytes},
             "decode_fp8_cache": {"us": t_fp8 * 1e3, "kv_gbs_fp8_bytes": dec_bytes / 2 / (t_fp8 * 1e-3) / 1e9,
                                  "speedup_over_bf16_cache": t_dec_b2b / t_fp8},
+            "decode_step_B1_L2304_in_cuda_graph": {"cluster_kernel_us": t_small, "split_kernel_us": t_small_split},
         },
         "gpu_launches": 3 * args.steps,
         "clocks": clocks,
@@ -514,7 +559,7 @@ def run_ours(args, rank, world):
 def run_profile_case(case: str):
     """A few launches of ONE kernel on a small case, for `ncu` captures (not a benchmark):
     prefill = B=1, S=8192 of the long_prefill workload (inputs 168 MB > L2); decode = the batched_decode batch;
-    rglru = the RG-LRU scan on B=16, T=2048, W=2560."""
+    rglru = the RG-LRU scan on B=16, T=2048, W=2560; decode_small = the cluster decode kernel on B=4 x 8192 tokens."""
     from paper_2608_21836_b200 import binding as l4l
 
     torch.cuda.set_device(0)
@@ -541,6 +586,15 @@ def run_profile_case(case: str):
         ws = l4l.new_rglru_workspace(B, T, W)
         for _ in range(3):
             l4l.l4l_rglru_scan(x, gx, ga, ap, state, y, ws)
+    elif case == "decode_small":
+        # the cluster kernel: B = 4 sequences of 8192 tokens of the 8B-shaped layer (134 MB of cache > L2)
+        w = wl.WORKLOADS["layer8b"]
+        db = wl.make_decode_batch(w, B=4, len_lo=8192, len_hi=8192, Lmax=8192, poison_tail=False)
+        q, ck, cv, lens = db.q.cuda(), db.cache_k.cuda(), db.cache_v.cuda(), db.kv_len.cuda()
+        o = torch.empty_like(q)
+        ws = l4l.new_workspace(l4l.L4L_OP_DECODE, 4, w.Hq, w.Hkv, w.D, 8192)
+        for _ in range(3):
+            l4l.l4l_attn_decode(q, o, ck, cv, lens, 8192, w.scale, ws)
     else:
         w = wl.WORKLOADS["batched_decode"]
         db = wl.make_decode_batch(w)
@@ -560,7 +614,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--profile-case", choices=["prefill", "decode", "rglru"], default=None,
+    ap.add_argument("--profile-case", choices=["prefill", "decode", "decode_small", "rglru"], default=None,
                     help="run three launches of one kernel on a small case and exit (for ncu)")
     args = ap.parse_args()
     if args.profile_case:

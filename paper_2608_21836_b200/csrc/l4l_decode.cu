@@ -969,18 +969,20 @@ DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_
     int n_dev = 0;
     const bool have_dev = cudaGetDeviceCount(&n_dev) == cudaSuccess && n_dev > 0;
     if (!have_dev) (void)cudaGetLastError();
-    // Prefer the 8-warp shape (one CTA per SM, ranges twice as long, so fewer sequences are cut between
-    // CTAs) whenever its shared memory fits, which it does for query-head groups of up to 4; else 4 warps.
+    // 128-wide heads: prefer the 8-warp shape (one CTA per SM, ranges twice as long, so fewer sequences are cut
+    // between CTAs) whenever its shared memory fits, which it does for query-head groups of up to 4; else 4 warps.
     static const int forced = [] {
         const char *e = getenv("L4L_DECODE_WARPS");      // debugging aid: force a shape
         return e ? atoi(e) : 0;
     }();
-    if (forced != 4) {
-        const DecodePlan p8 = plan_for_shape(B, Hq, Hkv, D, max_kv_len, ws_limit, 8, have_dev, fp8);
-        if (p8.fits && p8.ws_bytes <= ws_limit) return p8;
-        if (forced == 8) return p8;
-    }
-    return plan_for_shape(B, Hq, Hkv, D, max_kv_len, ws_limit, 4, have_dev, fp8);
+    // With 64-wide heads a tile carries half the bytes for the same per-tile work in the consumer warps, and two
+    // 4-warp CTAs per SM (two independent streams) hide that better than one 8-warp CTA: 4 warps first there.
+    const bool four_first = forced == 4 || (forced == 0 && D == 64);
+    const DecodePlan first = plan_for_shape(B, Hq, Hkv, D, max_kv_len, ws_limit, four_first ? 4 : 8, have_dev, fp8);
+    if ((first.fits && first.ws_bytes <= ws_limit) || forced != 0) return first;
+    const DecodePlan second = plan_for_shape(B, Hq, Hkv, D, max_kv_len, ws_limit, four_first ? 8 : 4, have_dev, fp8);
+    if (second.fits && second.ws_bytes <= ws_limit) return second;
+    return four_first ? first : second;          // neither fits: the 4-warp plan carries the diagnosis
 }
 
 l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, const int32_t *d_kv_lens,
