@@ -157,6 +157,9 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     // producer -> finisher: the pieces this CTA has started, in order (so that the finisher can look at a
     // piece's ticket while the piece is still being streamed)
     volatile uint32_t *posted_count = reinterpret_cast<volatile uint32_t *>(abort_flag + 1);
+    // producer -> finisher: how many pieces this CTA has in all (known once the last one has been started); the
+    // finisher leaves right after the last one
+    volatile uint32_t *pieces_total = posted_count + 1;
     PieceMeta *post_ring = reinterpret_cast<PieceMeta *>(lens_s + kMaxB + 4);
 
     const int warp = threadIdx.x >> 5;
@@ -171,6 +174,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
         mbar_init(comb_empty, 1);
         *abort_flag = 0;
         *posted_count = 0u;
+        *pieces_total = 0xffffffffu;
         fence_barrier_init();
         fence_proxy_async_smem();
     }
@@ -235,25 +239,41 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             const int my_end = range_begin((int)blockIdx.x + 1);
             uint32_t it = 0, n_posted = 0;
             bool ok = true;
-            // The walk over this CTA's pieces: the first one is located by a binary search over the prefix sums, every
+            // Order of work. If the range ends inside a sequence (the next CTA holds its tail and, walking forward,
+            // takes it first), that last piece is streamed FIRST and the rest of the range after it: both halves
+            // of a cut sequence are then finished early, their merge through the workspace (several round trips
+            // through a memory system that is saturated by the streams) happens in the background, and what a CTA
+            // ends with is a whole sequence or a tail whose head was finished long ago: no global round trip at
+            // the end of the kernel.
+            auto locate = [&](int g, int &b_, int &kvh_, int &len_, int &tiles_, int &first_) {
+                int lo = 0, hi = p.B;              // largest b with cum[b] <= g
+                while (hi - lo > 1) {
+                    const int mid = (lo + hi) >> 1;
+                    if (cum[mid] <= g) lo = mid; else hi = mid;
+                }
+                b_ = lo;
+                len_ = lens_s[lo];
+                tiles_ = (len_ + kTileT - 1) / kTileT;
+                kvh_ = (g - cum[lo]) / (tiles_ + 1);
+                first_ = cum[lo] + kvh_ * (tiles_ + 1);          // flattened index of this sequence's marker; tile t at +1+t
+            };
+            int b = 0, kvh = 0, len = 0, tiles_b = 0, seq_first = 0;
+            int split = my_end;                    // [split, my_end) goes first, then [my_begin, split)
+            if (my_end > my_begin) {
+                locate(my_end - 1, b, kvh, len, tiles_b, seq_first);
+                if (my_end - 1 > seq_first && seq_first + tiles_b + 1 > my_end) split = max(seq_first, my_begin);
+            }
+            // The walk over a range's pieces: the first one is located by a binary search over the prefix sums, every
             // later one starts a sequence (the next KV head of the same sequence, or the next sequence with tokens),
             // so its numbers follow from the previous piece without a search or a division.
-            int g = my_begin;
-            int b = 0, kvh = 0, len = 0, tiles_b = 0, seq_first = 0;
+            for (int pass = (split < my_end ? 0 : 1); pass < 2 && ok; ++pass) {
+            int g = pass == 0 ? split : my_begin;
+            const int g_end = pass == 0 ? my_end : split;
             bool located = false;
-            while (ok && g < my_end) {
+            while (ok && g < g_end) {
                 int first_cta;
                 if (!located) {
-                    int lo = 0, hi = p.B;          // largest b with cum[b] <= g
-                    while (hi - lo > 1) {
-                        const int mid = (lo + hi) >> 1;
-                        if (cum[mid] <= g) lo = mid; else hi = mid;
-                    }
-                    b = lo;
-                    len = lens_s[b];
-                    tiles_b = (len + kTileT - 1) / kTileT;
-                    kvh = (g - cum[b]) / (tiles_b + 1);
-                    seq_first = cum[b] + kvh * (tiles_b + 1);    // flattened index of this sequence's marker; tile t at +1+t
+                    if (pass == 1) locate(g, b, kvh, len, tiles_b, seq_first);   // pass 0 starts in the piece located above
                     first_cta = cta_of(seq_first + 1);
                     located = true;
                 } else {
@@ -267,7 +287,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     first_cta = (int)blockIdx.x;
                 }
                 const int tile_begin = max(g - seq_first - 1, 0);
-                const int tile_end = min(tiles_b, my_end - seq_first - 1);
+                const int tile_end = min(tiles_b, g_end - seq_first - 1);
                 if (tile_end <= tile_begin) break;                // only the marker fell into this range (at its very end)
                 const int npieces = (seq_first + tiles_b + 1 <= my_end) ? (int)blockIdx.x - first_cta + 1
                                                                         : cta_of(seq_first + tiles_b) - first_cta + 1;
@@ -340,6 +360,9 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 }
                 g = seq_first + 1 + tile_end;
             }
+            }
+            __threadfence_block();
+            *pieces_total = n_posted;
             if (ok) {
                 const uint32_t s = it % C::kStages;
                 const uint32_t ph = (it / C::kStages) & 1u;
@@ -370,16 +393,18 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             {
                 // every decision in this loop is taken by lane 0 and broadcast, so that the warp stays converged
                 const long long t0 = clock64();
-                bool have_post = false, dead = false;
+                bool have_post = false, dead = false, all_done = false;
                 while (true) {
                     int st = 0;                                       // 0: keep polling
                     if (lane == 0) {
-                        if (mbar_try_wait(comb_full, n & 1u)) st = 1;                                  // piece complete
+                        if (*pieces_total == n) st = 4;                                                // nothing left
+                        else if (mbar_try_wait(comb_full, n & 1u)) st = 1;                             // piece complete
                         else if (*abort_flag || clock64() - t0 > kWaitCycleBudget) st = 3;             // give up
                         else if (!have_post && (int32_t)(*posted_count - (n + 1u)) >= 0) st = 2;       // piece started
                     }
                     st = __shfl_sync(0xffffffffu, st, 0);
                     if (st == 1) break;
+                    if (st == 4) { all_done = true; break; }
                     if (st == 3) { dead = true; break; }
                     if (st == 2) {
                         have_post = true;
@@ -417,60 +442,84 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     *abort_flag = 1;
                     break;
                 }
+                if (all_done) break;
                 __syncwarp();                                         // lane 0's acquire covers the warp
             }
             const PieceMeta pm = *piece_meta;
-            if (pm.stop) break;
             const bool single = (pm.npieces == 1);
             const size_t bh0 = (size_t)pm.b * p.Hq + pm.kvh * p.G;
             int *tk = p.tickets + (size_t)pm.b * p.Hkv + pm.kvh;
             const int np = pm.npieces;
 
-            if (prefetched) {
-                // ---- this piece completes its sequence: merge the four warps' results, fold in the other
-                // pieces' partials fetched above, write the final output; nothing goes through the workspace
+            // ---- merge of the consumer warps' (max, sum, O). With at most 128 float4 outputs per piece (the usual
+            // case) a lane owns up to four of them and works on all four in lockstep, stage by stage, so that the
+            // four dependent chains overlap; the result is unnormalised, relative to the row maximum mloc.
+            float4 acc4[4];
+            float lsum4[4], mloc4[4];
+            int r4[4], d4s[4];
+            bool on4[4];
+            if (few_items) {
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     const int item = u * 32 + lane;
-                    if (item < p.G * kVec) {
-                        const int r = item / kVec, d4 = item % kVec;
-                        float mw[kConsumerWarps];
-                        float mloc = -INFINITY;
+                    on4[u] = item < p.G * kVec;
+                    r4[u] = on4[u] ? item / kVec : 0;
+                    d4s[u] = on4[u] ? item % kVec : 0;
+                    mloc4[u] = -INFINITY;
+                    acc4[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    lsum4[u] = 0.f;
+                }
 #pragma unroll
-                        for (int w = 0; w < kConsumerWarps; ++w) {
-                            mw[w] = comb[((size_t)w * p.G + r) * kPitch + D];
-                            mloc = fmaxf(mloc, mw[w]);
-                        }
-                        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                        float lsum = 0.f;
+                for (int w = 0; w < kConsumerWarps; ++w)
 #pragma unroll
-                        for (int w = 0; w < kConsumerWarps; ++w) {
-                            const float *row = comb + ((size_t)w * p.G + r) * kPitch;
-                            const float wgt = fast_exp2(mw[w] - mloc);
-                            const float4 v = *reinterpret_cast<const float4 *>(row + d4 * 4);
-                            acc.x += wgt * v.x; acc.y += wgt * v.y; acc.z += wgt * v.z; acc.w += wgt * v.w;
-                            lsum += wgt * row[D + 1];
-                        }
-                        // own piece in the same form as the stored partials: normalised output + log2-sum-exp
-                        const float inv_own = 1.f / lsum;
-                        const float lse_own = mloc + log2f(lsum);
-                        float mstar = fmaxf(lse_own, fmaxf(fmaxf(sl[u][0], sl[u][1]), fmaxf(sl[u][2], sl[u][3])));
-                        const float w_own = fast_exp2(lse_own - mstar) * inv_own;
-                        float4 out = make_float4(acc.x * w_own, acc.y * w_own, acc.z * w_own, acc.w * w_own);
-                        float wsum = fast_exp2(lse_own - mstar);
+                    for (int u = 0; u < 4; ++u)
+                        mloc4[u] = fmaxf(mloc4[u], comb[((size_t)w * p.G + r4[u]) * kPitch + D]);
 #pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            const float wc = fast_exp2(sl[u][c] - mstar);          // absent piece: 2^-inf = 0
-                            out.x += wc * sv[u][c].x; out.y += wc * sv[u][c].y;
-                            out.z += wc * sv[u][c].z; out.w += wc * sv[u][c].w;
-                            wsum += wc;
-                        }
-                        const float inv = 1.f / wsum;
+                for (int w = 0; w < kConsumerWarps; ++w)
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const float *row = comb + ((size_t)w * p.G + r4[u]) * kPitch;
+                        const float wgt = fast_exp2(row[D] - mloc4[u]);    // warp that saw no token: max = -inf -> 0
+                        const float4 v = *reinterpret_cast<const float4 *>(row + d4s[u] * 4);
+                        acc4[u].x += wgt * v.x; acc4[u].y += wgt * v.y; acc4[u].z += wgt * v.z; acc4[u].w += wgt * v.w;
+                        lsum4[u] += wgt * row[D + 1];
+                    }
+            }
+
+            if (prefetched) {
+                // ---- this piece completes its sequence: fold in the other pieces' partials fetched above and write
+                // the final output; nothing goes through the workspace (prefetched implies few_items)
+                float4 out4[4];
+                float wsum4[4], mstar4[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    // own piece in the same form as the stored partials: normalised output + log2-sum-exp
+                    const float inv_own = 1.f / lsum4[u];
+                    const float lse_own = mloc4[u] + log2f(lsum4[u]);
+                    mstar4[u] = fmaxf(lse_own, fmaxf(fmaxf(sl[u][0], sl[u][1]), fmaxf(sl[u][2], sl[u][3])));
+                    const float e_own = fast_exp2(lse_own - mstar4[u]);
+                    const float w_own = e_own * inv_own;
+                    out4[u] = make_float4(acc4[u].x * w_own, acc4[u].y * w_own, acc4[u].z * w_own, acc4[u].w * w_own);
+                    wsum4[u] = e_own;
+                }
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const float wc = fast_exp2(sl[u][c] - mstar4[u]);          // absent piece: 2^-inf = 0
+                        out4[u].x += wc * sv[u][c].x; out4[u].y += wc * sv[u][c].y;
+                        out4[u].z += wc * sv[u][c].z; out4[u].w += wc * sv[u][c].w;
+                        wsum4[u] += wc;
+                    }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    if (on4[u]) {
+                        const float inv = 1.f / wsum4[u];
                         uint2 packed;
-                        packed.x = pack_bf16x2(out.x * inv, out.y * inv);
-                        packed.y = pack_bf16x2(out.z * inv, out.w * inv);
-                        *reinterpret_cast<uint2 *>(p.o + (bh0 + r) * D + d4 * 4) = packed;
-                        if (d4 == 0 && p.lse) p.lse[bh0 + r] = (mstar + log2f(wsum)) * 0.6931471805599453f;
+                        packed.x = pack_bf16x2(out4[u].x * inv, out4[u].y * inv);
+                        packed.y = pack_bf16x2(out4[u].z * inv, out4[u].w * inv);
+                        *reinterpret_cast<uint2 *>(p.o + (bh0 + r4[u]) * D + d4s[u] * 4) = packed;
+                        if (d4s[u] == 0 && p.lse) p.lse[bh0 + r4[u]] = (mstar4[u] + log2f(wsum4[u])) * 0.6931471805599453f;
                     }
                 }
                 __syncwarp();
@@ -481,26 +530,9 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 continue;
             }
 
-            // merge the four consumer warps' (max, sum, O); each lane owns float4 pieces of the G x D outputs
-            for (int item = lane; item < p.G * kVec; item += 32) {
-                const int r = item / kVec, d4 = item % kVec;
-                float mw[kConsumerWarps];
-                float mstar = -INFINITY;
-#pragma unroll
-                for (int w = 0; w < kConsumerWarps; ++w) {
-                    mw[w] = comb[((size_t)w * p.G + r) * kPitch + D];
-                    mstar = fmaxf(mstar, mw[w]);
-                }
-                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                float lsum = 0.f;
-#pragma unroll
-                for (int w = 0; w < kConsumerWarps; ++w) {
-                    const float *row = comb + ((size_t)w * p.G + r) * kPitch;
-                    const float wgt = fast_exp2(mw[w] - mstar);    // warp that saw no token: max = -inf -> 0
-                    const float4 v = *reinterpret_cast<const float4 *>(row + d4 * 4);
-                    acc.x += wgt * v.x; acc.y += wgt * v.y; acc.z += wgt * v.z; acc.w += wgt * v.w;
-                    lsum += wgt * row[D + 1];
-                }
+            // this piece alone: straight to the output if it is the whole sequence, else (normalised, with its
+            // log2-sum-exp) to the workspace
+            auto emit = [&](int r, int d4, float4 acc, float lsum, float mstar) {
                 const float inv = 1.f / lsum;
                 acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
                 const size_t bh = bh0 + r;
@@ -515,6 +547,33 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     const size_t slot = bh * p.nsplit + pm.piece;
                     *reinterpret_cast<float4 *>(p.part_o + slot * D + d4 * 4) = acc;
                     if (d4 == 0) p.part_lse[slot] = lse2;
+                }
+            };
+            if (few_items) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (on4[u]) emit(r4[u], d4s[u], acc4[u], lsum4[u], mloc4[u]);
+            } else {
+                for (int item = lane; item < p.G * kVec; item += 32) {
+                    const int r = item / kVec, d4 = item % kVec;
+                    float mw[kConsumerWarps];
+                    float mstar = -INFINITY;
+#pragma unroll
+                    for (int w = 0; w < kConsumerWarps; ++w) {
+                        mw[w] = comb[((size_t)w * p.G + r) * kPitch + D];
+                        mstar = fmaxf(mstar, mw[w]);
+                    }
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                    float lsum = 0.f;
+#pragma unroll
+                    for (int w = 0; w < kConsumerWarps; ++w) {
+                        const float *row = comb + ((size_t)w * p.G + r) * kPitch;
+                        const float wgt = fast_exp2(mw[w] - mstar);    // warp that saw no token: max = -inf -> 0
+                        const float4 v = *reinterpret_cast<const float4 *>(row + d4 * 4);
+                        acc.x += wgt * v.x; acc.y += wgt * v.y; acc.z += wgt * v.z; acc.w += wgt * v.w;
+                        lsum += wgt * row[D + 1];
+                    }
+                    emit(r, d4, acc, lsum, mstar);
                 }
             }
             __syncwarp();
@@ -648,15 +707,8 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             const uint32_t ph = (it / C::kStages) & 1u;
             if (!mbar_wait(&full[s], ph, abort_flag)) break;
             const TileMeta mt = meta[s];
-            if (mt.flags & kFlagStop) {
-                // tell the finisher to stop (after it has drained the previous piece)
-                if (mbar_wait(comb_empty, (n_dumps & 1u) ^ 1u, abort_flag)) {
-                    if (warp == 0 && lane == 0) piece_meta->stop = 1;
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(comb_full);
-                }
-                break;
-            }
+            // end of this CTA's range: nothing to tell the finisher, which knows the number of pieces from the producer
+            if (mt.flags & kFlagStop) break;
 
             if (mt.flags & kFlagFirst) {
                 st.reset();
