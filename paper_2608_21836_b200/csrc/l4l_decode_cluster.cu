@@ -52,6 +52,7 @@ struct ClusterParams {
     unsigned *status;
     const int32_t *block_table;               // paged cache (null: contiguous)
     int table_stride, page_size, page_shift;
+    int tail_rows;                            // tokens per box of the tail maps (32, or the page size if that is smaller)
     // rotary embedding (+ optional RMS norm) of the step's q and k_new (null: inputs are final); only with the fused
     // append. The new token's position is kv_len - 1.
     const float *rope_cos, *rope_sin;         // [rope_n_pos, D/2]
@@ -116,7 +117,7 @@ __device__ __forceinline__ float2 ld_cluster_f2(uint32_t addr)
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
-                      const __grid_constant__ CUtensorMap tmap_k16, const __grid_constant__ CUtensorMap tmap_v16,
+                      const __grid_constant__ CUtensorMap tmap_k_tail, const __grid_constant__ CUtensorMap tmap_v_tail,
                       const ClusterParams p)
 {
     using C = ClusterCfg<D>;
@@ -154,8 +155,8 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
     if (warp == kW && lane == 0) {
         tma_prefetch_desc(&tmap_k);
         tma_prefetch_desc(&tmap_v);
-        tma_prefetch_desc(&tmap_k16);
-        tma_prefetch_desc(&tmap_v16);
+        tma_prefetch_desc(&tmap_k_tail);
+        tma_prefetch_desc(&tmap_v_tail);
     }
     // Programmatic dependent launch: everything above overlaps the tail of the previous kernel of the stream
     grid_dependency_wait();
@@ -186,10 +187,17 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                 const int tile = t_begin + it;
                 const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
                 if (!mbar_wait(&empty[s], ph ^ 1u, abort_flag)) break;
+                // The last tile of a sequence: if at most half of it holds tokens it comes in groups of p.tail_rows
+                // tokens (a few small boxes), else as a whole tile like the others (rows past the end of the sequence are
+                // never looked at, rows past the end of the cache arrive as zeros); with pages smaller than a tile only
+                // the pages that hold tokens are fetched. Neither a box nor a group straddles pages.
                 const int rem = len - tile * kTileT;
-                // the last tile of a sequence is fetched in 16-token groups: (almost) nothing past the end is read
-                const int groups = rem >= kTileT ? kTileT / 16 : (rem + 15) / 16;
-                const uint32_t kv_bytes = rem >= kTileT ? C::kStageBytes : (uint32_t)groups * 16u * 128u * C::kHalves * 2u;
+                const int groups = (rem + p.tail_rows - 1) / p.tail_rows;
+                const bool by_groups = rem < kTileT && groups * p.tail_rows * 2 <= kTileT;
+                const int box_rows = by_groups ? p.tail_rows : ((paged && p.page_size < kTileT) ? p.page_size : kTileT);
+                const int n_box = by_groups ? groups : ((rem >= kTileT || box_rows == kTileT) ? kTileT / box_rows
+                                                                                              : (rem + box_rows - 1) / box_rows);
+                const uint32_t kv_bytes = (uint32_t)n_box * box_rows * 128u * C::kHalves * 2u;
                 mbar_arrive_expect_tx(&full[s], kv_bytes + (it == 0 ? q_bytes + (with_rope ? kRopeBytes : 0u) : 0u));
                 if (it == 0) {
                     bulk_load_1d(q_smem, p.q + ((size_t)b * p.Hq + (size_t)kvh * p.G) * D, q_bytes, &full[s]);
@@ -200,12 +208,8 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                 }
                 uint8_t *dst = stages + (size_t)s * C::kStageBytes;
                 int c1, c2, c3;
-                // a full tile is one box (or one box per page when pages are smaller than the tile); neither a
-                // box nor a 16-token group straddles pages: page sizes are powers of two >= 16
-                const int box_rows = rem >= kTileT ? ((paged && p.page_size < kTileT) ? p.page_size : kTileT) : 16;
-                const int n_box = rem >= kTileT ? kTileT / box_rows : groups;
-                const CUtensorMap *tk = rem >= kTileT ? &tmap_k : &tmap_k16;
-                const CUtensorMap *tv = rem >= kTileT ? &tmap_v : &tmap_v16;
+                const CUtensorMap *tk = by_groups ? &tmap_k_tail : &tmap_k;
+                const CUtensorMap *tv = by_groups ? &tmap_v_tail : &tmap_v;
                 int page_of[kTileT / 16];                            // looked up together: independent loads
 #pragma unroll
                 for (int bx = 0; bx < kTileT / 16; ++bx)
@@ -524,19 +528,20 @@ l4l_status launch_decode_cluster(const void *q, void *o, const l4l_kv_cache &cac
     const size_t smem = (D == 128) ? cluster_smem_bytes<128>(G, stages) : cluster_smem_bytes<64>(G, stages);
     if (!((D == 128) ? configure_kernel<128>() : configure_kernel<64>())) return L4L_ERR_CUDA;
 
-    CUtensorMap tk, tv, tk16, tv16;   // tile-sized boxes, and 16-token boxes for the last tile of a sequence
+    CUtensorMap tk, tv, tk_tail, tv_tail;   // tile-sized boxes, and small boxes for a mostly empty last tile of a sequence
     TmapCoord coord, coord_v;
     const int outer = paged ? paged->num_pages : B;
     // pages smaller than a tile are fetched page by page: no box may exceed the page
     const int box_t = (paged && cache.max_len < kTileT) ? cache.max_len : kTileT;
+    const int tail_rows = (paged && cache.max_len < 32) ? cache.max_len : 32;
     if (!make_tmap(&tk, &coord, cache.k, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h, cache.stride_b, 64,
                    box_t, 2) ||
         !make_tmap(&tv, &coord_v, cache.v, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h, cache.stride_b,
                    64, box_t, 2) ||
-        !make_tmap(&tk16, &coord_v, cache.k, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
-                   cache.stride_b, 64, 16, 2) ||
-        !make_tmap(&tv16, &coord_v, cache.v, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
-                   cache.stride_b, 64, 16, 2))
+        !make_tmap(&tk_tail, &coord_v, cache.k, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
+                   cache.stride_b, 64, tail_rows, 2) ||
+        !make_tmap(&tv_tail, &coord_v, cache.v, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
+                   cache.stride_b, 64, tail_rows, 2))
         return L4L_ERR_CUDA;
     ClusterParams p;
     p.q = static_cast<const __nv_bfloat16 *>(q);
@@ -558,6 +563,7 @@ l4l_status launch_decode_cluster(const void *q, void *o, const l4l_kv_cache &cac
     p.block_table = paged ? paged->block_table : nullptr;
     p.table_stride = paged ? paged->table_stride : 0;
     p.page_size = paged ? cache.max_len : 0;
+    p.tail_rows = tail_rows;
     p.page_shift = 0;
     while (paged && (1 << p.page_shift) < cache.max_len) ++p.page_shift;
     p.rope_cos = rope ? rope->cos : nullptr;
@@ -582,8 +588,8 @@ l4l_status launch_decode_cluster(const void *q, void *o, const l4l_kv_cache &cac
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    const cudaError_t err = (D == 128) ? cudaLaunchKernelEx(&cfg, decode_cluster_kernel<128>, tk, tv, tk16, tv16, p)
-                                       : cudaLaunchKernelEx(&cfg, decode_cluster_kernel<64>, tk, tv, tk16, tv16, p);
+    const cudaError_t err = (D == 128) ? cudaLaunchKernelEx(&cfg, decode_cluster_kernel<128>, tk, tv, tk_tail, tv_tail, p)
+                                       : cudaLaunchKernelEx(&cfg, decode_cluster_kernel<64>, tk, tv, tk_tail, tv_tail, p);
     return err == cudaSuccess ? L4L_OK : L4L_ERR_CUDA;
 }
 
