@@ -298,7 +298,10 @@ l4l_status l4l_attn_prefill_chunk(l4l_tensor4 q, l4l_tensor4 o, l4l_kv_cache cac
  * already been appended and is included), query head h:
  *     o[b, h, :] = softmax_j( scale * q[b, h, :] . K[b, h/G, j, :],  j = 0..n-1 ) @ V[b, h/G, 0..n-1, :]
  * with no mask. n = 0 gives o = 0 and lse = -inf. Cache slots >= n are never allowed to
- * influence the result, whatever bits they hold.
+ * influence the result, whatever bits they hold (slots up to the end of the 256-token block that
+ * holds slot n-1 may be READ, inside cache.max_len only). Small batches (every (sequence, KV head)
+ * on its own thread-block cluster at once) run a kernel that merges through shared memory and
+ * leaves the workspace's partials unused; the workspace is required all the same.
  *   q, o         dense [B, Hq, D]
  *   d_kv_lens    device int32 [B], each 0 <= n <= max_kv_len
  *   max_kv_len   host upper bound of kv_lens (<= cache.max_len); used to size the split
