@@ -1048,12 +1048,12 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
     const int esz = fp8 ? 1 : 2;
     // paged: `cache` describes the page pool (stride_b = stride between pages, max_len = page size)
     if (paged && (k_new || v_new)) return L4L_ERR_UNSUPPORTED;
-    if (!fp8) {
+    {
         // small batches are latency-bound: one cluster per (sequence, KV head), no workspace round trips
-        const int width = decode_cluster_width(B, Hq, Hkv, D, max_kv_len);
+        const int width = decode_cluster_width(B, Hq, Hkv, D, max_kv_len, fp8 != nullptr);
         if (width > 0)
             return launch_decode_cluster(q, o, cache, d_kv_lens, max_kv_len, B, Hq, Hkv, D, scale, d_lse, workspace,
-                                         stream, k_new, v_new, paged, rope, width);
+                                         stream, k_new, v_new, paged, rope, fp8, width);
     }
     const int G = Hq / Hkv;
     const ShapeOps ops = pick_shape(D, plan.warps, fp8 != nullptr);

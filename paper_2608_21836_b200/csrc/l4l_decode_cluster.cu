@@ -13,9 +13,11 @@
 //   warps 0-7   16 tokens of every tile each, all query heads of the KV group as the M dimension of the warp
 //               MMAs (the same building blocks as the split kernel), fused append of the step's new token
 //
-// bf16 cache, contiguous or paged, with or without the rotary embedding (+ RMS norm) of the step's q and k fused
-// in. The fp8 cache stays on the split kernel.
+// bf16 cache (contiguous or paged, with or without the fused append and the rotary embedding (+ RMS norm) of the step's
+// q and k) or fp8 (e4m3) cache with per-KV-head scales (contiguous or paged; 256-token tiles, 32 tokens per warp and
+// tile, bytes widened to f16 in registers as in the split kernel).
 #include <cstdlib>
+#include <mutex>
 
 #include "l4l_internal.h"
 #include "l4l_rope_frag.cuh"
@@ -26,18 +28,23 @@ namespace l4l {
 namespace {
 
 constexpr int kW = 8;                          // consumer warps
-constexpr int kTileT = 16 * kW;                // tokens per tile
 constexpr int kThreads = (kW + 1) * 32;
 constexpr int kMaxCluster = 8;             // the portable limit; wider clusters schedule in too few places to pay
-constexpr uint32_t kHalfBytes = kTileT * 128;  // [tile tokens][64 bf16], swizzled
 
-template <int D>
+// F8: the cache holds e4m3 bytes (one byte per value, head_dim 128); a consumer warp then takes 32 tokens per tile.
+template <int D, bool F8>
 struct ClusterCfg {
-    static constexpr int kHalves = D / 64;
+    static_assert(!F8 || D == 128, "the fp8 path wants one 128-byte row per token");
+    static constexpr int kSub = F8 ? 2 : 1;                          // 16-token blocks a consumer warp takes per tile
+    static constexpr int kTileT = 16 * kW * kSub;                    // tokens per tile
+    static constexpr int kRowBytes = F8 ? D : 2 * D;                 // one token of one KV head
+    static constexpr int kHalves = kRowBytes / 128;                  // 128-byte column blocks of a tile
+    static constexpr int kBoxD = F8 ? 128 : 64;                      // elements per 128-byte box row
+    static constexpr uint32_t kHalfBytes = kTileT * 128;             // [tile tokens][128 bytes], swizzled
     static constexpr uint32_t kTileBytes = kHalves * kHalfBytes;     // one of K or V
     static constexpr uint32_t kStageBytes = 2 * kTileBytes;
     static constexpr int kPitch = D + 4;                             // floats per row: O[D], max, sum, pad
-    static constexpr int kMaxStages = (D == 128) ? 3 : 6;
+    static constexpr int kMaxStages = (kStageBytes >= 65536u) ? 3 : 6;
 };
 
 struct ClusterParams {
@@ -59,15 +66,16 @@ struct ClusterParams {
     const float *q_weight, *k_weight;         // [D] or null
     float norm_eps;
     int rope_n_pos;
+    const float *k_scale, *v_scale;           // fp8 cache: real value = e4m3 value * scale of its KV head, [Hkv]
     int B, Hq, Hkv, G, C, max_kv_len, stages;
     float scale_log2e;
     TmapCoord coord;
 };
 
-template <int D>
+template <int D, bool F8>
 size_t cluster_smem_bytes(int G, int stages)
 {
-    using C = ClusterCfg<D>;
+    using C = ClusterCfg<D, F8>;
     return 1024 /*alignment slack*/ + (size_t)stages * C::kStageBytes + (size_t)G * D * 2 +
            (size_t)(kW + 1) * G * C::kPitch * sizeof(float) + 3 * D * sizeof(float) +
            2 * C::kMaxStages * sizeof(uint64_t) + 64;
@@ -114,14 +122,15 @@ __device__ __forceinline__ float2 ld_cluster_f2(uint32_t addr)
     return v;
 }
 
-template <int D>
+template <int D, bool F8>
 __global__ void __launch_bounds__(kThreads, 1)
 decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
                       const __grid_constant__ CUtensorMap tmap_k_tail, const __grid_constant__ CUtensorMap tmap_v_tail,
                       const ClusterParams p)
 {
-    using C = ClusterCfg<D>;
-    constexpr int kPitch = C::kPitch, kVec = D / 4;
+    using C = ClusterCfg<D, F8>;
+    constexpr int kPitch = C::kPitch, kVec = D / 4, kTileT = C::kTileT;
+    constexpr uint32_t kHalfBytes = C::kHalfBytes;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     // the same offset in every CTA of the cluster (the dynamic segment starts at the same shared address)
@@ -223,8 +232,8 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                     uint8_t *db = dst + bx * box_rows * 128;          // whole 8-row groups: the swizzle phase is kept
 #pragma unroll
                     for (int hf = 0; hf < C::kHalves; ++hf) {
-                        tma_load_4d(db + hf * kHalfBytes, tk, &full[s], hf * 64, c1, c2, c3);
-                        tma_load_4d(db + C::kTileBytes + hf * kHalfBytes, tv, &full[s], hf * 64, c1, c2, c3);
+                        tma_load_4d(db + hf * kHalfBytes, tk, &full[s], hf * C::kBoxD, c1, c2, c3);
+                        tma_load_4d(db + C::kTileBytes + hf * kHalfBytes, tv, &full[s], hf * C::kBoxD, c1, c2, c3);
                     }
                 }
             }
@@ -235,6 +244,11 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
         st.reset();
         uint32_t qf[D / 16][4];
         const int r_lo = lane >> 2, r_hi = r_lo + 8;    // query heads of the group held in rows lane/4, lane/4 + 8
+        float k_sc = 1.f, v_sc = 1.f;                   // fp8 cache: scales of this KV head
+        if constexpr (F8) {
+            k_sc = __ldg(p.k_scale + kvh);
+            v_sc = __ldg(p.v_scale + kvh);
+        }
         for (int it = 0; it < n_mine; ++it) {
             const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
             if (!mbar_wait(&full[s], ph, abort_flag)) break;
@@ -245,21 +259,31 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                 const bool v_lo = r_lo < p.G, v_hi = r_hi < p.G;
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
-                    const int w = ks * 8 + (lane & 3);               // 32-bit word index in the row
-                    qf[ks][0] = v_lo ? qrow_lo[w] : 0u;
-                    qf[ks][1] = v_hi ? qrow_hi[w] : 0u;
-                    qf[ks][2] = v_lo ? qrow_lo[w + 4] : 0u;
-                    qf[ks][3] = v_hi ? qrow_hi[w + 4] : 0u;
+                    if constexpr (F8) {
+                        // f16 fragments with the k index permuted the way the fp8 K tiles arrive
+                        const int w = q_frag_f8_word(ks, 0, lane);
+                        qf[ks][0] = v_lo ? bf16x2_to_f16x2(qrow_lo[w]) : 0u;
+                        qf[ks][1] = v_hi ? bf16x2_to_f16x2(qrow_hi[w]) : 0u;
+                        qf[ks][2] = v_lo ? bf16x2_to_f16x2(qrow_lo[w + 1]) : 0u;
+                        qf[ks][3] = v_hi ? bf16x2_to_f16x2(qrow_hi[w + 1]) : 0u;
+                    } else {
+                        const int w = ks * 8 + (lane & 3);           // 32-bit word index in the row
+                        qf[ks][0] = v_lo ? qrow_lo[w] : 0u;
+                        qf[ks][1] = v_hi ? qrow_hi[w] : 0u;
+                        qf[ks][2] = v_lo ? qrow_lo[w + 4] : 0u;
+                        qf[ks][3] = v_hi ? qrow_hi[w + 4] : 0u;
+                    }
                 }
-                if (with_rope) rope_q_fragments<D>(qf, p.G, p.q_weight != nullptr, p.norm_eps, rope_cs, norm_w, lane);
+                if constexpr (!F8)
+                    if (with_rope) rope_q_fragments<D>(qf, p.G, p.q_weight != nullptr, p.norm_eps, rope_cs, norm_w, lane);
             }
             const int t0 = (t_begin + it) * kTileT;
             const uint32_t k_tile = smem_u32(stages + (size_t)s * C::kStageBytes);
             const uint32_t v_tile = k_tile + C::kTileBytes;
-            const int row0 = warp * 16;
+            const int row0 = warp * 16 * C::kSub;
             const int nvalid = len - (t0 + row0);                    // valid tokens in this warp's slice
             bool wrote_smem = false;
-            if (p.k_new != nullptr && nvalid > 0 && nvalid <= 16) {
+            if (!F8 && p.k_new != nullptr && nvalid > 0 && nvalid <= 16) {
                 // fused append: this slice holds the sequence's newest token. Its K/V arrive from the caller, not
                 // from the cache: patch the tile in shared memory and write the cache slot (exactly one warp of
                 // one CTA owns it)
@@ -285,7 +309,50 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                 wrote_smem = true;
                 __syncwarp();
             }
-            if (nvalid > 0) {
+            if constexpr (F8) {
+                if (nvalid > 0) {
+                    // 32 tokens per step: two 16-token blocks share one softmax update. A block with no valid token is
+                    // skipped (its rows may never have been fetched); in the last valid block the tokens past the end
+                    // get no weight and their V rows are cleared.
+                    constexpr int kSub = C::kSub;
+                    float sv[2 * kSub][4];
+                    const float sc = p.scale_log2e * k_sc;
+#pragma unroll
+                    for (int u = 0; u < kSub; ++u) {
+                        if (u == 0 || nvalid > 16 * u) {
+                            warp_qk_16x16_f8<D>(qf, k_tile, row0 + 16 * u, sv[2 * u], sv[2 * u + 1]);
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                sv[2 * u][e] *= sc;
+                                sv[2 * u + 1][e] *= sc;
+                            }
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) sv[2 * u][e] = sv[2 * u + 1][e] = -INFINITY;
+                        }
+                    }
+                    if (nvalid < 16 * kSub) {
+                        const int tok = 2 * (lane & 3);
+#pragma unroll
+                        for (int j = 0; j < 2 * kSub; ++j)
+#pragma unroll
+                            for (int e = 0; e < 4; ++e)
+                                if (8 * j + tok + (e & 1) >= nvalid) sv[j][e] = -INFINITY;
+                        uint8_t *vt = stages + (size_t)s * C::kStageBytes + C::kTileBytes;
+                        const int fetched_end = (nvalid + 15) & ~15;                 // end of the last valid block
+                        for (int i = lane; i < (fetched_end - nvalid) * 8; i += 32)
+                            *reinterpret_cast<uint4 *>(vt + (row0 + nvalid + i / 8) * 128 + ((i & 7) << 4)) =
+                                make_uint4(0u, 0u, 0u, 0u);
+                        wrote_smem = true;
+                        __syncwarp();
+                    }
+                    uint32_t pa[kSub][4];
+                    warp_softmax_tiles<D, true, 2 * kSub>(st, sv, pa);
+#pragma unroll
+                    for (int u = 0; u < kSub; ++u)
+                        if (u == 0 || nvalid > 16 * u) warp_pv_16x16_f8<D>(st, pa[u], v_tile, row0 + 16 * u);
+                }
+            } else if (nvalid > 0) {
                 float s_lo[4], s_hi[4];
                 warp_qk_16x16<D>(qf, k_tile, kHalfBytes, row0, s_lo, s_hi);
                 const int tok = 2 * (lane & 3);
@@ -327,19 +394,36 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
         l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
         l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
         float *cw = comb + (size_t)warp * p.G * kPitch;
+        // fp8: accumulator tiles alternate even / odd head dims (a tile pair gives this lane 4 consecutive dims) and O
+        // still lacks the V scale of its KV head
+        const float vs = F8 ? v_sc : 1.f;
         if (r_lo < p.G) {
             float *row = cw + (size_t)r_lo * kPitch;
             if ((lane & 3) == 0) { row[D] = st.m[0]; row[D + 1] = l0; }
+            if constexpr (F8) {
 #pragma unroll
-            for (int nt = 0; nt < D / 8; ++nt)
-                *reinterpret_cast<float2 *>(row + nt * 8 + 2 * (lane & 3)) = make_float2(st.o[nt][0], st.o[nt][1]);
+                for (int ch = 0; ch < D / 16; ++ch)
+                    *reinterpret_cast<float4 *>(row + ch * 16 + 4 * (lane & 3)) =
+                        make_float4(st.o[2 * ch][0] * vs, st.o[2 * ch + 1][0] * vs, st.o[2 * ch][1] * vs, st.o[2 * ch + 1][1] * vs);
+            } else {
+#pragma unroll
+                for (int nt = 0; nt < D / 8; ++nt)
+                    *reinterpret_cast<float2 *>(row + nt * 8 + 2 * (lane & 3)) = make_float2(st.o[nt][0], st.o[nt][1]);
+            }
         }
         if (r_hi < p.G) {
             float *row = cw + (size_t)r_hi * kPitch;
             if ((lane & 3) == 0) { row[D] = st.m[1]; row[D + 1] = l1; }
+            if constexpr (F8) {
 #pragma unroll
-            for (int nt = 0; nt < D / 8; ++nt)
-                *reinterpret_cast<float2 *>(row + nt * 8 + 2 * (lane & 3)) = make_float2(st.o[nt][2], st.o[nt][3]);
+                for (int ch = 0; ch < D / 16; ++ch)
+                    *reinterpret_cast<float4 *>(row + ch * 16 + 4 * (lane & 3)) =
+                        make_float4(st.o[2 * ch][2] * vs, st.o[2 * ch + 1][2] * vs, st.o[2 * ch][3] * vs, st.o[2 * ch + 1][3] * vs);
+            } else {
+#pragma unroll
+                for (int nt = 0; nt < D / 8; ++nt)
+                    *reinterpret_cast<float2 *>(row + nt * 8 + 2 * (lane & 3)) = make_float2(st.o[nt][2], st.o[nt][3]);
+            }
         }
     }
     __syncthreads();
@@ -429,13 +513,13 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
     }
 }
 
-template <int D>
+template <int D, bool F8>
 bool configure_kernel()
 {
     static bool done = false, ok = false;
     if (!done) {
         done = true;
-        ok = cudaFuncSetAttribute(decode_cluster_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) ==
+        ok = cudaFuncSetAttribute(decode_cluster_kernel<D, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) ==
              cudaSuccess;
         if (!ok) (void)cudaGetLastError();
     }
@@ -443,24 +527,26 @@ bool configure_kernel()
 }
 
 // Shared-memory stages that fit beside the merge scratch (0: none do).
-template <int D>
+template <int D, bool F8>
 int pick_stages(int G)
 {
-    for (int s = ClusterCfg<D>::kMaxStages; s >= 2; --s)
-        if (cluster_smem_bytes<D>(G, s) <= 227 * 1024) return s;
+    for (int s = ClusterCfg<D, F8>::kMaxStages; s >= 2; --s)
+        if (cluster_smem_bytes<D, F8>(G, s) <= 227 * 1024) return s;
     return 0;
 }
 
 // Clusters of C CTAs that the device can hold at once (0 if the shape cannot launch). Looked up once per shape.
-template <int D>
+template <int D, bool F8>
 int resident_clusters(int C, size_t smem)
 {
     struct Entry { int C; size_t smem; int n; };
     static Entry cache[16];
     static int n_cached = 0;
+    static std::mutex mutex;
+    std::lock_guard<std::mutex> lock(mutex);
     for (int i = 0; i < n_cached; ++i)
         if (cache[i].C == C && cache[i].smem == smem) return cache[i].n;
-    if (!configure_kernel<D>()) return 0;
+    if (!configure_kernel<D, F8>()) return 0;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(C, 1, 1);
     cfg.blockDim = dim3(kThreads);
@@ -471,7 +557,7 @@ int resident_clusters(int C, size_t smem)
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, decode_cluster_kernel<D>, &cfg) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveClusters(&n, decode_cluster_kernel<D, F8>, &cfg) != cudaSuccess) {
         (void)cudaGetLastError();
         n = 0;
     }
@@ -479,9 +565,31 @@ int resident_clusters(int C, size_t smem)
     return n;
 }
 
+// Host-side view of one instantiation.
+struct ClusterShape {
+    int tile_t;
+    int (*stages)(int G);
+    size_t (*smem)(int G, int stages);
+    int (*resident)(int C, size_t smem);
+    bool (*configure)();
+};
+
+template <int D, bool F8>
+ClusterShape shape_of()
+{
+    return ClusterShape{ClusterCfg<D, F8>::kTileT, &pick_stages<D, F8>, &cluster_smem_bytes<D, F8>, &resident_clusters<D, F8>,
+                        &configure_kernel<D, F8>};
+}
+
+ClusterShape pick_cluster_shape(int D, bool fp8)
+{
+    if (fp8) return shape_of<128, true>();
+    return D == 128 ? shape_of<128, false>() : shape_of<64, false>();
+}
+
 }  // namespace
 
-int decode_cluster_width(int B, int Hq, int Hkv, int D, int max_kv_len)
+int decode_cluster_width(int B, int Hq, int Hkv, int D, int max_kv_len, bool fp8)
 {
     // debugging aid: L4L_DECODE_CLUSTER=0 keeps every call on the split kernel, =N forces clusters of N where they fit
     int forced = -1;
@@ -491,10 +599,11 @@ int decode_cluster_width(int B, int Hq, int Hkv, int D, int max_kv_len)
     const long long units = (long long)B * Hkv;
     const int sms = sm_count();
     if (units <= 0 || units > 65535 || units > sms) return 0;
-    const int stages = (D == 128) ? pick_stages<128>(G) : pick_stages<64>(G);
+    const ClusterShape shape = pick_cluster_shape(D, fp8);
+    const int stages = shape.stages(G);
     if (stages == 0) return 0;
-    const size_t smem = (D == 128) ? cluster_smem_bytes<128>(G, stages) : cluster_smem_bytes<64>(G, stages);
-    const int tiles_max = max_kv_len > 0 ? (max_kv_len + kTileT - 1) / kTileT : 1;
+    const size_t smem = shape.smem(G, stages);
+    const int tiles_max = max_kv_len > 0 ? (max_kv_len + shape.tile_t - 1) / shape.tile_t : 1;
     // the widest power of two that keeps every cluster resident at once and gives every CTA at least one tile
     int C = 1;
     while (2 * C <= kMaxCluster && units * 2 * C <= sms && 2 * C <= tiles_max) C *= 2;
@@ -503,7 +612,7 @@ int decode_cluster_width(int B, int Hq, int Hkv, int D, int max_kv_len)
         while (2 * C <= forced && 2 * C <= kMaxCluster) C *= 2;
     }
     for (; C >= 1; C /= 2) {
-        const int n = (D == 128) ? resident_clusters<128>(C, smem) : resident_clusters<64>(C, smem);
+        const int n = shape.resident(C, smem);
         if (n >= units || (forced > 0 && n > 0)) break;
     }
     if (C < 1) return 0;
@@ -511,22 +620,28 @@ int decode_cluster_width(int B, int Hq, int Hkv, int D, int max_kv_len)
     // Beyond these bounds the even split of the whole tile stream over all SMs (the split kernel) wins: a lone CTA
     // per sequence streams at one SM's rate, and ragged lengths leave short sequences' CTAs idle.
     const int per_cta = (tiles_max + C - 1) / C;
-    if (per_cta > 32) return 0;
+    if (per_cta * shape.tile_t > 32 * 128) return 0;
     return C;
 }
 
 l4l_status launch_decode_cluster(const void *q, void *o, const l4l_kv_cache &cache, const int32_t *d_kv_lens,
                                  int max_kv_len, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
                                  void *workspace, cudaStream_t stream, const l4l_tensor4 *k_new,
-                                 const l4l_tensor4 *v_new, const PagedTable *paged, const RopeArgs *rope, int width)
+                                 const l4l_tensor4 *v_new, const PagedTable *paged, const RopeArgs *rope,
+                                 const Fp8Scales *fp8, int width)
 {
     if (paged && (k_new || v_new)) return L4L_ERR_UNSUPPORTED;
     if (rope && (!k_new || !v_new)) return L4L_ERR_UNSUPPORTED;      // only with the fused append
+    if (fp8 && (D != 128 || k_new || v_new || rope)) return L4L_ERR_UNSUPPORTED;
+    // fp8: cache.k / cache.v point at e4m3 bytes, the strides count bytes (= elements)
+    const int esz = fp8 ? 1 : 2, box_d = fp8 ? 128 : 64;
     const int G = Hq / Hkv;
-    const int stages = (D == 128) ? pick_stages<128>(G) : pick_stages<64>(G);
+    const ClusterShape shape = pick_cluster_shape(D, fp8 != nullptr);
+    const int kTileT = shape.tile_t;
+    const int stages = shape.stages(G);
     if (stages == 0 || width < 1 || width > kMaxCluster) return L4L_ERR_UNSUPPORTED;
-    const size_t smem = (D == 128) ? cluster_smem_bytes<128>(G, stages) : cluster_smem_bytes<64>(G, stages);
-    if (!((D == 128) ? configure_kernel<128>() : configure_kernel<64>())) return L4L_ERR_CUDA;
+    const size_t smem = shape.smem(G, stages);
+    if (!shape.configure()) return L4L_ERR_CUDA;
 
     CUtensorMap tk, tv, tk_tail, tv_tail;   // tile-sized boxes, and small boxes for a mostly empty last tile of a sequence
     TmapCoord coord, coord_v;
@@ -534,14 +649,14 @@ l4l_status launch_decode_cluster(const void *q, void *o, const l4l_kv_cache &cac
     // pages smaller than a tile are fetched page by page: no box may exceed the page
     const int box_t = (paged && cache.max_len < kTileT) ? cache.max_len : kTileT;
     const int tail_rows = (paged && cache.max_len < 32) ? cache.max_len : 32;
-    if (!make_tmap(&tk, &coord, cache.k, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h, cache.stride_b, 64,
-                   box_t, 2) ||
+    if (!make_tmap(&tk, &coord, cache.k, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h, cache.stride_b, box_d,
+                   box_t, esz) ||
         !make_tmap(&tv, &coord_v, cache.v, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h, cache.stride_b,
-                   64, box_t, 2) ||
+                   box_d, box_t, esz) ||
         !make_tmap(&tk_tail, &coord_v, cache.k, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
-                   cache.stride_b, 64, tail_rows, 2) ||
+                   cache.stride_b, box_d, tail_rows, esz) ||
         !make_tmap(&tv_tail, &coord_v, cache.v, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
-                   cache.stride_b, 64, tail_rows, 2))
+                   cache.stride_b, box_d, tail_rows, esz))
         return L4L_ERR_CUDA;
     ClusterParams p;
     p.q = static_cast<const __nv_bfloat16 *>(q);
@@ -572,6 +687,8 @@ l4l_status launch_decode_cluster(const void *q, void *o, const l4l_kv_cache &cac
     p.k_weight = rope ? rope->k_weight : nullptr;
     p.norm_eps = rope ? rope->eps : 0.f;
     p.rope_n_pos = rope ? rope->n_pos : 0;
+    p.k_scale = fp8 ? fp8->k_scale : nullptr;
+    p.v_scale = fp8 ? fp8->v_scale : nullptr;
     p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.G = G; p.C = width; p.max_kv_len = max_kv_len; p.stages = stages;
     p.scale_log2e = scale * 1.4426950408889634f;
     p.coord = coord;
@@ -588,8 +705,10 @@ l4l_status launch_decode_cluster(const void *q, void *o, const l4l_kv_cache &cac
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    const cudaError_t err = (D == 128) ? cudaLaunchKernelEx(&cfg, decode_cluster_kernel<128>, tk, tv, tk_tail, tv_tail, p)
-                                       : cudaLaunchKernelEx(&cfg, decode_cluster_kernel<64>, tk, tv, tk_tail, tv_tail, p);
+    const cudaError_t err =
+        fp8        ? cudaLaunchKernelEx(&cfg, decode_cluster_kernel<128, true>, tk, tv, tk_tail, tv_tail, p)
+        : D == 128 ? cudaLaunchKernelEx(&cfg, decode_cluster_kernel<128, false>, tk, tv, tk_tail, tv_tail, p)
+                   : cudaLaunchKernelEx(&cfg, decode_cluster_kernel<64, false>, tk, tv, tk_tail, tv_tail, p);
     return err == cudaSuccess ? L4L_OK : L4L_ERR_CUDA;
 }
 

@@ -76,11 +76,12 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
 
 // Small batches: one thread-block cluster per (sequence, KV head), partials merged through distributed shared
 // memory. decode_cluster_width returns the cluster size to use, or 0 if the split kernel should run.
-int decode_cluster_width(int B, int Hq, int Hkv, int D, int max_kv_len);
+int decode_cluster_width(int B, int Hq, int Hkv, int D, int max_kv_len, bool fp8);
 l4l_status launch_decode_cluster(const void *q, void *o, const l4l_kv_cache &cache, const int32_t *d_kv_lens,
                                  int max_kv_len, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
                                  void *workspace, cudaStream_t stream, const l4l_tensor4 *k_new,
-                                 const l4l_tensor4 *v_new, const PagedTable *paged, const RopeArgs *rope, int width);
+                                 const l4l_tensor4 *v_new, const PagedTable *paged, const RopeArgs *rope,
+                                 const Fp8Scales *fp8, int width);
 
 l4l_status launch_rope_kv_append(const l4l_tensor4 &q, const l4l_tensor4 &k_new, const l4l_tensor4 &v_new,
                                  const l4l_kv_cache &cache, const int32_t *d_pos, const int32_t *d_n_new, int T, int B,

@@ -27,7 +27,7 @@ def pytest_collection_modifyitems(config, items):
 # batches, the split kernel otherwise). The decode parity modules run once with the library's own choice and
 # once with every call kept on the split kernel, so that small test shapes cover both.
 _DECODE_MODULES = {"test_gpu_decode", "test_gpu_decode_append", "test_gpu_paged", "test_gpu_random_shapes",
-                   "test_gpu_cuda_graph", "test_gpu_rope_append"}
+                   "test_gpu_cuda_graph", "test_gpu_rope_append", "test_gpu_fp8"}
 
 
 def pytest_generate_tests(metafunc):

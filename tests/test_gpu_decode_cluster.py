@@ -130,6 +130,22 @@ def test_cluster_decode_step_with_rope_and_append(cluster_width, D, Hq, Hkv, nor
     rope_step_case(D, Hq, Hkv, norm)
 
 
+@pytest.mark.parametrize("cluster_width", WIDTHS, indirect=True)
+def test_cluster_decode_fp8_cache(cluster_width):
+    from test_gpu_fp8 import test_fp8_decode_matches_oracle as fp8_case
+
+    fp8_case(16, 2)
+    fp8_case(8, 8)
+
+
+@pytest.mark.parametrize("cluster_width", [1, 4, 8], indirect=True)
+@pytest.mark.parametrize("page", [16, 64, 256])
+def test_cluster_decode_fp8_paged(cluster_width, page):
+    from test_gpu_fp8 import test_fp8_paged_decode_matches_oracle as fp8_paged_case
+
+    fp8_paged_case(page)
+
+
 def test_library_choice_matches_split_kernel_result():
     # the same call on both kernels: results agree to rounding of the merge order
     lens = [2304]
