@@ -432,6 +432,14 @@ def run_ours(args, rank, world):
     t_rglru = timed(lambda: l4l.l4l_rglru_scan(rx, rgx, rga, r_ap, r_state, ry, ws_r), 10)
     rglru_bytes = rx.numel() * 8                          # 3 bf16 read + 1 written per (step, channel)
     dev_err_r = l4l.l4l_last_device_error(ws_r)
+    # the same bytes as 16 sequences of 2048 steps: 640 CTAs instead of 160 (which is 148 SMs + 12: the 12 SMs that
+    # get a second CTA set the time of the B=4 case)
+    rB2, rT2 = 16, 2048
+    r_state2 = torch.zeros(rB2, rW, dtype=torch.float32, device=dev)
+    ws_r2 = l4l.new_rglru_workspace(rB2, rT2, rW, device=dev)
+    v2 = lambda t: t.view(rB2, rT2, rW)
+    t_rglru2 = timed(lambda: l4l.l4l_rglru_scan(v2(rx), v2(rgx), v2(rga), r_ap, r_state2, v2(ry), ws_r2), 10)
+    dev_err_r |= l4l.l4l_last_device_error(ws_r2)
     del rx, rgx, rga, ry, filler
     dev_err = l4l.l4l_last_device_error(ws_p) | l4l.l4l_last_device_error(ws_d) | dev_err_r | err_small | err_small2
 
@@ -541,6 +549,9 @@ def run_ours(args, rank, world):
             "rglru_scan_B4_T8192_W2560": {"us": t_rglru * 1e3, "gbs": rglru_bytes / (t_rglru * 1e-3) / 1e9,
                                           "frac_of_measured_hbm": rglru_bytes / (t_rglru * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                           "bytes": rglru_bytes},
+            "rglru_scan_B16_T2048_W2560": {"us": t_rglru2 * 1e3, "gbs": rglru_bytes / (t_rglru2 * 1e-3) / 1e9,
+                                           "frac_of_measured_hbm": rglru_bytes / (t_rglru2 * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                           "bytes": rglru_bytes},
             "decode_fp8_cache": {"us": t_fp8 * 1e3, "kv_gbs_fp8_bytes": dec_bytes / 2 / (t_fp8 * 1e-3) / 1e9,
                                  "speedup_over_bf16_cache": t_dec_b2b / t_fp8},
             "decode_step_B1_L2304_in_cuda_graph": {"cluster_kernel_us": t_small, "split_kernel_us": t_small_split},
