@@ -261,7 +261,7 @@ def run_ours(args, rank, world):
     # ---- the decode kernel alone: launches back to back over three rotating copies of the cache (1.6 GB,
     # so every launch streams from HBM), one pair of CUDA events around the whole run
     caches = [(dck, dcv)] + [(dck.clone(), dcv.clone()) for _ in range(2)]
-    n_dec = max(20, args.steps)
+    n_dec = max(60, args.steps)
     for i in range(3):
         l4l.l4l_attn_decode(dq, do, caches[i][0], caches[i][1], dlen, Lmax, wd.scale, ws_d)
     barrier()

@@ -189,6 +189,9 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     // next kernel in the stream may begin its own prologue as soon as this grid's CTAs retire.
     grid_dependency_wait();
     grid_launch_dependents();
+    // the producer's first look at the lengths is requested now, so that its latency passes behind the barrier below
+    int early_len = 0;
+    if (warp == kProducerWarp && lane < p.B) early_len = p.kv_lens[lane];
     if (p.rope_cos != nullptr) {
         for (int i = threadIdx.x; i < D; i += blockDim.x) {
             norm_w[i] = p.q_weight ? __ldg(p.q_weight + i) : 1.f;
@@ -208,7 +211,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             const int b = b0 + lane;
             int n = 0;
             if (b < p.B) {
-                int len = p.kv_lens[b];
+                int len = b0 == 0 ? early_len : p.kv_lens[b];
                 len = len < 0 ? 0 : (len > p.max_kv_len ? p.max_kv_len : len);
                 lens_s[b] = len;
                 n = len > 0 ? ((len + kTileT - 1) / kTileT + 1) * p.Hkv : 0;
