@@ -570,7 +570,7 @@ def run_ours(args, rank, world):
 def run_profile_case(case: str):
     """A few launches of ONE kernel on a small case, for `ncu` captures (not a benchmark):
     prefill = B=1, S=8192 of the long_prefill workload (inputs 168 MB > L2); decode = the batched_decode batch;
-    rglru = the RG-LRU scan on B=16, T=2048, W=2560; decode_small = the cluster decode kernel on B=4 x 8192 tokens."""
+    rglru = the RG-LRU scan on B=16, T=2048, W=2560; decode_small = the cluster decode kernel on B=4 x 8192 tokens; rope = rope + norm + cache update on B=2, S=8192."""
     from paper_2608_21836_b200 import binding as l4l
 
     torch.cuda.set_device(0)
@@ -597,6 +597,20 @@ def run_profile_case(case: str):
         ws = l4l.new_rglru_workspace(B, T, W)
         for _ in range(3):
             l4l.l4l_rglru_scan(x, gx, ga, ap, state, y, ws)
+    elif case == "rope":
+        # rope + QK-norm + cache update of a whole prompt: B=2, S=8192 of the long_prefill shapes (403 MB moved)
+        w = wl.WORKLOADS["long_prefill"]
+        seq = wl.make_sequence(w, B=2)
+        q, k, v = seq.q.cuda(), seq.k.cuda(), seq.v.cuda()
+        ck = torch.empty(2, w.Hkv, seq.S, w.D, dtype=torch.bfloat16, device="cuda")
+        cv = torch.empty_like(ck)
+        cos, sin = wl.make_rope_tables(seq.S, w.D)
+        cos, sin = cos.cuda(), sin.cuda()
+        gamma = torch.ones(w.D, dtype=torch.float32, device="cuda")
+        pos = torch.zeros(2, dtype=torch.int32, device="cuda")
+        ws = l4l.new_workspace(l4l.L4L_OP_PREFILL, 2, w.Hq, w.Hkv, w.D, seq.S)     # only for the status word below
+        for _ in range(3):
+            l4l.l4l_rope_kv_append(q, k, v, ck, cv, pos, None, cos, sin, gamma, gamma, 1e-6)
     elif case == "decode_small":
         # the cluster kernel: B = 4 sequences of 8192 tokens of the 8B-shaped layer (134 MB of cache > L2)
         w = wl.WORKLOADS["layer8b"]
@@ -625,7 +639,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--profile-case", choices=["prefill", "decode", "decode_small", "rglru"], default=None,
+    ap.add_argument("--profile-case", choices=["prefill", "decode", "decode_small", "rope", "rglru"], default=None,
                     help="run three launches of one kernel on a small case and exit (for ncu)")
     args = ap.parse_args()
     if args.profile_case:
