@@ -40,7 +40,7 @@ constexpr int kPostRing = 16;               // pieces a producer can be ahead of
 // that calls of different shapes on one workspace can never write partials over counters another call
 // relies on being zero.
 constexpr size_t kTicketBytes = 128 * 1024;  // 32768 (sequence, KV head) pairs per launch
-constexpr int kMaxB = 512;                 // sequences per launch (prefix sums live in shared memory)
+constexpr int kMaxB = 384;                 // sequences per launch (prefix sums and lengths live in shared memory)
 
 // F8: the cache holds e4m3 bytes (one byte per value) instead of bf16.
 template <int D, int W, bool F8>
@@ -55,6 +55,27 @@ struct DecodeCfg {
     static constexpr uint32_t kTileBytes = kHalves * kHalfBytes;  // one of K or V
     static constexpr uint32_t kStageBytes = 2 * kTileBytes;
     static constexpr int kStages = (kStageBytes >= 32768u * (W / 4)) ? 3 : 6;   // 192 KB (96 KB with W = 4) in flight
+};
+
+// One row of `comb`: the unnormalised O of one query head of a piece as one consumer warp saw it, then its max and its
+// sum. Groups of 5 to 8 query heads at head_dim 128 (BigG) keep O as bf16 there, so that eight warps' rows still fit
+// beside the three 64 KB stages; max and sum stay fp32. (One rounding to bf16 per warp and piece, ahead of the merge.)
+template <int D, bool BigG>
+struct CombRow {
+    static constexpr int kBytes = BigG ? D * 2 + 16 : (D + 4) * 4;
+    static constexpr int kOffM = BigG ? D * 2 : D * 4;
+    static __device__ __forceinline__ float m(const uint8_t *row) { return *reinterpret_cast<const float *>(row + kOffM); }
+    static __device__ __forceinline__ float l(const uint8_t *row) { return *reinterpret_cast<const float *>(row + kOffM + 4); }
+    static __device__ __forceinline__ float4 v4(const uint8_t *row, int d4)
+    {
+        if constexpr (BigG) {
+            const uint2 u = *reinterpret_cast<const uint2 *>(row + d4 * 8);
+            return make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u), __uint_as_float(u.y << 16),
+                               __uint_as_float(u.y & 0xffff0000u));
+        } else {
+            return *reinterpret_cast<const float4 *>(row + d4 * 16);
+        }
+    }
 };
 
 struct TileMeta {
@@ -95,15 +116,16 @@ struct DecodeParams {
     int table_stride, page_size, page_shift;
     int tail_rows;            // tokens per box of tmap_k_tail / tmap_v_tail (32, or the page size if that is smaller)
     int B, Hq, Hkv, G, min_tiles, nsplit, max_kv_len;
+    int nfin;                 // finisher warps (BigG: one per 4 query heads of the group; else 1)
     float scale_log2e;
     TmapCoord coord;
 };
 
-template <int D, int W, bool F8>
+template <int D, int W, bool F8, bool BigG>
 size_t decode_smem_bytes(int G, int nsplit)
 {
     using C = DecodeCfg<D, W, F8>;
-    size_t comb = (size_t)W * G * (D + 4) * sizeof(float) + (size_t)((G * nsplit + 3) & ~3) * sizeof(float);
+    size_t comb = (size_t)W * G * CombRow<D, BigG>::kBytes + (size_t)((G * nsplit + 3) & ~3) * sizeof(float);
     // per stage: the K/V tiles, the piece's query rows and (rope fused into the step) the cos / sin rows of the
     // new token's position; per consumer warp: its private copy of those rows for the piece it is working on
     return 1024 /*alignment slack*/ + (size_t)C::kStages * (C::kStageBytes + (size_t)G * D * 2 + D * 4) + (size_t)W * D * 4 + 2 * D * 4 +
@@ -120,8 +142,8 @@ __device__ __forceinline__ void order_coords(const TmapCoord &c, int t, int h, i
     c3 = (c.pos_t == 3) ? t : (c.pos_h == 3) ? h : b;
 }
 
-template <int D, int W, bool F8>
-__global__ void __launch_bounds__((W + 2) * 32)
+template <int D, int W, bool F8, bool BigG>
+__global__ void __launch_bounds__((W + (BigG ? 3 : 2)) * 32)
 decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
                     const __grid_constant__ CUtensorMap tmap_k_tail, const __grid_constant__ CUtensorMap tmap_v_tail,
                     const DecodeParams p)
@@ -141,10 +163,10 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     float *rope_priv = reinterpret_cast<float *>(q_slots + (size_t)C::kStages * q_stride);   // [W][D] per-warp copy
     float *norm_w = rope_priv + (size_t)W * D;                           // q_weight | k_weight (when given)
     float *comb = norm_w + 2 * D;
-    constexpr int kPitch = D + 4;            // floats per row of `comb`: O[D], max, sum, pad (16-byte rows)
     constexpr int kVec = D / 4;
-    const int comb_floats = kConsumerWarps * p.G * kPitch;
-    float *merge_lse = comb + comb_floats;   // [G][nsplit] scratch of the finisher's second pass
+    using CR = CombRow<D, BigG>;
+    uint8_t *comb_b = reinterpret_cast<uint8_t *>(comb);
+    float *merge_lse = reinterpret_cast<float *>(comb_b + (size_t)kConsumerWarps * p.G * CR::kBytes);   // [G][nsplit] scratch of the finisher's second pass
     TileMeta *meta = reinterpret_cast<TileMeta *>(merge_lse + ((p.G * p.nsplit + 3) & ~3));   // keeps 16-byte alignment
     PieceMeta *piece_meta = reinterpret_cast<PieceMeta *>(meta + C::kStages);
     uint64_t *full = reinterpret_cast<uint64_t *>(piece_meta + 1);
@@ -171,7 +193,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             mbar_init(&empty[s], kConsumerWarps);
         }
         mbar_init(comb_full, kConsumerWarps);
-        mbar_init(comb_empty, 1);
+        mbar_init(comb_empty, BigG ? p.nfin : 1);
         *abort_flag = 0;
         *posted_count = 0u;
         *pieces_total = 0xffffffffu;
@@ -375,17 +397,23 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 }
             }
         }
-    } else if (warp == kFinisherWarp) {
+    } else if (warp >= kFinisherWarp) {
         // ------------------------------------------------------------------ finisher warp
+        // BigG: one finisher warp per 4 query heads of the group (so that a lane never owns more than four float4
+        // outputs of a piece), each with its own rows of `comb`, of the outputs and of the workspace, and its own ticket.
+        const int fin = BigG ? warp - kFinisherWarp : 0;
+        const int nfin = BigG ? p.nfin : 1;
+        const int g0 = BigG ? fin * 4 : 0;
+        const int gcnt = BigG ? min(4, p.G - g0) : p.G;
         // sequences with no cached token get o = 0, lse = -inf (no tile ever refers to them)
-        for (int b = blockIdx.x; b < p.B; b += gridDim.x) {
+        for (int b = blockIdx.x; fin == 0 && b < p.B; b += gridDim.x) {
             if (p.kv_lens[b] <= 0) {
                 for (int i = lane; i < p.Hq * D; i += 32) p.o[(size_t)b * p.Hq * D + i] = __float2bfloat16_rn(0.f);
                 if (p.lse)
                     for (int i = lane; i < p.Hq; i += 32) p.lse[(size_t)b * p.Hq + i] = -INFINITY;
             }
         }
-        const bool few_items = (p.G * kVec <= 4 * 32);     // each lane owns at most four float4 outputs of a piece
+        const bool few_items = (gcnt * kVec <= 4 * 32);     // each lane owns at most four float4 outputs of a piece
         for (uint32_t n = 0;; ++n) {
             // ---- While the consumers are still streaming piece n: if every other piece of its sequence has
             // already arrived (the usual case for the piece a CTA ends with), fetch their partials now, so
@@ -414,15 +442,15 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                         __threadfence_block();
                         const PieceMeta pp = post_ring[n % kPostRing];
                         if (few_items && pp.npieces > 1 && pp.npieces <= 4) {
-                            int *tk = p.tickets + (size_t)pp.b * p.Hkv + pp.kvh;
+                            int *tk = p.tickets + ((size_t)pp.b * p.Hkv + pp.kvh) * nfin + fin;
                             int seen = (lane == 0) ? ld_acquire_gpu(tk) : 0;
                             seen = __shfl_sync(0xffffffffu, seen, 0);
                             if (seen == pp.npieces - 1) {
-                                const size_t bh0 = (size_t)pp.b * p.Hq + pp.kvh * p.G;
+                                const size_t bh0 = (size_t)pp.b * p.Hq + pp.kvh * p.G + g0;
 #pragma unroll
                                 for (int u = 0; u < 4; ++u) {
                                     const int item = u * 32 + lane;
-                                    const bool on = item < p.G * kVec;
+                                    const bool on = item < gcnt * kVec;
                                     const int r = on ? item / kVec : 0, d4 = on ? item % kVec : 0;
                                     const float *pl = p.part_lse + (bh0 + r) * p.nsplit;
                                     const float4 *po =
@@ -450,8 +478,8 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             }
             const PieceMeta pm = *piece_meta;
             const bool single = (pm.npieces == 1);
-            const size_t bh0 = (size_t)pm.b * p.Hq + pm.kvh * p.G;
-            int *tk = p.tickets + (size_t)pm.b * p.Hkv + pm.kvh;
+            const size_t bh0 = (size_t)pm.b * p.Hq + pm.kvh * p.G + g0;
+            int *tk = p.tickets + ((size_t)pm.b * p.Hkv + pm.kvh) * nfin + fin;
             const int np = pm.npieces;
 
             // ---- merge of the consumer warps' (max, sum, O). With at most 128 float4 outputs per piece (the usual
@@ -465,7 +493,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     const int item = u * 32 + lane;
-                    on4[u] = item < p.G * kVec;
+                    on4[u] = item < gcnt * kVec;
                     r4[u] = on4[u] ? item / kVec : 0;
                     d4s[u] = on4[u] ? item % kVec : 0;
                     mloc4[u] = -INFINITY;
@@ -476,16 +504,16 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 for (int w = 0; w < kConsumerWarps; ++w)
 #pragma unroll
                     for (int u = 0; u < 4; ++u)
-                        mloc4[u] = fmaxf(mloc4[u], comb[((size_t)w * p.G + r4[u]) * kPitch + D]);
+                        mloc4[u] = fmaxf(mloc4[u], CR::m(comb_b + ((size_t)w * p.G + g0 + r4[u]) * CR::kBytes));
 #pragma unroll
                 for (int w = 0; w < kConsumerWarps; ++w)
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
-                        const float *row = comb + ((size_t)w * p.G + r4[u]) * kPitch;
-                        const float wgt = fast_exp2(row[D] - mloc4[u]);    // warp that saw no token: max = -inf -> 0
-                        const float4 v = *reinterpret_cast<const float4 *>(row + d4s[u] * 4);
+                        const uint8_t *row = comb_b + ((size_t)w * p.G + g0 + r4[u]) * CR::kBytes;
+                        const float wgt = fast_exp2(CR::m(row) - mloc4[u]);    // warp that saw no token: max = -inf -> 0
+                        const float4 v = CR::v4(row, d4s[u]);
                         acc4[u].x += wgt * v.x; acc4[u].y += wgt * v.y; acc4[u].z += wgt * v.z; acc4[u].w += wgt * v.w;
-                        lsum4[u] += wgt * row[D + 1];
+                        lsum4[u] += wgt * CR::l(row);
                     }
             }
 
@@ -557,24 +585,24 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 for (int u = 0; u < 4; ++u)
                     if (on4[u]) emit(r4[u], d4s[u], acc4[u], lsum4[u], mloc4[u]);
             } else {
-                for (int item = lane; item < p.G * kVec; item += 32) {
+                for (int item = lane; item < gcnt * kVec; item += 32) {
                     const int r = item / kVec, d4 = item % kVec;
                     float mw[kConsumerWarps];
                     float mstar = -INFINITY;
 #pragma unroll
                     for (int w = 0; w < kConsumerWarps; ++w) {
-                        mw[w] = comb[((size_t)w * p.G + r) * kPitch + D];
+                        mw[w] = CR::m(comb_b + ((size_t)w * p.G + g0 + r) * CR::kBytes);
                         mstar = fmaxf(mstar, mw[w]);
                     }
                     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
                     float lsum = 0.f;
 #pragma unroll
                     for (int w = 0; w < kConsumerWarps; ++w) {
-                        const float *row = comb + ((size_t)w * p.G + r) * kPitch;
+                        const uint8_t *row = comb_b + ((size_t)w * p.G + g0 + r) * CR::kBytes;
                         const float wgt = fast_exp2(mw[w] - mstar);    // warp that saw no token: max = -inf -> 0
-                        const float4 v = *reinterpret_cast<const float4 *>(row + d4 * 4);
+                        const float4 v = CR::v4(row, d4);
                         acc.x += wgt * v.x; acc.y += wgt * v.y; acc.z += wgt * v.z; acc.w += wgt * v.w;
-                        lsum += wgt * row[D + 1];
+                        lsum += wgt * CR::l(row);
                     }
                     emit(r, d4, acc, lsum, mstar);
                 }
@@ -597,7 +625,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     const int item = u * 32 + lane;
-                    const bool on = item < p.G * kVec;
+                    const bool on = item < gcnt * kVec;
                     const int r = on ? item / kVec : 0, d4 = on ? item % kVec : 0;
                     const float *pl = p.part_lse + (bh0 + r) * p.nsplit;
                     const float4 *po = reinterpret_cast<const float4 *>(p.part_o + (bh0 + r) * p.nsplit * D) + d4;
@@ -623,7 +651,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     const int item = u * 32 + lane;
-                    if (item < p.G * kVec) {
+                    if (item < gcnt * kVec) {
                         const int r = item / kVec, d4 = item % kVec;
                         const float mstar = fmaxf(fmaxf(sl[u][0], sl[u][1]), fmaxf(sl[u][2], sl[u][3]));
                         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -647,12 +675,12 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 continue;
             }
             // second pass: out = sum_c w_c o_c / sum_c w_c with w_c = 2^(lse_c - max_c lse_c)
-            for (int idx = lane; idx < p.G * np; idx += 32) {
+            for (int idx = lane; idx < gcnt * np; idx += 32) {
                 const int r = idx / np, c = idx % np;
-                merge_lse[r * p.nsplit + c] = __ldcg(p.part_lse + (bh0 + r) * p.nsplit + c);
+                merge_lse[(g0 + r) * p.nsplit + c] = __ldcg(p.part_lse + (bh0 + r) * p.nsplit + c);
             }
             __syncwarp();
-            for (int base = 0; base < p.G * kVec; base += 4 * 32) {
+            for (int base = 0; base < gcnt * kVec; base += 4 * 32) {
                 float4 res[4];
                 float lse_out[4];
 #pragma unroll
@@ -660,9 +688,9 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     const int item = base + u * 32 + lane;
                     res[u] = make_float4(0.f, 0.f, 0.f, 0.f);
                     lse_out[u] = 0.f;
-                    if (item < p.G * kVec) {
+                    if (item < gcnt * kVec) {
                         const int r = item / kVec, d4 = item % kVec;
-                        const float *wl = merge_lse + r * p.nsplit;
+                        const float *wl = merge_lse + (g0 + r) * p.nsplit;
                         float mstar = -INFINITY;
                         for (int c = 0; c < np; ++c) mstar = fmaxf(mstar, wl[c]);
                         const float4 *po = reinterpret_cast<const float4 *>(p.part_o + (bh0 + r) * p.nsplit * D) + d4;
@@ -683,7 +711,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     const int item = base + u * 32 + lane;
-                    if (item < p.G * kVec) {
+                    if (item < gcnt * kVec) {
                         const int r = item / kVec, d4 = item % kVec;
                         uint2 packed;
                         packed.x = pack_bf16x2(res[u].x, res[u].y);
@@ -875,14 +903,31 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
                 l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
                 l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
-                float *cw = comb + (size_t)warp * p.G * kPitch;
+                uint8_t *cw = comb_b + (size_t)warp * p.G * CR::kBytes;
                 // fp8: accumulator tiles alternate even / odd head dims (a tile pair gives this lane 4 consecutive
                 // dims) and O still lacks the V scale of its KV head
                 const float vs = F8 ? v_sc : 1.f;
                 if (r_lo < p.G) {
-                    float *row = cw + (size_t)r_lo * kPitch;
-                    if ((lane & 3) == 0) { row[D] = st.m[0]; row[D + 1] = l0; }
-                    if constexpr (F8) {
+                    uint8_t *rowb = cw + (size_t)r_lo * CR::kBytes;
+                    float *row = reinterpret_cast<float *>(rowb);
+                    if ((lane & 3) == 0) {
+                        *reinterpret_cast<float *>(rowb + CR::kOffM) = st.m[0];
+                        *reinterpret_cast<float *>(rowb + CR::kOffM + 4) = l0;
+                    }
+                    if constexpr (BigG) {
+                        // bf16 rows (groups of 5 to 8 heads occupy rows lane/4 only): the same elements, half the bytes
+                        if constexpr (F8) {
+#pragma unroll
+                            for (int ch = 0; ch < D / 16; ++ch)
+                                *reinterpret_cast<uint2 *>(rowb + (ch * 16 + 4 * (lane & 3)) * 2) =
+                                    make_uint2(pack_bf16x2(st.o[2 * ch][0] * vs, st.o[2 * ch + 1][0] * vs),
+                                               pack_bf16x2(st.o[2 * ch][1] * vs, st.o[2 * ch + 1][1] * vs));
+                        } else {
+#pragma unroll
+                            for (int nt = 0; nt < D / 8; ++nt)
+                                *reinterpret_cast<uint32_t *>(rowb + (nt * 8 + 2 * (lane & 3)) * 2) = pack_bf16x2(st.o[nt][0], st.o[nt][1]);
+                        }
+                    } else if constexpr (F8) {
 #pragma unroll
                         for (int ch = 0; ch < D / 16; ++ch)
                             *reinterpret_cast<float4 *>(row + ch * 16 + 4 * (lane & 3)) =
@@ -894,8 +939,8 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                             *reinterpret_cast<float2 *>(row + nt * 8 + 2 * (lane & 3)) = make_float2(st.o[nt][0], st.o[nt][1]);
                     }
                 }
-                if (r_hi < p.G) {
-                    float *row = cw + (size_t)r_hi * kPitch;
+                if (!BigG && r_hi < p.G) {
+                    float *row = reinterpret_cast<float *>(cw + (size_t)r_hi * CR::kBytes);
                     if ((lane & 3) == 0) { row[D] = st.m[1]; row[D + 1] = l1; }
                     if constexpr (F8) {
 #pragma unroll
@@ -928,20 +973,20 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
 }
 
 // Resident CTAs per SM for a given dynamic shared-memory size (0 on failure).
-template <int D, int W, bool F8>
+template <int D, int W, bool F8, bool BigG>
 int decode_blocks_per_sm(size_t smem)
 {
     static bool attr_set = false;
     if (!attr_set) {
         // the opt-in limit is per kernel: allow everything the SM has
-        if (cudaFuncSetAttribute(decode_split_kernel<D, W, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+        if (cudaFuncSetAttribute(decode_split_kernel<D, W, F8, BigG>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
             cudaSuccess)
             return 0;
         attr_set = true;
     }
     if (smem > 227 * 1024) return 0;
     int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_split_kernel<D, W, F8>, (W + 2) * 32, smem) != cudaSuccess)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_split_kernel<D, W, F8, BigG>, (W + (BigG ? 3 : 2)) * 32, smem) != cudaSuccess)
         return 0;
     return n;
 }
@@ -957,14 +1002,18 @@ struct ShapeOps {
     int (*blocks_per_sm)(size_t smem);
 };
 
-template <int D, int W, bool F8>
+template <int D, int W, bool F8, bool BigG = false>
 ShapeOps shape_ops()
 {
-    return ShapeOps{W, DecodeCfg<D, W, F8>::kTileT, &decode_smem_bytes<D, W, F8>, &decode_blocks_per_sm<D, W, F8>};
+    return ShapeOps{W, DecodeCfg<D, W, F8>::kTileT, &decode_smem_bytes<D, W, F8, BigG>, &decode_blocks_per_sm<D, W, F8, BigG>};
 }
 
-ShapeOps pick_shape(int D, int warps, bool fp8)
+// Groups of 5 to 8 query heads at head_dim 128 on the 8-warp shape: 16-bit hand-over rows and two finisher warps.
+bool is_big_group(int D, int warps, int G) { return D == 128 && warps == 8 && G > 4 && G <= 8; }
+
+ShapeOps pick_shape(int D, int warps, bool fp8, bool big = false)
 {
+    if (big) return fp8 ? shape_ops<128, 8, true, true>() : shape_ops<128, 8, false, true>();
     if (fp8) return warps == 8 ? shape_ops<128, 8, true>() : shape_ops<128, 4, true>();      // D == 128 only
     if (D == 128) return warps == 8 ? shape_ops<128, 8, false>() : shape_ops<128, 4, false>();
     return warps == 8 ? shape_ops<64, 8, false>() : shape_ops<64, 4, false>();
@@ -979,9 +1028,9 @@ DecodePlan plan_for_shape(int B, int Hq, int Hkv, int D, int max_kv_len, size_t 
     // scratch) when the real lengths are far below max_kv_len; it is raised until the partials fit the
     // caller's workspace and the shared memory fits the SM.
     DecodePlan pl;
-    const ShapeOps ops = pick_shape(D, warps, fp8);
-    pl.warps = warps;
     const int G = Hq / Hkv;
+    const ShapeOps ops = pick_shape(D, warps, fp8, is_big_group(D, warps, G));
+    pl.warps = warps;
     auto blocks = [&](int nsplit) {
         const size_t smem = ops.smem_bytes(G, nsplit);
         if (!have_dev) return smem <= 227 * 1024 ? (warps == 8 ? 1 : 2) : 0;   // sizing without a device
@@ -1059,7 +1108,9 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
                                          stream, k_new, v_new, paged, rope, fp8, width);
     }
     const int G = Hq / Hkv;
-    const ShapeOps ops = pick_shape(D, plan.warps, fp8 != nullptr);
+    const bool big = is_big_group(D, plan.warps, G);
+    const int nfin = big ? (G + 3) / 4 : 1;
+    const ShapeOps ops = pick_shape(D, plan.warps, fp8 != nullptr, big);
     const int kTileT = ops.tile_t;
     const size_t smem = ops.smem_bytes(G, plan.nsplit);
     if (ops.blocks_per_sm(smem) == 0) return L4L_ERR_CUDA;
@@ -1070,7 +1121,7 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
     float *part_lse = part_o + (size_t)B * Hq * plan.nsplit * D;
 
     // sequences per launch: bounded by the prefix-sum array in shared memory and by the ticket region
-    int slice = (int)(kTicketBytes / sizeof(int)) / Hkv;
+    int slice = (int)(kTicketBytes / sizeof(int)) / (Hkv * nfin);
     if (slice > kMaxB) slice = kMaxB;
     if (slice < 1) return L4L_ERR_UNSUPPORTED;
     for (int b0 = 0; b0 < B; b0 += slice) {
@@ -1106,6 +1157,7 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         p.status = reinterpret_cast<unsigned *>(ws);
         p.B = nb; p.Hq = Hq; p.Hkv = Hkv; p.G = G; p.min_tiles = plan.min_tiles; p.nsplit = plan.nsplit;
         p.max_kv_len = max_kv_len;
+        p.nfin = nfin;
         p.k_new = p.v_new = nullptr;
         p.new_sb = p.new_sh = 0;
         p.rope_cos = rope ? rope->cos : nullptr;
@@ -1136,7 +1188,7 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         p.coord = coord;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(plan.grid);
-        cfg.blockDim = dim3((plan.warps + 2) * 32);
+        cfg.blockDim = dim3((plan.warps + 1 + nfin) * 32);
         cfg.dynamicSmemBytes = smem;
         cfg.stream = stream;
         cudaLaunchAttribute attr[1];
@@ -1145,15 +1197,18 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         cudaError_t err;
-        if (fp8)
-            err = plan.warps == 8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 8, true>, tk, tv, tk_tail, tv_tail, p)
-                                  : cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 4, true>, tk, tv, tk_tail, tv_tail, p);
+        if (big)
+            err = fp8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 8, true, true>, tk, tv, tk_tail, tv_tail, p)
+                      : cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 8, false, true>, tk, tv, tk_tail, tv_tail, p);
+        else if (fp8)
+            err = plan.warps == 8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 8, true, false>, tk, tv, tk_tail, tv_tail, p)
+                                  : cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 4, true, false>, tk, tv, tk_tail, tv_tail, p);
         else if (D == 128)
-            err = plan.warps == 8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 8, false>, tk, tv, tk_tail, tv_tail, p)
-                                  : cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 4, false>, tk, tv, tk_tail, tv_tail, p);
+            err = plan.warps == 8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 8, false, false>, tk, tv, tk_tail, tv_tail, p)
+                                  : cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 4, false, false>, tk, tv, tk_tail, tv_tail, p);
         else
-            err = plan.warps == 8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<64, 8, false>, tk, tv, tk_tail, tv_tail, p)
-                                  : cudaLaunchKernelEx(&cfg, decode_split_kernel<64, 4, false>, tk, tv, tk_tail, tv_tail, p);
+            err = plan.warps == 8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<64, 8, false, false>, tk, tv, tk_tail, tv_tail, p)
+                                  : cudaLaunchKernelEx(&cfg, decode_split_kernel<64, 4, false, false>, tk, tv, tk_tail, tv_tail, p);
         if (err != cudaSuccess) return L4L_ERR_CUDA;
     }
     return L4L_OK;

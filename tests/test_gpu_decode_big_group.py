@@ -1,0 +1,74 @@
+"""Query-head groups of 5 to 8 at head_dim 128 on the split decode kernel: the consumer warps hand their results to two
+finisher warps in 16-bit rows (one rounding to bf16 per warp and piece ahead of the merge), so these shapes get their
+own parity cases: long ragged sequences cut between CTAs, the fused append, the fp8 cache."""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import l4l_oracle as orc
+from paper_2608_21836_b200 import binding as l4l
+from helpers import Guarded, assert_close_to_oracle, bits_equal, nan_bf16
+from test_gpu_decode import check_decode, random_batch
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(autouse=True)
+def split_kernel_only():
+    old = os.environ.get("L4L_DECODE_CLUSTER")
+    os.environ["L4L_DECODE_CLUSTER"] = "0"
+    yield
+    if old is None:
+        os.environ.pop("L4L_DECODE_CLUSTER", None)
+    else:
+        os.environ["L4L_DECODE_CLUSTER"] = old
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(40, 8), (48, 8), (56, 8), (64, 8), (8, 1), (5, 1)])
+def test_big_group_decode_long_ragged(Hq, Hkv):
+    lens = [4096, 0, 1, 129, 3000, 2049, 513, 17, 4000, 1234, 3333, 640]
+    q, ck, cv, kv_len = random_batch(len(lens), Hq, Hkv, 128, 4096, lens, seed=300 + Hq)
+    _, stats = check_decode(q, ck, cv, kv_len, 1.0 / math.sqrt(128))
+
+
+def test_big_group_decode_many_sequences_cut_between_ctas():
+    # enough tiles that every CTA streams a range and most sequences are cut once
+    g = torch.Generator().manual_seed(77)
+    lens = torch.randint(512, 4097, (40,), generator=g).tolist()
+    q, ck, cv, kv_len = random_batch(len(lens), 64, 8, 128, 4096, lens, seed=78)
+    check_decode(q, ck, cv, kv_len, 1.0 / math.sqrt(128))
+
+
+def test_big_group_decode_with_fused_append():
+    from test_gpu_decode_append import make_case
+
+    Hq, Hkv, D = 64, 8, 128
+    lens = [0, 1, 2, 16, 17, 128, 129, 300, 1000, 2048]
+    B, Lmax = len(lens), 2048
+    q, ck, cv, kn, vn, kv_len = make_case(B, Hq, Hkv, D, Lmax, lens, seed=41)
+    scale = 1.0 / math.sqrt(D)
+    pos = (kv_len - 1).clamp(min=0).numpy()
+    n_new = (kv_len > 0).to(torch.int32).numpy()
+    ek, ev = orc.kv_append(ck, cv, kn, vn, pos, n_new)
+    ek_t = torch.from_numpy(ek.view(np.int16)).view(torch.bfloat16)
+    ev_t = torch.from_numpy(ev.view(np.int16)).view(torch.bfloat16)
+    ref, _ = orc.decode(q, ek_t, ev_t, kv_len.numpy(), scale)
+    gk, gv, go = Guarded(ck), Guarded(cv), Guarded(nan_bf16((B, Hq, D)))
+    ws = l4l.new_workspace(l4l.L4L_OP_DECODE, B, Hq, Hkv, D, Lmax)
+    l4l.l4l_attn_decode_append(q.cuda(), go.t, gk.t, gv.t, kn.cuda(), vn.cuda(), kv_len.cuda(), Lmax, scale, ws)
+    torch.cuda.synchronize()
+    assert l4l.l4l_last_device_error(ws) == 0
+    for gd in (gk, gv, go):
+        assert gd.margins_intact()
+    assert bits_equal(gk.t, ek) and bits_equal(gv.t, ev)
+    assert_close_to_oracle(go.t, ref, "big-group decode_append o")
+
+
+def test_big_group_decode_fp8_cache():
+    from test_gpu_fp8 import test_fp8_decode_matches_oracle as fp8_case
+
+    fp8_case(64, 8)
+    fp8_case(40, 8)
