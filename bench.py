@@ -375,6 +375,21 @@ def run_ours(args, rank, world):
 
     t_fp8 = timed(fp8_step, 21)
     del c8
+    # the same cache with 64 query heads on the 8 KV heads (groups of 8: the 70B-class shape), three copies in rotation
+    Hq8 = 8 * Hkv
+    dq8 = torch.randn(Bd, Hq8, D, generator=torch.Generator().manual_seed(9)).to(torch.bfloat16).to(dev)
+    do8 = torch.empty_like(dq8)
+    ws_d8 = l4l.new_workspace(l4l.L4L_OP_DECODE, Bd, Hq8, Hkv, D, Lmax, device=dev)
+    c3 = [(dck, dcv)] + [(dck.clone(), dcv.clone()) for _ in range(2)]
+
+    def g8_step():
+        ck_i, cv_i = c3[rot[0] % 3]
+        rot[0] += 1
+        l4l.l4l_attn_decode(dq8, do8, ck_i, cv_i, dlen, Lmax, wd.scale, ws_d8)
+
+    t_g8 = timed(g8_step, 21)
+    err_g8 = l4l.l4l_last_device_error(ws_d8)
+    del c3
     # The decode phase of the 8B-shaped layer config (B = 1, 2048-token prompt, 256 steps): latency-bound, so the
     # steps (cache update fused in) are replayed from a CUDA graph, as a serving loop would issue them; once on the
     # kernel the library picks for this size (a thread-block cluster per KV head) and once held on the split kernel.
@@ -441,7 +456,7 @@ def run_ours(args, rank, world):
     t_rglru2 = timed(lambda: l4l.l4l_rglru_scan(v2(rx), v2(rgx), v2(rga), r_ap, r_state2, v2(ry), ws_r2), 10)
     dev_err_r |= l4l.l4l_last_device_error(ws_r2)
     del rx, rgx, rga, ry, filler
-    dev_err = l4l.l4l_last_device_error(ws_p) | l4l.l4l_last_device_error(ws_d) | dev_err_r | err_small | err_small2
+    dev_err = l4l.l4l_last_device_error(ws_p) | l4l.l4l_last_device_error(ws_d) | dev_err_r | err_small | err_small2 | err_g8
 
     # ---- end to end through the same entry points with HOST buffers (pinned), copies inside the timed region
     hq, hk, hv = seq.q.pin_memory(), seq.k.pin_memory(), seq.v.pin_memory()
@@ -554,6 +569,7 @@ def run_ours(args, rank, world):
                                            "bytes": rglru_bytes},
             "decode_fp8_cache": {"us": t_fp8 * 1e3, "kv_gbs_fp8_bytes": dec_bytes / 2 / (t_fp8 * 1e-3) / 1e9,
                                  "speedup_over_bf16_cache": t_dec_b2b / t_fp8},
+            "decode_64_query_heads_on_8_kv_heads": {"us": t_g8 * 1e3, "kv_gbs": dec_bytes / (t_g8 * 1e-3) / 1e9},
             "decode_step_B1_L2304_in_cuda_graph": {"cluster_kernel_us": t_small, "split_kernel_us": t_small_split},
         },
         "gpu_launches": 3 * args.steps,
