@@ -143,7 +143,7 @@ __device__ __forceinline__ void order_coords(const TmapCoord &c, int t, int h, i
 }
 
 template <int D, int W, bool F8, bool BigG>
-__global__ void __launch_bounds__((W + (BigG ? 3 : 2)) * 32)
+__global__ void __launch_bounds__((BigG ? 11 : W + 2) * 32)
 decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
                     const __grid_constant__ CUtensorMap tmap_k_tail, const __grid_constant__ CUtensorMap tmap_v_tail,
                     const DecodeParams p)
@@ -939,10 +939,26 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                             *reinterpret_cast<float2 *>(row + nt * 8 + 2 * (lane & 3)) = make_float2(st.o[nt][0], st.o[nt][1]);
                     }
                 }
-                if (!BigG && r_hi < p.G) {
-                    float *row = reinterpret_cast<float *>(cw + (size_t)r_hi * CR::kBytes);
-                    if ((lane & 3) == 0) { row[D] = st.m[1]; row[D + 1] = l1; }
-                    if constexpr (F8) {
+                if (r_hi < p.G) {
+                    uint8_t *rowb = cw + (size_t)r_hi * CR::kBytes;
+                    float *row = reinterpret_cast<float *>(rowb);
+                    if ((lane & 3) == 0) {
+                        *reinterpret_cast<float *>(rowb + CR::kOffM) = st.m[1];
+                        *reinterpret_cast<float *>(rowb + CR::kOffM + 4) = l1;
+                    }
+                    if constexpr (BigG) {
+                        if constexpr (F8) {
+#pragma unroll
+                            for (int ch = 0; ch < D / 16; ++ch)
+                                *reinterpret_cast<uint2 *>(rowb + (ch * 16 + 4 * (lane & 3)) * 2) =
+                                    make_uint2(pack_bf16x2(st.o[2 * ch][2] * vs, st.o[2 * ch + 1][2] * vs),
+                                               pack_bf16x2(st.o[2 * ch][3] * vs, st.o[2 * ch + 1][3] * vs));
+                        } else {
+#pragma unroll
+                            for (int nt = 0; nt < D / 8; ++nt)
+                                *reinterpret_cast<uint32_t *>(rowb + (nt * 8 + 2 * (lane & 3)) * 2) = pack_bf16x2(st.o[nt][2], st.o[nt][3]);
+                        }
+                    } else if constexpr (F8) {
 #pragma unroll
                         for (int ch = 0; ch < D / 16; ++ch)
                             *reinterpret_cast<float4 *>(row + ch * 16 + 4 * (lane & 3)) =
@@ -986,7 +1002,7 @@ int decode_blocks_per_sm(size_t smem)
     }
     if (smem > 227 * 1024) return 0;
     int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_split_kernel<D, W, F8, BigG>, (W + (BigG ? 3 : 2)) * 32, smem) != cudaSuccess)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_split_kernel<D, W, F8, BigG>, (BigG ? 11 : W + 2) * 32, smem) != cudaSuccess)
         return 0;
     return n;
 }
@@ -1008,11 +1024,17 @@ ShapeOps shape_ops()
     return ShapeOps{W, DecodeCfg<D, W, F8>::kTileT, &decode_smem_bytes<D, W, F8, BigG>, &decode_blocks_per_sm<D, W, F8, BigG>};
 }
 
-// Groups of 5 to 8 query heads at head_dim 128 on the 8-warp shape: 16-bit hand-over rows and two finisher warps.
-bool is_big_group(int D, int warps, int G) { return D == 128 && warps == 8 && G > 4 && G <= 8; }
+// Groups of more than 4 query heads at head_dim 128: 16-bit hand-over rows and one finisher warp per 4 heads. Up to 8
+// heads on the 8-warp shape; 9 to 16 heads on a 6-warp shape (96-token tiles: three 48 KB stages leave room for the
+// sixteen rows per warp, and 6 + 1 + 4 warps keep the block at 11 warps).
+bool is_big_group(int D, int warps, int G)
+{
+    return D == 128 && ((warps == 8 && G > 4 && G <= 8) || (warps == 6 && G > 8 && G <= 16));
+}
 
 ShapeOps pick_shape(int D, int warps, bool fp8, bool big = false)
 {
+    if (big && warps == 6) return fp8 ? shape_ops<128, 6, true, true>() : shape_ops<128, 6, false, true>();
     if (big) return fp8 ? shape_ops<128, 8, true, true>() : shape_ops<128, 8, false, true>();
     if (fp8) return warps == 8 ? shape_ops<128, 8, true>() : shape_ops<128, 4, true>();      // D == 128 only
     if (D == 128) return warps == 8 ? shape_ops<128, 8, false>() : shape_ops<128, 4, false>();
@@ -1033,7 +1055,7 @@ DecodePlan plan_for_shape(int B, int Hq, int Hkv, int D, int max_kv_len, size_t 
     pl.warps = warps;
     auto blocks = [&](int nsplit) {
         const size_t smem = ops.smem_bytes(G, nsplit);
-        if (!have_dev) return smem <= 227 * 1024 ? (warps == 8 ? 1 : 2) : 0;   // sizing without a device
+        if (!have_dev) return smem <= 227 * 1024 ? (warps == 4 ? 2 : 1) : 0;   // sizing without a device
         return ops.blocks_per_sm(smem);
     };
     int per_sm = blocks(2);
@@ -1068,11 +1090,17 @@ DecodePlan plan_for_shape(int B, int Hq, int Hkv, int D, int max_kv_len, size_t 
 
 }  // namespace
 
-DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_limit, bool fp8)
+DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_limit, bool fp8, bool paged)
 {
     int n_dev = 0;
     const bool have_dev = cudaGetDeviceCount(&n_dev) == cudaSuccess && n_dev > 0;
     if (!have_dev) (void)cudaGetLastError();
+    // groups of 9 to 16 query heads at head_dim 128: the 6-warp shape (contiguous caches: its 96-token tiles do not
+    // line up with pages)
+    if (D == 128 && Hq / Hkv > 8 && !paged) {
+        const DecodePlan six = plan_for_shape(B, Hq, Hkv, D, max_kv_len, ws_limit, 6, have_dev, fp8);
+        if (six.fits && six.ws_bytes <= ws_limit) return six;
+    }
     // 128-wide heads: prefer the 8-warp shape (one CTA per SM, ranges twice as long, so fewer sequences are cut
     // between CTAs) whenever its shared memory fits, which it does for query-head groups of up to 4; else 4 warps.
     static const int forced = [] {
@@ -1100,6 +1128,7 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
     const int esz = fp8 ? 1 : 2;
     // paged: `cache` describes the page pool (stride_b = stride between pages, max_len = page size)
     if (paged && (k_new || v_new)) return L4L_ERR_UNSUPPORTED;
+    if (paged && plan.warps == 6) return L4L_ERR_UNSUPPORTED;    // planned for a contiguous cache
     {
         // small batches are latency-bound: one cluster per (sequence, KV head), no workspace round trips
         const int width = decode_cluster_width(B, Hq, Hkv, D, max_kv_len, fp8 != nullptr);
@@ -1197,7 +1226,10 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         cudaError_t err;
-        if (big)
+        if (big && plan.warps == 6)
+            err = fp8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 6, true, true>, tk, tv, tk_tail, tv_tail, p)
+                      : cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 6, false, true>, tk, tv, tk_tail, tv_tail, p);
+        else if (big)
             err = fp8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 8, true, true>, tk, tv, tk_tail, tv_tail, p)
                       : cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 8, false, true>, tk, tv, tk_tail, tv_tail, p);
         else if (fp8)

@@ -36,14 +36,15 @@ bool make_tmap_rows_bf16(CUtensorMap *out, const void *base, int64_t n_cols, int
 int sm_count();
 
 struct DecodePlan {
-    int warps;       // kernel shape: 4 or 8 consumer warps (tile = 16 tokens per warp)
+    int warps;       // kernel shape: 4, 6 or 8 consumer warps (tile = 16 tokens per warp)
     bool fits;       // the shape's shared memory fits an SM
     int grid;        // persistent CTAs
     int min_tiles;   // floor on the 64-token tiles per CTA (bounds the pieces per sequence)
     int nsplit;      // max pieces a (sequence, KV head) can be cut into
     size_t ws_bytes; // status block + ticket counters + partials
 };
-DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_limit, bool fp8 = false);
+DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_limit, bool fp8 = false,
+                       bool paged = false);
 
 // Block table of a paged cache: token t of sequence b is in page block_table[b * table_stride + t / page_size].
 struct PagedTable {

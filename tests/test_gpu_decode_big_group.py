@@ -1,6 +1,7 @@
-"""Query-head groups of 5 to 8 at head_dim 128 on the split decode kernel: the consumer warps hand their results to two
-finisher warps in 16-bit rows (one rounding to bf16 per warp and piece ahead of the merge), so these shapes get their
-own parity cases: long ragged sequences cut between CTAs, the fused append, the fp8 cache."""
+"""Query-head groups of 5 to 16 at head_dim 128 on the split decode kernel: the consumer warps hand their results to one
+finisher warp per 4 heads in 16-bit rows (one rounding to bf16 per warp and piece ahead of the merge; 5 to 8 heads on
+the 8-warp shape, 9 to 16 on a 6-warp shape with 96-token tiles), so these shapes get their own parity cases: long
+ragged sequences cut between CTAs, the fused append, the fp8 cache."""
 import math
 import os
 
@@ -27,25 +28,28 @@ def split_kernel_only():
         os.environ["L4L_DECODE_CLUSTER"] = old
 
 
-@pytest.mark.parametrize("Hq,Hkv", [(40, 8), (48, 8), (56, 8), (64, 8), (8, 1), (5, 1)])
+@pytest.mark.parametrize("Hq,Hkv", [(40, 8), (48, 8), (56, 8), (64, 8), (8, 1), (5, 1), (72, 8), (96, 8), (128, 8), (16, 1),
+                                    (13, 1)])
 def test_big_group_decode_long_ragged(Hq, Hkv):
     lens = [4096, 0, 1, 129, 3000, 2049, 513, 17, 4000, 1234, 3333, 640]
     q, ck, cv, kv_len = random_batch(len(lens), Hq, Hkv, 128, 4096, lens, seed=300 + Hq)
     _, stats = check_decode(q, ck, cv, kv_len, 1.0 / math.sqrt(128))
 
 
-def test_big_group_decode_many_sequences_cut_between_ctas():
+@pytest.mark.parametrize("Hq", [64, 128])
+def test_big_group_decode_many_sequences_cut_between_ctas(Hq):
     # enough tiles that every CTA streams a range and most sequences are cut once
     g = torch.Generator().manual_seed(77)
     lens = torch.randint(512, 4097, (40,), generator=g).tolist()
-    q, ck, cv, kv_len = random_batch(len(lens), 64, 8, 128, 4096, lens, seed=78)
+    q, ck, cv, kv_len = random_batch(len(lens), Hq, 8, 128, 4096, lens, seed=78)
     check_decode(q, ck, cv, kv_len, 1.0 / math.sqrt(128))
 
 
-def test_big_group_decode_with_fused_append():
+@pytest.mark.parametrize("Hq", [64, 128])
+def test_big_group_decode_with_fused_append(Hq):
     from test_gpu_decode_append import make_case
 
-    Hq, Hkv, D = 64, 8, 128
+    Hkv, D = 8, 128
     lens = [0, 1, 2, 16, 17, 128, 129, 300, 1000, 2048]
     B, Lmax = len(lens), 2048
     q, ck, cv, kn, vn, kv_len = make_case(B, Hq, Hkv, D, Lmax, lens, seed=41)
@@ -72,3 +76,4 @@ def test_big_group_decode_fp8_cache():
 
     fp8_case(64, 8)
     fp8_case(40, 8)
+    fp8_case(128, 8)
