@@ -77,3 +77,26 @@ def test_big_group_decode_fp8_cache():
     fp8_case(64, 8)
     fp8_case(40, 8)
     fp8_case(128, 8)
+
+
+@pytest.mark.parametrize("Hq,page_size", [(64, 64), (64, 16), (128, 256), (128, 32)])
+def test_big_group_decode_paged(Hq, page_size):
+    # groups of 8 on the 8-warp shape; groups of 16 stay on the 4-warp shape with pages (96-token tiles would not line up)
+    B, Hkv, D = 6, 8, 128
+    lens = np.array([0, 1, 130, 700, 2048, 1999], np.int32)
+    g = torch.Generator().manual_seed(4321 + page_size + Hq)
+    max_pages = (2048 + page_size - 1) // page_size
+    n_pages = B * max_pages + 3
+    pool_k = torch.randn(n_pages, Hkv, page_size, D, generator=g).to(torch.bfloat16)
+    pool_v = torch.randn(n_pages, Hkv, page_size, D, generator=g).to(torch.bfloat16)
+    perm = torch.randperm(n_pages, generator=g)[:B * max_pages].to(torch.int32).view(B, max_pages)
+    q = torch.randn(B, Hq, D, generator=g).to(torch.bfloat16)
+    scale = 1.0 / math.sqrt(D)
+    ref, _ = orc.decode_paged(q, pool_k, pool_v, perm.numpy(), lens, scale)
+    o = torch.zeros(B, Hq, D, dtype=torch.bfloat16, device="cuda")
+    ws = l4l.new_workspace(l4l.L4L_OP_DECODE, B, Hq, Hkv, D, 2048)
+    l4l.l4l_attn_decode_paged(q.cuda(), o, pool_k.cuda(), pool_v.cuda(), perm.cuda(), torch.from_numpy(lens).cuda(),
+                              2048, scale, ws)
+    torch.cuda.synchronize()
+    assert l4l.l4l_last_device_error(ws) == 0
+    assert_close_to_oracle(o, ref, "big-group paged decode")
