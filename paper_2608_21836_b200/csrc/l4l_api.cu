@@ -196,8 +196,8 @@ size_t l4l_workspace_bytes(int op, int B, int Hq, int Hkv, int head_dim, int max
     if (op == L4L_OP_PREFILL) return kStatusBytes;
     if (op == L4L_OP_DECODE) {
         // the contiguous and the paged entry points may pick different kernel shapes: enough for either
-        const size_t a = plan_decode(B, Hq, Hkv, head_dim, max_len, (size_t)-1, false, false).ws_bytes;
-        const size_t b = plan_decode(B, Hq, Hkv, head_dim, max_len, (size_t)-1, false, true).ws_bytes;
+        const size_t a = plan_decode(B, Hq, Hkv, head_dim, max_len, (size_t)-1, false, 0).ws_bytes;
+        const size_t b = plan_decode(B, Hq, Hkv, head_dim, max_len, (size_t)-1, false, 64).ws_bytes;
         return a > b ? a : b;
     }
     return 0;
@@ -279,7 +279,7 @@ l4l_status l4l_attn_decode_paged(const void *q, void *o, l4l_paged_kv pool, cons
     if (max_kv_len < 0 || (long long)max_kv_len > (long long)table_stride * pool.page_size) return L4L_ERR_INVALID_ARG;
     if (!workspace || ws_bytes < kStatusBytes) return L4L_ERR_WORKSPACE;
     if (B == 0) return L4L_OK;
-    const DecodePlan plan = plan_decode(B, Hq, Hkv, head_dim, max_kv_len, ws_bytes, false, true);
+    const DecodePlan plan = plan_decode(B, Hq, Hkv, head_dim, max_kv_len, ws_bytes, false, pool.page_size);
     if (plan.ws_bytes > ws_bytes) return L4L_ERR_WORKSPACE;
     const PagedTable pt{d_block_table, table_stride, pool.num_pages};
     return launch_decode(q, o, pool_as_cache(pool), d_kv_lens, max_kv_len, B, Hq, Hkv, head_dim, scale, d_lse, workspace,
@@ -349,7 +349,7 @@ l4l_status l4l_attn_decode_paged_fp8(const void *q, void *o, l4l_paged_kv pool8,
     if (max_kv_len < 0 || (long long)max_kv_len > (long long)table_stride * pool8.page_size) return L4L_ERR_INVALID_ARG;
     if (!workspace || ws_bytes < kStatusBytes) return L4L_ERR_WORKSPACE;
     if (B == 0) return L4L_OK;
-    const DecodePlan plan = plan_decode(B, Hq, Hkv, head_dim, max_kv_len, ws_bytes, true, true);
+    const DecodePlan plan = plan_decode(B, Hq, Hkv, head_dim, max_kv_len, ws_bytes, true, pool8.page_size);
     if (plan.ws_bytes > ws_bytes) return L4L_ERR_WORKSPACE;
     const PagedTable pt{d_block_table, table_stride, pool8.num_pages};
     const Fp8Scales sc{d_k_scale, d_v_scale};

@@ -1090,14 +1090,14 @@ DecodePlan plan_for_shape(int B, int Hq, int Hkv, int D, int max_kv_len, size_t 
 
 }  // namespace
 
-DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_limit, bool fp8, bool paged)
+DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_limit, bool fp8, int page_size)
 {
     int n_dev = 0;
     const bool have_dev = cudaGetDeviceCount(&n_dev) == cudaSuccess && n_dev > 0;
     if (!have_dev) (void)cudaGetLastError();
-    // groups of 9 to 16 query heads at head_dim 128: the 6-warp shape (contiguous caches: its 96-token tiles do not
-    // line up with pages)
-    if (D == 128 && Hq / Hkv > 8 && !paged) {
+    // groups of 9 to 16 query heads at head_dim 128: the 6-warp shape (contiguous caches and pages of 16 or 32
+    // tokens: its 96-token tiles do not line up with larger pages)
+    if (D == 128 && Hq / Hkv > 8 && (page_size == 0 || page_size == 16 || page_size == 32)) {
         const DecodePlan six = plan_for_shape(B, Hq, Hkv, D, max_kv_len, ws_limit, 6, have_dev, fp8);
         if (six.fits && six.ws_bytes <= ws_limit) return six;
     }
@@ -1128,7 +1128,7 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
     const int esz = fp8 ? 1 : 2;
     // paged: `cache` describes the page pool (stride_b = stride between pages, max_len = page size)
     if (paged && (k_new || v_new)) return L4L_ERR_UNSUPPORTED;
-    if (paged && plan.warps == 6) return L4L_ERR_UNSUPPORTED;    // planned for a contiguous cache
+    if (paged && plan.warps == 6 && cache.max_len != 16 && cache.max_len != 32) return L4L_ERR_UNSUPPORTED;   // 96-token tiles
     {
         // small batches are latency-bound: one cluster per (sequence, KV head), no workspace round trips
         const int width = decode_cluster_width(B, Hq, Hkv, D, max_kv_len, fp8 != nullptr);

@@ -43,8 +43,10 @@ struct DecodePlan {
     int nsplit;      // max pieces a (sequence, KV head) can be cut into
     size_t ws_bytes; // status block + ticket counters + partials
 };
+// page_size: 0 for a contiguous cache, else the tokens per page of a paged cache (some kernel shapes need tiles
+// that line up with pages)
 DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_limit, bool fp8 = false,
-                       bool paged = false);
+                       int page_size = 0);
 
 // Block table of a paged cache: token t of sequence b is in page block_table[b * table_stride + t / page_size].
 struct PagedTable {

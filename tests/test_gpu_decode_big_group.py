@@ -79,9 +79,10 @@ def test_big_group_decode_fp8_cache():
     fp8_case(128, 8)
 
 
-@pytest.mark.parametrize("Hq,page_size", [(64, 64), (64, 16), (128, 256), (128, 32)])
+@pytest.mark.parametrize("Hq,page_size", [(64, 64), (64, 16), (128, 256), (128, 64), (128, 32), (128, 16)])
 def test_big_group_decode_paged(Hq, page_size):
-    # groups of 8 on the 8-warp shape; groups of 16 stay on the 4-warp shape with pages (96-token tiles would not line up)
+    # groups of 8 on the 8-warp shape; groups of 16 on the 6-warp shape with pages of 16 or 32 tokens (its 96-token
+    # tiles do not line up with larger pages: those stay on the 4-warp shape)
     B, Hkv, D = 6, 8, 128
     lens = np.array([0, 1, 130, 700, 2048, 1999], np.int32)
     g = torch.Generator().manual_seed(4321 + page_size + Hq)
