@@ -568,6 +568,7 @@ int resident_clusters(int C, size_t smem)
 // Host-side view of one instantiation.
 struct ClusterShape {
     int tile_t;
+    uint32_t stage_bytes;                      // K and V of one tile
     int (*stages)(int G);
     size_t (*smem)(int G, int stages);
     int (*resident)(int C, size_t smem);
@@ -577,7 +578,7 @@ struct ClusterShape {
 template <int D, bool F8>
 ClusterShape shape_of()
 {
-    return ClusterShape{ClusterCfg<D, F8>::kTileT, &pick_stages<D, F8>, &cluster_smem_bytes<D, F8>, &resident_clusters<D, F8>,
+    return ClusterShape{ClusterCfg<D, F8>::kTileT, ClusterCfg<D, F8>::kStageBytes, &pick_stages<D, F8>, &cluster_smem_bytes<D, F8>, &resident_clusters<D, F8>,
                         &configure_kernel<D, F8>};
 }
 
@@ -619,8 +620,10 @@ int decode_cluster_width(int B, int Hq, int Hkv, int D, int max_kv_len, bool fp8
     if (forced > 0) return C;
     // Beyond these bounds the even split of the whole tile stream over all SMs (the split kernel) wins: a lone CTA
     // per sequence streams at one SM's rate, and ragged lengths leave short sequences' CTAs idle.
-    const int per_cta = (tiles_max + C - 1) / C;
-    if (per_cta * shape.tile_t > 32 * 128) return 0;
+    // (measured on ragged batches of 8 to 16 sequences of up to 4096 tokens: with one CTA per sequence the cluster
+    // kernel wins up to about 1 MB of cache per CTA, with two or more up to about 2 MB)
+    const long long per_cta_bytes = (long long)((tiles_max + C - 1) / C) * shape.stage_bytes;
+    if (per_cta_bytes > (C == 1 ? (1ll << 20) : (2ll << 20))) return 0;
     return C;
 }
 
