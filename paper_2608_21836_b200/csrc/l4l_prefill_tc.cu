@@ -38,7 +38,7 @@ template <int D>
 struct TcCfg {
     static constexpr int kHalves = D / 64;
     static constexpr uint32_t kTileBytes = kHalves * kHalfBytes;        // one Q sub-tile, K tile or V tile
-    static constexpr int kSlots = (D == 128) ? 4 : 8;                    // ring of K/V tiles
+    static constexpr int kSlots = (D == 128) ? 5 : 8;                    // ring of K/V tiles
     static constexpr uint32_t kTmemCols = 512;
     static constexpr uint32_t kColS0 = 0, kColS1 = 128, kColO0 = 256, kColO1 = 256 + D;
     static constexpr int kNumBars = 1 + 2 * kSlots + 8;
