@@ -19,17 +19,20 @@ struct AppendParams {
     int B, T, Hkv, pieces, max_len;
 };
 
+// Idx: unsigned 32-bit when the piece count fits (the index arithmetic is four divisions per piece, which in 64 bits
+// cost more than the copy), 64-bit otherwise.
+template <typename Idx>
 __global__ void __launch_bounds__(256) kv_append_kernel(const AppendParams p)
 {
-    const long long total = (long long)p.B * p.T * p.Hkv * p.pieces;
-    for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
-         idx += (long long)gridDim.x * blockDim.x) {
-        const int piece = (int)(idx % p.pieces);
-        long long rest = idx / p.pieces;
-        const int g = (int)(rest % p.Hkv);
-        rest /= p.Hkv;
-        const int r = (int)(rest % p.T);
-        const int b = (int)(rest / p.T);
+    const Idx total = (Idx)p.B * (Idx)p.T * (Idx)p.Hkv * (Idx)p.pieces;
+    const Idx step = (Idx)gridDim.x * blockDim.x;
+    for (Idx idx = (Idx)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += step) {
+        const int piece = (int)(idx % (Idx)p.pieces);
+        Idx rest = idx / (Idx)p.pieces;
+        const int g = (int)(rest % (Idx)p.Hkv);
+        rest /= (Idx)p.Hkv;
+        const int r = (int)(rest % (Idx)p.T);
+        const int b = (int)(rest / (Idx)p.T);
         const int n = p.n_new ? p.n_new[b] : p.T;
         if (r >= n) continue;
         long long slot = (long long)p.write_pos[b] + r;
@@ -78,7 +81,11 @@ l4l_status launch_kv_append(const l4l_kv_cache &cache, const l4l_tensor4 &k_new,
     long long blocks = (total + 255) / 256;
     const long long cap = 8ll * sm_count();
     if (blocks > cap) blocks = cap;
-    kv_append_kernel<<<(int)blocks, 256, 0, stream>>>(p);
+    // (the 32-bit index also has to hold idx + grid step without wrapping)
+    if (total + blocks * 256 < (1ll << 32))
+        kv_append_kernel<uint32_t><<<(int)blocks, 256, 0, stream>>>(p);
+    else
+        kv_append_kernel<unsigned long long><<<(int)blocks, 256, 0, stream>>>(p);
     return cudaGetLastError() == cudaSuccess ? L4L_OK : L4L_ERR_CUDA;
 }
 
