@@ -36,7 +36,7 @@ FALLBACK_TFLOPS, FALLBACK_GBS = 1590.0, 6650.0
 # profiles/: prefill captured at B=1,S=8192 (155.8 MB) and scaled x4 to the bench's B=4 (traffic is proportional
 # to B); decode captured on the bench's own batch.
 NCU_TRAFFIC_PREFILL = 628.1e6   # 4 x (101.0 MB read + 56.1 MB written)
-NCU_TRAFFIC_DECODE = 302.2e6    # 295.9 MB read + 4.2 MB written
+NCU_TRAFFIC_DECODE = 302.2e6    # 297.8 MB read + 4.4 MB written
 
 
 def measured_peaks():
