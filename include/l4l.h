@@ -18,8 +18,8 @@
  * Further entry points widen that path, each documented at its declaration:
  *   l4l_attn_prefill_chunk (new tokens over a populated cache), l4l_attn_decode_append (cache
  *   update fused into the decode step), l4l_rope_kv_append (rotary embedding and QK-norm fused
- *   with the cache update), l4l_attn_decode_paged / l4l_kv_append_paged (page pool + block
- *   table), l4l_attn_decode_fp8 / l4l_kv_append_fp8 (e4m3 cache), l4l_attn_decode_static (no
+ *   with the cache update), l4l_attn_decode_paged / l4l_kv_append_paged / l4l_attn_decode_paged_append
+ *   (page pool + block table), l4l_attn_decode_fp8 / l4l_kv_append_fp8 (e4m3 cache), l4l_attn_decode_static (no
  *   caller workspace), and a second workload, l4l_rglru_scan (gated linear recurrence).
  *
  * Conventions shared by every call
@@ -144,6 +144,18 @@ l4l_status l4l_attn_decode_paged(const void *q, void *o, l4l_paged_kv pool, cons
                                  int table_stride, const int32_t *d_kv_lens, int max_kv_len,
                                  int B, int Hq, int Hkv, int head_dim, float scale, float *d_lse,
                                  void *workspace, size_t ws_bytes, l4l_stream stream);
+/*
+ * l4l_attn_decode_append over a paged cache: the step's newest token (k_new / v_new, [B, 1, Hkv, D]) goes to
+ * slot kv_lens[b] - 1 of sequence b, i.e. to page block_table[b][(kv_lens[b]-1) / page_size], bit for bit, and
+ * is attended with the rest in the same launch. Equivalent to l4l_kv_append_paged at that slot followed by
+ * l4l_attn_decode_paged; a sequence whose table has no valid page for the slot gets no write (as in
+ * l4l_kv_append_paged) and attends over zeros there. Sequences with kv_lens[b] = 0 append nothing.
+ */
+l4l_status l4l_attn_decode_paged_append(const void *q, void *o, l4l_paged_kv pool, const int32_t *d_block_table,
+                                        int table_stride, l4l_tensor4 k_new, l4l_tensor4 v_new,
+                                        const int32_t *d_kv_lens, int max_kv_len, int B, int Hq, int Hkv,
+                                        int head_dim, float scale, float *d_lse, void *workspace, size_t ws_bytes,
+                                        l4l_stream stream);
 
 /*
  * The same two operations over an fp8 cache (e4m3: 1 sign, 4 exponent, 3 mantissa bits, largest

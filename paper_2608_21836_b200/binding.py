@@ -24,7 +24,7 @@ EXPORTS = (
     "l4l_last_device_error", "l4l_kv_append", "l4l_attn_prefill", "l4l_attn_decode",
     "l4l_attn_decode_static", "l4l_attn_decode_append", "l4l_attn_prefill_chunk", "l4l_rope_kv_append",
     "l4l_kv_append_paged", "l4l_attn_decode_paged", "l4l_kv_append_fp8", "l4l_attn_decode_fp8", "l4l_rglru_scan", "l4l_rglru_workspace_bytes",
-    "l4l_attn_decode_paged_fp8", "l4l_attn_merge", "l4l_attn_decode_rope_append",
+    "l4l_attn_decode_paged_fp8", "l4l_attn_merge", "l4l_attn_decode_rope_append", "l4l_attn_decode_paged_append",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -89,6 +89,9 @@ def load() -> ctypes.CDLL:
     lib.l4l_attn_decode_paged.restype = c_int
     lib.l4l_attn_decode_paged.argtypes = [vp, vp, PagedKV, i32p, c_int, i32p, c_int, c_int, c_int, c_int, c_int,
                                           ctypes.c_float, vp, vp, c_size, vp]
+    lib.l4l_attn_decode_paged_append.restype = c_int
+    lib.l4l_attn_decode_paged_append.argtypes = [vp, vp, PagedKV, i32p, c_int, Tensor4, Tensor4, i32p, c_int, c_int, c_int,
+                                                 c_int, c_int, ctypes.c_float, vp, vp, c_size, vp]
     lib.l4l_kv_append_fp8.restype = c_int
     lib.l4l_kv_append_fp8.argtypes = [KVCache, Tensor4, Tensor4, i32p, i32p, c_int, c_int, c_int, c_int, vp, vp, vp]
     lib.l4l_attn_decode_fp8.restype = c_int
@@ -367,6 +370,32 @@ def l4l_attn_decode_paged(q, o, pool_k, pool_v, block_table, kv_lens, max_kv_len
                                       workspace.numel() * workspace.element_size(), _stream())
     if st != L4L_OK:
         raise L4LError(st, "l4l_attn_decode_paged")
+
+
+def l4l_attn_decode_paged_append(q, o, pool_k, pool_v, block_table, k_new, v_new, kv_lens, max_kv_len: int, scale: float,
+                                 workspace, lse=None) -> None:
+    """One launch per decode step over a paged cache: k_new / v_new ([B,1,Hkv,D]) go to slot kv_lens[b]-1 of sequence b
+    (the page the block table names) and are attended with the rest. Same result as l4l_kv_append_paged followed by
+    l4l_attn_decode_paged."""
+    _check_bf16_cuda(q, "q")
+    _check_bf16_cuda(o, "o")
+    if not (q.is_contiguous() and o.is_contiguous() and q.dim() == 3 and q.shape == o.shape):
+        raise ValueError("q and o must be dense [B, Hq, D]")
+    B, Hq, D = q.shape
+    Hkv = pool_k.shape[1]
+    if tuple(k_new.shape) != (B, 1, Hkv, D) or tuple(v_new.shape) != (B, 1, Hkv, D):
+        raise ValueError("k_new and v_new must be [B, 1, Hkv, D]")
+    if lse is not None and not (lse.is_cuda and lse.dtype == torch.float32 and lse.is_contiguous()
+                                and tuple(lse.shape) == (B, Hq)):
+        raise TypeError("lse must be a contiguous CUDA float32 tensor [B, Hq]")
+    tbl, stride = _block_table(block_table, B)
+    st = load().l4l_attn_decode_paged_append(q.data_ptr(), o.data_ptr(), paged_kv(pool_k, pool_v), tbl, stride,
+                                             tensor4(k_new), tensor4(v_new), _i32_dev(kv_lens, "kv_lens"),
+                                             int(max_kv_len), B, Hq, Hkv, D, float(scale),
+                                             None if lse is None else lse.data_ptr(), workspace.data_ptr(),
+                                             workspace.numel() * workspace.element_size(), _stream())
+    if st != L4L_OK:
+        raise L4LError(st, "l4l_attn_decode_paged_append")
 
 
 def kv_cache8(cache_k8, cache_v8) -> KVCache:

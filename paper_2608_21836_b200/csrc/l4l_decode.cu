@@ -113,7 +113,7 @@ struct DecodeParams {
     // paged cache (null: contiguous): token t of sequence b lives in page block_table[b * table_stride + t / page_size]
     // at offset t % page_size; the tensor maps then describe the page pool [pages, Hkv, page_size, D]
     const int32_t *block_table;
-    int table_stride, page_size, page_shift;
+    int table_stride, page_size, page_shift, num_pages;
     int tail_rows;            // tokens per box of tmap_k_tail / tmap_v_tail (32, or the page size if that is smaller)
     int B, Hq, Hkv, G, min_tiles, nsplit, max_kv_len;
     int nfin;                 // finisher warps (BigG: one per 4 query heads of the group; else 1)
@@ -802,14 +802,22 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     kk = rope_k_row<D>(kk, p.k_weight != nullptr, p.norm_eps, rope_priv + (size_t)warp * D, norm_w + D,
                                         mt.kv_len - 1 < p.rope_n_pos, lane);
                 if (lane < kChunks) {
-                    uint8_t *kt = stages + (size_t)s * C::kStageBytes;
-                    const uint32_t off = (lane >> 3) * C::kHalfBytes + swz128(last, lane & 7);
-                    *reinterpret_cast<uint4 *>(kt + off) = kk;
-                    *reinterpret_cast<uint4 *>(kt + C::kTileBytes + off) = vv;
-                    const size_t dst = (size_t)mt.b * p.c_sb + (size_t)mt.kvh * p.c_sh +
-                                       (size_t)(mt.kv_len - 1) * p.c_st + lane * 8;
-                    *reinterpret_cast<uint4 *>(p.cache_k + dst) = kk;
-                    *reinterpret_cast<uint4 *>(p.cache_v + dst) = vv;
+                    // the slot in the cache: with pages, behind the block table. No page there: nothing is written,
+                    // and the tile keeps the zeros that the fetch of a missing page delivers.
+                    long long outer = mt.b, slot = mt.kv_len - 1;
+                    if (p.block_table != nullptr) {
+                        outer = __ldg(p.block_table + (size_t)mt.b * p.table_stride + (slot >> p.page_shift));
+                        slot &= p.page_size - 1;
+                    }
+                    if (p.block_table == nullptr || (outer >= 0 && outer < p.num_pages)) {
+                        uint8_t *kt = stages + (size_t)s * C::kStageBytes;
+                        const uint32_t off = (lane >> 3) * C::kHalfBytes + swz128(last, lane & 7);
+                        *reinterpret_cast<uint4 *>(kt + off) = kk;
+                        *reinterpret_cast<uint4 *>(kt + C::kTileBytes + off) = vv;
+                        const size_t dst = (size_t)outer * p.c_sb + (size_t)mt.kvh * p.c_sh + (size_t)slot * p.c_st + lane * 8;
+                        *reinterpret_cast<uint4 *>(p.cache_k + dst) = kk;
+                        *reinterpret_cast<uint4 *>(p.cache_v + dst) = vv;
+                    }
                 }
                 wrote_smem = true;
                 __syncwarp();
@@ -1127,7 +1135,6 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
     if (fp8 && (D != 128 || k_new || v_new)) return L4L_ERR_UNSUPPORTED;
     const int esz = fp8 ? 1 : 2;
     // paged: `cache` describes the page pool (stride_b = stride between pages, max_len = page size)
-    if (paged && (k_new || v_new)) return L4L_ERR_UNSUPPORTED;
     if (paged && plan.warps == 6 && cache.max_len != 16 && cache.max_len != 32) return L4L_ERR_UNSUPPORTED;   // 96-token tiles
     {
         // small batches are latency-bound: one cluster per (sequence, KV head), no workspace round trips
@@ -1200,12 +1207,13 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         p.block_table = paged ? paged->block_table + (size_t)b0 * paged->table_stride : nullptr;
         p.table_stride = paged ? paged->table_stride : 0;
         p.page_size = paged ? cache.max_len : 0;
+        p.num_pages = paged ? paged->num_pages : 0;
         p.tail_rows = tail_rows;
         p.page_shift = 0;
         while (paged && (1 << p.page_shift) < cache.max_len) ++p.page_shift;
         // only the fused append (bf16, contiguous) writes through these
-        p.cache_k = static_cast<__nv_bfloat16 *>(cache.k) + (fp8 ? 0 : (size_t)b0 * cache.stride_b);
-        p.cache_v = static_cast<__nv_bfloat16 *>(cache.v) + (fp8 ? 0 : (size_t)b0 * cache.stride_b);
+        p.cache_k = static_cast<__nv_bfloat16 *>(cache.k) + ((fp8 || paged) ? 0 : (size_t)b0 * cache.stride_b);
+        p.cache_v = static_cast<__nv_bfloat16 *>(cache.v) + ((fp8 || paged) ? 0 : (size_t)b0 * cache.stride_b);
         p.c_sb = cache.stride_b; p.c_sh = cache.stride_h; p.c_st = cache.stride_t;
         if (k_new && v_new) {
             if (k_new->stride_b != v_new->stride_b || k_new->stride_h != v_new->stride_h) return L4L_ERR_UNSUPPORTED;

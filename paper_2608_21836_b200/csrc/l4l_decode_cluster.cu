@@ -58,7 +58,7 @@ struct ClusterParams {
     int64_t c_sb, c_sh, c_st;
     unsigned *status;
     const int32_t *block_table;               // paged cache (null: contiguous)
-    int table_stride, page_size, page_shift;
+    int table_stride, page_size, page_shift, num_pages;
     int tail_rows;                            // tokens per box of the tail maps (32, or the page size if that is smaller)
     // rotary embedding (+ optional RMS norm) of the step's q and k_new (null: inputs are final); only with the fused
     // append. The new token's position is kv_len - 1.
@@ -298,13 +298,22 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                 if (p.rope_cos != nullptr)                                      // all lanes: shuffles inside
                     kk = rope_k_row<D>(kk, p.k_weight != nullptr, p.norm_eps, rope_cs, norm_w + D, with_rope, lane);
                 if (lane < kChunks) {
-                    uint8_t *kt = stages + (size_t)s * C::kStageBytes;
-                    const uint32_t off = (lane >> 3) * kHalfBytes + swz128(last, lane & 7);
-                    *reinterpret_cast<uint4 *>(kt + off) = kk;
-                    *reinterpret_cast<uint4 *>(kt + C::kTileBytes + off) = vv;
-                    const size_t dst = (size_t)b * p.c_sb + (size_t)kvh * p.c_sh + (size_t)(len - 1) * p.c_st + lane * 8;
-                    *reinterpret_cast<uint4 *>(p.cache_k + dst) = kk;
-                    *reinterpret_cast<uint4 *>(p.cache_v + dst) = vv;
+                    // the slot in the cache: with pages, behind the block table. No page there: nothing is written,
+                    // and the tile keeps the zeros that the fetch of a missing page delivers.
+                    long long outer = b, slot = len - 1;
+                    if (p.block_table != nullptr) {
+                        outer = __ldg(p.block_table + (size_t)b * p.table_stride + (slot >> p.page_shift));
+                        slot &= p.page_size - 1;
+                    }
+                    if (p.block_table == nullptr || (outer >= 0 && outer < p.num_pages)) {
+                        uint8_t *kt = stages + (size_t)s * C::kStageBytes;
+                        const uint32_t off = (lane >> 3) * kHalfBytes + swz128(last, lane & 7);
+                        *reinterpret_cast<uint4 *>(kt + off) = kk;
+                        *reinterpret_cast<uint4 *>(kt + C::kTileBytes + off) = vv;
+                        const size_t dst = (size_t)outer * p.c_sb + (size_t)kvh * p.c_sh + (size_t)slot * p.c_st + lane * 8;
+                        *reinterpret_cast<uint4 *>(p.cache_k + dst) = kk;
+                        *reinterpret_cast<uint4 *>(p.cache_v + dst) = vv;
+                    }
                 }
                 wrote_smem = true;
                 __syncwarp();
@@ -633,8 +642,7 @@ l4l_status launch_decode_cluster(const void *q, void *o, const l4l_kv_cache &cac
                                  const l4l_tensor4 *v_new, const PagedTable *paged, const RopeArgs *rope,
                                  const Fp8Scales *fp8, int width)
 {
-    if (paged && (k_new || v_new)) return L4L_ERR_UNSUPPORTED;
-    if (rope && (!k_new || !v_new)) return L4L_ERR_UNSUPPORTED;      // only with the fused append
+    if (rope && (!k_new || !v_new || paged)) return L4L_ERR_UNSUPPORTED;      // only with the fused append, contiguous
     if (fp8 && (D != 128 || k_new || v_new || rope)) return L4L_ERR_UNSUPPORTED;
     // fp8: cache.k / cache.v point at e4m3 bytes, the strides count bytes (= elements)
     const int esz = fp8 ? 1 : 2, box_d = fp8 ? 128 : 64;
@@ -681,6 +689,7 @@ l4l_status launch_decode_cluster(const void *q, void *o, const l4l_kv_cache &cac
     p.block_table = paged ? paged->block_table : nullptr;
     p.table_stride = paged ? paged->table_stride : 0;
     p.page_size = paged ? cache.max_len : 0;
+    p.num_pages = paged ? paged->num_pages : 0;
     p.tail_rows = tail_rows;
     p.page_shift = 0;
     while (paged && (1 << p.page_shift) < cache.max_len) ++p.page_shift;
