@@ -193,7 +193,7 @@ l4l_status l4l_attn_decode_paged_fp8(const void *q, void *o, l4l_paged_kv pool8,
  * the rotated q attends over slots 0 .. kv_lens[b] - 1. Same result as l4l_rope_kv_append (T = 1) followed by
  * l4l_attn_decode, up to the last bf16 bit of the rotated values (the sum of squares of the norm is reduced
  * in a different order). q is NOT modified (the rotated values live in registers only). A position outside
- * [0, n_pos) leaves q and k unrotated. bf16 contiguous cache only.
+ * [0, n_pos) leaves q and k unrotated. bf16 caches only.
  *   arguments as for l4l_attn_decode_append and l4l_rope_kv_append
  */
 l4l_status l4l_attn_decode_rope_append(const void *q, void *o, l4l_kv_cache cache, l4l_tensor4 k_new, l4l_tensor4 v_new,
@@ -201,6 +201,14 @@ l4l_status l4l_attn_decode_rope_append(const void *q, void *o, l4l_kv_cache cach
                                        int head_dim, float scale, const float *d_cos, const float *d_sin, int n_pos,
                                        const float *d_q_weight, const float *d_k_weight, float norm_eps,
                                        float *d_lse, void *workspace, size_t ws_bytes, l4l_stream stream);
+/* The same step over a paged cache (l4l_attn_decode_paged_append with the rotation and normalisation of
+ * l4l_attn_decode_rope_append): the rotated k and v_new go to the page slot of position kv_lens[b] - 1. */
+l4l_status l4l_attn_decode_paged_rope_append(const void *q, void *o, l4l_paged_kv pool, const int32_t *d_block_table,
+                                             int table_stride, l4l_tensor4 k_new, l4l_tensor4 v_new,
+                                             const int32_t *d_kv_lens, int max_kv_len, int B, int Hq, int Hkv,
+                                             int head_dim, float scale, const float *d_cos, const float *d_sin, int n_pos,
+                                             const float *d_q_weight, const float *d_k_weight, float norm_eps,
+                                             float *d_lse, void *workspace, size_t ws_bytes, l4l_stream stream);
 
 /*
  * Merge of R partial decode results over DISJOINT parts of the same sequences' caches: the step that

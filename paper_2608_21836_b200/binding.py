@@ -25,6 +25,7 @@ EXPORTS = (
     "l4l_attn_decode_static", "l4l_attn_decode_append", "l4l_attn_prefill_chunk", "l4l_rope_kv_append",
     "l4l_kv_append_paged", "l4l_attn_decode_paged", "l4l_kv_append_fp8", "l4l_attn_decode_fp8", "l4l_rglru_scan", "l4l_rglru_workspace_bytes",
     "l4l_attn_decode_paged_fp8", "l4l_attn_merge", "l4l_attn_decode_rope_append", "l4l_attn_decode_paged_append",
+    "l4l_attn_decode_paged_rope_append",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -92,6 +93,10 @@ def load() -> ctypes.CDLL:
     lib.l4l_attn_decode_paged_append.restype = c_int
     lib.l4l_attn_decode_paged_append.argtypes = [vp, vp, PagedKV, i32p, c_int, Tensor4, Tensor4, i32p, c_int, c_int, c_int,
                                                  c_int, c_int, ctypes.c_float, vp, vp, c_size, vp]
+    lib.l4l_attn_decode_paged_rope_append.restype = c_int
+    lib.l4l_attn_decode_paged_rope_append.argtypes = [vp, vp, PagedKV, i32p, c_int, Tensor4, Tensor4, i32p, c_int, c_int,
+                                                      c_int, c_int, c_int, ctypes.c_float, vp, vp, c_int, vp, vp,
+                                                      ctypes.c_float, vp, vp, c_size, vp]
     lib.l4l_kv_append_fp8.restype = c_int
     lib.l4l_kv_append_fp8.argtypes = [KVCache, Tensor4, Tensor4, i32p, i32p, c_int, c_int, c_int, c_int, vp, vp, vp]
     lib.l4l_attn_decode_fp8.restype = c_int
@@ -396,6 +401,31 @@ def l4l_attn_decode_paged_append(q, o, pool_k, pool_v, block_table, k_new, v_new
                                              workspace.numel() * workspace.element_size(), _stream())
     if st != L4L_OK:
         raise L4LError(st, "l4l_attn_decode_paged_append")
+
+
+def l4l_attn_decode_paged_rope_append(q, o, pool_k, pool_v, block_table, k_new, v_new, kv_lens, max_kv_len: int,
+                                      scale: float, cos, sin, workspace, q_weight=None, k_weight=None, eps: float = 0.0,
+                                      lse=None) -> None:
+    """l4l_attn_decode_rope_append over a paged cache: rotation (+ optional RMS norm) of q and k_new at position
+    kv_lens - 1, write of the rotated k and of v_new into the page slot, attention: one launch."""
+    _check_bf16_cuda(q, "q")
+    _check_bf16_cuda(o, "o")
+    if not (q.is_contiguous() and o.is_contiguous() and q.dim() == 3 and q.shape == o.shape):
+        raise ValueError("q and o must be dense [B, Hq, D]")
+    B, Hq, D = q.shape
+    Hkv = pool_k.shape[1]
+    if tuple(k_new.shape) != (B, 1, Hkv, D) or tuple(v_new.shape) != (B, 1, Hkv, D):
+        raise ValueError("k_new and v_new must be [B, 1, Hkv, D]")
+    n_pos = cos.shape[0]
+    tbl, stride = _block_table(block_table, B)
+    st = load().l4l_attn_decode_paged_rope_append(
+        q.data_ptr(), o.data_ptr(), paged_kv(pool_k, pool_v), tbl, stride, tensor4(k_new, "k_new"), tensor4(v_new, "v_new"),
+        _i32_dev(kv_lens, "kv_lens"), int(max_kv_len), B, Hq, Hkv, D, float(scale),
+        _f32_dev(cos, "cos", (n_pos, D // 2)), _f32_dev(sin, "sin", (n_pos, D // 2)), n_pos,
+        _f32_dev(q_weight, "q_weight", (D,)), _f32_dev(k_weight, "k_weight", (D,)), float(eps),
+        None if lse is None else lse.data_ptr(), workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream())
+    if st != L4L_OK:
+        raise L4LError(st, "l4l_attn_decode_paged_rope_append")
 
 
 def kv_cache8(cache_k8, cache_v8) -> KVCache:

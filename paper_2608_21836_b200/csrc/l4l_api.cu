@@ -510,4 +510,29 @@ l4l_status l4l_attn_decode_rope_append(const void *q, void *o, l4l_kv_cache cach
                          static_cast<cudaStream_t>(stream), &k_new, &v_new, nullptr, nullptr, &rope);
 }
 
+l4l_status l4l_attn_decode_paged_rope_append(const void *q, void *o, l4l_paged_kv pool, const int32_t *d_block_table,
+                                             int table_stride, l4l_tensor4 k_new, l4l_tensor4 v_new,
+                                             const int32_t *d_kv_lens, int max_kv_len, int B, int Hq, int Hkv,
+                                             int head_dim, float scale, const float *d_cos, const float *d_sin, int n_pos,
+                                             const float *d_q_weight, const float *d_k_weight, float norm_eps,
+                                             float *d_lse, void *workspace, size_t ws_bytes, l4l_stream stream)
+{
+    l4l_status st = shape_status(B, Hq, Hkv, head_dim);
+    if (st != L4L_OK) return st;
+    if (!q || !o || !d_kv_lens || !d_block_table || !aligned16(q) || !aligned16(o)) return L4L_ERR_INVALID_ARG;
+    if (!pool_ok(pool) || table_stride <= 0) return L4L_ERR_INVALID_ARG;
+    if (!tensor4_ok(k_new) || !tensor4_ok(v_new)) return L4L_ERR_INVALID_ARG;
+    if (max_kv_len < 0 || (long long)max_kv_len > (long long)table_stride * pool.page_size) return L4L_ERR_INVALID_ARG;
+    if (!d_cos || !d_sin || n_pos < 0 || !(norm_eps >= 0.f)) return L4L_ERR_INVALID_ARG;
+    if (!aligned16(d_cos) || !aligned16(d_sin)) return L4L_ERR_INVALID_ARG;      // rows are fetched with bulk copies
+    if (!workspace || ws_bytes < kStatusBytes) return L4L_ERR_WORKSPACE;
+    if (B == 0) return L4L_OK;
+    const DecodePlan plan = plan_decode(B, Hq, Hkv, head_dim, max_kv_len, ws_bytes, false, pool.page_size);
+    if (plan.ws_bytes > ws_bytes) return L4L_ERR_WORKSPACE;
+    const PagedTable pt{d_block_table, table_stride, pool.num_pages};
+    const RopeArgs rope{d_cos, d_sin, d_q_weight, d_k_weight, norm_eps, n_pos};
+    return launch_decode(q, o, pool_as_cache(pool), d_kv_lens, max_kv_len, B, Hq, Hkv, head_dim, scale, d_lse, workspace,
+                         plan, static_cast<cudaStream_t>(stream), &k_new, &v_new, &pt, nullptr, &rope);
+}
+
 }  // extern "C"

@@ -1130,7 +1130,7 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
                          void *workspace, const DecodePlan &plan, cudaStream_t stream, const l4l_tensor4 *k_new,
                          const l4l_tensor4 *v_new, const PagedTable *paged, const Fp8Scales *fp8, const RopeArgs *rope)
 {
-    if (rope && (!k_new || !v_new || fp8 || paged)) return L4L_ERR_UNSUPPORTED;   // only with the plain fused append
+    if (rope && (!k_new || !v_new || fp8)) return L4L_ERR_UNSUPPORTED;   // only with the fused append, bf16 caches
     // fp8: cache.k / cache.v point at e4m3 bytes, the strides count bytes (= elements)
     if (fp8 && (D != 128 || k_new || v_new)) return L4L_ERR_UNSUPPORTED;
     const int esz = fp8 ? 1 : 2;

@@ -642,7 +642,7 @@ l4l_status launch_decode_cluster(const void *q, void *o, const l4l_kv_cache &cac
                                  const l4l_tensor4 *v_new, const PagedTable *paged, const RopeArgs *rope,
                                  const Fp8Scales *fp8, int width)
 {
-    if (rope && (!k_new || !v_new || paged)) return L4L_ERR_UNSUPPORTED;      // only with the fused append, contiguous
+    if (rope && (!k_new || !v_new)) return L4L_ERR_UNSUPPORTED;               // only with the fused append
     if (fp8 && (D != 128 || k_new || v_new || rope)) return L4L_ERR_UNSUPPORTED;
     // fp8: cache.k / cache.v point at e4m3 bytes, the strides count bytes (= elements)
     const int esz = fp8 ? 1 : 2, box_d = fp8 ? 128 : 64;

@@ -104,3 +104,56 @@ def test_paged_decode_append_rejects_bad_arguments():
         l4l.l4l_attn_decode_paged_append(q, q.clone(), pool, pool.clone(), table, kn, kn.clone(), lens, 33, 0.1, ws)
     with pytest.raises(ValueError):               # one new token per sequence
         l4l.l4l_attn_decode_paged_append(q, q.clone(), pool, pool.clone(), table, kn[:, :, :1], kn, lens, 16, 0.1, ws)
+
+
+# ---- the rope-fused step over a paged cache ----
+
+@pytest.mark.parametrize("kernel_choice", [None, 0, 2], indirect=True)
+@pytest.mark.parametrize("page", [16, 128])
+@pytest.mark.parametrize("Hq,Hkv,D,norm", [(32, 8, 128, True), (8, 2, 64, False), (64, 8, 128, True)])
+def test_paged_decode_rope_append_matches_oracle_chain(kernel_choice, page, Hq, Hkv, D, norm):
+    """Oracle chain: rotate (and normalise) q and k_new at position kv_len - 1, write the page slot, decode over the
+    pages; three consecutive steps on the same pool."""
+    from paper_2608_21836_b200.workloads import make_rope_tables
+    from test_gpu_rope_append import assert_bf16_close
+
+    lens = np.array([1, 16, 17, 128, 129, 600, 255, 0], np.int32)      # INCLUDING the new token at the first step
+    B, steps = len(lens), 3
+    pool_k, pool_v, table = build_pool(B, Hkv, D, page, [int(x) + steps for x in lens], seed=300 + page + Hq)
+    pool_k = torch.nan_to_num(pool_k, nan=0.5)                           # slots past the lengths: finite fill
+    pool_v = torch.nan_to_num(pool_v, nan=-0.25)
+    n_pos = 640
+    cos, sin = make_rope_tables(n_pos, D)
+    g = torch.Generator().manual_seed(31 + D + page)
+    qw = (torch.rand(D, generator=g) + 0.5) if norm else None
+    kw = (torch.rand(D, generator=g) + 0.5) if norm else None
+    eps = 1e-6 if norm else 0.0
+    scale = 1.0 / math.sqrt(D)
+    dpk, dpv = pool_k.cuda(), pool_v.cuda()
+    opk, opv = orc.bits(pool_k), orc.bits(pool_v)
+    dtab = torch.from_numpy(table).cuda()
+    max_len = int(lens.max()) + steps
+    ws = l4l.new_workspace(l4l.L4L_OP_DECODE, B, Hq, Hkv, D, max_len)
+    dcos, dsin = cos.cuda(), sin.cuda()
+    for s in range(steps):
+        q = torch.randn(B, Hq, D, generator=g).to(torch.bfloat16)
+        kn = torch.randn(B, 1, Hkv, D, generator=g).to(torch.bfloat16)
+        vn = torch.randn(B, 1, Hkv, D, generator=g).to(torch.bfloat16)
+        cur = np.where(lens > 0, lens + s, 0).astype(np.int32)
+        pos = np.maximum(cur - 1, 0)
+        # the oracle's rotation through a one-slot-per-position scratch cache, read back at the written slot
+        sk = np.zeros((B, Hkv, n_pos, D), np.uint16)
+        oq, sk, _, _, _ = orc.rope_kv_append(q.view(B, 1, Hq, D), kn, vn, sk, sk.copy(), pos, None, cos.numpy(), sin.numpy(),
+                                             None if qw is None else qw.numpy(), None if kw is None else kw.numpy(), eps)
+        k_rot = np.stack([sk[b, :, pos[b]] for b in range(B)])[:, None]           # [B, 1, Hkv, D] bits
+        opk, opv = orc.kv_append_paged(opk, opv, table, k_rot, vn, pos, (cur > 0).astype(np.int32))
+        ref, _ = orc.decode_paged(oq[:, 0], opk, opv, table, cur, scale)
+        o = torch.zeros(B, Hq, D, dtype=torch.bfloat16, device="cuda")
+        l4l.l4l_attn_decode_paged_rope_append(q.cuda(), o, dpk, dpv, dtab, kn.cuda(), vn.cuda(), torch.from_numpy(cur).cuda(),
+                                              max_len, scale, dcos, dsin, ws, q_weight=None if qw is None else qw.cuda(),
+                                              k_weight=None if kw is None else kw.cuda(), eps=eps)
+        torch.cuda.synchronize()
+        assert l4l.l4l_last_device_error(ws) == 0
+        assert_close_to_oracle(o.cpu(), ref, f"paged rope + append + decode, step {s}")
+    assert_bf16_close(dpk, opk, "pool k after the fused steps")
+    assert np.array_equal(orc.bits(dpv.cpu()), opv)
