@@ -586,7 +586,7 @@ def run_ours(args, rank, world):
 def run_profile_case(case: str):
     """A few launches of ONE kernel on a small case, for `ncu` captures (not a benchmark):
     prefill = B=1, S=8192 of the long_prefill workload (inputs 168 MB > L2); decode = the batched_decode batch;
-    rglru = the RG-LRU scan on B=16, T=2048, W=2560; decode_small = the cluster decode kernel on B=4 x 8192 tokens; rope = rope + norm + cache update on B=2, S=8192."""
+    rglru = the RG-LRU scan on B=16, T=2048, W=2560; decode_small = the cluster decode kernel on B=4 x 8192 tokens; decode_short = the warp-per-unit decode kernel on B=512 x 64..256 tokens; rope = rope + norm + cache update on B=2, S=8192."""
     from paper_2608_21836_b200 import binding as l4l
 
     torch.cuda.set_device(0)
@@ -636,6 +636,15 @@ def run_profile_case(case: str):
         ws = l4l.new_workspace(l4l.L4L_OP_DECODE, 4, w.Hq, w.Hkv, w.D, 8192)
         for _ in range(3):
             l4l.l4l_attn_decode(q, o, ck, cv, lens, 8192, w.scale, ws)
+    elif case == "decode_short":
+        # the warp-per-unit kernel: B = 512 sequences of 64 to 256 tokens of the 8B-shaped layer (338 MB of cache > L2)
+        w = wl.WORKLOADS["batched_decode"]
+        db = wl.make_decode_batch(w, B=512, len_lo=64, len_hi=256, Lmax=256, poison_tail=False)
+        q, ck, cv, lens = db.q.cuda(), db.cache_k.cuda(), db.cache_v.cuda(), db.kv_len.cuda()
+        o = torch.empty_like(q)
+        ws = l4l.new_workspace(l4l.L4L_OP_DECODE, 512, w.Hq, w.Hkv, w.D, 256)
+        for _ in range(3):
+            l4l.l4l_attn_decode(q, o, ck, cv, lens, 256, w.scale, ws)
     else:
         w = wl.WORKLOADS["batched_decode"]
         db = wl.make_decode_batch(w)
@@ -655,7 +664,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--profile-case", choices=["prefill", "decode", "decode_small", "rope", "rglru"], default=None,
+    ap.add_argument("--profile-case", choices=["prefill", "decode", "decode_small", "decode_short", "rope", "rglru"], default=None,
                     help="run three launches of one kernel on a small case and exit (for ncu)")
     args = ap.parse_args()
     if args.profile_case:

@@ -320,8 +320,10 @@ l4l_status l4l_attn_prefill_chunk(l4l_tensor4 q, l4l_tensor4 o, l4l_kv_cache cac
  * with no mask. n = 0 gives o = 0 and lse = -inf. Cache slots >= n are never allowed to
  * influence the result, whatever bits they hold (slots up to the end of the 256-token block that
  * holds slot n-1 may be READ, inside cache.max_len only). Small batches (every (sequence, KV head)
- * on its own thread-block cluster at once) run a kernel that merges through shared memory and
- * leaves the workspace's partials unused; the workspace is required all the same.
+ * on its own thread-block cluster at once) run a kernel that merges through shared memory, and
+ * hundreds of sequences of at most a few hundred tokens (by max_kv_len) one that gives every
+ * (sequence, KV head) to a single warp; both leave the workspace's partials unused; the
+ * workspace is required all the same.
  *   q, o         dense [B, Hq, D]
  *   d_kv_lens    device int32 [B], each 0 <= n <= max_kv_len
  *   max_kv_len   host upper bound of kv_lens (<= cache.max_len); used to size the split

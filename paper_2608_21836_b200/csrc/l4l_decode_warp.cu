@@ -1,0 +1,482 @@
+// Decode attention for MANY SHORT sequences: one warp owns a (sequence, KV head) from its first cached token to
+// the output row, so there is nothing to merge and nothing to hand over. The split kernel pays a fixed cost per
+// piece of a sequence (query rows, hand-over, finisher); with hundreds of sequences of a few hundred tokens
+// that cost is paid every tile or two and the kernel falls to a third of the HBM rate.
+//
+// Persistent CTAs of 8 warps. The (sequence, KV head) units are laid end to end in 16-token chunks; warp w of
+// all warps takes the units that START inside its equal share of that stream (whole units only: a warp's load
+// differs from the mean by at most one unit). A warp moves its chunks from the cache into a private ring in
+// shared memory with 16-byte asynchronous copies (cp.async: no barrier objects, no descriptors, rows past the
+// end of a sequence arrive as zeros), in the 128-byte-swizzled layout that the warp-level MMA blocks expect, and
+// stays S - 1 chunks ahead of its own arithmetic, across unit boundaries (the query rows of a unit travel with
+// the unit's first chunk). Contiguous or paged caches; optional fused append of the step's newest token.
+#include <cstdlib>
+#include <mutex>
+
+#include "l4l_internal.h"
+#include "l4l_ptx.cuh"
+#include "l4l_warp_attn.cuh"
+
+namespace l4l {
+
+namespace {
+
+constexpr int kMaxB = 1024;          // sequences per launch (lengths and prefix sums in shared memory)
+constexpr int kChunkT = 16;          // tokens per chunk = one MMA step of a warp
+
+struct WarpParams {
+    const __nv_bfloat16 *q;   // [B, Hq, D]
+    __nv_bfloat16 *o;         // [B, Hq, D]
+    float *lse;               // [B, Hq] or null
+    const int32_t *kv_lens;   // [B]
+    const __nv_bfloat16 *k_new, *v_new;   // fused append (null: none): element (b, kv head, d) at b*new_sb + kvh*new_sh + d
+    int64_t new_sb, new_sh;
+    __nv_bfloat16 *cache_k, *cache_v;
+    int64_t c_sb, c_sh, c_st;
+    const int32_t *block_table;           // paged cache (null: contiguous)
+    int table_stride, page_size, page_shift, num_pages;
+    int B, Hq, Hkv, G, max_kv_len, stages;
+    float scale_log2e;
+};
+
+template <int D>
+struct WarpCfg {
+    static constexpr int kHalves = D / 64;                            // 128-byte column blocks of a row
+    static constexpr uint32_t kHalfBytes = kChunkT * 128;             // [16 tokens][128 bytes], swizzled
+    static constexpr uint32_t kTileBytes = kHalves * kHalfBytes;      // K or V of one chunk
+    static constexpr int kRowPieces = D / 8;                          // 16-byte pieces per row
+    static constexpr int kCopies = kChunkT * kRowPieces / 32;         // cp.async per lane for K (and as many for V)
+};
+
+__host__ __device__ inline size_t stage_bytes(int D, int G)
+{
+    return (size_t)2 * (D / 64) * kChunkT * 128 + (size_t)G * D * 2;    // K, V, the unit's query rows
+}
+
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void *src, uint32_t src_bytes)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_16_full(uint32_t dst, const void *src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// Position of a warp in its list of units.
+struct Cursor {
+    int b, kvh, len, chunks, chunk;   // current unit, its length and chunk count, next chunk of it
+    int start;                        // the unit's first chunk in the flattened stream
+};
+
+template <int D, int kWarps>
+__global__ void __launch_bounds__(kWarps * 32) decode_warp_kernel(const WarpParams p)
+{
+    using C = WarpCfg<D>;
+    constexpr int kThreads = kWarps * 32;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    int *lens_s = reinterpret_cast<int *>(smem);                 // [kMaxB]
+    int *cum_s = lens_s + kMaxB;                                 // [kMaxB + 1] chunks of the sequences before b
+    int *warp_sums = cum_s + kMaxB + 1;                          // [kWarps] (16 at most)
+    const size_t sbytes = stage_bytes(D, p.G);
+    uint8_t *ring_base = smem + 9 * 1024;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint8_t *ring = ring_base + (size_t)warp * p.stages * sbytes;
+
+    grid_dependency_wait();
+    grid_launch_dependents();
+
+    // ---- lengths and the prefix sum of chunk counts (a sequence without tokens still owns one chunk of the
+    // stream, so that some warp writes its zero output)
+    constexpr int kPer = (kMaxB + kThreads - 1) / kThreads;
+    int mine[kPer], run = 0;
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) {
+        const int b = threadIdx.x * kPer + i;
+        int len = 0, ch = 0;
+        if (b < p.B) {
+            len = __ldg(p.kv_lens + b);
+            len = len < 0 ? 0 : (len > p.max_kv_len ? p.max_kv_len : len);
+            lens_s[b] = len;
+            ch = len > 0 ? (len + kChunkT - 1) / kChunkT : 1;
+        }
+        mine[i] = run;
+        run += ch;
+    }
+    int incl = run;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += v;
+    }
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    int before = incl - run;
+    for (int w = 0; w < warp; ++w) before += warp_sums[w];
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) {
+        const int b = threadIdx.x * kPer + i;
+        if (b <= p.B) cum_s[b] = before + mine[i];
+    }
+    if (kThreads * kPer == kMaxB && threadIdx.x == kThreads - 1 && p.B == kMaxB) cum_s[kMaxB] = before + run;
+    __syncthreads();
+
+    // ---- this warp's units: those that start inside its share [lo, hi) of the chunk stream
+    const long long total = (long long)cum_s[p.B] * p.Hkv;
+    const long long n_warps = (long long)gridDim.x * kWarps, gw = (long long)blockIdx.x * kWarps + warp;
+    const int lo = (int)(gw * total / n_warps), hi = (int)((gw + 1) * total / n_warps);
+    Cursor first;
+    {
+        int a = 0, z = p.B;                       // smallest b with Hkv * cum[b + 1] > lo
+        while (a < z) {
+            const int mid = (a + z) >> 1;
+            if ((long long)cum_s[mid + 1] * p.Hkv > lo) z = mid; else a = mid + 1;
+        }
+        first.b = a;
+        first.kvh = 0;
+        first.len = first.chunks = first.chunk = first.start = 0;
+        if (a < p.B) {
+            const int cb = cum_s[a + 1] - cum_s[a], base = cum_s[a] * p.Hkv;
+            int kvh = (lo - base + cb - 1) / cb;  // first unit of the sequence that starts at or after lo
+            if (kvh >= p.Hkv) {
+                first.b = a + 1;
+                kvh = 0;
+            }
+            first.kvh = kvh;
+            if (first.b < p.B) {
+                first.len = lens_s[first.b];
+                first.chunks = cum_s[first.b + 1] - cum_s[first.b];
+                first.start = cum_s[first.b] * p.Hkv + kvh * first.chunks;
+            }
+        }
+    }
+    auto live = [&](const Cursor &c) { return c.b < p.B && c.start < hi; };
+    auto advance = [&](Cursor &c) {               // to the next chunk, or the first chunk of the next unit
+        if (++c.chunk < c.chunks) return;
+        c.chunk = 0;
+        c.start += c.chunks;
+        if (++c.kvh == p.Hkv) {
+            c.kvh = 0;
+            if (++c.b < p.B) {
+                c.len = lens_s[c.b];
+                c.chunks = cum_s[c.b + 1] - cum_s[c.b];
+            }
+        }
+    };
+
+    // per-lane constants of the copies: piece i of a lane is row (32 i + lane) / kRowPieces, 16-byte piece
+    // (32 i + lane) % kRowPieces of the row
+    const int piece = lane % C::kRowPieces, row_of_lane = lane / C::kRowPieces;
+    constexpr int kRowsPerTrip = 32 / C::kRowPieces;
+    const uint32_t dst_half = (uint32_t)(piece >> 3) * C::kHalfBytes;
+
+    uint32_t soff[C::kCopies];                     // where this lane's pieces land inside a K (or V) tile
+#pragma unroll
+    for (int i = 0; i < C::kCopies; ++i) soff[i] = dst_half + swz128(i * kRowsPerTrip + row_of_lane, piece & 7);
+
+    auto issue = [&](const Cursor &c, int slot) {
+        uint8_t *st = ring + (size_t)slot * sbytes;
+        const uint32_t k_dst = smem_u32(st), v_dst = k_dst + C::kTileBytes;
+        const int t0 = c.chunk * kChunkT;
+        long long outer = c.b, slot_t = t0;
+        bool have = true;
+        if (p.block_table != nullptr) {
+            outer = __ldg(p.block_table + (size_t)c.b * p.table_stride + (t0 >> p.page_shift));
+            slot_t = t0 & (p.page_size - 1);
+            have = outer >= 0 && outer < p.num_pages;     // a page outside the pool reads as zeros
+            if (!have) outer = 0;
+        }
+        const size_t base = (size_t)outer * p.c_sb + (size_t)c.kvh * p.c_sh +
+                            (size_t)(slot_t + row_of_lane) * p.c_st + piece * 8;
+        const __nv_bfloat16 *ks = p.cache_k + base, *vs = p.cache_v + base;
+        const size_t step = (size_t)kRowsPerTrip * p.c_st;
+        const int nval = c.len - t0;               // rows of the chunk that hold tokens
+        if (have && (nval > kChunkT || (nval == kChunkT && p.k_new == nullptr))) {
+            // a full chunk of cached tokens (all but the last chunk of a unit): no predicates
+#pragma unroll
+            for (int i = 0; i < C::kCopies; ++i) {
+                cp_async_16_full(k_dst + soff[i], ks);
+                cp_async_16_full(v_dst + soff[i], vs);
+                ks += step;
+                vs += step;
+            }
+        } else {
+            const int newest = (p.k_new != nullptr) ? nval - 1 : -1;        // row of the chunk that the caller brings
+            const size_t new_off = (size_t)c.b * p.new_sb + (size_t)c.kvh * p.new_sh + piece * 8;
+#pragma unroll
+            for (int i = 0; i < C::kCopies; ++i) {
+                const int row = i * kRowsPerTrip + row_of_lane;
+                const bool valid = have && row < nval;
+                if (row == newest) {
+                    cp_async_16(k_dst + soff[i], p.k_new + new_off, 16u);
+                    cp_async_16(v_dst + soff[i], p.v_new + new_off, 16u);
+                } else {
+                    cp_async_16(k_dst + soff[i], valid ? ks : p.cache_k, valid ? 16u : 0u);
+                    cp_async_16(v_dst + soff[i], valid ? vs : p.cache_v, valid ? 16u : 0u);
+                }
+                ks += step;
+                vs += step;
+            }
+        }
+        if (c.chunk == 0) {                        // the unit's query rows: G x D bf16, unswizzled
+            const uint32_t q_dst = v_dst + C::kTileBytes;
+            const __nv_bfloat16 *qs = p.q + ((size_t)c.b * p.Hq + (size_t)c.kvh * p.G) * D;
+            for (int i = lane; i < p.G * C::kRowPieces; i += 32) cp_async_16_full(q_dst + i * 16, qs + i * 8);
+        }
+    };
+
+    // ---- prologue: S - 1 chunks in flight
+    Cursor head = first, tail = first;            // head: next chunk to fetch; tail: next chunk to compute
+    const int S = p.stages;
+    int head_slot = 0, tail_slot = 0;
+    for (int i = 0; i < S - 1; ++i) {
+        if (live(head)) {
+            issue(head, head_slot);
+            advance(head);
+        }
+        cp_async_commit();
+        head_slot = head_slot + 1 == S ? 0 : head_slot + 1;
+    }
+
+    WarpAttnState<D> st;
+    st.reset();
+    uint32_t qf[D / 16][4];
+    const int r_lo = lane >> 2, r_hi = r_lo + 8;
+    while (live(tail)) {
+        if (live(head)) {
+            issue(head, head_slot);
+            advance(head);
+        }
+        cp_async_commit();
+        head_slot = head_slot + 1 == S ? 0 : head_slot + 1;
+        switch (S) {                               // all but the newest S - 1 groups have landed
+        case 2: cp_async_wait<1>(); break;
+        case 3: cp_async_wait<2>(); break;
+        case 4: cp_async_wait<3>(); break;
+        case 5: cp_async_wait<4>(); break;
+        default: cp_async_wait<5>(); break;
+        }
+        __syncwarp();
+
+        uint8_t *stg = ring + (size_t)tail_slot * sbytes;
+        const uint32_t k_tile = smem_u32(stg), v_tile = k_tile + C::kTileBytes;
+        if (tail.chunk == 0) {
+            const uint32_t *qs = reinterpret_cast<const uint32_t *>(stg + 2 * C::kTileBytes);
+            const uint32_t *qrow_lo = qs + (size_t)r_lo * D / 2;
+            const uint32_t *qrow_hi = qs + (size_t)r_hi * D / 2;
+            const bool v_lo = r_lo < p.G, v_hi = r_hi < p.G;
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks) {
+                const int w = ks * 8 + (lane & 3);
+                qf[ks][0] = v_lo ? qrow_lo[w] : 0u;
+                qf[ks][1] = v_hi ? qrow_hi[w] : 0u;
+                qf[ks][2] = v_lo ? qrow_lo[w + 4] : 0u;
+                qf[ks][3] = v_hi ? qrow_hi[w + 4] : 0u;
+            }
+        }
+        const int t0 = tail.chunk * kChunkT;
+        const int nvalid = tail.len - t0;
+        if (nvalid > 0) {
+            if (p.k_new != nullptr && nvalid <= kChunkT) {
+                // fused append: the newest token came from the caller; its cache slot is written from the copy in
+                // shared memory (with pages: behind the block table; no page there: nothing is written)
+                const int row = nvalid - 1;
+                long long outer = tail.b, slot_t = tail.len - 1;
+                if (p.block_table != nullptr) {
+                    outer = __ldg(p.block_table + (size_t)tail.b * p.table_stride + (slot_t >> p.page_shift));
+                    slot_t &= p.page_size - 1;
+                }
+                const bool have = p.block_table == nullptr || (outer >= 0 && outer < p.num_pages);
+                if (lane < C::kRowPieces) {
+                    const uint32_t off = (uint32_t)(lane >> 3) * C::kHalfBytes + swz128(row, lane & 7);
+                    if (have) {
+                        const size_t dst = (size_t)outer * p.c_sb + (size_t)tail.kvh * p.c_sh + (size_t)slot_t * p.c_st + lane * 8;
+                        *reinterpret_cast<uint4 *>(p.cache_k + dst) = *reinterpret_cast<const uint4 *>(stg + off);
+                        *reinterpret_cast<uint4 *>(p.cache_v + dst) = *reinterpret_cast<const uint4 *>(stg + C::kTileBytes + off);
+                    } else {                       // as the cache would read: zeros
+                        *reinterpret_cast<uint4 *>(stg + off) = make_uint4(0u, 0u, 0u, 0u);
+                        *reinterpret_cast<uint4 *>(stg + C::kTileBytes + off) = make_uint4(0u, 0u, 0u, 0u);
+                    }
+                }
+                __syncwarp();
+            }
+            float s_lo[4], s_hi[4];
+            warp_qk_16x16<D>(qf, k_tile, C::kHalfBytes, 0, s_lo, s_hi);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                s_lo[e] *= p.scale_log2e;
+                s_hi[e] *= p.scale_log2e;
+            }
+            if (nvalid < kChunkT) {                // tokens past the end: no weight (their V rows arrived as zeros)
+                const int tok = 2 * (lane & 3);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    if (tok + (e & 1) >= nvalid) s_lo[e] = -INFINITY;
+                    if (tok + (e & 1) + 8 >= nvalid) s_hi[e] = -INFINITY;
+                }
+            }
+            uint32_t pa[4];
+            warp_softmax_16<D>(st, s_lo, s_hi, pa);
+            warp_pv_16x16<D>(st, pa, v_tile, C::kHalfBytes, 0);
+        }
+        if (tail.chunk + 1 == tail.chunks) {
+            // ---- the unit is complete: normalise and write its G output rows
+            float l0 = st.l[0], l1 = st.l[1];
+            l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+            l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+            l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+            l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+            const bool any = tail.len > 0;
+            const float i0 = any ? 1.f / l0 : 0.f, i1 = any ? 1.f / l1 : 0.f;
+            const size_t bh = (size_t)tail.b * p.Hq + (size_t)tail.kvh * p.G;
+            if (r_lo < p.G) {
+                __nv_bfloat16 *row = p.o + (bh + r_lo) * D + 2 * (lane & 3);
+#pragma unroll
+                for (int nt = 0; nt < D / 8; ++nt)
+                    *reinterpret_cast<uint32_t *>(row + nt * 8) = pack_bf16x2(st.o[nt][0] * i0, st.o[nt][1] * i0);
+                if ((lane & 3) == 0 && p.lse)
+                    p.lse[bh + r_lo] = any ? (st.m[0] + log2f(l0)) * 0.6931471805599453f : -INFINITY;
+            }
+            if (r_hi < p.G) {
+                __nv_bfloat16 *row = p.o + (bh + r_hi) * D + 2 * (lane & 3);
+#pragma unroll
+                for (int nt = 0; nt < D / 8; ++nt)
+                    *reinterpret_cast<uint32_t *>(row + nt * 8) = pack_bf16x2(st.o[nt][2] * i1, st.o[nt][3] * i1);
+                if ((lane & 3) == 0 && p.lse)
+                    p.lse[bh + r_hi] = any ? (st.m[1] + log2f(l1)) * 0.6931471805599453f : -INFINITY;
+            }
+            st.reset();
+        }
+        __syncwarp();                              // every lane is done with the slot before it is filled again
+        tail_slot = tail_slot + 1 == S ? 0 : tail_slot + 1;
+        advance(tail);
+    }
+    cp_async_wait<0>();
+}
+
+size_t warp_smem_bytes(int D, int G, int warps, int stages) { return 9 * 1024 + (size_t)warps * stages * stage_bytes(D, G); }
+
+template <int D, int W>
+int blocks_per_sm(size_t smem)
+{
+    struct Entry { size_t smem; int n; };
+    static Entry cache[8];
+    static int n_cached = 0;
+    static std::mutex mutex;
+    std::lock_guard<std::mutex> lock(mutex);
+    for (int i = 0; i < n_cached; ++i)
+        if (cache[i].smem == smem) return cache[i].n;
+    int n = 0;
+    if (cudaFuncSetAttribute(decode_warp_kernel<D, W>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_warp_kernel<D, W>, W * 32, smem) != cudaSuccess) {
+        (void)cudaGetLastError();
+        n = 0;
+    }
+    if (n_cached < 8) cache[n_cached++] = {smem, n};
+    return n;
+}
+
+// Warps per CTA and ring depth. The arithmetic of a warp is one dependent chain per chunk, so the SM wants as many
+// warps as its shared memory can give a ring of at least two chunks: 12 at head_dim 128 (groups of up to 4 query
+// heads; 8 above), 8 in each of two CTAs at head_dim 64.
+struct WarpShape { int warps, stages; };
+WarpShape pick_warp_shape(int D, int G)
+{
+    int warps = (D == 128 && G <= 4) ? 12 : 8;
+    if (const char *e = getenv("L4L_DECODE_WARP_WARPS")) {
+        const int w = atoi(e);
+        if (D == 128 && (w == 8 || w == 12)) warps = w;
+    }
+    const size_t limit = (D == 64 ? 113u : 227u) * 1024u;
+    for (int s = 5; s >= 2; --s)
+        if (warp_smem_bytes(D, G, warps, s) <= limit) return {warps, s};
+    return {warps, 0};
+}
+
+}  // namespace
+
+// Whether the warp-per-unit kernel should serve this decode call. L4L_DECODE_WARP=0 / 1 forces the answer (for
+// tests); shapes it cannot run are refused either way.
+bool decode_warp_eligible(int B, int Hq, int Hkv, int D, int max_kv_len, bool fp8, bool rope)
+{
+    const int G = Hq / Hkv;
+    if (fp8 || rope || G > 8 || pick_warp_shape(D, G).stages == 0) return false;
+    if (const char *e = getenv("L4L_DECODE_WARP")) return e[0] != '0';
+    // many units of a few chunks each: the regime where the split kernel pays its per-piece cost every tile or two.
+    // Thresholds measured against the split kernel (8 KV heads at head_dim 128, 12 at head_dim 64): with at most 256
+    // tokens per sequence it wins from about half a unit per resident warp, with at most 512 from about two.
+    const long long units = (long long)B * Hkv;
+    const long long slots = (long long)sm_count() * (D == 64 ? 16 : pick_warp_shape(D, G).warps);
+    if (max_kv_len <= 256) return units * 16 >= slots * 9;
+    if (max_kv_len <= 512) return units * 10 >= slots * 22;
+    return false;
+}
+
+l4l_status launch_decode_warp(const void *q, void *o, const l4l_kv_cache &cache, const int32_t *d_kv_lens,
+                              int max_kv_len, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
+                              cudaStream_t stream, const l4l_tensor4 *k_new, const l4l_tensor4 *v_new,
+                              const PagedTable *paged)
+{
+    const int G = Hq / Hkv;
+    const WarpShape shape = pick_warp_shape(D, G);
+    const int stages = shape.stages, kWarps = shape.warps;
+    if (stages == 0 || G > 8 || (k_new == nullptr) != (v_new == nullptr)) return L4L_ERR_UNSUPPORTED;
+    const size_t smem = warp_smem_bytes(D, G, kWarps, stages);
+    const int per_sm = D == 64 ? blocks_per_sm<64, 8>(smem)
+                               : (kWarps == 12 ? blocks_per_sm<128, 12>(smem) : blocks_per_sm<128, 8>(smem));
+    if (per_sm == 0) return L4L_ERR_CUDA;
+    for (int b0 = 0; b0 < B; b0 += kMaxB) {
+        const int nb = B - b0 < kMaxB ? B - b0 : kMaxB;
+        WarpParams p = {};
+        p.q = static_cast<const __nv_bfloat16 *>(q) + (size_t)b0 * Hq * D;
+        p.o = static_cast<__nv_bfloat16 *>(o) + (size_t)b0 * Hq * D;
+        p.lse = d_lse ? d_lse + (size_t)b0 * Hq : nullptr;
+        p.kv_lens = d_kv_lens + b0;
+        if (k_new) {
+            p.k_new = static_cast<const __nv_bfloat16 *>(k_new->ptr) + (size_t)b0 * k_new->stride_b;
+            p.v_new = static_cast<const __nv_bfloat16 *>(v_new->ptr) + (size_t)b0 * v_new->stride_b;
+            if (k_new->stride_b != v_new->stride_b || k_new->stride_h != v_new->stride_h) return L4L_ERR_UNSUPPORTED;
+            p.new_sb = k_new->stride_b;
+            p.new_sh = k_new->stride_h;
+        }
+        // paged: the pool as a whole, whatever the slice; contiguous: this slice's sequences
+        p.cache_k = static_cast<__nv_bfloat16 *>(cache.k) + (paged ? 0 : (size_t)b0 * cache.stride_b);
+        p.cache_v = static_cast<__nv_bfloat16 *>(cache.v) + (paged ? 0 : (size_t)b0 * cache.stride_b);
+        p.c_sb = cache.stride_b; p.c_sh = cache.stride_h; p.c_st = cache.stride_t;
+        p.block_table = paged ? paged->block_table + (size_t)b0 * paged->table_stride : nullptr;
+        p.table_stride = paged ? paged->table_stride : 0;
+        p.page_size = paged ? cache.max_len : 0;
+        p.num_pages = paged ? paged->num_pages : 0;
+        p.page_shift = 0;
+        while (paged && (1 << p.page_shift) < cache.max_len) ++p.page_shift;
+        p.B = nb; p.Hq = Hq; p.Hkv = Hkv; p.G = G; p.max_kv_len = max_kv_len; p.stages = stages;
+        p.scale_log2e = scale * 1.4426950408889634f;
+
+        // persistent: every resident warp gets its share; never more warps than units
+        long long blocks = (long long)per_sm * sm_count();
+        const long long units = (long long)nb * Hkv;
+        if (blocks * kWarps > units) blocks = (units + kWarps - 1) / kWarps;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)blocks, 1, 1);
+        cfg.blockDim = dim3(kWarps * 32, 1, 1);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        const cudaError_t err = D == 64 ? cudaLaunchKernelEx(&cfg, decode_warp_kernel<64, 8>, p)
+                                : (kWarps == 12 ? cudaLaunchKernelEx(&cfg, decode_warp_kernel<128, 12>, p)
+                                                : cudaLaunchKernelEx(&cfg, decode_warp_kernel<128, 8>, p));
+        if (err != cudaSuccess) {
+            (void)cudaGetLastError();
+            return L4L_ERR_CUDA;
+        }
+    }
+    return L4L_OK;
+}
+
+}  // namespace l4l

@@ -1,0 +1,124 @@
+"""The decode kernel for many short sequences (one warp per (sequence, KV head), no merge) against the fp64 oracle,
+forced on through L4L_DECODE_WARP for small shapes, and chosen by the library for the regime it is made for."""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import l4l_oracle as orc
+from paper_2608_21836_b200 import binding as l4l
+from helpers import Guarded, assert_close_to_oracle, bits_equal, nan_bf16
+from test_gpu_decode import check_decode, random_batch
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture
+def warp_kernel(request):
+    """'1': every eligible decode call runs on the warp kernel; '0': never; None: the library's choice."""
+    mode = getattr(request, "param", "1")
+    old = os.environ.get("L4L_DECODE_WARP")
+    if mode is None:
+        os.environ.pop("L4L_DECODE_WARP", None)
+    else:
+        os.environ["L4L_DECODE_WARP"] = mode
+    yield mode
+    if old is None:
+        os.environ.pop("L4L_DECODE_WARP", None)
+    else:
+        os.environ["L4L_DECODE_WARP"] = old
+
+
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("Hq,Hkv", [(8, 2), (8, 8), (8, 1), (3, 1), (6, 2), (32, 8)])
+def test_warp_decode_ragged_edge_lengths(warp_kernel, D, Hq, Hkv):
+    # around every boundary: empty, one token, 16-token chunks, more chunks than ring stages
+    lens = [0, 1, 2, 15, 16, 17, 31, 32, 33, 47, 48, 127, 128, 129, 255, 300, 0, 7]
+    q, ck, cv, kv_len = random_batch(len(lens), Hq, Hkv, D, 304, lens, seed=1900 + D + Hq)
+    check_decode(q, ck, cv, kv_len, 1.0 / math.sqrt(D))
+
+
+@pytest.mark.parametrize("B", [1, 7, 200, 1024, 1500])
+def test_warp_decode_batch_sizes(warp_kernel, B):
+    # fewer units than warps, one full launch slice, more than one slice
+    g = np.random.default_rng(B)
+    lens = g.integers(0, 200, size=B).tolist()
+    q, ck, cv, kv_len = random_batch(B, 8, 2, 128, 208, lens, seed=B)
+    check_decode(q, ck, cv, kv_len, 1.0 / math.sqrt(128))
+
+
+def test_warp_decode_long_sequences_too(warp_kernel):
+    # not its regime, but correct there as well: hundreds of chunks per unit
+    lens = [4000, 2500, 1, 4096]
+    q, ck, cv, kv_len = random_batch(4, 8, 2, 128, 4096, lens, seed=3)
+    check_decode(q, ck, cv, kv_len, 1.0 / math.sqrt(128))
+
+
+def test_warp_decode_extreme_scores_token_major_cache_and_clamp(warp_kernel):
+    lens = [300, 1, 129, 64]
+    q, ck, cv, kv_len = random_batch(4, 8, 2, 128, 384, lens, seed=77)
+    check_decode(q, ck, cv, kv_len, 1.0)
+    check_decode(q, ck, cv, kv_len, -0.25)
+    check_decode(q, ck, cv, kv_len, 1.0 / math.sqrt(128), strided_cache=True)
+    B, Hq, D = q.shape
+    clamp = 100                                   # kv_lens above max_kv_len are clamped to it
+    ref, _ = orc.decode(q, ck, cv, np.minimum(kv_len.numpy(), clamp), 0.1)
+    o = torch.zeros(B, Hq, D, dtype=torch.bfloat16, device="cuda")
+    ws = l4l.new_workspace(l4l.L4L_OP_DECODE, B, Hq, 2, D, clamp)
+    l4l.l4l_attn_decode(q.cuda(), o, ck.cuda(), cv.cuda(), kv_len.cuda(), clamp, 0.1, ws)
+    torch.cuda.synchronize()
+    assert_close_to_oracle(o, ref, "clamped decode")
+
+
+@pytest.mark.parametrize("D,Hq,Hkv", [(128, 8, 2), (64, 4, 4), (128, 8, 1), (128, 32, 8)])
+def test_warp_decode_with_fused_append(warp_kernel, D, Hq, Hkv):
+    from test_gpu_decode_append import make_case
+
+    lens = [0, 1, 2, 16, 17, 32, 33, 128, 129, 300, 255, 256]
+    B, Lmax = len(lens), 304
+    q, ck, cv, kn, vn, kv_len = make_case(B, Hq, Hkv, D, Lmax, lens, seed=140 + D + Hq)
+    scale = 1.0 / math.sqrt(D)
+    pos = (kv_len - 1).clamp(min=0).numpy()
+    n_new = (kv_len > 0).to(torch.int32).numpy()
+    ek, ev = orc.kv_append(ck, cv, kn, vn, pos, n_new)
+    ek_t = torch.from_numpy(ek.view(np.int16)).view(torch.bfloat16)
+    ev_t = torch.from_numpy(ev.view(np.int16)).view(torch.bfloat16)
+    ref, ref_lse = orc.decode(q, ek_t, ev_t, kv_len.numpy(), scale)
+    gk, gv, go = Guarded(ck), Guarded(cv), Guarded(nan_bf16((B, Hq, D)))
+    lse = torch.zeros(B, Hq, device="cuda")
+    ws = l4l.new_workspace(l4l.L4L_OP_DECODE, B, Hq, Hkv, D, Lmax)
+    l4l.l4l_attn_decode_append(q.cuda(), go.t, gk.t, gv.t, kn.cuda(), vn.cuda(), kv_len.cuda(), Lmax, scale, ws, lse=lse)
+    torch.cuda.synchronize()
+    assert l4l.l4l_last_device_error(ws) == 0
+    for g in (gk, gv, go):
+        assert g.margins_intact()
+    assert bits_equal(gk.t, ek) and bits_equal(gv.t, ev)
+    assert_close_to_oracle(go.t, ref, "warp decode_append o")
+    fin = np.isfinite(ref_lse)
+    assert np.abs(lse.cpu().double().numpy()[fin] - ref_lse[fin]).max() <= 2e-3
+    assert (lse.cpu().numpy()[~fin] == -np.inf).all()
+
+
+@pytest.mark.parametrize("page", [16, 64, 256])
+@pytest.mark.parametrize("Hq,Hkv,D", [(32, 8, 128), (12, 12, 64)])
+def test_warp_decode_paged_with_and_without_append(warp_kernel, page, Hq, Hkv, D):
+    from test_gpu_paged import test_paged_decode_matches_oracle
+    from test_gpu_paged_append import run_case
+
+    test_paged_decode_matches_oracle(page, Hq, Hkv, D)
+    lens = [1, 16, 17, 128, 129, 257, 300, 33, 0, 64]
+    run_case(len(lens), Hq, Hkv, D, page, lens, seed=2200 + page + D)
+    run_case(len(lens), Hq, Hkv, D, page, lens, seed=2300 + page + D, drop=(1, 4, 6))
+
+
+@pytest.mark.parametrize("warp_kernel", [None, "0"], indirect=True)
+def test_library_picks_the_warp_kernel_for_many_short_sequences(warp_kernel):
+    """B = 400 sequences of 1 to 256 tokens on 8 KV heads is inside the regime the library hands to the warp kernel;
+    the same call kept off it must agree within the tolerance of both."""
+    B, Hq, Hkv, D = 400, 32, 8, 128
+    g = np.random.default_rng(11)
+    lens = g.integers(1, 257, size=B).tolist()
+    q, ck, cv, kv_len = random_batch(B, Hq, Hkv, D, 256, lens, seed=12)
+    check_decode(q, ck, cv, kv_len, 1.0 / math.sqrt(D))
