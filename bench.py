@@ -432,6 +432,33 @@ def run_ours(args, rank, world):
         err = l4l.l4l_last_device_error(sws)
         return a0.elapsed_time(a1) / (5 * n) * 1e3, err
 
+    # hundreds of short sequences (B = 512 with 64 to 256 cached tokens, 338 MB > L2, three copies in rotation): the
+    # library's choice (a warp per (sequence, KV head)) and the same call held on the split kernel
+    def short_batch_us(split_only):
+        sb = wl.make_decode_batch(wd, B=512, len_lo=64, len_hi=256, Lmax=256, poison_tail=False)
+        nbytes = wl.decode_kv_bytes(wd.Hkv, wd.D, sb.kv_len.tolist())
+        cp = [(sb.cache_k.to(dev), sb.cache_v.to(dev)) for _ in range(3)]
+        sq, slen = sb.q.to(dev), sb.kv_len.to(dev)
+        so = torch.empty_like(sq)
+        sws = l4l.new_workspace(l4l.L4L_OP_DECODE, 512, wd.Hq, wd.Hkv, wd.D, 256, device=dev)
+        old = os.environ.get("L4L_DECODE_WARP")
+        if split_only:
+            os.environ["L4L_DECODE_WARP"] = "0"
+        try:
+            def step():
+                ck_i, cv_i = cp[rot[0] % 3]
+                rot[0] += 1
+                l4l.l4l_attn_decode(sq, so, ck_i, cv_i, slen, 256, wd.scale, sws)
+            t = timed(step, 21)
+        finally:
+            if old is None:
+                os.environ.pop("L4L_DECODE_WARP", None)
+            else:
+                os.environ["L4L_DECODE_WARP"] = old
+        return t, nbytes, l4l.l4l_last_device_error(sws)
+
+    t_short, short_bytes, err_short = short_batch_us(False)
+    t_short_split, _, err_short2 = short_batch_us(True)
     t_small, err_small = small_batch_step_us(2304, False)
     t_small_split, err_small2 = small_batch_step_us(2304, True)
     # second workload: the RG-LRU recurrence of a RecurrentGemma-2B-sized block (2560 channels) over a long prompt
@@ -456,7 +483,7 @@ def run_ours(args, rank, world):
     t_rglru2 = timed(lambda: l4l.l4l_rglru_scan(v2(rx), v2(rgx), v2(rga), r_ap, r_state2, v2(ry), ws_r2), 10)
     dev_err_r |= l4l.l4l_last_device_error(ws_r2)
     del rx, rgx, rga, ry, filler
-    dev_err = l4l.l4l_last_device_error(ws_p) | l4l.l4l_last_device_error(ws_d) | dev_err_r | err_small | err_small2 | err_g8
+    dev_err = l4l.l4l_last_device_error(ws_p) | l4l.l4l_last_device_error(ws_d) | dev_err_r | err_small | err_small2 | err_g8 | err_short | err_short2
 
     # ---- end to end through the same entry points with HOST buffers (pinned), copies inside the timed region
     hq, hk, hv = seq.q.pin_memory(), seq.k.pin_memory(), seq.v.pin_memory()
@@ -570,6 +597,8 @@ def run_ours(args, rank, world):
             "decode_fp8_cache": {"us": t_fp8 * 1e3, "kv_gbs_fp8_bytes": dec_bytes / 2 / (t_fp8 * 1e-3) / 1e9,
                                  "speedup_over_bf16_cache": t_dec_b2b / t_fp8},
             "decode_64_query_heads_on_8_kv_heads": {"us": t_g8 * 1e3, "kv_gbs": dec_bytes / (t_g8 * 1e-3) / 1e9},
+            "decode_B512_L64_to_256": {"warp_kernel_us": t_short * 1e3, "kv_gbs": short_bytes / (t_short * 1e-3) / 1e9,
+                                       "split_kernel_us": t_short_split * 1e3},
             "decode_step_B1_L2304_in_cuda_graph": {"cluster_kernel_us": t_small, "split_kernel_us": t_small_split},
         },
         "gpu_launches": 3 * args.steps,

@@ -3,9 +3,10 @@
 // piece of a sequence (query rows, hand-over, finisher); with hundreds of sequences of a few hundred tokens
 // that cost is paid every tile or two and the kernel falls to a third of the HBM rate.
 //
-// Persistent CTAs of 8 warps. The (sequence, KV head) units are laid end to end in 16-token chunks; warp w of
-// all warps takes the units that START inside its equal share of that stream (whole units only: a warp's load
-// differs from the mean by at most one unit). A warp moves its chunks from the cache into a private ring in
+// Persistent CTAs of 8 or 12 warps. The (sequence, KV head) units are laid end to end in 16-token chunks; a CTA
+// takes the units that START inside its equal share of that stream (whole units only), puts them in order of
+// descending length and hands them to its warps through a counter in shared memory, longest first, so that the
+// warps of a CTA finish together. A warp moves its chunks from the cache into a private ring in
 // shared memory with 16-byte asynchronous copies (cp.async: no barrier objects, no descriptors, rows past the
 // end of a sequence arrive as zeros), in the 128-byte-swizzled layout that the warp-level MMA blocks expect, and
 // stays S - 1 chunks ahead of its own arithmetic, across unit boundaries (the query rows of a unit travel with
@@ -22,6 +23,9 @@ namespace l4l {
 namespace {
 
 constexpr int kMaxB = 1024;          // sequences per launch (lengths and prefix sums in shared memory)
+constexpr int kMetaBytes = 11 * 1024; // lengths, prefix sums, unit order, queue: ahead of the rings
+constexpr int kMaxList = 512;        // units of a CTA that can be put in order
+constexpr int kFifo = 8;             // units the fetch side of a warp can be ahead of its compute side (power of two)
 constexpr int kChunkT = 16;          // tokens per chunk = one MMA step of a warp
 
 struct WarpParams {
@@ -68,7 +72,7 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 // Position of a warp in its list of units.
 struct Cursor {
     int b, kvh, len, chunks, chunk;   // current unit, its length and chunk count, next chunk of it
-    int start;                        // the unit's first chunk in the flattened stream
+    bool valid;                       // false: the queue is empty
 };
 
 template <int D, int kWarps>
@@ -80,8 +84,12 @@ __global__ void __launch_bounds__(kWarps * 32) decode_warp_kernel(const WarpPara
     int *lens_s = reinterpret_cast<int *>(smem);                 // [kMaxB]
     int *cum_s = lens_s + kMaxB;                                 // [kMaxB + 1] chunks of the sequences before b
     int *warp_sums = cum_s + kMaxB + 1;                          // [kWarps] (16 at most)
+    int *ctl = warp_sums + 16;                                   // first unit, end unit, queue position
+    int *fifo_s = ctl + 4;                                       // [kWarps][kFifo]
+    uint16_t *cnt_s = reinterpret_cast<uint16_t *>(fifo_s + 16 * kFifo);   // [kMaxList] chunks per unit of this CTA
+    uint16_t *order_s = cnt_s + kMaxList;                        // [kMaxList] units by descending chunk count
     const size_t sbytes = stage_bytes(D, p.G);
-    uint8_t *ring_base = smem + 9 * 1024;
+    uint8_t *ring_base = smem + kMetaBytes;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     uint8_t *ring = ring_base + (size_t)warp * p.stages * sbytes;
 
@@ -123,48 +131,83 @@ __global__ void __launch_bounds__(kWarps * 32) decode_warp_kernel(const WarpPara
     if (kThreads * kPer == kMaxB && threadIdx.x == kThreads - 1 && p.B == kMaxB) cum_s[kMaxB] = before + run;
     __syncthreads();
 
-    // ---- this warp's units: those that start inside its share [lo, hi) of the chunk stream
+    // ---- this CTA's units: those that start inside its equal share [lo, hi) of the chunk stream. Unit u is
+    // (sequence u / Hkv, KV head u % Hkv); units are ordered by their start, and every unit has at least one chunk.
     const long long total = (long long)cum_s[p.B] * p.Hkv;
-    const long long n_warps = (long long)gridDim.x * kWarps, gw = (long long)blockIdx.x * kWarps + warp;
-    const int lo = (int)(gw * total / n_warps), hi = (int)((gw + 1) * total / n_warps);
-    Cursor first;
-    {
-        int a = 0, z = p.B;                       // smallest b with Hkv * cum[b + 1] > lo
+    auto first_unit_at = [&](long long pos) -> int {          // first unit that starts at or after pos
+        if (pos >= total) return p.B * p.Hkv;
+        int a = 0, z = p.B;                                   // smallest b with Hkv * cum[b + 1] > pos
         while (a < z) {
             const int mid = (a + z) >> 1;
-            if ((long long)cum_s[mid + 1] * p.Hkv > lo) z = mid; else a = mid + 1;
+            if ((long long)cum_s[mid + 1] * p.Hkv > pos) z = mid; else a = mid + 1;
         }
-        first.b = a;
-        first.kvh = 0;
-        first.len = first.chunks = first.chunk = first.start = 0;
-        if (a < p.B) {
-            const int cb = cum_s[a + 1] - cum_s[a], base = cum_s[a] * p.Hkv;
-            int kvh = (lo - base + cb - 1) / cb;  // first unit of the sequence that starts at or after lo
-            if (kvh >= p.Hkv) {
-                first.b = a + 1;
-                kvh = 0;
-            }
-            first.kvh = kvh;
-            if (first.b < p.B) {
-                first.len = lens_s[first.b];
-                first.chunks = cum_s[first.b + 1] - cum_s[first.b];
-                first.start = cum_s[first.b] * p.Hkv + kvh * first.chunks;
-            }
-        }
-    }
-    auto live = [&](const Cursor &c) { return c.b < p.B && c.start < hi; };
-    auto advance = [&](Cursor &c) {               // to the next chunk, or the first chunk of the next unit
-        if (++c.chunk < c.chunks) return;
-        c.chunk = 0;
-        c.start += c.chunks;
-        if (++c.kvh == p.Hkv) {
-            c.kvh = 0;
-            if (++c.b < p.B) {
-                c.len = lens_s[c.b];
-                c.chunks = cum_s[c.b + 1] - cum_s[c.b];
-            }
-        }
+        const int cb = cum_s[a + 1] - cum_s[a];
+        const long long base = (long long)cum_s[a] * p.Hkv;
+        return a * p.Hkv + (int)((pos - base + cb - 1) / cb);  // KV head Hkv of sequence a = head 0 of a + 1
     };
+    if (threadIdx.x < 2) {
+        const long long pos = ((long long)blockIdx.x + threadIdx.x) * total / gridDim.x;
+        ctl[threadIdx.x] = first_unit_at(pos);
+    }
+    if (threadIdx.x == 2) ctl[2] = kWarps;                    // queue position of the next unit to hand out
+    __syncthreads();
+    const int u_first = ctl[0], n_units = ctl[1] - ctl[0];
+
+    // The units are handed to the warps longest first (every warp takes the next one when it has fetched its
+    // current one to the end), which evens out the finishing times of the warps: order_s = the CTA's units by
+    // descending chunk count (rank sort; a CTA has a few dozen units). Lists too long for the array keep their order.
+    const bool sorted = n_units <= kMaxList;
+    if (sorted) {
+        for (int j = threadIdx.x; j < n_units; j += kThreads) {
+            const int b = (u_first + j) / p.Hkv;
+            cnt_s[j] = (uint16_t)min(cum_s[b + 1] - cum_s[b], 65535);
+        }
+        __syncthreads();
+        for (int j = threadIdx.x; j < n_units; j += kThreads) {
+            const int mine_c = cnt_s[j];
+            int rank = 0;
+            for (int k = 0; k < n_units; ++k) {
+                const int c = cnt_s[k];
+                rank += (c > mine_c || (c == mine_c && k < j)) ? 1 : 0;
+            }
+            order_s[rank] = (uint16_t)j;
+        }
+        __syncthreads();
+    }
+    int *fifo = fifo_s + warp * kFifo;            // queue positions that the fetch side took, for the compute side
+    int fifo_wr = 0, fifo_rd = 0;
+    auto load_unit = [&](Cursor &c, int pos) {    // the unit at queue position pos (pos >= n_units: none)
+        c.chunk = 0;
+        c.valid = pos < n_units;
+        if (!c.valid) return;
+        const int u = u_first + (sorted ? (int)order_s[pos] : pos);
+        c.b = u / p.Hkv;
+        c.kvh = u - c.b * p.Hkv;
+        c.len = lens_s[c.b];
+        c.chunks = cum_s[c.b + 1] - cum_s[c.b];
+    };
+    auto live = [&](const Cursor &c) { return c.valid; };
+    auto advance_head = [&](Cursor &c) {          // next chunk, or the first chunk of the next unit in the queue
+        if (++c.chunk < c.chunks) return;
+        int pos = 0;
+        if (lane == 0) pos = atomicAdd(&ctl[2], 1);
+        pos = __shfl_sync(0xffffffffu, pos, 0);
+        fifo[fifo_wr & (kFifo - 1)] = pos;        // all lanes, the same value
+        ++fifo_wr;
+        load_unit(c, pos);
+    };
+    auto advance_tail = [&](Cursor &c) {          // the fetch side is ahead: it has taken the next unit already
+        if (++c.chunk < c.chunks) return;
+        if (fifo_rd == fifo_wr) {
+            c.valid = false;
+            return;
+        }
+        load_unit(c, fifo[fifo_rd & (kFifo - 1)]);
+        ++fifo_rd;
+    };
+    Cursor first;
+    first.b = first.kvh = first.len = first.chunks = 0;
+    load_unit(first, warp);
 
     // per-lane constants of the copies: piece i of a lane is row (32 i + lane) / kRowPieces, 16-byte piece
     // (32 i + lane) % kRowPieces of the row
@@ -234,7 +277,7 @@ __global__ void __launch_bounds__(kWarps * 32) decode_warp_kernel(const WarpPara
     for (int i = 0; i < S - 1; ++i) {
         if (live(head)) {
             issue(head, head_slot);
-            advance(head);
+            advance_head(head);
         }
         cp_async_commit();
         head_slot = head_slot + 1 == S ? 0 : head_slot + 1;
@@ -247,7 +290,7 @@ __global__ void __launch_bounds__(kWarps * 32) decode_warp_kernel(const WarpPara
     while (live(tail)) {
         if (live(head)) {
             issue(head, head_slot);
-            advance(head);
+            advance_head(head);
         }
         cp_async_commit();
         head_slot = head_slot + 1 == S ? 0 : head_slot + 1;
@@ -351,12 +394,12 @@ __global__ void __launch_bounds__(kWarps * 32) decode_warp_kernel(const WarpPara
         }
         __syncwarp();                              // every lane is done with the slot before it is filled again
         tail_slot = tail_slot + 1 == S ? 0 : tail_slot + 1;
-        advance(tail);
+        advance_tail(tail);
     }
     cp_async_wait<0>();
 }
 
-size_t warp_smem_bytes(int D, int G, int warps, int stages) { return 9 * 1024 + (size_t)warps * stages * stage_bytes(D, G); }
+size_t warp_smem_bytes(int D, int G, int warps, int stages) { return kMetaBytes + (size_t)warps * stages * stage_bytes(D, G); }
 
 template <int D, int W>
 int blocks_per_sm(size_t smem)
@@ -406,11 +449,12 @@ bool decode_warp_eligible(int B, int Hq, int Hkv, int D, int max_kv_len, bool fp
     if (const char *e = getenv("L4L_DECODE_WARP")) return e[0] != '0';
     // many units of a few chunks each: the regime where the split kernel pays its per-piece cost every tile or two.
     // Thresholds measured against the split kernel (8 KV heads at head_dim 128, 12 at head_dim 64): with at most 256
-    // tokens per sequence it wins from about half a unit per resident warp, with at most 512 from about two.
+    // tokens per sequence it wins from about half a unit per resident warp, with at most 512 from about one (two at
+    // head_dim 64).
     const long long units = (long long)B * Hkv;
     const long long slots = (long long)sm_count() * (D == 64 ? 16 : pick_warp_shape(D, G).warps);
     if (max_kv_len <= 256) return units * 16 >= slots * 9;
-    if (max_kv_len <= 512) return units * 10 >= slots * 22;
+    if (max_kv_len <= 512) return units * 10 >= slots * (D == 64 ? 22 : 11);
     return false;
 }
 
