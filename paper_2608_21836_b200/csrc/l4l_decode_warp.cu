@@ -423,15 +423,11 @@ int blocks_per_sm(size_t smem)
 
 // Warps per CTA and ring depth. The arithmetic of a warp is one dependent chain per chunk, so the SM wants as many
 // warps as its shared memory can give a ring of at least two chunks: 12 at head_dim 128 (groups of up to 4 query
-// heads; 8 above), 8 in each of two CTAs at head_dim 64.
+// heads; 8 for groups of 5 to 16), 8 in each of two CTAs at head_dim 64.
 struct WarpShape { int warps, stages; };
 WarpShape pick_warp_shape(int D, int G)
 {
-    int warps = (D == 128 && G <= 4) ? 12 : 8;
-    if (const char *e = getenv("L4L_DECODE_WARP_WARPS")) {
-        const int w = atoi(e);
-        if (D == 128 && (w == 8 || w == 12)) warps = w;
-    }
+    const int warps = (D == 128 && G <= 4) ? 12 : 8;
     const size_t limit = (D == 64 ? 113u : 227u) * 1024u;
     for (int s = 5; s >= 2; --s)
         if (warp_smem_bytes(D, G, warps, s) <= limit) return {warps, s};
@@ -445,7 +441,7 @@ WarpShape pick_warp_shape(int D, int G)
 bool decode_warp_eligible(int B, int Hq, int Hkv, int D, int max_kv_len, bool fp8, bool rope)
 {
     const int G = Hq / Hkv;
-    if (fp8 || rope || G > 8 || pick_warp_shape(D, G).stages == 0) return false;
+    if (fp8 || rope || G > 16 || pick_warp_shape(D, G).stages == 0) return false;
     if (const char *e = getenv("L4L_DECODE_WARP")) return e[0] != '0';
     // many units of a few chunks each: the regime where the split kernel pays its per-piece cost every tile or two.
     // Thresholds measured against the split kernel (8 KV heads at head_dim 128, 12 at head_dim 64): with at most 256
@@ -466,7 +462,7 @@ l4l_status launch_decode_warp(const void *q, void *o, const l4l_kv_cache &cache,
     const int G = Hq / Hkv;
     const WarpShape shape = pick_warp_shape(D, G);
     const int stages = shape.stages, kWarps = shape.warps;
-    if (stages == 0 || G > 8 || (k_new == nullptr) != (v_new == nullptr)) return L4L_ERR_UNSUPPORTED;
+    if (stages == 0 || G > 16 || (k_new == nullptr) != (v_new == nullptr)) return L4L_ERR_UNSUPPORTED;
     const size_t smem = warp_smem_bytes(D, G, kWarps, stages);
     const int per_sm = D == 64 ? blocks_per_sm<64, 8>(smem)
                                : (kWarps == 12 ? blocks_per_sm<128, 12>(smem) : blocks_per_sm<128, 8>(smem));

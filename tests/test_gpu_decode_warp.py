@@ -32,7 +32,7 @@ def warp_kernel(request):
 
 
 @pytest.mark.parametrize("D", [64, 128])
-@pytest.mark.parametrize("Hq,Hkv", [(8, 2), (8, 8), (8, 1), (3, 1), (6, 2), (32, 8)])
+@pytest.mark.parametrize("Hq,Hkv", [(8, 2), (8, 8), (8, 1), (3, 1), (6, 2), (32, 8), (16, 1), (24, 2)])
 def test_warp_decode_ragged_edge_lengths(warp_kernel, D, Hq, Hkv):
     # around every boundary: empty, one token, 16-token chunks, more chunks than ring stages
     lens = [0, 1, 2, 15, 16, 17, 31, 32, 33, 47, 48, 127, 128, 129, 255, 300, 0, 7]
@@ -72,7 +72,7 @@ def test_warp_decode_extreme_scores_token_major_cache_and_clamp(warp_kernel):
     assert_close_to_oracle(o, ref, "clamped decode")
 
 
-@pytest.mark.parametrize("D,Hq,Hkv", [(128, 8, 2), (64, 4, 4), (128, 8, 1), (128, 32, 8)])
+@pytest.mark.parametrize("D,Hq,Hkv", [(128, 8, 2), (64, 4, 4), (128, 8, 1), (128, 32, 8), (128, 16, 1), (64, 26, 2)])
 def test_warp_decode_with_fused_append(warp_kernel, D, Hq, Hkv):
     from test_gpu_decode_append import make_case
 
