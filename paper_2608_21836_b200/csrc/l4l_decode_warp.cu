@@ -421,17 +421,38 @@ int blocks_per_sm(size_t smem)
     return n;
 }
 
-// Warps per CTA and ring depth. The arithmetic of a warp is one dependent chain per chunk, so the SM wants as many
-// warps as its shared memory can give a ring of at least two chunks: 12 at head_dim 128 (groups of up to 4 query
-// heads; 8 for groups of 5 to 16), 8 in each of two CTAs at head_dim 64.
-struct WarpShape { int warps, stages; };
-WarpShape pick_warp_shape(int D, int G)
+// Warps per CTA and ring depth. A CTA's shared memory holds a fixed number of chunks (24 at head_dim 128 with groups
+// of up to 4 query heads); it is divided among as many warps as the CTA has units to work on at a time. With many
+// units per SM the arithmetic of a warp (one dependent chain per chunk) is the bound and 12 warps with 2-chunk
+// rings are fastest; with few units per SM a warp's chain of memory round trips is the bound and fewer warps with
+// deeper rings (up to 6 chunks) are. head_dim 64 runs two CTAs per SM (of 8 warps at most: registers).
+struct WarpShape { int warps, stages, ctas_per_sm; };
+WarpShape pick_warp_shape(int D, int G, long long units)
 {
-    const int warps = (D == 128 && G <= 4) ? 12 : 8;
-    const size_t limit = (D == 64 ? 113u : 227u) * 1024u;
-    for (int s = 5; s >= 2; --s)
-        if (warp_smem_bytes(D, G, warps, s) <= limit) return {warps, s};
-    return {warps, 0};
+    const int cps = D == 64 ? 2 : 1;
+    const size_t budget = (D == 64 ? 113u : 227u) * 1024u - kMetaBytes;
+    const int total = (int)(budget / stage_bytes(D, G));             // chunks of ring per CTA
+    const long long ctas = (long long)sm_count() * cps;
+    const long long per_cta = (units + ctas - 1) / ctas;
+    const int wmax = (D == 128 && total >= 24) ? 12 : 8;
+    int warps = 4;
+    for (int w : {4, 6, 8, 12}) {
+        if (w > wmax) break;
+        warps = w;
+        if (w >= per_cta) break;
+    }
+    const int stages = total / warps < 6 ? total / warps : 6;
+    return {warps, stages >= 2 ? stages : 0, cps};
+}
+
+using WarpKernel = void (*)(const WarpParams);
+struct KernelEntry { WarpKernel fn; int (*blocks)(size_t); };
+template <int D, int W>
+KernelEntry entry() { return {decode_warp_kernel<D, W>, &blocks_per_sm<D, W>}; }
+KernelEntry pick_kernel(int D, int warps)
+{
+    if (D == 64) return warps == 4 ? entry<64, 4>() : warps == 6 ? entry<64, 6>() : entry<64, 8>();
+    return warps == 4 ? entry<128, 4>() : warps == 6 ? entry<128, 6>() : warps == 8 ? entry<128, 8>() : entry<128, 12>();
 }
 
 }  // namespace
@@ -441,16 +462,16 @@ WarpShape pick_warp_shape(int D, int G)
 bool decode_warp_eligible(int B, int Hq, int Hkv, int D, int max_kv_len, bool fp8, bool rope)
 {
     const int G = Hq / Hkv;
-    if (fp8 || rope || G > 16 || pick_warp_shape(D, G).stages == 0) return false;
+    const long long units = (long long)B * Hkv;
+    if (fp8 || rope || G > 16 || pick_warp_shape(D, G, units).stages == 0) return false;
     if (const char *e = getenv("L4L_DECODE_WARP")) return e[0] != '0';
     // many units of a few chunks each: the regime where the split kernel pays its per-piece cost every tile or two.
-    // Thresholds measured against the split kernel (8 KV heads at head_dim 128, 12 at head_dim 64): with at most 256
-    // tokens per sequence it wins from about half a unit per resident warp, with at most 512 from about one (two at
-    // head_dim 64).
-    const long long units = (long long)B * Hkv;
-    const long long slots = (long long)sm_count() * (D == 64 ? 16 : pick_warp_shape(D, G).warps);
-    if (max_kv_len <= 256) return units * 16 >= slots * 9;
-    if (max_kv_len <= 512) return units * 10 >= slots * (D == 64 ? 22 : 11);
+    // Thresholds measured against the split kernel in CUDA graphs (8 KV heads at head_dim 128, 12 at head_dim 64),
+    // in units per SM: with at most 256 tokens per sequence it wins from 3 units per SM (8 at head_dim 64), with
+    // at most 512 from 10 (30).
+    const long long sms = sm_count();
+    if (max_kv_len <= 256) return units >= (D == 64 ? 8 : 3) * sms;
+    if (max_kv_len <= 512) return units >= (D == 64 ? 30 : 10) * sms;
     return false;
 }
 
@@ -460,15 +481,17 @@ l4l_status launch_decode_warp(const void *q, void *o, const l4l_kv_cache &cache,
                               const PagedTable *paged)
 {
     const int G = Hq / Hkv;
-    const WarpShape shape = pick_warp_shape(D, G);
-    const int stages = shape.stages, kWarps = shape.warps;
-    if (stages == 0 || G > 16 || (k_new == nullptr) != (v_new == nullptr)) return L4L_ERR_UNSUPPORTED;
-    const size_t smem = warp_smem_bytes(D, G, kWarps, stages);
-    const int per_sm = D == 64 ? blocks_per_sm<64, 8>(smem)
-                               : (kWarps == 12 ? blocks_per_sm<128, 12>(smem) : blocks_per_sm<128, 8>(smem));
-    if (per_sm == 0) return L4L_ERR_CUDA;
+    if (G > 16 || (k_new == nullptr) != (v_new == nullptr)) return L4L_ERR_UNSUPPORTED;
     for (int b0 = 0; b0 < B; b0 += kMaxB) {
         const int nb = B - b0 < kMaxB ? B - b0 : kMaxB;
+        const long long units = (long long)nb * Hkv;
+        const WarpShape shape = pick_warp_shape(D, G, units);
+        const int stages = shape.stages, kWarps = shape.warps;
+        if (stages == 0) return L4L_ERR_UNSUPPORTED;
+        const size_t smem = warp_smem_bytes(D, G, kWarps, stages);
+        const KernelEntry kernel = pick_kernel(D, kWarps);
+        const int per_sm = kernel.blocks(smem);
+        if (per_sm == 0) return L4L_ERR_CUDA;
         WarpParams p = {};
         p.q = static_cast<const __nv_bfloat16 *>(q) + (size_t)b0 * Hq * D;
         p.o = static_cast<__nv_bfloat16 *>(o) + (size_t)b0 * Hq * D;
@@ -494,10 +517,9 @@ l4l_status launch_decode_warp(const void *q, void *o, const l4l_kv_cache &cache,
         p.B = nb; p.Hq = Hq; p.Hkv = Hkv; p.G = G; p.max_kv_len = max_kv_len; p.stages = stages;
         p.scale_log2e = scale * 1.4426950408889634f;
 
-        // persistent: every resident warp gets its share; never more warps than units
+        // persistent: every resident CTA gets its share of the stream; never more CTAs than units
         long long blocks = (long long)per_sm * sm_count();
-        const long long units = (long long)nb * Hkv;
-        if (blocks * kWarps > units) blocks = (units + kWarps - 1) / kWarps;
+        if (blocks > units) blocks = units;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)blocks, 1, 1);
         cfg.blockDim = dim3(kWarps * 32, 1, 1);
@@ -508,9 +530,7 @@ l4l_status launch_decode_warp(const void *q, void *o, const l4l_kv_cache &cache,
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        const cudaError_t err = D == 64 ? cudaLaunchKernelEx(&cfg, decode_warp_kernel<64, 8>, p)
-                                : (kWarps == 12 ? cudaLaunchKernelEx(&cfg, decode_warp_kernel<128, 12>, p)
-                                                : cudaLaunchKernelEx(&cfg, decode_warp_kernel<128, 8>, p));
+        const cudaError_t err = cudaLaunchKernelEx(&cfg, kernel.fn, p);
         if (err != cudaSuccess) {
             (void)cudaGetLastError();
             return L4L_ERR_CUDA;
