@@ -615,7 +615,7 @@ def run_ours(args, rank, world):
 def run_profile_case(case: str):
     """A few launches of ONE kernel on a small case, for `ncu` captures (not a benchmark):
     prefill = B=1, S=8192 of the long_prefill workload (inputs 168 MB > L2); decode = the batched_decode batch;
-    rglru = the RG-LRU scan on B=16, T=2048, W=2560; decode_small = the cluster decode kernel on B=4 x 8192 tokens; decode_short = the warp-per-unit decode kernel on B=512 x 64..256 tokens; rope = rope + norm + cache update on B=2, S=8192."""
+    rglru = the RG-LRU scan on B=16, T=2048, W=2560; decode_small = the cluster decode kernel on B=4 x 8192 tokens; decode_short = the warp-per-unit decode kernel on B=512 x 64..256 tokens; decode_fp8 = the split kernel on the batched_decode batch in an fp8 cache; rope = rope + norm + cache update on B=2, S=8192."""
     from paper_2608_21836_b200 import binding as l4l
 
     torch.cuda.set_device(0)
@@ -665,6 +665,21 @@ def run_profile_case(case: str):
         ws = l4l.new_workspace(l4l.L4L_OP_DECODE, 4, w.Hq, w.Hkv, w.D, 8192)
         for _ in range(3):
             l4l.l4l_attn_decode(q, o, ck, cv, lens, 8192, w.scale, ws)
+    elif case == "decode_fp8":
+        # the split kernel on an fp8 (e4m3) cache: the batched_decode batch quantised with one scale per KV head
+        w = wl.WORKLOADS["batched_decode"]
+        db = wl.make_decode_batch(w, poison_tail=False)
+        q, lens = db.q.cuda(), db.kv_len.cuda()
+        B, Lmax = w.decode_B, w.decode_Lmax
+        k8 = torch.zeros(B, w.Hkv, Lmax, w.D, dtype=torch.uint8, device="cuda")
+        v8 = torch.zeros_like(k8)
+        sc = torch.full((w.Hkv,), 4.5 / 448, dtype=torch.float32, device="cuda")
+        l4l.l4l_kv_append_fp8(k8, v8, db.cache_k.cuda().permute(0, 2, 1, 3), db.cache_v.cuda().permute(0, 2, 1, 3),
+                              torch.zeros(B, dtype=torch.int32, device="cuda"), sc, sc)
+        o = torch.empty_like(q)
+        ws = l4l.new_workspace(l4l.L4L_OP_DECODE, B, w.Hq, w.Hkv, w.D, Lmax)
+        for _ in range(3):
+            l4l.l4l_attn_decode_fp8(q, o, k8, v8, sc, sc, lens, Lmax, w.scale, ws)
     elif case == "decode_short":
         # the warp-per-unit kernel: B = 512 sequences of 64 to 256 tokens of the 8B-shaped layer (338 MB of cache > L2)
         w = wl.WORKLOADS["batched_decode"]
@@ -693,7 +708,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--profile-case", choices=["prefill", "decode", "decode_small", "decode_short", "rope", "rglru"], default=None,
+    ap.add_argument("--profile-case", choices=["prefill", "decode", "decode_small", "decode_short", "decode_fp8", "rope", "rglru"], default=None,
                     help="run three launches of one kernel on a small case and exit (for ncu)")
     args = ap.parse_args()
     if args.profile_case:
