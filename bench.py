@@ -459,6 +459,44 @@ def run_ours(args, rank, world):
 
     t_short, short_bytes, err_short = short_batch_us(False)
     t_short_split, _, err_short2 = short_batch_us(True)
+    # the other configurations of the workload list, each as its own kernel timing: the prefill of the 8B-shaped layer
+    # config (B = 1, S = 2048) and of the small MHA model (B = 8, S = 512, head_dim 64), and the MHA decode batch
+    # (B = 64 at context 1024; 201 MB, three cache copies in rotation)
+    def other_prefill(name):
+        w2 = wl.WORKLOADS[name]
+        sq = wl.make_sequence(w2, T=0)
+        q2, k2, v2 = sq.q.to(dev), sq.k.to(dev), sq.v.to(dev)
+        o2 = torch.empty_like(q2)
+        B2, S2 = q2.shape[0], q2.shape[1]
+        ck2 = torch.empty(B2, w2.Hkv, S2, w2.D, dtype=torch.bfloat16, device=dev)
+        cv2 = torch.empty_like(ck2)
+        l2 = torch.full((B2,), S2, dtype=torch.int32, device=dev)
+        ws2 = l4l.new_workspace(l4l.L4L_OP_PREFILL, B2, w2.Hq, w2.Hkv, w2.D, S2, device=dev)
+        t = timed(lambda: l4l.l4l_attn_prefill(q2, k2, v2, o2, l2, w2.scale, ws2, cache_k=ck2, cache_v=cv2), 20)
+        fl = wl.prefill_flops(w2.Hq, w2.D, [S2] * B2)
+        return {"us": t * 1e3, "tflops": fl / (t * 1e-3) / 1e12, "device_error": l4l.l4l_last_device_error(ws2)}
+
+    def other_decode(name):
+        w2 = wl.WORKLOADS[name]
+        sb = wl.make_decode_batch(w2, poison_tail=False)
+        nbytes = wl.decode_kv_bytes(w2.Hkv, w2.D, sb.kv_len.tolist())
+        cp = [(sb.cache_k.to(dev), sb.cache_v.to(dev)) for _ in range(3)]
+        q2, l2 = sb.q.to(dev), sb.kv_len.to(dev)
+        o2 = torch.empty_like(q2)
+        ws2 = l4l.new_workspace(l4l.L4L_OP_DECODE, w2.decode_B, w2.Hq, w2.Hkv, w2.D, w2.decode_Lmax, device=dev)
+
+        def step():
+            ck_i, cv_i = cp[rot[0] % 3]
+            rot[0] += 1
+            l4l.l4l_attn_decode(q2, o2, ck_i, cv_i, l2, w2.decode_Lmax, w2.scale, ws2)
+        t = timed(step, 21)
+        return {"us": t * 1e3, "kv_gbs": nbytes / (t * 1e-3) / 1e9, "device_error": l4l.l4l_last_device_error(ws2)}
+
+    other = {"layer8b_prefill_B1_S2048": other_prefill("layer8b"), "mha_small_prefill_B8_S512": other_prefill("mha_small"),
+             "mha_small_decode_B64_L1024": other_decode("mha_small")}
+    err_other = 0
+    for v_ in other.values():
+        err_other |= v_.pop("device_error")
     t_small, err_small = small_batch_step_us(2304, False)
     t_small_split, err_small2 = small_batch_step_us(2304, True)
     # second workload: the RG-LRU recurrence of a RecurrentGemma-2B-sized block (2560 channels) over a long prompt
@@ -483,7 +521,7 @@ def run_ours(args, rank, world):
     t_rglru2 = timed(lambda: l4l.l4l_rglru_scan(v2(rx), v2(rgx), v2(rga), r_ap, r_state2, v2(ry), ws_r2), 10)
     dev_err_r |= l4l.l4l_last_device_error(ws_r2)
     del rx, rgx, rga, ry, filler
-    dev_err = l4l.l4l_last_device_error(ws_p) | l4l.l4l_last_device_error(ws_d) | dev_err_r | err_small | err_small2 | err_g8 | err_short | err_short2
+    dev_err = l4l.l4l_last_device_error(ws_p) | l4l.l4l_last_device_error(ws_d) | dev_err_r | err_small | err_small2 | err_g8 | err_short | err_short2 | err_other
 
     # ---- end to end through the same entry points with HOST buffers (pinned), copies inside the timed region
     hq, hk, hv = seq.q.pin_memory(), seq.k.pin_memory(), seq.v.pin_memory()
@@ -597,6 +635,7 @@ def run_ours(args, rank, world):
             "decode_fp8_cache": {"us": t_fp8 * 1e3, "kv_gbs_fp8_bytes": dec_bytes / 2 / (t_fp8 * 1e-3) / 1e9,
                                  "speedup_over_bf16_cache": t_dec_b2b / t_fp8},
             "decode_64_query_heads_on_8_kv_heads": {"us": t_g8 * 1e3, "kv_gbs": dec_bytes / (t_g8 * 1e-3) / 1e9},
+            "other_configs": other,
             "decode_B512_L64_to_256": {"warp_kernel_us": t_short * 1e3, "kv_gbs": short_bytes / (t_short * 1e-3) / 1e9,
                                        "split_kernel_us": t_short_split * 1e3},
             "decode_step_B1_L2304_in_cuda_graph": {"cluster_kernel_us": t_small, "split_kernel_us": t_small_split},
