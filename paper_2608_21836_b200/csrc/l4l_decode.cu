@@ -114,6 +114,7 @@ struct DecodeParams {
     // at offset t % page_size; the tensor maps then describe the page pool [pages, Hkv, page_size, D]
     const int32_t *block_table;
     int table_stride, page_size, page_shift, num_pages;
+    int page_box;             // paged: tokens per box of tmap_k / tmap_v (divides the tile, never straddles a page)
     int tail_rows;            // tokens per box of tmap_k_tail / tmap_v_tail (32, or the page size if that is smaller)
     int B, Hq, Hkv, G, min_tiles, nsplit, max_kv_len;
     int nfin;                 // finisher warps (BigG: one per 4 query heads of the group; else 1)
@@ -343,7 +344,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     const int rem = len - tile * kTileT;
                     const int groups = (rem + p.tail_rows - 1) / p.tail_rows;
                     const bool by_groups = rem < kTileT && groups * p.tail_rows * 2 <= kTileT;
-                    const int box_rows = by_groups ? p.tail_rows : ((paged && p.page_size < kTileT) ? p.page_size : kTileT);
+                    const int box_rows = by_groups ? p.tail_rows : (paged ? p.page_box : kTileT);
                     const int n_box = by_groups ? groups : ((rem >= kTileT || box_rows == kTileT) ? kTileT / box_rows
                                                                                                   : (rem + box_rows - 1) / box_rows);
                     const uint32_t kv_bytes = (uint32_t)n_box * box_rows * 128u * C::kHalves * 2u;
@@ -1103,9 +1104,9 @@ DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_
     int n_dev = 0;
     const bool have_dev = cudaGetDeviceCount(&n_dev) == cudaSuccess && n_dev > 0;
     if (!have_dev) (void)cudaGetLastError();
-    // groups of 9 to 16 query heads at head_dim 128: the 6-warp shape (contiguous caches and pages of 16 or 32
-    // tokens: its 96-token tiles do not line up with larger pages)
-    if (D == 128 && Hq / Hkv > 8 && (page_size == 0 || page_size == 16 || page_size == 32)) {
+    // groups of 9 to 16 query heads at head_dim 128: the 6-warp shape (its 96-token tiles are fetched in 32-token
+    // boxes from pages they do not line up with)
+    if (D == 128 && Hq / Hkv > 8) {
         const DecodePlan six = plan_for_shape(B, Hq, Hkv, D, max_kv_len, ws_limit, 6, have_dev, fp8);
         if (six.fits && six.ws_bytes <= ws_limit) return six;
     }
@@ -1135,7 +1136,6 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
     if (fp8 && (D != 128 || k_new || v_new)) return L4L_ERR_UNSUPPORTED;
     const int esz = fp8 ? 1 : 2;
     // paged: `cache` describes the page pool (stride_b = stride between pages, max_len = page size)
-    if (paged && plan.warps == 6 && cache.max_len != 16 && cache.max_len != 32) return L4L_ERR_UNSUPPORTED;   // 96-token tiles
     // hundreds of short sequences: one warp per (sequence, KV head), nothing to merge
     if (decode_warp_eligible(B, Hq, Hkv, D, max_kv_len, fp8 != nullptr, rope != nullptr))
         return launch_decode_warp(q, o, cache, d_kv_lens, max_kv_len, B, Hq, Hkv, D, scale, d_lse, stream, k_new, v_new,
@@ -1174,8 +1174,10 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         const uint8_t *kb = static_cast<const uint8_t *>(cache.k) + first * esz;
         const uint8_t *vb = static_cast<const uint8_t *>(cache.v) + first * esz;
         const int box_d = fp8 ? 128 : 64;
-        // pages smaller than a tile are fetched page by page: no box may exceed the page
-        const int box_t = (paged && cache.max_len < kTileT) ? cache.max_len : kTileT;
+        // no box may straddle pages: pages smaller than a tile are fetched page by page, and tiles that are not a
+        // power of two (96 tokens) over larger pages in 32-token boxes (page sizes are powers of two >= 16)
+        int box_t = kTileT;
+        if (paged) box_t = (kTileT % cache.max_len == 0) ? cache.max_len : (cache.max_len % kTileT == 0 ? kTileT : 32);
         const int tail_rows = (paged && cache.max_len < 32) ? cache.max_len : 32;
         if (!make_tmap(&tk, &coord, kb, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
                        cache.stride_b, box_d, box_t, esz) ||
@@ -1211,6 +1213,7 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         p.block_table = paged ? paged->block_table + (size_t)b0 * paged->table_stride : nullptr;
         p.table_stride = paged ? paged->table_stride : 0;
         p.page_size = paged ? cache.max_len : 0;
+        p.page_box = box_t;
         p.num_pages = paged ? paged->num_pages : 0;
         p.tail_rows = tail_rows;
         p.page_shift = 0;

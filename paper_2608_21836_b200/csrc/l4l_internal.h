@@ -43,8 +43,8 @@ struct DecodePlan {
     int nsplit;      // max pieces a (sequence, KV head) can be cut into
     size_t ws_bytes; // status block + ticket counters + partials
 };
-// page_size: 0 for a contiguous cache, else the tokens per page of a paged cache (some kernel shapes need tiles
-// that line up with pages)
+// page_size: 0 for a contiguous cache, else the tokens per page of a paged cache (kept for shapes whose tiles must
+// line up with pages; none does at present)
 DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_limit, bool fp8 = false,
                        int page_size = 0);
 
