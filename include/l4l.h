@@ -19,8 +19,9 @@
  *   l4l_attn_prefill_chunk (new tokens over a populated cache), l4l_attn_decode_append (cache
  *   update fused into the decode step), l4l_rope_kv_append (rotary embedding and QK-norm fused
  *   with the cache update), l4l_attn_decode_paged / l4l_kv_append_paged / l4l_attn_decode_paged_append
- *   (page pool + block table), l4l_attn_decode_fp8 / l4l_kv_append_fp8 (e4m3 cache), l4l_attn_decode_static (no
- *   caller workspace), and a second workload, l4l_rglru_scan (gated linear recurrence).
+ *   (page pool + block table), l4l_attn_decode_fp8 / l4l_kv_append_fp8 / l4l_attn_decode_append_fp8
+ *   (e4m3 cache), l4l_attn_decode_static (no caller workspace), and a second workload,
+ *   l4l_rglru_scan (gated linear recurrence).
  *
  * Conventions shared by every call
  *   - All tensors are bf16 (16-bit words) in DEVICE memory unless a parameter says "host".
@@ -184,6 +185,20 @@ l4l_status l4l_attn_decode_paged_fp8(const void *q, void *o, l4l_paged_kv pool8,
                                      const int32_t *d_kv_lens, int max_kv_len, int B, int Hq, int Hkv,
                                      int head_dim, float scale, float *d_lse, void *workspace,
                                      size_t ws_bytes, l4l_stream stream);
+/* l4l_attn_decode_append over an fp8 cache: the step's newest token (bf16 k_new / v_new, [B, 1, Hkv, D]) is
+ * quantised with the arithmetic of l4l_kv_append_fp8 (the stored codes are the same, bit for bit), written to
+ * slot kv_lens[b] - 1 and attended with the rest in the same launch. Contiguous cache, or page pool + block
+ * table (rules of l4l_attn_decode_paged_append). */
+l4l_status l4l_attn_decode_append_fp8(const void *q, void *o, l4l_kv_cache cache8, const float *d_k_scale,
+                                      const float *d_v_scale, l4l_tensor4 k_new, l4l_tensor4 v_new,
+                                      const int32_t *d_kv_lens, int max_kv_len, int B, int Hq, int Hkv,
+                                      int head_dim, float scale, float *d_lse, void *workspace, size_t ws_bytes,
+                                      l4l_stream stream);
+l4l_status l4l_attn_decode_paged_append_fp8(const void *q, void *o, l4l_paged_kv pool8, const float *d_k_scale,
+                                            const float *d_v_scale, const int32_t *d_block_table, int table_stride,
+                                            l4l_tensor4 k_new, l4l_tensor4 v_new, const int32_t *d_kv_lens,
+                                            int max_kv_len, int B, int Hq, int Hkv, int head_dim, float scale,
+                                            float *d_lse, void *workspace, size_t ws_bytes, l4l_stream stream);
 
 /*
  * The whole decode step of one attention layer in ONE launch: rotary embedding (and optional per-head RMS

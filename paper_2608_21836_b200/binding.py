@@ -25,7 +25,7 @@ EXPORTS = (
     "l4l_attn_decode_static", "l4l_attn_decode_append", "l4l_attn_prefill_chunk", "l4l_rope_kv_append",
     "l4l_kv_append_paged", "l4l_attn_decode_paged", "l4l_kv_append_fp8", "l4l_attn_decode_fp8", "l4l_rglru_scan", "l4l_rglru_workspace_bytes",
     "l4l_attn_decode_paged_fp8", "l4l_attn_merge", "l4l_attn_decode_rope_append", "l4l_attn_decode_paged_append",
-    "l4l_attn_decode_paged_rope_append",
+    "l4l_attn_decode_paged_rope_append", "l4l_attn_decode_append_fp8", "l4l_attn_decode_paged_append_fp8",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -97,6 +97,12 @@ def load() -> ctypes.CDLL:
     lib.l4l_attn_decode_paged_rope_append.argtypes = [vp, vp, PagedKV, i32p, c_int, Tensor4, Tensor4, i32p, c_int, c_int,
                                                       c_int, c_int, c_int, ctypes.c_float, vp, vp, c_int, vp, vp,
                                                       ctypes.c_float, vp, vp, c_size, vp]
+    lib.l4l_attn_decode_append_fp8.restype = c_int
+    lib.l4l_attn_decode_append_fp8.argtypes = [vp, vp, KVCache, vp, vp, Tensor4, Tensor4, i32p, c_int, c_int, c_int, c_int,
+                                               c_int, ctypes.c_float, vp, vp, c_size, vp]
+    lib.l4l_attn_decode_paged_append_fp8.restype = c_int
+    lib.l4l_attn_decode_paged_append_fp8.argtypes = [vp, vp, PagedKV, vp, vp, i32p, c_int, Tensor4, Tensor4, i32p, c_int,
+                                                     c_int, c_int, c_int, c_int, ctypes.c_float, vp, vp, c_size, vp]
     lib.l4l_kv_append_fp8.restype = c_int
     lib.l4l_kv_append_fp8.argtypes = [KVCache, Tensor4, Tensor4, i32p, i32p, c_int, c_int, c_int, c_int, vp, vp, vp]
     lib.l4l_attn_decode_fp8.restype = c_int
@@ -520,6 +526,34 @@ def l4l_attn_decode_paged_fp8(q, o, pool_k8, pool_v8, k_scale, v_scale, block_ta
                                           workspace.numel() * workspace.element_size(), _stream())
     if st != L4L_OK:
         raise L4LError(st, "l4l_attn_decode_paged_fp8")
+
+
+def l4l_attn_decode_append_fp8(q, o, cache_k8, cache_v8, k_scale, v_scale, k_new, v_new, kv_lens, max_kv_len: int,
+                               scale: float, workspace, lse=None, block_table=None) -> None:
+    """One launch per decode step over an fp8 cache: bf16 k_new / v_new ([B,1,Hkv,128]) are quantised as
+    l4l_kv_append_fp8 does, written to slot kv_lens[b]-1 and attended with the rest. With block_table, cache_k8 /
+    cache_v8 are a page pool [pages, Hkv, page_size, 128]."""
+    _check_bf16_cuda(q, "q")
+    _check_bf16_cuda(o, "o")
+    if not (q.is_contiguous() and o.is_contiguous() and q.dim() == 3 and q.shape == o.shape):
+        raise ValueError("q and o must be dense [B, Hq, D]")
+    B, Hq, D = q.shape
+    Hkv = cache_k8.shape[1]
+    if tuple(k_new.shape) != (B, 1, Hkv, D) or tuple(v_new.shape) != (B, 1, Hkv, D):
+        raise ValueError("k_new and v_new must be [B, 1, Hkv, D]")
+    c = kv_cache8(cache_k8, cache_v8)
+    common = (tensor4(k_new, "k_new"), tensor4(v_new, "v_new"), _i32_dev(kv_lens, "kv_lens"), int(max_kv_len), B, Hq, Hkv,
+              D, float(scale), None if lse is None else lse.data_ptr(), workspace.data_ptr(),
+              workspace.numel() * workspace.element_size(), _stream())
+    ks, vs = _f32_dev(k_scale, "k_scale", (Hkv,)), _f32_dev(v_scale, "v_scale", (Hkv,))
+    if block_table is None:
+        st = load().l4l_attn_decode_append_fp8(q.data_ptr(), o.data_ptr(), c, ks, vs, *common)
+    else:
+        pool = PagedKV(c.k, c.v, c.stride_b, c.stride_h, c.stride_t, cache_k8.shape[2], cache_k8.shape[0])
+        tbl, stride = _block_table(block_table, B)
+        st = load().l4l_attn_decode_paged_append_fp8(q.data_ptr(), o.data_ptr(), pool, ks, vs, tbl, stride, *common)
+    if st != L4L_OK:
+        raise L4LError(st, "l4l_attn_decode_append_fp8")
 
 
 def l4l_attn_merge(o_parts, lse_parts, o, lse=None) -> None:

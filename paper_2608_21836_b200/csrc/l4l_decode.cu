@@ -24,6 +24,7 @@
 #include <cstdlib>
 #include <mutex>
 
+#include "l4l_fp8_quant.cuh"
 #include "l4l_internal.h"
 #include "l4l_rope_frag.cuh"
 #include "l4l_warp_attn.cuh"
@@ -824,6 +825,36 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 __syncwarp();
             }
             if constexpr (F8) {
+                if (p.k_new != nullptr && nvalid > 0 && nvalid <= 16 * C::kSub) {
+                    // fused append into an fp8 cache: the newest token's K/V rows are quantised here exactly as the
+                    // cache update quantises them (same division, same rounding), patched into the tile and written
+                    // to their cache slot; 8 lanes, 16 values each
+                    const int last = row0 + nvalid - 1;
+                    if (lane < 8) {
+                        const size_t src = (size_t)mt.b * p.new_sb + (size_t)mt.kvh * p.new_sh + lane * 16;
+                        const uint4 *ks = reinterpret_cast<const uint4 *>(p.k_new + src);
+                        const uint4 *vs = reinterpret_cast<const uint4 *>(p.v_new + src);
+                        const uint4 kq = quantise16(__ldg(ks), __ldg(ks + 1), k_sc);
+                        const uint4 vq = quantise16(__ldg(vs), __ldg(vs + 1), v_sc);
+                        long long outer = mt.b, slot = mt.kv_len - 1;
+                        if (p.block_table != nullptr) {
+                            outer = __ldg(p.block_table + (size_t)mt.b * p.table_stride + (slot >> p.page_shift));
+                            slot &= p.page_size - 1;
+                        }
+                        if (p.block_table == nullptr || (outer >= 0 && outer < p.num_pages)) {
+                            uint8_t *kt = stages + (size_t)s * C::kStageBytes;
+                            const uint32_t off = swz128(last, lane);
+                            *reinterpret_cast<uint4 *>(kt + off) = kq;
+                            *reinterpret_cast<uint4 *>(kt + C::kTileBytes + off) = vq;
+                            // fp8 caches: the strides count bytes
+                            const size_t dst = (size_t)outer * p.c_sb + (size_t)mt.kvh * p.c_sh + (size_t)slot * p.c_st + lane * 16;
+                            *reinterpret_cast<uint4 *>(reinterpret_cast<uint8_t *>(p.cache_k) + dst) = kq;
+                            *reinterpret_cast<uint4 *>(reinterpret_cast<uint8_t *>(p.cache_v) + dst) = vq;
+                        }
+                    }
+                    wrote_smem = true;
+                    __syncwarp();
+                }
                 if (nvalid > 0) {
                     // 32 tokens per step: two 16-token blocks share one softmax update. A block with no valid
                     // token is skipped (its rows may never have been fetched); in the last valid block the
@@ -1133,7 +1164,7 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
 {
     if (rope && (!k_new || !v_new || fp8)) return L4L_ERR_UNSUPPORTED;   // only with the fused append, bf16 caches
     // fp8: cache.k / cache.v point at e4m3 bytes, the strides count bytes (= elements)
-    if (fp8 && (D != 128 || k_new || v_new)) return L4L_ERR_UNSUPPORTED;
+    if (fp8 && D != 128) return L4L_ERR_UNSUPPORTED;
     const int esz = fp8 ? 1 : 2;
     // paged: `cache` describes the page pool (stride_b = stride between pages, max_len = page size)
     // hundreds of short sequences: one warp per (sequence, KV head), nothing to merge
@@ -1218,9 +1249,10 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         p.tail_rows = tail_rows;
         p.page_shift = 0;
         while (paged && (1 << p.page_shift) < cache.max_len) ++p.page_shift;
-        // only the fused append (bf16, contiguous) writes through these
-        p.cache_k = static_cast<__nv_bfloat16 *>(cache.k) + ((fp8 || paged) ? 0 : (size_t)b0 * cache.stride_b);
-        p.cache_v = static_cast<__nv_bfloat16 *>(cache.v) + ((fp8 || paged) ? 0 : (size_t)b0 * cache.stride_b);
+        // only the fused append writes through these: the slice's sequences, or the whole pool of a paged cache
+        const size_t base_bytes = paged ? 0 : (size_t)b0 * cache.stride_b * esz;
+        p.cache_k = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(cache.k) + base_bytes);
+        p.cache_v = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(cache.v) + base_bytes);
         p.c_sb = cache.stride_b; p.c_sh = cache.stride_h; p.c_st = cache.stride_t;
         if (k_new && v_new) {
             if (k_new->stride_b != v_new->stride_b || k_new->stride_h != v_new->stride_h) return L4L_ERR_UNSUPPORTED;

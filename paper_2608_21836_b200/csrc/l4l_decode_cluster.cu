@@ -19,6 +19,7 @@
 #include <cstdlib>
 #include <mutex>
 
+#include "l4l_fp8_quant.cuh"
 #include "l4l_internal.h"
 #include "l4l_rope_frag.cuh"
 #include "l4l_warp_attn.cuh"
@@ -319,6 +320,36 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                 __syncwarp();
             }
             if constexpr (F8) {
+                if (p.k_new != nullptr && nvalid > 0 && nvalid <= 16 * C::kSub) {
+                    // fused append into an fp8 cache: the newest token's K/V rows are quantised here exactly as the
+                    // cache update quantises them (same division, same rounding), patched into the tile and written
+                    // to their cache slot; 8 lanes, 16 values each
+                    const int last = row0 + nvalid - 1;
+                    if (lane < 8) {
+                        const size_t src = (size_t)b * p.new_sb + (size_t)kvh * p.new_sh + lane * 16;
+                        const uint4 *ks = reinterpret_cast<const uint4 *>(p.k_new + src);
+                        const uint4 *vs = reinterpret_cast<const uint4 *>(p.v_new + src);
+                        const uint4 kq = quantise16(__ldg(ks), __ldg(ks + 1), k_sc);
+                        const uint4 vq = quantise16(__ldg(vs), __ldg(vs + 1), v_sc);
+                        long long outer = b, slot = len - 1;
+                        if (p.block_table != nullptr) {
+                            outer = __ldg(p.block_table + (size_t)b * p.table_stride + (slot >> p.page_shift));
+                            slot &= p.page_size - 1;
+                        }
+                        if (p.block_table == nullptr || (outer >= 0 && outer < p.num_pages)) {
+                            uint8_t *kt = stages + (size_t)s * C::kStageBytes;
+                            const uint32_t off = swz128(last, lane);
+                            *reinterpret_cast<uint4 *>(kt + off) = kq;
+                            *reinterpret_cast<uint4 *>(kt + C::kTileBytes + off) = vq;
+                            // fp8 caches: the strides count bytes
+                            const size_t dst = (size_t)outer * p.c_sb + (size_t)kvh * p.c_sh + (size_t)slot * p.c_st + lane * 16;
+                            *reinterpret_cast<uint4 *>(reinterpret_cast<uint8_t *>(p.cache_k) + dst) = kq;
+                            *reinterpret_cast<uint4 *>(reinterpret_cast<uint8_t *>(p.cache_v) + dst) = vq;
+                        }
+                    }
+                    wrote_smem = true;
+                    __syncwarp();
+                }
                 if (nvalid > 0) {
                     // 32 tokens per step: two 16-token blocks share one softmax update. A block with no valid token is
                     // skipped (its rows may never have been fetched); in the last valid block the tokens past the end
@@ -643,7 +674,7 @@ l4l_status launch_decode_cluster(const void *q, void *o, const l4l_kv_cache &cac
                                  const Fp8Scales *fp8, int width)
 {
     if (rope && (!k_new || !v_new)) return L4L_ERR_UNSUPPORTED;               // only with the fused append
-    if (fp8 && (D != 128 || k_new || v_new || rope)) return L4L_ERR_UNSUPPORTED;
+    if (fp8 && (D != 128 || rope)) return L4L_ERR_UNSUPPORTED;
     // fp8: cache.k / cache.v point at e4m3 bytes, the strides count bytes (= elements)
     const int esz = fp8 ? 1 : 2, box_d = fp8 ? 128 : 64;
     const int G = Hq / Hkv;

@@ -1,8 +1,7 @@
 // Cache update for an fp8 (e4m3) KV cache: the new tokens' bf16 K and V rows are divided by the scale
 // of their KV head and rounded to e4m3 (nearest even, saturating at +-448) on the way into the cache.
 // One thread turns 16 bf16 values of a K row and of the matching V row into 16 bytes each.
-#include <cuda_fp8.h>
-
+#include "l4l_fp8_quant.cuh"
 #include "l4l_internal.h"
 #include "l4l_ptx.cuh"
 
@@ -19,28 +18,6 @@ struct AppendFp8Params {
     const float *k_scale, *v_scale;  // [Hkv]
     int B, T, Hkv, pieces, max_len;
 };
-
-// 8 bf16 values / scale -> 8 e4m3 bytes (two 32-bit words). The quotient is an IEEE fp32 division, so
-// the stored code is RN_e4m3(RN_fp32(x / scale)) exactly.
-__device__ __forceinline__ uint2 quantise8(const uint4 &v, float scale)
-{
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-    uint32_t out[2];
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-        uint32_t packed = 0;
-#pragma unroll
-        for (int j = 0; j < 2; ++j) {
-            const uint32_t word = w[2 * i + j];
-            const float lo = __fdiv_rn(__uint_as_float(word << 16), scale);
-            const float hi = __fdiv_rn(__uint_as_float(word & 0xffff0000u), scale);
-            const uint32_t two = __nv_cvt_float2_to_fp8x2(make_float2(lo, hi), __NV_SATFINITE, __NV_E4M3);
-            packed |= (two & 0xffffu) << (16 * j);
-        }
-        out[i] = packed;
-    }
-    return make_uint2(out[0], out[1]);
-}
 
 __global__ void __launch_bounds__(256) kv_append_fp8_kernel(const AppendFp8Params p)
 {

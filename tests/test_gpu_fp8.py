@@ -152,3 +152,92 @@ def test_fp8_paged_decode_matches_oracle(page):
     torch.cuda.synchronize()
     assert l4l.l4l_last_device_error(ws) == 0
     assert_close_to_oracle(o.cpu(), ref, f"fp8 paged decode, page {page}")
+
+
+# ---- the decode step that appends the newest token to the fp8 cache itself ----
+
+def _fp8_append_case(Hq, Hkv, lens, seed, page=None, Lmax=2304):
+    """Reference = the oracle's fp8 append at slot kv_len - 1 followed by its fp8 decode; the codes in the cache must
+    come back bit for bit. With `page`, the cache is a page pool behind a shuffled block table."""
+    D = 128
+    B = len(lens)
+    g = torch.Generator().manual_seed(seed)
+    ck8 = random_codes((B, Hkv, Lmax, D), g, 7)
+    cv8 = random_codes((B, Hkv, Lmax, D), g, 7)
+    for b, L in enumerate(lens):                             # the new token's slot and everything after it: NaN codes
+        ck8[b, :, max(L - 1, 0):] = 0x7F
+        cv8[b, :, max(L - 1, 0):] = 0xFF
+    q = torch.randn(B, Hq, D, generator=g).to(torch.bfloat16)
+    kn = (torch.randn(B, 1, Hkv, D, generator=g) * 0.7).to(torch.bfloat16)
+    vn = (torch.randn(B, 1, Hkv, D, generator=g) * 0.7).to(torch.bfloat16)
+    ks, vs = torch.rand(Hkv, generator=g) + 0.5, torch.rand(Hkv, generator=g) + 0.25
+    scale = 1.0 / math.sqrt(D)
+    kv = np.array(lens, np.int32)
+    pos, n_new = np.maximum(kv - 1, 0), (kv > 0).astype(np.int32)
+    ref_k, ref_v = orc.kv_append_fp8(ck8, cv8, kn, vn, pos, n_new, ks.numpy(), vs.numpy())
+    ref, ref_lse = orc.decode_fp8(q, ref_k, ref_v, kv, ks.numpy(), vs.numpy(), scale)
+    go = Guarded(torch.zeros(B, Hq, D, dtype=torch.bfloat16))
+    lse = torch.zeros(B, Hq, device="cuda")
+    ws = l4l.new_workspace(l4l.L4L_OP_DECODE, B, Hq, Hkv, D, Lmax)
+    if page is None:
+        gk, gv = Guarded(ck8), Guarded(cv8)
+        l4l.l4l_attn_decode_append_fp8(q.cuda(), go.t, gk.t, gv.t, ks.cuda(), vs.cuda(), kn.cuda(), vn.cuda(),
+                                       torch.from_numpy(kv).cuda(), Lmax, scale, ws, lse=lse)
+        torch.cuda.synchronize()
+        got_k, got_v = gk.t.cpu().numpy(), gv.t.cpu().numpy()
+        assert gk.margins_intact() and gv.margins_intact()
+    else:
+        per = Lmax // page
+        n_pages = B * per + 3
+        perm = torch.randperm(n_pages, generator=g)[:B * per].view(B, per)
+        pool_k = torch.full((n_pages, Hkv, page, D), 0x7F, dtype=torch.uint8)
+        pool_v = torch.full((n_pages, Hkv, page, D), 0xFF, dtype=torch.uint8)
+        for b in range(B):
+            for i in range(per):
+                pool_k[perm[b, i]] = ck8[b, :, i * page:(i + 1) * page]
+                pool_v[perm[b, i]] = cv8[b, :, i * page:(i + 1) * page]
+        gk, gv = Guarded(pool_k), Guarded(pool_v)
+        l4l.l4l_attn_decode_append_fp8(q.cuda(), go.t, gk.t, gv.t, ks.cuda(), vs.cuda(), kn.cuda(), vn.cuda(),
+                                       torch.from_numpy(kv).cuda(), Lmax, scale, ws, lse=lse,
+                                       block_table=perm.to(torch.int32).cuda())
+        torch.cuda.synchronize()
+        assert gk.margins_intact() and gv.margins_intact()
+        pk, pv = gk.t.cpu(), gv.t.cpu()
+        got_k = torch.stack([torch.cat([pk[perm[b, i]] for i in range(per)], dim=1) for b in range(B)]).numpy()
+        got_v = torch.stack([torch.cat([pv[perm[b, i]] for i in range(per)], dim=1) for b in range(B)]).numpy()
+    assert l4l.l4l_last_device_error(ws) == 0
+    assert go.margins_intact()
+    assert np.array_equal(got_k, ref_k) and np.array_equal(got_v, ref_v)
+    assert_close_to_oracle(go.t.cpu(), ref, "fp8 decode + append")
+    fin = np.isfinite(ref_lse)
+    assert np.abs(lse.cpu().double().numpy()[fin] - ref_lse[fin]).max() <= 2e-3
+    assert (lse.cpu().numpy()[~fin] == -np.inf).all()
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(32, 8), (8, 8), (16, 2), (64, 8)])
+def test_fp8_decode_with_fused_append(Hq, Hkv):
+    # the new token at the start, in the middle and at the end of 32-token steps and 256-token tiles; an empty sequence
+    lens = [1, 2, 16, 17, 32, 33, 255, 256, 257, 700, 1024, 2049, 2304, 0, 333]
+    _fp8_append_case(Hq, Hkv, lens, seed=3000 + Hq)
+
+
+@pytest.mark.parametrize("page", [16, 64, 256])
+def test_fp8_paged_decode_with_fused_append(page):
+    lens = [1, 17, 255, 256, 257, 1500, 0, 640, 2304]
+    _fp8_append_case(16, 4, lens, seed=3100 + page, page=page)
+
+
+@pytest.mark.parametrize("width", [1, 2, 8])
+def test_fp8_fused_append_on_the_cluster_kernel(width):
+    import os
+
+    old = os.environ.get("L4L_DECODE_CLUSTER")
+    os.environ["L4L_DECODE_CLUSTER"] = str(width)
+    try:
+        _fp8_append_case(8, 2, [1, 32, 33, 256, 257, 1000, 0, 2304], seed=3200 + width)
+        _fp8_append_case(8, 2, [1, 33, 257, 1000, 0, 2304], seed=3300 + width, page=64)
+    finally:
+        if old is None:
+            os.environ.pop("L4L_DECODE_CLUSTER", None)
+        else:
+            os.environ["L4L_DECODE_CLUSTER"] = old
