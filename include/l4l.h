@@ -408,6 +408,15 @@ l4l_status l4l_attn_decode_static(const void *q, void *o, l4l_kv_cache cache,
 const char *l4l_status_string(l4l_status status);
 
 /*
+ * Which kernel the decode entry points would run for these sizes on the current device, without launching
+ * anything (for tests and tuning): 0 = the split kernel (*detail = consumer warps per CTA), 1 = the cluster
+ * kernel (*detail = CTAs per cluster), 2 = the warp-per-unit kernel, -1 = sizes the decode calls reject.
+ * fp8: non-zero for an e4m3 cache. detail may be NULL. The environment overrides that the library reads
+ * (L4L_DECODE_CLUSTER, L4L_DECODE_WARP, L4L_DECODE_WARPS: debugging aids) are honoured here as there.
+ */
+int l4l_decode_kernel_choice(int B, int Hq, int Hkv, int head_dim, int max_kv_len, int fp8, int *detail);
+
+/*
  * Synchronises `stream`, reads the workspace's status block and returns 0 if no bounded wait
  * has run out since the last l4l_workspace_init(), else a non-zero code identifying the wait
  * (bit 0: decode pipeline, bit 1: prefill pipeline). Returns -1 if the read itself fails.

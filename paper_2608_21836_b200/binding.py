@@ -26,6 +26,7 @@ EXPORTS = (
     "l4l_kv_append_paged", "l4l_attn_decode_paged", "l4l_kv_append_fp8", "l4l_attn_decode_fp8", "l4l_rglru_scan", "l4l_rglru_workspace_bytes",
     "l4l_attn_decode_paged_fp8", "l4l_attn_merge", "l4l_attn_decode_rope_append", "l4l_attn_decode_paged_append",
     "l4l_attn_decode_paged_rope_append", "l4l_attn_decode_append_fp8", "l4l_attn_decode_paged_append_fp8",
+    "l4l_decode_kernel_choice",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -103,6 +104,8 @@ def load() -> ctypes.CDLL:
     lib.l4l_attn_decode_paged_append_fp8.restype = c_int
     lib.l4l_attn_decode_paged_append_fp8.argtypes = [vp, vp, PagedKV, vp, vp, i32p, c_int, Tensor4, Tensor4, i32p, c_int,
                                                      c_int, c_int, c_int, c_int, ctypes.c_float, vp, vp, c_size, vp]
+    lib.l4l_decode_kernel_choice.restype = c_int
+    lib.l4l_decode_kernel_choice.argtypes = [c_int, c_int, c_int, c_int, c_int, c_int, ctypes.POINTER(c_int)]
     lib.l4l_kv_append_fp8.restype = c_int
     lib.l4l_kv_append_fp8.argtypes = [KVCache, Tensor4, Tensor4, i32p, i32p, c_int, c_int, c_int, c_int, vp, vp, vp]
     lib.l4l_attn_decode_fp8.restype = c_int
@@ -554,6 +557,14 @@ def l4l_attn_decode_append_fp8(q, o, cache_k8, cache_v8, k_scale, v_scale, k_new
         st = load().l4l_attn_decode_paged_append_fp8(q.data_ptr(), o.data_ptr(), pool, ks, vs, tbl, stride, *common)
     if st != L4L_OK:
         raise L4LError(st, "l4l_attn_decode_append_fp8")
+
+
+def l4l_decode_kernel_choice(B: int, Hq: int, Hkv: int, D: int, max_kv_len: int, fp8: bool = False):
+    """(name, detail) of the kernel the decode calls would run for these sizes on the current device: ("split", consumer
+    warps), ("cluster", CTAs per cluster) or ("warp", 0); None for sizes the calls reject."""
+    detail = ctypes.c_int(0)
+    k = load().l4l_decode_kernel_choice(B, Hq, Hkv, D, int(max_kv_len), int(bool(fp8)), ctypes.byref(detail))
+    return None if k < 0 else (("split", "cluster", "warp")[k], detail.value)
 
 
 def l4l_attn_merge(o_parts, lse_parts, o, lse=None) -> None:

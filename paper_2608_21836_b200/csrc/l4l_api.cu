@@ -583,4 +583,20 @@ l4l_status l4l_attn_decode_paged_rope_append(const void *q, void *o, l4l_paged_k
                          plan, static_cast<cudaStream_t>(stream), &k_new, &v_new, &pt, nullptr, &rope);
 }
 
+int l4l_decode_kernel_choice(int B, int Hq, int Hkv, int head_dim, int max_kv_len, int fp8, int *detail)
+{
+    if (detail) *detail = 0;
+    if (shape_status(B, Hq, Hkv, head_dim) != L4L_OK || B == 0 || max_kv_len < 0 || (fp8 && head_dim != 128)) return -1;
+    // the order launch_decode asks in
+    if (decode_warp_eligible(B, Hq, Hkv, head_dim, max_kv_len, fp8 != 0, false)) return 2;
+    const int width = decode_cluster_width(B, Hq, Hkv, head_dim, max_kv_len, fp8 != 0);
+    if (width > 0) {
+        if (detail) *detail = width;
+        return 1;
+    }
+    const DecodePlan plan = plan_decode(B, Hq, Hkv, head_dim, max_kv_len, ~(size_t)0, fp8 != 0);
+    if (detail) *detail = plan.warps;
+    return 0;
+}
+
 }  // extern "C"

@@ -122,3 +122,22 @@ def test_library_picks_the_warp_kernel_for_many_short_sequences(warp_kernel):
     lens = g.integers(1, 257, size=B).tolist()
     q, ck, cv, kv_len = random_batch(B, Hq, Hkv, D, 256, lens, seed=12)
     check_decode(q, ck, cv, kv_len, 1.0 / math.sqrt(D))
+
+
+@pytest.mark.parametrize("warp_kernel", [None], indirect=True)
+def test_kernel_choice_by_problem_size(warp_kernel):
+    """The three decode kernels and the regimes the library gives them (8B-shaped layer: 32 query heads on 8 KV heads)."""
+    old = os.environ.pop("L4L_DECODE_CLUSTER", None)
+    try:
+        assert l4l.l4l_decode_kernel_choice(1, 32, 8, 128, 2304) == ("cluster", 8)          # one sequence: latency-bound
+        assert l4l.l4l_decode_kernel_choice(4, 32, 8, 128, 2304)[0] == "cluster"
+        assert l4l.l4l_decode_kernel_choice(32, 32, 8, 128, 4096) == ("split", 8)            # the benchmark batch
+        assert l4l.l4l_decode_kernel_choice(64, 12, 12, 64, 1024) == ("split", 4)            # small MHA model
+        assert l4l.l4l_decode_kernel_choice(512, 32, 8, 128, 256) == ("warp", 0)             # hundreds of short sequences
+        assert l4l.l4l_decode_kernel_choice(512, 32, 8, 128, 4096)[0] == "split"             # ... but not long ones
+        assert l4l.l4l_decode_kernel_choice(512, 32, 8, 128, 256, fp8=True)[0] == "split"    # fp8: not on the warp kernel
+        assert l4l.l4l_decode_kernel_choice(32, 128, 8, 128, 4096) == ("split", 6)           # groups of 16 query heads
+        assert l4l.l4l_decode_kernel_choice(1, 32, 8, 96, 128) is None                       # unsupported head_dim
+    finally:
+        if old is not None:
+            os.environ["L4L_DECODE_CLUSTER"] = old
