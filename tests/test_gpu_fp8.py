@@ -241,3 +241,10 @@ def test_fp8_fused_append_on_the_cluster_kernel(width):
             os.environ.pop("L4L_DECODE_CLUSTER", None)
         else:
             os.environ["L4L_DECODE_CLUSTER"] = old
+
+
+def test_fp8_fused_append_batch_of_several_launch_slices():
+    g = np.random.default_rng(23)
+    lens = g.integers(0, 300, size=420).tolist()             # more than the 384 sequences of one launch
+    _fp8_append_case(8, 2, lens, seed=3400, Lmax=320)
+    _fp8_append_case(8, 2, lens, seed=3401, page=32, Lmax=320)

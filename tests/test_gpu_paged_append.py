@@ -157,3 +157,21 @@ def test_paged_decode_rope_append_matches_oracle_chain(kernel_choice, page, Hq, 
         assert_close_to_oracle(o.cpu(), ref, f"paged rope + append + decode, step {s}")
     assert_bf16_close(dpk, opk, "pool k after the fused steps")
     assert np.array_equal(orc.bits(dpv.cpu()), opv)
+
+
+# ---- batches larger than one launch slice (384 sequences on the split kernel, 1024 on the warp-per-unit kernel) ----
+
+@pytest.mark.parametrize("kernel_choice", [None], indirect=True)
+def test_paged_decode_append_batch_of_several_launch_slices_split_kernel(kernel_choice):
+    g = np.random.default_rng(21)
+    lens = g.integers(0, 700, size=450).tolist()             # longer than the warp-per-unit kernel's regime
+    assert l4l.l4l_decode_kernel_choice(len(lens), 8, 2, 128, max(lens))[0] == "split"
+    run_case(len(lens), 8, 2, 128, 64, lens, seed=515)
+
+
+@pytest.mark.parametrize("kernel_choice", [None], indirect=True)
+def test_paged_decode_append_batch_of_several_launch_slices_warp_kernel(kernel_choice):
+    g = np.random.default_rng(22)
+    lens = g.integers(0, 120, size=1100).tolist()
+    assert l4l.l4l_decode_kernel_choice(len(lens), 8, 2, 128, max(lens))[0] == "warp"
+    run_case(len(lens), 8, 2, 128, 16, lens, seed=516)
