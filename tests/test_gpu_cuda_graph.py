@@ -96,3 +96,55 @@ def test_prefill_in_a_cuda_graph():
     assert l4l.l4l_last_device_error(ws) == 0
     valid = torch.arange(S).view(1, S) < torch.tensor([S, 77]).view(B, 1)
     assert_close_to_oracle(o.cpu()[valid], ref[valid.numpy()], "prefill in a graph")
+
+
+def test_fused_decode_steps_of_many_short_sequences_in_a_cuda_graph():
+    """The warp-per-unit kernel (hundreds of short sequences) with the fused append, captured once and replayed over
+    four growing steps: lengths, queries and new tokens change in place between replays."""
+    B, Hq, Hkv, D, Lmax = 160, 8, 4, 128, 128
+    g = torch.Generator().manual_seed(12)
+    rng = np.random.default_rng(12)
+    ck = torch.randn(B, Hkv, Lmax, D, generator=g).to(torch.bfloat16)
+    cv = torch.randn(B, Hkv, Lmax, D, generator=g).to(torch.bfloat16)
+    cur = rng.integers(0, 100, size=B).astype(np.int32)        # tokens cached so far
+    dck, dcv = ck.cuda(), cv.cuda()
+    q = torch.zeros(B, Hq, D, dtype=torch.bfloat16, device="cuda")
+    kn = torch.zeros(B, 1, Hkv, D, dtype=torch.bfloat16, device="cuda")
+    vn = torch.zeros_like(kn)
+    lens = torch.zeros(B, dtype=torch.int32, device="cuda")
+    o = torch.zeros_like(q)
+    ws = l4l.new_workspace(l4l.L4L_OP_DECODE, B, Hq, Hkv, D, Lmax)
+    scale = 1.0 / math.sqrt(D)
+    if l4l.l4l_decode_kernel_choice(B, Hq, Hkv, D, Lmax)[0] != "warp":      # held on another kernel by the environment
+        pytest.skip("the warp-per-unit kernel is not the library's choice under this setting")
+
+    def step():
+        l4l.l4l_attn_decode_append(q, o, dck, dcv, kn, vn, lens, Lmax, scale, ws)
+
+    ref_k, ref_v = orc.bits(ck).copy(), orc.bits(cv).copy()
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        lens.copy_(torch.from_numpy(cur + 1))
+        step()                                                  # warm-up: appends zeros at `cur`
+    torch.cuda.current_stream().wait_stream(s)
+    torch.cuda.synchronize()
+    zeros = torch.zeros(B, 1, Hkv, D).to(torch.bfloat16)
+    ref_k, ref_v = orc.kv_append(ref_k, ref_v, zeros, zeros, cur, np.ones(B, np.int32))
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    for it in range(4):
+        qi = torch.randn(B, Hq, D, generator=g).to(torch.bfloat16)
+        ki = torch.randn(B, 1, Hkv, D, generator=g).to(torch.bfloat16)
+        vi = torch.randn(B, 1, Hkv, D, generator=g).to(torch.bfloat16)
+        q.copy_(qi); kn.copy_(ki); vn.copy_(vi)
+        lens.copy_(torch.from_numpy(cur + 1))
+        graph.replay()
+        torch.cuda.synchronize()
+        ref_k, ref_v = orc.kv_append(ref_k, ref_v, ki, vi, cur, np.ones(B, np.int32))
+        ref, _ = orc.decode(qi, ref_k, ref_v, cur + 1, scale)
+        assert_close_to_oracle(o.cpu(), ref, f"graph replay {it}")
+        cur = cur + 1
+    assert l4l.l4l_last_device_error(ws) == 0
+    assert np.array_equal(orc.bits(dck.cpu()), ref_k) and np.array_equal(orc.bits(dcv.cpu()), ref_v)
