@@ -508,6 +508,12 @@ def test_paged_decode_is_decode_over_the_pages_laid_end_to_end():
     ck2, cv2 = orc.kv_append(ck, cv, k_new, v_new, pos, np.array([2, 3, 3], np.int32))
     assert np.array_equal(orc.gather_pages(pk2, perm, Lmax), ck2)
     assert np.array_equal(orc.gather_pages(pv2, perm, Lmax), cv2)
+    # a slot whose table entry names no page of the pool is dropped: the pools come back untouched for that sequence
+    perm3 = perm.copy()
+    perm3[1, 7 // page] = -1
+    perm3[2, 1 // page] = n_pages
+    pk3, pv3 = orc.kv_append_paged(pool_k, pool_v, perm3, k_new[:, :1], v_new[:, :1], pos, np.array([0, 1, 1], np.int32))
+    assert np.array_equal(pk3, orc.bits(pool_k)) and np.array_equal(pv3, orc.bits(pool_v))
 
 
 # --------------------------------------------------------------------------- fp8 (e4m3) cache
