@@ -3,7 +3,8 @@
 // piece of a sequence (query rows, hand-over, finisher); with hundreds of sequences of a few hundred tokens
 // that cost is paid every tile or two and the kernel falls to a third of the HBM rate.
 //
-// Persistent CTAs of 8 or 12 warps. The (sequence, KV head) units are laid end to end in 16-token chunks; a CTA
+// Persistent CTAs of 4 to 12 warps (the fewer units per SM, the fewer warps and the deeper their rings). The
+// (sequence, KV head) units are laid end to end in 16-token chunks; a CTA
 // takes the units that START inside its equal share of that stream (whole units only), puts them in order of
 // descending length and hands them to its warps through a counter in shared memory, longest first, so that the
 // warps of a CTA finish together. A warp moves its chunks from the cache into a private ring in
