@@ -355,6 +355,13 @@ def run_ours(args, rank, world):
         l4l.l4l_attn_decode_paged(dq, do, pk_i, pv_i, tbl_i, dlen, Lmax, wd.scale, ws_d)
 
     t_paged = timed(paged_step, 21)
+
+    def paged_fused_step():                                   # the same with the cache update of the step fused in
+        pk_i, pv_i, tbl_i = pools[rot[0] % 3]
+        rot[0] += 1
+        l4l.l4l_attn_decode_paged_append(dq, do, pk_i, pv_i, tbl_i, dkn, dvn, dlen, Lmax, wd.scale, ws_d)
+
+    t_paged_fused = timed(paged_fused_step, 21)
     del pools
     # decode over an fp8 (e4m3) cache: the same batch quantised by the library's own append (N(0,1) data, 4.5 sigma
     # at full scale), three copies in rotation
@@ -374,6 +381,13 @@ def run_ours(args, rank, world):
         l4l.l4l_attn_decode_fp8(dq, do, k8, v8, k_sc, k_sc, dlen, Lmax, wd.scale, ws_d)
 
     t_fp8 = timed(fp8_step, 21)
+
+    def fp8_fused_step():                                     # the new token quantised and appended in the same launch
+        k8, v8 = c8[rot[0] % 3]
+        rot[0] += 1
+        l4l.l4l_attn_decode_append_fp8(dq, do, k8, v8, k_sc, k_sc, dkn, dvn, dlen, Lmax, wd.scale, ws_d)
+
+    t_fp8_fused = timed(fp8_fused_step, 21)
     del c8
     # the same cache with 64 query heads on the 8 KV heads (groups of 8: the 70B-class shape), three copies in rotation
     Hq8 = 8 * Hkv
@@ -625,7 +639,8 @@ def run_ours(args, rank, world):
             "prefill_from_cache": {"ms": t_chunk, "tflops": pre_flops / (t_chunk * 1e-3) / 1e12},
             "decode_with_fused_append": {"us": t_fused * 1e3, "kv_gbs": dec_bytes / (t_fused * 1e-3) / 1e9},
             "decode_step_rope_norm_append_attention": {"one_launch_us": t_step1 * 1e3, "two_launches_us": t_step3 * 1e3},
-            "decode_paged_64": {"us": t_paged * 1e3, "kv_gbs": dec_bytes / (t_paged * 1e-3) / 1e9},
+            "decode_paged_64": {"us": t_paged * 1e3, "kv_gbs": dec_bytes / (t_paged * 1e-3) / 1e9,
+                                "with_fused_append_us": t_paged_fused * 1e3},
             "rglru_scan_B4_T8192_W2560": {"us": t_rglru * 1e3, "gbs": rglru_bytes / (t_rglru * 1e-3) / 1e9,
                                           "frac_of_measured_hbm": rglru_bytes / (t_rglru * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                           "bytes": rglru_bytes},
@@ -633,7 +648,7 @@ def run_ours(args, rank, world):
                                            "frac_of_measured_hbm": rglru_bytes / (t_rglru2 * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                            "bytes": rglru_bytes},
             "decode_fp8_cache": {"us": t_fp8 * 1e3, "kv_gbs_fp8_bytes": dec_bytes / 2 / (t_fp8 * 1e-3) / 1e9,
-                                 "speedup_over_bf16_cache": t_dec_b2b / t_fp8},
+                                 "speedup_over_bf16_cache": t_dec_b2b / t_fp8, "with_fused_append_us": t_fp8_fused * 1e3},
             "decode_64_query_heads_on_8_kv_heads": {"us": t_g8 * 1e3, "kv_gbs": dec_bytes / (t_g8 * 1e-3) / 1e9},
             "other_configs": other,
             "decode_B512_L64_to_256": {"warp_kernel_us": t_short * 1e3, "kv_gbs": short_bytes / (t_short * 1e-3) / 1e9,
