@@ -141,3 +141,43 @@ def test_kernel_choice_by_problem_size(warp_kernel):
     finally:
         if old is not None:
             os.environ["L4L_DECODE_CLUSTER"] = old
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_warp_decode_random_shapes(warp_kernel, seed):
+    """Seeded random shapes, length mixes, page sizes and group sizes through the warp-per-unit kernel (forced on),
+    without and with the fused append: a net for the index arithmetic of its unit queue and rings."""
+    from test_gpu_random_shapes import random_lengths
+    from test_gpu_paged import build_pool
+
+    rng = np.random.default_rng(7000 + seed)
+    D = int(rng.choice([64, 128]))
+    Hkv = int(rng.choice([1, 2, 3, 8]))
+    G = int(rng.choice([1, 2, 4, 5, 8, 12, 16]))
+    Hq = Hkv * G
+    B = int(rng.choice([1, 2, 9, 40, 150, 700]))
+    Lmax = int(rng.choice([48, 96, 300, 700]))
+    lens = random_lengths(rng, B, Lmax)
+    q, ck, cv, kv_len = random_batch(B, Hq, Hkv, D, Lmax, lens.tolist(), seed=seed)
+    scale = float(rng.choice([1.0 / math.sqrt(D), 0.05, -0.03]))
+    check_decode(q, ck, cv, kv_len, scale)
+    # fused append over a paged copy of the same lengths (the new token is the last one of every sequence)
+    page = int(rng.choice([16, 32, 64, 128]))
+    g = torch.Generator().manual_seed(100 + seed)
+    pool_k, pool_v, table = build_pool(B, Hkv, D, page, lens.tolist(), seed=200 + seed)
+    kn = torch.randn(B, 1, Hkv, D, generator=g).to(torch.bfloat16)
+    vn = torch.randn(B, 1, Hkv, D, generator=g).to(torch.bfloat16)
+    pos = np.maximum(lens - 1, 0)
+    ref_k, ref_v = orc.kv_append_paged(pool_k, pool_v, table, kn, vn, pos, (lens > 0).astype(np.int32))
+    ref, _ = orc.decode_paged(q, ref_k, ref_v, table, lens, scale)
+    gk, gv = Guarded(pool_k), Guarded(pool_v)
+    o = torch.zeros(B, Hq, D, dtype=torch.bfloat16, device="cuda")
+    max_len = max(int(lens.max()), 1)
+    ws = l4l.new_workspace(l4l.L4L_OP_DECODE, B, Hq, Hkv, D, max_len)
+    l4l.l4l_attn_decode_paged_append(q.cuda(), o, gk.t, gv.t, torch.from_numpy(table).cuda(), kn.cuda(), vn.cuda(),
+                                     torch.from_numpy(lens).cuda(), max_len, scale, ws)
+    torch.cuda.synchronize()
+    assert l4l.l4l_last_device_error(ws) == 0
+    assert gk.margins_intact() and gv.margins_intact()
+    assert np.array_equal(orc.bits(gk.t.cpu()), ref_k) and np.array_equal(orc.bits(gv.t.cpu()), ref_v)
+    assert_close_to_oracle(o.cpu(), ref, f"paged decode + append, seed {seed}")
