@@ -588,7 +588,7 @@ int l4l_decode_kernel_choice(int B, int Hq, int Hkv, int head_dim, int max_kv_le
     if (detail) *detail = 0;
     if (shape_status(B, Hq, Hkv, head_dim) != L4L_OK || B == 0 || max_kv_len < 0 || (fp8 && head_dim != 128)) return -1;
     // the order launch_decode asks in
-    if (decode_warp_eligible(B, Hq, Hkv, head_dim, max_kv_len, fp8 != 0, false)) return 2;
+    if (decode_warp_eligible(B, Hq, Hkv, head_dim, max_kv_len, fp8 != 0, false, false)) return 2;
     const int width = decode_cluster_width(B, Hq, Hkv, head_dim, max_kv_len, fp8 != 0);
     if (width > 0) {
         if (detail) *detail = width;

@@ -1168,9 +1168,9 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
     const int esz = fp8 ? 1 : 2;
     // paged: `cache` describes the page pool (stride_b = stride between pages, max_len = page size)
     // hundreds of short sequences: one warp per (sequence, KV head), nothing to merge
-    if (decode_warp_eligible(B, Hq, Hkv, D, max_kv_len, fp8 != nullptr, rope != nullptr))
+    if (decode_warp_eligible(B, Hq, Hkv, D, max_kv_len, fp8 != nullptr, rope != nullptr, k_new != nullptr))
         return launch_decode_warp(q, o, cache, d_kv_lens, max_kv_len, B, Hq, Hkv, D, scale, d_lse, stream, k_new, v_new,
-                                  paged);
+                                  paged, fp8);
     {
         // small batches are latency-bound: one cluster per (sequence, KV head), no workspace round trips
         const int width = decode_cluster_width(B, Hq, Hkv, D, max_kv_len, fp8 != nullptr);

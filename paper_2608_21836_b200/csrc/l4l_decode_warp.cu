@@ -11,7 +11,8 @@
 // shared memory with 16-byte asynchronous copies (cp.async: no barrier objects, no descriptors, rows past the
 // end of a sequence arrive as zeros), in the 128-byte-swizzled layout that the warp-level MMA blocks expect, and
 // stays S - 1 chunks ahead of its own arithmetic, across unit boundaries (the query rows of a unit travel with
-// the unit's first chunk). Contiguous or paged caches; optional fused append of the step's newest token.
+// the unit's first chunk). Contiguous or paged caches, bf16 or fp8 (e4m3, per-KV-head scales); optional fused
+// append of the step's newest token (bf16 caches).
 #include <cstdlib>
 #include <mutex>
 
@@ -40,22 +41,24 @@ struct WarpParams {
     int64_t c_sb, c_sh, c_st;
     const int32_t *block_table;           // paged cache (null: contiguous)
     int table_stride, page_size, page_shift, num_pages;
+    const float *k_scale, *v_scale;       // fp8 cache: real value = e4m3 value * scale of its KV head, [Hkv]
     int B, Hq, Hkv, G, max_kv_len, stages;
     float scale_log2e;
 };
 
-template <int D>
+template <int D, bool F8>
 struct WarpCfg {
-    static constexpr int kHalves = D / 64;                            // 128-byte column blocks of a row
+    static constexpr int kRowBytes = F8 ? D : 2 * D;                  // one token of one KV head
+    static constexpr int kHalves = kRowBytes / 128;                   // 128-byte column blocks of a row
     static constexpr uint32_t kHalfBytes = kChunkT * 128;             // [16 tokens][128 bytes], swizzled
     static constexpr uint32_t kTileBytes = kHalves * kHalfBytes;      // K or V of one chunk
-    static constexpr int kRowPieces = D / 8;                          // 16-byte pieces per row
+    static constexpr int kRowPieces = kRowBytes / 16;                 // 16-byte pieces per row
     static constexpr int kCopies = kChunkT * kRowPieces / 32;         // cp.async per lane for K (and as many for V)
 };
 
-__host__ __device__ inline size_t stage_bytes(int D, int G)
+__host__ __device__ inline size_t stage_bytes(int D, int G, bool f8)
 {
-    return (size_t)2 * (D / 64) * kChunkT * 128 + (size_t)G * D * 2;    // K, V, the unit's query rows
+    return (size_t)2 * ((f8 ? D : 2 * D) / 128) * kChunkT * 128 + (size_t)G * D * 2;    // K, V, the unit's query rows
 }
 
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void *src, uint32_t src_bytes)
@@ -76,10 +79,12 @@ struct Cursor {
     bool valid;                       // false: the queue is empty
 };
 
-template <int D, int kWarps>
+template <int D, int kWarps, bool F8>
 __global__ void __launch_bounds__(kWarps * 32) decode_warp_kernel(const WarpParams p)
 {
-    using C = WarpCfg<D>;
+    static_assert(!F8 || D == 128, "the fp8 path wants one 128-byte row per token");
+    using C = WarpCfg<D, F8>;
+    constexpr int kEsz = F8 ? 1 : 2;
     constexpr int kThreads = kWarps * 32;
     extern __shared__ __align__(1024) uint8_t smem[];
     int *lens_s = reinterpret_cast<int *>(smem);                 // [kMaxB]
@@ -89,7 +94,7 @@ __global__ void __launch_bounds__(kWarps * 32) decode_warp_kernel(const WarpPara
     int *fifo_s = ctl + 4;                                       // [kWarps][kFifo]
     uint16_t *cnt_s = reinterpret_cast<uint16_t *>(fifo_s + 16 * kFifo);   // [kMaxList] chunks per unit of this CTA
     uint16_t *order_s = cnt_s + kMaxList;                        // [kMaxList] units by descending chunk count
-    const size_t sbytes = stage_bytes(D, p.G);
+    const size_t sbytes = stage_bytes(D, p.G, F8);
     uint8_t *ring_base = smem + kMetaBytes;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     uint8_t *ring = ring_base + (size_t)warp * p.stages * sbytes;
@@ -232,10 +237,12 @@ __global__ void __launch_bounds__(kWarps * 32) decode_warp_kernel(const WarpPara
             have = outer >= 0 && outer < p.num_pages;     // a page outside the pool reads as zeros
             if (!have) outer = 0;
         }
-        const size_t base = (size_t)outer * p.c_sb + (size_t)c.kvh * p.c_sh +
-                            (size_t)(slot_t + row_of_lane) * p.c_st + piece * 8;
-        const __nv_bfloat16 *ks = p.cache_k + base, *vs = p.cache_v + base;
-        const size_t step = (size_t)kRowsPerTrip * p.c_st;
+        // byte addresses: an fp8 cache counts its strides in bytes, a bf16 cache in 2-byte elements
+        const size_t base = ((size_t)outer * p.c_sb + (size_t)c.kvh * p.c_sh + (size_t)(slot_t + row_of_lane) * p.c_st) * kEsz +
+                            piece * 16;
+        const uint8_t *kbase = reinterpret_cast<const uint8_t *>(p.cache_k), *vbase = reinterpret_cast<const uint8_t *>(p.cache_v);
+        const uint8_t *ks = kbase + base, *vs = vbase + base;
+        const size_t step = (size_t)kRowsPerTrip * p.c_st * kEsz;
         const int nval = c.len - t0;               // rows of the chunk that hold tokens
         if (have && (nval > kChunkT || (nval == kChunkT && p.k_new == nullptr))) {
             // a full chunk of cached tokens (all but the last chunk of a unit): no predicates
@@ -257,8 +264,8 @@ __global__ void __launch_bounds__(kWarps * 32) decode_warp_kernel(const WarpPara
                     cp_async_16(k_dst + soff[i], p.k_new + new_off, 16u);
                     cp_async_16(v_dst + soff[i], p.v_new + new_off, 16u);
                 } else {
-                    cp_async_16(k_dst + soff[i], valid ? ks : p.cache_k, valid ? 16u : 0u);
-                    cp_async_16(v_dst + soff[i], valid ? vs : p.cache_v, valid ? 16u : 0u);
+                    cp_async_16(k_dst + soff[i], valid ? ks : kbase, valid ? 16u : 0u);
+                    cp_async_16(v_dst + soff[i], valid ? vs : vbase, valid ? 16u : 0u);
                 }
                 ks += step;
                 vs += step;
@@ -267,7 +274,7 @@ __global__ void __launch_bounds__(kWarps * 32) decode_warp_kernel(const WarpPara
         if (c.chunk == 0) {                        // the unit's query rows: G x D bf16, unswizzled
             const uint32_t q_dst = v_dst + C::kTileBytes;
             const __nv_bfloat16 *qs = p.q + ((size_t)c.b * p.Hq + (size_t)c.kvh * p.G) * D;
-            for (int i = lane; i < p.G * C::kRowPieces; i += 32) cp_async_16_full(q_dst + i * 16, qs + i * 8);
+            for (int i = lane; i < p.G * (D / 8); i += 32) cp_async_16_full(q_dst + i * 16, qs + i * 8);
         }
     };
 
@@ -288,6 +295,7 @@ __global__ void __launch_bounds__(kWarps * 32) decode_warp_kernel(const WarpPara
     st.reset();
     uint32_t qf[D / 16][4];
     const int r_lo = lane >> 2, r_hi = r_lo + 8;
+    float k_sc = 1.f, v_sc = 1.f;                  // fp8 cache: scales of the unit's KV head
     while (live(tail)) {
         if (live(head)) {
             issue(head, head_slot);
@@ -313,17 +321,30 @@ __global__ void __launch_bounds__(kWarps * 32) decode_warp_kernel(const WarpPara
             const bool v_lo = r_lo < p.G, v_hi = r_hi < p.G;
 #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks) {
-                const int w = ks * 8 + (lane & 3);
-                qf[ks][0] = v_lo ? qrow_lo[w] : 0u;
-                qf[ks][1] = v_hi ? qrow_hi[w] : 0u;
-                qf[ks][2] = v_lo ? qrow_lo[w + 4] : 0u;
-                qf[ks][3] = v_hi ? qrow_hi[w + 4] : 0u;
+                if constexpr (F8) {
+                    // f16 fragments with the k index permuted the way the fp8 K rows arrive
+                    const int w = q_frag_f8_word(ks, 0, lane);
+                    qf[ks][0] = v_lo ? bf16x2_to_f16x2(qrow_lo[w]) : 0u;
+                    qf[ks][1] = v_hi ? bf16x2_to_f16x2(qrow_hi[w]) : 0u;
+                    qf[ks][2] = v_lo ? bf16x2_to_f16x2(qrow_lo[w + 1]) : 0u;
+                    qf[ks][3] = v_hi ? bf16x2_to_f16x2(qrow_hi[w + 1]) : 0u;
+                } else {
+                    const int w = ks * 8 + (lane & 3);
+                    qf[ks][0] = v_lo ? qrow_lo[w] : 0u;
+                    qf[ks][1] = v_hi ? qrow_hi[w] : 0u;
+                    qf[ks][2] = v_lo ? qrow_lo[w + 4] : 0u;
+                    qf[ks][3] = v_hi ? qrow_hi[w + 4] : 0u;
+                }
+            }
+            if constexpr (F8) {
+                k_sc = __ldg(p.k_scale + tail.kvh);
+                v_sc = __ldg(p.v_scale + tail.kvh);
             }
         }
         const int t0 = tail.chunk * kChunkT;
         const int nvalid = tail.len - t0;
         if (nvalid > 0) {
-            if (p.k_new != nullptr && nvalid <= kChunkT) {
+            if (!F8 && p.k_new != nullptr && nvalid <= kChunkT) {
                 // fused append: the newest token came from the caller; its cache slot is written from the copy in
                 // shared memory (with pages: behind the block table; no page there: nothing is written)
                 const int row = nvalid - 1;
@@ -347,11 +368,15 @@ __global__ void __launch_bounds__(kWarps * 32) decode_warp_kernel(const WarpPara
                 __syncwarp();
             }
             float s_lo[4], s_hi[4];
-            warp_qk_16x16<D>(qf, k_tile, C::kHalfBytes, 0, s_lo, s_hi);
+            if constexpr (F8)
+                warp_qk_16x16_f8<D>(qf, k_tile, 0, s_lo, s_hi);
+            else
+                warp_qk_16x16<D>(qf, k_tile, C::kHalfBytes, 0, s_lo, s_hi);
+            const float sc = F8 ? p.scale_log2e * k_sc : p.scale_log2e;
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                s_lo[e] *= p.scale_log2e;
-                s_hi[e] *= p.scale_log2e;
+                s_lo[e] *= sc;
+                s_hi[e] *= sc;
             }
             if (nvalid < kChunkT) {                // tokens past the end: no weight (their V rows arrived as zeros)
                 const int tok = 2 * (lane & 3);
@@ -362,8 +387,11 @@ __global__ void __launch_bounds__(kWarps * 32) decode_warp_kernel(const WarpPara
                 }
             }
             uint32_t pa[4];
-            warp_softmax_16<D>(st, s_lo, s_hi, pa);
-            warp_pv_16x16<D>(st, pa, v_tile, C::kHalfBytes, 0);
+            warp_softmax_16<D, F8>(st, s_lo, s_hi, pa);        // fp8: weights as f16 for the f16 MMAs
+            if constexpr (F8)
+                warp_pv_16x16_f8<D>(st, pa, v_tile, 0);
+            else
+                warp_pv_16x16<D>(st, pa, v_tile, C::kHalfBytes, 0);
         }
         if (tail.chunk + 1 == tail.chunks) {
             // ---- the unit is complete: normalise and write its G output rows
@@ -375,19 +403,41 @@ __global__ void __launch_bounds__(kWarps * 32) decode_warp_kernel(const WarpPara
             const bool any = tail.len > 0;
             const float i0 = any ? 1.f / l0 : 0.f, i1 = any ? 1.f / l1 : 0.f;
             const size_t bh = (size_t)tail.b * p.Hq + (size_t)tail.kvh * p.G;
+            // fp8: accumulator tiles alternate even / odd head dims (a tile pair gives this lane 4 consecutive dims) and O
+            // still lacks the V scale of its KV head
             if (r_lo < p.G) {
-                __nv_bfloat16 *row = p.o + (bh + r_lo) * D + 2 * (lane & 3);
+                if constexpr (F8) {
+                    __nv_bfloat16 *row = p.o + (bh + r_lo) * D + 4 * (lane & 3);
+                    const float f = i0 * v_sc;
 #pragma unroll
-                for (int nt = 0; nt < D / 8; ++nt)
-                    *reinterpret_cast<uint32_t *>(row + nt * 8) = pack_bf16x2(st.o[nt][0] * i0, st.o[nt][1] * i0);
+                    for (int ch = 0; ch < D / 16; ++ch)
+                        *reinterpret_cast<uint2 *>(row + ch * 16) =
+                            make_uint2(pack_bf16x2(st.o[2 * ch][0] * f, st.o[2 * ch + 1][0] * f),
+                                       pack_bf16x2(st.o[2 * ch][1] * f, st.o[2 * ch + 1][1] * f));
+                } else {
+                    __nv_bfloat16 *row = p.o + (bh + r_lo) * D + 2 * (lane & 3);
+#pragma unroll
+                    for (int nt = 0; nt < D / 8; ++nt)
+                        *reinterpret_cast<uint32_t *>(row + nt * 8) = pack_bf16x2(st.o[nt][0] * i0, st.o[nt][1] * i0);
+                }
                 if ((lane & 3) == 0 && p.lse)
                     p.lse[bh + r_lo] = any ? (st.m[0] + log2f(l0)) * 0.6931471805599453f : -INFINITY;
             }
             if (r_hi < p.G) {
-                __nv_bfloat16 *row = p.o + (bh + r_hi) * D + 2 * (lane & 3);
+                if constexpr (F8) {
+                    __nv_bfloat16 *row = p.o + (bh + r_hi) * D + 4 * (lane & 3);
+                    const float f = i1 * v_sc;
 #pragma unroll
-                for (int nt = 0; nt < D / 8; ++nt)
-                    *reinterpret_cast<uint32_t *>(row + nt * 8) = pack_bf16x2(st.o[nt][2] * i1, st.o[nt][3] * i1);
+                    for (int ch = 0; ch < D / 16; ++ch)
+                        *reinterpret_cast<uint2 *>(row + ch * 16) =
+                            make_uint2(pack_bf16x2(st.o[2 * ch][2] * f, st.o[2 * ch + 1][2] * f),
+                                       pack_bf16x2(st.o[2 * ch][3] * f, st.o[2 * ch + 1][3] * f));
+                } else {
+                    __nv_bfloat16 *row = p.o + (bh + r_hi) * D + 2 * (lane & 3);
+#pragma unroll
+                    for (int nt = 0; nt < D / 8; ++nt)
+                        *reinterpret_cast<uint32_t *>(row + nt * 8) = pack_bf16x2(st.o[nt][2] * i1, st.o[nt][3] * i1);
+                }
                 if ((lane & 3) == 0 && p.lse)
                     p.lse[bh + r_hi] = any ? (st.m[1] + log2f(l1)) * 0.6931471805599453f : -INFINITY;
             }
@@ -400,9 +450,12 @@ __global__ void __launch_bounds__(kWarps * 32) decode_warp_kernel(const WarpPara
     cp_async_wait<0>();
 }
 
-size_t warp_smem_bytes(int D, int G, int warps, int stages) { return kMetaBytes + (size_t)warps * stages * stage_bytes(D, G); }
+size_t warp_smem_bytes(int D, int G, int warps, int stages, bool f8)
+{
+    return kMetaBytes + (size_t)warps * stages * stage_bytes(D, G, f8);
+}
 
-template <int D, int W>
+template <int D, int W, bool F8>
 int blocks_per_sm(size_t smem)
 {
     struct Entry { size_t smem; int n; };
@@ -413,8 +466,8 @@ int blocks_per_sm(size_t smem)
     for (int i = 0; i < n_cached; ++i)
         if (cache[i].smem == smem) return cache[i].n;
     int n = 0;
-    if (cudaFuncSetAttribute(decode_warp_kernel<D, W>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_warp_kernel<D, W>, W * 32, smem) != cudaSuccess) {
+    if (cudaFuncSetAttribute(decode_warp_kernel<D, W, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_warp_kernel<D, W, F8>, W * 32, smem) != cudaSuccess) {
         (void)cudaGetLastError();
         n = 0;
     }
@@ -428,11 +481,11 @@ int blocks_per_sm(size_t smem)
 // rings are fastest; with few units per SM a warp's chain of memory round trips is the bound and fewer warps with
 // deeper rings (up to 6 chunks) are. head_dim 64 runs two CTAs per SM (of 8 warps at most: registers).
 struct WarpShape { int warps, stages, ctas_per_sm; };
-WarpShape pick_warp_shape(int D, int G, long long units)
+WarpShape pick_warp_shape(int D, int G, long long units, bool f8)
 {
     const int cps = D == 64 ? 2 : 1;
     const size_t budget = (D == 64 ? 113u : 227u) * 1024u - kMetaBytes;
-    const int total = (int)(budget / stage_bytes(D, G));             // chunks of ring per CTA
+    const int total = (int)(budget / stage_bytes(D, G, f8));         // chunks of ring per CTA
     const long long ctas = (long long)sm_count() * cps;
     const long long per_cta = (units + ctas - 1) / ctas;
     const int wmax = (D == 128 && total >= 24) ? 12 : 8;
@@ -448,23 +501,29 @@ WarpShape pick_warp_shape(int D, int G, long long units)
 
 using WarpKernel = void (*)(const WarpParams);
 struct KernelEntry { WarpKernel fn; int (*blocks)(size_t); };
-template <int D, int W>
-KernelEntry entry() { return {decode_warp_kernel<D, W>, &blocks_per_sm<D, W>}; }
-KernelEntry pick_kernel(int D, int warps)
+template <int D, int W, bool F8>
+KernelEntry entry() { return {decode_warp_kernel<D, W, F8>, &blocks_per_sm<D, W, F8>}; }
+KernelEntry pick_kernel(int D, int warps, bool f8)
 {
-    if (D == 64) return warps == 4 ? entry<64, 4>() : warps == 6 ? entry<64, 6>() : entry<64, 8>();
-    return warps == 4 ? entry<128, 4>() : warps == 6 ? entry<128, 6>() : warps == 8 ? entry<128, 8>() : entry<128, 12>();
+    if (f8)                                                       // head_dim 128 only
+        return warps == 4 ? entry<128, 4, true>() : warps == 6 ? entry<128, 6, true>()
+               : warps == 8 ? entry<128, 8, true>() : entry<128, 12, true>();
+    if (D == 64) return warps == 4 ? entry<64, 4, false>() : warps == 6 ? entry<64, 6, false>() : entry<64, 8, false>();
+    return warps == 4 ? entry<128, 4, false>() : warps == 6 ? entry<128, 6, false>()
+           : warps == 8 ? entry<128, 8, false>() : entry<128, 12, false>();
 }
 
 }  // namespace
 
 // Whether the warp-per-unit kernel should serve this decode call. L4L_DECODE_WARP=0 / 1 forces the answer (for
 // tests); shapes it cannot run are refused either way.
-bool decode_warp_eligible(int B, int Hq, int Hkv, int D, int max_kv_len, bool fp8, bool rope)
+bool decode_warp_eligible(int B, int Hq, int Hkv, int D, int max_kv_len, bool fp8, bool rope, bool append)
 {
     const int G = Hq / Hkv;
     const long long units = (long long)B * Hkv;
-    if (fp8 || rope || G > 16 || pick_warp_shape(D, G, units).stages == 0) return false;
+    // fp8 caches: plain decode only (the fused append of an fp8 cache quantises the new token, which this kernel's
+    // copy path cannot do on the way)
+    if (rope || (fp8 && (append || D != 128)) || G > 16 || pick_warp_shape(D, G, units, fp8).stages == 0) return false;
     if (const char *e = getenv("L4L_DECODE_WARP")) return e[0] != '0';
     // many units of a few chunks each: the regime where the split kernel pays its per-piece cost every tile or two.
     // Thresholds measured against the split kernel in CUDA graphs (8 KV heads at head_dim 128, 12 at head_dim 64),
@@ -479,18 +538,19 @@ bool decode_warp_eligible(int B, int Hq, int Hkv, int D, int max_kv_len, bool fp
 l4l_status launch_decode_warp(const void *q, void *o, const l4l_kv_cache &cache, const int32_t *d_kv_lens,
                               int max_kv_len, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
                               cudaStream_t stream, const l4l_tensor4 *k_new, const l4l_tensor4 *v_new,
-                              const PagedTable *paged)
+                              const PagedTable *paged, const Fp8Scales *fp8)
 {
     const int G = Hq / Hkv;
-    if (G > 16 || (k_new == nullptr) != (v_new == nullptr)) return L4L_ERR_UNSUPPORTED;
+    const bool f8 = fp8 != nullptr;
+    if (G > 16 || (k_new == nullptr) != (v_new == nullptr) || (f8 && (k_new || D != 128))) return L4L_ERR_UNSUPPORTED;
     for (int b0 = 0; b0 < B; b0 += kMaxB) {
         const int nb = B - b0 < kMaxB ? B - b0 : kMaxB;
         const long long units = (long long)nb * Hkv;
-        const WarpShape shape = pick_warp_shape(D, G, units);
+        const WarpShape shape = pick_warp_shape(D, G, units, f8);
         const int stages = shape.stages, kWarps = shape.warps;
         if (stages == 0) return L4L_ERR_UNSUPPORTED;
-        const size_t smem = warp_smem_bytes(D, G, kWarps, stages);
-        const KernelEntry kernel = pick_kernel(D, kWarps);
+        const size_t smem = warp_smem_bytes(D, G, kWarps, stages, f8);
+        const KernelEntry kernel = pick_kernel(D, kWarps, f8);
         const int per_sm = kernel.blocks(smem);
         if (per_sm == 0) return L4L_ERR_CUDA;
         WarpParams p = {};
@@ -506,8 +566,12 @@ l4l_status launch_decode_warp(const void *q, void *o, const l4l_kv_cache &cache,
             p.new_sh = k_new->stride_h;
         }
         // paged: the pool as a whole, whatever the slice; contiguous: this slice's sequences
-        p.cache_k = static_cast<__nv_bfloat16 *>(cache.k) + (paged ? 0 : (size_t)b0 * cache.stride_b);
-        p.cache_v = static_cast<__nv_bfloat16 *>(cache.v) + (paged ? 0 : (size_t)b0 * cache.stride_b);
+        // (fp8: the strides count bytes)
+        const size_t base_bytes = paged ? 0 : (size_t)b0 * cache.stride_b * (f8 ? 1 : 2);
+        p.cache_k = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(cache.k) + base_bytes);
+        p.cache_v = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(cache.v) + base_bytes);
+        p.k_scale = f8 ? fp8->k_scale : nullptr;
+        p.v_scale = f8 ? fp8->v_scale : nullptr;
         p.c_sb = cache.stride_b; p.c_sh = cache.stride_h; p.c_st = cache.stride_t;
         p.block_table = paged ? paged->block_table + (size_t)b0 * paged->table_stride : nullptr;
         p.table_stride = paged ? paged->table_stride : 0;

@@ -135,7 +135,7 @@ def test_kernel_choice_by_problem_size(warp_kernel):
         assert l4l.l4l_decode_kernel_choice(64, 12, 12, 64, 1024) == ("split", 4)            # small MHA model
         assert l4l.l4l_decode_kernel_choice(512, 32, 8, 128, 256) == ("warp", 0)             # hundreds of short sequences
         assert l4l.l4l_decode_kernel_choice(512, 32, 8, 128, 4096)[0] == "split"             # ... but not long ones
-        assert l4l.l4l_decode_kernel_choice(512, 32, 8, 128, 256, fp8=True)[0] == "split"    # fp8: not on the warp kernel
+        assert l4l.l4l_decode_kernel_choice(512, 32, 8, 128, 256, fp8=True)[0] == "warp"     # also with an fp8 cache
         assert l4l.l4l_decode_kernel_choice(32, 128, 8, 128, 4096) == ("split", 6)           # groups of 16 query heads
         assert l4l.l4l_decode_kernel_choice(1, 32, 8, 96, 128) is None                       # unsupported head_dim
     finally:
@@ -181,3 +181,49 @@ def test_warp_decode_random_shapes(warp_kernel, seed):
     assert gk.margins_intact() and gv.margins_intact()
     assert np.array_equal(orc.bits(gk.t.cpu()), ref_k) and np.array_equal(orc.bits(gv.t.cpu()), ref_v)
     assert_close_to_oracle(o.cpu(), ref, f"paged decode + append, seed {seed}")
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(32, 8), (8, 8), (16, 2), (16, 1)])
+def test_warp_decode_fp8_cache(warp_kernel, Hq, Hkv):
+    """The fp8 (e4m3) variant of the warp-per-unit kernel against the oracle over the codes: contiguous and paged
+    caches; the fused append of an fp8 cache is not this kernel's (the call must still be served, by the split kernel)."""
+    import test_gpu_fp8 as f8
+
+    assert l4l.l4l_decode_kernel_choice(13, Hq, Hkv, 128, 2304, fp8=True)[0] == "warp"       # forced on by the fixture
+    f8.test_fp8_decode_matches_oracle(Hq, Hkv)
+    f8._fp8_append_case(Hq, Hkv, [1, 16, 17, 33, 255, 300, 0], seed=3500 + Hq, Lmax=320)
+
+
+@pytest.mark.parametrize("page", [16, 64, 256])
+def test_warp_decode_fp8_paged_cache(warp_kernel, page):
+    import test_gpu_fp8 as f8
+
+    f8.test_fp8_paged_decode_matches_oracle(page)
+
+
+def test_warp_decode_fp8_many_short_sequences(warp_kernel):
+    import test_gpu_fp8 as f8
+
+    rng = np.random.default_rng(5)
+    B, Hq, Hkv, D, Lmax = 600, 8, 4, 128, 160
+    lens = rng.integers(0, Lmax + 1, size=B)
+    g = torch.Generator().manual_seed(6)
+    ck8 = f8.random_codes((B, Hkv, Lmax, D), g, 7)
+    cv8 = f8.random_codes((B, Hkv, Lmax, D), g, 7)
+    for b, L in enumerate(lens):
+        ck8[b, :, L:] = 0x7F
+        cv8[b, :, L:] = 0xFF
+    q = torch.randn(B, Hq, D, generator=g).to(torch.bfloat16)
+    ks, vs = torch.rand(Hkv, generator=g) + 0.5, torch.rand(Hkv, generator=g) + 0.25
+    scale = 1.0 / math.sqrt(D)
+    ref, ref_lse = orc.decode_fp8(q, ck8, cv8, lens.astype(np.int32), ks.numpy(), vs.numpy(), scale)
+    o = torch.zeros(B, Hq, D, dtype=torch.bfloat16, device="cuda")
+    lse = torch.zeros(B, Hq, device="cuda")
+    ws = l4l.new_workspace(l4l.L4L_OP_DECODE, B, Hq, Hkv, D, Lmax)
+    l4l.l4l_attn_decode_fp8(q.cuda(), o, ck8.cuda(), cv8.cuda(), ks.cuda(), vs.cuda(),
+                            torch.from_numpy(lens.astype(np.int32)).cuda(), Lmax, scale, ws, lse=lse)
+    torch.cuda.synchronize()
+    assert_close_to_oracle(o.cpu(), ref, "fp8 decode, many short sequences")
+    fin = np.isfinite(ref_lse)
+    assert np.abs(lse.cpu().double().numpy()[fin] - ref_lse[fin]).max() <= 2e-3
+    assert (lse.cpu().numpy()[~fin] == -np.inf).all()
