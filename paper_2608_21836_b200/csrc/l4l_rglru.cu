@@ -32,7 +32,9 @@ constexpr int kCb = 64;          // channels per CTA (two per lane)
 constexpr int kStages = 2;       // TMA buffers per warp
 constexpr uint32_t kArrayBytes = kTb * kCb * 2;
 constexpr uint32_t kStageBytes = 3 * kArrayBytes;
-// kTeam warps per CTA, each taking every kTeam-th tile: 8 for sequences, 1 for a single tile (decode steps)
+// kTeam warps per CTA, each taking every kTeam-th tile: 8 for sequences, 16 when the launch has no more strips
+// than the GPU has SMs (one CTA per SM then, and a strip's rate is set by how many tiles it has in flight),
+// 1 for a single tile (decode steps)
 constexpr size_t smem_bytes(int team)
 {
     return 128 + (size_t)team * kStages * kStageBytes + (team * kStages + team) * 8 + 2 * kCb * 4 + 64;
@@ -253,9 +255,15 @@ l4l_status launch_rglru_scan(const void *x, const void *gate_x, const void *gate
         !make_tmap_rows_bf16(&tga, gate_a, W, T, B, W, (int64_t)T * W, kCb, kTb))
         return L4L_ERR_CUDA;
     static bool configured = false;
+    static int sm_count = 0;
     if (!configured) {
-        if (cudaFuncSetAttribute(rglru_scan_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)smem_bytes(8)) != cudaSuccess)
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+            cudaFuncSetAttribute(rglru_scan_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem_bytes(8)) != cudaSuccess ||
+            cudaFuncSetAttribute(rglru_scan_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem_bytes(16)) != cudaSuccess)
             return L4L_ERR_CUDA;
         configured = true;
     }
@@ -267,6 +275,8 @@ l4l_status launch_rglru_scan(const void *x, const void *gate_x, const void *gate
     const dim3 grid((W + kCb - 1) / kCb, B);
     if (T <= kTb)
         rglru_scan_kernel<1><<<grid, 32, smem_bytes(1), stream>>>(tx, tgx, tga, p);
+    else if ((long long)grid.x * grid.y <= sm_count && T >= 16 * 2 * kTb)
+        rglru_scan_kernel<16><<<grid, 16 * 32, smem_bytes(16), stream>>>(tx, tgx, tga, p);
     else
         rglru_scan_kernel<8><<<grid, 8 * 32, smem_bytes(8), stream>>>(tx, tgx, tga, p);
     return cudaGetLastError() == cudaSuccess ? L4L_OK : L4L_ERR_CUDA;
