@@ -32,6 +32,9 @@
  *   - The caller owns every buffer. The library allocates no device memory, enqueues its
  *     kernels on the caller's stream and never synchronises (l4l_last_device_error excepted).
  *     Sequence lengths live in device memory; only upper bounds come from the host.
+ *   - Every call works on the device that is current in the calling thread (all its pointers
+ *     belong to that device); the one-time set-up of each kernel is kept per device, so one
+ *     process may drive several GPUs, one at a time per call.
  *   - Errors: arguments are validated on the host BEFORE anything is launched; a non-zero
  *     status means no kernel of that call ran. Nothing throws, nothing traps on the device.
  *     Unsupported shapes return L4L_ERR_UNSUPPORTED; there is no fallback path.

@@ -1032,7 +1032,10 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
 template <int D, int W, bool F8, bool BigG>
 int decode_blocks_per_sm(size_t smem)
 {
-    static bool attr_set = false;
+    static bool attr_set_on[kDeviceSlots] = {};
+    const int slot = device_slot();
+    if (slot < 0) return 0;
+    bool &attr_set = attr_set_on[slot];
     if (!attr_set) {
         // the opt-in limit is per kernel: allow everything the SM has
         if (cudaFuncSetAttribute(decode_split_kernel<D, W, F8, BigG>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=

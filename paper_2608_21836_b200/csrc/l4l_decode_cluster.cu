@@ -556,7 +556,10 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
 template <int D, bool F8>
 bool configure_kernel()
 {
-    static bool done = false, ok = false;
+    static bool done_on[kDeviceSlots] = {}, ok_on[kDeviceSlots] = {};
+    const int slot = device_slot();
+    if (slot < 0) return false;
+    bool &done = done_on[slot], &ok = ok_on[slot];
     if (!done) {
         done = true;
         ok = cudaFuncSetAttribute(decode_cluster_kernel<D, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) ==

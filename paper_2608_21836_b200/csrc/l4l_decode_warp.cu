@@ -458,20 +458,22 @@ size_t warp_smem_bytes(int D, int G, int warps, int stages, bool f8)
 template <int D, int W, bool F8>
 int blocks_per_sm(size_t smem)
 {
-    struct Entry { size_t smem; int n; };
-    static Entry cache[8];
+    struct Entry { size_t smem; int dev; int n; };
+    static Entry cache[16];
     static int n_cached = 0;
     static std::mutex mutex;
+    const int dev = device_slot();
+    if (dev < 0) return 0;
     std::lock_guard<std::mutex> lock(mutex);
     for (int i = 0; i < n_cached; ++i)
-        if (cache[i].smem == smem) return cache[i].n;
+        if (cache[i].smem == smem && cache[i].dev == dev) return cache[i].n;
     int n = 0;
     if (cudaFuncSetAttribute(decode_warp_kernel<D, W, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_warp_kernel<D, W, F8>, W * 32, smem) != cudaSuccess) {
         (void)cudaGetLastError();
         n = 0;
     }
-    if (n_cached < 8) cache[n_cached++] = {smem, n};
+    if (n_cached < 16) cache[n_cached++] = {smem, dev, n};
     return n;
 }
 

@@ -10,6 +10,16 @@
 
 namespace l4l {
 
+// One-time set-up of a kernel (the shared-memory opt-in, occupancy look-ups) holds for one device only, so the
+// "already done" flags are kept per device ordinal. Slot of the current device, or -1 if it cannot be had.
+constexpr int kDeviceSlots = 64;
+inline int device_slot()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kDeviceSlots) return -1;
+    return dev;
+}
+
 // Where each logical coordinate (token, head, batch) sits among coordinates 1..3 of a 4-D
 // tensor map whose coordinate 0 is head_dim. Dimensions are ordered by ascending stride.
 struct TmapCoord {

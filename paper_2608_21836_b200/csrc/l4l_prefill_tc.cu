@@ -533,7 +533,10 @@ l4l_status launch_t(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensor
                     const TcParams &p, cudaStream_t stream)
 {
     using C = TcCfg<D>;
-    static bool configured = false;
+    static bool configured_on[kDeviceSlots] = {};
+    const int slot = device_slot();
+    if (slot < 0) return L4L_ERR_CUDA;
+    bool &configured = configured_on[slot];
     if (!configured) {
         if (cudaFuncSetAttribute(prefill_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)C::kSmemBytes) != cudaSuccess)

@@ -254,12 +254,14 @@ l4l_status launch_rglru_scan(const void *x, const void *gate_x, const void *gate
         !make_tmap_rows_bf16(&tgx, gate_x, W, T, B, W, (int64_t)T * W, kCb, kTb) ||
         !make_tmap_rows_bf16(&tga, gate_a, W, T, B, W, (int64_t)T * W, kCb, kTb))
         return L4L_ERR_CUDA;
-    static bool configured = false;
-    static int sm_count = 0;
+    static bool configured_on[kDeviceSlots] = {};
+    static int sm_count_on[kDeviceSlots] = {};
+    const int slot = device_slot();
+    if (slot < 0) return L4L_ERR_CUDA;
+    bool &configured = configured_on[slot];
+    int &sm_count = sm_count_on[slot];
     if (!configured) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, slot) != cudaSuccess ||
             cudaFuncSetAttribute(rglru_scan_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)smem_bytes(8)) != cudaSuccess ||
             cudaFuncSetAttribute(rglru_scan_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
