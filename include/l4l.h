@@ -59,7 +59,7 @@ typedef enum {
     L4L_ERR_UNSUPPORTED = 2, /* head_dim / head grouping outside the supported set             */
     L4L_ERR_WORKSPACE = 3,   /* workspace missing or too small                                  */
     L4L_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed (launch, tensor-map encode) */
-    L4L_ERR_TIMEOUT = 5      /* a bounded device-side wait ran out (see l4l_last_device_error)  */
+    L4L_ERR_TIMEOUT = 5      /* a bounded device-side wait ran out (returned by l4l_check_status) */
 } l4l_status;
 
 /* A cudaStream_t, passed as an opaque pointer (NULL = the legacy default stream). */
@@ -362,7 +362,10 @@ l4l_status l4l_attn_decode(const void *q, void *o, l4l_kv_cache cache,
  * 0..n-1 with that newest token taken from k_new / v_new. Equivalent to l4l_kv_append at slot n-1
  * followed by l4l_attn_decode; sequences with n = 0 append nothing and give o = 0.
  *   k_new, v_new  [B, 1, Hkv, D] views (stride_t unused); both with the same strides
- * Everything else as in l4l_attn_decode.
+ * Everything else as in l4l_attn_decode, except for a sequence whose kv_lens[b] exceeds the host bound
+ * max_kv_len (a caller error): l4l_attn_decode ignores the tokens past the bound, whereas here the new token
+ * has no slot inside the bound, so the sequence is treated as empty: nothing is written to the cache, o[b] = 0
+ * and lse[b] = -inf. The same holds for every other entry point that fuses the append.
  */
 l4l_status l4l_attn_decode_append(const void *q, void *o, l4l_kv_cache cache,
                                   l4l_tensor4 k_new, l4l_tensor4 v_new,
@@ -398,8 +401,8 @@ l4l_status l4l_attn_decode_append(const void *q, void *o, l4l_kv_cache cache,
  *     in it; each call therefore clears the status block and the ticket counters on `stream` before its
  *     kernel. Two calls that can overlap on the GPU (different streams, no ordering between them) race
  *     on the array and give wrong results: order them, or give one of them a workspace.
- *   - A bounded device-side wait that runs out is recorded in the array's status block, which this
- *     entry point does not expose; callers that must observe it use l4l_attn_decode.
+ *   - A bounded device-side wait that runs out is recorded in the array's status block;
+ *     l4l_check_status(NULL, stream) reads it.
  */
 #define L4L_STATIC_SCRATCH_BYTES (8u << 20)
 l4l_status l4l_attn_decode_static(const void *q, void *o, l4l_kv_cache cache,
@@ -414,17 +417,49 @@ const char *l4l_status_string(l4l_status status);
  * Which kernel the decode entry points would run for these sizes on the current device, without launching
  * anything (for tests and tuning): 0 = the split kernel (*detail = consumer warps per CTA), 1 = the cluster
  * kernel (*detail = CTAs per cluster), 2 = the warp-per-unit kernel, -1 = sizes the decode calls reject.
- * fp8: non-zero for an e4m3 cache. detail may be NULL. The environment overrides that the library reads
- * (L4L_DECODE_CLUSTER, L4L_DECODE_WARP, L4L_DECODE_WARPS: debugging aids) are honoured here as there.
+ * fp8: non-zero for an e4m3 cache. detail may be NULL. The overrides of l4l_set_decode_override are honoured
+ * here as in the decode calls.
  */
 int l4l_decode_kernel_choice(int B, int Hq, int Hkv, int head_dim, int max_kv_len, int fp8, int *detail);
 
 /*
+ * Tuning override of the decode kernel choice, process-wide (for tests and benchmarks that must hold a call on
+ * one kernel; a serving loop has no reason to call it). No counterpart in the paper.
+ *   cluster      -1 library's choice; 0 never the cluster kernel; N > 0 clusters of N CTAs where they fit
+ *   warp         -1 library's choice; 0 never the warp-per-unit kernel; 1 that kernel wherever it can run
+ *   split_warps   0 library's choice; 4 or 8 consumer warps per CTA of the split kernel
+ * The decode calls never read the environment; L4L_DECODE_CLUSTER, L4L_DECODE_WARP and L4L_DECODE_WARPS are
+ * read once, when the library is loaded, as the initial values of these three settings.
+ */
+void l4l_set_decode_override(int cluster, int warp, int split_warps);
+
+/*
  * Synchronises `stream`, reads the workspace's status block and returns 0 if no bounded wait
  * has run out since the last l4l_workspace_init(), else a non-zero code identifying the wait
- * (bit 0: decode pipeline, bit 1: prefill pipeline). Returns -1 if the read itself fails.
+ * (bit 0: decode pipeline, bit 1: prefill pipeline, bit 2: scan pipeline, bit 3: the self-test). Returns -1 if
+ * the read itself fails.
  */
 int l4l_last_device_error(void *workspace, l4l_stream stream);
+
+/*
+ * The same check as a status: synchronises `stream` and returns L4L_OK if no bounded device-side wait has run
+ * out since the status block was last cleared, L4L_ERR_TIMEOUT if one has (the kernels of that call gave up and
+ * returned; their outputs are not valid), L4L_ERR_CUDA if the block cannot be read. workspace = NULL checks the
+ * status block of the library's own scratch array on the current device, the one l4l_attn_decode_static uses
+ * (that entry point clears it at every call, so the answer is about the latest such call). After
+ * L4L_ERR_TIMEOUT, l4l_workspace_init makes the workspace usable again.
+ */
+l4l_status l4l_check_status(void *workspace, l4l_stream stream);
+
+/*
+ * Self-test of the time-out path (no counterpart in the paper; not part of the hot path). Launches one warp
+ * that waits, with the library's bounded-wait routine and a budget of `budget_cycles` SM clock cycles (clamped
+ * to [1000, 2^24], i.e. a few milliseconds at most), on a pipeline barrier that nothing ever completes. The wait
+ * runs out, the kernel records bit 3 in the workspace's status block and returns normally: the context stays
+ * usable, nothing traps. Afterwards l4l_last_device_error() reports a non-zero code and l4l_check_status()
+ * L4L_ERR_TIMEOUT until l4l_workspace_init() is called. workspace: any workspace of this library (>= 256 bytes).
+ */
+l4l_status l4l_selftest_wait_expiry(void *workspace, size_t ws_bytes, long long budget_cycles, l4l_stream stream);
 
 /* Library version, "major.minor". */
 const char *l4l_version(void);

@@ -26,7 +26,7 @@ EXPORTS = (
     "l4l_kv_append_paged", "l4l_attn_decode_paged", "l4l_kv_append_fp8", "l4l_attn_decode_fp8", "l4l_rglru_scan", "l4l_rglru_workspace_bytes",
     "l4l_attn_decode_paged_fp8", "l4l_attn_merge", "l4l_attn_decode_rope_append", "l4l_attn_decode_paged_append",
     "l4l_attn_decode_paged_rope_append", "l4l_attn_decode_append_fp8", "l4l_attn_decode_paged_append_fp8",
-    "l4l_decode_kernel_choice",
+    "l4l_decode_kernel_choice", "l4l_set_decode_override", "l4l_check_status", "l4l_selftest_wait_expiry",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -106,6 +106,12 @@ def load() -> ctypes.CDLL:
                                                      c_int, c_int, c_int, c_int, ctypes.c_float, vp, vp, c_size, vp]
     lib.l4l_decode_kernel_choice.restype = c_int
     lib.l4l_decode_kernel_choice.argtypes = [c_int, c_int, c_int, c_int, c_int, c_int, ctypes.POINTER(c_int)]
+    lib.l4l_set_decode_override.restype = None
+    lib.l4l_set_decode_override.argtypes = [c_int, c_int, c_int]
+    lib.l4l_check_status.restype = c_int
+    lib.l4l_check_status.argtypes = [vp, vp]
+    lib.l4l_selftest_wait_expiry.restype = c_int
+    lib.l4l_selftest_wait_expiry.argtypes = [vp, c_size, ctypes.c_longlong, vp]
     lib.l4l_kv_append_fp8.restype = c_int
     lib.l4l_kv_append_fp8.argtypes = [KVCache, Tensor4, Tensor4, i32p, i32p, c_int, c_int, c_int, c_int, vp, vp, vp]
     lib.l4l_attn_decode_fp8.restype = c_int
@@ -565,6 +571,47 @@ def l4l_decode_kernel_choice(B: int, Hq: int, Hkv: int, D: int, max_kv_len: int,
     detail = ctypes.c_int(0)
     k = load().l4l_decode_kernel_choice(B, Hq, Hkv, D, int(max_kv_len), int(bool(fp8)), ctypes.byref(detail))
     return None if k < 0 else (("split", "cluster", "warp")[k], detail.value)
+
+
+_override = {"cluster": -1, "warp": -1, "split_warps": 0}
+
+
+def l4l_set_decode_override(cluster: int = -1, warp: int = -1, split_warps: int = 0) -> None:
+    """Process-wide tuning override of the decode kernel choice (see the header); the defaults restore the library's own
+    choice."""
+    load().l4l_set_decode_override(int(cluster), int(warp), int(split_warps))
+    _override.update(cluster=int(cluster), warp=int(warp), split_warps=int(split_warps))
+
+
+class decode_override:
+    """``with decode_override(cluster=0): ...`` holds the decode calls of the block on one kernel and puts the previous
+    settings back afterwards. Only the settings that are named change."""
+
+    def __init__(self, cluster: Optional[int] = None, warp: Optional[int] = None, split_warps: Optional[int] = None):
+        self.want = {k: v for k, v in (("cluster", cluster), ("warp", warp), ("split_warps", split_warps)) if v is not None}
+
+    def __enter__(self):
+        self.old = dict(_override)
+        l4l_set_decode_override(**{**self.old, **self.want})
+        return self
+
+    def __exit__(self, *exc):
+        l4l_set_decode_override(**self.old)
+        return False
+
+
+def l4l_check_status(workspace: Optional[torch.Tensor] = None) -> int:
+    """L4L_OK, or L4L_ERR_TIMEOUT if a bounded device-side wait has run out since the status block was cleared
+    (synchronises the stream). workspace=None: the status block of the library's own scratch array."""
+    return int(load().l4l_check_status(None if workspace is None else workspace.data_ptr(), _stream()))
+
+
+def l4l_selftest_wait_expiry(workspace: torch.Tensor, budget_cycles: int = 100000) -> None:
+    """Launches the one-warp kernel whose bounded wait runs out by construction (see the header)."""
+    st = load().l4l_selftest_wait_expiry(workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                         int(budget_cycles), _stream())
+    if st != L4L_OK:
+        raise L4LError(st, "l4l_selftest_wait_expiry")
 
 
 def l4l_attn_merge(o_parts, lse_parts, o, lse=None) -> None:

@@ -1,6 +1,8 @@
 // C-ABI entry points: host-side validation, workspace sizing, tensor-map construction.
 // Nothing here touches the data path; every operation runs in the kernels of the other
 // translation units.
+#include <atomic>
+#include <cstdlib>
 #include <mutex>
 
 #include "l4l_internal.h"
@@ -54,20 +56,55 @@ l4l_status shape_status(int B, int Hq, int Hkv, int D)
 
 int sm_count()
 {
-    static int n = 0;
+    // per device: one process may drive GPUs that differ in SM count (or in how they are partitioned)
+    static std::atomic<int> n_on[kDeviceSlots];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kDeviceSlots) {
+        (void)cudaGetLastError();
+        return 148;
+    }
+    int n = n_on[dev].load(std::memory_order_relaxed);
     if (n == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+            (void)cudaGetLastError();
             n = 148;
+        }
+        n_on[dev].store(n, std::memory_order_relaxed);
     }
     return n;
+}
+
+std::mutex &setup_mutex()
+{
+    static std::mutex m;
+    return m;
+}
+
+namespace {
+
+std::atomic<int> g_override_cluster{-1}, g_override_warp{-1}, g_override_split_warps{0};
+
+// The environment is read once, when the library is loaded.
+const bool g_override_seeded = [] {
+    if (const char *e = getenv("L4L_DECODE_CLUSTER")) g_override_cluster = atoi(e);
+    if (const char *e = getenv("L4L_DECODE_WARP")) g_override_warp = (e[0] != '0') ? 1 : 0;
+    if (const char *e = getenv("L4L_DECODE_WARPS")) g_override_split_warps = atoi(e);
+    return true;
+}();
+
+}  // namespace
+
+DecodeOverride decode_override()
+{
+    return DecodeOverride{g_override_cluster.load(std::memory_order_relaxed), g_override_warp.load(std::memory_order_relaxed),
+                          g_override_split_warps.load(std::memory_order_relaxed)};
 }
 
 namespace {
 
 // A serving loop calls with the same buffers step after step: remember the last few encoded maps
-// (a tensor map is a pure function of these arguments).
+// (a tensor map is a pure function of these arguments; it encodes an address and a layout, nothing of the
+// device, and under unified addressing an address names one device's memory, so the key needs no device).
 struct TmapKey {
     const void *base;
     int D, box_d, box_t, elem_bytes;
@@ -581,6 +618,13 @@ l4l_status l4l_attn_decode_paged_rope_append(const void *q, void *o, l4l_paged_k
     const RopeArgs rope{d_cos, d_sin, d_q_weight, d_k_weight, norm_eps, n_pos};
     return launch_decode(q, o, pool_as_cache(pool), d_kv_lens, max_kv_len, B, Hq, Hkv, head_dim, scale, d_lse, workspace,
                          plan, static_cast<cudaStream_t>(stream), &k_new, &v_new, &pt, nullptr, &rope);
+}
+
+void l4l_set_decode_override(int cluster, int warp, int split_warps)
+{
+    g_override_cluster = cluster < 0 ? -1 : cluster;
+    g_override_warp = warp < 0 ? -1 : (warp ? 1 : 0);
+    g_override_split_warps = (split_warps == 4 || split_warps == 8) ? split_warps : 0;
 }
 
 int l4l_decode_kernel_choice(int B, int Hq, int Hkv, int head_dim, int max_kv_len, int fp8, int *detail)

@@ -236,7 +236,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             int n = 0;
             if (b < p.B) {
                 int len = b0 == 0 ? early_len : p.kv_lens[b];
-                len = len < 0 ? 0 : (len > p.max_kv_len ? p.max_kv_len : len);
+                len = len < 0 ? 0 : (len > p.max_kv_len ? (p.k_new ? 0 : p.max_kv_len) : len);   // over the host's bound: decode ignores the extra tokens, a fused append treats the sequence as empty
                 lens_s[b] = len;
                 n = len > 0 ? ((len + kTileT - 1) / kTileT + 1) * p.Hkv : 0;
             }
@@ -1036,6 +1036,7 @@ int decode_blocks_per_sm(size_t smem)
     const int slot = device_slot();
     if (slot < 0) return 0;
     bool &attr_set = attr_set_on[slot];
+    std::lock_guard<std::mutex> lock(setup_mutex());
     if (!attr_set) {
         // the opt-in limit is per kernel: allow everything the SM has
         if (cudaFuncSetAttribute(decode_split_kernel<D, W, F8, BigG>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
@@ -1146,10 +1147,7 @@ DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int max_kv_len, size_t ws_
     }
     // 128-wide heads: prefer the 8-warp shape (one CTA per SM, ranges twice as long, so fewer sequences are cut
     // between CTAs) whenever its shared memory fits, which it does for query-head groups of up to 4; else 4 warps.
-    static const int forced = [] {
-        const char *e = getenv("L4L_DECODE_WARPS");      // debugging aid: force a shape
-        return e ? atoi(e) : 0;
-    }();
+    const int forced = decode_override().split_warps;    // tuning override: force a shape
     // With 64-wide heads a tile carries half the bytes for the same per-tile work in the consumer warps, and two
     // 4-warp CTAs per SM (two independent streams) hide that better than one 8-warp CTA: 4 warps first there.
     const bool four_first = forced == 4 || (forced == 0 && D == 64);
@@ -1317,6 +1315,8 @@ constexpr int kMaxDevices = 64;
 void *g_static_scratch_addr[kMaxDevices] = {nullptr};
 std::mutex g_static_scratch_mutex;
 
+}  // namespace
+
 // Device address of the scratch array on the current device, or nullptr if the look-up fails.
 void *static_scratch_on_current_device()
 {
@@ -1333,8 +1333,6 @@ void *static_scratch_on_current_device()
     }
     return g_static_scratch_addr[dev];
 }
-
-}  // namespace
 
 }  // namespace l4l
 

@@ -172,7 +172,7 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
     grid_dependency_wait();
     grid_launch_dependents();
     int len = __ldg(p.kv_lens + b);
-    len = len < 0 ? 0 : (len > p.max_kv_len ? p.max_kv_len : len);
+    len = len < 0 ? 0 : (len > p.max_kv_len ? (p.k_new ? 0 : p.max_kv_len) : len);   // over the host's bound: decode ignores the extra tokens, a fused append treats the sequence as empty
     const bool with_rope = p.rope_cos != nullptr && len - 1 < p.rope_n_pos;   // a position outside the table: rows stay as they are
     if (p.rope_cos != nullptr) {
         for (int i = threadIdx.x; i < D; i += kThreads) {
@@ -560,6 +560,7 @@ bool configure_kernel()
     const int slot = device_slot();
     if (slot < 0) return false;
     bool &done = done_on[slot], &ok = ok_on[slot];
+    std::lock_guard<std::mutex> lock(setup_mutex());
     if (!done) {
         done = true;
         ok = cudaFuncSetAttribute(decode_cluster_kernel<D, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) ==
@@ -582,14 +583,16 @@ int pick_stages(int G)
 template <int D, bool F8>
 int resident_clusters(int C, size_t smem)
 {
-    struct Entry { int C; size_t smem; int n; };
-    static Entry cache[16];
+    struct Entry { int C; size_t smem; int dev; int n; };
+    static Entry cache[32];
     static int n_cached = 0;
     static std::mutex mutex;
+    const int dev = device_slot();
+    if (dev < 0) return 0;
+    if (!configure_kernel<D, F8>()) return 0;
     std::lock_guard<std::mutex> lock(mutex);
     for (int i = 0; i < n_cached; ++i)
-        if (cache[i].C == C && cache[i].smem == smem) return cache[i].n;
-    if (!configure_kernel<D, F8>()) return 0;
+        if (cache[i].C == C && cache[i].smem == smem && cache[i].dev == dev) return cache[i].n;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(C, 1, 1);
     cfg.blockDim = dim3(kThreads);
@@ -604,7 +607,7 @@ int resident_clusters(int C, size_t smem)
         (void)cudaGetLastError();
         n = 0;
     }
-    if (n_cached < 16) cache[n_cached++] = Entry{C, smem, n};
+    if (n_cached < 32) cache[n_cached++] = Entry{C, smem, dev, n};
     return n;
 }
 
@@ -635,9 +638,8 @@ ClusterShape pick_cluster_shape(int D, bool fp8)
 
 int decode_cluster_width(int B, int Hq, int Hkv, int D, int max_kv_len, bool fp8)
 {
-    // debugging aid: L4L_DECODE_CLUSTER=0 keeps every call on the split kernel, =N forces clusters of N where they fit
-    int forced = -1;
-    if (const char *e = getenv("L4L_DECODE_CLUSTER")) forced = atoi(e);
+    // tuning override: 0 keeps every call on the split kernel, N forces clusters of N where they fit
+    const int forced = decode_override().cluster;
     if (forced == 0) return 0;
     const int G = Hq / Hkv;
     const long long units = (long long)B * Hkv;

@@ -112,7 +112,7 @@ __global__ void __launch_bounds__(kWarps * 32) decode_warp_kernel(const WarpPara
         int len = 0, ch = 0;
         if (b < p.B) {
             len = __ldg(p.kv_lens + b);
-            len = len < 0 ? 0 : (len > p.max_kv_len ? p.max_kv_len : len);
+            len = len < 0 ? 0 : (len > p.max_kv_len ? (p.k_new ? 0 : p.max_kv_len) : len);   // over the host's bound: decode ignores the extra tokens, a fused append treats the sequence as empty
             lens_s[b] = len;
             ch = len > 0 ? (len + kChunkT - 1) / kChunkT : 1;
         }
@@ -517,7 +517,7 @@ KernelEntry pick_kernel(int D, int warps, bool f8)
 
 }  // namespace
 
-// Whether the warp-per-unit kernel should serve this decode call. L4L_DECODE_WARP=0 / 1 forces the answer (for
+// Whether the warp-per-unit kernel should serve this decode call. The tuning override (l4l_set_decode_override) forces the answer (for
 // tests); shapes it cannot run are refused either way.
 bool decode_warp_eligible(int B, int Hq, int Hkv, int D, int max_kv_len, bool fp8, bool rope, bool append)
 {
@@ -526,7 +526,7 @@ bool decode_warp_eligible(int B, int Hq, int Hkv, int D, int max_kv_len, bool fp
     // fp8 caches: plain decode only (the fused append of an fp8 cache quantises the new token, which this kernel's
     // copy path cannot do on the way)
     if (rope || (fp8 && (append || D != 128)) || G > 16 || pick_warp_shape(D, G, units, fp8).stages == 0) return false;
-    if (const char *e = getenv("L4L_DECODE_WARP")) return e[0] != '0';
+    if (const int forced = decode_override().warp; forced >= 0) return forced != 0;
     // many units of a few chunks each: the regime where the split kernel pays its per-piece cost every tile or two.
     // Thresholds measured against the split kernel in CUDA graphs (8 KV heads at head_dim 128, 12 at head_dim 64),
     // in units per SM: with at most 256 tokens per sequence it wins from 3 units per SM (8 at head_dim 64), with

@@ -3,6 +3,7 @@
 
 #include <cuda.h>
 #include <cuda_runtime.h>
+#include <mutex>
 #include <stddef.h>
 #include <stdint.h>
 
@@ -19,6 +20,20 @@ inline int device_slot()
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kDeviceSlots) return -1;
     return dev;
 }
+
+// One mutex for every "first call on this device" set-up (shared-memory opt-ins, occupancy look-ups): those
+// flags are read and written from whichever host thread launches first.
+std::mutex &setup_mutex();
+
+// Tuning overrides of the decode kernel choice (tests and benchmarks use them to hold a call on one kernel).
+// Seeded once, when the library is loaded, from L4L_DECODE_CLUSTER / L4L_DECODE_WARP / L4L_DECODE_WARPS, and
+// changed afterwards only through l4l_set_decode_override: no decode call reads the environment.
+struct DecodeOverride {
+    int cluster;       // -1: library's choice, 0: never the cluster kernel, N > 0: clusters of N where they fit
+    int warp;          // -1: library's choice, 0: never the warp-per-unit kernel, 1: always where it can run
+    int split_warps;   // 0: library's choice, 4 or 8: consumer warps of the split kernel
+};
+DecodeOverride decode_override();
 
 // Where each logical coordinate (token, head, batch) sits among coordinates 1..3 of a 4-D
 // tensor map whose coordinate 0 is head_dim. Dimensions are ordered by ascending stride.

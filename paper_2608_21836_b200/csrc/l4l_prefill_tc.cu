@@ -536,12 +536,15 @@ l4l_status launch_t(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensor
     static bool configured_on[kDeviceSlots] = {};
     const int slot = device_slot();
     if (slot < 0) return L4L_ERR_CUDA;
-    bool &configured = configured_on[slot];
-    if (!configured) {
-        if (cudaFuncSetAttribute(prefill_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)C::kSmemBytes) != cudaSuccess)
-            return L4L_ERR_CUDA;
-        configured = true;
+    {
+        std::lock_guard<std::mutex> lock(setup_mutex());
+        bool &configured = configured_on[slot];
+        if (!configured) {
+            if (cudaFuncSetAttribute(prefill_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)C::kSmemBytes) != cudaSuccess)
+                return L4L_ERR_CUDA;
+            configured = true;
+        }
     }
     const long long grid = (long long)p.n_qblocks * p.Hq * p.B;
     if (grid > 0x7fffffffll) return L4L_ERR_UNSUPPORTED;

@@ -17,6 +17,7 @@ constexpr int kStatusInfoWord = 1;      // where it happened (role / barrier id)
 constexpr unsigned kErrDecodeWait = 1u;
 constexpr unsigned kErrPrefillWait = 2u;
 constexpr unsigned kErrScanWait = 4u;
+constexpr unsigned kErrSelfTestWait = 8u;
 constexpr size_t kStatusBytes = 256;
 
 // Cycle budget of one bounded wait (~0.25 s at 2 GHz): far above any legitimate latency.
@@ -125,6 +126,26 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
         if ((++polls & 0xffu) == 0) {
             if (*abort_flag) return false;
             if (clock64() - t0 > kWaitCycleBudget) {
+                *abort_flag = 1;
+                return false;
+            }
+            if (polls > 4096u) __nanosleep(64);
+        }
+    }
+}
+
+// The same wait with the budget as an argument (the time-out self-test uses a short one).
+__device__ __forceinline__ bool mbar_wait_budget(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
+                                                 long long budget_cycles)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    uint32_t polls = 0;
+    while (true) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((++polls & 0xffu) == 0) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > budget_cycles) {
                 *abort_flag = 1;
                 return false;
             }

@@ -194,6 +194,10 @@ rglru_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 av[t] = a;
                 const uint64_t mxh = mul_f32x2(mul_f32x2(pack_f32x2(m0, m1), half2), xv);   // m x / 2
                 bv[t] = fma_f32x2(th_x, mxh, mxh);                                         // m x sigmoid(gate_x)
+                if constexpr (!kPlain) {
+                    // rows past the end are caller memory that may hold anything (0 * NaN is NaN): select, not multiply
+                    if (t >= n) bv[t] = zero2;
+                }
             }
         };
         if (resets == 0u && n == kTb)
@@ -258,16 +262,20 @@ l4l_status launch_rglru_scan(const void *x, const void *gate_x, const void *gate
     static int sm_count_on[kDeviceSlots] = {};
     const int slot = device_slot();
     if (slot < 0) return L4L_ERR_CUDA;
-    bool &configured = configured_on[slot];
-    int &sm_count = sm_count_on[slot];
-    if (!configured) {
-        if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, slot) != cudaSuccess ||
-            cudaFuncSetAttribute(rglru_scan_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)smem_bytes(8)) != cudaSuccess ||
-            cudaFuncSetAttribute(rglru_scan_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)smem_bytes(16)) != cudaSuccess)
-            return L4L_ERR_CUDA;
-        configured = true;
+    int sm_count;
+    {
+        std::lock_guard<std::mutex> lock(setup_mutex());
+        bool &configured = configured_on[slot];
+        if (!configured) {
+            if (cudaDeviceGetAttribute(&sm_count_on[slot], cudaDevAttrMultiProcessorCount, slot) != cudaSuccess ||
+                cudaFuncSetAttribute(rglru_scan_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)smem_bytes(8)) != cudaSuccess ||
+                cudaFuncSetAttribute(rglru_scan_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)smem_bytes(16)) != cudaSuccess)
+                return L4L_ERR_CUDA;
+            configured = true;
+        }
+        sm_count = sm_count_on[slot];
     }
     RglruParams p;
     p.a_param = d_a_param; p.position = d_position; p.seq_lens = d_seq_lens; p.state = d_state;

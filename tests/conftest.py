@@ -28,6 +28,7 @@ def pytest_collection_modifyitems(config, items):
 # once with every call kept on the split kernel, so that small test shapes cover both.
 _DECODE_MODULES = {"test_gpu_decode", "test_gpu_decode_append", "test_gpu_paged", "test_gpu_random_shapes",
                    "test_gpu_cuda_graph", "test_gpu_rope_append", "test_gpu_fp8"}
+# (the static-scratch test pins its shapes to the split kernel itself and asserts that choice)
 
 
 def pytest_generate_tests(metafunc):
@@ -39,14 +40,8 @@ def pytest_generate_tests(metafunc):
 
 @pytest.fixture
 def decode_kernel_choice(request):
+    from paper_2608_21836_b200 import binding as l4l
+
     mode = getattr(request, "param", "auto")
-    old = os.environ.get("L4L_DECODE_CLUSTER")
-    if mode == "split":
-        os.environ["L4L_DECODE_CLUSTER"] = "0"
-    else:
-        os.environ.pop("L4L_DECODE_CLUSTER", None)
-    yield mode
-    if old is None:
-        os.environ.pop("L4L_DECODE_CLUSTER", None)
-    else:
-        os.environ["L4L_DECODE_CLUSTER"] = old
+    with l4l.decode_override(cluster=0 if mode == "split" else -1):
+        yield mode

@@ -85,3 +85,32 @@ def test_decode_append_steps_equal_prefill_rows_layer8b():
     ref, _ = orc.prefill_rows(seq.q, seq.k, seq.v, np.full(B, S + T, np.int32), w.scale, rows)
     got = torch.stack([outs[b, t, h] for b in range(B) for t in steps for h in range(Hq)])
     assert_close_to_oracle(got, ref, "layer8b fused decode steps")
+
+
+@pytest.mark.parametrize("B,Lmax", [(3, 512), (40, 512)])
+def test_decode_append_length_beyond_the_host_bound_leaves_the_cache_alone(B, Lmax):
+    """A sequence whose device length exceeds the host bound has no slot for its new token inside the bound: the
+    fused step must not write it over a valid slot. It is treated as empty (o = 0, lse = -inf, nothing written);
+    the other sequences of the batch are unaffected. Small batch: cluster kernel; 40 x 8 units: split kernel."""
+    Hq, Hkv, D, bound = 16, 8, 128, 256
+    lens = [200] * B
+    lens[1] = 300                                            # > bound (but inside the cache)
+    q, ck, cv, kn, vn, kv_len = make_case(B, Hq, Hkv, D, Lmax, lens, seed=640 + B)
+    ck, cv = torch.nan_to_num(ck.float()).to(torch.bfloat16), torch.nan_to_num(cv.float()).to(torch.bfloat16)
+    scale = 1.0 / math.sqrt(D)
+    ok = torch.tensor([b != 1 for b in range(B)])
+    pos = (kv_len - 1).numpy()
+    ek, ev = orc.kv_append(ck, cv, kn, vn, pos, ok.to(torch.int32).numpy())
+    ek_t = torch.from_numpy(ek.view(np.int16)).view(torch.bfloat16)
+    ev_t = torch.from_numpy(ev.view(np.int16)).view(torch.bfloat16)
+    ref, _ = orc.decode(q, ek_t, ev_t, torch.where(ok, kv_len, torch.zeros_like(kv_len)).numpy(), scale)
+    dk, dv = ck.cuda(), cv.cuda()
+    o = nan_bf16((B, Hq, D)).cuda()
+    lse = torch.full((B, Hq), float("nan"), device="cuda")
+    ws = l4l.new_workspace(l4l.L4L_OP_DECODE, B, Hq, Hkv, D, bound)
+    l4l.l4l_attn_decode_append(q.cuda(), o, dk, dv, kn.cuda(), vn.cuda(), kv_len.cuda(), bound, scale, ws, lse=lse)
+    torch.cuda.synchronize()
+    assert l4l.l4l_last_device_error(ws) == 0
+    assert bits_equal(dk, ek) and bits_equal(dv, ev)         # sequence 1's cache untouched, the others got their row
+    assert_close_to_oracle(o, ref, "decode_append with one over-long sequence")
+    assert torch.isneginf(lse[1]).all() and torch.isfinite(lse[ok.cuda()]).all()

@@ -19,13 +19,8 @@ pytestmark = pytest.mark.gpu
 
 @pytest.fixture(autouse=True)
 def split_kernel_only():
-    old = os.environ.get("L4L_DECODE_CLUSTER")
-    os.environ["L4L_DECODE_CLUSTER"] = "0"
-    yield
-    if old is None:
-        os.environ.pop("L4L_DECODE_CLUSTER", None)
-    else:
-        os.environ["L4L_DECODE_CLUSTER"] = old
+    with l4l.decode_override(cluster=0):
+        yield
 
 
 @pytest.mark.parametrize("Hq,Hkv", [(40, 8), (48, 8), (56, 8), (64, 8), (8, 1), (5, 1), (72, 8), (96, 8), (128, 8), (16, 1),

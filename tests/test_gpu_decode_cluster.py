@@ -17,13 +17,8 @@ pytestmark = pytest.mark.gpu
 
 @pytest.fixture
 def cluster_width(request):
-    old = os.environ.get("L4L_DECODE_CLUSTER")
-    os.environ["L4L_DECODE_CLUSTER"] = str(request.param)
-    yield request.param
-    if old is None:
-        os.environ.pop("L4L_DECODE_CLUSTER", None)
-    else:
-        os.environ["L4L_DECODE_CLUSTER"] = old
+    with l4l.decode_override(cluster=int(request.param)):
+        yield request.param
 
 
 WIDTHS = [1, 2, 4, 8]
@@ -151,16 +146,12 @@ def test_library_choice_matches_split_kernel_result():
     lens = [2304]
     q, ck, cv, kv_len = random_batch(1, 32, 8, 128, 2304, lens, seed=3)
     outs = []
-    for mode in ("0", None):
-        if mode is None:
-            os.environ.pop("L4L_DECODE_CLUSTER", None)
-        else:
-            os.environ["L4L_DECODE_CLUSTER"] = mode
-        o = torch.zeros(1, 32, 128, dtype=torch.bfloat16, device="cuda")
-        ws = l4l.new_workspace(l4l.L4L_OP_DECODE, 1, 32, 8, 128, 2304)
-        l4l.l4l_attn_decode(q.cuda(), o, ck.cuda(), cv.cuda(), kv_len.cuda(), 2304, 1.0 / math.sqrt(128), ws)
-        torch.cuda.synchronize()
-        assert l4l.l4l_last_device_error(ws) == 0
-        outs.append(o.float().cpu())
-    os.environ.pop("L4L_DECODE_CLUSTER", None)
+    for mode in (0, -1):
+        with l4l.decode_override(cluster=mode):
+            o = torch.zeros(1, 32, 128, dtype=torch.bfloat16, device="cuda")
+            ws = l4l.new_workspace(l4l.L4L_OP_DECODE, 1, 32, 8, 128, 2304)
+            l4l.l4l_attn_decode(q.cuda(), o, ck.cuda(), cv.cuda(), kv_len.cuda(), 2304, 1.0 / math.sqrt(128), ws)
+            torch.cuda.synchronize()
+            assert l4l.l4l_last_device_error(ws) == 0
+            outs.append(o.float().cpu())
     assert (outs[0] - outs[1]).abs().max() <= 2e-2

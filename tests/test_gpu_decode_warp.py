@@ -1,5 +1,5 @@
 """The decode kernel for many short sequences (one warp per (sequence, KV head), no merge) against the fp64 oracle,
-forced on through L4L_DECODE_WARP for small shapes, and chosen by the library for the regime it is made for."""
+forced on through the tuning override for small shapes, and chosen by the library for the regime it is made for."""
 import math
 import os
 
@@ -19,16 +19,8 @@ pytestmark = pytest.mark.gpu
 def warp_kernel(request):
     """'1': every eligible decode call runs on the warp kernel; '0': never; None: the library's choice."""
     mode = getattr(request, "param", "1")
-    old = os.environ.get("L4L_DECODE_WARP")
-    if mode is None:
-        os.environ.pop("L4L_DECODE_WARP", None)
-    else:
-        os.environ["L4L_DECODE_WARP"] = mode
-    yield mode
-    if old is None:
-        os.environ.pop("L4L_DECODE_WARP", None)
-    else:
-        os.environ["L4L_DECODE_WARP"] = old
+    with l4l.decode_override(warp=-1 if mode is None else int(mode)):
+        yield mode
 
 
 @pytest.mark.parametrize("D", [64, 128])
@@ -127,8 +119,7 @@ def test_library_picks_the_warp_kernel_for_many_short_sequences(warp_kernel):
 @pytest.mark.parametrize("warp_kernel", [None], indirect=True)
 def test_kernel_choice_by_problem_size(warp_kernel):
     """The three decode kernels and the regimes the library gives them (8B-shaped layer: 32 query heads on 8 KV heads)."""
-    old = os.environ.pop("L4L_DECODE_CLUSTER", None)
-    try:
+    with l4l.decode_override(cluster=-1):
         assert l4l.l4l_decode_kernel_choice(1, 32, 8, 128, 2304) == ("cluster", 8)          # one sequence: latency-bound
         assert l4l.l4l_decode_kernel_choice(4, 32, 8, 128, 2304)[0] == "cluster"
         assert l4l.l4l_decode_kernel_choice(32, 32, 8, 128, 4096) == ("split", 8)            # the benchmark batch
@@ -138,9 +129,6 @@ def test_kernel_choice_by_problem_size(warp_kernel):
         assert l4l.l4l_decode_kernel_choice(512, 32, 8, 128, 256, fp8=True)[0] == "warp"     # also with an fp8 cache
         assert l4l.l4l_decode_kernel_choice(32, 128, 8, 128, 4096) == ("split", 6)           # groups of 16 query heads
         assert l4l.l4l_decode_kernel_choice(1, 32, 8, 96, 128) is None                       # unsupported head_dim
-    finally:
-        if old is not None:
-            os.environ["L4L_DECODE_CLUSTER"] = old
 
 
 @pytest.mark.parametrize("seed", range(16))

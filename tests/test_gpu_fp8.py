@@ -229,18 +229,9 @@ def test_fp8_paged_decode_with_fused_append(page):
 
 @pytest.mark.parametrize("width", [1, 2, 8])
 def test_fp8_fused_append_on_the_cluster_kernel(width):
-    import os
-
-    old = os.environ.get("L4L_DECODE_CLUSTER")
-    os.environ["L4L_DECODE_CLUSTER"] = str(width)
-    try:
+    with l4l.decode_override(cluster=width):
         _fp8_append_case(8, 2, [1, 32, 33, 256, 257, 1000, 0, 2304], seed=3200 + width)
         _fp8_append_case(8, 2, [1, 33, 257, 1000, 0, 2304], seed=3300 + width, page=64)
-    finally:
-        if old is None:
-            os.environ.pop("L4L_DECODE_CLUSTER", None)
-        else:
-            os.environ["L4L_DECODE_CLUSTER"] = old
 
 
 def test_fp8_fused_append_batch_of_several_launch_slices():

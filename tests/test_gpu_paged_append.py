@@ -50,16 +50,8 @@ def run_case(B, Hq, Hkv, D, page, lens, seed, drop=()):
 
 @pytest.fixture
 def kernel_choice(request):
-    old = os.environ.get("L4L_DECODE_CLUSTER")
-    if request.param is None:
-        os.environ.pop("L4L_DECODE_CLUSTER", None)
-    else:
-        os.environ["L4L_DECODE_CLUSTER"] = str(request.param)
-    yield request.param
-    if old is None:
-        os.environ.pop("L4L_DECODE_CLUSTER", None)
-    else:
-        os.environ["L4L_DECODE_CLUSTER"] = old
+    with l4l.decode_override(cluster=-1 if request.param is None else int(request.param)):
+        yield request.param
 
 
 # None: the library's own choice; 0: split kernel; 1..8: cluster kernel of that width

@@ -11,7 +11,7 @@ import torch
 
 from oracle import l4l_oracle as orc
 from paper_2608_21836_b200 import binding as l4l
-from helpers import Guarded
+from helpers import Guarded, nan_bf16
 
 pytestmark = pytest.mark.gpu
 SENTINEL = 0x4D4D
@@ -36,6 +36,7 @@ def check(y_gpu, st_gpu, y_ref, st_ref, valid):
     assert np.isfinite(got[valid]).all()
     assert err.max() <= 1e-2, f"max-abs {err.max():.3g}"
     assert err.mean() <= 1.5e-3, f"mean-abs {err.mean():.3g}"
+    assert torch.isfinite(st_gpu).all()
     serr = np.abs(st_gpu.cpu().double().numpy() - st_ref)
     assert serr.max() <= 5e-3, f"state max-abs {serr.max():.3g}"
 
@@ -50,6 +51,10 @@ def test_rglru_matches_oracle(B, T, W):
     if T > 40:
         pos[0, 37:] = torch.arange(T - 37, dtype=torch.int32)        # a second segment inside sequence 0
     lens = [T] + [max(1, T - 7 * i) for i in range(1, B)]
+    # rows past a sequence's length are caller memory that may hold anything: NaN there must reach neither y nor the state
+    dead = torch.arange(T).view(1, T, 1) >= torch.tensor(lens).view(B, 1, 1)
+    nan = nan_bf16((1,))
+    x, gx, ga = torch.where(dead, nan, x), torch.where(dead, nan, gx), torch.where(dead, nan, ga)
     y_ref, st_ref = orc.rglru(x, gx, ga, ap.numpy(), state=h0.double().numpy(), position=pos.numpy(), seq_len=lens)
     gy = Guarded(torch.full((B, T, W), SENTINEL, dtype=torch.int16).view(torch.bfloat16))
     gs = Guarded(h0)

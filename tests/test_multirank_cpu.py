@@ -53,6 +53,20 @@ def test_whole_job_value_is_additive_over_replicas_and_single_rank_needs_no_proc
     assert abs(bench.whole_job_value(8, 2.2e12, 2.0) - 8 * one) < 1e-9
 
 
+def test_plain_gpus_flag_starts_one_rank_per_gpu():
+    """`python bench.py --gpus N` without a launcher re-runs itself as N ranks on 127.0.0.1."""
+    sys.path.insert(0, ROOT)
+    import bench
+
+    cmd = bench.spawn_command(4, ["--gpus", "4", "--steps", "3"], port=29999)
+    assert cmd[1:3] == ["-m", "torch.distributed.run"]
+    assert "--nproc-per-node=4" in cmd and "--nnodes=1" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[cmd.index("--master-port") + 1] == "29999"
+    assert cmd[-5] == os.path.join(ROOT, "bench.py") and cmd[-4:] == ["--gpus", "4", "--steps", "3"]
+    # a port is found when none is given
+    assert int(bench.spawn_command(2, [])[bench.spawn_command(2, []).index("--master-port") + 1]) > 0
+
+
 # --------------------------------------------------------------------------- context-parallel decode plumbing
 def _lse_merge_f64(o_parts, lse_parts):
     """The merge formula in float64 torch ops (stand-in for the CUDA merge kernel on CPU ranks)."""
