@@ -266,7 +266,7 @@ def run_ours(args, rank, world):
     #   overlapped  N launches back to back between ONE pair of events: with programmatic stream serialization the
     #               prologue of a launch runs under the tail of the one before, so this mean is a pipelined rate
     #   pairs       the same loop with an event pair around every launch (median and best of the per-launch times)
-    #   single      one launch alone: a write of 1 GiB first (flushes L2, and keeps the GPU busy until the host has
+    #   single      one launch alone: a pass over 1 GiB first (flushes L2, and keeps the GPU busy until the host has
     #               the launch and both events queued), then event, launch, event; median and best over repeats
     caches = [(dck, dcv)] + [(dck.clone(), dcv.clone()) for _ in range(2)]
     n_dec = max(60, args.steps)
@@ -287,16 +287,19 @@ def run_ours(args, rank, world):
     barrier()
     t_dec_b2b = d0.elapsed_time(d1) / n_dec
 
-    def launch_times(fn, n, alone):
+    def launch_times(fn, n, alone, flush="read"):
         """Per-launch device times (ms) of n calls of fn(i): back to back with an event pair around each, or each
-        one alone behind a 1 GiB write."""
+        one alone behind an L2 flush over 1 GiB. flush = "read" (a reduction over the buffer: L2 ends up full of
+        clean lines, so the launch sees a cold cache and nothing else) or "write" (a memset: L2 ends up full of
+        DIRTY lines, whose write-back to HBM then competes with the launch's own traffic, as it does behind any
+        kernel that has just written a large output)."""
         pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
         if not alone:
             for _ in range(6):
                 filler.zero_()
         for i, (a, b) in enumerate(pairs):
             if alone:
-                filler.zero_()
+                filler.sum() if flush == "read" else filler.zero_()
             a.record()
             fn(i)
             b.record()
@@ -308,6 +311,7 @@ def run_ours(args, rank, world):
 
     dec_pairs = launch_times(decode_i, n_dec, alone=False)
     dec_single = launch_times(decode_i, 30, alone=True)
+    dec_single_dirty = launch_times(decode_i, 30, alone=True, flush="write")
     sampler = ClockSampler(local)
     sampler.start()
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
@@ -666,7 +670,11 @@ def run_ours(args, rank, world):
                    "pct_nominal_8000": 100 * dec_gbs_single / NOMINAL_GBS,
                    "pct_measured": 100 * dec_gbs_single / peaks["hbm_gbs"],
                    "single_launch_us": {"median": med(dec_single) * 1e3, "best": dec_single[0] * 1e3,
-                                        "launches": len(dec_single), "how": "1 GiB write, event, one launch, event"},
+                                        "launches": len(dec_single),
+                                        "how": "1 GiB read (L2 cold and clean), event, one launch, event",
+                                        "behind_a_1GiB_write_median": med(dec_single_dirty) * 1e3,
+                                        "behind_a_1GiB_write_note": "L2 full of dirty lines: their write-back shares "
+                                                                    "HBM with the launch"},
                    "event_pairs_us": {"median": med(dec_pairs) * 1e3, "best": dec_pairs[0] * 1e3,
                                       "launches": len(dec_pairs), "how": "back to back, an event pair around each launch"},
                    "overlapped_us": {"mean": t_dec_b2b * 1e3, "launches": n_dec, "kv_gbs": dec_gbs,

@@ -409,7 +409,8 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
         const int gcnt = BigG ? min(4, p.G - g0) : p.G;
         // sequences with no cached token get o = 0, lse = -inf (no tile ever refers to them)
         for (int b = blockIdx.x; fin == 0 && b < p.B; b += gridDim.x) {
-            if (p.kv_lens[b] <= 0) {
+            const int raw = p.kv_lens[b];
+            if (raw <= 0 || (p.k_new != nullptr && raw > p.max_kv_len)) {      // the same rule as the producer's clamp
                 for (int i = lane; i < p.Hq * D; i += 32) p.o[(size_t)b * p.Hq * D + i] = __float2bfloat16_rn(0.f);
                 if (p.lse)
                     for (int i = lane; i < p.Hq; i += 32) p.lse[(size_t)b * p.Hq + i] = -INFINITY;
