@@ -359,6 +359,13 @@ def run_ours(args, rank, world):
     del q_rot
     rope_bytes = 2 * q.numel() * 2 + 2 * (k.numel() + v.numel()) * 2       # q read + written, k/v read, cache written
     t_chunk = timed(lambda: l4l.l4l_attn_prefill_chunk(q, o, pk, pv, zeros_b, plens, wp.scale, ws_p), 5)
+    # a chunk of 4096 new tokens per sequence over 4096 cached ones, the chunk's K/V written by the same launch
+    half = S // 2
+    past_b = torch.full((Bp,), half, dtype=torch.int32, device=dev)
+    qlen_b = torch.full((Bp,), half, dtype=torch.int32, device=dev)
+    t_chunk_append = timed(lambda: l4l.l4l_attn_prefill_chunk_append(q[:, half:], k[:, half:], v[:, half:], o[:, half:], pk, pv,
+                                                                     past_b, qlen_b, wp.scale, ws_p), 5)
+    chunk_flops = 4 * D * Hq * Bp * (half * half + half * (half + 1) // 2)
     t_fused = timed(lambda: l4l.l4l_attn_decode_append(dq, do, dck, dcv, dkn, dvn, dlen, Lmax, wd.scale, ws_d), 20)
     # the whole decode step of a layer: rope + norm of the new token's q and k, append, attention: one launch, against
     # the three launches rope_kv_append (T = 1) + decode
@@ -701,6 +708,8 @@ def run_ours(args, rank, world):
                                     "frac_of_measured_hbm": rope_bytes / (t_rope * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                     "bytes": rope_bytes},
             "prefill_from_cache": {"ms": t_chunk, "tflops": pre_flops / (t_chunk * 1e-3) / 1e12},
+            "prefill_chunk_4096_over_4096_cached_with_fused_append": {"ms": t_chunk_append,
+                                                                      "tflops": chunk_flops / (t_chunk_append * 1e-3) / 1e12},
             "decode_with_fused_append": {"us": t_fused * 1e3, "kv_gbs": dec_bytes / (t_fused * 1e-3) / 1e9},
             "decode_step_rope_norm_append_attention": {"one_launch_us": t_step1 * 1e3, "two_launches_us": t_step3 * 1e3},
             "decode_paged_64": {"us": t_paged * 1e3, "kv_gbs": dec_bytes / (t_paged * 1e-3) / 1e9,

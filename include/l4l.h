@@ -16,7 +16,8 @@
  *   l4l_kv_append                : the cache update (an exact copy).
  *
  * Further entry points widen that path, each documented at its declaration:
- *   l4l_attn_prefill_chunk (new tokens over a populated cache), l4l_attn_decode_append (cache
+ *   l4l_attn_prefill_chunk (new tokens over a populated cache; _append / _paged_append with the cache
+ *   update fused in, over a contiguous or a paged cache), l4l_attn_decode_append (cache
  *   update fused into the decode step), l4l_rope_kv_append (rotary embedding and QK-norm fused
  *   with the cache update), l4l_attn_decode_paged / l4l_kv_append_paged / l4l_attn_decode_paged_append
  *   (page pool + block table), l4l_attn_decode_fp8 / l4l_kv_append_fp8 / l4l_attn_decode_append_fp8
@@ -299,8 +300,8 @@ l4l_status l4l_rope_kv_append(l4l_tensor4 q, l4l_tensor4 k_new, l4l_tensor4 v_ne
  * Causal prefill. For every sequence b with L = seq_lens[b] tokens, query head h, row i < L:
  *     o[b, i, h, :] = softmax_j( scale * q[b, i, h, :] . k[b, j, h/G, :],  j = 0..i ) @ v[b, 0..i, h/G, :]
  * and, when cache.k != NULL, cache slots 0..L-1 of sequence b receive k and v bit for bit
- * (the prompt starts an empty cache; prefill over an already populated cache is not
- * supported). Rows i >= L of o / lse and cache slots >= L are left untouched; q/k/v rows
+ * (the prompt starts an empty cache; for new tokens over a populated cache see
+ * l4l_attn_prefill_chunk_append). Rows i >= L of o / lse and cache slots >= L are left untouched; q/k/v rows
  * >= L may hold anything.
  *   q, o         [B, S_max, Hq, D] views       k, v   [B, S_max, Hkv, D] views
  *   d_seq_lens   device int32 [B], each 0 <= L <= S_max (and <= cache.max_len when caching)
@@ -330,6 +331,35 @@ l4l_status l4l_attn_prefill_chunk(l4l_tensor4 q, l4l_tensor4 o, l4l_kv_cache cac
                                   const int32_t *d_past_lens, const int32_t *d_q_lens, int S_max,
                                   int B, int Hq, int Hkv, int head_dim, float scale,
                                   float *d_lse, void *workspace, size_t ws_bytes, l4l_stream stream);
+
+/*
+ * The same chunk prefill with the cache update fused in (the paper's cache contract: the phase that produces
+ * tokens updates the state exactly once; here in the same launch, as l4l_attn_prefill does for a prompt). The
+ * chunk's K and V come from k_new / v_new; for sequence b with P = past_lens[b] and L = q_lens[b]:
+ *     cache slots P .. P+L-1 receive k_new[b, 0..L-1] and v_new[b, 0..L-1] bit for bit, and
+ *     o[b, i, h, :] = attention of q[b, i, h, :] over the cached tokens 0..P-1 and the new tokens 0..i.
+ * Equivalent to l4l_kv_append at slot P followed by l4l_attn_prefill_chunk. Cache slots below P are only read,
+ * slots from P+L on are neither read into a result nor written; new tokens whose slot lies outside the cache
+ * (P + i >= cache.max_len) are still attended (from k_new / v_new) but not stored. P = 0 is an ordinary prefill.
+ *   q, o          [B, S_max, Hq, D] views;   k_new, v_new  [B, S_max, Hkv, D] views (the chunk's tokens)
+ *   everything else as in l4l_attn_prefill_chunk
+ */
+l4l_status l4l_attn_prefill_chunk_append(l4l_tensor4 q, l4l_tensor4 k_new, l4l_tensor4 v_new, l4l_tensor4 o,
+                                         l4l_kv_cache cache, const int32_t *d_past_lens, const int32_t *d_q_lens,
+                                         int S_max, int B, int Hq, int Hkv, int head_dim, float scale,
+                                         float *d_lse, void *workspace, size_t ws_bytes, l4l_stream stream);
+
+/*
+ * l4l_attn_prefill_chunk_append over a paged cache (pool + block table, as in l4l_attn_decode_paged): the tokens
+ * cached before are read page by page, the chunk's K and V are written to the page slots the block table names.
+ * A slot whose table entry is not a page of the pool (or lies beyond table_stride entries) is read as zeros
+ * (only slots >= P can be in that state in a well-formed table) and is not written.
+ */
+l4l_status l4l_attn_prefill_chunk_paged_append(l4l_tensor4 q, l4l_tensor4 k_new, l4l_tensor4 v_new, l4l_tensor4 o,
+                                               l4l_paged_kv pool, const int32_t *d_block_table, int table_stride,
+                                               const int32_t *d_past_lens, const int32_t *d_q_lens, int S_max,
+                                               int B, int Hq, int Hkv, int head_dim, float scale,
+                                               float *d_lse, void *workspace, size_t ws_bytes, l4l_stream stream);
 
 /*
  * Decode. For every sequence b with n = kv_lens[b] cached tokens (the current token has

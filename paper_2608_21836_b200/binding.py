@@ -26,6 +26,7 @@ EXPORTS = (
     "l4l_kv_append_paged", "l4l_attn_decode_paged", "l4l_kv_append_fp8", "l4l_attn_decode_fp8", "l4l_rglru_scan", "l4l_rglru_workspace_bytes",
     "l4l_attn_decode_paged_fp8", "l4l_attn_merge", "l4l_attn_decode_rope_append", "l4l_attn_decode_paged_append",
     "l4l_attn_decode_paged_rope_append", "l4l_attn_decode_append_fp8", "l4l_attn_decode_paged_append_fp8",
+    "l4l_attn_prefill_chunk_append", "l4l_attn_prefill_chunk_paged_append",
     "l4l_decode_kernel_choice", "l4l_set_decode_override", "l4l_check_status", "l4l_selftest_wait_expiry",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
@@ -135,6 +136,12 @@ def load() -> ctypes.CDLL:
     lib.l4l_attn_prefill_chunk.restype = c_int
     lib.l4l_attn_prefill_chunk.argtypes = [Tensor4, Tensor4, KVCache, i32p, i32p, c_int, c_int, c_int, c_int, c_int,
                                            ctypes.c_float, vp, vp, c_size, vp]
+    lib.l4l_attn_prefill_chunk_append.restype = c_int
+    lib.l4l_attn_prefill_chunk_append.argtypes = [Tensor4, Tensor4, Tensor4, Tensor4, KVCache, i32p, i32p, c_int, c_int,
+                                                  c_int, c_int, c_int, ctypes.c_float, vp, vp, c_size, vp]
+    lib.l4l_attn_prefill_chunk_paged_append.restype = c_int
+    lib.l4l_attn_prefill_chunk_paged_append.argtypes = [Tensor4, Tensor4, Tensor4, Tensor4, PagedKV, i32p, c_int, i32p, i32p,
+                                                        c_int, c_int, c_int, c_int, c_int, ctypes.c_float, vp, vp, c_size, vp]
     lib.l4l_attn_decode_append.restype = c_int
     lib.l4l_attn_decode_append.argtypes = [vp, vp, KVCache, Tensor4, Tensor4, i32p, c_int, c_int, c_int, c_int, c_int,
                                            ctypes.c_float, vp, vp, c_size, vp]
@@ -314,6 +321,30 @@ def l4l_attn_prefill_chunk(q, o, cache_k, cache_v, past_lens, q_lens, scale: flo
                                        workspace.numel() * workspace.element_size(), _stream())
     if st != L4L_OK:
         raise L4LError(st, "l4l_attn_prefill_chunk")
+
+
+def l4l_attn_prefill_chunk_append(q, k_new, v_new, o, cache_k, cache_v, past_lens, q_lens, scale: float, workspace,
+                                  lse=None, block_table=None) -> None:
+    """Chunk of new tokens over a populated cache with the cache update fused in (one launch). q,o [B,S,Hq,D];
+    k_new, v_new [B,S,Hkv,D] go to slots past..past+q_len-1. With block_table (CUDA int32 [B, n]) cache_k / cache_v
+    are a page pool [pages,Hkv,page_size,D]; without it a contiguous cache [B,Hkv,max_len,D]."""
+    B, S, Hq, D = q.shape
+    Hkv = k_new.shape[2]
+    if lse is not None and not (lse.is_cuda and lse.dtype == torch.float32 and lse.is_contiguous()
+                                and tuple(lse.shape) == (B, Hq, S)):
+        raise TypeError("lse must be a contiguous CUDA float32 tensor [B, Hq, S]")
+    common = (_i32_dev(past_lens, "past_lens"), _i32_dev(q_lens, "q_lens"), S, B, Hq, Hkv, D, float(scale),
+              None if lse is None else lse.data_ptr(), workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+              _stream())
+    if block_table is None:
+        st = load().l4l_attn_prefill_chunk_append(tensor4(q, "q"), tensor4(k_new, "k_new"), tensor4(v_new, "v_new"),
+                                                  tensor4(o, "o"), kv_cache(cache_k, cache_v), *common)
+    else:
+        tbl, stride = _block_table(block_table, B)
+        st = load().l4l_attn_prefill_chunk_paged_append(tensor4(q, "q"), tensor4(k_new, "k_new"), tensor4(v_new, "v_new"),
+                                                        tensor4(o, "o"), paged_kv(cache_k, cache_v), tbl, stride, *common)
+    if st != L4L_OK:
+        raise L4LError(st, "l4l_attn_prefill_chunk_append")
 
 
 def _f32_dev(t, name: str, shape=None):

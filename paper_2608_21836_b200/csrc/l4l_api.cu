@@ -522,8 +522,10 @@ l4l_status l4l_attn_prefill(l4l_tensor4 q, l4l_tensor4 k, l4l_tensor4 v, l4l_ten
     }
     if (!workspace || ws_bytes < kStatusBytes) return L4L_ERR_WORKSPACE;
     if (B == 0 || S_max == 0) return L4L_OK;
-    return launch_prefill(q, k, v, o, cache, d_seq_lens, S_max, B, Hq, Hkv, head_dim, scale, d_lse, workspace,
-                          static_cast<cudaStream_t>(stream));
+    // a fresh prompt: every key comes from k / v, nothing is cached before; the cache (if given) is written
+    const PrefillKV kv{k, v, S_max, false, nullptr, nullptr, (cache.k && cache.v) ? &cache : nullptr};
+    return launch_prefill_tc(q, o, kv, d_seq_lens, nullptr, S_max, B, Hq, Hkv, head_dim, scale, d_lse, workspace,
+                             static_cast<cudaStream_t>(stream));
 }
 
 l4l_status l4l_attn_prefill_chunk(l4l_tensor4 q, l4l_tensor4 o, l4l_kv_cache cache, const int32_t *d_past_lens,
@@ -536,8 +538,49 @@ l4l_status l4l_attn_prefill_chunk(l4l_tensor4 q, l4l_tensor4 o, l4l_kv_cache cac
     if (!tensor4_ok(q) || !tensor4_ok(o) || !cache_ok(cache)) return L4L_ERR_INVALID_ARG;
     if (!workspace || ws_bytes < kStatusBytes) return L4L_ERR_WORKSPACE;
     if (B == 0 || S_max == 0) return L4L_OK;
-    return launch_prefill_chunk(q, o, cache, d_past_lens, d_q_lens, S_max, B, Hq, Hkv, head_dim, scale, d_lse,
-                                workspace, static_cast<cudaStream_t>(stream));
+    // the caller has appended the chunk already: its keys are read from the cache too, viewed as [B, slot, Hkv, D]
+    const l4l_tensor4 k{cache.k, cache.stride_b, cache.stride_t, cache.stride_h};
+    const l4l_tensor4 v{cache.v, cache.stride_b, cache.stride_t, cache.stride_h};
+    const PrefillKV kv{k, v, cache.max_len, true, &cache, nullptr, nullptr};
+    return launch_prefill_tc(q, o, kv, d_q_lens, d_past_lens, S_max, B, Hq, Hkv, head_dim, scale, d_lse, workspace,
+                             static_cast<cudaStream_t>(stream));
+}
+
+l4l_status l4l_attn_prefill_chunk_append(l4l_tensor4 q, l4l_tensor4 k_new, l4l_tensor4 v_new, l4l_tensor4 o,
+                                         l4l_kv_cache cache, const int32_t *d_past_lens, const int32_t *d_q_lens,
+                                         int S_max, int B, int Hq, int Hkv, int head_dim, float scale, float *d_lse,
+                                         void *workspace, size_t ws_bytes, l4l_stream stream)
+{
+    l4l_status st = shape_status(B, Hq, Hkv, head_dim);
+    if (st != L4L_OK) return st;
+    if (S_max < 0 || !d_past_lens || !d_q_lens) return L4L_ERR_INVALID_ARG;
+    if (!tensor4_ok(q) || !tensor4_ok(k_new) || !tensor4_ok(v_new) || !tensor4_ok(o) || !cache_ok(cache))
+        return L4L_ERR_INVALID_ARG;
+    if (!workspace || ws_bytes < kStatusBytes) return L4L_ERR_WORKSPACE;
+    if (B == 0 || S_max == 0) return L4L_OK;
+    const PrefillKV kv{k_new, v_new, S_max, false, &cache, nullptr, &cache};
+    return launch_prefill_tc(q, o, kv, d_q_lens, d_past_lens, S_max, B, Hq, Hkv, head_dim, scale, d_lse, workspace,
+                             static_cast<cudaStream_t>(stream));
+}
+
+l4l_status l4l_attn_prefill_chunk_paged_append(l4l_tensor4 q, l4l_tensor4 k_new, l4l_tensor4 v_new, l4l_tensor4 o,
+                                               l4l_paged_kv pool, const int32_t *d_block_table, int table_stride,
+                                               const int32_t *d_past_lens, const int32_t *d_q_lens, int S_max, int B,
+                                               int Hq, int Hkv, int head_dim, float scale, float *d_lse, void *workspace,
+                                               size_t ws_bytes, l4l_stream stream)
+{
+    l4l_status st = shape_status(B, Hq, Hkv, head_dim);
+    if (st != L4L_OK) return st;
+    if (S_max < 0 || !d_past_lens || !d_q_lens || !d_block_table || table_stride <= 0) return L4L_ERR_INVALID_ARG;
+    if (!tensor4_ok(q) || !tensor4_ok(k_new) || !tensor4_ok(v_new) || !tensor4_ok(o) || !pool_ok(pool))
+        return L4L_ERR_INVALID_ARG;
+    if (!workspace || ws_bytes < kStatusBytes) return L4L_ERR_WORKSPACE;
+    if (B == 0 || S_max == 0) return L4L_OK;
+    const l4l_kv_cache as_cache = pool_as_cache(pool);
+    const PagedTable pt{d_block_table, table_stride, pool.num_pages};
+    const PrefillKV kv{k_new, v_new, S_max, false, &as_cache, &pt, &as_cache};
+    return launch_prefill_tc(q, o, kv, d_q_lens, d_past_lens, S_max, B, Hq, Hkv, head_dim, scale, d_lse, workspace,
+                             static_cast<cudaStream_t>(stream));
 }
 
 l4l_status l4l_attn_decode(const void *q, void *o, l4l_kv_cache cache, const int32_t *d_kv_lens, int max_kv_len,

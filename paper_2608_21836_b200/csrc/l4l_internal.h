@@ -139,20 +139,21 @@ l4l_status launch_rglru_scan(const void *x, const void *gate_x, const void *gate
                              int W, void *workspace, size_t ws_bytes, cudaStream_t stream);
 size_t rglru_workspace_bytes(int B, int T, int W);
 
-l4l_status launch_prefill(const l4l_tensor4 &q, const l4l_tensor4 &k, const l4l_tensor4 &v,
-                          const l4l_tensor4 &o, const l4l_kv_cache &cache, const int32_t *d_seq_lens,
-                          int S_max, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
-                          void *workspace, cudaStream_t stream);
+// Where one prefill launch takes its keys and values from, and where it puts them.
+struct PrefillKV {
+    l4l_tensor4 k_new, v_new;     // K/V of the new tokens (a prompt, or a chunk) as [B, T, Hkv, D] views ...
+    int new_extent;               // ... with this many token rows
+    bool new_at_past;             // those views are the cache itself: row r of sequence b is slot past[b] + r
+    const l4l_kv_cache *past;     // the tokens cached before are read from here (a contiguous cache, or with `paged`
+                                  // the page pool: stride_b = stride between pages, max_len = page size); null: none
+    const PagedTable *paged;      // block table of a paged cache; null: contiguous
+    const l4l_kv_cache *write;    // the new tokens' K/V are written here in the same pass; null: nothing is written
+};
 
-// tcgen05 / tensor-memory prefill kernel. k, v: where the keys and values are read from, as [B, T, Hkv, D]
-// views with kv_extent token slots. d_past_lens (may be null): tokens ahead of the chunk, per sequence.
-l4l_status launch_prefill_tc(const l4l_tensor4 &q, const l4l_tensor4 &k, const l4l_tensor4 &v,
-                             const l4l_tensor4 &o, const l4l_kv_cache &cache, const int32_t *d_seq_lens,
-                             int S_max, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
-                             void *workspace, cudaStream_t stream, const int32_t *d_past_lens, int kv_extent);
-
-l4l_status launch_prefill_chunk(const l4l_tensor4 &q, const l4l_tensor4 &o, const l4l_kv_cache &cache,
-                                const int32_t *d_past_lens, const int32_t *d_q_lens, int S_max, int B, int Hq,
-                                int Hkv, int D, float scale, float *d_lse, void *workspace, cudaStream_t stream);
+// tcgen05 / tensor-memory prefill kernel: a fresh prompt (no past), or a chunk of new tokens over a populated
+// cache. d_past_lens (may be null): tokens ahead of the chunk, per sequence.
+l4l_status launch_prefill_tc(const l4l_tensor4 &q, const l4l_tensor4 &o, const PrefillKV &kv, const int32_t *d_seq_lens,
+                             const int32_t *d_past_lens, int S_max, int B, int Hq, int Hkv, int D, float scale,
+                             float *d_lse, void *workspace, cudaStream_t stream);
 
 }  // namespace l4l

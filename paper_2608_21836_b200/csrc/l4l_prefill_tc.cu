@@ -14,8 +14,12 @@
 //               from TMEM and V as an MN-major shared-memory operand; owns the TMEM allocation
 //   warps 10-11 help with the cache copy, which runs beside the last iterations
 //
-// The same kernel serves a chunk of new tokens over a populated cache (per-sequence offset `past`: row i is
-// position past + i, K/V come from the cache layout, the causal diagonal may then cross two tiles per sub-tile).
+// The same kernel serves a chunk of new tokens over a populated cache. The key axis of a sequence is then two runs
+// of 128-token tiles: the `past` tokens cached before (tiles of the cache, contiguous or paged, aligned to slot 0;
+// every query row sees all of them, the last tile may be partly filled) followed by the new tokens (tiles aligned
+// to the chunk's first token, so the causal diagonal sits exactly as in a fresh prompt, which is the case past = 0).
+// The new tokens' K/V come from the caller's tensors (and are written to the cache in the same pass) or, when the
+// caller has appended them already, from the cache itself at slot past + row.
 // A whole sub-tile's output leaves through the shared memory that held its Q rows and TMA stores.
 //
 // TMEM columns: S0 [0,128) S1 [128,256) O0 [256,256+D) O1 [256+D,256+2D); P_i aliases the first 64
@@ -48,16 +52,20 @@ struct TcCfg {
 struct TcParams {
     __nv_bfloat16 *o;
     int64_t o_sb, o_st, o_sh;
-    __nv_bfloat16 *cache_k, *cache_v;
-    int64_t c_sb, c_sh, c_st;
-    int cache_max_len;
-    const int32_t *seq_lens;
-    const int32_t *past_lens;   // null: fresh prompt (keys come from k/v); else keys come from the cache views
+    __nv_bfloat16 *cache_k, *cache_v;   // destination of the fused cache write (null: nothing is written)
+    int64_t c_sb, c_sh, c_st;           // its strides (paged: c_sb is the stride between pages)
+    int cache_slots;                    // token slots per sequence that may be written
+    const int32_t *seq_lens;            // [B] new tokens per sequence (prompt or chunk length)
+    const int32_t *past_lens;           // [B] tokens cached ahead of them, or null (none)
+    const int32_t *block_table;         // paged cache: [B, table_stride] page ids; null: contiguous cache
+    int table_stride, page_shift, page_size, num_pages;
+    int new_at_past;                    // the new tokens' K/V are read from the cache itself: row r is slot past + r
+    int cache_box_t;                    // token rows per TMA box of a cache tile (128, or the page size if smaller)
     float *lse;
     unsigned *status;
     int S_max, B, Hq, Hkv, G, n_qblocks;
     float scale_log2e;
-    TmapCoord cq, ckv, co;
+    TmapCoord cq, ckv, co, ckc;         // ckv: maps of the new tokens' K/V; ckc: maps of the cache (tokens before)
 };
 
 __device__ __forceinline__ void order_coords(const TmapCoord &c, int t, int h, int b, int &c1, int &c2, int &c3)
@@ -92,6 +100,7 @@ template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                   const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_o,
+                  const __grid_constant__ CUtensorMap tmap_kc, const __grid_constant__ CUtensorMap tmap_vc,
                   const TcParams p)
 {
     using C = TcCfg<D>;
@@ -151,31 +160,58 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     // TMEM is taken).
     const int L = L_raw < 0 ? 0 : (L_raw > p.S_max ? p.S_max : L_raw);
     if (q0 >= L) return;
-    // Tokens already in the cache ahead of this chunk (0 for a fresh prompt): query row i sees keys
-    // 0 .. past + i. kv_total keys exist in all.
+    // Tokens already in the cache ahead of these (0 for a fresh prompt): n_cache tiles, seen by every row.
     const int past = past_raw < 0 ? 0 : past_raw;
-    const int kv_total = past + L;
-    // sub-tile i (rows q0 + 128 i ..) visits K/V tiles 0 .. tile of its last valid row's last key
+    const int n_cache = (past + kRows - 1) / kRows;
+    // sub-tile i (rows q0 + 128 i ..) visits the tiles of the past and the new tokens' tiles up to its diagonal
     int n_sub[2];
-    n_sub[0] = (past + min(q0 + kRows - 1, L - 1)) / kRows + 1;
-    n_sub[1] = (q0 + kRows < L) ? (past + min(q0 + 2 * kRows - 1, L - 1)) / kRows + 1 : 0;
+    n_sub[0] = n_cache + min(q0 + kRows - 1, L - 1) / kRows + 1;
+    n_sub[1] = (q0 + kRows < L) ? n_cache + min(q0 + 2 * kRows - 1, L - 1) / kRows + 1 : 0;
     const int n_kv = max(n_sub[0], n_sub[1]);
     // Q and the first ring-ful of K/V tiles need no waiting: requested before the block-wide barrier
     const int n_pre = min(2 * n_kv, C::kSlots);
     auto request_tile = [&](int idx) {
         const uint32_t s = idx % C::kSlots;
+        const int j = idx >> 1;
+        uint8_t *dst = ring + (size_t)s * C::kTileBytes;
         int c1, c2, c3;
         mbar_arrive_expect_tx(&kv_full[s], C::kTileBytes);
-        order_coords(p.ckv, (idx >> 1) * kRows, kvh, b, c1, c2, c3);
-        const CUtensorMap *tm = (idx & 1) ? &tmap_v : &tmap_k;
+        if (j >= n_cache) {
+            // a tile of the new tokens
+            order_coords(p.ckv, (p.new_at_past ? past : 0) + (j - n_cache) * kRows, kvh, b, c1, c2, c3);
+            const CUtensorMap *tm = (idx & 1) ? &tmap_v : &tmap_k;
 #pragma unroll
-        for (int hf = 0; hf < C::kHalves; ++hf)
-            tma_load_4d(ring + (size_t)s * C::kTileBytes + hf * kHalfBytes, tm, &kv_full[s], hf * 64, c1, c2, c3);
+            for (int hf = 0; hf < C::kHalves; ++hf) tma_load_4d(dst + hf * kHalfBytes, tm, &kv_full[s], hf * 64, c1, c2, c3);
+        } else if (p.block_table == nullptr) {
+            // a tile of the tokens cached before, contiguous cache
+            order_coords(p.ckc, j * kRows, kvh, b, c1, c2, c3);
+            const CUtensorMap *tm = (idx & 1) ? &tmap_vc : &tmap_kc;
+#pragma unroll
+            for (int hf = 0; hf < C::kHalves; ++hf) tma_load_4d(dst + hf * kHalfBytes, tm, &kv_full[s], hf * 64, c1, c2, c3);
+        } else {
+            // ... paged cache: one box per page that the tile touches (a page never straddles tiles or boxes). A
+            // table entry outside the pool becomes an out-of-range coordinate, which reads zeros.
+            const CUtensorMap *tm = (idx & 1) ? &tmap_vc : &tmap_kc;
+            const int32_t *row = p.block_table + (size_t)b * p.table_stride;
+            for (int r0 = 0; r0 < kRows; r0 += p.cache_box_t) {
+                const int slot0 = j * kRows + r0, entry = slot0 >> p.page_shift;
+                int page = entry < p.table_stride ? __ldg(row + entry) : -1;
+                if (page < 0 || page >= p.num_pages) page = p.num_pages;
+                order_coords(p.ckc, slot0 & (p.page_size - 1), kvh, page, c1, c2, c3);
+#pragma unroll
+                for (int hf = 0; hf < C::kHalves; ++hf)
+                    tma_load_4d(dst + hf * kHalfBytes + r0 * 128, tm, &kv_full[s], hf * 64, c1, c2, c3);
+            }
+        }
     };
     if (producer_lane) {
         tma_prefetch_desc(&tmap_q);
         tma_prefetch_desc(&tmap_k);
         tma_prefetch_desc(&tmap_v);
+        if (n_cache > 0) {
+            tma_prefetch_desc(&tmap_kc);
+            tma_prefetch_desc(&tmap_vc);
+        }
         int c1, c2, c3;
         mbar_arrive_expect_tx(q_full, 2 * C::kTileBytes);
         order_coords(p.cq, q0, h, b, c1, c2, c3);
@@ -199,26 +235,36 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     tcgen05_fence_after_sync();
     const uint32_t tmem_base = *tmem_base_smem;
 
-    // The block's diagonal K/V tiles (2*qb and 2*qb+1) go to the cache (first query head of a KV group
-    // only, so each row is written once). They are the last tiles loaded, so their ring slots are never
-    // refilled; the copy runs beside the last iterations, shared by three warps. Rows >= L are not written.
+    // The block's diagonal K/V tiles (tiles 2*qb and 2*qb+1 of the new tokens) go to the cache, at slot past + row
+    // (first query head of a KV group only, so each row is written once). They are the last tiles loaded, so their
+    // ring slots are never refilled; the copy runs beside the last iterations, shared by three warps. Rows >= L
+    // and slots the cache does not have are not written.
     const bool writes_cache = p.cache_k != nullptr && (h % p.G) == 0;
     auto copy_diagonal_tiles = [&](int part) {
         if (!writes_cache) return;
-        const int lim = min(L, p.cache_max_len);
-        for (int j = 2 * qb; j < n_kv; ++j) {
+        for (int j = n_cache + 2 * qb; j < n_kv; ++j) {
+            const int r_base = (j - n_cache) * kRows;              // first row of the tile among the new tokens
             for (int kv = 0; kv < 2; ++kv) {
                 const int idx = 2 * j + kv;
                 const uint32_t s = idx % C::kSlots, ph = (idx / C::kSlots) & 1u;
                 if (!mbar_wait(&kv_full[s], ph, abort_flag)) return;
                 const uint8_t *src = ring + (size_t)s * C::kTileBytes;
-                __nv_bfloat16 *dst_base = (kv ? p.cache_v : p.cache_k) + b * p.c_sb + kvh * p.c_sh;
+                __nv_bfloat16 *dst_all = kv ? p.cache_v : p.cache_k;
                 constexpr int kChunks = D / 8;
-                const int rows = min(kRows, lim - j * kRows);
+                const int rows = min(min(kRows, L - r_base), p.cache_slots - past - r_base);
                 for (int i = part * 32 + lane; i < rows * kChunks; i += 96) {
                     const int r = i / kChunks, ch = i % kChunks;
+                    const int slot = past + r_base + r;
+                    __nv_bfloat16 *dst;
+                    if (p.block_table == nullptr) {
+                        dst = dst_all + b * p.c_sb + kvh * p.c_sh + (int64_t)slot * p.c_st;
+                    } else {
+                        const int page = __ldg(p.block_table + (size_t)b * p.table_stride + (slot >> p.page_shift));
+                        if (page < 0 || page >= p.num_pages) continue;          // no page behind this slot
+                        dst = dst_all + (int64_t)page * p.c_sb + kvh * p.c_sh + (int64_t)(slot & (p.page_size - 1)) * p.c_st;
+                    }
                     const uint4 val = *reinterpret_cast<const uint4 *>(src + (ch >> 3) * kHalfBytes + swz128(r, ch & 7));
-                    *reinterpret_cast<uint4 *>(dst_base + (int64_t)(j * kRows + r) * p.c_st + ch * 8) = val;
+                    *reinterpret_cast<uint4 *>(dst + ch * 8) = val;
                 }
             }
         }
@@ -300,7 +346,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
             const int iv = 2 * j + 1, ik = 2 * j + 2;
             const uint32_t sv = iv % C::kSlots, sk = ik % C::kSlots;
             if (!mbar_wait(&kv_full[sv], (iv / C::kSlots) & 1u, abort_flag)) { ok = false; break; }
-            const int first_dead = kv_total - j * kRows;          // V rows >= this hold no valid token
+            // V rows >= this hold no valid token (the partly filled last tile of the past, or of the new tokens)
+            const int first_dead = j < n_cache ? past - j * kRows : L - (j - n_cache) * kRows;
             if (first_dead < kRows) {
                 // may hold any bits (NaN included): clear, so that a zero weight times garbage cannot appear
                 uint8_t *vt = ring + (size_t)sv * C::kTileBytes;
@@ -347,7 +394,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
         const uint32_t tmem_s = tmem_base + lane_base + (i ? C::kColS1 : C::kColS0);
         const uint32_t tmem_o = tmem_base + lane_base + (i ? C::kColO1 : C::kColO0);
         const int n_mine = n_sub[i];
-        const int mask_from = (past + q0 + i * kRows) / kRows;   // first K/V tile that holds a key some row must not see
+        // Tiles that need a mask: the last tile of the past when it is partly filled (columns past its end, the same
+        // for every row), and the sub-tile's diagonal tile among the new tokens (row t sees columns 0..t).
+        const int j_ragged = (past & (kRows - 1)) ? n_cache - 1 : -1;
+        const int j_diag = n_cache + 2 * qb + i;
         const float c = p.scale_log2e;
         float m = -INFINITY, l = 0.f;
         bool ok = true;
@@ -363,10 +413,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
             // Row maximum of the scaled scores (log2 domain). Off the diagonal the maximum is taken over the
             // raw scores with independent 3-input max chains and scaled once (min for a negative scale);
             // on the diagonal tile the causal mask is applied to the scaled scores first.
-            const bool diag = (j >= mask_from);
+            const bool diag = (j == j_ragged) || (j >= j_diag);
             float mx;
             if (diag) {
-                const int lim = past + row - j * kRows;            // columns > lim are in the future
+                const int lim = (j == j_ragged) ? (past & (kRows - 1)) - 1 : t;   // columns > lim hold no visible key
                 float a0 = -INFINITY, a1 = -INFINITY, a2 = -INFINITY, a3 = -INFINITY;
 #pragma unroll
                 for (int qd = 0; qd < 4; ++qd)
@@ -530,7 +580,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
 
 template <int D>
 l4l_status launch_t(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const CUtensorMap &to,
-                    const TcParams &p, cudaStream_t stream)
+                    const CUtensorMap &tkc, const CUtensorMap &tvc, const TcParams &p, cudaStream_t stream)
 {
     using C = TcCfg<D>;
     static bool configured_on[kDeviceSlots] = {};
@@ -558,31 +608,56 @@ l4l_status launch_t(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensor
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, prefill_tc_kernel<D>, tq, tk, tv, to, p) == cudaSuccess ? L4L_OK : L4L_ERR_CUDA;
+    return cudaLaunchKernelEx(&cfg, prefill_tc_kernel<D>, tq, tk, tv, to, tkc, tvc, p) == cudaSuccess ? L4L_OK : L4L_ERR_CUDA;
 }
 
 }  // namespace
 
-l4l_status launch_prefill_tc(const l4l_tensor4 &q, const l4l_tensor4 &k, const l4l_tensor4 &v,
-                             const l4l_tensor4 &o, const l4l_kv_cache &cache, const int32_t *d_seq_lens,
-                             int S_max, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
-                             void *workspace, cudaStream_t stream, const int32_t *d_past_lens, int kv_extent)
+l4l_status launch_prefill_tc(const l4l_tensor4 &q, const l4l_tensor4 &o, const PrefillKV &kv, const int32_t *d_seq_lens,
+                             const int32_t *d_past_lens, int S_max, int B, int Hq, int Hkv, int D, float scale,
+                             float *d_lse, void *workspace, cudaStream_t stream)
 {
-    CUtensorMap tq, tk, tv, to;
-    TmapCoord cq, ck, cv, co;
+    CUtensorMap tq, tk, tv, to, tkc, tvc;
+    TmapCoord cq, ck, cv, co, ckc, cvc;
     if (!make_tmap_bf16(&tq, &cq, q.ptr, D, S_max, Hq, B, q.stride_t, q.stride_h, q.stride_b, 64, kRows) ||
         !make_tmap_bf16(&to, &co, o.ptr, D, S_max, Hq, B, o.stride_t, o.stride_h, o.stride_b, 64, kRows) ||
-        !make_tmap_bf16(&tk, &ck, k.ptr, D, kv_extent, Hkv, B, k.stride_t, k.stride_h, k.stride_b, 64, kRows) ||
-        !make_tmap_bf16(&tv, &cv, v.ptr, D, kv_extent, Hkv, B, v.stride_t, v.stride_h, v.stride_b, 64, kRows))
+        !make_tmap_bf16(&tk, &ck, kv.k_new.ptr, D, kv.new_extent, Hkv, B, kv.k_new.stride_t, kv.k_new.stride_h,
+                        kv.k_new.stride_b, 64, kRows) ||
+        !make_tmap_bf16(&tv, &cv, kv.v_new.ptr, D, kv.new_extent, Hkv, B, kv.v_new.stride_t, kv.v_new.stride_h,
+                        kv.v_new.stride_b, 64, kRows))
         return L4L_ERR_CUDA;
     if (ck.pos_t != cv.pos_t || ck.pos_h != cv.pos_h || ck.pos_b != cv.pos_b) return L4L_ERR_UNSUPPORTED;
-    TcParams p;
+    TcParams p = {};
+    // the tokens cached before: tiles of the cache (one box per tile), or of the page pool (one box per page if the
+    // pages are smaller than a tile); without a past the kernel never touches these two maps
+    tkc = tk; tvc = tv; ckc = ck;
+    p.cache_box_t = kRows;
+    if (kv.past) {
+        const l4l_kv_cache &c = *kv.past;
+        const int outer = kv.paged ? kv.paged->num_pages : B;
+        if (kv.paged && c.max_len < kRows) p.cache_box_t = c.max_len;
+        if (!make_tmap_bf16(&tkc, &ckc, c.k, D, c.max_len, Hkv, outer, c.stride_t, c.stride_h, c.stride_b, 64, p.cache_box_t) ||
+            !make_tmap_bf16(&tvc, &cvc, c.v, D, c.max_len, Hkv, outer, c.stride_t, c.stride_h, c.stride_b, 64, p.cache_box_t))
+            return L4L_ERR_CUDA;
+    }
     p.o = static_cast<__nv_bfloat16 *>(o.ptr);
     p.o_sb = o.stride_b; p.o_st = o.stride_t; p.o_sh = o.stride_h;
-    p.cache_k = static_cast<__nv_bfloat16 *>(cache.k);
-    p.cache_v = static_cast<__nv_bfloat16 *>(cache.v);
-    p.c_sb = cache.stride_b; p.c_sh = cache.stride_h; p.c_st = cache.stride_t;
-    p.cache_max_len = cache.max_len;
+    if (kv.write) {
+        p.cache_k = static_cast<__nv_bfloat16 *>(kv.write->k);
+        p.cache_v = static_cast<__nv_bfloat16 *>(kv.write->v);
+        p.c_sb = kv.write->stride_b; p.c_sh = kv.write->stride_h; p.c_st = kv.write->stride_t;
+        const long long slots = kv.paged ? (long long)kv.paged->table_stride * kv.write->max_len : kv.write->max_len;
+        p.cache_slots = slots > 0x7fffffffll ? 0x7fffffff : (int)slots;
+    }
+    if (kv.paged) {
+        const int page_size = kv.past ? kv.past->max_len : kv.write->max_len;
+        p.block_table = kv.paged->block_table;
+        p.table_stride = kv.paged->table_stride;
+        p.num_pages = kv.paged->num_pages;
+        p.page_size = page_size;
+        while ((1 << p.page_shift) < page_size) ++p.page_shift;
+    }
+    p.new_at_past = kv.new_at_past ? 1 : 0;
     p.seq_lens = d_seq_lens;
     p.past_lens = d_past_lens;
     p.lse = d_lse;
@@ -590,8 +665,8 @@ l4l_status launch_prefill_tc(const l4l_tensor4 &q, const l4l_tensor4 &k, const l
     p.S_max = S_max; p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.G = Hq / Hkv;
     p.n_qblocks = (S_max + 2 * kRows - 1) / (2 * kRows);
     p.scale_log2e = scale * 1.4426950408889634f;
-    p.cq = cq; p.ckv = ck; p.co = co;
-    return (D == 128) ? launch_t<128>(tq, tk, tv, to, p, stream) : launch_t<64>(tq, tk, tv, to, p, stream);
+    p.cq = cq; p.ckv = ck; p.co = co; p.ckc = ckc;
+    return (D == 128) ? launch_t<128>(tq, tk, tv, to, tkc, tvc, p, stream) : launch_t<64>(tq, tk, tv, to, tkc, tvc, p, stream);
 }
 
 }  // namespace l4l
