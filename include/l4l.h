@@ -264,6 +264,13 @@ l4l_status l4l_attn_merge(const void *o_parts, const float *d_lse_parts, int R, 
  *                status block: the state is handed from tile to tile on chip)
  */
 size_t l4l_rglru_workspace_bytes(int B, int T, int W);
+
+/*
+ * Channels per strip (64, 32 or 16) that l4l_rglru_scan would give one thread block for these sizes on the
+ * current device, without launching anything (for tests and tuning; no counterpart in the paper): narrower
+ * strips are taken when 64-channel ones would load the SMs unevenly. -1 for sizes the scan rejects.
+ */
+int l4l_rglru_strip_channels(int B, int T, int W);
 l4l_status l4l_rglru_scan(const void *x, const void *gate_x, const void *gate_a, const float *d_a_param,
                           const int32_t *d_position, const int32_t *d_seq_lens, float *d_state, void *y,
                           int B, int T, int W, void *workspace, size_t ws_bytes, l4l_stream stream);

@@ -26,7 +26,7 @@ EXPORTS = (
     "l4l_kv_append_paged", "l4l_attn_decode_paged", "l4l_kv_append_fp8", "l4l_attn_decode_fp8", "l4l_rglru_scan", "l4l_rglru_workspace_bytes",
     "l4l_attn_decode_paged_fp8", "l4l_attn_merge", "l4l_attn_decode_rope_append", "l4l_attn_decode_paged_append",
     "l4l_attn_decode_paged_rope_append", "l4l_attn_decode_append_fp8", "l4l_attn_decode_paged_append_fp8",
-    "l4l_attn_prefill_chunk_append", "l4l_attn_prefill_chunk_paged_append",
+    "l4l_attn_prefill_chunk_append", "l4l_attn_prefill_chunk_paged_append", "l4l_rglru_strip_channels",
     "l4l_decode_kernel_choice", "l4l_set_decode_override", "l4l_check_status", "l4l_selftest_wait_expiry",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
@@ -128,6 +128,8 @@ def load() -> ctypes.CDLL:
     lib.l4l_attn_merge.argtypes = [vp, vp, c_int, vp, vp, c_int, c_int, c_int, vp]
     lib.l4l_rglru_workspace_bytes.restype = c_size
     lib.l4l_rglru_workspace_bytes.argtypes = [c_int, c_int, c_int]
+    lib.l4l_rglru_strip_channels.restype = c_int
+    lib.l4l_rglru_strip_channels.argtypes = [c_int, c_int, c_int]
     lib.l4l_rglru_scan.restype = c_int
     lib.l4l_rglru_scan.argtypes = [vp, vp, vp, vp, i32p, i32p, vp, vp, c_int, c_int, c_int, vp, c_size, vp]
     lib.l4l_rope_kv_append.restype = c_int
@@ -643,6 +645,11 @@ def l4l_selftest_wait_expiry(workspace: torch.Tensor, budget_cycles: int = 10000
                                          int(budget_cycles), _stream())
     if st != L4L_OK:
         raise L4LError(st, "l4l_selftest_wait_expiry")
+
+
+def l4l_rglru_strip_channels(B: int, T: int, W: int) -> int:
+    """Channels per strip (64, 32 or 16) the scan would use for these sizes on the current device."""
+    return int(load().l4l_rglru_strip_channels(int(B), int(T), int(W)))
 
 
 def l4l_attn_merge(o_parts, lse_parts, o, lse=None) -> None:

@@ -487,6 +487,13 @@ l4l_status l4l_rglru_scan(const void *x, const void *gate_x, const void *gate_a,
                              ws_bytes, static_cast<cudaStream_t>(stream));
 }
 
+int l4l_rglru_strip_channels(int B, int T, int W)
+{
+    if (B <= 0 || T <= 0 || W <= 0 || W % 8 != 0) return -1;
+    const int split = rglru_strip_split(B, T, W);
+    return split == 0 ? 64 : 64 / split;
+}
+
 size_t l4l_rglru_workspace_bytes(int B, int T, int W)
 {
     if (B < 0 || T < 0 || W <= 0) return 0;

@@ -138,6 +138,9 @@ l4l_status launch_rglru_scan(const void *x, const void *gate_x, const void *gate
                              const int32_t *d_position, const int32_t *d_seq_lens, float *d_state, void *y, int B, int T,
                              int W, void *workspace, size_t ws_bytes, cudaStream_t stream);
 size_t rglru_workspace_bytes(int B, int T, int W);
+// the scan's shape for these sizes on the current device: 0 = 64-channel strips, teams of 16 warps; 1, 2, 4 = teams of
+// 8 warps on strips of 64, 32, 16 channels
+int rglru_strip_split(int B, int T, int W);
 
 // Where one prefill launch takes its keys and values from, and where it puts them.
 struct PrefillKV {

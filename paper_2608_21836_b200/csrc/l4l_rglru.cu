@@ -18,6 +18,13 @@
 // 8 bytes per (step, channel) move through HBM (3 bf16 read, 1 written) against 4 MUFU operations per
 // channel (two tanh.approx sigmoids, ex2.approx, sqrt.approx) and about 25 issued instructions per channel
 // pair and step.
+//
+// Narrow strips (template parameter kSplit = 2 or 4). A strip is one serial chain, so a launch is as long as the
+// most loaded SM's chains: 160 strips on 148 SMs put two on twelve SMs and take twice the time of 148. For such
+// launches the strips are made 32 or 16 channels wide, and a warp then owns kSplit CONSECUTIVE time tiles at once:
+// lane = (sub-tile, channel pair), so every instruction still does 32 lanes' worth of work. Everything per lane is
+// unchanged; the start states of a warp's later sub-tiles come from the earlier ones by kSplit - 1 shuffles
+// (h <- A h + E) inside step 3. Twice or four times as many CTAs of half or a quarter of the work spread evenly.
 #include <type_traits>
 
 #include "l4l_internal.h"
@@ -28,9 +35,9 @@ namespace l4l {
 namespace {
 
 constexpr int kTb = 16;          // time steps per tile
-constexpr int kCb = 64;          // channels per CTA (two per lane)
+constexpr int kCb = 64;          // channels per CTA at kSplit = 1 (two per lane); kCb / kSplit otherwise
 constexpr int kStages = 2;       // TMA buffers per warp
-constexpr uint32_t kArrayBytes = kTb * kCb * 2;
+constexpr uint32_t kArrayBytes = kTb * kCb * 2;   // one array of a warp's tile: (kTb * kSplit) steps x (kCb / kSplit) channels
 constexpr uint32_t kStageBytes = 3 * kArrayBytes;
 // kTeam warps per CTA, each taking every kTeam-th tile: 8 for sequences, 16 when the launch has no more strips
 // than the GPU has SMs (one CTA per SM then, and a strip's rate is set by how many tiles it has in flight),
@@ -67,7 +74,7 @@ __device__ __forceinline__ float sqrt_approx(float x)
 // two bf16 in one word -> packed fp32x2 (low half first)
 __device__ __forceinline__ uint64_t widen2(uint32_t w) { return pack_u32x2(w << 16, w & 0xffff0000u); }
 
-template <int kTeam>
+template <int kTeam, int kSplit>
 __global__ void __launch_bounds__(kTeam * 32)
 rglru_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_gx,
                   const __grid_constant__ CUtensorMap tmap_ga, const RglruParams p)
@@ -80,12 +87,16 @@ rglru_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     float *carry = reinterpret_cast<float *>(handed + kTeam);                  // [2][kCb]: start state of tile j in slot j & 1
     volatile int *abort_flag = reinterpret_cast<volatile int *>(carry + 2 * kCb);
 
+    constexpr int kCw = kCb / kSplit;                    // channels of this CTA's strip
+    constexpr int kPairs = kCw / 2;                      // lanes per sub-tile (one channel pair each)
+    constexpr int kSteps = kTb * kSplit;                 // time steps a warp owns at a time (kSplit sub-tiles of kTb)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int b = blockIdx.y, c0 = blockIdx.x * kCb;
+    const int sub = lane / kPairs, cp = lane % kPairs;   // this lane's sub-tile and channel pair
+    const int b = blockIdx.y, c0 = blockIdx.x * kCw;
     int L = p.seq_lens ? p.seq_lens[b] : p.T;
     L = L < 0 ? 0 : (L > p.T ? p.T : L);
-    const int n_tiles = (L + kTb - 1) / kTb;
-    const int c = c0 + 2 * lane;
+    const int n_tiles = (L + kSteps - 1) / kSteps;
+    const int c = c0 + 2 * cp;
     const bool live = c < p.W;                           // W is even: both channels or neither
 
     if (threadIdx.x == 0) {
@@ -95,9 +106,9 @@ rglru_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         fence_barrier_init();
         fence_proxy_async_smem();
     }
-    if (warp == 0) {
+    if (warp == 0 && sub == 0) {
         const float2 st = live ? *reinterpret_cast<const float2 *>(p.state + (size_t)b * p.W + c) : make_float2(0.f, 0.f);
-        *reinterpret_cast<float2 *>(carry + 2 * lane) = st;                    // slot 0: the caller's state starts tile 0
+        *reinterpret_cast<float2 *>(carry + 2 * cp) = st;                      // slot 0: the caller's state starts tile 0
     }
     __syncthreads();
     if (threadIdx.x == 0) mbar_arrive(&handed[0]);
@@ -112,9 +123,9 @@ rglru_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             const uint32_t s = k % kStages;
             mbar_arrive_expect_tx(&my_full[s], kStageBytes);
             uint8_t *dst = my_stages + s * kStageBytes;
-            tma_load_3d(dst, &tmap_x, &my_full[s], c0, tile * kTb, b);
-            tma_load_3d(dst + kArrayBytes, &tmap_gx, &my_full[s], c0, tile * kTb, b);
-            tma_load_3d(dst + 2 * kArrayBytes, &tmap_ga, &my_full[s], c0, tile * kTb, b);
+            tma_load_3d(dst, &tmap_x, &my_full[s], c0, tile * kSteps, b);
+            tma_load_3d(dst + kArrayBytes, &tmap_gx, &my_full[s], c0, tile * kSteps, b);
+            tma_load_3d(dst + 2 * kArrayBytes, &tmap_ga, &my_full[s], c0, tile * kSteps, b);
         }
     };
     if (lane == 0) {
@@ -139,11 +150,17 @@ rglru_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     uint32_t *yrow = reinterpret_cast<uint32_t *>(p.y + (size_t)b * p.T * p.W + c);
     const size_t y_step = (size_t)p.W / 2;               // 32-bit words between time steps
     auto resets_of = [&](int tile) -> unsigned {
-        // bit t: step tile*kTb + t is the first token of a segment (position 0)
+        // bit t: step t of THIS LANE'S sub-tile is the first token of a segment (position 0)
         if (!p.position || tile >= n_tiles) return 0u;
-        const int t = tile * kTb + lane;
-        const int pos = (lane < kTb && t < L) ? __ldg(p.position + (size_t)b * p.T + t) : 1;
-        return __ballot_sync(0xffffffffu, pos == 0);
+        unsigned mine = 0u;
+#pragma unroll
+        for (int part = 0; part < (kSteps + 31) / 32; ++part) {
+            const int t = tile * kSteps + part * 32 + lane;
+            const int pos = (part * 32 + lane < kSteps && t < L) ? __ldg(p.position + (size_t)b * p.T + t) : 1;
+            const unsigned bits = __ballot_sync(0xffffffffu, pos == 0);
+            if ((sub * kTb) / 32 == part) mine = (bits >> ((sub * kTb) % 32)) & 0xffffu;
+        }
+        return mine;
     };
     unsigned reset_next = resets_of(warp);
 
@@ -152,10 +169,11 @@ rglru_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         const unsigned resets = reset_next;
         reset_next = resets_of(tile + kTeam);            // in flight while this tile is processed
         if (!mbar_wait(&my_full[s], ph, abort_flag)) break;
-        const uint32_t *xs = reinterpret_cast<const uint32_t *>(my_stages + s * kStageBytes) + lane;
+        // the tile in shared memory: kSteps rows of kPairs words; this lane reads rows sub * kTb .. of column cp
+        const uint32_t *xs = reinterpret_cast<const uint32_t *>(my_stages + s * kStageBytes) + sub * kTb * kPairs + cp;
         const uint32_t *gxs = xs + kTb * kCb / 2, *gas = gxs + kTb * kCb / 2;
-        const int t0 = tile * kTb;
-        const int n = min(kTb, L - t0);
+        const int t0 = tile * kSteps + sub * kTb;            // first step of this lane's sub-tile
+        const int n = max(0, min(kTb, L - t0));
         // ---- a_t and b_t = m_t i_t x_t of all steps of the tile (independent of the state). Tiles without a
         // reset and without a ragged end (nearly all) take the version without the per-step selects.
         uint64_t av[kTb], bv[kTb];
@@ -163,10 +181,10 @@ rglru_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             constexpr bool kPlain = decltype(plain_tag)::value;
 #pragma unroll
             for (int t = 0; t < kTb; ++t) {
-                const uint64_t xv = widen2(xs[t * (kCb / 2)]);
+                const uint64_t xv = widen2(xs[t * kPairs]);
                 float g0, g1, r0, r1;
-                unpack_f32x2(mul_f32x2(widen2(gxs[t * (kCb / 2)]), half2), g0, g1);
-                unpack_f32x2(mul_f32x2(widen2(gas[t * (kCb / 2)]), half2), r0, r1);
+                unpack_f32x2(mul_f32x2(widen2(gxs[t * kPairs]), half2), g0, g1);
+                unpack_f32x2(mul_f32x2(widen2(gas[t * kPairs]), half2), r0, r1);
                 const uint64_t th_x = pack_f32x2(tanh_approx(g0), tanh_approx(g1));   // sigmoid = 0.5 tanh(z/2) + 0.5
                 const uint64_t th_a = pack_f32x2(tanh_approx(r0), tanh_approx(r1));
                 const uint64_t la2 = fma_f32x2(th_a, k2h, k2h);                        // log2(a) = k2 * sigmoid(gate_a)
@@ -182,7 +200,7 @@ rglru_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 unpack_f32x2(z, z0, z1);
                 float m0 = sqrt_approx(z0 > -0.0625f ? s0 : d0), m1 = sqrt_approx(z1 > -0.0625f ? s1 : d1);
                 if constexpr (!kPlain) {
-                    if ((resets >> t) & 1u) {                                          // uniform across the warp
+                    if ((resets >> t) & 1u) {                                          // uniform across a sub-tile's lanes
                         a = zero2;
                         m0 = m1 = 1.f;
                     }
@@ -200,7 +218,7 @@ rglru_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 }
             }
         };
-        if (resets == 0u && n == kTb)
+        if (__all_sync(0xffffffffu, resets == 0u && n == kTb))
             gates(std::true_type{});
         else
             gates(std::false_type{});
@@ -219,21 +237,31 @@ rglru_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         // warp cannot reach its next arrival here before this warp has handed the present tile on, so the
         // phases are seen one by one.
         if (!mbar_wait(&handed[warp], k & 1u, abort_flag)) break;
-        const float2 hs = *reinterpret_cast<const float2 *>(carry + (tile & 1) * kCb + 2 * lane);
-        uint64_t h2 = pack_f32x2(hs.x, hs.y);
+        const float2 hs = *reinterpret_cast<const float2 *>(carry + (tile & 1) * kCb + 2 * cp);
+        uint64_t h2 = pack_f32x2(hs.x, hs.y);                                  // start state of the warp's first sub-tile
         {
+            // start states of the later sub-tiles, and the end state of the warp's steps: h <- A h + E along the
+            // sub-tiles, the state travelling kPairs lanes up at each step
             float e0, e1;
             unpack_f32x2(fma_f32x2(A, h2, E), e0, e1);
-            *reinterpret_cast<float2 *>(carry + ((tile + 1) & 1) * kCb + 2 * lane) = make_float2(e0, e1);
+#pragma unroll
+            for (int u = 1; u < kSplit; ++u) {
+                const float i0 = __shfl_up_sync(0xffffffffu, e0, kPairs), i1 = __shfl_up_sync(0xffffffffu, e1, kPairs);
+                if (sub == u) {
+                    h2 = pack_f32x2(i0, i1);
+                    unpack_f32x2(fma_f32x2(A, h2, E), e0, e1);
+                }
+            }
+            if (sub == kSplit - 1) *reinterpret_cast<float2 *>(carry + ((tile + 1) & 1) * kCb + 2 * cp) = make_float2(e0, e1);
             __syncwarp();
             if (lane == 0) mbar_arrive(&handed[(warp + 1) % kTeam]);           // release: the slot is written
-            if (tile + 1 == n_tiles && live)                                   // the sequence ends here
+            if (tile + 1 == n_tiles && live && sub == kSplit - 1)              // the sequence ends here
                 *reinterpret_cast<float2 *>(p.state + (size_t)b * p.W + c) = make_float2(e0, e1);
         }
         // ---- the recurrence proper, one packed FMA per step, and the outputs
 #pragma unroll
         for (int t = 0; t < kTb; ++t) {
-            if (t < n) {                                                       // uniform across the warp
+            if (t < n) {                                                       // uniform across a sub-tile's lanes
                 h2 = fma_f32x2(av[t], h2, bv[t]);
                 float h0, h1;
                 unpack_f32x2(h2, h0, h1);
@@ -249,47 +277,81 @@ rglru_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
 
 size_t rglru_workspace_bytes(int, int, int) { return kStatusBytes; }
 
+namespace {
+
+template <int kTeam, int kSplit>
+l4l_status launch_shape(const void *x, const void *gate_x, const void *gate_a, const RglruParams &p, cudaStream_t stream)
+{
+    // one opt-in per instantiation and device
+    static bool configured_on[kDeviceSlots] = {};
+    const int slot = device_slot();
+    if (slot < 0) return L4L_ERR_CUDA;
+    {
+        std::lock_guard<std::mutex> lock(setup_mutex());
+        if (!configured_on[slot]) {
+            if (cudaFuncSetAttribute(rglru_scan_kernel<kTeam, kSplit>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)smem_bytes(kTeam)) != cudaSuccess)
+                return L4L_ERR_CUDA;
+            configured_on[slot] = true;
+        }
+    }
+    constexpr int kCw = kCb / kSplit;
+    CUtensorMap tx, tgx, tga;
+    if (!make_tmap_rows_bf16(&tx, x, p.W, p.T, p.B, p.W, (int64_t)p.T * p.W, kCw, kTb * kSplit) ||
+        !make_tmap_rows_bf16(&tgx, gate_x, p.W, p.T, p.B, p.W, (int64_t)p.T * p.W, kCw, kTb * kSplit) ||
+        !make_tmap_rows_bf16(&tga, gate_a, p.W, p.T, p.B, p.W, (int64_t)p.T * p.W, kCw, kTb * kSplit))
+        return L4L_ERR_CUDA;
+    const dim3 grid((p.W + kCw - 1) / kCw, p.B);
+    rglru_scan_kernel<kTeam, kSplit><<<grid, kTeam * 32, smem_bytes(kTeam), stream>>>(tx, tgx, tga, p);
+    return cudaGetLastError() == cudaSuccess ? L4L_OK : L4L_ERR_CUDA;
+}
+
+}  // namespace
+
 l4l_status launch_rglru_scan(const void *x, const void *gate_x, const void *gate_a, const float *d_a_param,
                              const int32_t *d_position, const int32_t *d_seq_lens, float *d_state, void *y, int B, int T,
                              int W, void *workspace, size_t, cudaStream_t stream)
 {
-    CUtensorMap tx, tgx, tga;
-    if (!make_tmap_rows_bf16(&tx, x, W, T, B, W, (int64_t)T * W, kCb, kTb) ||
-        !make_tmap_rows_bf16(&tgx, gate_x, W, T, B, W, (int64_t)T * W, kCb, kTb) ||
-        !make_tmap_rows_bf16(&tga, gate_a, W, T, B, W, (int64_t)T * W, kCb, kTb))
-        return L4L_ERR_CUDA;
-    static bool configured_on[kDeviceSlots] = {};
-    static int sm_count_on[kDeviceSlots] = {};
-    const int slot = device_slot();
-    if (slot < 0) return L4L_ERR_CUDA;
-    int sm_count;
-    {
-        std::lock_guard<std::mutex> lock(setup_mutex());
-        bool &configured = configured_on[slot];
-        if (!configured) {
-            if (cudaDeviceGetAttribute(&sm_count_on[slot], cudaDevAttrMultiProcessorCount, slot) != cudaSuccess ||
-                cudaFuncSetAttribute(rglru_scan_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)smem_bytes(8)) != cudaSuccess ||
-                cudaFuncSetAttribute(rglru_scan_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)smem_bytes(16)) != cudaSuccess)
-                return L4L_ERR_CUDA;
-            configured = true;
-        }
-        sm_count = sm_count_on[slot];
-    }
     RglruParams p;
     p.a_param = d_a_param; p.position = d_position; p.seq_lens = d_seq_lens; p.state = d_state;
     p.y = static_cast<__nv_bfloat16 *>(y);
     p.status = static_cast<unsigned *>(workspace);
     p.B = B; p.T = T; p.W = W;
-    const dim3 grid((W + kCb - 1) / kCb, B);
-    if (T <= kTb)
-        rglru_scan_kernel<1><<<grid, 32, smem_bytes(1), stream>>>(tx, tgx, tga, p);
-    else if ((long long)grid.x * grid.y <= sm_count && T >= 16 * 2 * kTb)
-        rglru_scan_kernel<16><<<grid, 16 * 32, smem_bytes(16), stream>>>(tx, tgx, tga, p);
-    else
-        rglru_scan_kernel<8><<<grid, 8 * 32, smem_bytes(8), stream>>>(tx, tgx, tga, p);
-    return cudaGetLastError() == cudaSuccess ? L4L_OK : L4L_ERR_CUDA;
+    if (T <= kTb) return launch_shape<1, 1>(x, gate_x, gate_a, p, stream);
+    const int split = rglru_strip_split(B, T, W);
+    if (split == 0) return launch_shape<16, 1>(x, gate_x, gate_a, p, stream);
+    if (split == 4) return launch_shape<8, 4>(x, gate_x, gate_a, p, stream);
+    if (split == 2) return launch_shape<8, 2>(x, gate_x, gate_a, p, stream);
+    return launch_shape<8, 1>(x, gate_x, gate_a, p, stream);
+}
+
+// 0: 64-channel strips with teams of 16 warps; 1, 2, 4: teams of 8 warps on strips of 64, 32, 16 channels.
+int rglru_strip_split(int B, int T, int W)
+{
+    if (T <= kTb) return 1;
+    const long long sms = sm_count();
+    // A strip is a serial chain that keeps an SM's issue slots busy, so a launch takes as long as the most loaded
+    // SM. Estimated time of that SM, in units of one 64-channel strip on an SM of its own: k CTAs of 1/s strip each
+    // take k / s; a lone team of 8 warps reaches about three quarters of the issue rate that two co-resident teams
+    // or one team of 16 warps reach.
+    auto fullest = [&](int s) { return ((long long)((W + kCb / s - 1) / (kCb / s)) * B + sms - 1) / sms; };
+    int best = 1;
+    double best_time = fullest(1) >= 2 ? (double)fullest(1) : 1.0 / 0.74;
+    if (fullest(1) == 1 && T >= 16 * 2 * kTb) {
+        best = 0;
+        best_time = 1.0;
+    }
+    // narrower strips have to win by a tenth or more (their warps pay two or four dependent steps in the hand-off
+    // instead of one), and the sequence has to be long enough for their wider tiles
+    for (int s = 2; s <= 4; s *= 2) {
+        const long long k = fullest(s);
+        const double time = k >= 2 ? (double)k / s : (1.0 / s) / 0.74;
+        if (time < 0.9 * best_time && T >= 8 * kTb * s) {
+            best = s;
+            best_time = time;
+        }
+    }
+    return best;
 }
 
 }  // namespace l4l

@@ -41,11 +41,16 @@ def check(y_gpu, st_gpu, y_ref, st_ref, valid):
     assert serr.max() <= 5e-3, f"state max-abs {serr.max():.3g}"
 
 
-@pytest.mark.parametrize("B,T,W", [(2, 300, 2560), (1, 1237, 200), (3, 65, 40), (1, 1, 64), (5, 1000, 96), (1, 16, 64), (2, 17, 128)])
+@pytest.mark.parametrize("B,T,W", [(2, 300, 2560), (1, 1237, 200), (3, 65, 40), (1, 1, 64), (5, 1000, 96), (1, 16, 64), (2, 17, 128),
+                                   (4, 300, 2560), (4, 600, 2560), (5, 520, 2440), (19, 530, 512)])
 def test_rglru_matches_oracle(B, T, W):
     """Sequences of many tiles (eight warps hand the state on from tile to tile), of exactly one tile (the one-warp
     variant) and just past it; a second segment inside a sequence, ragged lengths, a channel count that does not fill
-    the last 64-channel strip."""
+    the last strip; launches of 149 to 200 strips, which the library cuts into 32- or 16-channel strips (a warp
+    then owns two or four consecutive time tiles)."""
+    if (B, W) in ((4, 2560), (5, 2440), (19, 512)):                    # 160, 195 and 152 strips at 64 channels
+        assert l4l.l4l_rglru_strip_channels(B, T, W) in (16, 32)
+        assert l4l.l4l_rglru_strip_channels(4, 600, 2560) == 16 and l4l.l4l_rglru_strip_channels(4, 300, 2560) == 32
     x, gx, ga, ap, h0 = make(B, T, W, 1100 + T)
     pos = torch.arange(T, dtype=torch.int32).repeat(B, 1)
     if T > 40:
