@@ -1,8 +1,10 @@
 // Causal prefill on the 5th-generation tensor cores (tcgen05.mma, accumulators in tensor memory).
 //
-// One CTA owns 256 consecutive query rows of one (sequence, query head): two 128-row sub-tiles
-// whose S = Q K^T and O += P V products ping-pong on the tensor pipe while the other sub-tile's
-// softmax runs on the CUDA cores.
+// One CTA owns two 128-row sub-tiles whose S = Q K^T and O += P V products ping-pong on the tensor
+// pipe while the other sub-tile's softmax runs on the CUDA cores. The two sub-tiles are the same 128
+// query rows of TWO query heads that share a KV head (query-head groups of even size: both sub-tiles
+// then visit the same K/V tiles, their causal spans are equal, and work items are half as coarse), or
+// 256 consecutive rows of ONE query head (odd group sizes, multi-head attention included).
 //
 //   warps 0-3   softmax of sub-tile 0: thread t owns row t (= TMEM lane t): reads S from TMEM,
 //               keeps the running max / sum in fp32, writes P (bf16) back into TMEM over S
@@ -64,6 +66,7 @@ struct TcParams {
     float *lse;
     unsigned *status;
     int S_max, B, Hq, Hkv, G, n_qblocks;
+    int pair_heads;                     // the two sub-tiles are two query heads of one KV group at the same 128 rows
     float scale_log2e;
     TmapCoord cq, ckv, co, ckc;         // ckv: maps of the new tokens' K/V; ckc: maps of the cache (tokens before)
 };
@@ -106,16 +109,22 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     using C = TcCfg<D>;
     // ---- which block: heaviest (longest causal span) blocks first, heads of a KV group adjacent
     grid_dependency_wait();                       // seq_lens may have been written by the previous kernel
-    const int per_block = p.Hq * p.B;
-    const int qb = p.n_qblocks - 1 - (int)(blockIdx.x / per_block);
+    // pair mode: sub-tile i is query head h + i at rows q0 ..; else: head h at rows q0 + 128 i ..
+    const bool pair = p.pair_heads != 0;
+    const int heads = pair ? p.Hq / 2 : p.Hq;
+    const int per_block = heads * p.B;
+    const int qb = p.n_qblocks - 1 - (int)(blockIdx.x / per_block);     // block of 128 (pair mode) or 256 rows
     const int hb = blockIdx.x % per_block;
-    const int h = hb % p.Hq, b = hb / p.Hq;
+    const int h = pair ? 2 * (hb % heads) : hb % heads, b = hb / heads;
     const int kvh = h / p.G;
+    const int sub_rows = pair ? 0 : kRows;                // rows between the two sub-tiles
+    const int sub_heads = pair ? 1 : 0;                   // heads between them
+    const int diag0 = pair ? qb : 2 * qb;                 // tile (among the new tokens) of sub-tile 0's diagonal
     // The two lengths are requested now and first looked at after the barrier / TMEM set-up below, so that
     // their latency is hidden behind it.
     const int L_raw = __ldg(p.seq_lens + b);
     const int past_raw = p.past_lens ? __ldg(p.past_lens + b) : 0;
-    const int q0 = qb * 2 * kRows;
+    const int q0 = qb * (pair ? kRows : 2 * kRows);
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -166,7 +175,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     // sub-tile i (rows q0 + 128 i ..) visits the tiles of the past and the new tokens' tiles up to its diagonal
     int n_sub[2];
     n_sub[0] = n_cache + min(q0 + kRows - 1, L - 1) / kRows + 1;
-    n_sub[1] = (q0 + kRows < L) ? n_cache + min(q0 + 2 * kRows - 1, L - 1) / kRows + 1 : 0;
+    n_sub[1] = (q0 + sub_rows < L) ? n_cache + min(q0 + sub_rows + kRows - 1, L - 1) / kRows + 1 : 0;
     const int n_kv = max(n_sub[0], n_sub[1]);
     // Q and the first ring-ful of K/V tiles need no waiting: requested before the block-wide barrier
     const int n_pre = min(2 * n_kv, C::kSlots);
@@ -218,7 +227,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
 #pragma unroll
         for (int hf = 0; hf < C::kHalves; ++hf) tma_load_4d(q_smem + hf * kHalfBytes, &tmap_q, q_full, hf * 64, c1, c2, c3);
         request_tile(0);                                   // K_0 right behind Q_0: the first product needs both
-        order_coords(p.cq, q0 + kRows, h, b, c1, c2, c3);
+        order_coords(p.cq, q0 + sub_rows, h + sub_heads, b, c1, c2, c3);
 #pragma unroll
         for (int hf = 0; hf < C::kHalves; ++hf)
             tma_load_4d(q_smem + C::kTileBytes + hf * kHalfBytes, &tmap_q, q_full, hf * 64, c1, c2, c3);
@@ -235,14 +244,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     tcgen05_fence_after_sync();
     const uint32_t tmem_base = *tmem_base_smem;
 
-    // The block's diagonal K/V tiles (tiles 2*qb and 2*qb+1 of the new tokens) go to the cache, at slot past + row
+    // The block's diagonal K/V tiles (one or two tiles of the new tokens, from diag0 on) go to the cache, at slot past + row
     // (first query head of a KV group only, so each row is written once). They are the last tiles loaded, so their
     // ring slots are never refilled; the copy runs beside the last iterations, shared by three warps. Rows >= L
     // and slots the cache does not have are not written.
     const bool writes_cache = p.cache_k != nullptr && (h % p.G) == 0;
     auto copy_diagonal_tiles = [&](int part) {
         if (!writes_cache) return;
-        for (int j = n_cache + 2 * qb; j < n_kv; ++j) {
+        for (int j = n_cache + diag0; j < n_kv; ++j) {
             const int r_base = (j - n_cache) * kRows;              // first row of the tile among the new tokens
             for (int kv = 0; kv < 2; ++kv) {
                 const int idx = 2 * j + kv;
@@ -389,7 +398,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
         // ============================================================ softmax + epilogue warpgroups
         const int i = warp >> 2;                                   // sub-tile
         const int t = threadIdx.x & 127;                           // row within the sub-tile == TMEM lane
-        const int row = q0 + i * kRows + t;                        // token index of this thread's query row
+        const int row = q0 + i * sub_rows + t;                     // token index of this thread's query row
+        const int hq = h + i * sub_heads;                          // ... and its query head
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t tmem_s = tmem_base + lane_base + (i ? C::kColS1 : C::kColS0);
         const uint32_t tmem_o = tmem_base + lane_base + (i ? C::kColO1 : C::kColO0);
@@ -397,7 +407,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
         // Tiles that need a mask: the last tile of the past when it is partly filled (columns past its end, the same
         // for every row), and the sub-tile's diagonal tile among the new tokens (row t sees columns 0..t).
         const int j_ragged = (past & (kRows - 1)) ? n_cache - 1 : -1;
-        const int j_diag = n_cache + 2 * qb + i;
+        const int j_diag = n_cache + (pair ? diag0 : diag0 + i);
         const float c = p.scale_log2e;
         float m = -INFINITY, l = 0.f;
         bool ok = true;
@@ -515,11 +525,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
             tcgen05_fence_after_sync();
             const float inv = 1.f / l;
             const bool valid = row < L;
-            __nv_bfloat16 *orow = p.o + b * p.o_sb + (int64_t)row * p.o_st + h * p.o_sh;
+            __nv_bfloat16 *orow = p.o + b * p.o_sb + (int64_t)row * p.o_st + hq * p.o_sh;
             // A sub-tile whose 128 rows are all valid leaves through shared memory and one TMA store per 64
             // columns (coalesced, asynchronous): the rows are staged where Q_i was, which no MMA reads any more
             // (o_full follows the last of them). A ragged sub-tile writes its valid rows directly.
-            const bool whole = q0 + i * kRows + kRows <= L;
+            const bool whole = q0 + i * sub_rows + kRows <= L;
             uint8_t *stage = q_smem + i * C::kTileBytes;
 #pragma unroll
             for (int qd = 0; qd < D / 32; ++qd) {
@@ -554,7 +564,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
                 mbar_arrive(&o_staged[i]);
                 if (t == 0 && mbar_wait(&o_staged[i], 0, abort_flag)) {
                     int c1, c2, c3;
-                    order_coords(p.co, q0 + i * kRows, h, b, c1, c2, c3);
+                    order_coords(p.co, q0 + i * sub_rows, hq, b, c1, c2, c3);
 #pragma unroll
                     for (int hf = 0; hf < C::kHalves; ++hf) tma_store_4d(&tmap_o, stage + hf * kHalfBytes, hf * 64, c1, c2, c3);
                     tma_store_commit();
@@ -562,7 +572,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
                 }
             }
             if (valid && p.lse)
-                p.lse[((size_t)b * p.Hq + h) * p.S_max + row] = (m + log2f(l)) * 0.6931471805599453f;
+                p.lse[((size_t)b * p.Hq + hq) * p.S_max + row] = (m + log2f(l)) * 0.6931471805599453f;
         }
     }
 
@@ -596,7 +606,7 @@ l4l_status launch_t(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensor
             configured = true;
         }
     }
-    const long long grid = (long long)p.n_qblocks * p.Hq * p.B;
+    const long long grid = (long long)p.n_qblocks * (p.pair_heads ? p.Hq / 2 : p.Hq) * p.B;
     if (grid > 0x7fffffffll) return L4L_ERR_UNSUPPORTED;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
@@ -663,7 +673,8 @@ l4l_status launch_prefill_tc(const l4l_tensor4 &q, const l4l_tensor4 &o, const P
     p.lse = d_lse;
     p.status = static_cast<unsigned *>(workspace);
     p.S_max = S_max; p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.G = Hq / Hkv;
-    p.n_qblocks = (S_max + 2 * kRows - 1) / (2 * kRows);
+    p.pair_heads = (p.G % 2 == 0) ? 1 : 0;
+    p.n_qblocks = p.pair_heads ? (S_max + kRows - 1) / kRows : (S_max + 2 * kRows - 1) / (2 * kRows);
     p.scale_log2e = scale * 1.4426950408889634f;
     p.cq = cq; p.ckv = ck; p.co = co; p.ckc = ckc;
     return (D == 128) ? launch_t<128>(tq, tk, tv, to, tkc, tvc, p, stream) : launch_t<64>(tq, tk, tv, to, tkc, tvc, p, stream);
