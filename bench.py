@@ -34,9 +34,9 @@ METRIC = "decode-attn HBM GB/s & prefill-attn TFLOP/s, each as % of B200 peak"
 NOMINAL_TFLOPS, NOMINAL_GBS = 2250.0, 8000.0
 FALLBACK_TFLOPS, FALLBACK_GBS = 1590.0, 6650.0
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
-# profiles/: prefill captured at B=1,S=8192 (155.8 MB) and scaled x4 to the bench's B=4 (traffic is proportional
+# profiles/: prefill captured at B=1,S=8192 (160.2 MB) and scaled x4 to the bench's B=4 (traffic is proportional
 # to B); decode captured on the bench's own batch.
-NCU_TRAFFIC_PREFILL = 628.1e6   # 4 x (101.0 MB read + 56.1 MB written)
+NCU_TRAFFIC_PREFILL = 640.8e6   # 4 x (102.1 MB read + 58.1 MB written)
 NCU_TRAFFIC_DECODE = 302.2e6    # 297.8 MB read + 4.4 MB written
 
 
@@ -744,7 +744,7 @@ def run_ours(args, rank, world):
 def run_profile_case(case: str):
     """A few launches of ONE kernel on a small case, for `ncu` captures (not a benchmark):
     prefill = B=1, S=8192 of the long_prefill workload (inputs 168 MB > L2); decode = the batched_decode batch;
-    rglru = the RG-LRU scan on B=16, T=2048, W=2560; decode_small = the cluster decode kernel on B=4 x 8192 tokens; decode_short = the warp-per-unit decode kernel on B=512 x 64..256 tokens; decode_fp8 = the split kernel on the batched_decode batch in an fp8 cache; rope = rope + norm + cache update on B=2, S=8192."""
+    rglru = the RG-LRU scan on B=16, T=2048, W=2560; rglru_long = the same bytes as B=4, T=8192 (narrow strips); decode_small = the cluster decode kernel on B=4 x 8192 tokens; decode_short = the warp-per-unit decode kernel on B=512 x 64..256 tokens; decode_fp8 = the split kernel on the batched_decode batch in an fp8 cache; rope = rope + norm + cache update on B=2, S=8192."""
     from paper_2608_21836_b200 import binding as l4l
 
     torch.cuda.set_device(0)
@@ -759,8 +759,10 @@ def run_profile_case(case: str):
         ws = l4l.new_workspace(l4l.L4L_OP_PREFILL, 1, w.Hq, w.Hkv, w.D, seq.S)
         for _ in range(3):
             l4l.l4l_attn_prefill(q, k, v, o, lens, w.scale, ws, cache_k=ck, cache_v=cv)
-    elif case == "rglru":
-        B, T, W = 16, 2048, 2560                          # 503 MB of inputs, 168 MB of output
+    elif case in ("rglru", "rglru_long"):
+        # 503 MB of inputs, 168 MB of output; rglru: 640 strips of 64 channels; rglru_long: 4 sequences of 8192 steps,
+        # which the library cuts into 640 strips of 16 channels (160 strips of 64 would load 148 SMs unevenly)
+        B, T, W = (16, 2048, 2560) if case == "rglru" else (4, 8192, 2560)
         gen = torch.Generator().manual_seed(1006)
         x = torch.randn(B, T, W, generator=gen).to(torch.bfloat16).cuda()
         gx = (torch.randn(B, T, W, generator=gen) * 2).to(torch.bfloat16).cuda()
@@ -848,7 +850,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--profile-case", choices=["prefill", "decode", "decode_small", "decode_short", "decode_fp8", "rope", "rglru"], default=None,
+    ap.add_argument("--profile-case", choices=["prefill", "decode", "decode_small", "decode_short", "decode_fp8", "rope", "rglru", "rglru_long"], default=None,
                     help="run three launches of one kernel on a small case and exit (for ncu)")
     args = ap.parse_args()
     if args.profile_case:
