@@ -146,3 +146,46 @@ def test_prefill_family_random(seed):
     for b in range(B):
         if qlen[b] > 0:
             assert_close_to_oracle(oc[b, :qlen[b]].cpu(), ref[b, past[b]:lens[b]], f"chunk seed {seed} sequence {b}")
+    # ... and the same cut through the fused call: a fresh cache that holds only the prefix, the chunk's K/V handed in
+    # and written by the same launch; once contiguous, once as a page pool of a random page size
+    kc = torch.zeros(B, Sc, Hkv, D, dtype=torch.bfloat16)
+    vc = torch.zeros(B, Sc, Hkv, D, dtype=torch.bfloat16)
+    for b in range(B):
+        kc[b, :qlen[b]] = k[b, past[b]:lens[b]]
+        vc[b, :qlen[b]] = v[b, past[b]:lens[b]]
+    want_k, want_v = k.permute(0, 2, 1, 3).contiguous(), v.permute(0, 2, 1, 3).contiguous()       # [B, Hkv, S, D]
+    live = torch.arange(S).view(1, 1, S, 1) < torch.from_numpy(lens).view(B, 1, 1, 1)
+    prefix = torch.arange(S).view(1, 1, S, 1) < torch.from_numpy(past).view(B, 1, 1, 1)
+    nan = nan_bf16((1,))
+    ck2 = torch.where(prefix, want_k, nan).contiguous().cuda()
+    cv2 = torch.where(prefix, want_v, nan).contiguous().cuda()
+    oc2 = torch.zeros(B, Sc, Hq, D, dtype=torch.bfloat16, device="cuda")
+    l4l.l4l_attn_prefill_chunk_append(qc.cuda(), kc.cuda(), vc.cuda(), oc2, ck2, cv2, torch.from_numpy(past).cuda(),
+                                      torch.from_numpy(qlen).cuda(), scale, ws)
+    torch.cuda.synchronize()
+    assert l4l.l4l_last_device_error(ws) == 0
+    assert torch.equal(torch.where(live, ck2.cpu(), nan).view(torch.int16), torch.where(live, want_k, nan).view(torch.int16))
+    assert torch.equal(torch.where(live, cv2.cpu(), nan).view(torch.int16), torch.where(live, want_v, nan).view(torch.int16))
+    page = int(rng.choice([16, 32, 64, 128]))
+    n_per = (S + page - 1) // page
+    perm = torch.from_numpy(rng.permutation(B * n_per + 2)[:B * n_per].astype(np.int32)).view(B, n_per)
+    pool_k = nan_bf16((B * n_per + 2, Hkv, page, D)).clone()
+    pool_v = nan_bf16((B * n_per + 2, Hkv, page, D)).clone()
+    pad_k = torch.cat([torch.where(prefix, want_k, nan), nan_bf16((B, Hkv, n_per * page - S, D))], dim=2)
+    pad_v = torch.cat([torch.where(prefix, want_v, nan), nan_bf16((B, Hkv, n_per * page - S, D))], dim=2)
+    for b in range(B):
+        for i in range(n_per):
+            pool_k[perm[b, i]] = pad_k[b, :, i * page:(i + 1) * page]
+            pool_v[perm[b, i]] = pad_v[b, :, i * page:(i + 1) * page]
+    dpk, dpv = pool_k.cuda(), pool_v.cuda()
+    oc3 = torch.zeros(B, Sc, Hq, D, dtype=torch.bfloat16, device="cuda")
+    l4l.l4l_attn_prefill_chunk_append(qc.cuda(), kc.cuda(), vc.cuda(), oc3, dpk, dpv, torch.from_numpy(past).cuda(),
+                                      torch.from_numpy(qlen).cuda(), scale, ws, block_table=perm.cuda())
+    torch.cuda.synchronize()
+    assert l4l.l4l_last_device_error(ws) == 0
+    got_k = torch.from_numpy(orc.gather_pages(dpk.cpu(), perm.numpy(), S).view(np.int16)).view(torch.bfloat16)
+    assert torch.equal(torch.where(live, got_k, nan).view(torch.int16), torch.where(live, want_k, nan).view(torch.int16))
+    for b in range(B):
+        if qlen[b] > 0:
+            assert_close_to_oracle(oc2[b, :qlen[b]].cpu(), ref[b, past[b]:lens[b]], f"fused chunk seed {seed} sequence {b}")
+            assert_close_to_oracle(oc3[b, :qlen[b]].cpu(), ref[b, past[b]:lens[b]], f"paged fused chunk seed {seed} sequence {b}")
