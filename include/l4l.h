@@ -171,7 +171,10 @@ l4l_status l4l_attn_decode_paged_append(const void *q, void *o, l4l_paged_kv poo
  *   l4l_kv_append_fp8  : stores RN_e4m3( fp32(x) / k_scale[g] ) (IEEE fp32 division, then round to
  *                        nearest even, saturating at +-448; NaN stays NaN); other rules as l4l_kv_append.
  *   l4l_attn_decode_fp8: l4l_attn_decode over the values the bytes stand for (the widening to f16 in
- *                        the kernel is exact; q and the softmax weights are used as f16). head_dim 128 only.
+ *                        the kernel is exact; q and the softmax weights are used as f16). At head_dim 64 (this
+ *                        entry point and the other fp8 decode calls) two tokens share a 128-byte tile row, so the
+ *                        token rows of the cache (of each page) must lie back to back (stride_t = 64) and the
+ *                        number of slots must be even, else L4L_ERR_UNSUPPORTED.
  *   d_k_scale, d_v_scale   device float [Hkv], > 0
  */
 l4l_status l4l_kv_append_fp8(l4l_kv_cache cache8, l4l_tensor4 k_new, l4l_tensor4 v_new,

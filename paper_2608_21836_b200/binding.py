@@ -500,7 +500,8 @@ def l4l_kv_append_fp8(cache_k8, cache_v8, k_new, v_new, write_pos, k_scale, v_sc
 
 def l4l_attn_decode_fp8(q, o, cache_k8, cache_v8, k_scale, v_scale, kv_lens, max_kv_len: int, scale: float, workspace,
                         lse=None) -> None:
-    """Decode over an fp8 (e4m3) cache with per-KV-head scales. q,o dense bf16 [B,Hq,D]; head_dim 128."""
+    """Decode over an fp8 (e4m3) cache with per-KV-head scales. q,o dense bf16 [B,Hq,D] (at head_dim 64 the cache's
+    token rows must be dense and even in number)."""
     _check_bf16_cuda(q, "q")
     _check_bf16_cuda(o, "o")
     if not (q.is_contiguous() and o.is_contiguous() and q.dim() == 3 and q.shape == o.shape):

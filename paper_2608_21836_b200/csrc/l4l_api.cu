@@ -375,7 +375,6 @@ l4l_status l4l_attn_decode_fp8(const void *q, void *o, l4l_kv_cache cache8, cons
 {
     l4l_status st = shape_status(B, Hq, Hkv, head_dim);
     if (st != L4L_OK) return st;
-    if (head_dim != 128) return L4L_ERR_UNSUPPORTED;          // one 128-byte row per token
     if (!q || !o || !d_kv_lens || !d_k_scale || !d_v_scale || !aligned16(q) || !aligned16(o)) return L4L_ERR_INVALID_ARG;
     if (!cache8_ok(cache8)) return L4L_ERR_INVALID_ARG;
     if (max_kv_len < 0 || max_kv_len > cache8.max_len) return L4L_ERR_INVALID_ARG;
@@ -395,7 +394,6 @@ l4l_status l4l_attn_decode_paged_fp8(const void *q, void *o, l4l_paged_kv pool8,
 {
     l4l_status st = shape_status(B, Hq, Hkv, head_dim);
     if (st != L4L_OK) return st;
-    if (head_dim != 128) return L4L_ERR_UNSUPPORTED;
     if (!q || !o || !d_kv_lens || !d_block_table || !d_k_scale || !d_v_scale || !aligned16(q) || !aligned16(o))
         return L4L_ERR_INVALID_ARG;
     auto s16 = [](int64_t s) { return s >= 0 && (s % 16) == 0; };
@@ -421,7 +419,6 @@ l4l_status l4l_attn_decode_append_fp8(const void *q, void *o, l4l_kv_cache cache
 {
     l4l_status st = shape_status(B, Hq, Hkv, head_dim);
     if (st != L4L_OK) return st;
-    if (head_dim != 128) return L4L_ERR_UNSUPPORTED;          // one 128-byte row per token
     if (!q || !o || !d_kv_lens || !d_k_scale || !d_v_scale || !aligned16(q) || !aligned16(o)) return L4L_ERR_INVALID_ARG;
     if (!cache8_ok(cache8) || !tensor4_ok(k_new) || !tensor4_ok(v_new)) return L4L_ERR_INVALID_ARG;
     if (max_kv_len < 0 || max_kv_len > cache8.max_len) return L4L_ERR_INVALID_ARG;
@@ -442,7 +439,6 @@ l4l_status l4l_attn_decode_paged_append_fp8(const void *q, void *o, l4l_paged_kv
 {
     l4l_status st = shape_status(B, Hq, Hkv, head_dim);
     if (st != L4L_OK) return st;
-    if (head_dim != 128) return L4L_ERR_UNSUPPORTED;
     if (!q || !o || !d_kv_lens || !d_block_table || !d_k_scale || !d_v_scale || !aligned16(q) || !aligned16(o))
         return L4L_ERR_INVALID_ARG;
     auto s16 = [](int64_t s) { return s >= 0 && (s % 16) == 0; };
@@ -680,7 +676,7 @@ void l4l_set_decode_override(int cluster, int warp, int split_warps)
 int l4l_decode_kernel_choice(int B, int Hq, int Hkv, int head_dim, int max_kv_len, int fp8, int *detail)
 {
     if (detail) *detail = 0;
-    if (shape_status(B, Hq, Hkv, head_dim) != L4L_OK || B == 0 || max_kv_len < 0 || (fp8 && head_dim != 128)) return -1;
+    if (shape_status(B, Hq, Hkv, head_dim) != L4L_OK || B == 0 || max_kv_len < 0 || false) return -1;
     // the order launch_decode asks in
     if (decode_warp_eligible(B, Hq, Hkv, head_dim, max_kv_len, fp8 != 0, false, false)) return 2;
     const int width = decode_cluster_width(B, Hq, Hkv, head_dim, max_kv_len, fp8 != 0);

@@ -46,13 +46,16 @@ constexpr int kMaxB = 384;                 // sequences per launch (prefix sums 
 // F8: the cache holds e4m3 bytes (one byte per value) instead of bf16.
 template <int D, int W, bool F8>
 struct DecodeCfg {
-    static_assert(!F8 || D == 128, "the fp8 path wants one 128-byte row per token");
     static constexpr int kSub = F8 ? 2 : 1;                       // 16-token blocks a consumer warp takes per tile
     static constexpr int kTileT = 16 * W * kSub;                  // tokens per TMA tile
     static constexpr int kRowBytes = F8 ? D : 2 * D;              // one token of one KV head
-    static constexpr int kHalves = kRowBytes / 128;               // 128-byte column blocks of a tile
+    // fp8 at head_dim 64: a token is 64 bytes, and two consecutive tokens make one 128-byte row of the tile (the
+    // cache must be dense in the token dimension); everywhere else a token is one row of every 128-byte column block
+    static constexpr int kTokPerRow = kRowBytes < 128 ? 2 : 1;
+    static constexpr int kTokBytes = 128 / kTokPerRow;            // bytes of a token in one column block
+    static constexpr int kHalves = kRowBytes < 128 ? 1 : kRowBytes / 128;   // 128-byte column blocks of a tile
     static constexpr int kBoxD = F8 ? 128 : 64;                   // elements per 128-byte box row
-    static constexpr uint32_t kHalfBytes = kTileT * 128;          // [tile tokens][128 bytes], swizzled
+    static constexpr uint32_t kHalfBytes = kTileT * kTokBytes;    // [tile rows][128 bytes], swizzled
     static constexpr uint32_t kTileBytes = kHalves * kHalfBytes;  // one of K or V
     static constexpr uint32_t kStageBytes = 2 * kTileBytes;
     static constexpr int kStages = (kStageBytes >= 32768u * (W / 4)) ? 3 : 6;   // 192 KB (96 KB with W = 4) in flight
@@ -348,7 +351,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     const int box_rows = by_groups ? p.tail_rows : (paged ? p.page_box : kTileT);
                     const int n_box = by_groups ? groups : ((rem >= kTileT || box_rows == kTileT) ? kTileT / box_rows
                                                                                                   : (rem + box_rows - 1) / box_rows);
-                    const uint32_t kv_bytes = (uint32_t)n_box * box_rows * 128u * C::kHalves * 2u;
+                    const uint32_t kv_bytes = (uint32_t)n_box * box_rows * (uint32_t)C::kTokBytes * C::kHalves * 2u;
                     // with the rope fused into the step, the piece's first tile also brings the cos / sin rows of
                     // the new token's position (kv_len - 1), if the table has it
                     const bool with_rope = first && p.rope_cos != nullptr && len - 1 < p.rope_n_pos;
@@ -376,8 +379,8 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                         if (bx >= n_box) break;
                         int tt = tile * kTileT + bx * box_rows;
                         if (paged) tt &= p.page_size - 1;
-                        order_coords(p.coord, tt, kvh, page_of[bx], c1, c2, c3);
-                        uint8_t *db = dst + bx * box_rows * 128;  // whole 8-row groups: the swizzle phase is kept
+                        order_coords(p.coord, tt / C::kTokPerRow, kvh, page_of[bx], c1, c2, c3);
+                        uint8_t *db = dst + bx * box_rows * C::kTokBytes;  // whole 8-row groups: the swizzle phase is kept
 #pragma unroll
                         for (int hf = 0; hf < C::kHalves; ++hf) {
                             tma_load_4d(db + hf * C::kHalfBytes, tk, &full[s], hf * C::kBoxD, c1, c2, c3);
@@ -831,7 +834,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     // cache update quantises them (same division, same rounding), patched into the tile and written
                     // to their cache slot; 8 lanes, 16 values each
                     const int last = row0 + nvalid - 1;
-                    if (lane < 8) {
+                    if (lane < D / 16) {
                         const size_t src = (size_t)mt.b * p.new_sb + (size_t)mt.kvh * p.new_sh + lane * 16;
                         const uint4 *ks = reinterpret_cast<const uint4 *>(p.k_new + src);
                         const uint4 *vs = reinterpret_cast<const uint4 *>(p.v_new + src);
@@ -844,7 +847,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                         }
                         if (p.block_table == nullptr || (outer >= 0 && outer < p.num_pages)) {
                             uint8_t *kt = stages + (size_t)s * C::kStageBytes;
-                            const uint32_t off = swz128(last, lane);
+                            const uint32_t off = tok_chunk_f8<D>(0u, (uint32_t)last, (uint32_t)lane);
                             *reinterpret_cast<uint4 *>(kt + off) = kq;
                             *reinterpret_cast<uint4 *>(kt + C::kTileBytes + off) = vq;
                             // fp8 caches: the strides count bytes
@@ -886,8 +889,9 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                                 if (8 * j + tok + (e & 1) >= nvalid) sv[j][e] = -INFINITY;
                         uint8_t *vt = stages + (size_t)s * C::kStageBytes + C::kTileBytes;
                         const int fetched_end = (nvalid + 15) & ~15;                 // end of the last valid block
-                        for (int i = lane; i < (fetched_end - nvalid) * 8; i += 32)
-                            *reinterpret_cast<uint4 *>(vt + (row0 + nvalid + i / 8) * 128 + ((i & 7) << 4)) =
+                        constexpr int kCh = D / 16;                                   // 16-byte chunks of a token
+                        for (int i = lane; i < (fetched_end - nvalid) * kCh; i += 32)
+                            *reinterpret_cast<uint4 *>(vt + tok_chunk_f8<D>(0u, (uint32_t)(row0 + nvalid + i / kCh), (uint32_t)(i % kCh))) =
                                 make_uint4(0u, 0u, 0u, 0u);
                         wrote_smem = true;
                         __syncwarp();
@@ -1081,7 +1085,8 @@ ShapeOps pick_shape(int D, int warps, bool fp8, bool big = false)
 {
     if (big && warps == 6) return fp8 ? shape_ops<128, 6, true, true>() : shape_ops<128, 6, false, true>();
     if (big) return fp8 ? shape_ops<128, 8, true, true>() : shape_ops<128, 8, false, true>();
-    if (fp8) return warps == 8 ? shape_ops<128, 8, true>() : shape_ops<128, 4, true>();      // D == 128 only
+    if (fp8 && D == 64) return warps == 8 ? shape_ops<64, 8, true>() : shape_ops<64, 4, true>();
+    if (fp8) return warps == 8 ? shape_ops<128, 8, true>() : shape_ops<128, 4, true>();
     if (D == 128) return warps == 8 ? shape_ops<128, 8, false>() : shape_ops<128, 4, false>();
     return warps == 8 ? shape_ops<64, 8, false>() : shape_ops<64, 4, false>();
 }
@@ -1166,7 +1171,10 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
 {
     if (rope && (!k_new || !v_new || fp8)) return L4L_ERR_UNSUPPORTED;   // only with the fused append, bf16 caches
     // fp8: cache.k / cache.v point at e4m3 bytes, the strides count bytes (= elements)
-    if (fp8 && D != 128) return L4L_ERR_UNSUPPORTED;
+    // fp8 at head_dim 64: two 64-byte tokens make one 128-byte tile row, so the token rows of the cache (or of a page)
+    // must lie back to back and come in pairs
+    const bool pair_rows = fp8 && D == 64;
+    if (pair_rows && (cache.stride_t != 64 || (cache.max_len & 1))) return L4L_ERR_UNSUPPORTED;
     const int esz = fp8 ? 1 : 2;
     // paged: `cache` describes the page pool (stride_b = stride between pages, max_len = page size)
     // hundreds of short sequences: one warp per (sequence, KV head), nothing to merge
@@ -1212,14 +1220,17 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         int box_t = kTileT;
         if (paged) box_t = (kTileT % cache.max_len == 0) ? cache.max_len : (cache.max_len % kTileT == 0 ? kTileT : 32);
         const int tail_rows = (paged && cache.max_len < 32) ? cache.max_len : 32;
-        if (!make_tmap(&tk, &coord, kb, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
-                       cache.stride_b, box_d, box_t, esz) ||
-            !make_tmap(&tv, &coord_v, vb, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
-                       cache.stride_b, box_d, box_t, esz) ||
-            !make_tmap(&tk_tail, &coord_v, kb, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
-                       cache.stride_b, box_d, tail_rows, esz) ||
-            !make_tmap(&tv_tail, &coord_v, vb, D, cache.max_len, Hkv, outer, cache.stride_t, cache.stride_h,
-                       cache.stride_b, box_d, tail_rows, esz))
+        // what the maps see as a row: a token, or (fp8 at head_dim 64) a pair of tokens
+        const int tpr = pair_rows ? 2 : 1, map_d = pair_rows ? 128 : D;
+        const int64_t map_rows = cache.max_len / tpr, map_st = cache.stride_t * tpr;
+        if (!make_tmap(&tk, &coord, kb, map_d, map_rows, Hkv, outer, map_st, cache.stride_h,
+                       cache.stride_b, box_d, box_t / tpr, esz) ||
+            !make_tmap(&tv, &coord_v, vb, map_d, map_rows, Hkv, outer, map_st, cache.stride_h,
+                       cache.stride_b, box_d, box_t / tpr, esz) ||
+            !make_tmap(&tk_tail, &coord_v, kb, map_d, map_rows, Hkv, outer, map_st, cache.stride_h,
+                       cache.stride_b, box_d, tail_rows / tpr, esz) ||
+            !make_tmap(&tv_tail, &coord_v, vb, map_d, map_rows, Hkv, outer, map_st, cache.stride_h,
+                       cache.stride_b, box_d, tail_rows / tpr, esz))
             return L4L_ERR_CUDA;
         DecodeParams p;
         p.q = static_cast<const __nv_bfloat16 *>(q) + (size_t)b0 * Hq * D;
@@ -1281,6 +1292,9 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         else if (big)
             err = fp8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 8, true, true>, tk, tv, tk_tail, tv_tail, p)
                       : cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 8, false, true>, tk, tv, tk_tail, tv_tail, p);
+        else if (fp8 && D == 64)
+            err = plan.warps == 8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<64, 8, true, false>, tk, tv, tk_tail, tv_tail, p)
+                                  : cudaLaunchKernelEx(&cfg, decode_split_kernel<64, 4, true, false>, tk, tv, tk_tail, tv_tail, p);
         else if (fp8)
             err = plan.warps == 8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 8, true, false>, tk, tv, tk_tail, tv_tail, p)
                                   : cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 4, true, false>, tk, tv, tk_tail, tv_tail, p);

@@ -640,7 +640,7 @@ int decode_cluster_width(int B, int Hq, int Hkv, int D, int max_kv_len, bool fp8
 {
     // tuning override: 0 keeps every call on the split kernel, N forces clusters of N where they fit
     const int forced = decode_override().cluster;
-    if (forced == 0) return 0;
+    if (forced == 0 || (fp8 && D != 128)) return 0;       // fp8 at head_dim 64 runs on the split kernel only
     const int G = Hq / Hkv;
     const long long units = (long long)B * Hkv;
     const int sms = sm_count();

@@ -148,7 +148,9 @@ __device__ __forceinline__ void warp_softmax_tiles(WarpAttnState<D> &st, const f
 }
 
 // ----------------------------------------------------------------------------- fp8 (e4m3) K/V tiles
-// A tile is [tile_tokens][128 bytes] (D = 128 values per token), 128-byte swizzled. The values are
+// A tile is rows of 128 bytes, 128-byte swizzled: one token per row at D = 128, TWO consecutive tokens per row at
+// D = 64 (token 2r in bytes 0..63 of row r, token 2r+1 in bytes 64..127: a dense cache of 64-byte token rows seen as
+// rows of 128). tok_chunk_f8 gives the address of 16-byte chunk c (16 head dims) of a token either way. The values are
 // widened to f16 in registers (exact) and multiplied with f16 MMAs. ldmatrix moves 16-bit units, so a
 // thread receives 4 consecutive head-dim bytes of a K row where the MMA wants two separate pairs: the
 // k index of QK^T is therefore permuted (MMA slots 2c, 2c+1, 2c+8, 2c+9 of a 16-block hold head dims
@@ -156,6 +158,15 @@ __device__ __forceinline__ void warp_softmax_tiles(WarpAttnState<D> &st, const f
 // transposing ldmatrix delivers, per thread, two tokens of an EVEN and an ODD head dim: the 8-column
 // MMA tiles of O alternate even / odd dims (tile 2j: dims 16j + 2x, tile 2j+1: dims 16j + 2x + 1 in
 // column x); a thread's accumulators of a tile pair are then 4 consecutive head dims.
+
+// Shared-memory address of head dims [16c, 16c+16) of token `tok` of an fp8 tile.
+template <int D>
+__device__ __forceinline__ uint32_t tok_chunk_f8(uint32_t tile, uint32_t tok, uint32_t c)
+{
+    static_assert(D == 128 || D == 64, "one or two tokens per 128-byte row");
+    if constexpr (D == 128) return tile + swz128(tok, c);
+    else return tile + swz128(tok >> 1, ((tok & 1u) << 2) + c);
+}
 
 // 32-bit word (two bf16) of a q row that feeds A-fragment register `reg` (0..3) of k-step ks, as f16x2.
 __device__ __forceinline__ int q_frag_f8_word(int ks, int reg, int lane) { return ks * 8 + 2 * (lane & 3) + (reg >> 1); }
@@ -169,7 +180,6 @@ template <int D>
 __device__ __forceinline__ void warp_qk_16x16_f8(const uint32_t (&qf)[D / 16][4], uint32_t k_tile, int row0,
                                                  float (&s_lo)[4], float (&s_hi)[4])
 {
-    static_assert(D == 128, "one 128-byte row per token");
     const int lane = threadIdx.x & 31;
     s_lo[0] = s_lo[1] = s_lo[2] = s_lo[3] = 0.f;
     s_hi[0] = s_hi[1] = s_hi[2] = s_hi[3] = 0.f;
@@ -178,7 +188,7 @@ __device__ __forceinline__ void warp_qk_16x16_f8(const uint32_t (&qf)[D / 16][4]
 #pragma unroll
     for (int qd = 0; qd < D / 32; ++qd) {
         uint32_t r0, r1, r2, r3;
-        ldmatrix_x4(k_tile + swz128(row, 2 * qd + csel), r0, r1, r2, r3);
+        ldmatrix_x4(tok_chunk_f8<D>(k_tile, row, 2 * qd + csel), r0, r1, r2, r3);
         mma_f16_16816(s_lo, qf[2 * qd], e4m3x2_to_f16x2(r0), e4m3x2_to_f16x2(r0 >> 16));
         mma_f16_16816(s_lo, qf[2 * qd + 1], e4m3x2_to_f16x2(r1), e4m3x2_to_f16x2(r1 >> 16));
         mma_f16_16816(s_hi, qf[2 * qd], e4m3x2_to_f16x2(r2), e4m3x2_to_f16x2(r2 >> 16));
@@ -189,14 +199,13 @@ __device__ __forceinline__ void warp_qk_16x16_f8(const uint32_t (&qf)[D / 16][4]
 template <int D>
 __device__ __forceinline__ void warp_pv_16x16_f8(WarpAttnState<D> &st, const uint32_t (&pa)[4], uint32_t v_tile, int row0)
 {
-    static_assert(D == 128, "one 128-byte row per token");
     const int lane = threadIdx.x & 31;
     const uint32_t row = row0 + (((lane >> 3) & 1) << 3) + (lane & 7);   // matrices 1,3: tokens +8
     const uint32_t csel = lane >> 4;                                      // matrices 2,3: next 16 head dims
 #pragma unroll
     for (int qd = 0; qd < D / 32; ++qd) {
         uint32_t r0, r1, r2, r3;
-        ldmatrix_x4_trans(v_tile + swz128(row, 2 * qd + csel), r0, r1, r2, r3);
+        ldmatrix_x4_trans(tok_chunk_f8<D>(v_tile, row, 2 * qd + csel), r0, r1, r2, r3);
         // bytes (tok, even) (tok, odd) (tok+1, even) (tok+1, odd) -> (tok, even) (tok+1, even) | (tok, odd) (tok+1, odd)
         const uint32_t x0 = __byte_perm(r0, 0u, 0x3120), x1 = __byte_perm(r1, 0u, 0x3120);
         const uint32_t x2 = __byte_perm(r2, 0u, 0x3120), x3 = __byte_perm(r3, 0u, 0x3120);

@@ -20,12 +20,13 @@ def random_codes(shape, g, max_exp_field=11):
     return c
 
 
-@pytest.mark.parametrize("Hq,Hkv", [(32, 8), (8, 8), (16, 2)])
-def test_fp8_decode_matches_oracle(Hq, Hkv):
-    D, Lmax = 128, 2304
+@pytest.mark.parametrize("D", [128, 64])
+@pytest.mark.parametrize("Hq,Hkv", [(32, 8), (8, 8), (16, 2), (12, 12)])
+def test_fp8_decode_matches_oracle(Hq, Hkv, D):
+    Lmax = 2304
     lens = [1, 15, 16, 17, 127, 128, 129, 700, 1024, 2049, 2304, 0, 333]
     B = len(lens)
-    g = torch.Generator().manual_seed(1000 + Hq)
+    g = torch.Generator().manual_seed(1000 + Hq + D)
     ck8 = random_codes((B, Hkv, Lmax, D), g, 7)              # |k| < 2
     cv8 = random_codes((B, Hkv, Lmax, D), g, 7)              # |v| < 2: the absolute tolerance presumes O(1) outputs
     for b, L in enumerate(lens):                             # slots past the end hold the NaN code
@@ -100,24 +101,69 @@ def test_fp8_append_is_bit_exact(D):
     assert np.array_equal(gk.t.cpu().numpy(), ref_k) and np.array_equal(gv.t.cpu().numpy(), ref_v)
 
 
-def test_fp8_decode_rejects_head_dim_64():
+def test_fp8_decode_at_head_dim_64_wants_dense_token_rows_in_pairs():
+    """At head_dim 64 two tokens share a 128-byte tile row: the cache's token rows must lie back to back (stride 64)
+    and the slot count must be even; anything else is refused on the host."""
     q = torch.zeros(1, 4, 64, dtype=torch.bfloat16, device="cuda")
-    c8 = torch.zeros(1, 2, 32, 64, dtype=torch.uint8, device="cuda")
     sc = torch.ones(2, device="cuda")
+    one = torch.ones(1, dtype=torch.int32, device="cuda")
     ws = l4l.new_workspace(l4l.L4L_OP_DECODE, 1, 4, 2, 64, 32)
-    with pytest.raises(l4l.L4LError):
-        l4l.l4l_attn_decode_fp8(q, q.clone(), c8, c8.clone(), sc, sc, torch.ones(1, dtype=torch.int32, device="cuda"),
-                                32, 0.1, ws)
+    odd = torch.zeros(1, 2, 33, 64, dtype=torch.uint8, device="cuda")                       # odd number of slots
+    with pytest.raises(l4l.L4LError) as e:
+        l4l.l4l_attn_decode_fp8(q, q.clone(), odd, odd.clone(), sc, sc, one, 32, 0.1, ws)
+    assert e.value.status == l4l.L4L_ERR_UNSUPPORTED
+    wide = torch.zeros(1, 2, 32, 128, dtype=torch.uint8, device="cuda")[..., :64]           # token rows 128 bytes apart
+    with pytest.raises(l4l.L4LError) as e:
+        l4l.l4l_attn_decode_fp8(q, q.clone(), wide, torch.zeros(1, 2, 32, 128, dtype=torch.uint8, device="cuda")[..., :64],
+                                sc, sc, one, 32, 0.1, ws)
+    assert e.value.status == l4l.L4L_ERR_UNSUPPORTED
+    ok = torch.zeros(1, 2, 32, 64, dtype=torch.uint8, device="cuda")
+    l4l.l4l_attn_decode_fp8(q, q.clone(), ok, ok.clone(), sc, sc, one, 32, 0.1, ws)
+    torch.cuda.synchronize()
+    assert l4l.l4l_last_device_error(ws) == 0
 
 
+def test_fp8_decode_small_mha_shape_at_full_size():
+    """The small MHA model's decode batch (Hq = Hkv = 12, head_dim 64, B = 64 at context 1024) over an fp8 cache written
+    by the library's own append."""
+    from paper_2608_21836_b200 import workloads as wl
+
+    w = wl.WORKLOADS["mha_small"]
+    db = wl.make_decode_batch(w, poison_tail=False)
+    B, Hq, Hkv, D, Lmax = w.decode_B, w.Hq, w.Hkv, w.D, w.decode_Lmax
+    sc = torch.full((Hkv,), 4.5 / 448, dtype=torch.float32)
+    k8 = torch.zeros(B, Hkv, Lmax, D, dtype=torch.uint8, device="cuda")
+    v8 = torch.zeros_like(k8)
+    l4l.l4l_kv_append_fp8(k8, v8, db.cache_k.cuda().permute(0, 2, 1, 3), db.cache_v.cuda().permute(0, 2, 1, 3),
+                          torch.zeros(B, dtype=torch.int32, device="cuda"), sc.cuda(), sc.cuda())
+    torch.cuda.synchronize()
+    # the codes against the oracle's quantisation on a slice (the oracle's encoder is slow): two sequences, 96 slots
+    nb, nt = 2, 96
+    ref_k, ref_v = orc.kv_append_fp8(np.zeros((nb, Hkv, nt, D), np.uint8), np.zeros((nb, Hkv, nt, D), np.uint8),
+                                     db.cache_k[:nb, :, :nt].permute(0, 2, 1, 3).contiguous(),
+                                     db.cache_v[:nb, :, :nt].permute(0, 2, 1, 3).contiguous(),
+                                     np.zeros(nb, np.int32), None, sc.numpy(), sc.numpy())
+    assert np.array_equal(k8[:nb, :, :nt].cpu().numpy(), ref_k) and np.array_equal(v8[:nb, :, :nt].cpu().numpy(), ref_v)
+    ref_k, ref_v = k8.cpu().numpy(), v8.cpu().numpy()
+    ref, _ = orc.decode_fp8(db.q, ref_k, ref_v, db.kv_len.numpy(), sc.numpy(), sc.numpy(), w.scale)
+    o = torch.zeros(B, Hq, D, dtype=torch.bfloat16, device="cuda")
+    ws = l4l.new_workspace(l4l.L4L_OP_DECODE, B, Hq, Hkv, D, Lmax)
+    assert l4l.l4l_decode_kernel_choice(B, Hq, Hkv, D, Lmax, fp8=True)[0] == "split"
+    l4l.l4l_attn_decode_fp8(db.q.cuda(), o, k8, v8, sc.cuda(), sc.cuda(), db.kv_len.cuda(), Lmax, w.scale, ws)
+    torch.cuda.synchronize()
+    assert l4l.l4l_last_device_error(ws) == 0
+    assert_close_to_oracle(o.cpu(), ref, "fp8 decode, small MHA shape")
+
+
+@pytest.mark.parametrize("D", [128, 64])
 @pytest.mark.parametrize("page", [16, 64, 256])
-def test_fp8_paged_decode_matches_oracle(page):
+def test_fp8_paged_decode_matches_oracle(page, D):
     """An fp8 page pool behind a block table: the oracle gathers the pages (codes are bytes: the gather is the same
     indexing as for bf16) and decodes over the codes."""
-    Hq, Hkv, D = 16, 4, 128
+    Hq, Hkv = 16, 4
     lens = [1, 17, 255, 256, 257, 1500, 0, 640]
     B = len(lens)
-    g = torch.Generator().manual_seed(2000 + page)
+    g = torch.Generator().manual_seed(2000 + page + D)
     need = [(L + page - 1) // page for L in lens]
     n_pages = sum(need) + 4
     table = np.full((B, max(need) + 1), -1, np.int32)
@@ -156,10 +202,9 @@ def test_fp8_paged_decode_matches_oracle(page):
 
 # ---- the decode step that appends the newest token to the fp8 cache itself ----
 
-def _fp8_append_case(Hq, Hkv, lens, seed, page=None, Lmax=2304):
+def _fp8_append_case(Hq, Hkv, lens, seed, page=None, Lmax=2304, D=128):
     """Reference = the oracle's fp8 append at slot kv_len - 1 followed by its fp8 decode; the codes in the cache must
     come back bit for bit. With `page`, the cache is a page pool behind a shuffled block table."""
-    D = 128
     B = len(lens)
     g = torch.Generator().manual_seed(seed)
     ck8 = random_codes((B, Hkv, Lmax, D), g, 7)
@@ -239,3 +284,10 @@ def test_fp8_fused_append_batch_of_several_launch_slices():
     lens = g.integers(0, 300, size=420).tolist()             # more than the 384 sequences of one launch
     _fp8_append_case(8, 2, lens, seed=3400, Lmax=320)
     _fp8_append_case(8, 2, lens, seed=3401, page=32, Lmax=320)
+
+
+@pytest.mark.parametrize("page", [None, 16, 128])
+def test_fp8_fused_append_at_head_dim_64(page, decode_kernel_choice):
+    lens = [1, 2, 31, 32, 33, 255, 256, 257, 1000, 0, 2303, 2304]
+    _fp8_append_case(12, 12, lens, seed=3500 + (page or 0), page=page, D=64)
+    _fp8_append_case(8, 2, lens, seed=3600 + (page or 0), page=page, D=64)
