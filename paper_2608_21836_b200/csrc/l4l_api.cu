@@ -676,7 +676,7 @@ void l4l_set_decode_override(int cluster, int warp, int split_warps)
 int l4l_decode_kernel_choice(int B, int Hq, int Hkv, int head_dim, int max_kv_len, int fp8, int *detail)
 {
     if (detail) *detail = 0;
-    if (shape_status(B, Hq, Hkv, head_dim) != L4L_OK || B == 0 || max_kv_len < 0 || false) return -1;
+    if (shape_status(B, Hq, Hkv, head_dim) != L4L_OK || B == 0 || max_kv_len < 0) return -1;
     // the order launch_decode asks in
     if (decode_warp_eligible(B, Hq, Hkv, head_dim, max_kv_len, fp8 != 0, false, false)) return 2;
     const int width = decode_cluster_width(B, Hq, Hkv, head_dim, max_kv_len, fp8 != 0);

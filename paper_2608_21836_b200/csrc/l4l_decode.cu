@@ -1180,7 +1180,7 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
     // hundreds of short sequences: one warp per (sequence, KV head), nothing to merge
     if (decode_warp_eligible(B, Hq, Hkv, D, max_kv_len, fp8 != nullptr, rope != nullptr, k_new != nullptr))
         return launch_decode_warp(q, o, cache, d_kv_lens, max_kv_len, B, Hq, Hkv, D, scale, d_lse, stream, k_new, v_new,
-                                  paged, fp8);
+                                  paged, fp8, rope);
     {
         // small batches are latency-bound: one cluster per (sequence, KV head), no workspace round trips
         const int width = decode_cluster_width(B, Hq, Hkv, D, max_kv_len, fp8 != nullptr);

@@ -18,6 +18,7 @@
 
 #include "l4l_internal.h"
 #include "l4l_ptx.cuh"
+#include "l4l_rope_frag.cuh"
 #include "l4l_warp_attn.cuh"
 
 namespace l4l {
@@ -42,6 +43,12 @@ struct WarpParams {
     const int32_t *block_table;           // paged cache (null: contiguous)
     int table_stride, page_size, page_shift, num_pages;
     const float *k_scale, *v_scale;       // fp8 cache: real value = e4m3 value * scale of its KV head, [Hkv]
+    // rotary embedding (+ optional RMS norm) of the step's q and k_new inside the kernel (null: inputs are final); only
+    // together with the fused append, bf16 caches. The new token's position is kv_len - 1.
+    const float *rope_cos, *rope_sin;     // [rope_n_pos, D/2]
+    const float *q_weight, *k_weight;     // [D] or null
+    float norm_eps;
+    int rope_n_pos;
     int B, Hq, Hkv, G, max_kv_len, stages;
     float scale_log2e;
 };
@@ -56,10 +63,14 @@ struct WarpCfg {
     static constexpr int kCopies = kChunkT * kRowPieces / 32;         // cp.async per lane for K (and as many for V)
 };
 
-__host__ __device__ inline size_t stage_bytes(int D, int G, bool f8)
+__host__ __device__ inline size_t stage_bytes(int D, int G, bool f8, bool rope)
 {
-    return (size_t)2 * ((f8 ? D : 2 * D) / 128) * kChunkT * 128 + (size_t)G * D * 2;    // K, V, the unit's query rows
+    // K, V, the unit's query rows, and (rope fused into the step) the cos | sin rows of the unit's newest position
+    return (size_t)2 * ((f8 ? D : 2 * D) / 128) * kChunkT * 128 + (size_t)G * D * 2 + (rope ? (size_t)D * 4 : 0);
 }
+// Beside the rings when the rope is fused in: every warp's copy of its unit's cos | sin rows (a unit's first stage is
+// recycled long before its last chunk, which holds the new token), and the two norm weight rows.
+__host__ __device__ inline size_t rope_extra_bytes(int D, int warps, bool rope) { return rope ? (size_t)(warps + 2) * D * 4 : 0; }
 
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void *src, uint32_t src_bytes)
 {
@@ -94,10 +105,19 @@ __global__ void __launch_bounds__(kWarps * 32) decode_warp_kernel(const WarpPara
     int *fifo_s = ctl + 4;                                       // [kWarps][kFifo]
     uint16_t *cnt_s = reinterpret_cast<uint16_t *>(fifo_s + 16 * kFifo);   // [kMaxList] chunks per unit of this CTA
     uint16_t *order_s = cnt_s + kMaxList;                        // [kMaxList] units by descending chunk count
-    const size_t sbytes = stage_bytes(D, p.G, F8);
+    const bool fused_rope = !F8 && p.rope_cos != nullptr;
+    const size_t sbytes = stage_bytes(D, p.G, F8, fused_rope);
     uint8_t *ring_base = smem + kMetaBytes;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     uint8_t *ring = ring_base + (size_t)warp * p.stages * sbytes;
+    float *rope_priv = reinterpret_cast<float *>(ring_base + (size_t)kWarps * p.stages * sbytes) + (size_t)warp * D;   // cos | sin of this warp's unit
+    float *norm_w = reinterpret_cast<float *>(ring_base + (size_t)kWarps * p.stages * sbytes) + (size_t)kWarps * D;   // q_weight | k_weight
+    if (fused_rope) {
+        for (int i = threadIdx.x; i < D; i += kThreads) {
+            norm_w[i] = p.q_weight ? __ldg(p.q_weight + i) : 1.f;
+            norm_w[D + i] = p.k_weight ? __ldg(p.k_weight + i) : 1.f;
+        }
+    }
 
     grid_dependency_wait();
     grid_launch_dependents();
@@ -275,6 +295,12 @@ __global__ void __launch_bounds__(kWarps * 32) decode_warp_kernel(const WarpPara
             const uint32_t q_dst = v_dst + C::kTileBytes;
             const __nv_bfloat16 *qs = p.q + ((size_t)c.b * p.Hq + (size_t)c.kvh * p.G) * D;
             for (int i = lane; i < p.G * (D / 8); i += 32) cp_async_16_full(q_dst + i * 16, qs + i * 8);
+            if (fused_rope && c.len >= 1 && c.len - 1 < p.rope_n_pos) {
+                // cos | sin of the unit's newest position, behind the query rows: D/8 pieces of 16 bytes each
+                const uint32_t r_dst = q_dst + (uint32_t)p.G * D * 2;
+                const float *row = (lane < D / 8 ? p.rope_cos : p.rope_sin) + (size_t)(c.len - 1) * (D / 2);
+                if (lane < D / 4) cp_async_16_full(r_dst + lane * 16, row + (lane % (D / 8)) * 4);
+            }
         }
     };
 
@@ -339,6 +365,14 @@ __global__ void __launch_bounds__(kWarps * 32) decode_warp_kernel(const WarpPara
             if constexpr (F8) {
                 k_sc = __ldg(p.k_scale + tail.kvh);
                 v_sc = __ldg(p.v_scale + tail.kvh);
+            } else if (fused_rope && tail.len >= 1 && tail.len - 1 < p.rope_n_pos) {
+                // keep the unit's cos | sin rows (its first stage is recycled before the chunk with the new token), then
+                // rotate the q fragments in registers
+                const float4 *src = reinterpret_cast<const float4 *>(stg + 2 * C::kTileBytes + (size_t)p.G * D * 2);
+                __syncwarp();
+                for (int i = lane; i < D / 4; i += 32) reinterpret_cast<float4 *>(rope_priv)[i] = src[i];
+                __syncwarp();
+                rope_q_fragments<D>(qf, p.G, p.q_weight != nullptr, p.norm_eps, rope_priv, norm_w, lane);
             }
         }
         const int t0 = tail.chunk * kChunkT;
@@ -354,8 +388,15 @@ __global__ void __launch_bounds__(kWarps * 32) decode_warp_kernel(const WarpPara
                     slot_t &= p.page_size - 1;
                 }
                 const bool have = p.block_table == nullptr || (outer >= 0 && outer < p.num_pages);
+                const uint32_t off = lane < C::kRowPieces ? (uint32_t)(lane >> 3) * C::kHalfBytes + swz128(row, lane & 7) : 0u;
+                if (fused_rope) {
+                    // the k row arrived as the caller holds it: rotate (+ normalise) it where it sits (all lanes: shuffles)
+                    uint4 kk = make_uint4(0u, 0u, 0u, 0u);
+                    if (lane < C::kRowPieces) kk = *reinterpret_cast<const uint4 *>(stg + off);
+                    kk = rope_k_row<D>(kk, p.k_weight != nullptr, p.norm_eps, rope_priv, norm_w + D, tail.len - 1 < p.rope_n_pos, lane);
+                    if (lane < C::kRowPieces) *reinterpret_cast<uint4 *>(stg + off) = kk;
+                }
                 if (lane < C::kRowPieces) {
-                    const uint32_t off = (uint32_t)(lane >> 3) * C::kHalfBytes + swz128(row, lane & 7);
                     if (have) {
                         const size_t dst = (size_t)outer * p.c_sb + (size_t)tail.kvh * p.c_sh + (size_t)slot_t * p.c_st + lane * 8;
                         *reinterpret_cast<uint4 *>(p.cache_k + dst) = *reinterpret_cast<const uint4 *>(stg + off);
@@ -450,9 +491,9 @@ __global__ void __launch_bounds__(kWarps * 32) decode_warp_kernel(const WarpPara
     cp_async_wait<0>();
 }
 
-size_t warp_smem_bytes(int D, int G, int warps, int stages, bool f8)
+size_t warp_smem_bytes(int D, int G, int warps, int stages, bool f8, bool rope)
 {
-    return kMetaBytes + (size_t)warps * stages * stage_bytes(D, G, f8);
+    return kMetaBytes + (size_t)warps * stages * stage_bytes(D, G, f8, rope) + rope_extra_bytes(D, warps, rope);
 }
 
 template <int D, int W, bool F8>
@@ -483,11 +524,11 @@ int blocks_per_sm(size_t smem)
 // rings are fastest; with few units per SM a warp's chain of memory round trips is the bound and fewer warps with
 // deeper rings (up to 6 chunks) are. head_dim 64 runs two CTAs per SM (of 8 warps at most: registers).
 struct WarpShape { int warps, stages, ctas_per_sm; };
-WarpShape pick_warp_shape(int D, int G, long long units, bool f8)
+WarpShape pick_warp_shape(int D, int G, long long units, bool f8, bool rope = false)
 {
     const int cps = D == 64 ? 2 : 1;
-    const size_t budget = (D == 64 ? 113u : 227u) * 1024u - kMetaBytes;
-    const int total = (int)(budget / stage_bytes(D, G, f8));         // chunks of ring per CTA
+    const size_t budget = (D == 64 ? 113u : 227u) * 1024u - kMetaBytes - rope_extra_bytes(D, 12, rope);
+    const int total = (int)(budget / stage_bytes(D, G, f8, rope));   // chunks of ring per CTA
     const long long ctas = (long long)sm_count() * cps;
     const long long per_cta = (units + ctas - 1) / ctas;
     const int wmax = (D == 128 && total >= 24) ? 12 : 8;
@@ -525,7 +566,9 @@ bool decode_warp_eligible(int B, int Hq, int Hkv, int D, int max_kv_len, bool fp
     const long long units = (long long)B * Hkv;
     // fp8 caches: plain decode only (the fused append of an fp8 cache quantises the new token, which this kernel's
     // copy path cannot do on the way)
-    if (rope || (fp8 && (append || D != 128)) || G > 16 || pick_warp_shape(D, G, units, fp8).stages == 0) return false;
+    if ((rope && (fp8 || !append)) || (fp8 && (append || D != 128)) || G > 16 ||
+        pick_warp_shape(D, G, units, fp8, rope).stages == 0)
+        return false;
     if (const int forced = decode_override().warp; forced >= 0) return forced != 0;
     // many units of a few chunks each: the regime where the split kernel pays its per-piece cost every tile or two.
     // Thresholds measured against the split kernel in CUDA graphs (8 KV heads at head_dim 128, 12 at head_dim 64),
@@ -540,18 +583,19 @@ bool decode_warp_eligible(int B, int Hq, int Hkv, int D, int max_kv_len, bool fp
 l4l_status launch_decode_warp(const void *q, void *o, const l4l_kv_cache &cache, const int32_t *d_kv_lens,
                               int max_kv_len, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
                               cudaStream_t stream, const l4l_tensor4 *k_new, const l4l_tensor4 *v_new,
-                              const PagedTable *paged, const Fp8Scales *fp8)
+                              const PagedTable *paged, const Fp8Scales *fp8, const RopeArgs *rope)
 {
     const int G = Hq / Hkv;
     const bool f8 = fp8 != nullptr;
     if (G > 16 || (k_new == nullptr) != (v_new == nullptr) || (f8 && (k_new || D != 128))) return L4L_ERR_UNSUPPORTED;
+    if (rope && (f8 || !k_new)) return L4L_ERR_UNSUPPORTED;
     for (int b0 = 0; b0 < B; b0 += kMaxB) {
         const int nb = B - b0 < kMaxB ? B - b0 : kMaxB;
         const long long units = (long long)nb * Hkv;
-        const WarpShape shape = pick_warp_shape(D, G, units, f8);
+        const WarpShape shape = pick_warp_shape(D, G, units, f8, rope != nullptr);
         const int stages = shape.stages, kWarps = shape.warps;
         if (stages == 0) return L4L_ERR_UNSUPPORTED;
-        const size_t smem = warp_smem_bytes(D, G, kWarps, stages, f8);
+        const size_t smem = warp_smem_bytes(D, G, kWarps, stages, f8, rope != nullptr);
         const KernelEntry kernel = pick_kernel(D, kWarps, f8);
         const int per_sm = kernel.blocks(smem);
         if (per_sm == 0) return L4L_ERR_CUDA;
@@ -574,6 +618,12 @@ l4l_status launch_decode_warp(const void *q, void *o, const l4l_kv_cache &cache,
         p.cache_v = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(cache.v) + base_bytes);
         p.k_scale = f8 ? fp8->k_scale : nullptr;
         p.v_scale = f8 ? fp8->v_scale : nullptr;
+        p.rope_cos = rope ? rope->cos : nullptr;
+        p.rope_sin = rope ? rope->sin : nullptr;
+        p.q_weight = rope ? rope->q_weight : nullptr;
+        p.k_weight = rope ? rope->k_weight : nullptr;
+        p.norm_eps = rope ? rope->eps : 0.f;
+        p.rope_n_pos = rope ? rope->n_pos : 0;
         p.c_sb = cache.stride_b; p.c_sh = cache.stride_h; p.c_st = cache.stride_t;
         p.block_table = paged ? paged->block_table + (size_t)b0 * paged->table_stride : nullptr;
         p.table_stride = paged ? paged->table_stride : 0;

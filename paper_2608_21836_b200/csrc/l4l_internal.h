@@ -111,13 +111,13 @@ l4l_status launch_decode_cluster(const void *q, void *o, const l4l_kv_cache &cac
                                  const l4l_tensor4 *v_new, const PagedTable *paged, const RopeArgs *rope,
                                  const Fp8Scales *fp8, int width);
 
-// Many short sequences: one warp per (sequence, KV head), no merge (bf16 caches, fp8 caches without the fused append, groups of up to 16 query heads, no
-// rotary fusion). decode_warp_eligible says whether launch_decode should hand the call over.
+// Many short sequences: one warp per (sequence, KV head), no merge (bf16 caches with or without the fused append and
+// the rotary fusion, fp8 caches without them, groups of up to 16 query heads). decode_warp_eligible says whether launch_decode should hand the call over.
 bool decode_warp_eligible(int B, int Hq, int Hkv, int D, int max_kv_len, bool fp8, bool rope, bool append);
 l4l_status launch_decode_warp(const void *q, void *o, const l4l_kv_cache &cache, const int32_t *d_kv_lens,
                               int max_kv_len, int B, int Hq, int Hkv, int D, float scale, float *d_lse,
                               cudaStream_t stream, const l4l_tensor4 *k_new, const l4l_tensor4 *v_new,
-                              const PagedTable *paged, const Fp8Scales *fp8);
+                              const PagedTable *paged, const Fp8Scales *fp8, const RopeArgs *rope);
 
 l4l_status launch_rope_kv_append(const l4l_tensor4 &q, const l4l_tensor4 &k_new, const l4l_tensor4 &v_new,
                                  const l4l_kv_cache &cache, const int32_t *d_pos, const int32_t *d_n_new, int T, int B,

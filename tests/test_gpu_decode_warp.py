@@ -178,7 +178,7 @@ def test_warp_decode_fp8_cache(warp_kernel, Hq, Hkv):
     import test_gpu_fp8 as f8
 
     assert l4l.l4l_decode_kernel_choice(13, Hq, Hkv, 128, 2304, fp8=True)[0] == "warp"       # forced on by the fixture
-    f8.test_fp8_decode_matches_oracle(Hq, Hkv)
+    f8.test_fp8_decode_matches_oracle(Hq, Hkv, 128)
     f8._fp8_append_case(Hq, Hkv, [1, 16, 17, 33, 255, 300, 0], seed=3500 + Hq, Lmax=320)
 
 
@@ -186,7 +186,7 @@ def test_warp_decode_fp8_cache(warp_kernel, Hq, Hkv):
 def test_warp_decode_fp8_paged_cache(warp_kernel, page):
     import test_gpu_fp8 as f8
 
-    f8.test_fp8_paged_decode_matches_oracle(page)
+    f8.test_fp8_paged_decode_matches_oracle(page, 128)
 
 
 def test_warp_decode_fp8_many_short_sequences(warp_kernel):
@@ -215,3 +215,68 @@ def test_warp_decode_fp8_many_short_sequences(warp_kernel):
     fin = np.isfinite(ref_lse)
     assert np.abs(lse.cpu().double().numpy()[fin] - ref_lse[fin]).max() <= 2e-3
     assert (lse.cpu().numpy()[~fin] == -np.inf).all()
+
+
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("Hq,Hkv", [(8, 2), (4, 4), (16, 1), (32, 8)])
+@pytest.mark.parametrize("norm", [False, True])
+@pytest.mark.parametrize("page", [None, 32])
+def test_warp_decode_step_with_rope_and_append_in_one_launch(warp_kernel, D, Hq, Hkv, norm, page):
+    """The whole decode step (rotary embedding and optional RMS norm of the new token's q and k, cache update,
+    attention) on the warp-per-unit kernel, against the oracle chain rope -> append -> decode over several steps."""
+    from paper_2608_21836_b200.workloads import make_rope_tables
+    from test_gpu_rope_append import assert_bf16_close
+
+    B, Lmax, steps, n_pos = 9, 320, 3, 320
+    lens = np.array([1, 2, 16, 17, 33, 128, 129, 250, 310], np.int32)     # kv_len INCLUDING the new token at the first step
+    g = torch.Generator().manual_seed(1900 + D + Hq + norm)
+    ck = torch.randn(B, Hkv, Lmax, D, generator=g).to(torch.bfloat16)
+    cv = torch.randn(B, Hkv, Lmax, D, generator=g).to(torch.bfloat16)
+    cos, sin = make_rope_tables(n_pos, D)
+    qw = (torch.rand(D, generator=g) + 0.5) if norm else None
+    kw = (torch.rand(D, generator=g) + 0.5) if norm else None
+    eps = 1e-6 if norm else 0.0
+    scale = 1.0 / math.sqrt(D)
+    ock, ocv = orc.bits(ck), orc.bits(cv)
+    if page is None:
+        dck, dcv, table = ck.cuda(), cv.cuda(), None
+    else:
+        n_per = Lmax // page
+        table = torch.randperm(B * n_per, generator=g).view(B, n_per).to(torch.int32)
+        pool_k = torch.zeros(B * n_per, Hkv, page, D, dtype=torch.bfloat16)
+        pool_v = torch.zeros_like(pool_k)
+        for b in range(B):
+            for i in range(n_per):
+                pool_k[table[b, i]] = ck[b, :, i * page:(i + 1) * page]
+                pool_v[table[b, i]] = cv[b, :, i * page:(i + 1) * page]
+        dck, dcv = pool_k.cuda(), pool_v.cuda()
+    ws = l4l.new_workspace(l4l.L4L_OP_DECODE, B, Hq, Hkv, D, Lmax)
+    dcos, dsin = cos.cuda(), sin.cuda()
+    assert l4l.l4l_decode_kernel_choice(B, Hq, Hkv, D, Lmax)[0] == "warp"           # forced on by the fixture
+    for s in range(steps):
+        q = torch.randn(B, Hq, D, generator=g).to(torch.bfloat16)
+        kn = torch.randn(B, 1, Hkv, D, generator=g).to(torch.bfloat16)
+        vn = torch.randn(B, 1, Hkv, D, generator=g).to(torch.bfloat16)
+        cur = lens + s
+        oq, ock, ocv, _, _ = orc.rope_kv_append(q.view(B, 1, Hq, D), kn, vn, ock, ocv, cur - 1, None, cos.numpy(),
+                                                sin.numpy(), None if qw is None else qw.numpy(),
+                                                None if kw is None else kw.numpy(), eps)
+        ref, _ = orc.decode(oq[:, 0], ock, ocv, cur, scale)
+        o = torch.zeros(B, Hq, D, dtype=torch.bfloat16, device="cuda")
+        kwargs = dict(q_weight=None if qw is None else qw.cuda(), k_weight=None if kw is None else kw.cuda(), eps=eps)
+        if page is None:
+            l4l.l4l_attn_decode_rope_append(q.cuda(), o, dck, dcv, kn.cuda(), vn.cuda(), torch.from_numpy(cur).cuda(), Lmax,
+                                            scale, dcos, dsin, ws, **kwargs)
+        else:
+            l4l.l4l_attn_decode_paged_rope_append(q.cuda(), o, dck, dcv, table.cuda(), kn.cuda(), vn.cuda(),
+                                                  torch.from_numpy(cur).cuda(), Lmax, scale, dcos, dsin, ws, **kwargs)
+        torch.cuda.synchronize()
+        assert l4l.l4l_last_device_error(ws) == 0
+        assert_close_to_oracle(o.cpu(), ref, f"warp kernel: rope + append + decode, step {s}")
+    if page is None:
+        assert_bf16_close(dck, ock, "cache k after the fused steps")
+        assert np.array_equal(orc.bits(dcv.cpu()), ocv)
+    else:
+        got_k = orc.gather_pages(dck.cpu(), table.numpy(), Lmax)
+        assert_bf16_close(torch.from_numpy(got_k.view(np.int16)).view(torch.bfloat16), ock, "paged cache k after the fused steps")
+        assert np.array_equal(orc.gather_pages(dcv.cpu(), table.numpy(), Lmax), ocv)
