@@ -140,6 +140,16 @@ size_t decode_smem_bytes(int G, int nsplit)
            kPostRing * sizeof(PieceMeta);
 }
 
+// n / d for 0 <= n < 2^23, 0 < d < 2^23 without the integer-division sequence (the producer lane's partition
+// arithmetic sits on the path to the first load of the kernel): a float quotient, corrected by at most one.
+__device__ __forceinline__ int small_div(int n, int d)
+{
+    int q = (int)__fdividef((float)n, (float)d);
+    if (q * d > n) --q;
+    if ((q + 1) * d <= n) ++q;
+    return q;
+}
+
 __device__ __forceinline__ void order_coords(const TmapCoord &c, int t, int h, int b, int &c1, int &c2, int &c3)
 {
     c1 = (c.pos_t == 1) ? t : (c.pos_h == 1) ? h : b;
@@ -260,11 +270,11 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             // Even split of the tile stream: the first `rem` CTAs take q+1 tiles, the others q, so that
             // no CTA idles; if that would be fewer than the floor, every CTA takes the floor instead (and
             // the last CTAs get nothing).
-            int q = total / (int)gridDim.x, rem = total % (int)gridDim.x;
+            int q = small_div(total, (int)gridDim.x), rem = total - q * (int)gridDim.x;
             if (q < p.min_tiles) { q = p.min_tiles; rem = 0; }
             const int big = rem * (q + 1);                 // tiles covered by the CTAs that take q+1
             auto range_begin = [&](int c) { return min(total, c * q + min(c, rem)); };
-            auto cta_of = [&](int t) { return t < big ? t / (q + 1) : rem + (t - big) / q; };
+            auto cta_of = [&](int t) { return t < big ? small_div(t, q + 1) : rem + small_div(t - big, q); };
             const int my_begin = range_begin((int)blockIdx.x);
             const int my_end = range_begin((int)blockIdx.x + 1);
             uint32_t it = 0, n_posted = 0;
@@ -284,7 +294,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 b_ = lo;
                 len_ = lens_s[lo];
                 tiles_ = (len_ + kTileT - 1) / kTileT;
-                kvh_ = (g - cum[lo]) / (tiles_ + 1);
+                kvh_ = small_div(g - cum[lo], tiles_ + 1);
                 first_ = cum[lo] + kvh_ * (tiles_ + 1);          // flattened index of this sequence's marker; tile t at +1+t
             };
             int b = 0, kvh = 0, len = 0, tiles_b = 0, seq_first = 0;
@@ -346,11 +356,16 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     // tile only the pages that hold tokens are fetched.
                     const bool paged = p.block_table != nullptr;
                     const int rem = len - tile * kTileT;
-                    const int groups = (rem + p.tail_rows - 1) / p.tail_rows;
-                    const bool by_groups = rem < kTileT && groups * p.tail_rows * 2 <= kTileT;
-                    const int box_rows = by_groups ? p.tail_rows : (paged ? p.page_box : kTileT);
-                    const int n_box = by_groups ? groups : ((rem >= kTileT || box_rows == kTileT) ? kTileT / box_rows
-                                                                                                  : (rem + box_rows - 1) / box_rows);
+                    // (a whole tile of a contiguous cache, which is nearly every tile, is one box: no division on that path)
+                    bool by_groups = false;
+                    int box_rows = kTileT, n_box = 1;
+                    if (rem < kTileT || paged) {
+                        const int groups = (rem + p.tail_rows - 1) / p.tail_rows;
+                        by_groups = rem < kTileT && groups * p.tail_rows * 2 <= kTileT;
+                        box_rows = by_groups ? p.tail_rows : (paged ? p.page_box : kTileT);
+                        n_box = by_groups ? groups : ((rem >= kTileT || box_rows == kTileT) ? kTileT / box_rows
+                                                                                              : (rem + box_rows - 1) / box_rows);
+                    }
                     const uint32_t kv_bytes = (uint32_t)n_box * box_rows * (uint32_t)C::kTokBytes * C::kHalves * 2u;
                     // with the rope fused into the step, the piece's first tile also brings the cos / sin rows of
                     // the new token's position (kv_len - 1), if the table has it

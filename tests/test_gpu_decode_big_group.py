@@ -69,9 +69,9 @@ def test_big_group_decode_with_fused_append(Hq):
 def test_big_group_decode_fp8_cache():
     from test_gpu_fp8 import test_fp8_decode_matches_oracle as fp8_case
 
-    fp8_case(64, 8)
-    fp8_case(40, 8)
-    fp8_case(128, 8)
+    fp8_case(64, 8, 128)
+    fp8_case(40, 8, 128)
+    fp8_case(128, 8, 128)
 
 
 @pytest.mark.parametrize("Hq,page_size", [(64, 64), (64, 16), (128, 256), (128, 64), (128, 32), (128, 16)])

@@ -129,8 +129,8 @@ def test_cluster_decode_step_with_rope_and_append(cluster_width, D, Hq, Hkv, nor
 def test_cluster_decode_fp8_cache(cluster_width):
     from test_gpu_fp8 import test_fp8_decode_matches_oracle as fp8_case
 
-    fp8_case(16, 2)
-    fp8_case(8, 8)
+    fp8_case(16, 2, 128)
+    fp8_case(8, 8, 128)
 
 
 @pytest.mark.parametrize("cluster_width", [1, 4, 8], indirect=True)
@@ -138,7 +138,7 @@ def test_cluster_decode_fp8_cache(cluster_width):
 def test_cluster_decode_fp8_paged(cluster_width, page):
     from test_gpu_fp8 import test_fp8_paged_decode_matches_oracle as fp8_paged_case
 
-    fp8_paged_case(page)
+    fp8_paged_case(page, 128)
 
 
 def test_library_choice_matches_split_kernel_result():
