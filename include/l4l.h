@@ -20,8 +20,8 @@
  *   update fused in, over a contiguous or a paged cache), l4l_attn_decode_append (cache
  *   update fused into the decode step), l4l_rope_kv_append (rotary embedding and QK-norm fused
  *   with the cache update), l4l_attn_decode_paged / l4l_kv_append_paged / l4l_attn_decode_paged_append
- *   (page pool + block table), l4l_attn_decode_fp8 / l4l_kv_append_fp8 / l4l_attn_decode_append_fp8
- *   (e4m3 cache), l4l_attn_decode_static (no caller workspace), and a second workload,
+ *   (page pool + block table), l4l_attn_decode_fp8 / l4l_kv_append_fp8 / l4l_attn_decode_append_fp8 /
+ *   l4l_attn_decode_rope_append_fp8 (e4m3 cache), l4l_attn_decode_static (no caller workspace), and a second workload,
  *   l4l_rglru_scan (gated linear recurrence).
  *
  * Conventions shared by every call
@@ -215,7 +215,7 @@ l4l_status l4l_attn_decode_paged_append_fp8(const void *q, void *o, l4l_paged_kv
  * the rotated q attends over slots 0 .. kv_lens[b] - 1. Same result as l4l_rope_kv_append (T = 1) followed by
  * l4l_attn_decode, up to the last bf16 bit of the rotated values (the sum of squares of the norm is reduced
  * in a different order). q is NOT modified (the rotated values live in registers only). A position outside
- * [0, n_pos) leaves q and k unrotated. bf16 caches only.
+ * [0, n_pos) leaves q and k unrotated.
  *   arguments as for l4l_attn_decode_append and l4l_rope_kv_append
  */
 l4l_status l4l_attn_decode_rope_append(const void *q, void *o, l4l_kv_cache cache, l4l_tensor4 k_new, l4l_tensor4 v_new,
@@ -231,6 +231,24 @@ l4l_status l4l_attn_decode_paged_rope_append(const void *q, void *o, l4l_paged_k
                                              int head_dim, float scale, const float *d_cos, const float *d_sin, int n_pos,
                                              const float *d_q_weight, const float *d_k_weight, float norm_eps,
                                              float *d_lse, void *workspace, size_t ws_bytes, l4l_stream stream);
+/* The same step over an e4m3 cache (contiguous, or a page pool behind a block table): k_new is rotated (and
+ * normalised) as above, rounded to bf16, and then quantised with the arithmetic of l4l_kv_append_fp8, so the stored
+ * codes are those of l4l_rope_kv_append followed by l4l_kv_append_fp8 (up to the last bf16 bit of the rotated values
+ * when the norm is on, as above); v_new is quantised as it is. Rules of l4l_attn_decode_append_fp8 /
+ * l4l_attn_decode_paged_append_fp8 for the cache, of l4l_attn_decode_rope_append for the tables. */
+l4l_status l4l_attn_decode_rope_append_fp8(const void *q, void *o, l4l_kv_cache cache8, const float *d_k_scale,
+                                           const float *d_v_scale, l4l_tensor4 k_new, l4l_tensor4 v_new,
+                                           const int32_t *d_kv_lens, int max_kv_len, int B, int Hq, int Hkv,
+                                           int head_dim, float scale, const float *d_cos, const float *d_sin, int n_pos,
+                                           const float *d_q_weight, const float *d_k_weight, float norm_eps,
+                                           float *d_lse, void *workspace, size_t ws_bytes, l4l_stream stream);
+l4l_status l4l_attn_decode_paged_rope_append_fp8(const void *q, void *o, l4l_paged_kv pool8, const float *d_k_scale,
+                                                 const float *d_v_scale, const int32_t *d_block_table, int table_stride,
+                                                 l4l_tensor4 k_new, l4l_tensor4 v_new, const int32_t *d_kv_lens,
+                                                 int max_kv_len, int B, int Hq, int Hkv, int head_dim, float scale,
+                                                 const float *d_cos, const float *d_sin, int n_pos,
+                                                 const float *d_q_weight, const float *d_k_weight, float norm_eps,
+                                                 float *d_lse, void *workspace, size_t ws_bytes, l4l_stream stream);
 
 /*
  * Merge of R partial decode results over DISJOINT parts of the same sequences' caches: the step that

@@ -28,6 +28,7 @@ EXPORTS = (
     "l4l_attn_decode_paged_rope_append", "l4l_attn_decode_append_fp8", "l4l_attn_decode_paged_append_fp8",
     "l4l_attn_prefill_chunk_append", "l4l_attn_prefill_chunk_paged_append", "l4l_rglru_strip_channels",
     "l4l_decode_kernel_choice", "l4l_set_decode_override", "l4l_check_status", "l4l_selftest_wait_expiry",
+    "l4l_attn_decode_rope_append_fp8", "l4l_attn_decode_paged_rope_append_fp8",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -105,6 +106,14 @@ def load() -> ctypes.CDLL:
     lib.l4l_attn_decode_paged_append_fp8.restype = c_int
     lib.l4l_attn_decode_paged_append_fp8.argtypes = [vp, vp, PagedKV, vp, vp, i32p, c_int, Tensor4, Tensor4, i32p, c_int,
                                                      c_int, c_int, c_int, c_int, ctypes.c_float, vp, vp, c_size, vp]
+    lib.l4l_attn_decode_rope_append_fp8.restype = c_int
+    lib.l4l_attn_decode_rope_append_fp8.argtypes = [vp, vp, KVCache, vp, vp, Tensor4, Tensor4, i32p, c_int, c_int, c_int,
+                                                    c_int, c_int, ctypes.c_float, vp, vp, c_int, vp, vp, ctypes.c_float,
+                                                    vp, vp, c_size, vp]
+    lib.l4l_attn_decode_paged_rope_append_fp8.restype = c_int
+    lib.l4l_attn_decode_paged_rope_append_fp8.argtypes = [vp, vp, PagedKV, vp, vp, i32p, c_int, Tensor4, Tensor4, i32p,
+                                                          c_int, c_int, c_int, c_int, c_int, ctypes.c_float, vp, vp, c_int,
+                                                          vp, vp, ctypes.c_float, vp, vp, c_size, vp]
     lib.l4l_decode_kernel_choice.restype = c_int
     lib.l4l_decode_kernel_choice.argtypes = [c_int, c_int, c_int, c_int, c_int, c_int, ctypes.POINTER(c_int)]
     lib.l4l_set_decode_override.restype = None
@@ -474,6 +483,38 @@ def l4l_attn_decode_paged_rope_append(q, o, pool_k, pool_v, block_table, k_new, 
         None if lse is None else lse.data_ptr(), workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream())
     if st != L4L_OK:
         raise L4LError(st, "l4l_attn_decode_paged_rope_append")
+
+
+def l4l_attn_decode_rope_append_fp8(q, o, cache_k8, cache_v8, k_scale, v_scale, k_new, v_new, kv_lens, max_kv_len: int,
+                                    scale: float, cos, sin, workspace, q_weight=None, k_weight=None, eps: float = 0.0,
+                                    lse=None, block_table=None) -> None:
+    """One launch per decode step over an fp8 cache with the rotation fused in: q and k_new are rotated (+ optional RMS
+    norm) at position kv_lens - 1, the rotated k (rounded to bf16) and v_new are quantised as l4l_kv_append_fp8 does and
+    written to slot kv_lens - 1, the rotated q attends. With block_table, the caches are a page pool."""
+    _check_bf16_cuda(q, "q")
+    _check_bf16_cuda(o, "o")
+    if not (q.is_contiguous() and o.is_contiguous() and q.dim() == 3 and q.shape == o.shape):
+        raise ValueError("q and o must be dense [B, Hq, D]")
+    B, Hq, D = q.shape
+    Hkv = cache_k8.shape[1]
+    if tuple(k_new.shape) != (B, 1, Hkv, D) or tuple(v_new.shape) != (B, 1, Hkv, D):
+        raise ValueError("k_new and v_new must be [B, 1, Hkv, D]")
+    n_pos = cos.shape[0]
+    c = kv_cache8(cache_k8, cache_v8)
+    common = (tensor4(k_new, "k_new"), tensor4(v_new, "v_new"), _i32_dev(kv_lens, "kv_lens"), int(max_kv_len), B, Hq, Hkv,
+              D, float(scale), _f32_dev(cos, "cos", (n_pos, D // 2)), _f32_dev(sin, "sin", (n_pos, D // 2)), n_pos,
+              _f32_dev(q_weight, "q_weight", (D,)), _f32_dev(k_weight, "k_weight", (D,)), float(eps),
+              None if lse is None else lse.data_ptr(), workspace.data_ptr(),
+              workspace.numel() * workspace.element_size(), _stream())
+    ks, vs = _f32_dev(k_scale, "k_scale", (Hkv,)), _f32_dev(v_scale, "v_scale", (Hkv,))
+    if block_table is None:
+        st = load().l4l_attn_decode_rope_append_fp8(q.data_ptr(), o.data_ptr(), c, ks, vs, *common)
+    else:
+        pool = PagedKV(c.k, c.v, c.stride_b, c.stride_h, c.stride_t, cache_k8.shape[2], cache_k8.shape[0])
+        tbl, stride = _block_table(block_table, B)
+        st = load().l4l_attn_decode_paged_rope_append_fp8(q.data_ptr(), o.data_ptr(), pool, ks, vs, tbl, stride, *common)
+    if st != L4L_OK:
+        raise L4LError(st, "l4l_attn_decode_rope_append_fp8")
 
 
 def kv_cache8(cache_k8, cache_v8) -> KVCache:

@@ -666,6 +666,62 @@ l4l_status l4l_attn_decode_paged_rope_append(const void *q, void *o, l4l_paged_k
                          plan, static_cast<cudaStream_t>(stream), &k_new, &v_new, &pt, nullptr, &rope);
 }
 
+l4l_status l4l_attn_decode_rope_append_fp8(const void *q, void *o, l4l_kv_cache cache8, const float *d_k_scale,
+                                           const float *d_v_scale, l4l_tensor4 k_new, l4l_tensor4 v_new,
+                                           const int32_t *d_kv_lens, int max_kv_len, int B, int Hq, int Hkv, int head_dim,
+                                           float scale, const float *d_cos, const float *d_sin, int n_pos,
+                                           const float *d_q_weight, const float *d_k_weight, float norm_eps, float *d_lse,
+                                           void *workspace, size_t ws_bytes, l4l_stream stream)
+{
+    l4l_status st = shape_status(B, Hq, Hkv, head_dim);
+    if (st != L4L_OK) return st;
+    if (!q || !o || !d_kv_lens || !d_k_scale || !d_v_scale || !aligned16(q) || !aligned16(o)) return L4L_ERR_INVALID_ARG;
+    if (!cache8_ok(cache8) || !tensor4_ok(k_new) || !tensor4_ok(v_new)) return L4L_ERR_INVALID_ARG;
+    if (max_kv_len < 0 || max_kv_len > cache8.max_len) return L4L_ERR_INVALID_ARG;
+    if (!d_cos || !d_sin || n_pos < 0 || !(norm_eps >= 0.f)) return L4L_ERR_INVALID_ARG;
+    if (!aligned16(d_cos) || !aligned16(d_sin)) return L4L_ERR_INVALID_ARG;      // rows are fetched with bulk copies
+    if (!workspace || ws_bytes < kStatusBytes) return L4L_ERR_WORKSPACE;
+    if (B == 0) return L4L_OK;
+    const DecodePlan plan = plan_decode(B, Hq, Hkv, head_dim, max_kv_len, ws_bytes, true);
+    if (plan.ws_bytes > ws_bytes) return L4L_ERR_WORKSPACE;
+    const Fp8Scales sc{d_k_scale, d_v_scale};
+    const RopeArgs rope{d_cos, d_sin, d_q_weight, d_k_weight, norm_eps, n_pos};
+    return launch_decode(q, o, cache8, d_kv_lens, max_kv_len, B, Hq, Hkv, head_dim, scale, d_lse, workspace, plan,
+                         static_cast<cudaStream_t>(stream), &k_new, &v_new, nullptr, &sc, &rope);
+}
+
+l4l_status l4l_attn_decode_paged_rope_append_fp8(const void *q, void *o, l4l_paged_kv pool8, const float *d_k_scale,
+                                                 const float *d_v_scale, const int32_t *d_block_table, int table_stride,
+                                                 l4l_tensor4 k_new, l4l_tensor4 v_new, const int32_t *d_kv_lens,
+                                                 int max_kv_len, int B, int Hq, int Hkv, int head_dim, float scale,
+                                                 const float *d_cos, const float *d_sin, int n_pos,
+                                                 const float *d_q_weight, const float *d_k_weight, float norm_eps,
+                                                 float *d_lse, void *workspace, size_t ws_bytes, l4l_stream stream)
+{
+    l4l_status st = shape_status(B, Hq, Hkv, head_dim);
+    if (st != L4L_OK) return st;
+    if (!q || !o || !d_kv_lens || !d_block_table || !d_k_scale || !d_v_scale || !aligned16(q) || !aligned16(o))
+        return L4L_ERR_INVALID_ARG;
+    auto s16 = [](int64_t s) { return s >= 0 && (s % 16) == 0; };
+    if (!pool8.k || !pool8.v || !aligned16(pool8.k) || !aligned16(pool8.v) || !s16(pool8.stride_page) ||
+        !s16(pool8.stride_h) || !s16(pool8.stride_t) || pool8.num_pages <= 0 || pool8.page_size < 16 ||
+        pool8.page_size > (1 << 20) || (pool8.page_size & (pool8.page_size - 1)) != 0 || table_stride <= 0)
+        return L4L_ERR_INVALID_ARG;
+    if (!tensor4_ok(k_new) || !tensor4_ok(v_new)) return L4L_ERR_INVALID_ARG;
+    if (max_kv_len < 0 || (long long)max_kv_len > (long long)table_stride * pool8.page_size) return L4L_ERR_INVALID_ARG;
+    if (!d_cos || !d_sin || n_pos < 0 || !(norm_eps >= 0.f)) return L4L_ERR_INVALID_ARG;
+    if (!aligned16(d_cos) || !aligned16(d_sin)) return L4L_ERR_INVALID_ARG;      // rows are fetched with bulk copies
+    if (!workspace || ws_bytes < kStatusBytes) return L4L_ERR_WORKSPACE;
+    if (B == 0) return L4L_OK;
+    const DecodePlan plan = plan_decode(B, Hq, Hkv, head_dim, max_kv_len, ws_bytes, true, pool8.page_size);
+    if (plan.ws_bytes > ws_bytes) return L4L_ERR_WORKSPACE;
+    const PagedTable pt{d_block_table, table_stride, pool8.num_pages};
+    const Fp8Scales sc{d_k_scale, d_v_scale};
+    const RopeArgs rope{d_cos, d_sin, d_q_weight, d_k_weight, norm_eps, n_pos};
+    return launch_decode(q, o, pool_as_cache(pool8), d_kv_lens, max_kv_len, B, Hq, Hkv, head_dim, scale, d_lse, workspace,
+                         plan, static_cast<cudaStream_t>(stream), &k_new, &v_new, &pt, &sc, &rope);
+}
+
 void l4l_set_decode_override(int cluster, int warp, int split_warps)
 {
     g_override_cluster = cluster < 0 ? -1 : cluster;

@@ -775,12 +775,12 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     if constexpr (F8) {
-                        // f16 fragments with the k index permuted the way the fp8 K tiles arrive
+                        // the k index permuted the way the fp8 K tiles arrive (bf16 pairs here, f16 below)
                         const int w = q_frag_f8_word(ks, 0, lane);
-                        qf[ks][0] = v_lo ? bf16x2_to_f16x2(qrow_lo[w]) : 0u;
-                        qf[ks][1] = v_hi ? bf16x2_to_f16x2(qrow_hi[w]) : 0u;
-                        qf[ks][2] = v_lo ? bf16x2_to_f16x2(qrow_lo[w + 1]) : 0u;
-                        qf[ks][3] = v_hi ? bf16x2_to_f16x2(qrow_hi[w + 1]) : 0u;
+                        qf[ks][0] = v_lo ? qrow_lo[w] : 0u;
+                        qf[ks][1] = v_hi ? qrow_hi[w] : 0u;
+                        qf[ks][2] = v_lo ? qrow_lo[w + 1] : 0u;
+                        qf[ks][3] = v_hi ? qrow_hi[w + 1] : 0u;
                     } else {
                         const int w = ks * 8 + (lane & 3);           // 32-bit word index in the row
                         qf[ks][0] = v_lo ? qrow_lo[w] : 0u;
@@ -789,16 +789,20 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                         qf[ks][3] = v_hi ? qrow_hi[w + 4] : 0u;
                     }
                 }
-                if constexpr (!F8) {
-                    if (p.rope_cos != nullptr && mt.kv_len - 1 < p.rope_n_pos) {
-                        // keep this piece's cos | sin rows in the warp's own scratch (the stage is recycled long
-                        // before the tile with the new token arrives), then rotate the q fragments in registers
-                        float *mine = rope_priv + (size_t)warp * D;
-                        const float4 *src = reinterpret_cast<const float4 *>(q_slots + (size_t)s * q_stride + q_bytes);
-                        for (int i = lane; i < D / 4; i += 32) reinterpret_cast<float4 *>(mine)[i] = src[i];
-                        __syncwarp();
-                        rope_q_fragments<D>(qf, p.G, p.q_weight != nullptr, p.norm_eps, mine, norm_w, lane);
-                    }
+                if (p.rope_cos != nullptr && mt.kv_len - 1 < p.rope_n_pos) {
+                    // keep this piece's cos | sin rows in the warp's own scratch (the stage is recycled long
+                    // before the tile with the new token arrives), then rotate the q fragments in registers
+                    float *mine = rope_priv + (size_t)warp * D;
+                    const float4 *src = reinterpret_cast<const float4 *>(q_slots + (size_t)s * q_stride + q_bytes);
+                    for (int i = lane; i < D / 4; i += 32) reinterpret_cast<float4 *>(mine)[i] = src[i];
+                    __syncwarp();
+                    rope_q_fragments<D, F8>(qf, p.G, p.q_weight != nullptr, p.norm_eps, mine, norm_w, lane);
+                }
+                if constexpr (F8) {
+#pragma unroll
+                    for (int ks = 0; ks < D / 16; ++ks)
+#pragma unroll
+                        for (int r = 0; r < 4; ++r) qf[ks][r] = bf16x2_to_f16x2(qf[ks][r]);
                 }
             }
 
@@ -849,11 +853,25 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     // cache update quantises them (same division, same rounding), patched into the tile and written
                     // to their cache slot; 8 lanes, 16 values each
                     const int last = row0 + nvalid - 1;
+                    // the k row: straight from the caller, or (rope fused into the step) rotated first, in the
+                    // arrangement of the bf16 path (8 values per lane), rounded to bf16 and regrouped
+                    uint4 ka = make_uint4(0u, 0u, 0u, 0u), kb = ka;
+                    if (p.rope_cos != nullptr) {
+                        uint4 kk = make_uint4(0u, 0u, 0u, 0u);
+                        if (lane < D / 8)
+                            kk = __ldg(reinterpret_cast<const uint4 *>(p.k_new + (size_t)mt.b * p.new_sb + (size_t)mt.kvh * p.new_sh + lane * 8));
+                        kk = rope_k_row<D>(kk, p.k_weight != nullptr, p.norm_eps, rope_priv + (size_t)warp * D, norm_w + D,
+                                            mt.kv_len - 1 < p.rope_n_pos, lane);
+                        regroup_row_16(kk, lane, ka, kb);
+                    } else if (lane < D / 16) {
+                        const uint4 *ks = reinterpret_cast<const uint4 *>(p.k_new + (size_t)mt.b * p.new_sb + (size_t)mt.kvh * p.new_sh + lane * 16);
+                        ka = __ldg(ks);
+                        kb = __ldg(ks + 1);
+                    }
                     if (lane < D / 16) {
                         const size_t src = (size_t)mt.b * p.new_sb + (size_t)mt.kvh * p.new_sh + lane * 16;
-                        const uint4 *ks = reinterpret_cast<const uint4 *>(p.k_new + src);
                         const uint4 *vs = reinterpret_cast<const uint4 *>(p.v_new + src);
-                        const uint4 kq = quantise16(__ldg(ks), __ldg(ks + 1), k_sc);
+                        const uint4 kq = quantise16(ka, kb, k_sc);
                         const uint4 vq = quantise16(__ldg(vs), __ldg(vs + 1), v_sc);
                         long long outer = mt.b, slot = mt.kv_len - 1;
                         if (p.block_table != nullptr) {
@@ -1184,7 +1202,7 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
                          void *workspace, const DecodePlan &plan, cudaStream_t stream, const l4l_tensor4 *k_new,
                          const l4l_tensor4 *v_new, const PagedTable *paged, const Fp8Scales *fp8, const RopeArgs *rope)
 {
-    if (rope && (!k_new || !v_new || fp8)) return L4L_ERR_UNSUPPORTED;   // only with the fused append, bf16 caches
+    if (rope && (!k_new || !v_new)) return L4L_ERR_UNSUPPORTED;   // only with the fused append
     // fp8: cache.k / cache.v point at e4m3 bytes, the strides count bytes (= elements)
     // fp8 at head_dim 64: two 64-byte tokens make one 128-byte tile row, so the token rows of the cache (or of a page)
     // must lie back to back and come in pairs

@@ -13,7 +13,9 @@ namespace l4l {
 // The q rows live in the A fragments of the warp MMA: a thread holds, per 16-column k-step, columns 2c, 2c+1
 // (registers 0: row lane/4, 1: row lane/4 + 8) and 2c+8, 2c+9 (registers 2, 3), c = lane % 4. The partner of
 // column i is column i + D/2, i.e. the same register of the k-step D/32 further on: no data leaves the thread.
-template <int D>
+// kF8Cols: the fragments of the e4m3-cache kernels, whose k index is permuted the way the byte tiles arrive (registers
+// 0, 1 hold columns 4c, 4c+1 of the k-step, registers 2, 3 columns 4c+2, 4c+3); still bf16 pairs at this point.
+template <int D, bool kF8Cols = false>
 __device__ __forceinline__ void rope_q_fragments(uint32_t (&qf)[D / 16][4], int G, bool with_norm, float norm_eps,
                                                  const float *cos_sin, const float *weight, int lane)
 {
@@ -42,7 +44,8 @@ __device__ __forceinline__ void rope_q_fragments(uint32_t (&qf)[D / 16][4], int 
     for (int ks = 0; ks < kHalf; ++ks)
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
-            const int col = 16 * ks + 2 * c + ((r >> 1) << 3);               // first-half column of element 0
+            const int col = kF8Cols ? 16 * ks + 4 * c + ((r >> 1) << 1)
+                                    : 16 * ks + 2 * c + ((r >> 1) << 3);    // first-half column of element 0
             float x1[2] = {__uint_as_float(qf[ks][r] << 16), __uint_as_float(qf[ks][r] & 0xffff0000u)};
             float x2[2] = {__uint_as_float(qf[ks + kHalf][r] << 16), __uint_as_float(qf[ks + kHalf][r] & 0xffff0000u)};
             float y1[2], y2[2];
@@ -104,6 +107,17 @@ __device__ __forceinline__ uint4 rope_k_row(uint4 kk, bool with_norm, float norm
     }
     if (!in_table) return kk;
     return make_uint4(pack_bf16x2(y[0], y[1]), pack_bf16x2(y[2], y[3]), pack_bf16x2(y[4], y[5]), pack_bf16x2(y[6], y[7]));
+}
+
+// The rotated row regrouped for the e4m3 quantiser: from 8 values per lane (lanes < D/8) to 16 values per lane
+// (lanes < D/16) as two 16-byte pieces. Every lane of the warp must call this.
+__device__ __forceinline__ void regroup_row_16(const uint4 &kk, int lane, uint4 &a, uint4 &b)
+{
+    const int src = (2 * lane) & 31;
+    a.x = __shfl_sync(0xffffffffu, kk.x, src);     a.y = __shfl_sync(0xffffffffu, kk.y, src);
+    a.z = __shfl_sync(0xffffffffu, kk.z, src);     a.w = __shfl_sync(0xffffffffu, kk.w, src);
+    b.x = __shfl_sync(0xffffffffu, kk.x, src + 1); b.y = __shfl_sync(0xffffffffu, kk.y, src + 1);
+    b.z = __shfl_sync(0xffffffffu, kk.z, src + 1); b.w = __shfl_sync(0xffffffffu, kk.w, src + 1);
 }
 
 }  // namespace l4l
