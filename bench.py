@@ -432,6 +432,14 @@ def run_ours(args, rank, world):
         l4l.l4l_attn_decode_append_fp8(dq, do, k8, v8, k_sc, k_sc, dkn, dvn, dlen, Lmax, wd.scale, ws_d)
 
     t_fp8_fused = timed(fp8_fused_step, 21)
+
+    def fp8_rope_step():                                      # ... and with rope + norm of the new token's q and k fused in too
+        k8, v8 = c8[rot[0] % 3]
+        rot[0] += 1
+        l4l.l4l_attn_decode_rope_append_fp8(dq, do, k8, v8, k_sc, k_sc, dkn, dvn, dlen, Lmax, wd.scale, cos_d, sin_d, ws_d,
+                                            q_weight=gamma, k_weight=gamma, eps=1e-6)
+
+    t_fp8_rope = timed(fp8_rope_step, 21)
     del c8
     # the same cache with 64 query heads on the 8 KV heads (groups of 8: the 70B-class shape), three copies in rotation
     Hq8 = 8 * Hkv
@@ -739,7 +747,8 @@ def run_ours(args, rank, world):
                                            "frac_of_measured_hbm": rglru_bytes / (t_rglru2 * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                            "bytes": rglru_bytes},
             "decode_fp8_cache": {"us": t_fp8 * 1e3, "kv_gbs_fp8_bytes": dec_bytes / 2 / (t_fp8 * 1e-3) / 1e9,
-                                 "speedup_over_bf16_cache": t_dec_b2b / t_fp8, "with_fused_append_us": t_fp8_fused * 1e3},
+                                 "speedup_over_bf16_cache": t_dec_b2b / t_fp8, "with_fused_append_us": t_fp8_fused * 1e3,
+                                 "with_rope_norm_and_append_us": t_fp8_rope * 1e3},
             "decode_64_query_heads_on_8_kv_heads": {"us": t_g8 * 1e3, "kv_gbs": dec_bytes / (t_g8 * 1e-3) / 1e9},
             "other_configs": other,
             "decode_B512_L64_to_256": {"warp_kernel_us": t_short * 1e3, "kv_gbs": short_bytes / (t_short * 1e-3) / 1e9,

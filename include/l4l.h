@@ -214,7 +214,7 @@ l4l_status l4l_attn_decode_paged_append_fp8(const void *q, void *o, l4l_paged_kv
  * l4l_rope_kv_append at that position, the rotated k and v_new are written to cache slot kv_lens[b] - 1, and
  * the rotated q attends over slots 0 .. kv_lens[b] - 1. Same result as l4l_rope_kv_append (T = 1) followed by
  * l4l_attn_decode, up to the last bf16 bit of the rotated values (the sum of squares of the norm is reduced
- * in a different order). q is NOT modified (the rotated values live in registers only). A position outside
+ * in a different order). q is NOT modified (the rotated values live on chip only). A position outside
  * [0, n_pos) leaves q and k unrotated.
  *   arguments as for l4l_attn_decode_append and l4l_rope_kv_append
  */

@@ -157,7 +157,9 @@ __device__ __forceinline__ void order_coords(const TmapCoord &c, int t, int h, i
     c3 = (c.pos_t == 3) ? t : (c.pos_h == 3) ? h : b;
 }
 
-template <int D, int W, bool F8, bool BigG>
+// R8: an e4m3-cache kernel that also carries the rope-fused step. A build of its own, so that the rotation code does
+// not weigh on the registers of the plain fp8 kernels, which are bound by their consumer warps (bf16 kernels always carry it).
+template <int D, int W, bool F8, bool BigG, bool R8 = false>
 __global__ void __launch_bounds__((BigG ? 11 : W + 2) * 32)
 decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
                     const __grid_constant__ CUtensorMap tmap_k_tail, const __grid_constant__ CUtensorMap tmap_v_tail,
@@ -198,6 +200,8 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     // finisher leaves right after the last one
     volatile uint32_t *pieces_total = posted_count + 1;
     PieceMeta *post_ring = reinterpret_cast<PieceMeta *>(lens_s + kMaxB + 4);
+    // consumers among themselves: the piece's query rows have been rotated in place (rope fused into the step)
+    uint64_t *q_rotated = reinterpret_cast<uint64_t *>((reinterpret_cast<uintptr_t>(post_ring + kPostRing) + 7) & ~(uintptr_t)7);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -208,6 +212,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             mbar_init(&empty[s], kConsumerWarps);
         }
         mbar_init(comb_full, kConsumerWarps);
+        mbar_init(q_rotated, kConsumerWarps);
         mbar_init(comb_empty, BigG ? p.nfin : 1);
         *abort_flag = 0;
         *posted_count = 0u;
@@ -752,6 +757,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
         const int r_lo = lane >> 2;          // query head within the group held in rows lane/4, lane/4+8
         const int r_hi = r_lo + 8;
         uint32_t n_dumps = 0;                // pieces handed to the finisher so far
+        uint32_t n_rotated = 0;              // pieces whose query rows were rotated (phase of q_rotated)
         float k_sc = 1.f, v_sc = 1.f;        // fp8 cache: scales of the piece's KV head (read once per piece)
 
         for (uint32_t it = 0;; ++it) {
@@ -768,6 +774,26 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     k_sc = __ldg(p.k_scale + mt.kvh);
                     v_sc = __ldg(p.v_scale + mt.kvh);
                 }
+                if constexpr (!F8 || R8) {
+                    if (p.rope_cos != nullptr && mt.kv_len - 1 < p.rope_n_pos) {
+                        // Rope fused into the step: the piece's query rows are rotated in place in the stage's slot, row g by
+                        // consumer warp g mod W, before anybody builds fragments from them. Every warp also keeps the
+                        // cos | sin rows in its own scratch: the stage is recycled long before the tile with the new
+                        // token (whose k row needs them) arrives.
+                        uint8_t *slot = q_slots + (size_t)s * q_stride;
+                        float *mine = rope_priv + (size_t)warp * D;
+                        const float4 *src = reinterpret_cast<const float4 *>(slot + q_bytes);
+                        for (int i = lane; i < D / 4; i += 32) reinterpret_cast<float4 *>(mine)[i] = src[i];
+                        __syncwarp();
+                        for (int g = warp; g < p.G; g += kConsumerWarps)
+                            rope_row_in_smem<D>(reinterpret_cast<uint32_t *>(slot) + (size_t)g * (D / 2), mine, p.q_weight != nullptr,
+                                                p.norm_eps, norm_w, lane);
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(q_rotated);
+                        if (!mbar_wait(q_rotated, n_rotated & 1u, abort_flag)) break;
+                        ++n_rotated;
+                    }
+                }
                 const uint32_t *qs = reinterpret_cast<const uint32_t *>(q_slots + (size_t)s * q_stride);
                 const uint32_t *qrow_lo = qs + (size_t)r_lo * D / 2;
                 const uint32_t *qrow_hi = qs + (size_t)r_hi * D / 2;
@@ -775,12 +801,12 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     if constexpr (F8) {
-                        // the k index permuted the way the fp8 K tiles arrive (bf16 pairs here, f16 below)
+                        // f16 fragments with the k index permuted the way the fp8 K tiles arrive
                         const int w = q_frag_f8_word(ks, 0, lane);
-                        qf[ks][0] = v_lo ? qrow_lo[w] : 0u;
-                        qf[ks][1] = v_hi ? qrow_hi[w] : 0u;
-                        qf[ks][2] = v_lo ? qrow_lo[w + 1] : 0u;
-                        qf[ks][3] = v_hi ? qrow_hi[w + 1] : 0u;
+                        qf[ks][0] = v_lo ? bf16x2_to_f16x2(qrow_lo[w]) : 0u;
+                        qf[ks][1] = v_hi ? bf16x2_to_f16x2(qrow_hi[w]) : 0u;
+                        qf[ks][2] = v_lo ? bf16x2_to_f16x2(qrow_lo[w + 1]) : 0u;
+                        qf[ks][3] = v_hi ? bf16x2_to_f16x2(qrow_hi[w + 1]) : 0u;
                     } else {
                         const int w = ks * 8 + (lane & 3);           // 32-bit word index in the row
                         qf[ks][0] = v_lo ? qrow_lo[w] : 0u;
@@ -788,21 +814,6 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                         qf[ks][2] = v_lo ? qrow_lo[w + 4] : 0u;
                         qf[ks][3] = v_hi ? qrow_hi[w + 4] : 0u;
                     }
-                }
-                if (p.rope_cos != nullptr && mt.kv_len - 1 < p.rope_n_pos) {
-                    // keep this piece's cos | sin rows in the warp's own scratch (the stage is recycled long
-                    // before the tile with the new token arrives), then rotate the q fragments in registers
-                    float *mine = rope_priv + (size_t)warp * D;
-                    const float4 *src = reinterpret_cast<const float4 *>(q_slots + (size_t)s * q_stride + q_bytes);
-                    for (int i = lane; i < D / 4; i += 32) reinterpret_cast<float4 *>(mine)[i] = src[i];
-                    __syncwarp();
-                    rope_q_fragments<D, F8>(qf, p.G, p.q_weight != nullptr, p.norm_eps, mine, norm_w, lane);
-                }
-                if constexpr (F8) {
-#pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks)
-#pragma unroll
-                        for (int r = 0; r < 4; ++r) qf[ks][r] = bf16x2_to_f16x2(qf[ks][r]);
                 }
             }
 
@@ -856,14 +867,19 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     // the k row: straight from the caller, or (rope fused into the step) rotated first, in the
                     // arrangement of the bf16 path (8 values per lane), rounded to bf16 and regrouped
                     uint4 ka = make_uint4(0u, 0u, 0u, 0u), kb = ka;
-                    if (p.rope_cos != nullptr) {
-                        uint4 kk = make_uint4(0u, 0u, 0u, 0u);
-                        if (lane < D / 8)
-                            kk = __ldg(reinterpret_cast<const uint4 *>(p.k_new + (size_t)mt.b * p.new_sb + (size_t)mt.kvh * p.new_sh + lane * 8));
-                        kk = rope_k_row<D>(kk, p.k_weight != nullptr, p.norm_eps, rope_priv + (size_t)warp * D, norm_w + D,
-                                            mt.kv_len - 1 < p.rope_n_pos, lane);
-                        regroup_row_16(kk, lane, ka, kb);
-                    } else if (lane < D / 16) {
+                    bool rotated = false;
+                    if constexpr (R8) {
+                        if (p.rope_cos != nullptr) {
+                            uint4 kk = make_uint4(0u, 0u, 0u, 0u);
+                            if (lane < D / 8)
+                                kk = __ldg(reinterpret_cast<const uint4 *>(p.k_new + (size_t)mt.b * p.new_sb + (size_t)mt.kvh * p.new_sh + lane * 8));
+                            kk = rope_k_row<D>(kk, p.k_weight != nullptr, p.norm_eps, rope_priv + (size_t)warp * D, norm_w + D,
+                                                mt.kv_len - 1 < p.rope_n_pos, lane);
+                            regroup_row_16(kk, lane, ka, kb);
+                            rotated = true;
+                        }
+                    }
+                    if (!rotated && lane < D / 16) {
                         const uint4 *ks = reinterpret_cast<const uint4 *>(p.k_new + (size_t)mt.b * p.new_sb + (size_t)mt.kvh * p.new_sh + lane * 16);
                         ka = __ldg(ks);
                         kb = __ldg(ks + 1);
@@ -1067,7 +1083,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
 }
 
 // Resident CTAs per SM for a given dynamic shared-memory size (0 on failure).
-template <int D, int W, bool F8, bool BigG>
+template <int D, int W, bool F8, bool BigG, bool R8 = false>
 int decode_blocks_per_sm(size_t smem)
 {
     static bool attr_set_on[kDeviceSlots] = {};
@@ -1077,14 +1093,14 @@ int decode_blocks_per_sm(size_t smem)
     std::lock_guard<std::mutex> lock(setup_mutex());
     if (!attr_set) {
         // the opt-in limit is per kernel: allow everything the SM has
-        if (cudaFuncSetAttribute(decode_split_kernel<D, W, F8, BigG>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+        if (cudaFuncSetAttribute(decode_split_kernel<D, W, F8, BigG, R8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
             cudaSuccess)
             return 0;
         attr_set = true;
     }
     if (smem > 227 * 1024) return 0;
     int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_split_kernel<D, W, F8, BigG>, (BigG ? 11 : W + 2) * 32, smem) != cudaSuccess)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_split_kernel<D, W, F8, BigG, R8>, (BigG ? 11 : W + 2) * 32, smem) != cudaSuccess)
         return 0;
     return n;
 }
@@ -1100,10 +1116,10 @@ struct ShapeOps {
     int (*blocks_per_sm)(size_t smem);
 };
 
-template <int D, int W, bool F8, bool BigG = false>
+template <int D, int W, bool F8, bool BigG = false, bool R8 = false>
 ShapeOps shape_ops()
 {
-    return ShapeOps{W, DecodeCfg<D, W, F8>::kTileT, &decode_smem_bytes<D, W, F8, BigG>, &decode_blocks_per_sm<D, W, F8, BigG>};
+    return ShapeOps{W, DecodeCfg<D, W, F8>::kTileT, &decode_smem_bytes<D, W, F8, BigG>, &decode_blocks_per_sm<D, W, F8, BigG, R8>};
 }
 
 // Groups of more than 4 query heads at head_dim 128: 16-bit hand-over rows and one finisher warp per 4 heads. Up to 8
@@ -1114,8 +1130,14 @@ bool is_big_group(int D, int warps, int G)
     return D == 128 && ((warps == 8 && G > 4 && G <= 8) || (warps == 6 && G > 8 && G <= 16));
 }
 
-ShapeOps pick_shape(int D, int warps, bool fp8, bool big = false)
+ShapeOps pick_shape(int D, int warps, bool fp8, bool big = false, bool rope8 = false)
 {
+    if (fp8 && rope8) {          // the e4m3-cache kernels that carry the rope-fused step
+        if (big && warps == 6) return shape_ops<128, 6, true, true, true>();
+        if (big) return shape_ops<128, 8, true, true, true>();
+        if (D == 64) return warps == 8 ? shape_ops<64, 8, true, false, true>() : shape_ops<64, 4, true, false, true>();
+        return warps == 8 ? shape_ops<128, 8, true, false, true>() : shape_ops<128, 4, true, false, true>();
+    }
     if (big && warps == 6) return fp8 ? shape_ops<128, 6, true, true>() : shape_ops<128, 6, false, true>();
     if (big) return fp8 ? shape_ops<128, 8, true, true>() : shape_ops<128, 8, false, true>();
     if (fp8 && D == 64) return warps == 8 ? shape_ops<64, 8, true>() : shape_ops<64, 4, true>();
@@ -1224,7 +1246,8 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
     const int G = Hq / Hkv;
     const bool big = is_big_group(D, plan.warps, G);
     const int nfin = big ? (G + 3) / 4 : 1;
-    const ShapeOps ops = pick_shape(D, plan.warps, fp8 != nullptr, big);
+    const bool rope8 = fp8 != nullptr && rope != nullptr;
+    const ShapeOps ops = pick_shape(D, plan.warps, fp8 != nullptr, big, rope8);
     const int kTileT = ops.tile_t;
     const size_t smem = ops.smem_bytes(G, plan.nsplit);
     if (ops.blocks_per_sm(smem) == 0) return L4L_ERR_CUDA;
@@ -1319,7 +1342,16 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         cudaError_t err;
-        if (big && plan.warps == 6)
+        if (rope8 && big)
+            err = plan.warps == 6 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 6, true, true, true>, tk, tv, tk_tail, tv_tail, p)
+                                  : cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 8, true, true, true>, tk, tv, tk_tail, tv_tail, p);
+        else if (rope8 && D == 64)
+            err = plan.warps == 8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<64, 8, true, false, true>, tk, tv, tk_tail, tv_tail, p)
+                                  : cudaLaunchKernelEx(&cfg, decode_split_kernel<64, 4, true, false, true>, tk, tv, tk_tail, tv_tail, p);
+        else if (rope8)
+            err = plan.warps == 8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 8, true, false, true>, tk, tv, tk_tail, tv_tail, p)
+                                  : cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 4, true, false, true>, tk, tv, tk_tail, tv_tail, p);
+        else if (big && plan.warps == 6)
             err = fp8 ? cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 6, true, true>, tk, tv, tk_tail, tv_tail, p)
                       : cudaLaunchKernelEx(&cfg, decode_split_kernel<128, 6, false, true>, tk, tv, tk_tail, tv_tail, p);
         else if (big)

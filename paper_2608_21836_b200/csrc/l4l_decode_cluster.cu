@@ -146,7 +146,8 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
     constexpr uint32_t kRopeBytes = D * 4;
     uint64_t *full = reinterpret_cast<uint64_t *>(norm_w + 2 * D);
     uint64_t *empty = full + C::kMaxStages;
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(empty + C::kMaxStages);
+    uint64_t *q_rotated = empty + C::kMaxStages;     // consumers among themselves: the query rows have been rotated in place
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(q_rotated + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rank = blockIdx.x;                 // cluster = the gridDim.x CTAs of one blockIdx.y
@@ -158,6 +159,7 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
             mbar_init(&full[s], 1);
             mbar_init(&empty[s], kW);
         }
+        mbar_init(q_rotated, kW);
         *abort_flag = 0;
         fence_barrier_init();
         fence_proxy_async_smem();
@@ -254,6 +256,17 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
             const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
             if (!mbar_wait(&full[s], ph, abort_flag)) break;
             if (it == 0) {
+                if (with_rope) {
+                    // rope fused into the step: the query rows are rotated in place in shared memory, row g by consumer
+                    // warp g mod kW, before anybody builds fragments from them (small code: it runs once, from a cold
+                    // instruction cache)
+                    for (int g = warp; g < p.G; g += kW)
+                        rope_row_in_smem<D>(reinterpret_cast<uint32_t *>(q_smem) + (size_t)g * (D / 2), rope_cs, p.q_weight != nullptr,
+                                            p.norm_eps, norm_w, lane);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(q_rotated);
+                    if (!mbar_wait(q_rotated, 0u, abort_flag)) break;
+                }
                 const uint32_t *qs = reinterpret_cast<const uint32_t *>(q_smem);
                 const uint32_t *qrow_lo = qs + (size_t)r_lo * D / 2;
                 const uint32_t *qrow_hi = qs + (size_t)r_hi * D / 2;
@@ -261,12 +274,12 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     if constexpr (F8) {
-                        // the k index permuted the way the fp8 K tiles arrive (bf16 pairs here, f16 below)
+                        // f16 fragments with the k index permuted the way the fp8 K tiles arrive
                         const int w = q_frag_f8_word(ks, 0, lane);
-                        qf[ks][0] = v_lo ? qrow_lo[w] : 0u;
-                        qf[ks][1] = v_hi ? qrow_hi[w] : 0u;
-                        qf[ks][2] = v_lo ? qrow_lo[w + 1] : 0u;
-                        qf[ks][3] = v_hi ? qrow_hi[w + 1] : 0u;
+                        qf[ks][0] = v_lo ? bf16x2_to_f16x2(qrow_lo[w]) : 0u;
+                        qf[ks][1] = v_hi ? bf16x2_to_f16x2(qrow_hi[w]) : 0u;
+                        qf[ks][2] = v_lo ? bf16x2_to_f16x2(qrow_lo[w + 1]) : 0u;
+                        qf[ks][3] = v_hi ? bf16x2_to_f16x2(qrow_hi[w + 1]) : 0u;
                     } else {
                         const int w = ks * 8 + (lane & 3);           // 32-bit word index in the row
                         qf[ks][0] = v_lo ? qrow_lo[w] : 0u;
@@ -274,13 +287,6 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                         qf[ks][2] = v_lo ? qrow_lo[w + 4] : 0u;
                         qf[ks][3] = v_hi ? qrow_hi[w + 4] : 0u;
                     }
-                }
-                if (with_rope) rope_q_fragments<D, F8>(qf, p.G, p.q_weight != nullptr, p.norm_eps, rope_cs, norm_w, lane);
-                if constexpr (F8) {
-#pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks)
-#pragma unroll
-                        for (int r = 0; r < 4; ++r) qf[ks][r] = bf16x2_to_f16x2(qf[ks][r]);
                 }
             }
             const int t0 = (t_begin + it) * kTileT;

@@ -13,9 +13,9 @@ namespace l4l {
 // The q rows live in the A fragments of the warp MMA: a thread holds, per 16-column k-step, columns 2c, 2c+1
 // (registers 0: row lane/4, 1: row lane/4 + 8) and 2c+8, 2c+9 (registers 2, 3), c = lane % 4. The partner of
 // column i is column i + D/2, i.e. the same register of the k-step D/32 further on: no data leaves the thread.
-// kF8Cols: the fragments of the e4m3-cache kernels, whose k index is permuted the way the byte tiles arrive (registers
-// 0, 1 hold columns 4c, 4c+1 of the k-step, registers 2, 3 columns 4c+2, 4c+3); still bf16 pairs at this point.
-template <int D, bool kF8Cols = false>
+// (The warp-per-unit kernel rotates this way: every warp has its own query rows. The split and the cluster kernel,
+// where all warps of a CTA share the rows, rotate them once in shared memory instead: rope_row_in_smem below.)
+template <int D>
 __device__ __forceinline__ void rope_q_fragments(uint32_t (&qf)[D / 16][4], int G, bool with_norm, float norm_eps,
                                                  const float *cos_sin, const float *weight, int lane)
 {
@@ -44,8 +44,7 @@ __device__ __forceinline__ void rope_q_fragments(uint32_t (&qf)[D / 16][4], int 
     for (int ks = 0; ks < kHalf; ++ks)
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
-            const int col = kF8Cols ? 16 * ks + 4 * c + ((r >> 1) << 1)
-                                    : 16 * ks + 2 * c + ((r >> 1) << 3);    // first-half column of element 0
+            const int col = 16 * ks + 2 * c + ((r >> 1) << 3);               // first-half column of element 0
             float x1[2] = {__uint_as_float(qf[ks][r] << 16), __uint_as_float(qf[ks][r] & 0xffff0000u)};
             float x2[2] = {__uint_as_float(qf[ks + kHalf][r] << 16), __uint_as_float(qf[ks + kHalf][r] & 0xffff0000u)};
             float y1[2], y2[2];
@@ -64,6 +63,44 @@ __device__ __forceinline__ void rope_q_fragments(uint32_t (&qf)[D / 16][4], int 
                 qf[ks + kHalf][r] = pack_bf16x2(y2[0], y2[1]);
             }
         }
+}
+
+// One query row rotated in place in shared memory by one warp: lane l owns the words l (elements 2l, 2l+1) and
+// D/4 + l (their partners, D/2 columns further on); lanes >= D/4 idle. Small code on purpose: it runs once per
+// piece, from a cold instruction cache. All lanes of the warp must call this (shuffles).
+template <int D>
+__device__ __forceinline__ void rope_row_in_smem(uint32_t *row, const float *cos_sin, bool with_norm, float norm_eps,
+                                                 const float *weight, int lane)
+{
+    constexpr int kWords = D / 4;                       // 32-bit words per half row
+    const bool on = lane < kWords;
+    const uint32_t w1 = on ? row[lane] : 0u, w2 = on ? row[kWords + lane] : 0u;
+    float x1[2] = {__uint_as_float(w1 << 16), __uint_as_float(w1 & 0xffff0000u)};
+    float x2[2] = {__uint_as_float(w2 << 16), __uint_as_float(w2 & 0xffff0000u)};
+    if (with_norm) {
+        float ss = fmaf(x1[0], x1[0], fmaf(x1[1], x1[1], fmaf(x2[0], x2[0], x2[1] * x2[1])));
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, d);
+        const float rinv = rsqrtf(ss * (1.f / D) + norm_eps);
+        if (on) {
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                x1[e] = x1[e] * rinv * weight[2 * lane + e];
+                x2[e] = x2[e] * rinv * weight[D / 2 + 2 * lane + e];
+            }
+        }
+    }
+    if (on) {
+        float y1[2], y2[2];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            const float cs = cos_sin[2 * lane + e], sn = cos_sin[D / 2 + 2 * lane + e];
+            y1[e] = fmaf(-x2[e], sn, x1[e] * cs);
+            y2[e] = fmaf(x1[e], sn, x2[e] * cs);
+        }
+        row[lane] = pack_bf16x2(y1[0], y1[1]);
+        row[kWords + lane] = pack_bf16x2(y2[0], y2[1]);
+    }
 }
 
 // The new token's k row as the patching warp holds it: lane l < D/8 has elements [8l, 8l + 8). The partner chunk
