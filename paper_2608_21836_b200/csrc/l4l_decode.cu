@@ -133,7 +133,7 @@ size_t decode_smem_bytes(int G, int nsplit)
     size_t comb = (size_t)W * G * CombRow<D, BigG>::kBytes + (size_t)((G * nsplit + 3) & ~3) * sizeof(float);
     // per stage: the K/V tiles, the piece's query rows and (rope fused into the step) the cos / sin rows of the
     // new token's position; per consumer warp: its private copy of those rows for the piece it is working on
-    return 1024 /*alignment slack*/ + (size_t)C::kStages * (C::kStageBytes + (size_t)G * D * 2 + D * 4) + (size_t)W * D * 4 + 2 * D * 4 +
+    return 1024 /*alignment slack*/ + (size_t)C::kStages * (C::kStageBytes + (size_t)G * D * 2 + D * 4 + (BigG ? 0 : 2 * D * 2)) + (size_t)W * D * 4 + 2 * D * 4 +
            comb +
            C::kStages * sizeof(TileMeta) +
            sizeof(PieceMeta) + (2 * C::kStages + 2) * sizeof(uint64_t) + (2 * kMaxB + 1) * sizeof(int) + 64 +
@@ -176,7 +176,10 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     uint8_t *q_slots = stages + (size_t)C::kStages * C::kStageBytes;     // per stage: the piece's G query rows ...
     const uint32_t q_bytes = (uint32_t)p.G * D * 2;
     constexpr uint32_t kRopeBytes = D * 4;                               // ... and cos | sin of the new token's position
-    const uint32_t q_stride = q_bytes + kRopeBytes;
+    // ... and (fused append; not on the big-group shapes, whose shared memory is full) the step's new k row and v row,
+    // which arrive with the tile they are patched into, so that the patching warp does not wait for global memory there
+    constexpr uint32_t kNewBytes = BigG ? 0 : 2 * D * 2;
+    const uint32_t q_stride = q_bytes + kRopeBytes + kNewBytes;
     float *rope_priv = reinterpret_cast<float *>(q_slots + (size_t)C::kStages * q_stride);   // [W][D] per-warp copy
     float *norm_w = rope_priv + (size_t)W * D;                           // q_weight | k_weight (when given)
     float *comb = norm_w + 2 * D;
@@ -371,20 +374,6 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                         n_box = by_groups ? groups : ((rem >= kTileT || box_rows == kTileT) ? kTileT / box_rows
                                                                                               : (rem + box_rows - 1) / box_rows);
                     }
-                    const uint32_t kv_bytes = (uint32_t)n_box * box_rows * (uint32_t)C::kTokBytes * C::kHalves * 2u;
-                    // with the rope fused into the step, the piece's first tile also brings the cos / sin rows of
-                    // the new token's position (kv_len - 1), if the table has it
-                    const bool with_rope = first && p.rope_cos != nullptr && len - 1 < p.rope_n_pos;
-                    mbar_arrive_expect_tx(&full[s], kv_bytes + (first ? q_bytes : 0u) + (with_rope ? kRopeBytes : 0u));
-                    if (first)
-                        bulk_load_1d(q_slots + (size_t)s * q_stride, p.q + ((size_t)b * p.Hq + (size_t)kvh * p.G) * D,
-                                     q_bytes, &full[s]);
-                    if (with_rope) {
-                        uint8_t *rs = q_slots + (size_t)s * q_stride + q_bytes;
-                        bulk_load_1d(rs, p.rope_cos + (size_t)(len - 1) * (D / 2), kRopeBytes / 2, &full[s]);
-                        bulk_load_1d(rs + kRopeBytes / 2, p.rope_sin + (size_t)(len - 1) * (D / 2), kRopeBytes / 2, &full[s]);
-                    }
-                    uint8_t *dst = stages + (size_t)s * C::kStageBytes;
                     // Neither a box nor a group straddles pages: page sizes are powers of two >= 16 and p.tail_rows is at
                     // most the page size. A page id outside the pool makes the box read zeros, never memory.
                     const int32_t *pages = paged ? p.block_table + (size_t)b * p.table_stride : nullptr;
@@ -394,6 +383,35 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
 #pragma unroll
                     for (int bx = 0; bx < kTileT / 16; ++bx)
                         page_of[bx] = (paged && bx < n_box) ? __ldg(pages + ((tile * kTileT + bx * box_rows) >> p.page_shift)) : b;
+                    // paged fused append: the page of the newest token's slot (it lies in the last box fetched)
+                    if (paged && p.k_new != nullptr && tile + 1 == tiles_b) {
+                        int pg = page_of[0];
+#pragma unroll
+                        for (int bx = 1; bx < kTileT / 16; ++bx) pg = (bx < n_box) ? page_of[bx] : pg;
+                        mt.pad = pg;
+                    }
+                    const uint32_t kv_bytes = (uint32_t)n_box * box_rows * (uint32_t)C::kTokBytes * C::kHalves * 2u;
+                    // with the rope fused into the step, the piece's first tile also brings the cos / sin rows of
+                    // the new token's position (kv_len - 1), if the table has it
+                    const bool with_rope = first && p.rope_cos != nullptr && len - 1 < p.rope_n_pos;
+                    const bool with_new = kNewBytes != 0 && p.k_new != nullptr && tile + 1 == tiles_b;   // the tile of the newest token
+                    mbar_arrive_expect_tx(&full[s], kv_bytes + (first ? q_bytes : 0u) + (with_rope ? kRopeBytes : 0u) +
+                                                        (with_new ? kNewBytes : 0u));
+                    if (with_new) {
+                        uint8_t *ns = q_slots + (size_t)s * q_stride + q_bytes + kRopeBytes;
+                        const size_t src = (size_t)b * p.new_sb + (size_t)kvh * p.new_sh;
+                        bulk_load_1d(ns, p.k_new + src, kNewBytes / 2, &full[s]);
+                        bulk_load_1d(ns + kNewBytes / 2, p.v_new + src, kNewBytes / 2, &full[s]);
+                    }
+                    if (first)
+                        bulk_load_1d(q_slots + (size_t)s * q_stride, p.q + ((size_t)b * p.Hq + (size_t)kvh * p.G) * D,
+                                     q_bytes, &full[s]);
+                    if (with_rope) {
+                        uint8_t *rs = q_slots + (size_t)s * q_stride + q_bytes;
+                        bulk_load_1d(rs, p.rope_cos + (size_t)(len - 1) * (D / 2), kRopeBytes / 2, &full[s]);
+                        bulk_load_1d(rs + kRopeBytes / 2, p.rope_sin + (size_t)(len - 1) * (D / 2), kRopeBytes / 2, &full[s]);
+                    }
+                    uint8_t *dst = stages + (size_t)s * C::kStageBytes;
 #pragma unroll
                     for (int bx = 0; bx < kTileT / 16; ++bx) {
                         if (bx >= n_box) break;
@@ -830,9 +848,15 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 constexpr int kChunks = D / 8;
                 uint4 kk = make_uint4(0u, 0u, 0u, 0u), vv = kk;
                 if (lane < kChunks) {
-                    const size_t src = (size_t)mt.b * p.new_sb + (size_t)mt.kvh * p.new_sh + lane * 8;
-                    kk = __ldg(reinterpret_cast<const uint4 *>(p.k_new + src));
-                    vv = __ldg(reinterpret_cast<const uint4 *>(p.v_new + src));
+                    if constexpr (kNewBytes != 0) {          // the rows came with this tile
+                        const uint4 *ns = reinterpret_cast<const uint4 *>(q_slots + (size_t)s * q_stride + q_bytes + kRopeBytes);
+                        kk = ns[lane];
+                        vv = ns[kChunks + lane];
+                    } else {
+                        const size_t src = (size_t)mt.b * p.new_sb + (size_t)mt.kvh * p.new_sh + lane * 8;
+                        kk = __ldg(reinterpret_cast<const uint4 *>(p.k_new + src));
+                        vv = __ldg(reinterpret_cast<const uint4 *>(p.v_new + src));
+                    }
                 }
                 if (p.rope_cos != nullptr)                                      // all lanes: shuffles inside
                     kk = rope_k_row<D>(kk, p.k_weight != nullptr, p.norm_eps, rope_priv + (size_t)warp * D, norm_w + D,
@@ -842,7 +866,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     // and the tile keeps the zeros that the fetch of a missing page delivers.
                     long long outer = mt.b, slot = mt.kv_len - 1;
                     if (p.block_table != nullptr) {
-                        outer = __ldg(p.block_table + (size_t)mt.b * p.table_stride + (slot >> p.page_shift));
+                        outer = mt.pad;                                          // looked up by the producer
                         slot &= p.page_size - 1;
                     }
                     if (p.block_table == nullptr || (outer >= 0 && outer < p.num_pages)) {
@@ -871,27 +895,44 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     if constexpr (R8) {
                         if (p.rope_cos != nullptr) {
                             uint4 kk = make_uint4(0u, 0u, 0u, 0u);
-                            if (lane < D / 8)
-                                kk = __ldg(reinterpret_cast<const uint4 *>(p.k_new + (size_t)mt.b * p.new_sb + (size_t)mt.kvh * p.new_sh + lane * 8));
+                            if (lane < D / 8) {
+                                if constexpr (kNewBytes != 0)
+                                    kk = reinterpret_cast<const uint4 *>(q_slots + (size_t)s * q_stride + q_bytes + kRopeBytes)[lane];
+                                else
+                                    kk = __ldg(reinterpret_cast<const uint4 *>(p.k_new + (size_t)mt.b * p.new_sb + (size_t)mt.kvh * p.new_sh + lane * 8));
+                            }
                             kk = rope_k_row<D>(kk, p.k_weight != nullptr, p.norm_eps, rope_priv + (size_t)warp * D, norm_w + D,
                                                 mt.kv_len - 1 < p.rope_n_pos, lane);
                             regroup_row_16(kk, lane, ka, kb);
                             rotated = true;
                         }
                     }
-                    if (!rotated && lane < D / 16) {
-                        const uint4 *ks = reinterpret_cast<const uint4 *>(p.k_new + (size_t)mt.b * p.new_sb + (size_t)mt.kvh * p.new_sh + lane * 16);
-                        ka = __ldg(ks);
-                        kb = __ldg(ks + 1);
+                    uint4 va = make_uint4(0u, 0u, 0u, 0u), vb = va;
+                    if (lane < D / 16) {
+                        if constexpr (kNewBytes != 0) {      // the rows came with this tile
+                            const uint4 *ns = reinterpret_cast<const uint4 *>(q_slots + (size_t)s * q_stride + q_bytes + kRopeBytes);
+                            if (!rotated) {
+                                ka = ns[2 * lane];
+                                kb = ns[2 * lane + 1];
+                            }
+                            va = ns[D / 8 + 2 * lane];
+                            vb = ns[D / 8 + 2 * lane + 1];
+                        } else {
+                            const size_t src = (size_t)mt.b * p.new_sb + (size_t)mt.kvh * p.new_sh + lane * 16;
+                            if (!rotated) {
+                                ka = __ldg(reinterpret_cast<const uint4 *>(p.k_new + src));
+                                kb = __ldg(reinterpret_cast<const uint4 *>(p.k_new + src) + 1);
+                            }
+                            va = __ldg(reinterpret_cast<const uint4 *>(p.v_new + src));
+                            vb = __ldg(reinterpret_cast<const uint4 *>(p.v_new + src) + 1);
+                        }
                     }
                     if (lane < D / 16) {
-                        const size_t src = (size_t)mt.b * p.new_sb + (size_t)mt.kvh * p.new_sh + lane * 16;
-                        const uint4 *vs = reinterpret_cast<const uint4 *>(p.v_new + src);
                         const uint4 kq = quantise16(ka, kb, k_sc);
-                        const uint4 vq = quantise16(__ldg(vs), __ldg(vs + 1), v_sc);
+                        const uint4 vq = quantise16(va, vb, v_sc);
                         long long outer = mt.b, slot = mt.kv_len - 1;
                         if (p.block_table != nullptr) {
-                            outer = __ldg(p.block_table + (size_t)mt.b * p.table_stride + (slot >> p.page_shift));
+                            outer = mt.pad;                                      // looked up by the producer
                             slot &= p.page_size - 1;
                         }
                         if (p.block_table == nullptr || (outer >= 0 && outer < p.num_pages)) {

@@ -78,7 +78,7 @@ size_t cluster_smem_bytes(int G, int stages)
 {
     using C = ClusterCfg<D, F8>;
     return 1024 /*alignment slack*/ + (size_t)stages * C::kStageBytes + (size_t)G * D * 2 +
-           (size_t)(kW + 1) * G * C::kPitch * sizeof(float) + 3 * D * sizeof(float) +
+           (size_t)(kW + 1) * G * C::kPitch * sizeof(float) + 4 * D * sizeof(float) +
            2 * C::kMaxStages * sizeof(uint64_t) + 64;
 }
 
@@ -144,7 +144,11 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
     float *rope_cs = part + (size_t)p.G * kPitch;                    // cos | sin of the new token's position
     float *norm_w = rope_cs + D;                                     // q_weight | k_weight
     constexpr uint32_t kRopeBytes = D * 4;
-    uint64_t *full = reinterpret_cast<uint64_t *>(norm_w + 2 * D);
+    // fused append: the step's new k row and v row (bf16), fetched with the first tile so that the warp that patches
+    // them into the last tile does not wait for global memory there
+    uint8_t *new_rows = reinterpret_cast<uint8_t *>(norm_w + 2 * D);
+    constexpr uint32_t kNewBytes = 2 * D * 2;
+    uint64_t *full = reinterpret_cast<uint64_t *>(new_rows + kNewBytes);
     uint64_t *empty = full + C::kMaxStages;
     uint64_t *q_rotated = empty + C::kMaxStages;     // consumers among themselves: the query rows have been rotated in place
     volatile int *abort_flag = reinterpret_cast<volatile int *>(q_rotated + 1);
@@ -176,6 +180,10 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
     int len = __ldg(p.kv_lens + b);
     len = len < 0 ? 0 : (len > p.max_kv_len ? (p.k_new ? 0 : p.max_kv_len) : len);   // over the host's bound: decode ignores the extra tokens, a fused append treats the sequence as empty
     const bool with_rope = p.rope_cos != nullptr && len - 1 < p.rope_n_pos;   // a position outside the table: rows stay as they are
+    // fused append over a paged cache: the page of the new token's slot, looked up now rather than when its tile arrives
+    long long new_page = b;
+    if (p.k_new != nullptr && p.block_table != nullptr && len > 0)
+        new_page = __ldg(p.block_table + (size_t)b * p.table_stride + ((len - 1) >> p.page_shift));
     if (p.rope_cos != nullptr) {
         for (int i = threadIdx.x; i < D; i += kThreads) {
             norm_w[i] = p.q_weight ? __ldg(p.q_weight + i) : 1.f;
@@ -210,9 +218,15 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                 const int n_box = by_groups ? groups : ((rem >= kTileT || box_rows == kTileT) ? kTileT / box_rows
                                                                                               : (rem + box_rows - 1) / box_rows);
                 const uint32_t kv_bytes = (uint32_t)n_box * box_rows * 128u * C::kHalves * 2u;
-                mbar_arrive_expect_tx(&full[s], kv_bytes + (it == 0 ? q_bytes + (with_rope ? kRopeBytes : 0u) : 0u));
+                mbar_arrive_expect_tx(&full[s], kv_bytes + (it == 0 ? q_bytes + (with_rope ? kRopeBytes : 0u) +
+                                                                              (p.k_new != nullptr ? kNewBytes : 0u) : 0u));
                 if (it == 0) {
                     bulk_load_1d(q_smem, p.q + ((size_t)b * p.Hq + (size_t)kvh * p.G) * D, q_bytes, &full[s]);
+                    if (p.k_new != nullptr) {
+                        const size_t src = (size_t)b * p.new_sb + (size_t)kvh * p.new_sh;
+                        bulk_load_1d(new_rows, p.k_new + src, kNewBytes / 2, &full[s]);
+                        bulk_load_1d(new_rows + kNewBytes / 2, p.v_new + src, kNewBytes / 2, &full[s]);
+                    }
                     if (with_rope) {
                         bulk_load_1d(rope_cs, p.rope_cos + (size_t)(len - 1) * (D / 2), kRopeBytes / 2, &full[s]);
                         bulk_load_1d(rope_cs + D / 2, p.rope_sin + (size_t)(len - 1) * (D / 2), kRopeBytes / 2, &full[s]);
@@ -303,9 +317,8 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                 constexpr int kChunks = D / 8;
                 uint4 kk = make_uint4(0u, 0u, 0u, 0u), vv = kk;
                 if (lane < kChunks) {
-                    const size_t src = (size_t)b * p.new_sb + (size_t)kvh * p.new_sh + lane * 8;
-                    kk = __ldg(reinterpret_cast<const uint4 *>(p.k_new + src));
-                    vv = __ldg(reinterpret_cast<const uint4 *>(p.v_new + src));
+                    kk = reinterpret_cast<const uint4 *>(new_rows)[lane];
+                    vv = reinterpret_cast<const uint4 *>(new_rows + kNewBytes / 2)[lane];
                 }
                 if (p.rope_cos != nullptr)                                      // all lanes: shuffles inside
                     kk = rope_k_row<D>(kk, p.k_weight != nullptr, p.norm_eps, rope_cs, norm_w + D, with_rope, lane);
@@ -314,7 +327,7 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                     // and the tile keeps the zeros that the fetch of a missing page delivers.
                     long long outer = b, slot = len - 1;
                     if (p.block_table != nullptr) {
-                        outer = __ldg(p.block_table + (size_t)b * p.table_stride + (slot >> p.page_shift));
+                        outer = new_page;
                         slot &= p.page_size - 1;
                     }
                     if (p.block_table == nullptr || (outer >= 0 && outer < p.num_pages)) {
@@ -341,23 +354,20 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                     uint4 ka = make_uint4(0u, 0u, 0u, 0u), kb = ka;
                     if (p.rope_cos != nullptr) {
                         uint4 kk = make_uint4(0u, 0u, 0u, 0u);
-                        if (lane < D / 8)
-                            kk = __ldg(reinterpret_cast<const uint4 *>(p.k_new + (size_t)b * p.new_sb + (size_t)kvh * p.new_sh + lane * 8));
+                        if (lane < D / 8) kk = reinterpret_cast<const uint4 *>(new_rows)[lane];
                         kk = rope_k_row<D>(kk, p.k_weight != nullptr, p.norm_eps, rope_cs, norm_w + D, with_rope, lane);
                         regroup_row_16(kk, lane, ka, kb);
                     } else if (lane < 8) {
-                        const uint4 *ks = reinterpret_cast<const uint4 *>(p.k_new + (size_t)b * p.new_sb + (size_t)kvh * p.new_sh + lane * 16);
-                        ka = __ldg(ks);
-                        kb = __ldg(ks + 1);
+                        ka = reinterpret_cast<const uint4 *>(new_rows)[2 * lane];
+                        kb = reinterpret_cast<const uint4 *>(new_rows)[2 * lane + 1];
                     }
                     if (lane < 8) {
-                        const size_t src = (size_t)b * p.new_sb + (size_t)kvh * p.new_sh + lane * 16;
-                        const uint4 *vs = reinterpret_cast<const uint4 *>(p.v_new + src);
+                        const uint4 *vs = reinterpret_cast<const uint4 *>(new_rows + kNewBytes / 2);
                         const uint4 kq = quantise16(ka, kb, k_sc);
-                        const uint4 vq = quantise16(__ldg(vs), __ldg(vs + 1), v_sc);
+                        const uint4 vq = quantise16(vs[2 * lane], vs[2 * lane + 1], v_sc);
                         long long outer = b, slot = len - 1;
                         if (p.block_table != nullptr) {
-                            outer = __ldg(p.block_table + (size_t)b * p.table_stride + (slot >> p.page_shift));
+                            outer = new_page;
                             slot &= p.page_size - 1;
                         }
                         if (p.block_table == nullptr || (outer >= 0 && outer < p.num_pages)) {
