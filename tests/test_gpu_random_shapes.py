@@ -189,3 +189,113 @@ def test_prefill_family_random(seed):
         if qlen[b] > 0:
             assert_close_to_oracle(oc2[b, :qlen[b]].cpu(), ref[b, past[b]:lens[b]], f"fused chunk seed {seed} sequence {b}")
             assert_close_to_oracle(oc3[b, :qlen[b]].cpu(), ref[b, past[b]:lens[b]], f"paged fused chunk seed {seed} sequence {b}")
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_decode_step_family_random(seed):
+    """The fused decode steps on seeded random shapes: cache update fused in (contiguous and paged), the same with rope +
+    norm of the new token, and both over an fp8 cache, each against the oracle chain (rope ->) append -> decode."""
+    from paper_2608_21836_b200.workloads import make_rope_tables
+    from test_gpu_decode_append import make_case
+    from test_gpu_fp8 import random_codes
+    from helpers import bits_equal
+
+    rng = np.random.default_rng(6000 + seed)
+    D = int(rng.choice([64, 128]))
+    Hkv = int(rng.choice([1, 2, 3, 8]))
+    G = int(rng.choice([1, 2, 4, 5, 8]))
+    Hq = Hkv * G
+    B = int(rng.choice([1, 3, 9, 40]))
+    page = int(rng.choice([16, 32, 64, 128]))
+    Lmax = int(rng.choice([128, 640, 2176]))                       # multiples of every page size
+    lens = np.maximum(random_lengths(rng, B, Lmax), rng.integers(0, 2, B)).astype(np.int32)   # kv_len INCLUDING the new token
+    q, ck, cv, kn, vn, kv_len = make_case(B, Hq, Hkv, D, Lmax, lens.tolist(), seed=seed)
+    scale = 1.0 / math.sqrt(D)
+    pos, n_new = np.maximum(lens - 1, 0), (lens > 0).astype(np.int32)
+    dl = torch.from_numpy(lens).cuda()
+    ws = l4l.new_workspace(l4l.L4L_OP_DECODE, B, Hq, Hkv, D, Lmax)
+    as_t = lambda bits: torch.from_numpy(bits.view(np.int16).copy()).view(torch.bfloat16)
+    n_per = Lmax // page
+    perm = torch.from_numpy(rng.permutation(B * n_per + 3)[: B * n_per].astype(np.int32)).view(B, n_per)
+
+    def to_pool(c, fill):
+        pool = fill((B * n_per + 3, Hkv, page, D))
+        pool[perm.reshape(-1).long()] = c.view(B, Hkv, n_per, page, D).permute(0, 2, 1, 3, 4).reshape(-1, Hkv, page, D)
+        return pool.cuda()
+
+    def from_pool(pool):
+        return pool.cpu()[perm.reshape(-1).long()].view(B, n_per, Hkv, page, D).permute(0, 2, 1, 3, 4).reshape(B, Hkv, Lmax, D)
+
+    def done(o, ref, what):
+        torch.cuda.synchronize()
+        assert l4l.l4l_last_device_error(ws) == 0
+        assert_close_to_oracle(o.cpu(), ref, f"{what}, seed {seed}")
+
+    # ---- bf16 cache: fused append, contiguous and paged
+    ek, ev = orc.kv_append(ck, cv, kn, vn, pos, n_new)
+    ref, _ = orc.decode(q, as_t(ek), as_t(ev), lens, scale)
+    dck, dcv, o = ck.cuda(), cv.cuda(), torch.zeros(B, Hq, D, dtype=torch.bfloat16, device="cuda")
+    l4l.l4l_attn_decode_append(q.cuda(), o, dck, dcv, kn.cuda(), vn.cuda(), dl, Lmax, scale, ws)
+    done(o, ref, "fused append")
+    assert bits_equal(dck, ek) and bits_equal(dcv, ev)
+    pk, pv, o = to_pool(ck, nan_bf16), to_pool(cv, nan_bf16), torch.zeros(B, Hq, D, dtype=torch.bfloat16, device="cuda")
+    l4l.l4l_attn_decode_paged_append(q.cuda(), o, pk, pv, perm.cuda(), kn.cuda(), vn.cuda(), dl, Lmax, scale, ws)
+    done(o, ref, f"paged fused append, page {page}")
+    assert bits_equal(from_pool(pk), ek) and bits_equal(from_pool(pv), ev)
+
+    # ---- the same with rope + norm of the new token (table over every position)
+    cos, sin = make_rope_tables(Lmax, D)
+    g = torch.Generator().manual_seed(seed + 77)
+    norm = bool(rng.integers(0, 2))
+    qw = (torch.rand(D, generator=g) + 0.5) if norm else None
+    kw = (torch.rand(D, generator=g) + 0.5) if norm else None
+    eps = 1e-6 if norm else 0.0
+    oq, rk, rv, _, _ = orc.rope_kv_append(q.view(B, 1, Hq, D), kn, vn, ck, cv, pos, n_new, cos.numpy(), sin.numpy(),
+                                          None if qw is None else qw.numpy(), None if kw is None else kw.numpy(), eps)
+    ref_r, _ = orc.decode(as_t(oq[:, 0]), as_t(rk), as_t(rv), lens, scale)
+    wargs = dict(q_weight=None if qw is None else qw.cuda(), k_weight=None if kw is None else kw.cuda(), eps=eps)
+    dck, dcv, o = ck.cuda(), cv.cuda(), torch.zeros(B, Hq, D, dtype=torch.bfloat16, device="cuda")
+    l4l.l4l_attn_decode_rope_append(q.cuda(), o, dck, dcv, kn.cuda(), vn.cuda(), dl, Lmax, scale, cos.cuda(), sin.cuda(), ws, **wargs)
+    done(o, ref_r, "rope step")
+    assert bits_equal(dcv, rv)
+    pk, pv, o = to_pool(ck, nan_bf16), to_pool(cv, nan_bf16), torch.zeros(B, Hq, D, dtype=torch.bfloat16, device="cuda")
+    l4l.l4l_attn_decode_paged_rope_append(q.cuda(), o, pk, pv, perm.cuda(), kn.cuda(), vn.cuda(), dl, Lmax, scale, cos.cuda(),
+                                          sin.cuda(), ws, **wargs)
+    done(o, ref_r, f"paged rope step, page {page}")
+    assert bits_equal(from_pool(pv), rv)
+
+    # ---- fp8 cache (head_dim 64: on the split kernel, which wants an even number of slots): fused append and rope step
+    if D == 64:
+        return
+    tg = torch.Generator().manual_seed(seed + 99)
+    c8k, c8v = random_codes((B, Hkv, Lmax, D), tg, 7), random_codes((B, Hkv, Lmax, D), tg, 7)
+    for b in range(B):
+        c8k[b, :, max(int(lens[b]) - 1, 0):] = 0x7F
+        c8v[b, :, max(int(lens[b]) - 1, 0):] = 0xFF
+    ks = torch.from_numpy(rng.uniform(0.5, 1.5, Hkv).astype(np.float32))
+    vs = torch.from_numpy(rng.uniform(0.25, 1.25, Hkv).astype(np.float32))
+    kn7, vn7 = (kn.float() * 0.7).to(torch.bfloat16), (vn.float() * 0.7).to(torch.bfloat16)
+    e8k, e8v = orc.kv_append_fp8(c8k, c8v, kn7, vn7, pos, n_new, ks.numpy(), vs.numpy())
+    ref8, _ = orc.decode_fp8(q, e8k, e8v, lens, ks.numpy(), vs.numpy(), scale)
+    u8 = lambda shape: torch.full(shape, 0x7F, dtype=torch.uint8)
+    d8k, d8v, o = c8k.cuda(), c8v.cuda(), torch.zeros(B, Hq, D, dtype=torch.bfloat16, device="cuda")
+    l4l.l4l_attn_decode_append_fp8(q.cuda(), o, d8k, d8v, ks.cuda(), vs.cuda(), kn7.cuda(), vn7.cuda(), dl, Lmax, scale, ws)
+    done(o, ref8, "fp8 fused append")
+    assert np.array_equal(d8k.cpu().numpy(), e8k) and np.array_equal(d8v.cpu().numpy(), e8v)
+    p8k, p8v, o = to_pool(c8k, u8), to_pool(c8v, u8), torch.zeros(B, Hq, D, dtype=torch.bfloat16, device="cuda")
+    l4l.l4l_attn_decode_append_fp8(q.cuda(), o, p8k, p8v, ks.cuda(), vs.cuda(), kn7.cuda(), vn7.cuda(), dl, Lmax, scale, ws,
+                                   block_table=perm.cuda())
+    done(o, ref8, f"fp8 paged fused append, page {page}")
+    assert np.array_equal(from_pool(p8k).numpy(), e8k) and np.array_equal(from_pool(p8v).numpy(), e8v)
+    # rope step over the fp8 cache: the rotated k row of the oracle (bf16), quantised by the oracle
+    scratch = torch.zeros(B, Hkv, Lmax, D, dtype=torch.bfloat16)
+    oq7, sk, _, _, _ = orc.rope_kv_append(q.view(B, 1, Hq, D), kn7, vn7, scratch, scratch, pos, n_new, cos.numpy(), sin.numpy(),
+                                          None if qw is None else qw.numpy(), None if kw is None else kw.numpy(), eps)
+    k_rot = as_t(np.stack([sk[b, :, pos[b], :] for b in range(B)])[:, None])
+    r8k, r8v = orc.kv_append_fp8(c8k, c8v, k_rot, vn7, pos, n_new, ks.numpy(), vs.numpy())
+    ref8r, _ = orc.decode_fp8(as_t(oq7[:, 0]), r8k, r8v, lens, ks.numpy(), vs.numpy(), scale)
+    d8k, d8v, o = c8k.cuda(), c8v.cuda(), torch.zeros(B, Hq, D, dtype=torch.bfloat16, device="cuda")
+    l4l.l4l_attn_decode_rope_append_fp8(q.cuda(), o, d8k, d8v, ks.cuda(), vs.cuda(), kn7.cuda(), vn7.cuda(), dl, Lmax, scale,
+                                        cos.cuda(), sin.cuda(), ws, **wargs)
+    done(o, ref8r, "fp8 rope step")
+    assert np.array_equal(d8v.cpu().numpy(), r8v)
