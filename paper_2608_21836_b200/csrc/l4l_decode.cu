@@ -3,7 +3,8 @@
 // change the tile element type and the producer's coordinates, nothing else).
 //
 // One launch. The cache of every (sequence, KV head) is cut into tiles of 16*W tokens (W = 4 or 8
-// consumer warps; twice that for fp8, where a warp takes 32 tokens per step); the flattened tile stream (sequence-major, then KV head, then position) is divided
+// consumer warps; twice that for fp8 caches and for 64-wide heads, where a warp takes 32 tokens per step); the
+// flattened tile stream (sequence-major, then KV head, then position) is divided
 // among persistent CTAs as evenly as whole tiles allow, so every CTA streams the same number of bytes
 // (to within one tile) whatever the length mix. A CTA's range may
 // start or end inside a sequence: each (sequence, KV head) is thus covered by one or more
@@ -46,7 +47,9 @@ constexpr int kMaxB = 384;                 // sequences per launch (prefix sums 
 // F8: the cache holds e4m3 bytes (one byte per value) instead of bf16.
 template <int D, int W, bool F8>
 struct DecodeCfg {
-    static constexpr int kSub = F8 ? 2 : 1;                       // 16-token blocks a consumer warp takes per tile
+    // 16-token blocks a consumer warp takes per tile: two (one softmax update per 32 tokens) for fp8 caches and for
+    // 64-wide heads, where a token is half the bytes and the per-token bookkeeping weighs twice as much
+    static constexpr int kSub = (F8 || D == 64) ? 2 : 1;
     static constexpr int kTileT = 16 * W * kSub;                  // tokens per TMA tile
     static constexpr int kRowBytes = F8 ? D : 2 * D;              // one token of one KV head
     // fp8 at head_dim 64: a token is 64 bytes, and two consecutive tokens make one 128-byte row of the tile (the
@@ -840,7 +843,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             const int row0 = warp * 16 * C::kSub;
             const int nvalid = mt.kv_len - (mt.t0 + row0);       // valid tokens in this warp's slice
             bool wrote_smem = false;
-            if (!F8 && p.k_new != nullptr && nvalid > 0 && nvalid <= 16) {
+            if (!F8 && p.k_new != nullptr && nvalid > 0 && nvalid <= 16 * C::kSub) {
                 // fused append: this slice holds the sequence's newest token (row `last` of the tile). Its K/V
                 // arrive from the caller, not from the cache: patch the tile in shared memory and write the
                 // cache slot (each slot belongs to exactly one CTA's range and one warp's slice).
@@ -993,26 +996,38 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                         if (u == 0 || nvalid > 16 * u) warp_pv_16x16_f8<D>(st, pa[u], v_tile, row0 + 16 * u);
                 }
             } else if (nvalid > 0) {
-                float s_lo[4], s_hi[4];
-                float sc = p.scale_log2e;
-                warp_qk_16x16<D>(qf, k_tile, C::kHalfBytes, row0, s_lo, s_hi);
-                const int tok = 2 * (lane & 3);
+                // kSub 16-token blocks per step share one softmax update. A block with no valid token is skipped (its
+                // rows may never have been fetched); in the last valid block the tokens past the end of the sequence get
+                // no weight, and their V rows (which may hold any bits, NaN included) are cleared so that 0 * garbage
+                // cannot appear.
+                constexpr int kSub = C::kSub;
+                float sv[2 * kSub][4];
+                const float sc = p.scale_log2e;
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    s_lo[e] *= sc;
-                    s_hi[e] *= sc;
-                }
-                if (nvalid < 16) {
-                    // tokens past the end of the sequence: no weight, and their V rows (which may
-                    // hold any bits, NaN included) are cleared so that 0 * garbage cannot appear
+                for (int u = 0; u < kSub; ++u) {
+                    if (u == 0 || nvalid > 16 * u) {
+                        warp_qk_16x16<D>(qf, k_tile, C::kHalfBytes, row0 + 16 * u, sv[2 * u], sv[2 * u + 1]);
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        if (tok + (e & 1) >= nvalid) s_lo[e] = -INFINITY;
-                        if (tok + (e & 1) + 8 >= nvalid) s_hi[e] = -INFINITY;
+                        for (int e = 0; e < 4; ++e) {
+                            sv[2 * u][e] *= sc;
+                            sv[2 * u + 1][e] *= sc;
+                        }
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) sv[2 * u][e] = sv[2 * u + 1][e] = -INFINITY;
                     }
+                }
+                if (nvalid < 16 * kSub) {
+                    const int tok = 2 * (lane & 3);
+#pragma unroll
+                    for (int j = 0; j < 2 * kSub; ++j)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            if (8 * j + tok + (e & 1) >= nvalid) sv[j][e] = -INFINITY;
                     uint8_t *vt = stages + (size_t)s * C::kStageBytes + C::kTileBytes;
                     const int chunks_per_row = C::kRowBytes / 16;
-                    for (int i = lane; i < (16 - nvalid) * chunks_per_row; i += 32) {
+                    const int fetched_end = (nvalid + 15) & ~15;                 // end of the last valid block
+                    for (int i = lane; i < (fetched_end - nvalid) * chunks_per_row; i += 32) {
                         const int r = row0 + nvalid + i / chunks_per_row;
                         const int ch = i % chunks_per_row;
                         *reinterpret_cast<uint4 *>(vt + (ch >> 3) * C::kHalfBytes + r * 128 + ((ch & 7) << 4)) =
@@ -1021,9 +1036,11 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     wrote_smem = true;
                     __syncwarp();
                 }
-                uint32_t pa[4];
-                warp_softmax_16<D>(st, s_lo, s_hi, pa);
-                warp_pv_16x16<D>(st, pa, v_tile, C::kHalfBytes, row0);
+                uint32_t pa[kSub][4];
+                warp_softmax_tiles<D, false, 2 * kSub>(st, sv, pa);
+#pragma unroll
+                for (int u = 0; u < kSub; ++u)
+                    if (u == 0 || nvalid > 16 * u) warp_pv_16x16<D>(st, pa[u], v_tile, C::kHalfBytes, row0 + 16 * u);
             }
 
             if (wrote_smem) fence_proxy_async_smem();   // generic writes before the next TMA fill
