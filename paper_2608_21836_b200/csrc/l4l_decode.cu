@@ -290,6 +290,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             const int my_end = range_begin((int)blockIdx.x + 1);
             uint32_t it = 0, n_posted = 0;
             bool ok = true;
+            const uint64_t stream_policy = l2_policy_evict_first();     // the cache is read once
             // Order of work. If the range ends inside a sequence (the next CTA holds its tail and, walking forward,
             // takes it first), that last piece is streamed FIRST and the rest of the range after it: both halves
             // of a cut sequence are then finished early, their merge through the workspace (several round trips
@@ -424,8 +425,8 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                         uint8_t *db = dst + bx * box_rows * C::kTokBytes;  // whole 8-row groups: the swizzle phase is kept
 #pragma unroll
                         for (int hf = 0; hf < C::kHalves; ++hf) {
-                            tma_load_4d(db + hf * C::kHalfBytes, tk, &full[s], hf * C::kBoxD, c1, c2, c3);
-                            tma_load_4d(db + C::kTileBytes + hf * C::kHalfBytes, tv, &full[s], hf * C::kBoxD, c1, c2, c3);
+                            tma_load_4d_policy(db + hf * C::kHalfBytes, tk, &full[s], hf * C::kBoxD, c1, c2, c3, stream_policy);
+                            tma_load_4d_policy(db + C::kTileBytes + hf * C::kHalfBytes, tv, &full[s], hf * C::kBoxD, c1, c2, c3, stream_policy);
                         }
                     }
                 }

@@ -173,6 +173,28 @@ __device__ __forceinline__ void tma_load_4d(void *smem_dst, const void *tmap, ui
         : "memory");
 }
 
+// L2 eviction policy for data that is read once (a streamed cache): its lines are the first to be replaced, so that a
+// stream larger than the L2 recycles its own lines instead of pushing out what an earlier kernel left there (dirty
+// output lines, whose write-back would otherwise share HBM with the stream).
+__device__ __forceinline__ uint64_t l2_policy_evict_first()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+
+// The 4-D tiled load with an L2 policy.
+__device__ __forceinline__ void tma_load_4d_policy(void *smem_dst, const void *tmap, uint64_t *bar, int c0, int c1,
+                                                   int c2, int c3, uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
+        ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_u32(bar)), "r"(c0), "r"(c1),
+        "r"(c2), "r"(c3), "l"(policy)
+        : "memory");
+}
+
 // 3-D tiled load global -> shared (same rules as the 4-D form).
 __device__ __forceinline__ void tma_load_3d(void *smem_dst, const void *tmap, uint64_t *bar, int c0, int c1, int c2)
 {
