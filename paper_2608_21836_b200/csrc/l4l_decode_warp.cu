@@ -80,6 +80,12 @@ __device__ __forceinline__ void cp_async_16_full(uint32_t dst, const void *src)
 {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
+// The same for data that is read once (whole chunks of the cache): an L2 evict-first policy, so that the stream recycles
+// its own lines instead of pushing out what an earlier kernel left in the L2.
+__device__ __forceinline__ void cp_async_16_stream(uint32_t dst, const void *src, uint64_t policy)
+{
+    asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "l"(policy) : "memory");
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
@@ -245,6 +251,8 @@ __global__ void __launch_bounds__(kWarps * 32) decode_warp_kernel(const WarpPara
 #pragma unroll
     for (int i = 0; i < C::kCopies; ++i) soff[i] = dst_half + swz128(i * kRowsPerTrip + row_of_lane, piece & 7);
 
+    uint64_t stream_policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(stream_policy));
     auto issue = [&](const Cursor &c, int slot) {
         uint8_t *st = ring + (size_t)slot * sbytes;
         const uint32_t k_dst = smem_u32(st), v_dst = k_dst + C::kTileBytes;
@@ -268,8 +276,8 @@ __global__ void __launch_bounds__(kWarps * 32) decode_warp_kernel(const WarpPara
             // a full chunk of cached tokens (all but the last chunk of a unit): no predicates
 #pragma unroll
             for (int i = 0; i < C::kCopies; ++i) {
-                cp_async_16_full(k_dst + soff[i], ks);
-                cp_async_16_full(v_dst + soff[i], vs);
+                cp_async_16_stream(k_dst + soff[i], ks, stream_policy);
+                cp_async_16_stream(v_dst + soff[i], vs, stream_policy);
                 ks += step;
                 vs += step;
             }
