@@ -124,6 +124,7 @@ struct DecodeParams {
     int page_box;             // paged: tokens per box of tmap_k / tmap_v (divides the tile, never straddles a page)
     int tail_rows;            // tokens per box of tmap_k_tail / tmap_v_tail (32, or the page size if that is smaller)
     int B, Hq, Hkv, G, min_tiles, nsplit, max_kv_len;
+    int stream_once;          // load K/V with the L2 evict-first policy (large caches)
     int nfin;                 // finisher warps (BigG: one per 4 query heads of the group; else 1)
     float scale_log2e;
     TmapCoord coord;
@@ -290,7 +291,8 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             const int my_end = range_begin((int)blockIdx.x + 1);
             uint32_t it = 0, n_posted = 0;
             bool ok = true;
-            const uint64_t stream_policy = l2_policy_evict_first();     // the cache is read once
+            // a large cache is read once per step: its lines go first; a small one stays L2-resident between steps
+            const uint64_t stream_policy = p.stream_once ? l2_policy_evict_first() : l2_policy_evict_normal();
             // Order of work. If the range ends inside a sequence (the next CTA holds its tail and, walking forward,
             // takes it first), that last piece is streamed FIRST and the rest of the range after it: both halves
             // of a cut sequence are then finished early, their merge through the workspace (several round trips
@@ -1358,6 +1360,7 @@ l4l_status launch_decode(const void *q, void *o, const l4l_kv_cache &cache, cons
         p.status = reinterpret_cast<unsigned *>(ws);
         p.B = nb; p.Hq = Hq; p.Hkv = Hkv; p.G = G; p.min_tiles = plan.min_tiles; p.nsplit = plan.nsplit;
         p.max_kv_len = max_kv_len;
+        p.stream_once = decode_streams_once(B, Hkv, D, max_kv_len, fp8 != nullptr) ? 1 : 0;
         p.nfin = nfin;
         p.k_new = p.v_new = nullptr;
         p.new_sb = p.new_sh = 0;

@@ -69,6 +69,7 @@ struct ClusterParams {
     int rope_n_pos;
     const float *k_scale, *v_scale;           // fp8 cache: real value = e4m3 value * scale of its KV head, [Hkv]
     int B, Hq, Hkv, G, C, max_kv_len, stages;
+    int stream_once;          // load K/V with the L2 evict-first policy (large caches)
     float scale_log2e;
     TmapCoord coord;
 };
@@ -203,6 +204,8 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
         if (lane == 0) {
             const bool paged = p.block_table != nullptr;
             const int32_t *pages = paged ? p.block_table + (size_t)b * p.table_stride : nullptr;
+            // a large cache is read once per step: its lines go first; a small one stays L2-resident between steps
+            const uint64_t stream_policy = p.stream_once ? l2_policy_evict_first() : l2_policy_evict_normal();
             for (int it = 0; it < n_mine; ++it) {
                 const int tile = t_begin + it;
                 const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
@@ -249,8 +252,8 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                     uint8_t *db = dst + bx * box_rows * 128;          // whole 8-row groups: the swizzle phase is kept
 #pragma unroll
                     for (int hf = 0; hf < C::kHalves; ++hf) {
-                        tma_load_4d(db + hf * kHalfBytes, tk, &full[s], hf * C::kBoxD, c1, c2, c3);
-                        tma_load_4d(db + C::kTileBytes + hf * kHalfBytes, tv, &full[s], hf * C::kBoxD, c1, c2, c3);
+                        tma_load_4d_policy(db + hf * kHalfBytes, tk, &full[s], hf * C::kBoxD, c1, c2, c3, stream_policy);
+                        tma_load_4d_policy(db + C::kTileBytes + hf * kHalfBytes, tv, &full[s], hf * C::kBoxD, c1, c2, c3, stream_policy);
                     }
                 }
             }
@@ -772,6 +775,7 @@ l4l_status launch_decode_cluster(const void *q, void *o, const l4l_kv_cache &cac
     p.k_scale = fp8 ? fp8->k_scale : nullptr;
     p.v_scale = fp8 ? fp8->v_scale : nullptr;
     p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.G = G; p.C = width; p.max_kv_len = max_kv_len; p.stages = stages;
+    p.stream_once = decode_streams_once(B, Hkv, D, max_kv_len, fp8 != nullptr) ? 1 : 0;
     p.scale_log2e = scale * 1.4426950408889634f;
     p.coord = coord;
 

@@ -50,6 +50,7 @@ struct WarpParams {
     float norm_eps;
     int rope_n_pos;
     int B, Hq, Hkv, G, max_kv_len, stages;
+    int stream_once;          // copy whole chunks with the L2 evict-first policy (large caches)
     float scale_log2e;
 };
 
@@ -251,8 +252,8 @@ __global__ void __launch_bounds__(kWarps * 32) decode_warp_kernel(const WarpPara
 #pragma unroll
     for (int i = 0; i < C::kCopies; ++i) soff[i] = dst_half + swz128(i * kRowsPerTrip + row_of_lane, piece & 7);
 
-    uint64_t stream_policy;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(stream_policy));
+    // a large cache is read once per step: its lines go first; a small one stays L2-resident between steps
+    const uint64_t stream_policy = p.stream_once ? l2_policy_evict_first() : l2_policy_evict_normal();
     auto issue = [&](const Cursor &c, int slot) {
         uint8_t *st = ring + (size_t)slot * sbytes;
         const uint32_t k_dst = smem_u32(st), v_dst = k_dst + C::kTileBytes;
@@ -640,6 +641,7 @@ l4l_status launch_decode_warp(const void *q, void *o, const l4l_kv_cache &cache,
         p.page_shift = 0;
         while (paged && (1 << p.page_shift) < cache.max_len) ++p.page_shift;
         p.B = nb; p.Hq = Hq; p.Hkv = Hkv; p.G = G; p.max_kv_len = max_kv_len; p.stages = stages;
+        p.stream_once = decode_streams_once(B, Hkv, D, max_kv_len, fp8 != nullptr) ? 1 : 0;
         p.scale_log2e = scale * 1.4426950408889634f;
 
         // persistent: every resident CTA gets its share of the stream; never more CTAs than units

@@ -60,6 +60,14 @@ bool make_tmap_rows_bf16(CUtensorMap *out, const void *base, int64_t n_cols, int
 
 int sm_count();
 
+// Whether a decode launch should load its K/V with the L2 evict-first policy: yes when the cache it may stream is large
+// against the L2 (it is read once per step and would otherwise push out what earlier kernels left there, dirty lines
+// included); no for small caches, which stay L2-resident from one step to the next and are better off without the hint.
+inline bool decode_streams_once(int B, int Hkv, int D, int max_kv_len, bool fp8)
+{
+    return (size_t)B * Hkv * (size_t)max_kv_len * D * (fp8 ? 1 : 2) * 2 >= ((size_t)64 << 20);
+}
+
 struct DecodePlan {
     int warps;       // kernel shape: 4, 6 or 8 consumer warps (tile = 16 tokens per warp)
     bool fits;       // the shape's shared memory fits an SM

@@ -183,6 +183,14 @@ __device__ __forceinline__ uint64_t l2_policy_evict_first()
     return pol;
 }
 
+// The policy that changes nothing (for code that always passes a policy and picks it at run time).
+__device__ __forceinline__ uint64_t l2_policy_evict_normal()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+
 // The 4-D tiled load with an L2 policy.
 __device__ __forceinline__ void tma_load_4d_policy(void *smem_dst, const void *tmap, uint64_t *bar, int c0, int c1,
                                                    int c2, int c3, uint64_t policy)
